@@ -1,0 +1,181 @@
+/*
+ * hbmm.h -- C ABI of the B200 (sm_100a) Hadamard Binary Matrix Multiply library.
+ *
+ * The library implements the inference path of HadaNets ("HadaNets: Flexible
+ * Quantization Strategies for Neural Networks"): a tensor X (rows x K, row-major)
+ * is represented as the Hadamard product  X~ = delta (.) Sign(X)  of a
+ * full-precision tensor delta (the mean absolute value of every run of beta
+ * consecutive row elements; Section 3, Eq. 1-4) and a binary tensor that is
+ * bit-packed along the row (Section 4).  The product of two such operands is
+ * formed from one signed +-1 dot product per K-group (XNOR/popcount) and two
+ * full-precision multiplies per group (Section 4.2, Eq. 7).
+ *
+ * General conventions
+ *   - Every data pointer is DEVICE memory owned by the caller unless a comment
+ *     says "host".  Operand descriptors and geometry structs are host memory and
+ *     are read before the call returns.  The library never allocates, frees or
+ *     keeps a pointer, except where an entry point says otherwise.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     All work is enqueued on it; no call synchronises the host.
+ *   - Every call returns an hbmm_status.  Argument errors are detected on the
+ *     host before anything is launched; a failed launch returns HBMM_ERR_CUDA.
+ *   - Matrices are row-major.  A is M x K (rows = samples / output pixels), W is
+ *     N x K (rows = filters; the paper's W^f = Reshape(W, (filters, -1))), and
+ *     C = A~ * W~^T is M x N in fp32.
+ */
+#ifndef HBMM_H_
+#define HBMM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  HBMM_OK = 0,
+  HBMM_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, leading dimension too small, K mismatch */
+  HBMM_ERR_UNSUPPORTED = 2, /* a beta / dtype / path combination this build does not implement        */
+  HBMM_ERR_ALIGNMENT = 3,   /* a pointer or leading dimension violates the stated alignment           */
+  HBMM_ERR_WORKSPACE = 4,   /* workspace missing or smaller than the *_workspace_bytes query          */
+  HBMM_ERR_CUDA = 5,        /* the CUDA runtime reported an error at launch                            */
+  HBMM_ERR_TIMEOUT = 6      /* a bounded device-side wait expired (kernels never spin unbounded)       */
+} hbmm_status;
+
+typedef enum { HBMM_F32 = 0, HBMM_BF16 = 1 } hbmm_dtype;
+
+/* Which contraction kernel hbmm_gemm_ex runs for two packed operands. */
+typedef enum {
+  HBMM_PATH_AUTO = 0,   /* the fastest path that supports the operands                                 */
+  HBMM_PATH_POPC = 1,   /* XOR + __popc on the integer pipe, fp32 group-scale epilogue in registers    */
+  HBMM_PATH_B1MMA = 2,  /* legacy mma.sync b1 (xor.popc) tensor instruction, beta multiple of 128      */
+  HBMM_PATH_TENSOR = 3  /* sign bits expanded to +-1 e4m3 in shared memory, tensor-core group dots     */
+} hbmm_path;
+
+/*
+ * One Hadamard-binary operand (Section 3, Fig. 1): rows x K, scale groups of beta
+ * consecutive elements along K.
+ *   beta >= 2 : packed form.  `bits` and `scales` are used, `dense` is ignored.
+ *       bits   : uint32 [rows, ld_words]; element k of a row is bit (k % 32), least significant
+ *                first, of word (k / 32); bit 1 <=> Sign = +1 (x >= 0), bit 0 <=> -1 (the paper's
+ *                packing example, Section 4).  Bits at positions >= K and words >= ceil(K/32)
+ *                are zero.  ld_words is a multiple of 4 (16-byte rows); 16-byte aligned.
+ *       scales : [rows, ld_scales] of scale_dtype; entry g is the mean |x| over columns
+ *                [g*beta, min((g+1)*beta, K)) (a tail group is averaged over its own length);
+ *                entries g >= ceil(K/beta) are zero.  ld_scales is a multiple of 4 (fp32) or 8
+ *                (bf16); 16-byte aligned.  bf16 scales are the fp32 scale rounded to nearest even.
+ *       Supported beta: multiples of 32, and any beta >= K (one group per row, the XNOR-Net case
+ *       of Section 5).  Sub-word beta (2..16) returns HBMM_ERR_UNSUPPORTED.
+ *   beta == 1 : the tensor stays at full precision (X~ = X; the paper's first/last layers and the
+ *       HBWN mode).  `dense` [rows, ld_dense] of dense_dtype is used, bits/scales are ignored.
+ */
+typedef struct {
+  int64_t rows;
+  int64_t K;
+  int32_t beta;
+  int32_t scale_dtype; /* hbmm_dtype */
+  uint32_t *bits;
+  int64_t ld_words;
+  void *scales;
+  int64_t ld_scales;
+  const void *dense;
+  int64_t ld_dense;
+  int32_t dense_dtype; /* hbmm_dtype */
+  int32_t reserved;
+} hbmm_operand;
+
+/* Convolution geometry: NCHW input [B, C, H, W], kh x kw filters. */
+typedef struct {
+  int32_t B, C, H, W;
+  int32_t kh, kw;
+  int32_t stride_h, stride_w;
+  int32_t pad_h, pad_w;
+} hbmm_conv_geom;
+
+/*
+ * Storage of a packed operand (Fig. 1; Section 3.2 and 4.1: a binarized tensor costs about
+ * 1 + X/beta bits per element, X the scale width, i.e. beta*X/(beta+X) times less than full
+ * precision).  Pure host arithmetic, no CUDA call.  Outputs (host pointers, any may be NULL):
+ * bytes of the bit tensor, bytes of the scale tensor, and the two leading dimensions to put in
+ * the descriptor.  Errors: INVALID_ARG (rows, K <= 0, beta < 2, bad dtype).
+ */
+hbmm_status hbmm_operand_bytes(int64_t rows, int64_t K, int32_t beta, int32_t scale_dtype,
+                               size_t *bits_bytes, size_t *scales_bytes,
+                               int64_t *ld_words, int64_t *ld_scales);
+
+/*
+ * Hadamard binarization and bit-packing of a row-major tensor (Section 3, Eq. 1-4; packing
+ * Section 4).  x: device, [rows, ldx] of x_dtype, ldx >= K.  out: host descriptor whose rows, K,
+ * beta, scale_dtype, bits, ld_words, scales, ld_scales are set by the caller (buffers sized by
+ * hbmm_operand_bytes); the call fills bits and scales, including their zero padding.
+ * Sign(0) = Sign(-0) = +1.  NaN inputs are outside the contract.
+ * Errors: INVALID_ARG, UNSUPPORTED (beta), ALIGNMENT (bits/scales not 16-byte aligned or
+ * ld_words / ld_scales not as hbmm_operand_bytes returns), CUDA.
+ */
+hbmm_status hbmm_quantize(const void *x, int32_t x_dtype, int64_t rows, int64_t K, int64_t ldx,
+                          const hbmm_operand *out, void *stream);
+
+/* Bytes of scratch hbmm_gemm needs for these operands (currently 0 for every path; the query
+ * exists so callers stay correct if a path grows a workspace).  bytes: host pointer. */
+hbmm_status hbmm_gemm_workspace_bytes(const hbmm_operand *A, const hbmm_operand *W, size_t *bytes);
+
+/*
+ * C[m,n] = sum_k A~[m,k] * W~[n,k]  (Eq. 7 regrouped: per K-segment one signed +-1 dot product
+ * D = n_valid - 2*popcount(xor) and the product of the two segment scales).
+ *   A: M x K, packed (beta_a >= 2) or dense bf16/fp32 (beta_a == 1: the HBWN mode, full-precision
+ *      activations times Hadamard-binary weights).   W: N x K, packed.  A.K == W.K.
+ *   When beta_a != beta_w the larger must be a multiple of the smaller; the work is done on the
+ *   finer segmentation (Section 4.2).
+ *   C: device fp32 [M, ldc], ldc >= N, 16-byte aligned with ldc % 4 == 0.  Fully overwritten
+ *   in columns < N.  workspace may be NULL when the query returns 0.
+ * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, WORKSPACE, CUDA.
+ */
+hbmm_status hbmm_gemm(const hbmm_operand *A, const hbmm_operand *W, float *C, int64_t ldc,
+                      void *workspace, size_t workspace_bytes, void *stream);
+
+/* Same as hbmm_gemm with the contraction kernel chosen by the caller (hbmm_path); a path that
+ * cannot run these operands returns HBMM_ERR_UNSUPPORTED.  For measurement and tests. */
+hbmm_status hbmm_gemm_ex(const hbmm_operand *A, const hbmm_operand *W, float *C, int64_t ldc,
+                         void *workspace, size_t workspace_bytes, int32_t path, void *stream);
+
+/*
+ * The integer term of Eq. 7 on its own: D[m,n,t] = signed +-1 dot product of K-segment t
+ * (segment length min(beta_a, beta_w); T = ceil(K / segment) segments), int32, device
+ * [M, N, T] contiguous.  Both operands packed.  Meant for checking the popcount path
+ * bit-exactly; not tuned.  Errors as hbmm_gemm.
+ */
+hbmm_status hbmm_gemm_partials(const hbmm_operand *A, const hbmm_operand *W, int32_t *D,
+                               int32_t path, void *stream);
+
+/* Scratch for hbmm_conv_im2col: the packed (or, for beta_a == 1, bf16 dense) im2col operand.
+ * bytes: host pointer. */
+hbmm_status hbmm_conv_workspace_bytes(const hbmm_conv_geom *g, int32_t beta_a, int32_t a_scale_dtype,
+                                      const hbmm_operand *W, size_t *bytes);
+
+/*
+ * Convolution as HBMM.  Row m = (b, yo, xo) of the implicit activation matrix gathers
+ * A[m,k] = x[b, c, yo*stride_h + i - pad_h, xo*stride_w + j - pad_w] (0 outside the image) with
+ * k = (c, i, j), c slowest -- the column order of W^f = Reshape(W, (filters, -1)) (Algorithm 1,
+ * Section 3.1.1).  beta_a >= 2: every such row is Hadamard-binarized along k (the grouping Eq. 7
+ * is stated for), packed into the workspace, and multiplied by W as in hbmm_gemm.  beta_a == 1:
+ * HBWN, rows are gathered as bf16.  x: device NCHW of x_dtype.  W: packed, N x (C*kh*kw).
+ * C_out: device fp32 [B*Ho*Wo, ldc] (the NHWC output), alignment as in hbmm_gemm.
+ * workspace: device, 256-byte aligned, at least hbmm_conv_workspace_bytes.
+ * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, WORKSPACE, CUDA.
+ */
+hbmm_status hbmm_conv_im2col(const void *x, int32_t x_dtype, const hbmm_conv_geom *g,
+                             int32_t beta_a, int32_t a_scale_dtype, const hbmm_operand *W,
+                             float *C_out, int64_t ldc, void *workspace, size_t workspace_bytes,
+                             void *stream);
+
+/* Static, NUL-terminated description of a status code (host). */
+const char *hbmm_status_string(int32_t status);
+
+/* Library version, major*10000 + minor*100 + patch. */
+int32_t hbmm_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HBMM_H_ */

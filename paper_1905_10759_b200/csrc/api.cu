@@ -1,0 +1,268 @@
+// C-ABI layer: argument validation on the host, then dispatch to the kernel launchers.
+// Nothing here allocates device memory or synchronises; see include/hbmm.h for the contract.
+#include <cstdint>
+#include <cstddef>
+#include "../../include/hbmm.h"
+#include "kernels.h"
+
+using namespace hbmm;
+
+namespace {
+
+constexpr int32_t kVersion = 100;  // 0.1.0
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool valid_dtype(int32_t d) { return d == HBMM_F32 || d == HBMM_BF16; }
+inline int64_t round_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
+
+inline int64_t words_ld(int64_t K) { return round_up((K + 31) / 32, 4); }
+inline int64_t scales_ld(int64_t K, int32_t beta, int32_t dtype) {
+  return round_up(num_groups(K, beta), dtype == HBMM_BF16 ? 8 : 4);
+}
+
+// beta values the packed kernels implement: whole words per group, or one group per row.
+inline bool beta_supported(int64_t K, int32_t beta) { return beta >= 2 && (beta % 32 == 0 || beta >= K); }
+
+hbmm_status check_packed(const hbmm_operand* op, bool need_buffers = true) {
+  if (!op) return HBMM_ERR_INVALID_ARG;
+  if (op->rows <= 0 || op->K <= 0 || op->beta < 2) return HBMM_ERR_INVALID_ARG;
+  if (!valid_dtype(op->scale_dtype)) return HBMM_ERR_INVALID_ARG;
+  if (!beta_supported(op->K, op->beta)) return HBMM_ERR_UNSUPPORTED;
+  if (need_buffers) {
+    if (!op->bits || !op->scales) return HBMM_ERR_INVALID_ARG;
+    if (op->ld_words < (op->K + 31) / 32 || op->ld_scales < num_groups(op->K, op->beta)) return HBMM_ERR_INVALID_ARG;
+    if (!aligned16(op->bits) || !aligned16(op->scales)) return HBMM_ERR_ALIGNMENT;
+    if (op->ld_words % 4 != 0) return HBMM_ERR_ALIGNMENT;
+    if (op->ld_scales % (op->scale_dtype == HBMM_BF16 ? 8 : 4) != 0) return HBMM_ERR_ALIGNMENT;
+  }
+  return HBMM_OK;
+}
+
+PackedView view_of(const hbmm_operand* op) {
+  PackedView v;
+  v.bits = op->bits; v.scales = op->scales; v.rows = op->rows; v.K = op->K;
+  v.ld_words = op->ld_words; v.ld_scales = op->ld_scales; v.beta = op->beta;
+  v.scale_bf16 = op->scale_dtype == HBMM_BF16;
+  return v;
+}
+
+// Both packed: the coarser grouping must be a whole number of the finer groups.
+bool segments_compatible(const hbmm_operand* A, const hbmm_operand* W) {
+  const bool a_one = A->beta >= A->K, w_one = W->beta >= W->K;
+  if (a_one || w_one) return true;
+  const int64_t lo = A->beta < W->beta ? A->beta : W->beta, hi = A->beta < W->beta ? W->beta : A->beta;
+  return hi % lo == 0;
+}
+
+hbmm_status check_c(const float* C, int64_t ldc, int64_t N) {
+  if (!C || ldc < N) return HBMM_ERR_INVALID_ARG;
+  if (!aligned16(C) || ldc % 4 != 0) return HBMM_ERR_ALIGNMENT;
+  return HBMM_OK;
+}
+
+hbmm_status gemm_checked(const hbmm_operand* A, const hbmm_operand* W, float* C, int64_t ldc,
+                         int32_t path, cudaStream_t stream) {
+  if (!A || !W) return HBMM_ERR_INVALID_ARG;
+  if (W->beta == 1) return HBMM_ERR_UNSUPPORTED;  // the weight operand is always Hadamard-binary
+  hbmm_status st = check_packed(W);
+  if (st != HBMM_OK) return st;
+  if (path < HBMM_PATH_AUTO || path > HBMM_PATH_TENSOR) return HBMM_ERR_INVALID_ARG;
+  if (A->beta == 1) {
+    if (A->rows <= 0 || A->K <= 0 || !A->dense || A->ld_dense < A->K || !valid_dtype(A->dense_dtype))
+      return HBMM_ERR_INVALID_ARG;
+    if (A->K != W->K) return HBMM_ERR_INVALID_ARG;
+    if ((st = check_c(C, ldc, W->rows)) != HBMM_OK) return st;
+    if (path == HBMM_PATH_POPC || path == HBMM_PATH_B1MMA) return HBMM_ERR_UNSUPPORTED;
+    DenseView dv;
+    dv.data = A->dense; dv.rows = A->rows; dv.K = A->K; dv.ld = A->ld_dense; dv.bf16 = A->dense_dtype == HBMM_BF16;
+    return launch_hbwn(dv, view_of(W), C, ldc, path == HBMM_PATH_TENSOR ? 1 : 0, stream) == cudaSuccess
+               ? HBMM_OK : HBMM_ERR_CUDA;
+  }
+  if ((st = check_packed(A)) != HBMM_OK) return st;
+  if (A->K != W->K) return HBMM_ERR_INVALID_ARG;
+  if (!segments_compatible(A, W)) return HBMM_ERR_UNSUPPORTED;
+  if ((st = check_c(C, ldc, W->rows)) != HBMM_OK) return st;
+  const PackedView a = view_of(A), w = view_of(W);
+  cudaError_t e;
+  switch (path) {
+    case HBMM_PATH_POPC: e = launch_gemm_popc(a, w, C, ldc, stream); break;
+    case HBMM_PATH_B1MMA:
+      if (!gemm_b1_supported(a, w)) return HBMM_ERR_UNSUPPORTED;
+      e = launch_gemm_b1(a, w, C, ldc, stream);
+      break;
+    case HBMM_PATH_TENSOR:
+      if (!gemm_tensor_supported(a, w)) return HBMM_ERR_UNSUPPORTED;
+      e = launch_gemm_tensor(a, w, C, ldc, stream);
+      break;
+    default:
+      if (gemm_tensor_supported(a, w)) e = launch_gemm_tensor(a, w, C, ldc, stream);
+      else e = launch_gemm_popc(a, w, C, ldc, stream);
+      break;
+  }
+  return e == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
+}
+
+hbmm_status check_geom(const hbmm_conv_geom* g, ConvGeom* out) {
+  if (!g) return HBMM_ERR_INVALID_ARG;
+  if (g->B <= 0 || g->C <= 0 || g->H <= 0 || g->W <= 0 || g->kh <= 0 || g->kw <= 0 || g->stride_h <= 0 ||
+      g->stride_w <= 0 || g->pad_h < 0 || g->pad_w < 0)
+    return HBMM_ERR_INVALID_ARG;
+  const int64_t ho = (static_cast<int64_t>(g->H) + 2 * g->pad_h - g->kh) / g->stride_h + 1;
+  const int64_t wo = (static_cast<int64_t>(g->W) + 2 * g->pad_w - g->kw) / g->stride_w + 1;
+  if (g->H + 2 * g->pad_h < g->kh || g->W + 2 * g->pad_w < g->kw || ho <= 0 || wo <= 0) return HBMM_ERR_INVALID_ARG;
+  if (static_cast<int64_t>(g->C) * g->kh * g->kw > INT32_MAX) return HBMM_ERR_INVALID_ARG;
+  out->B = g->B; out->C = g->C; out->H = g->H; out->W = g->W; out->kh = g->kh; out->kw = g->kw;
+  out->sh = g->stride_h; out->sw = g->stride_w; out->ph = g->pad_h; out->pw = g->pad_w;
+  out->Ho = static_cast<int32_t>(ho); out->Wo = static_cast<int32_t>(wo);
+  return HBMM_OK;
+}
+
+struct ConvLayout {
+  int64_t M, K, ld_words, ld_scales, ld_dense;
+  size_t bits_bytes, scales_bytes, total;
+};
+
+ConvLayout conv_layout(const ConvGeom& g, int32_t beta_a, int32_t scale_dtype) {
+  ConvLayout L{};
+  L.M = static_cast<int64_t>(g.B) * g.Ho * g.Wo;
+  L.K = static_cast<int64_t>(g.C) * g.kh * g.kw;
+  if (beta_a == 1) {
+    L.ld_dense = round_up(L.K, 8);
+    L.total = static_cast<size_t>(L.M) * L.ld_dense * 2;
+  } else {
+    L.ld_words = words_ld(L.K);
+    L.ld_scales = scales_ld(L.K, beta_a, scale_dtype);
+    L.bits_bytes = static_cast<size_t>(round_up(L.M * L.ld_words * 4, 256));
+    L.scales_bytes = static_cast<size_t>(round_up(L.M * L.ld_scales * (scale_dtype == HBMM_BF16 ? 2 : 4), 256));
+    L.total = L.bits_bytes + L.scales_bytes;
+  }
+  return L;
+}
+
+}  // namespace
+
+extern "C" {
+
+hbmm_status hbmm_operand_bytes(int64_t rows, int64_t K, int32_t beta, int32_t scale_dtype,
+                               size_t* bits_bytes, size_t* scales_bytes, int64_t* ld_words, int64_t* ld_scales) {
+  if (rows <= 0 || K <= 0 || beta < 2 || !valid_dtype(scale_dtype)) return HBMM_ERR_INVALID_ARG;
+  const int64_t lw = words_ld(K), ls = scales_ld(K, beta, scale_dtype);
+  if (bits_bytes) *bits_bytes = static_cast<size_t>(rows) * lw * 4;
+  if (scales_bytes) *scales_bytes = static_cast<size_t>(rows) * ls * (scale_dtype == HBMM_BF16 ? 2 : 4);
+  if (ld_words) *ld_words = lw;
+  if (ld_scales) *ld_scales = ls;
+  return HBMM_OK;
+}
+
+hbmm_status hbmm_quantize(const void* x, int32_t x_dtype, int64_t rows, int64_t K, int64_t ldx,
+                          const hbmm_operand* out, void* stream) {
+  if (!x || !out || rows <= 0 || K <= 0 || ldx < K || !valid_dtype(x_dtype)) return HBMM_ERR_INVALID_ARG;
+  if (out->rows != rows || out->K != K) return HBMM_ERR_INVALID_ARG;
+  hbmm_status st = check_packed(out);
+  if (st != HBMM_OK) return st;
+  if ((reinterpret_cast<uintptr_t>(x) % (x_dtype == HBMM_BF16 ? 2 : 4)) != 0) return HBMM_ERR_ALIGNMENT;
+  const cudaError_t e = launch_quantize(x, x_dtype == HBMM_BF16, rows, K, ldx, out->bits, out->ld_words, out->scales,
+                                        out->ld_scales, out->scale_dtype == HBMM_BF16, out->beta,
+                                        static_cast<cudaStream_t>(stream));
+  if (e == cudaErrorInvalidValue) return HBMM_ERR_UNSUPPORTED;
+  return e == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
+}
+
+hbmm_status hbmm_gemm_workspace_bytes(const hbmm_operand* A, const hbmm_operand* W, size_t* bytes) {
+  if (!A || !W || !bytes) return HBMM_ERR_INVALID_ARG;
+  *bytes = 0;
+  return HBMM_OK;
+}
+
+hbmm_status hbmm_gemm(const hbmm_operand* A, const hbmm_operand* W, float* C, int64_t ldc, void* workspace,
+                      size_t workspace_bytes, void* stream) {
+  (void)workspace; (void)workspace_bytes;
+  return gemm_checked(A, W, C, ldc, HBMM_PATH_AUTO, static_cast<cudaStream_t>(stream));
+}
+
+hbmm_status hbmm_gemm_ex(const hbmm_operand* A, const hbmm_operand* W, float* C, int64_t ldc, void* workspace,
+                         size_t workspace_bytes, int32_t path, void* stream) {
+  (void)workspace; (void)workspace_bytes;
+  return gemm_checked(A, W, C, ldc, path, static_cast<cudaStream_t>(stream));
+}
+
+hbmm_status hbmm_gemm_partials(const hbmm_operand* A, const hbmm_operand* W, int32_t* D, int32_t path, void* stream) {
+  hbmm_status st;
+  if ((st = check_packed(A)) != HBMM_OK) return st;
+  if ((st = check_packed(W)) != HBMM_OK) return st;
+  if (!D || A->K != W->K) return HBMM_ERR_INVALID_ARG;
+  if (!segments_compatible(A, W)) return HBMM_ERR_UNSUPPORTED;
+  const PackedView a = view_of(A), w = view_of(W);
+  cudaError_t e;
+  if (path == HBMM_PATH_AUTO || path == HBMM_PATH_POPC) {
+    e = launch_partials_popc(a, w, D, static_cast<cudaStream_t>(stream));
+  } else if (path == HBMM_PATH_B1MMA) {
+    if (!gemm_b1_supported(a, w)) return HBMM_ERR_UNSUPPORTED;
+    e = launch_partials_b1(a, w, D, static_cast<cudaStream_t>(stream));
+  } else {
+    return HBMM_ERR_UNSUPPORTED;
+  }
+  return e == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
+}
+
+hbmm_status hbmm_conv_workspace_bytes(const hbmm_conv_geom* g, int32_t beta_a, int32_t a_scale_dtype,
+                                      const hbmm_operand* W, size_t* bytes) {
+  ConvGeom cg;
+  hbmm_status st = check_geom(g, &cg);
+  if (st != HBMM_OK) return st;
+  if (!bytes || !W || beta_a < 1 || !valid_dtype(a_scale_dtype)) return HBMM_ERR_INVALID_ARG;
+  const int64_t K = static_cast<int64_t>(cg.C) * cg.kh * cg.kw;
+  if (beta_a >= 2 && !beta_supported(K, beta_a)) return HBMM_ERR_UNSUPPORTED;
+  *bytes = conv_layout(cg, beta_a, a_scale_dtype).total;
+  return HBMM_OK;
+}
+
+hbmm_status hbmm_conv_im2col(const void* x, int32_t x_dtype, const hbmm_conv_geom* g, int32_t beta_a,
+                             int32_t a_scale_dtype, const hbmm_operand* W, float* C_out, int64_t ldc,
+                             void* workspace, size_t workspace_bytes, void* stream) {
+  ConvGeom cg;
+  hbmm_status st = check_geom(g, &cg);
+  if (st != HBMM_OK) return st;
+  if (!x || !W || beta_a < 1 || !valid_dtype(x_dtype) || !valid_dtype(a_scale_dtype)) return HBMM_ERR_INVALID_ARG;
+  if ((st = check_packed(W)) != HBMM_OK) return st;
+  const ConvLayout L = conv_layout(cg, beta_a, a_scale_dtype);
+  if (W->K != L.K) return HBMM_ERR_INVALID_ARG;
+  if (beta_a >= 2 && !beta_supported(L.K, beta_a)) return HBMM_ERR_UNSUPPORTED;
+  if ((st = check_c(C_out, ldc, W->rows)) != HBMM_OK) return st;
+  if (!workspace || workspace_bytes < L.total) return HBMM_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return HBMM_ERR_ALIGNMENT;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  hbmm_operand A{};
+  A.rows = L.M; A.K = L.K; A.beta = beta_a; A.scale_dtype = a_scale_dtype;
+  if (beta_a == 1) {
+    if (launch_im2col_bf16(x, x_dtype == HBMM_BF16, cg, workspace, L.ld_dense, s) != cudaSuccess) return HBMM_ERR_CUDA;
+    A.dense = workspace; A.ld_dense = L.ld_dense; A.dense_dtype = HBMM_BF16;
+  } else {
+    A.bits = static_cast<uint32_t*>(workspace);
+    A.scales = static_cast<char*>(workspace) + L.bits_bytes;
+    A.ld_words = L.ld_words; A.ld_scales = L.ld_scales;
+    hbmm_operand Aseg = A;
+    if (!segments_compatible(&Aseg, W)) return HBMM_ERR_UNSUPPORTED;
+    if (launch_im2col_quantize(x, x_dtype == HBMM_BF16, cg, beta_a, A.bits, A.ld_words, A.scales, A.ld_scales,
+                               a_scale_dtype == HBMM_BF16, s) != cudaSuccess)
+      return HBMM_ERR_CUDA;
+  }
+  return gemm_checked(&A, W, C_out, ldc, HBMM_PATH_AUTO, s);
+}
+
+const char* hbmm_status_string(int32_t status) {
+  switch (status) {
+    case HBMM_OK: return "ok";
+    case HBMM_ERR_INVALID_ARG: return "invalid argument";
+    case HBMM_ERR_UNSUPPORTED: return "unsupported beta / dtype / path combination";
+    case HBMM_ERR_ALIGNMENT: return "pointer or leading dimension violates the required alignment";
+    case HBMM_ERR_WORKSPACE: return "workspace missing or too small";
+    case HBMM_ERR_CUDA: return "CUDA runtime error at launch";
+    case HBMM_ERR_TIMEOUT: return "bounded device-side wait expired";
+    default: return "unknown status";
+  }
+}
+
+int32_t hbmm_version(void) { return kVersion; }
+
+}  // extern "C"

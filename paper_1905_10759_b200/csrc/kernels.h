@@ -1,0 +1,68 @@
+// Internal launcher interface between the C-ABI layer (api.cu) and the kernel files.
+// Host-only declarations; every launcher enqueues on `stream` and returns the launch status.
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace hbmm {
+
+// Device-side view of one packed Hadamard-binary operand (validated by the caller).
+struct PackedView {
+  const uint32_t* bits;   // [rows, ld_words]
+  const void* scales;     // [rows, ld_scales], fp32 or bf16
+  int64_t rows, K;
+  int64_t ld_words, ld_scales;
+  int32_t beta;           // group length along K; >= K means one group per row
+  int32_t scale_bf16;     // 0: fp32 scales, 1: bf16 scales
+};
+
+// Dense full-precision operand (beta = 1).
+struct DenseView {
+  const void* data;       // [rows, ld]
+  int64_t rows, K, ld;
+  int32_t bf16;           // 0: fp32, 1: bf16
+};
+
+struct ConvGeom {
+  int32_t B, C, H, W, kh, kw, sh, sw, ph, pw, Ho, Wo;
+};
+
+// ceil(K / beta) with beta clamped to K (one group per row when beta >= K).
+inline int64_t num_groups(int64_t K, int64_t beta) { return beta >= K ? 1 : (K + beta - 1) / beta; }
+
+cudaError_t launch_quantize(const void* x, int x_bf16, int64_t rows, int64_t K, int64_t ldx,
+                            uint32_t* bits, int64_t ld_words, void* scales, int64_t ld_scales,
+                            int scale_bf16, int32_t beta, cudaStream_t stream);
+
+// Packed x packed contraction on the integer pipe (XOR + POPC).
+cudaError_t launch_gemm_popc(const PackedView& A, const PackedView& W, float* C, int64_t ldc,
+                             cudaStream_t stream);
+cudaError_t launch_partials_popc(const PackedView& A, const PackedView& W, int32_t* D,
+                                 cudaStream_t stream);
+
+// Packed x packed contraction on the legacy b1 tensor instruction (segment multiple of 128 bits).
+bool gemm_b1_supported(const PackedView& A, const PackedView& W);
+cudaError_t launch_gemm_b1(const PackedView& A, const PackedView& W, float* C, int64_t ldc,
+                           cudaStream_t stream);
+cudaError_t launch_partials_b1(const PackedView& A, const PackedView& W, int32_t* D,
+                               cudaStream_t stream);
+
+// Packed x packed contraction with +-1 e4m3 operands on the tensor cores.
+bool gemm_tensor_supported(const PackedView& A, const PackedView& W);
+cudaError_t launch_gemm_tensor(const PackedView& A, const PackedView& W, float* C, int64_t ldc,
+                               cudaStream_t stream);
+
+// Dense x packed contraction (HBWN).
+// tensor = 0: sign-select on the fp32 pipe; 1: bf16 tensor-core path (falls back when unsupported).
+cudaError_t launch_hbwn(const DenseView& A, const PackedView& W, float* C, int64_t ldc, int tensor,
+                        cudaStream_t stream);
+
+// im2col gather fused with Hadamard binarization (packed output), and bf16 dense gather.
+cudaError_t launch_im2col_quantize(const void* x, int x_bf16, const ConvGeom& g, int32_t beta,
+                                   uint32_t* bits, int64_t ld_words, void* scales, int64_t ld_scales,
+                                   int scale_bf16, cudaStream_t stream);
+cudaError_t launch_im2col_bf16(const void* x, int x_bf16, const ConvGeom& g, void* out, int64_t ld,
+                               cudaStream_t stream);
+
+}  // namespace hbmm

@@ -1,0 +1,225 @@
+"""Python binding of the HBMM C-ABI library (``include/hbmm.h``).
+
+Argument marshalling only: every function here has the name of the C entry point it
+calls and passes device pointers of torch tensors straight through; all arithmetic
+runs in the CUDA kernels of ``libhbmm.so``.  Importing this module loads the library
+and raises if it has not been built -- there is no fallback of any kind.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libhbmm.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        "libhbmm.so is missing (%s); build it with `python -m paper_1905_10759_b200.build` "
+        "or __graft_entry__.build()" % LIB_PATH)
+
+_lib = ctypes.CDLL(LIB_PATH)
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(7)
+F32, BF16 = 0, 1
+PATH_AUTO, PATH_POPC, PATH_B1MMA, PATH_TENSOR = 0, 1, 2, 3
+
+EXPORTS = [
+    "hbmm_operand_bytes", "hbmm_quantize", "hbmm_gemm_workspace_bytes", "hbmm_gemm", "hbmm_gemm_ex",
+    "hbmm_gemm_partials", "hbmm_conv_workspace_bytes", "hbmm_conv_im2col", "hbmm_status_string",
+    "hbmm_version",
+]
+
+
+class hbmm_operand(ctypes.Structure):
+    _fields_ = [
+        ("rows", ctypes.c_int64), ("K", ctypes.c_int64),
+        ("beta", ctypes.c_int32), ("scale_dtype", ctypes.c_int32),
+        ("bits", ctypes.c_void_p), ("ld_words", ctypes.c_int64),
+        ("scales", ctypes.c_void_p), ("ld_scales", ctypes.c_int64),
+        ("dense", ctypes.c_void_p), ("ld_dense", ctypes.c_int64),
+        ("dense_dtype", ctypes.c_int32), ("reserved", ctypes.c_int32),
+    ]
+
+
+class hbmm_conv_geom(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("B", "C", "H", "W", "kh", "kw", "stride_h", "stride_w", "pad_h", "pad_w")]
+
+
+_i32, _i64, _vp, _sz = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p, ctypes.c_size_t
+_P = ctypes.POINTER
+_lib.hbmm_operand_bytes.argtypes = [_i64, _i64, _i32, _i32, _P(_sz), _P(_sz), _P(_i64), _P(_i64)]
+_lib.hbmm_quantize.argtypes = [_vp, _i32, _i64, _i64, _i64, _P(hbmm_operand), _vp]
+_lib.hbmm_gemm_workspace_bytes.argtypes = [_P(hbmm_operand), _P(hbmm_operand), _P(_sz)]
+_lib.hbmm_gemm.argtypes = [_P(hbmm_operand), _P(hbmm_operand), _vp, _i64, _vp, _sz, _vp]
+_lib.hbmm_gemm_ex.argtypes = [_P(hbmm_operand), _P(hbmm_operand), _vp, _i64, _vp, _sz, _i32, _vp]
+_lib.hbmm_gemm_partials.argtypes = [_P(hbmm_operand), _P(hbmm_operand), _vp, _i32, _vp]
+_lib.hbmm_conv_workspace_bytes.argtypes = [_P(hbmm_conv_geom), _i32, _i32, _P(hbmm_operand), _P(_sz)]
+_lib.hbmm_conv_im2col.argtypes = [_vp, _i32, _P(hbmm_conv_geom), _i32, _i32, _P(hbmm_operand), _vp, _i64,
+                                  _vp, _sz, _vp]
+_lib.hbmm_status_string.argtypes = [_i32]
+_lib.hbmm_status_string.restype = ctypes.c_char_p
+_lib.hbmm_version.restype = _i32
+for _n in EXPORTS[:8]:
+    getattr(_lib, _n).restype = _i32
+
+
+class HbmmError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s: %s (status %d)" % (where, status_string(status), status))
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise HbmmError(status, where)
+
+
+def status_string(status: int) -> str:
+    return _lib.hbmm_status_string(status).decode()
+
+
+def version() -> int:
+    return int(_lib.hbmm_version())
+
+
+def _dtype_code(dt: torch.dtype) -> int:
+    if dt == torch.float32:
+        return F32
+    if dt == torch.bfloat16:
+        return BF16
+    raise TypeError("only float32 and bfloat16 tensors are accepted, got %s" % dt)
+
+
+def _stream(stream: Optional[torch.cuda.Stream]) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+def _dev_ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("device tensor expected")
+    return t.data_ptr()
+
+
+def operand_bytes(rows: int, K: int, beta: int, scale_dtype: int):
+    """hbmm_operand_bytes -> (bits_bytes, scales_bytes, ld_words, ld_scales)."""
+    bb, sb, lw, ls = _sz(), _sz(), _i64(), _i64()
+    _check(_lib.hbmm_operand_bytes(rows, K, beta, scale_dtype, bb, sb, lw, ls), "hbmm_operand_bytes")
+    return bb.value, sb.value, lw.value, ls.value
+
+
+@dataclass
+class Operand:
+    """A descriptor plus the torch tensors that own its device buffers."""
+    desc: hbmm_operand
+    bits: Optional[torch.Tensor] = None     # int32 view of the uint32 words [rows, ld_words]
+    scales: Optional[torch.Tensor] = None   # [rows, ld_scales] float32 / bfloat16
+    dense: Optional[torch.Tensor] = None    # [rows, ld_dense] for beta == 1
+
+    @property
+    def rows(self) -> int:
+        return self.desc.rows
+
+    @property
+    def K(self) -> int:
+        return self.desc.K
+
+    @property
+    def beta(self) -> int:
+        return self.desc.beta
+
+
+def alloc_operand(rows: int, K: int, beta: int, scale_dtype: int = F32, device="cuda") -> Operand:
+    """Allocate the buffers of a packed operand (sizes from hbmm_operand_bytes) and fill its descriptor."""
+    _, _, lw, ls = operand_bytes(rows, K, beta, scale_dtype)
+    bits = torch.empty((rows, lw), dtype=torch.int32, device=device)
+    scales = torch.empty((rows, ls), dtype=torch.float32 if scale_dtype == F32 else torch.bfloat16, device=device)
+    return wrap_packed(bits, scales, K, beta)
+
+
+def wrap_packed(bits: torch.Tensor, scales: torch.Tensor, K: int, beta: int) -> Operand:
+    """Descriptor over existing device buffers (bits int32/uint32-as-int32 [rows, ld_words])."""
+    d = hbmm_operand()
+    d.rows, d.K, d.beta = bits.shape[0], K, beta
+    d.scale_dtype = _dtype_code(scales.dtype)
+    d.bits, d.ld_words = bits.data_ptr(), bits.stride(0)
+    d.scales, d.ld_scales = scales.data_ptr(), scales.stride(0)
+    return Operand(d, bits=bits, scales=scales)
+
+
+def wrap_dense(a: torch.Tensor) -> Operand:
+    """beta = 1 operand over a row-major [rows, K] device tensor (fp32 or bf16)."""
+    d = hbmm_operand()
+    d.rows, d.K, d.beta = a.shape[0], a.shape[1], 1
+    d.dense, d.ld_dense, d.dense_dtype = a.data_ptr(), a.stride(0), _dtype_code(a.dtype)
+    return Operand(d, dense=a)
+
+
+def quantize(x: torch.Tensor, out: Operand, stream=None) -> Operand:
+    """hbmm_quantize: Hadamard-binarize and pack the rows of ``x`` [rows, K] into ``out``."""
+    if x.dim() != 2 or x.stride(1) != 1:
+        raise ValueError("x must be a row-major 2-D tensor")
+    _check(_lib.hbmm_quantize(_dev_ptr(x), _dtype_code(x.dtype), x.shape[0], x.shape[1], x.stride(0),
+                              ctypes.byref(out.desc), _stream(stream)), "hbmm_quantize")
+    return out
+
+
+def gemm_workspace_bytes(A: Operand, W: Operand) -> int:
+    n = _sz()
+    _check(_lib.hbmm_gemm_workspace_bytes(ctypes.byref(A.desc), ctypes.byref(W.desc), n), "hbmm_gemm_workspace_bytes")
+    return n.value
+
+
+def gemm(A: Operand, W: Operand, C: torch.Tensor, workspace: Optional[torch.Tensor] = None, stream=None):
+    """hbmm_gemm: C[M, N] (fp32, row-major, caller-allocated) = A~ W~^T."""
+    ws_ptr = _dev_ptr(workspace)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(_lib.hbmm_gemm(ctypes.byref(A.desc), ctypes.byref(W.desc), _dev_ptr(C), C.stride(0), ws_ptr, ws_bytes,
+                          _stream(stream)), "hbmm_gemm")
+    return C
+
+
+def gemm_ex(A: Operand, W: Operand, C: torch.Tensor, path: int, workspace: Optional[torch.Tensor] = None,
+            stream=None):
+    ws_ptr = _dev_ptr(workspace)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(_lib.hbmm_gemm_ex(ctypes.byref(A.desc), ctypes.byref(W.desc), _dev_ptr(C), C.stride(0), ws_ptr, ws_bytes,
+                             path, _stream(stream)), "hbmm_gemm_ex")
+    return C
+
+
+def gemm_partials(A: Operand, W: Operand, D: torch.Tensor, path: int = PATH_AUTO, stream=None):
+    """hbmm_gemm_partials: D int32 [M, N, T] contiguous."""
+    _check(_lib.hbmm_gemm_partials(ctypes.byref(A.desc), ctypes.byref(W.desc), _dev_ptr(D), path, _stream(stream)),
+           "hbmm_gemm_partials")
+    return D
+
+
+def make_geom(B, C, H, W, kh, kw, stride=(1, 1), pad=(0, 0)) -> hbmm_conv_geom:
+    return hbmm_conv_geom(B, C, H, W, kh, kw, stride[0], stride[1], pad[0], pad[1])
+
+
+def conv_workspace_bytes(geom: hbmm_conv_geom, beta_a: int, a_scale_dtype: int, W: Operand) -> int:
+    n = _sz()
+    _check(_lib.hbmm_conv_workspace_bytes(ctypes.byref(geom), beta_a, a_scale_dtype, ctypes.byref(W.desc), n),
+           "hbmm_conv_workspace_bytes")
+    return n.value
+
+
+def conv_im2col(x: torch.Tensor, geom: hbmm_conv_geom, beta_a: int, a_scale_dtype: int, W: Operand,
+                C_out: torch.Tensor, workspace: torch.Tensor, stream=None):
+    """hbmm_conv_im2col: x NCHW contiguous; C_out fp32 [B*Ho*Wo, N]."""
+    if not x.is_contiguous():
+        raise ValueError("x must be a contiguous NCHW tensor")
+    _check(_lib.hbmm_conv_im2col(_dev_ptr(x), _dtype_code(x.dtype), ctypes.byref(geom), beta_a, a_scale_dtype,
+                                 ctypes.byref(W.desc), _dev_ptr(C_out), C_out.stride(0), _dev_ptr(workspace),
+                                 workspace.numel() * workspace.element_size(), _stream(stream)), "hbmm_conv_im2col")
+    return C_out

@@ -1,0 +1,277 @@
+"""GPU parity: every result of the CUDA library is compared with the CPU oracle on the same seeded
+inputs, through the C-ABI binding.  Bits and integer partials must match exactly; scales within the
+bound of an fp32 pairwise sum; products within 1e-5 of the magnitude reference sum |deltaA*deltaW*D|."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1905_10759_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+RTOL = 1e-5          # fp32 products (relative to sum_t |deltaA * deltaW * D_t|)
+RTOL_BF16 = 1e-2     # paths whose inputs or scales are stored in bf16, end to end from raw data
+
+
+@pytest.fixture(scope="module")
+def hb():
+    from paper_1905_10759_b200 import hbmm
+    return hbmm
+
+
+def _gu():
+    import gpu_util
+    return gpu_util
+
+
+# ------------------------------------------------------------------ quantize / pack
+QUANT_CASES = [
+    # rows, K, beta, x bf16?, scale dtype, ldx pad
+    (256, 256, 32, False, 0, 0),
+    (37, 100, 32, False, 0, 0),
+    (5, 45, 32, False, 0, 3),      # ragged K, unaligned rows -> scalar loads
+    (64, 576, 32, False, 0, 0),
+    (64, 576, 64, False, 1, 0),
+    (33, 576, 128, False, 0, 0),   # 128 does not divide 576: tail group of 64
+    (16, 1152, 256, False, 0, 0),  # general path
+    (7, 384, 96, False, 0, 0),     # group of three words
+    (9, 577, 577, False, 0, 0),    # one group per row, ragged
+    (3, 4608, 4608, False, 1, 0),
+    (130, 1000, 64, True, 0, 0),   # bf16 input
+    (20, 333, 32, True, 1, 8),
+    (11, 2048, 256, True, 0, 0),
+    (1, 1, 32, False, 0, 0),
+]
+
+
+@pytest.mark.parametrize("rows,K,beta,xbf16,sdt,ldpad", QUANT_CASES)
+def test_quantize_bits_exact_scales_within_bound(hb, rows, K, beta, xbf16, sdt, ldpad):
+    gu = _gu()
+    x = inputs.normal((rows, K), 1000 + rows + K + beta)
+    x[0, 0] = 0.0
+    if K > 2:
+        x[rows // 2, 1] = -0.0
+    if xbf16:
+        xb, x = inputs.as_bf16(x)
+    delta, sign = oracle.quantize(x, beta)
+    xd = torch.zeros((rows, K + ldpad), dtype=torch.float32)
+    xd[:, :K] = torch.from_numpy(x)
+    xd = xd.cuda()
+    if xbf16:
+        xd = xd.to(torch.bfloat16)  # exact: values are bf16-representable
+    out = hb.alloc_operand(rows, K, beta, sdt)
+    out.bits.fill_(-1)
+    out.scales.fill_(float("nan"))
+    hb.quantize(xd[:, :K], out)
+    torch.cuda.synchronize()
+    bits = gu.host_bits(out.bits)
+    assert np.array_equal(bits, oracle.pack(sign, bits.shape[1]))          # includes zero pad bits / words
+    G = delta.shape[1]
+    sc = out.scales.float().cpu().numpy().astype(np.float64)
+    assert np.all(sc[:, G:] == 0.0)
+    be = gu.eff_beta(beta, K)
+    depth = int(np.ceil(np.log2(be))) + int(np.ceil(be / 1024)) + 2     # pairwise tree (+ lane-strided part)
+    tol = depth * gu.U
+    if sdt == hb.BF16:
+        tol += 2.0 ** -8                                                  # half an ulp of bf16 (8 significant bits)
+    np.testing.assert_allclose(sc[:, :G], delta, rtol=tol, atol=0)
+
+
+def test_quantize_signs_of_special_values(hb):
+    gu = _gu()
+    x = np.zeros((2, 64), dtype=np.float32)
+    x[0, :] = [(-1.0) ** k * 1e-38 * (k % 3) for k in range(64)]   # zeros, +-tiny
+    x[1, ::2] = -0.0
+    x[1, 1::2] = np.float32(3e36)   # 16 of them still sum below the fp32 maximum
+    out = hb.alloc_operand(2, 64, 32, 0)
+    hb.quantize(torch.from_numpy(x).cuda(), out)
+    delta, sign = oracle.quantize(x, 32)
+    assert np.array_equal(gu.host_bits(out.bits), oracle.pack(sign, 4))
+    np.testing.assert_allclose(out.scales.cpu().numpy()[:, :2], delta, rtol=8 * gu.U)
+
+
+# ------------------------------------------------------------------ integer partials (bit exact)
+PARTIAL_CASES = [(33, 17, 256, 32, 32), (20, 9, 100, 32, 64), (8, 8, 576, 128, 32), (5, 6, 333, 333, 32),
+                 (4, 3, 384, 96, 96), (6, 7, 77, 77, 77), (3, 5, 1024, 256, 64)]
+
+
+@pytest.mark.parametrize("M,N,K,ba,bw", PARTIAL_CASES)
+def test_partials_bit_exact(hb, M, N, K, ba, bw):
+    gu = _gu()
+    a = inputs.normal((M, K), 2000 + M + K)
+    w = inputs.normal((N, K), 3000 + N + K)
+    A, _, sa = gu.oracle_operand(a, ba)
+    W, _, sw = gu.oracle_operand(w, bw)
+    d_ref, _ = oracle.partials(sa, sw, gu.eff_beta(ba, K), gu.eff_beta(bw, K))
+    D = torch.empty(d_ref.shape, dtype=torch.int32, device="cuda")
+    hb.gemm_partials(A, W, D, hb.PATH_POPC)
+    assert np.array_equal(D.cpu().numpy(), d_ref)
+
+
+# ------------------------------------------------------------------ packed x packed contraction
+GEMM_CASES = [
+    # M, N, K, beta_a, beta_w, scale dtype
+    (256, 256, 256, 32, 32, 0),      # the 256^3 configuration
+    (130, 70, 100, 32, 32, 0),       # ragged everywhere, tail segment of 4 bits
+    (300, 64, 576, 32, 32, 0),       # narrow-N tile
+    (129, 200, 576, 64, 64, 0),
+    (77, 129, 576, 128, 128, 0),     # 576 = 4*128 + 64: short tail segment
+    (64, 96, 1024, 256, 256, 0),
+    (100, 100, 512, 32, 128, 0),     # beta_a < beta_w: finer segmentation decides
+    (100, 100, 512, 128, 32, 1),     # and the other way, bf16 scales
+    (65, 63, 384, 96, 96, 0),        # generic segment length
+    (50, 60, 333, 333, 333, 0),      # XNOR-Net case, one scale per row
+    (50, 60, 320, 320, 32, 0),       # one group per row against beta 32
+    (40, 1000, 4096, 64, 64, 0),     # FC-style ragged N = 1000
+    (1, 1000, 4096, 64, 64, 0),      # batch 1
+    (3, 5, 31, 32, 32, 0),           # K below one word
+]
+
+
+def _paths(hb):
+    return [hb.PATH_POPC, hb.PATH_B1MMA, hb.PATH_TENSOR, hb.PATH_AUTO]
+
+
+@pytest.mark.parametrize("M,N,K,ba,bw,sdt", GEMM_CASES)
+def test_gemm_matches_oracle_on_every_path(hb, M, N, K, ba, bw, sdt):
+    gu = _gu()
+    a = inputs.normal((M, K), 4000 + M + K + ba)
+    w = inputs.he_normal(N, K, 5000 + N + K + bw)
+    A, da, sa = gu.oracle_operand(a, ba, sdt)
+    W, dw, sw = gu.oracle_operand(w, bw, sdt)
+    c_ref, absref = oracle.hbmm_from_quantized(da, sa, gu.eff_beta(ba, K), dw, sw, gu.eff_beta(bw, K))
+    ran = 0
+    for path in _paths(hb):
+        ldc = (N + 3) // 4 * 4 + 4
+        C = torch.full((M, ldc), float("nan"), device="cuda")
+        try:
+            hb.gemm_ex(A, W, C, path)
+        except hb.HbmmError as e:
+            assert e.status == hb.ERR_UNSUPPORTED and path not in (hb.PATH_POPC, hb.PATH_AUTO)
+            continue
+        ran += 1
+        out = C.cpu().numpy()
+        assert np.isnan(out[:, N:]).all()          # nothing written beyond column N
+        gu.assert_close_rel_absref(out[:, :N], c_ref, absref, RTOL, "path %d" % path)
+    assert ran >= 2
+
+
+@pytest.mark.parametrize("M,N,K,beta", [(200, 130, 576, 32), (70, 64, 1152, 64), (33, 140, 640, 128)])
+def test_unit_scales_give_exact_integers(hb, M, N, K, beta):
+    """All scales 1: C must equal K - 2*popc(xor) exactly (every value is a small integer in fp32)."""
+    gu = _gu()
+    rng = np.random.default_rng(M + N)
+    sa = rng.choice(np.array([-1, 1], dtype=np.int8), size=(M, K))
+    sw = rng.choice(np.array([-1, 1], dtype=np.int8), size=(N, K))
+    G = oracle.n_groups(K, beta)
+    _, _, lw, ls = hb.operand_bytes(M, K, beta, hb.F32)
+    A = hb.wrap_packed(gu.dev_bits(oracle.pack(sa, lw)), gu.scales_to_dev(np.ones((M, G)), hb.F32, ls), K, beta)
+    W = hb.wrap_packed(gu.dev_bits(oracle.pack(sw, lw)), gu.scales_to_dev(np.ones((N, G)), hb.F32, ls), K, beta)
+    ref = sa.astype(np.int32) @ sw.astype(np.int32).T
+    for path in _paths(hb):
+        C = torch.empty((M, (N + 3) // 4 * 4), device="cuda")
+        try:
+            hb.gemm_ex(A, W, C, path)
+        except hb.HbmmError as e:
+            assert e.status == hb.ERR_UNSUPPORTED
+            continue
+        assert np.array_equal(C.cpu().numpy()[:, :N], ref.astype(np.float32)), path
+
+
+def test_quantize_then_gemm_end_to_end(hb):
+    """Raw fp32 inputs through hbmm_quantize and hbmm_gemm against the oracle from raw inputs."""
+    gu = _gu()
+    M, N, K = 256, 256, 256
+    a = inputs.normal((M, K), inputs.SEEDS["square256"][0])
+    w = inputs.normal((N, K), inputs.SEEDS["square256"][1])
+    for sdt, rtol in [(hb.F32, RTOL), (hb.BF16, RTOL_BF16)]:
+        A = hb.quantize(torch.from_numpy(a).cuda(), hb.alloc_operand(M, K, 32, sdt))
+        W = hb.quantize(torch.from_numpy(w).cuda(), hb.alloc_operand(N, K, 32, sdt))
+        C = torch.empty((M, N), device="cuda")
+        hb.gemm(A, W, C)
+        c_ref, absref = oracle.hbmm(a, w, 32, 32, None)       # exact scales: the GPU's rounding is inside rtol
+        gu.assert_close_rel_absref(C.cpu().numpy(), c_ref, absref, rtol)
+
+
+# ------------------------------------------------------------------ HBWN (beta_a = 1)
+HBWN_CASES = [(256, 64, 576, 32, True), (100, 130, 1152, 32, True), (65, 70, 100, 32, True), (40, 33, 576, 64, False),
+              (30, 40, 333, 333, True), (129, 256, 2304, 32, True), (8, 16, 64, 32, False)]
+
+
+def _hbwn_rtol(gu, K, beta_w):
+    be = gu.eff_beta(beta_w, K)
+    return (be + -(-K // be) + 4) * 2 * gu.U       # sequential fp32 sums inside and across groups, x2 margin
+
+
+@pytest.mark.parametrize("M,N,K,bw,abf16", HBWN_CASES)
+def test_hbwn_matches_oracle(hb, M, N, K, bw, abf16):
+    gu = _gu()
+    a = inputs.normal((M, K), 6000 + M + K)
+    w = inputs.he_normal(N, K, 7000 + N + K)
+    if abf16:
+        _, a = inputs.as_bf16(a)
+    W, dw, sw = gu.oracle_operand(w, bw)
+    c_ref, absref = oracle.hbwn_from_quantized(a, dw, sw, gu.eff_beta(bw, K))
+    ad = torch.from_numpy(a).cuda()
+    if abf16:
+        ad = ad.to(torch.bfloat16)
+    rtol = _hbwn_rtol(gu, K, bw)
+    assert rtol < RTOL_BF16
+    for path in (hb.PATH_AUTO, hb.PATH_TENSOR):
+        C = torch.full((M, (N + 3) // 4 * 4), float("nan"), device="cuda")
+        hb.gemm_ex(hb.wrap_dense(ad), W, C, path)
+        gu.assert_close_rel_absref(C.cpu().numpy()[:, :N], c_ref, absref, rtol, "hbwn path %d" % path)
+
+
+# ------------------------------------------------------------------ convolution front end
+CONV_CASES = [
+    # B, C, H, W, N, kh, kw, stride, pad, beta_a, beta_w, signed, x bf16
+    (2, 64, 8, 8, 64, 3, 3, 1, 1, 32, 32, True, False),
+    (2, 64, 8, 8, 64, 3, 3, 1, 1, 32, 32, False, False),    # post-ReLU: every sign bit is 1
+    (3, 32, 7, 9, 40, 3, 3, 1, 1, 64, 32, True, False),
+    (2, 16, 9, 9, 20, 3, 3, 2, 0, 32, 32, True, False),     # stride 2, no padding
+    (1, 8, 6, 6, 12, 5, 5, 1, 2, 200, 200, True, False),    # one group per row
+    (2, 24, 5, 5, 16, 1, 1, 1, 0, 32, 32, True, True),      # 1x1, bf16 input, K = 24 below a word
+    (2, 64, 8, 8, 64, 3, 3, 1, 1, 1, 32, True, True),       # HBWN
+    (2, 20, 7, 7, 33, 3, 3, 1, 1, 1, 32, False, False),     # HBWN from fp32 input (rounded to bf16 rows)
+]
+
+
+@pytest.mark.parametrize("B,C,H,W,N,kh,kw,st,pd,ba,bw,signed,xbf16", CONV_CASES)
+def test_conv_im2col_matches_oracle(hb, B, C, H, W, N, kh, kw, st, pd, ba, bw, signed, xbf16):
+    gu = _gu()
+    shape = inputs.ConvShape("t", B, C, H, W, N, kh, kw, st, pd)
+    x = inputs.conv_activation(shape, 8000 + C + H, signed=signed)
+    if xbf16 or ba == 1:
+        _, xr = inputs.as_bf16(x)     # HBWN rows are bf16: the oracle sees the same rounded values
+    else:
+        xr = x
+    if xbf16:
+        x = xr
+    K = C * kh * kw
+    w = inputs.he_normal(N, K, 9000 + N)
+    Wop, dw, sw = gu.oracle_operand(w, bw)
+    a_rows = oracle.im2col(xr, kh, kw, (st, st), (pd, pd))
+    if ba == 1:
+        c_ref, absref = oracle.hbwn_from_quantized(a_rows, dw, sw, gu.eff_beta(bw, K))
+        rtol = _hbwn_rtol(gu, K, bw)
+    else:
+        da, sa = oracle.quantize(a_rows, gu.eff_beta(ba, K))
+        c_ref, absref = oracle.hbmm_from_quantized(da, sa, gu.eff_beta(ba, K), dw, sw, gu.eff_beta(bw, K))
+        rtol = RTOL
+    geom = hb.make_geom(B, C, H, W, kh, kw, (st, st), (pd, pd))
+    xd = torch.from_numpy(x).cuda()
+    if xbf16:
+        xd = xd.to(torch.bfloat16)
+    nbytes = hb.conv_workspace_bytes(geom, ba, hb.F32, Wop)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    M = c_ref.shape[0]
+    Cout = torch.full((M, (N + 3) // 4 * 4), float("nan"), device="cuda")
+    hb.conv_im2col(xd, geom, ba, hb.F32, Wop, Cout, ws)
+    gu.assert_close_rel_absref(Cout.cpu().numpy()[:, :N], c_ref, absref, rtol)
+    if ba > 1:
+        # the packed activation operand left in the workspace: bits exact
+        _, _, lw, ls = hb.operand_bytes(M, K, ba, hb.F32)
+        bits = ws[: M * lw * 4].view(torch.int32).reshape(M, lw)
+        assert np.array_equal(gu.host_bits(bits), oracle.pack(sa, lw))
