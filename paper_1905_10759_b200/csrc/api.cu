@@ -72,10 +72,10 @@ hbmm_status gemm_checked(const hbmm_operand* A, const hbmm_operand* W, float* C,
       return HBMM_ERR_INVALID_ARG;
     if (A->K != W->K) return HBMM_ERR_INVALID_ARG;
     if ((st = check_c(C, ldc, W->rows)) != HBMM_OK) return st;
-    if (path == HBMM_PATH_POPC || path == HBMM_PATH_B1MMA) return HBMM_ERR_UNSUPPORTED;
+    if (path == HBMM_PATH_B1MMA) return HBMM_ERR_UNSUPPORTED;
     DenseView dv;
     dv.data = A->dense; dv.rows = A->rows; dv.K = A->K; dv.ld = A->ld_dense; dv.bf16 = A->dense_dtype == HBMM_BF16;
-    return launch_hbwn(dv, view_of(W), C, ldc, path == HBMM_PATH_TENSOR ? 1 : 0, stream) == cudaSuccess
+    return launch_hbwn(dv, view_of(W), C, ldc, path == HBMM_PATH_TENSOR ? 1 : (path == HBMM_PATH_POPC ? 2 : 0), stream) == cudaSuccess
                ? HBMM_OK : HBMM_ERR_CUDA;
   }
   if ((st = check_packed(A)) != HBMM_OK) return st;

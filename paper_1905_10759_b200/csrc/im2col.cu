@@ -72,6 +72,56 @@ im2col_quantize_kernel(const void* __restrict__ x, int x_bf16, const ConvGeom g,
   for (int64_t z = grp; z < ld_scales; z++) store_scale(scales, scale_bf16, m * ld_scales + z, 0.0f);
 }
 
+// One thread per (row m, scale group g): the 32 lanes of a warp hold 32 consecutive m for the
+// same group, so every tap is a coalesced read along an image row and each thread emits whole
+// words plus the group's scale.  Used when beta < K; blocks are 32 rows x 8 groups.
+__global__ void __launch_bounds__(256)
+im2col_quantize_groups_kernel(const void* __restrict__ x, int x_bf16, const ConvGeom g, int64_t M, int64_t K,
+                              int beta_words, int64_t G, int64_t n_words, uint32_t* __restrict__ bits,
+                              int64_t ld_words, void* __restrict__ scales, int64_t ld_scales, int scale_bf16) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t m = static_cast<int64_t>(blockIdx.x) * 32 + lane;
+  const int64_t grp = static_cast<int64_t>(blockIdx.y) * 8 + warp;
+  if (m >= M || grp >= G) return;
+  const int xo = static_cast<int>(m % g.Wo);
+  const int yo = static_cast<int>((m / g.Wo) % g.Ho);
+  const int64_t b = m / (static_cast<int64_t>(g.Wo) * g.Ho);
+  const int taps = g.kh * g.kw;
+  const int64_t HW = static_cast<int64_t>(g.H) * g.W;
+  const int y0 = yo * g.sh - g.ph, x0 = xo * g.sw - g.pw;
+  const int64_t k_begin = grp * beta_words * 32;
+  int64_t k_end = k_begin + static_cast<int64_t>(beta_words) * 32;
+  if (k_end > K) k_end = K;
+  int c = static_cast<int>(k_begin / taps);
+  int r = static_cast<int>(k_begin - static_cast<int64_t>(c) * taps);
+  int i = r / g.kw, j = r - i * g.kw;
+  const int64_t base = b * g.C * HW;
+  uint32_t* brow = bits + m * ld_words;
+  float gsum = 0.0f;
+  for (int64_t kw0 = k_begin; kw0 < k_end; kw0 += 32) {
+    uint32_t word = 0;
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+    const int nk = (k_end - kw0 < 32) ? static_cast<int>(k_end - kw0) : 32;
+#pragma unroll 4
+    for (int e = 0; e < nk; e++) {
+      const int y = y0 + i, xx = x0 + j;
+      float v = 0.0f;
+      if (y >= 0 && y < g.H && xx >= 0 && xx < g.W) v = load_x(x, x_bf16, base + c * HW + static_cast<int64_t>(y) * g.W + xx);
+      word |= (v >= 0.0f ? 1u : 0u) << e;
+      const float av = fabsf(v);
+      if ((e & 3) == 0) s0 += av; else if ((e & 3) == 1) s1 += av; else if ((e & 3) == 2) s2 += av; else s3 += av;
+      if (++j == g.kw) { j = 0; if (++i == g.kh) { i = 0; c++; } }
+    }
+    brow[kw0 >> 5] = word;
+    gsum += (s0 + s1) + (s2 + s3);
+  }
+  store_scale(scales, scale_bf16, m * ld_scales + grp, gsum / static_cast<float>(k_end - k_begin));
+  if (grp == G - 1) {
+    for (int64_t w = n_words; w < ld_words; w++) brow[w] = 0u;
+    for (int64_t z = G; z < ld_scales; z++) store_scale(scales, scale_bf16, m * ld_scales + z, 0.0f);
+  }
+}
+
 __global__ void __launch_bounds__(256)
 im2col_bf16_kernel(const void* __restrict__ x, int x_bf16, const ConvGeom g, int64_t M, int64_t K,
                    __nv_bfloat16* __restrict__ out, int64_t ld) {
@@ -103,6 +153,12 @@ cudaError_t launch_im2col_quantize(const void* x, int x_bf16, const ConvGeom& g,
   const int64_t M = static_cast<int64_t>(g.B) * g.Ho * g.Wo, K = static_cast<int64_t>(g.C) * g.kh * g.kw;
   const int64_t beta_eff = beta >= K ? K : beta;
   const int64_t G = num_groups(K, beta);
+  if (beta < K && beta % 32 == 0) {
+    dim3 grid(static_cast<unsigned>((M + 31) / 32), static_cast<unsigned>((G + 7) / 8));
+    im2col_quantize_groups_kernel<<<grid, 256, 0, stream>>>(x, x_bf16, g, M, K, beta / 32, G, (K + 31) / 32, bits,
+                                                             ld_words, scales, ld_scales, scale_bf16);
+    return cudaGetLastError();
+  }
   const int64_t blocks = (M + kThreads - 1) / kThreads;
   im2col_quantize_kernel<<<static_cast<unsigned>(blocks), kThreads, 0, stream>>>(
       x, x_bf16, g, M, K, beta_eff, G, bits, ld_words, scales, ld_scales, scale_bf16);

@@ -54,8 +54,8 @@ cudaError_t launch_gemm_tensor(const PackedView& A, const PackedView& W, float* 
                                cudaStream_t stream);
 
 // Dense x packed contraction (HBWN).
-// tensor = 0: sign-select on the fp32 pipe; 1: bf16 tensor-core path (falls back when unsupported).
-cudaError_t launch_hbwn(const DenseView& A, const PackedView& W, float* C, int64_t ldc, int tensor,
+// kind = 0: fastest available; 1: bf16 tensor-core path (falls back when unsupported); 2: sign-select.
+cudaError_t launch_hbwn(const DenseView& A, const PackedView& W, float* C, int64_t ldc, int kind,
                         cudaStream_t stream);
 
 // im2col gather fused with Hadamard binarization (packed output), and bf16 dense gather.

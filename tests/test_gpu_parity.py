@@ -196,7 +196,9 @@ def test_quantize_then_gemm_end_to_end(hb):
 
 # ------------------------------------------------------------------ HBWN (beta_a = 1)
 HBWN_CASES = [(256, 64, 576, 32, True), (100, 130, 1152, 32, True), (65, 70, 100, 32, True), (40, 33, 576, 64, False),
-              (30, 40, 333, 333, True), (129, 256, 2304, 32, True), (8, 16, 64, 32, False)]
+              (30, 40, 333, 333, True), (129, 256, 2304, 32, True), (8, 16, 64, 32, False), (300, 64, 576, 64, True),
+              (130, 200, 672, 128, True), (70, 50, 96, 64, True), (257, 129, 1160, 1160, True), (33, 64, 40, 32, True),
+              (64, 72, 384, 96, True)]
 
 
 def _hbwn_rtol(gu, K, beta_w):
@@ -218,7 +220,7 @@ def test_hbwn_matches_oracle(hb, M, N, K, bw, abf16):
         ad = ad.to(torch.bfloat16)
     rtol = _hbwn_rtol(gu, K, bw)
     assert rtol < RTOL_BF16
-    for path in (hb.PATH_AUTO, hb.PATH_TENSOR):
+    for path in (hb.PATH_AUTO, hb.PATH_TENSOR, hb.PATH_POPC):   # POPC selects the fp32 sign-select kernel
         C = torch.full((M, (N + 3) // 4 * 4), float("nan"), device="cuda")
         hb.gemm_ex(hb.wrap_dense(ad), W, C, path)
         gu.assert_close_rel_absref(C.cpu().numpy()[:, :N], c_ref, absref, rtol, "hbwn path %d" % path)
