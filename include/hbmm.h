@@ -169,6 +169,34 @@ hbmm_status hbmm_conv_im2col(const void *x, int32_t x_dtype, const hbmm_conv_geo
                              float *C_out, int64_t ldc, void *workspace, size_t workspace_bytes,
                              void *stream);
 
+/*
+ * hbmm_conv_im2col for callers that cannot allocate device memory.  (No counterpart in the
+ * paper: this is a deployment convenience, not part of the method.)
+ *
+ * Who needs it: code that runs inside a host framework or inference server whose allocator
+ * already owns all device memory, plugins that are handed nothing but tensor pointers and a
+ * stream, and real-time loops where cudaMalloc/cudaFree (which synchronise the device) are
+ * not allowed.  Such callers can pass inputs and outputs but have nowhere to get a workspace.
+ *
+ * Same arguments, results and errors as hbmm_conv_im2col, without the workspace: the packed
+ * activation operand is kept in a fixed array of HBMM_STATIC_SCRATCH_BYTES inside the library's
+ * device image (every GPU that loads the library holds that much memory until the process
+ * exits).  The call allocates and frees nothing.  A problem whose hbmm_conv_workspace_bytes
+ * exceeds HBMM_STATIC_SCRATCH_BYTES is rejected with HBMM_ERR_WORKSPACE before anything is
+ * launched (this includes every realistic beta_a == 1 problem, whose bf16 row matrix is large).
+ *
+ * The first call on each device looks up the array's device address (the device must be
+ * current); make that first call outside any stream capture.  All calls on a device share the
+ * one array: it keeps whatever the last call left, which is harmless because each call rewrites
+ * all of the region it reads (nothing has to start at zero), but two calls whose kernels can
+ * overlap on the GPU (different streams, or different host threads on different streams) race
+ * on it -- serialise them on one stream or with events.
+ */
+#define HBMM_STATIC_SCRATCH_BYTES ((size_t)32 << 20) /* 32 MiB */
+hbmm_status hbmm_conv_im2col_static(const void *x, int32_t x_dtype, const hbmm_conv_geom *g,
+                                    int32_t beta_a, int32_t a_scale_dtype, const hbmm_operand *W,
+                                    float *C_out, int64_t ldc, void *stream);
+
 /* Static, NUL-terminated description of a status code (host). */
 const char *hbmm_status_string(int32_t status);
 

@@ -31,8 +31,9 @@ PATH_AUTO, PATH_POPC, PATH_B1MMA, PATH_TENSOR = 0, 1, 2, 3
 EXPORTS = [
     "hbmm_operand_bytes", "hbmm_quantize", "hbmm_gemm_workspace_bytes", "hbmm_gemm", "hbmm_gemm_ex",
     "hbmm_gemm_partials", "hbmm_conv_workspace_bytes", "hbmm_conv_im2col", "hbmm_status_string",
-    "hbmm_version",
+    "hbmm_version", "hbmm_conv_im2col_static",
 ]
+STATIC_SCRATCH_BYTES = 32 << 20
 
 
 class hbmm_operand(ctypes.Structure):
@@ -62,6 +63,8 @@ _lib.hbmm_gemm_partials.argtypes = [_P(hbmm_operand), _P(hbmm_operand), _vp, _i3
 _lib.hbmm_conv_workspace_bytes.argtypes = [_P(hbmm_conv_geom), _i32, _i32, _P(hbmm_operand), _P(_sz)]
 _lib.hbmm_conv_im2col.argtypes = [_vp, _i32, _P(hbmm_conv_geom), _i32, _i32, _P(hbmm_operand), _vp, _i64,
                                   _vp, _sz, _vp]
+_lib.hbmm_conv_im2col_static.argtypes = [_vp, _i32, _P(hbmm_conv_geom), _i32, _i32, _P(hbmm_operand), _vp, _i64, _vp]
+_lib.hbmm_conv_im2col_static.restype = _i32
 _lib.hbmm_status_string.argtypes = [_i32]
 _lib.hbmm_status_string.restype = ctypes.c_char_p
 _lib.hbmm_version.restype = _i32
@@ -222,4 +225,17 @@ def conv_im2col(x: torch.Tensor, geom: hbmm_conv_geom, beta_a: int, a_scale_dtyp
     _check(_lib.hbmm_conv_im2col(_dev_ptr(x), _dtype_code(x.dtype), ctypes.byref(geom), beta_a, a_scale_dtype,
                                  ctypes.byref(W.desc), _dev_ptr(C_out), C_out.stride(0), _dev_ptr(workspace),
                                  workspace.numel() * workspace.element_size(), _stream(stream)), "hbmm_conv_im2col")
+    return C_out
+
+
+def conv_im2col_static(x: torch.Tensor, geom: hbmm_conv_geom, beta_a: int, a_scale_dtype: int, W: Operand,
+                       C_out: torch.Tensor, stream=None):
+    """hbmm_conv_im2col_static: hbmm_conv_im2col without a caller workspace, for callers that cannot
+    allocate device memory; the scratch is a fixed STATIC_SCRATCH_BYTES array inside the library.
+    Calls that may overlap on the GPU share that array and must be serialised by the caller."""
+    if not x.is_contiguous():
+        raise ValueError("x must be a contiguous NCHW tensor")
+    _check(_lib.hbmm_conv_im2col_static(_dev_ptr(x), _dtype_code(x.dtype), ctypes.byref(geom), beta_a, a_scale_dtype,
+                                        ctypes.byref(W.desc), _dev_ptr(C_out), C_out.stride(0), _stream(stream)),
+           "hbmm_conv_im2col_static")
     return C_out
