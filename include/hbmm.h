@@ -50,7 +50,7 @@ typedef enum {
   HBMM_PATH_AUTO = 0,   /* the fastest path that supports the operands                                 */
   HBMM_PATH_POPC = 1,   /* XOR + __popc on the integer pipe, fp32 group-scale epilogue in registers    */
   HBMM_PATH_B1MMA = 2,  /* legacy mma.sync b1 (xor.popc) tensor instruction, beta multiple of 128      */
-  HBMM_PATH_TENSOR = 3  /* sign bits expanded to +-1 e4m3 in shared memory, tensor-core group dots     */
+  HBMM_PATH_TENSOR = 3  /* sign bits expanded to +-1 e4m3 in shared memory, tcgen05 group dots in TMEM  */
 } hbmm_path;
 
 /*
@@ -196,6 +196,15 @@ hbmm_status hbmm_conv_im2col(const void *x, int32_t x_dtype, const hbmm_conv_geo
 hbmm_status hbmm_conv_im2col_static(const void *x, int32_t x_dtype, const hbmm_conv_geom *g,
                                     int32_t beta_a, int32_t a_scale_dtype, const hbmm_operand *W,
                                     float *C_out, int64_t ldc, void *stream);
+
+/*
+ * Device-side health word of the tensor-core contraction.  Its kernels never spin without a
+ * limit: a wait on a barrier that does not complete in time records a code (1 producer, 2/3/4
+ * MMA issue, 5 epilogue), makes the kernel drain and return, and leaves the output undefined.
+ * This call copies the word back (it synchronises the device) and returns HBMM_ERR_TIMEOUT when
+ * it is non-zero, HBMM_OK otherwise.  code: host pointer, may be NULL.
+ */
+hbmm_status hbmm_last_device_error(int32_t *code);
 
 /* Static, NUL-terminated description of a status code (host). */
 const char *hbmm_status_string(int32_t status);

@@ -250,6 +250,13 @@ hbmm_status hbmm_conv_im2col(const void* x, int32_t x_dtype, const hbmm_conv_geo
   return gemm_checked(&A, W, C_out, ldc, HBMM_PATH_AUTO, s);
 }
 
+hbmm_status hbmm_last_device_error(int32_t* code) {
+  int c = 0;
+  if (read_umma_error(&c) != cudaSuccess) return HBMM_ERR_CUDA;
+  if (code) *code = c;
+  return c == 0 ? HBMM_OK : HBMM_ERR_TIMEOUT;
+}
+
 const char* hbmm_status_string(int32_t status) {
   switch (status) {
     case HBMM_OK: return "ok";

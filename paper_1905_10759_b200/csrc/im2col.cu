@@ -145,6 +145,220 @@ im2col_bf16_kernel(const void* __restrict__ x, int x_bf16, const ConvGeom g, int
   }
 }
 
+// ---- shared-memory tiled front ends (stride_w == 1, any kh x kw / padding / stride_h) ----------------
+// A block owns RB consecutive output rows (b, yo .. yo+RB-1) and a contiguous range of input
+// channels that it walks in chunks of 32.  The input rows a chunk needs are staged in shared
+// memory with their zero halo (coalesced reads, each element fetched once per block), a small
+// table maps the chunk-local k to its tile offset, and the results leave the block as contiguous
+// runs per output row.
+
+constexpr int kTileCC = 32;   // channels per chunk: 32 * kh * kw elements = whole K-words and whole 16-byte pieces
+
+struct TilePlan {
+  int RB;             // output rows per block
+  int rows_in;        // staged input rows: (RB - 1) * sh + kh
+  int span;           // staged row length: Wo - 1 + kw
+  int yo_blocks;      // ceil(Ho / RB)
+  int splits;         // channel ranges (grid.y)
+  int chunks_per_split;
+};
+
+inline TilePlan make_plan(const ConvGeom& g, int sms) {
+  TilePlan p;
+  p.RB = 112 / g.Wo;
+  if (p.RB < 1) p.RB = 1;
+  if (p.RB > g.Ho) p.RB = g.Ho;
+  p.rows_in = (p.RB - 1) * g.sh + g.kh;
+  p.span = g.Wo - 1 + g.kw;
+  p.yo_blocks = (g.Ho + p.RB - 1) / p.RB;
+  const int chunks = (g.C + kTileCC - 1) / kTileCC;
+  const int64_t row_blocks = static_cast<int64_t>(g.B) * p.yo_blocks;
+  int splits = 1;
+  while (row_blocks * splits < 2LL * sms && splits * 2 <= chunks) splits *= 2;
+  p.chunks_per_split = (chunks + splits - 1) / splits;
+  p.splits = (chunks + p.chunks_per_split - 1) / p.chunks_per_split;
+  return p;
+}
+
+template <typename T, typename Conv>
+__device__ __forceinline__ void stage_tile(T* tile, const void* __restrict__ x, int x_bf16, const ConvGeom& g,
+                                           int64_t b, int c0, int cc, int yo0, const TilePlan& tp, Conv conv) {
+  // Work items are (staged row (c, r), block of 32 consecutive columns); a warp takes them eight at a
+  // time so that eight independent global loads are in flight before the first shared-memory store.
+  constexpr int BATCH = 8;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  const int y_base = yo0 * g.sh - g.ph;
+  const int xblocks = (tp.span + 31) / 32;
+  const int items = cc * tp.rows_in * xblocks;
+  for (int it0 = warp * BATCH; it0 < items; it0 += nwarps * BATCH) {
+    float v[BATCH];
+    int dst[BATCH];
+#pragma unroll
+    for (int u = 0; u < BATCH; u++) {
+      const int it = it0 + u;
+      v[u] = 0.0f;
+      dst[u] = -1;
+      if (it < items) {
+        const int row = it / xblocks, xx = (it - row * xblocks) * 32 + lane;
+        const int c = row / tp.rows_in, r = row - c * tp.rows_in;
+        const int y = y_base + r, xi = xx - g.pw;
+        if (xx < tp.span) {
+          dst[u] = row * tp.span + xx;
+          if (y >= 0 && y < g.H && xi >= 0 && xi < g.W)
+            v[u] = load_x(x, x_bf16, ((b * g.C + c0 + c) * static_cast<int64_t>(g.H) + y) * g.W + xi);
+        }
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < BATCH; u++)
+      if (dst[u] >= 0) tile[dst[u]] = conv(v[u]);
+  }
+}
+
+// chunk-local k -> offset of tap (c, i, j) inside the staged tile (for the pixel at the tile origin)
+__device__ __forceinline__ void build_offsets(unsigned short* off, int cc, const ConvGeom& g, const TilePlan& tp) {
+  const int taps = g.kh * g.kw;
+  for (int k = threadIdx.x; k < cc * taps; k += blockDim.x) {
+    const int c = k / taps, r = k - c * taps, i = r / g.kw, j = r - i * g.kw;
+    off[k] = static_cast<unsigned short>((c * tp.rows_in + i) * tp.span + j);
+  }
+}
+
+struct ToBf16 { __device__ unsigned short operator()(float v) const { return __bfloat16_as_ushort(__float2bfloat16_rn(v)); } };
+struct KeepF32 { __device__ float operator()(float v) const { return v; } };
+
+// bf16 rows for HBWN.  Each thread writes 16-byte pieces (8 consecutive k) of an output row.
+__global__ void __launch_bounds__(256)
+im2col_bf16_tiled_kernel(const void* __restrict__ x, int x_bf16, const ConvGeom g, const TilePlan tp, int64_t K,
+                         __nv_bfloat16* __restrict__ out, int64_t ld) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int taps = g.kh * g.kw;
+  unsigned short* off = reinterpret_cast<unsigned short*>(smem_raw);                       // [32 * taps]
+  unsigned short* tile = off + ((kTileCC * taps + 7) / 8) * 8;                             // [32 * rows_in * span]
+  const int64_t b = blockIdx.x / tp.yo_blocks;
+  const int yo0 = static_cast<int>(blockIdx.x % tp.yo_blocks) * tp.RB;
+  const int rows = (g.Ho - yo0 < tp.RB) ? g.Ho - yo0 : tp.RB;
+  const int pixels = rows * g.Wo;
+  const int chunk_first = blockIdx.y * tp.chunks_per_split;
+  for (int ch = chunk_first; ch < chunk_first + tp.chunks_per_split; ch++) {
+    const int c0 = ch * kTileCC;
+    if (c0 >= g.C) break;
+    const int cc = (g.C - c0 < kTileCC) ? g.C - c0 : kTileCC;
+    const bool last_chunk = c0 + cc == g.C;
+    __syncthreads();                              // previous chunk's readers are done with tile / off
+    if (ch == chunk_first || cc != kTileCC) build_offsets(off, cc, g, tp);
+    stage_tile<unsigned short>(tile, x, x_bf16, g, b, c0, cc, yo0, tp, ToBf16());
+    __syncthreads();
+    const int k_lo = c0 * taps;                                               // multiple of 8
+    const int k_end = k_lo + cc * taps;                                       // valid elements end here
+    const int k_hi = last_chunk ? static_cast<int>(ld) : k_end;               // the last chunk also writes the padding
+    const int pieces = (k_hi - k_lo + 7) / 8;
+    // walk (pixel, piece) pairs with piece fastest, without divisions
+    int pc = threadIdx.x % pieces, pix = threadIdx.x / pieces;
+    const int dpc = 256 % pieces, dpix = 256 / pieces;
+    int ry = pix / g.Wo, xo = pix - ry * g.Wo;
+    while (pix < pixels) {
+      const int kl = pc * 8;                                                  // chunk-local k of the piece
+      const unsigned short* base = tile + ry * g.sh * tp.span + xo;
+      unsigned short v[8];
+#pragma unroll
+      for (int e = 0; e < 8; e++) v[e] = (k_lo + kl + e < k_end) ? base[off[kl + e]] : static_cast<unsigned short>(0);
+      const int64_t m = (b * g.Ho + yo0 + ry) * g.Wo + xo;
+      uint4 o;
+      o.x = v[0] | (static_cast<uint32_t>(v[1]) << 16); o.y = v[2] | (static_cast<uint32_t>(v[3]) << 16);
+      o.z = v[4] | (static_cast<uint32_t>(v[5]) << 16); o.w = v[6] | (static_cast<uint32_t>(v[7]) << 16);
+      *reinterpret_cast<uint4*>(out + m * ld + k_lo + kl) = o;
+      pc += dpc; pix += dpix; xo += dpix;
+      if (pc >= pieces) { pc -= pieces; pix++; xo++; }
+      while (xo >= g.Wo) { xo -= g.Wo; ry++; }
+    }
+  }
+}
+
+// Packed front end for beta = 32: one thread per (output pixel, K-word); the 32 lanes of a warp
+// hold 32 consecutive pixels of the same word, so the tap offsets are warp-uniform and the tile
+// reads are consecutive.  Words and scales of the block's channel range are collected in shared
+// memory and written out as contiguous runs per output row.
+__global__ void __launch_bounds__(256)
+im2col_quantize_tiled_kernel(const void* __restrict__ x, int x_bf16, const ConvGeom g, const TilePlan tp, int64_t K,
+                             int64_t G, int64_t n_words, uint32_t* __restrict__ bits, int64_t ld_words,
+                             void* __restrict__ scales, int64_t ld_scales, int scale_bf16) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int taps = g.kh * g.kw;
+  const int max_pixels = tp.RB * g.Wo;
+  const int split_words = tp.chunks_per_split * taps;          // words this block produces per pixel (upper bound)
+  float* tile = reinterpret_cast<float*>(smem_raw);                                        // [32 * rows_in * span]
+  uint32_t* out_bits = reinterpret_cast<uint32_t*>(tile + kTileCC * tp.rows_in * tp.span);  // [max_pixels][split_words + 1]
+  float* out_scale = reinterpret_cast<float*>(out_bits + max_pixels * (split_words + 1));  // same shape
+  unsigned short* off = reinterpret_cast<unsigned short*>(out_scale + max_pixels * (split_words + 1));
+  const int ldo = split_words + 1;                             // odd-ish pitch: fewer bank conflicts on the column writes
+  const int64_t b = blockIdx.x / tp.yo_blocks;
+  const int yo0 = static_cast<int>(blockIdx.x % tp.yo_blocks) * tp.RB;
+  const int rows = (g.Ho - yo0 < tp.RB) ? g.Ho - yo0 : tp.RB;
+  const int pixels = rows * g.Wo;
+  const int pix_pad = (pixels + 31) / 32 * 32;                 // keep a warp on one word
+  const int chunk_first = blockIdx.y * tp.chunks_per_split;
+  int words_done = 0;                                          // words produced so far by this block
+  bool wrote_last = false;
+  for (int ch = chunk_first; ch < chunk_first + tp.chunks_per_split; ch++) {
+    const int c0 = ch * kTileCC;
+    if (c0 >= g.C) break;
+    const int cc = (g.C - c0 < kTileCC) ? g.C - c0 : kTileCC;
+    wrote_last = c0 + cc == g.C;
+    __syncthreads();
+    if (ch == chunk_first || cc != kTileCC) build_offsets(off, cc, g, tp);
+    stage_tile<float>(tile, x, x_bf16, g, b, c0, cc, yo0, tp, KeepF32());
+    __syncthreads();
+    const int chunk_elems = cc * taps;
+    const int words = (chunk_elems + 31) / 32;
+    for (int idx = threadIdx.x; idx < pix_pad * words; idx += 256) {
+      const int w = idx / pix_pad, pix = idx - w * pix_pad;
+      if (pix >= pixels) continue;
+      const int ry = pix / g.Wo, xo = pix - ry * g.Wo;
+      const int k_begin = w * 32;
+      const int nk = (chunk_elems - k_begin < 32) ? chunk_elems - k_begin : 32;
+      const float* base = tile + ry * g.sh * tp.span + xo;
+      const unsigned short* o = off + k_begin;
+      uint32_t word = 0;
+      float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+      if (nk == 32) {
+#pragma unroll
+        for (int e = 0; e < 32; e += 4) {
+          const float v0 = base[o[e]], v1 = base[o[e + 1]], v2 = base[o[e + 2]], v3 = base[o[e + 3]];
+          word |= (v0 >= 0.0f ? 1u : 0u) << e;
+          word |= (v1 >= 0.0f ? 1u : 0u) << (e + 1);
+          word |= (v2 >= 0.0f ? 1u : 0u) << (e + 2);
+          word |= (v3 >= 0.0f ? 1u : 0u) << (e + 3);
+          s0 += fabsf(v0); s1 += fabsf(v1); s2 += fabsf(v2); s3 += fabsf(v3);
+        }
+      } else {
+        for (int e = 0; e < nk; e++) {
+          const float v = base[o[e]];
+          word |= (v >= 0.0f ? 1u : 0u) << e;
+          s0 += fabsf(v);
+        }
+      }
+      out_bits[pix * ldo + words_done + w] = word;
+      out_scale[pix * ldo + words_done + w] = ((s0 + s1) + (s2 + s3)) / static_cast<float>(nk);
+    }
+    words_done += words;
+  }
+  __syncthreads();
+  // contiguous runs: for each pixel the block's words, then (last range only) the zero padding
+  const int64_t word0 = static_cast<int64_t>(chunk_first) * kTileCC * taps / 32;
+  const int run_bits = wrote_last ? static_cast<int>(ld_words - word0) : words_done;
+  const int run_scale = wrote_last ? static_cast<int>(ld_scales - word0) : words_done;
+  const int64_t m_base = (b * g.Ho + yo0) * g.Wo;
+  for (int idx = threadIdx.x; idx < pixels * run_bits; idx += 256) {
+    const int pix = idx / run_bits, w = idx - pix * run_bits;
+    bits[(m_base + pix) * ld_words + word0 + w] = (w < words_done) ? out_bits[pix * ldo + w] : 0u;
+  }
+  for (int idx = threadIdx.x; idx < pixels * run_scale; idx += 256) {
+    const int pix = idx / run_scale, w = idx - pix * run_scale;
+    store_scale(scales, scale_bf16, (m_base + pix) * ld_scales + word0 + w, (w < words_done) ? out_scale[pix * ldo + w] : 0.0f);
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_im2col_quantize(const void* x, int x_bf16, const ConvGeom& g, int32_t beta,
@@ -153,6 +367,28 @@ cudaError_t launch_im2col_quantize(const void* x, int x_bf16, const ConvGeom& g,
   const int64_t M = static_cast<int64_t>(g.B) * g.Ho * g.Wo, K = static_cast<int64_t>(g.C) * g.kh * g.kw;
   const int64_t beta_eff = beta >= K ? K : beta;
   const int64_t G = num_groups(K, beta);
+  if (beta == 32 && beta < K && g.sw == 1) {
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const TilePlan tp = make_plan(g, sms);
+    const int taps = g.kh * g.kw;
+    const size_t smem = static_cast<size_t>(kTileCC) * tp.rows_in * tp.span * 4 +
+                        2 * static_cast<size_t>(tp.RB) * g.Wo * (tp.chunks_per_split * taps + 1) * 4 +
+                        static_cast<size_t>(kTileCC) * taps * 2 + 16;
+    if (smem <= 160 * 1024 && static_cast<int64_t>(kTileCC) * tp.rows_in * tp.span < 65536) {
+      static size_t configured = 0;
+      if (smem > 48 * 1024 && smem > configured) {
+        if (cudaFuncSetAttribute(im2col_quantize_tiled_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 160 * 1024) != cudaSuccess) return cudaGetLastError();
+        configured = 160 * 1024;
+      }
+      dim3 grid(static_cast<unsigned>(static_cast<int64_t>(g.B) * tp.yo_blocks), static_cast<unsigned>(tp.splits));
+      im2col_quantize_tiled_kernel<<<grid, 256, smem, stream>>>(x, x_bf16, g, tp, K, G, (K + 31) / 32, bits, ld_words,
+                                                                scales, ld_scales, scale_bf16);
+      return cudaGetLastError();
+    }
+  }
   if (beta < K && beta % 32 == 0) {
     dim3 grid(static_cast<unsigned>((M + 31) / 32), static_cast<unsigned>((G + 7) / 8));
     im2col_quantize_groups_kernel<<<grid, 256, 0, stream>>>(x, x_bf16, g, M, K, beta / 32, G, (K + 31) / 32, bits,
@@ -168,6 +404,19 @@ cudaError_t launch_im2col_quantize(const void* x, int x_bf16, const ConvGeom& g,
 cudaError_t launch_im2col_bf16(const void* x, int x_bf16, const ConvGeom& g, void* out, int64_t ld,
                                cudaStream_t stream) {
   const int64_t M = static_cast<int64_t>(g.B) * g.Ho * g.Wo, K = static_cast<int64_t>(g.C) * g.kh * g.kw;
+  if (g.sw == 1 && ld % 8 == 0 && reinterpret_cast<uintptr_t>(out) % 16 == 0) {
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const TilePlan tp = make_plan(g, sms);
+    const int taps = g.kh * g.kw;
+    const size_t smem = static_cast<size_t>((kTileCC * taps + 7) / 8 * 8) * 2 + static_cast<size_t>(kTileCC) * tp.rows_in * tp.span * 2;
+    if (smem <= 48 * 1024 && static_cast<int64_t>(kTileCC) * tp.rows_in * tp.span < 65536) {
+      dim3 grid(static_cast<unsigned>(static_cast<int64_t>(g.B) * tp.yo_blocks), static_cast<unsigned>(tp.splits));
+      im2col_bf16_tiled_kernel<<<grid, 256, smem, stream>>>(x, x_bf16, g, tp, K, reinterpret_cast<__nv_bfloat16*>(out), ld);
+      return cudaGetLastError();
+    }
+  }
   int64_t blocks = (M * ld + 255) / 256;
   if (blocks > 148 * 64) blocks = 148 * 64;
   im2col_bf16_kernel<<<static_cast<unsigned>(blocks), 256, 0, stream>>>(x, x_bf16, g, M, K,

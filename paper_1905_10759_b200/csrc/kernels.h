@@ -48,7 +48,9 @@ cudaError_t launch_gemm_b1(const PackedView& A, const PackedView& W, float* C, i
 cudaError_t launch_partials_b1(const PackedView& A, const PackedView& W, int32_t* D,
                                cudaStream_t stream);
 
-// Packed x packed contraction with +-1 e4m3 operands on the tensor cores.
+// Packed x packed contraction with +-1 e4m3 operands on the tensor cores (tcgen05 / TMEM).
+// read_umma_error copies the device-side error word (0 = no bounded wait ever expired); it synchronises.
+cudaError_t read_umma_error(int* code);
 bool gemm_tensor_supported(const PackedView& A, const PackedView& W);
 cudaError_t launch_gemm_tensor(const PackedView& A, const PackedView& W, float* C, int64_t ldc,
                                cudaStream_t stream);

@@ -31,7 +31,7 @@ PATH_AUTO, PATH_POPC, PATH_B1MMA, PATH_TENSOR = 0, 1, 2, 3
 EXPORTS = [
     "hbmm_operand_bytes", "hbmm_quantize", "hbmm_gemm_workspace_bytes", "hbmm_gemm", "hbmm_gemm_ex",
     "hbmm_gemm_partials", "hbmm_conv_workspace_bytes", "hbmm_conv_im2col", "hbmm_status_string",
-    "hbmm_version", "hbmm_conv_im2col_static",
+    "hbmm_version", "hbmm_conv_im2col_static", "hbmm_last_device_error",
 ]
 STATIC_SCRATCH_BYTES = 32 << 20
 
@@ -65,6 +65,8 @@ _lib.hbmm_conv_im2col.argtypes = [_vp, _i32, _P(hbmm_conv_geom), _i32, _i32, _P(
                                   _vp, _sz, _vp]
 _lib.hbmm_conv_im2col_static.argtypes = [_vp, _i32, _P(hbmm_conv_geom), _i32, _i32, _P(hbmm_operand), _vp, _i64, _vp]
 _lib.hbmm_conv_im2col_static.restype = _i32
+_lib.hbmm_last_device_error.argtypes = [_P(_i32)]
+_lib.hbmm_last_device_error.restype = _i32
 _lib.hbmm_status_string.argtypes = [_i32]
 _lib.hbmm_status_string.restype = ctypes.c_char_p
 _lib.hbmm_version.restype = _i32
@@ -239,3 +241,12 @@ def conv_im2col_static(x: torch.Tensor, geom: hbmm_conv_geom, beta_a: int, a_sca
                                         ctypes.byref(W.desc), _dev_ptr(C_out), C_out.stride(0), _stream(stream)),
            "hbmm_conv_im2col_static")
     return C_out
+
+
+def last_device_error() -> int:
+    """hbmm_last_device_error: 0 when no bounded device-side wait has ever expired (synchronises)."""
+    code = _i32(0)
+    st = _lib.hbmm_last_device_error(ctypes.byref(code))
+    if st not in (OK, ERR_TIMEOUT):
+        raise HbmmError(st, "hbmm_last_device_error")
+    return int(code.value)

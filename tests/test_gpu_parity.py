@@ -17,7 +17,8 @@ RTOL_BF16 = 1e-2     # paths whose inputs or scales are stored in bf16, end to e
 @pytest.fixture(scope="module")
 def hb():
     from paper_1905_10759_b200 import hbmm
-    return hbmm
+    yield hbmm
+    assert hbmm.last_device_error() == 0      # no bounded device-side wait expired during these tests
 
 
 def _gu():
