@@ -8,7 +8,8 @@
 // warps read each finished segment from TMEM and apply C += (deltaA * D) * deltaW in fp32
 // registers, so every group keeps its own full-precision scale exactly as in the popcount path.
 //
-// CTA = 128 rows x TN columns, one CTA per SM (it owns all 512 TMEM columns).
+// CTA tile = 128 rows x TN columns; one persistent CTA per SM (it owns all 512 TMEM columns)
+// walks the tiles of the output.
 //   warps 0-7   : epilogue (warp w reads TMEM lanes 32*(w%4).., warps 0-3 the left half of the
 //                 columns, warps 4-7 the right half); they take most of the register file
 //   warps 8-11  : producers: packed words -> e4m3 bytes in the UMMA K-major core-matrix layout
@@ -32,8 +33,8 @@ constexpr int kProducerWarps = 4;                         // warpgroup 2
 constexpr int kFirstProducerWarp = kEpilogueWarps;        // warps 8..11
 constexpr int kMmaWarp = kEpilogueWarps + kProducerWarps; // warp 12 (warps 13..15 only rebalance registers)
 constexpr int kThreads = 16 * 32;                         // 512: four warpgroups
-constexpr int kRegsEpilogue = 200;                        // 256 threads x 200 + 256 threads x 56 = 64 K registers
-constexpr int kRegsOther = 56;
+constexpr int kRegsEpilogue = 184;                        // 256 threads x 184 + 256 threads x 72 = 64 K registers
+constexpr int kRegsOther = 72;
 constexpr int TM = 128;
 constexpr int WPS = 4;            // K-words per stage
 constexpr int STAGES = 4;
@@ -116,6 +117,44 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 template <int R> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(R)); }
 template <int R> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(R)); }
 
+// Two fp32 lanes per instruction (halves the issue slots of the scale epilogue).
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+
+// Four sign bits (in bits 0..3 or 4..7 of `v`, selected by the multiplier) -> four e4m3 bytes:
+// the multiply copies bit i to bit 8*i+7, the sign position of byte i; 0xB8 = -1.0, 0x38 = +1.0.
+__device__ __forceinline__ uint32_t signs_lo(uint32_t v) { return (((v & 0x0Fu) * 0x10204080u) & 0x80808080u) ^ 0xB8B8B8B8u; }
+__device__ __forceinline__ uint32_t signs_hi(uint32_t v) { return (((v & 0xF0u) * 0x01020408u) & 0x80808080u) ^ 0xB8B8B8B8u; }
+
+// Four packed K-words of one tile row -> 4 x 32 e4m3 bytes in the UMMA core-matrix layout of a stage:
+// [word][K-half (16 bytes)][row / 8][row % 8][16 bytes].
+__device__ __forceinline__ void expand_words(unsigned char* stage_base, int rows, int row, const uint4& w4) {
+  const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+  for (int q = 0; q < 4; q++) {
+    unsigned char* base = stage_base + q * rows * 32 + (row >> 3) * 128 + (row & 7) * 16;
+    const uint32_t y0 = w[q] & 0xFF, y1 = (w[q] >> 8) & 0xFF, y2 = (w[q] >> 16) & 0xFF, y3 = w[q] >> 24;
+    *reinterpret_cast<uint4*>(base) = make_uint4(signs_lo(y0), signs_hi(y0), signs_lo(y1), signs_hi(y1));              // K bytes 0..15
+    *reinterpret_cast<uint4*>(base + rows * 16) = make_uint4(signs_lo(y2), signs_hi(y2), signs_lo(y3), signs_hi(y3));  // K bytes 16..31
+  }
+}
+
 // K-major operand without swizzle: core matrices of 8 rows x 16 bytes stored contiguously
 // (128 bytes); `sbo` = byte distance between 8-row groups, `lbo` = byte distance between the two
 // 16-byte K-chunks of one K = 32 instruction.  Descriptor version 1, layout type 0.
@@ -142,8 +181,7 @@ struct Smem {
   static constexpr int OFF_B = OFF_A + STAGES * A_STAGE;
   static constexpr int OFF_SA = OFF_B + STAGES * B_STAGE;               // [STAGES][WPS][TM] float
   static constexpr int OFF_SW = OFF_SA + STAGES * WPS * TM * 4;         // [STAGES][WPS][TN] float
-  static constexpr int OFF_LUT = OFF_SW + STAGES * WPS * TN * 4;        // [256] uint2
-  static constexpr int OFF_BAR = OFF_LUT + 256 * 8;
+  static constexpr int OFF_BAR = OFF_SW + STAGES * WPS * TN * 4;
   static constexpr int NBUF = 512 / TN;                                 // TMEM accumulator buffers
   // barriers: full[STAGES], empty[STAGES], tfull[NBUF], tempty[NBUF], drain
   static constexpr int NBAR = 2 * STAGES + 2 * NBUF + 1;
@@ -153,7 +191,16 @@ struct Smem {
   static constexpr int BYTES = USED > 120 * 1024 ? USED : 120 * 1024;
 };
 
-template <int TN>
+// What one producer thread has fetched for one stage: four K-words and their scales for its A row
+// and its B row.
+struct Fetched {
+  uint4 wa, wb;
+  float fa[WPS], fb[WPS];
+};
+
+// FAST: one K-word per segment, both operands with beta = 32 and fp32 scales -- the four scales of a
+// stage are then one 16-byte vector per row, like the four words.
+template <int TN, bool FAST>
 __global__ void __launch_bounds__(kThreads, 1)
 hbmm_umma_kernel(const Args g) {
   using S = Smem<TN>;
@@ -167,25 +214,16 @@ hbmm_umma_kernel(const Args g) {
   uint64_t* drain = tempty + NBUF;
   uint32_t* tmem_base_ptr = reinterpret_cast<uint32_t*>(smem + S::OFF_MISC);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + S::OFF_MISC + 4);
-  uint2* lut = reinterpret_cast<uint2*>(smem + S::OFF_LUT);
   float* sA = reinterpret_cast<float*>(smem + S::OFF_SA);
   float* sW = reinterpret_cast<float*>(smem + S::OFF_SW);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int64_t m0 = static_cast<int64_t>(blockIdx.y) * TM, n0 = static_cast<int64_t>(blockIdx.x) * TN;
-  const int64_t n_stages = (g.n_words + WPS - 1) / WPS;
-  const int64_t n_segs = (g.n_words + g.seg_words - 1) / g.seg_words;
+  const int64_t tiles_n = (g.N + TN - 1) / TN, tiles_m = (g.M + TM - 1) / TM;
+  const int64_t n_tiles = tiles_m * tiles_n;
+  const int64_t n_stages = (g.n_words + WPS - 1) / WPS;                 // per tile
+  const int64_t n_segs = (g.n_words + g.seg_words - 1) / g.seg_words;   // per tile
 
   // ---- set-up
-  if (tid < 256) {  // byte of sign bits -> eight e4m3 bytes: 0x38 = +1.0 for bit 1, 0xB8 = -1.0 for bit 0
-    uint32_t lo = 0, hi = 0;
-#pragma unroll
-    for (int i = 0; i < 4; i++) {
-      lo |= (((tid >> i) & 1) ? 0x38u : 0xB8u) << (8 * i);
-      hi |= (((tid >> (i + 4)) & 1) ? 0x38u : 0xB8u) << (8 * i);
-    }
-    lut[tid] = make_uint2(lo, hi);
-  }
   if (tid == 0) {
     for (int s = 0; s < STAGES; s++) {
       mbar_init(&full[s], kProducerWarps);            // one arrival per producer warp
@@ -208,106 +246,148 @@ hbmm_umma_kernel(const Args g) {
   tc_fence_after();
   const uint32_t tmem_base = *tmem_base_ptr;
 
+  // The CTA is persistent: it walks tiles blockIdx.x, blockIdx.x + gridDim.x, ... and the stage and
+  // accumulator rings simply continue across tiles (gst / gseg count stages / segments since launch).
   if (warp >= kFirstProducerWarp && warp < kMmaWarp) {
     // =========================== producers ===========================
     reg_dec<kRegsOther>();
-    const int p = tid - kFirstProducerWarp * 32;   // 0..127: A row p and B row p
+    const int p = tid - kFirstProducerWarp * 32;   // 0..127: A row p and B row p of the tile
     const bool b_row = p < TN;
-    const int64_t m = m0 + p, n = n0 + p;
-    const bool a_in = m < g.M, b_in = b_row && n < g.N;
-    const uint32_t* a_ptr = g.a_bits + (a_in ? m : 0) * g.lda_w;
-    const uint32_t* b_ptr = g.w_bits + (b_in ? n : 0) * g.ldw_w;
-    const int64_t a_srow = (a_in ? m : 0) * g.lda_s, b_srow = (b_in ? n : 0) * g.ldw_s;
-    // running position of the next word to fetch: segment phase and the two group indices
-    int in_seg = 0, in_ga = 0, in_gw = 0;
-    int64_t ga = 0, gw = 0;
-    float cur_a = 0.0f, cur_w = 0.0f;
-    bool need_a = true, need_w = true;
-    uint4 wa, wb;
-    float fa[WPS], fb[WPS];
-    auto fetch = [&](int64_t st) {
-      const int64_t kw = st * WPS;
-      wa = make_uint4(0, 0, 0, 0);
-      wb = make_uint4(0, 0, 0, 0);
-      if (a_in && kw < g.lda_w) wa = __ldg(reinterpret_cast<const uint4*>(a_ptr + kw));
-      if (b_in && kw < g.ldw_w) wb = __ldg(reinterpret_cast<const uint4*>(b_ptr + kw));
-#pragma unroll
-      for (int q = 0; q < WPS; q++) {
-        const bool live = kw + q < g.n_words;
-        if (need_a) { cur_a = (a_in && live && ga < g.Ga) ? load_scale(g.a_scales, g.a_bf16, a_srow + ga) : 0.0f; need_a = false; }
-        if (need_w) { cur_w = (b_in && live && gw < g.Gw) ? load_scale(g.w_scales, g.w_bf16, b_srow + gw) : 0.0f; need_w = false; }
-        fa[q] = live ? cur_a : 0.0f;
-        fb[q] = live ? cur_w : 0.0f;
-        if (++in_seg == g.seg_words) {           // next word starts a new segment
-          in_seg = 0;
-          if (++in_ga == g.ra) { in_ga = 0; ga++; need_a = true; }
-          if (++in_gw == g.rw) { in_gw = 0; gw++; need_w = true; }
+    int64_t gst = 0;
+    bool ok = true;
+    if (FAST) {
+      // ---- one K-word per segment, fp32 scales: the four scales of a stage are one 16-byte vector
+      // like the four words.  All four loads of the next stage are in flight while this one is expanded.
+      const int64_t my_tiles = (n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x;
+      const int64_t total = my_tiles * n_stages;           // stages this CTA will produce
+      uint4 wa, wb, nwa, nwb;
+      float4 fa, fb, nfa, nfb;
+      auto fetch4 = [&](int64_t gs, uint4& xa, float4& ya, uint4& xb, float4& yb) {
+        const int64_t tile = blockIdx.x + (gs / n_stages) * gridDim.x, kw = (gs % n_stages) * WPS;
+        const int64_t m = (tile / tiles_n) * TM + p, n = (tile % tiles_n) * TN + p;
+        xa = make_uint4(0, 0, 0, 0); xb = make_uint4(0, 0, 0, 0);
+        ya = make_float4(0.f, 0.f, 0.f, 0.f); yb = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (m < g.M) {
+          if (kw < g.lda_w) xa = __ldg(reinterpret_cast<const uint4*>(g.a_bits + m * g.lda_w + kw));
+          if (kw < g.lda_s) ya = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(g.a_scales) + m * g.lda_s + kw));
         }
+        if (b_row && n < g.N) {
+          if (kw < g.ldw_w) xb = __ldg(reinterpret_cast<const uint4*>(g.w_bits + n * g.ldw_w + kw));
+          if (kw < g.ldw_s) yb = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(g.w_scales) + n * g.ldw_s + kw));
+        }
+      };
+      if (total > 0) fetch4(0, wa, fa, wb, fb);
+      for (; gst < total; gst++) {
+        if (gst + 1 < total) fetch4(gst + 1, nwa, nfa, nwb, nfb);
+        const int s = static_cast<int>(gst % STAGES);
+        if (gst >= STAGES && !mbar_wait(&empty[s], static_cast<uint32_t>(((gst / STAGES) & 1) ^ 1), abort_flag, 1)) break;
+        expand_words(smem + S::OFF_A + s * S::A_STAGE, TM, p, wa);
+        float* sa_dst = sA + s * WPS * TM + p;
+        sa_dst[0] = fa.x; sa_dst[TM] = fa.y; sa_dst[2 * TM] = fa.z; sa_dst[3 * TM] = fa.w;
+        if (b_row) {
+          expand_words(smem + S::OFF_B + s * S::B_STAGE, TN, p, wb);
+          float* sw_dst = sW + s * WPS * TN + p;
+          sw_dst[0] = fb.x; sw_dst[TN] = fb.y; sw_dst[2 * TN] = fb.z; sw_dst[3 * TN] = fb.w;
+        }
+        fence_async_proxy();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&full[s]);
+        wa = nwa; wb = nwb; fa = nfa; fb = nfb;
       }
-    };
-    auto expand_row = [&](unsigned char* tile, int rows, int row, const uint4& w4) {
-      const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+    } else
+    for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      const int64_t m = (tile / tiles_n) * TM + p, n = (tile % tiles_n) * TN + p;
+      const bool a_in = m < g.M, b_in = b_row && n < g.N;
+      const uint32_t* a_ptr = g.a_bits + (a_in ? m : 0) * g.lda_w;
+      const uint32_t* b_ptr = g.w_bits + (b_in ? n : 0) * g.ldw_w;
+      const int64_t a_srow = (a_in ? m : 0) * g.lda_s, b_srow = (b_in ? n : 0) * g.ldw_s;
+      // running position of the next word to fetch: segment phase and the two group indices
+      int in_seg = 0, in_ga = 0, in_gw = 0;
+      int64_t ga = 0, gw = 0;
+      auto fetch = [&](int64_t st, Fetched& f) {
+        const int64_t kw = st * WPS;
+        f.wa = make_uint4(0, 0, 0, 0);
+        f.wb = make_uint4(0, 0, 0, 0);
+        if (a_in && kw < g.lda_w) f.wa = __ldg(reinterpret_cast<const uint4*>(a_ptr + kw));
+        if (b_in && kw < g.ldw_w) f.wb = __ldg(reinterpret_cast<const uint4*>(b_ptr + kw));
+        // first decide which scale every word needs (no loaded value is touched here) ...
+        int64_t ia[WPS], iw[WPS];
 #pragma unroll
-      for (int q = 0; q < WPS; q++) {
-        unsigned char* base = tile + q * rows * 32 + (row >> 3) * 128 + (row & 7) * 16;
-        const uint2 b0 = lut[w[q] & 0xFF], b1 = lut[(w[q] >> 8) & 0xFF];
-        const uint2 b2 = lut[(w[q] >> 16) & 0xFF], b3 = lut[w[q] >> 24];
-        *reinterpret_cast<uint4*>(base) = make_uint4(b0.x, b0.y, b1.x, b1.y);                 // K bytes 0..15
-        *reinterpret_cast<uint4*>(base + rows * 16) = make_uint4(b2.x, b2.y, b3.x, b3.y);     // K bytes 16..31
+        for (int q = 0; q < WPS; q++) {
+          const bool live = kw + q < g.n_words;
+          ia[q] = (a_in && live && ga < g.Ga) ? a_srow + ga : -1;
+          iw[q] = (b_in && live && gw < g.Gw) ? b_srow + gw : -1;
+          if (++in_seg == g.seg_words) {           // next word starts a new segment
+            in_seg = 0;
+            if (++in_ga == g.ra) { in_ga = 0; ga++; }
+            if (++in_gw == g.rw) { in_gw = 0; gw++; }
+          }
+        }
+        // ... then issue the loads back to back (repeated indices hit the same cache line)
+#pragma unroll
+        for (int q = 0; q < WPS; q++) {
+          f.fa[q] = 0.0f; f.fb[q] = 0.0f;
+          if (ia[q] >= 0) f.fa[q] = load_scale(g.a_scales, g.a_bf16, ia[q]);
+          if (iw[q] >= 0) f.fb[q] = load_scale(g.w_scales, g.w_bf16, iw[q]);
+        }
+      };
+      Fetched cur, nxt;
+      fetch(0, cur);
+      for (int64_t st = 0; st < n_stages; st++, gst++) {
+        if (st + 1 < n_stages) fetch(st + 1, nxt);     // in flight while this stage is expanded
+        const int s = static_cast<int>(gst % STAGES);
+        if (gst >= STAGES && !mbar_wait(&empty[s], static_cast<uint32_t>(((gst / STAGES) & 1) ^ 1), abort_flag, 1)) { ok = false; break; }
+        expand_words(smem + S::OFF_A + s * S::A_STAGE, TM, p, cur.wa);
+#pragma unroll
+        for (int q = 0; q < WPS; q++) sA[(s * WPS + q) * TM + p] = cur.fa[q];
+        if (b_row) {
+          expand_words(smem + S::OFF_B + s * S::B_STAGE, TN, p, cur.wb);
+#pragma unroll
+          for (int q = 0; q < WPS; q++) sW[(s * WPS + q) * TN + p] = cur.fb[q];
+        }
+        fence_async_proxy();          // make the generic-proxy stores visible to the tensor core
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&full[s]);
+        cur = nxt;
       }
-    };
-    if (n_stages > 0) fetch(0);
-    for (int64_t st = 0; st < n_stages; st++) {
-      const int s = static_cast<int>(st % STAGES);
-      const uint32_t par = static_cast<uint32_t>((st / STAGES) & 1);
-      if (st >= STAGES && !mbar_wait(&empty[s], par ^ 1, abort_flag, 1)) break;
-      expand_row(smem + S::OFF_A + s * S::A_STAGE, TM, p, wa);
-#pragma unroll
-      for (int q = 0; q < WPS; q++) sA[(s * WPS + q) * TM + p] = fa[q];
-      if (b_row) {
-        expand_row(smem + S::OFF_B + s * S::B_STAGE, TN, p, wb);
-#pragma unroll
-        for (int q = 0; q < WPS; q++) sW[(s * WPS + q) * TN + p] = fb[q];
-      }
-      if (st + 1 < n_stages) fetch(st + 1);
-      fence_async_proxy();          // make the generic-proxy stores visible to the tensor core
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&full[s]);
     }
   } else if (warp == kMmaWarp) {
     // =========================== MMA issuer ===========================
     reg_dec<kRegsOther>();
     if (lane == 0) {
       constexpr uint32_t idesc = instr_desc_f8(TN);
-      int64_t seg = 0;      // segment being accumulated
+      int64_t gst = 0, gseg = 0;
       bool ok = true;
-      for (int64_t st = 0; st < n_stages && ok; st++) {
-        const int s = static_cast<int>(st % STAGES);
-        if (!mbar_wait(&full[s], static_cast<uint32_t>((st / STAGES) & 1), abort_flag, 2)) { ok = false; break; }
-        tc_fence_after();
-        const uint32_t a_addr = smem_u32(smem + S::OFF_A + s * S::A_STAGE);
-        const uint32_t b_addr = smem_u32(smem + S::OFF_B + s * S::B_STAGE);
-        for (int q = 0; q < WPS; q++) {
-          const int64_t kw = st * WPS + q;
-          if (kw >= g.n_words) break;
-          const int64_t in_seg = kw - seg * g.seg_words;
-          const int buf = static_cast<int>(seg % NBUF);
-          if (in_seg == 0 && seg >= NBUF) {
-            if (!mbar_wait(&tempty[buf], static_cast<uint32_t>(((seg / NBUF) & 1) ^ 1), abort_flag, 3)) { ok = false; break; }
-            tc_fence_after();
+      for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        int64_t in_seg = 0;
+        for (int64_t st = 0; st < n_stages && ok; st++, gst++) {
+          const int s = static_cast<int>(gst % STAGES);
+          if (!mbar_wait(&full[s], static_cast<uint32_t>((gst / STAGES) & 1), abort_flag, 2)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(smem + S::OFF_A + s * S::A_STAGE);
+          const uint32_t b_addr = smem_u32(smem + S::OFF_B + s * S::B_STAGE);
+          for (int q = 0; q < WPS; q++) {
+            const int64_t kw = st * WPS + q;
+            if (kw >= g.n_words) break;
+            const int buf = static_cast<int>(gseg % NBUF);
+            if (in_seg == 0 && gseg >= NBUF) {
+              if (!mbar_wait(&tempty[buf], static_cast<uint32_t>(((gseg / NBUF) & 1) ^ 1), abort_flag, 3)) { ok = false; break; }
+              tc_fence_after();
+            }
+            umma_f8(tmem_base + buf * TN,
+                    smem_desc(a_addr + q * S::A_WORD_BYTES, TM * 16, 128),
+                    smem_desc(b_addr + q * S::B_WORD_BYTES, TN * 16, 128), idesc, in_seg != 0 ? 1u : 0u);
+            if (++in_seg == g.seg_words || kw == g.n_words - 1) {
+              umma_commit(&tfull[buf]);     // segment complete: hand the accumulator to the epilogue
+              gseg++;
+              in_seg = 0;
+            }
           }
-          umma_f8(tmem_base + buf * TN,
-                  smem_desc(a_addr + q * S::A_WORD_BYTES, TM * 16, 128),
-                  smem_desc(b_addr + q * S::B_WORD_BYTES, TN * 16, 128), idesc, in_seg != 0 ? 1u : 0u);
-          if (in_seg == g.seg_words - 1 || kw == g.n_words - 1) {
-            umma_commit(&tfull[buf]);     // segment complete: hand the accumulator to the epilogue
-            seg++;
-          }
+          umma_commit(&empty[s]);           // stage's bytes are free once these MMAs have read them
         }
-        umma_commit(&empty[s]);           // stage's bytes are free once these MMAs have read them
       }
       umma_commit(drain);
-      mbar_wait(drain, 0, abort_flag, 4); // every MMA has retired before TMEM is released
+      mbar_wait(drain, 0, abort_flag, 4);   // every MMA has retired before TMEM is released
     }
     __syncwarp();
   } else if (warp < kEpilogueWarps) {
@@ -316,57 +396,62 @@ hbmm_umma_kernel(const Args g) {
     const int wg = warp >> 2;                       // column half
     const int row = (warp & 3) * 32 + lane;         // TMEM lane = tile row
     const uint32_t t_lane = static_cast<uint32_t>((warp & 3) * 32) << 16;
-    float acc[HALF];
-#pragma unroll
-    for (int j = 0; j < HALF; j++) acc[j] = 0.0f;
+    int64_t gseg = 0, gst_base = 0, released = 0;   // released: stages handed back to the producers so far
     bool ok = true;
-    int64_t released = 0;   // stages this warp has handed back to the producers
-    for (int64_t seg = 0; seg < n_segs && ok; seg++) {
-      const int buf = static_cast<int>(seg % NBUF);
-      if (!mbar_wait(&tfull[buf], static_cast<uint32_t>((seg / NBUF) & 1), abort_flag, 5)) { ok = false; break; }
-      tc_fence_after();
-      int64_t kw_last = (seg + 1) * g.seg_words - 1;        // the word that carries this segment's scales
-      if (kw_last > g.n_words - 1) kw_last = g.n_words - 1;
-      const int64_t st = kw_last / WPS;
-      const int s = static_cast<int>(st % STAGES), q = static_cast<int>(kw_last % WPS);
-      const float sa = sA[(s * WPS + q) * TM + row];
-      const float* swp = sW + (s * WPS + q) * TN + wg * HALF;
-      uint32_t d[HALF / 32][32];
+    for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, gst_base += n_stages) {
+      uint64_t acc[HALF / 2];                       // two fp32 outputs per register pair
 #pragma unroll
-      for (int c = 0; c < HALF / 32; c++) tmem_ld32(tmem_base + t_lane + buf * TN + wg * HALF + c * 32, d[c]);
-      tmem_ld_wait();
+      for (int j = 0; j < HALF / 2; j++) acc[j] = 0ull;
+      for (int64_t seg = 0; seg < n_segs; seg++, gseg++) {
+        const int buf = static_cast<int>(gseg % NBUF);
+        if (!mbar_wait(&tfull[buf], static_cast<uint32_t>((gseg / NBUF) & 1), abort_flag, 5)) { ok = false; break; }
+        tc_fence_after();
+        int64_t kw_last = (seg + 1) * g.seg_words - 1;        // the word that carries this segment's scales
+        if (kw_last > g.n_words - 1) kw_last = g.n_words - 1;
+        const int64_t st = gst_base + kw_last / WPS;
+        const int s = static_cast<int>(st % STAGES), q = static_cast<int>(kw_last % WPS);
+        const float sa = sA[(s * WPS + q) * TM + row];
+        const uint64_t sa2 = pack2(sa, sa);
+        const float* swp = sW + (s * WPS + q) * TN + wg * HALF;
+        uint32_t d[HALF / 32][32];
 #pragma unroll
-      for (int c = 0; c < HALF / 32; c++)
+        for (int c = 0; c < HALF / 32; c++) tmem_ld32(tmem_base + t_lane + buf * TN + wg * HALF + c * 32, d[c]);
+        tmem_ld_wait();
 #pragma unroll
-        for (int j = 0; j < 32; j += 4) {
-          const float4 sw = *reinterpret_cast<const float4*>(swp + c * 32 + j);
-          acc[c * 32 + j + 0] = fmaf(sa * __uint_as_float(d[c][j + 0]), sw.x, acc[c * 32 + j + 0]);
-          acc[c * 32 + j + 1] = fmaf(sa * __uint_as_float(d[c][j + 1]), sw.y, acc[c * 32 + j + 1]);
-          acc[c * 32 + j + 2] = fmaf(sa * __uint_as_float(d[c][j + 2]), sw.z, acc[c * 32 + j + 2]);
-          acc[c * 32 + j + 3] = fmaf(sa * __uint_as_float(d[c][j + 3]), sw.w, acc[c * 32 + j + 3]);
+        for (int c = 0; c < HALF / 32; c++)
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            const float4 sw = *reinterpret_cast<const float4*>(swp + c * 32 + j);
+            const uint64_t t0 = mul2(sa2, pack2(__uint_as_float(d[c][j + 0]), __uint_as_float(d[c][j + 1])));
+            const uint64_t t1 = mul2(sa2, pack2(__uint_as_float(d[c][j + 2]), __uint_as_float(d[c][j + 3])));
+            acc[(c * 32 + j) / 2] = fma2(t0, pack2(sw.x, sw.y), acc[(c * 32 + j) / 2]);
+            acc[(c * 32 + j) / 2 + 1] = fma2(t1, pack2(sw.z, sw.w), acc[(c * 32 + j) / 2 + 1]);
+          }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(&tempty[buf]);
+          // release every stage whose words are now all consumed (their scales will not be read again)
+          int64_t done_words = (seg + 1) * g.seg_words;
+          if (done_words > g.n_words) done_words = g.n_words;
+          const int64_t consumed = gst_base + ((done_words == g.n_words) ? n_stages : done_words / WPS);
+          for (; released < consumed; released++) mbar_arrive(&empty[released % STAGES]);
         }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) {
-        mbar_arrive(&tempty[buf]);
-        // release every stage whose words are now all consumed (their scales will not be read again)
-        int64_t done_words = (seg + 1) * g.seg_words;
-        if (done_words > g.n_words) done_words = g.n_words;
-        const int64_t consumed = (done_words == g.n_words) ? n_stages : done_words / WPS;
-        for (; released < consumed; released++) mbar_arrive(&empty[released % STAGES]);
       }
-    }
-    if (ok) {
-      const int64_t m = m0 + row;
-      if (m < g.M) {
-        float* dst = g.C + m * g.ldc + n0 + wg * HALF;
+      if (ok) {
+        const int64_t m = (tile / tiles_n) * TM + row, nb = (tile % tiles_n) * TN + wg * HALF;
+        if (m < g.M) {
+          float* dst = g.C + m * g.ldc + nb;
 #pragma unroll
-        for (int j = 0; j < HALF; j += 4) {
-          const int64_t n = n0 + wg * HALF + j;
-          if (n + 3 < g.N) *reinterpret_cast<float4*>(dst + j) = make_float4(acc[j], acc[j + 1], acc[j + 2], acc[j + 3]);
-          else
-            for (int e = 0; e < 4; e++)
-              if (n + e < g.N) dst[j + e] = acc[j + e];
+          for (int j = 0; j < HALF; j += 4) {
+            float v[4];
+            unpack2(acc[j / 2], v[0], v[1]);
+            unpack2(acc[j / 2 + 1], v[2], v[3]);
+            if (nb + j + 3 < g.N) *reinterpret_cast<float4*>(dst + j) = make_float4(v[0], v[1], v[2], v[3]);
+            else
+              for (int e = 0; e < 4; e++)
+                if (nb + j + e < g.N) dst[j + e] = v[e];
+          }
         }
       }
     }
@@ -381,6 +466,25 @@ hbmm_umma_kernel(const Args g) {
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
   }
+}
+
+template <int TN, bool FAST>
+cudaError_t launch_umma(const Args& g, cudaStream_t stream) {
+  using S = Smem<TN>;
+  static bool configured = false;
+  static int sms = 0;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(hbmm_umma_kernel<TN, FAST>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::BYTES);
+    if (e != cudaSuccess) return e;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    configured = true;
+  }
+  const int64_t tiles = ((g.M + TM - 1) / TM) * ((g.N + TN - 1) / TN);
+  const unsigned grid = static_cast<unsigned>(tiles < sms ? tiles : sms);   // one persistent CTA per SM
+  hbmm_umma_kernel<TN, FAST><<<grid, kThreads, S::BYTES, stream>>>(g);
+  return cudaGetLastError();
 }
 
 }  // namespace
@@ -412,27 +516,9 @@ cudaError_t launch_gemm_tensor(const PackedView& A, const PackedView& W, float* 
   g.rw = static_cast<int32_t>(w_one ? T : W.beta / seg);
   g.Ga = num_groups(A.K, A.beta);
   g.Gw = num_groups(W.K, W.beta);
-  static bool configured[2] = {false, false};
-  if (g.N <= 64) {
-    using S = Smem<64>;
-    if (!configured[0]) {
-      cudaError_t e = cudaFuncSetAttribute(hbmm_umma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::BYTES);
-      if (e != cudaSuccess) return e;
-      configured[0] = true;
-    }
-    dim3 grid(static_cast<unsigned>((g.N + 63) / 64), static_cast<unsigned>((g.M + TM - 1) / TM));
-    hbmm_umma_kernel<64><<<grid, kThreads, S::BYTES, stream>>>(g);
-  } else {
-    using S = Smem<128>;
-    if (!configured[1]) {
-      cudaError_t e = cudaFuncSetAttribute(hbmm_umma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::BYTES);
-      if (e != cudaSuccess) return e;
-      configured[1] = true;
-    }
-    dim3 grid(static_cast<unsigned>((g.N + 127) / 128), static_cast<unsigned>((g.M + TM - 1) / TM));
-    hbmm_umma_kernel<128><<<grid, kThreads, S::BYTES, stream>>>(g);
-  }
-  return cudaGetLastError();
+  const bool fast = g.seg_words == 1 && g.ra == 1 && g.rw == 1 && !g.a_bf16 && !g.w_bf16;
+  if (fast) return g.N <= 64 ? launch_umma<64, true>(g, stream) : launch_umma<128, true>(g, stream);
+  return g.N <= 64 ? launch_umma<64, false>(g, stream) : launch_umma<128, false>(g, stream);
 }
 
 cudaError_t read_umma_error(int* code) {
