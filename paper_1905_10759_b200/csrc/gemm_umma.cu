@@ -1,20 +1,28 @@
 // HBMM contraction of two packed operands on the 5th-generation tensor cores (tcgen05 / TMEM).
 //
-// Section 4.2, Eq. 7: per K-segment one signed +-1 dot product and two full-precision multiplies.
-// Here the +-1 dot of a segment is a dense contraction: the sign bits of both operands are
-// expanded to +-1.0 in e4m3 (one byte per element, products and sums of at most a few thousand
-// +-1 terms are exact in the fp32 accumulator), and one tcgen05.mma (kind::f8f6f4, K = 32) per
-// 32-bit K-word accumulates the segment's dot for a 128 x TN tile in tensor memory.  The epilogue
-// warps read each finished segment from TMEM and apply C += (deltaA * D) * deltaW in fp32
-// registers, so every group keeps its own full-precision scale exactly as in the popcount path.
+// Section 4.2, Eq. 7: per K-segment one signed +-1 dot product D and two full-precision multiplies,
+//   C[m,n] += (deltaA[m,seg] * deltaW[n,seg]) * D[m,n].
+// Both factors of every term are produced by the tensor cores:
+//   * D: the sign bits of both operands are expanded to +-1.0 in e4m3 (one byte per element; sums of
+//     a few thousand +-1 products are exact in the fp32 accumulator) and one tcgen05.mma
+//     (kind::f8f6f4, K = 32) per 32-bit K-word accumulates the segment's dot of a 128 x TN tile in
+//     tensor memory.
+//   * S = deltaA (x) deltaW: each fp32 scale is split into three bf16 pieces a = a1 + a2 + a3
+//     (24 significant bits), and one small tcgen05.mma (kind::f16, K = 16, six non-zero columns)
+//     forms a1w1 + a1w2 + a2w1 + a2w2 + a1w3 + a3w1 -- every bf16 x bf16 product is exact in fp32
+//     and the omitted cross terms are below 2^-26 of the product -- so the scale product of the
+//     whole tile arrives in tensor memory at fp32 accuracy without touching the FMA pipe.
+// The epilogue warps then read D and S from TMEM and do one fp32 FMA per output and segment,
+// C += S * D, two outputs per instruction (fma.rn.f32x2).  Every group keeps its own full-precision
+// scale exactly as in the popcount path.
 //
 // CTA tile = 128 rows x TN columns; one persistent CTA per SM (it owns all 512 TMEM columns)
 // walks the tiles of the output.
 //   warps 0-7   : epilogue (warp w reads TMEM lanes 32*(w%4).., warps 0-3 the left half of the
 //                 columns, warps 4-7 the right half); they take most of the register file
-//   warps 8-11  : producers: packed words -> e4m3 bytes in the UMMA K-major core-matrix layout
-//                 (8 rows x 16 bytes contiguous), plus the segment scales of the stage
-//   warp  12    : TMEM allocation and the single MMA-issuing thread
+//   warps 8-11  : A producers, warps 12-15 : B producers: packed words -> e4m3 bytes and scales ->
+//                 bf16 pieces, both in the UMMA K-major core-matrix layout (8 rows x 16 bytes contiguous)
+//   warp  16    : TMEM allocation and the single MMA-issuing thread (warps 17-19 only hand registers over)
 // A stage holds four K-words; stages and TMEM accumulator buffers are rings guarded by
 // mbarriers.  Every wait is bounded: when a limit expires the thread records an error code in
 // global memory, raises a CTA-wide abort flag that all other waits observe, and the kernel
@@ -29,12 +37,12 @@ __device__ int g_umma_error = 0;  // 0 = ok; otherwise the code of the first wai
 namespace {
 
 constexpr int kEpilogueWarps = 8;                         // warpgroups 0 and 1
-constexpr int kProducerWarps = 4;                         // warpgroup 2
-constexpr int kFirstProducerWarp = kEpilogueWarps;        // warps 8..11
-constexpr int kMmaWarp = kEpilogueWarps + kProducerWarps; // warp 12 (warps 13..15 only rebalance registers)
-constexpr int kThreads = 16 * 32;                         // 512: four warpgroups
-constexpr int kRegsEpilogue = 184;                        // 256 threads x 184 + 256 threads x 72 = 64 K registers
-constexpr int kRegsOther = 72;
+constexpr int kProducerWarps = 8;                         // warpgroup 2 (A rows) and warpgroup 3 (B rows)
+constexpr int kFirstProducerWarp = kEpilogueWarps;        // warps 8..15
+constexpr int kMmaWarp = kEpilogueWarps + kProducerWarps; // warp 16
+constexpr int kThreads = 20 * 32;                         // 640: five warpgroups
+constexpr int kRegsEpilogue = 144;                        // 256 x 144 + 384 x 64 = 61440 = 640 x 96, the CTA's register allocation at launch
+constexpr int kRegsOther = 64;
 constexpr int TM = 128;
 constexpr int WPS = 4;            // K-words per stage
 constexpr int STAGES = 4;
@@ -118,23 +126,25 @@ template <int R> __device__ __forceinline__ void reg_inc() { asm volatile("setma
 template <int R> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(R)); }
 
 // Two fp32 lanes per instruction (halves the issue slots of the scale epilogue).
-__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+__device__ __forceinline__ uint64_t pack2(uint32_t lo, uint32_t hi) {
   uint64_t r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
   return r;
 }
 __device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
   asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
 }
-__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
-  uint64_t r;
-  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-  return r;
-}
 __device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
   uint64_t r;
   asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
   return r;
+}
+// D[tmem] = A[smem desc] * B[smem desc]^T, 128 x N x 16, bf16 operands, fp32 result (overwrites).
+__device__ __forceinline__ void umma_bf16_overwrite(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, 0, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc) : "memory");
 }
 
 // Four sign bits (in bits 0..3 or 4..7 of `v`, selected by the multiplier) -> four e4m3 bytes:
@@ -155,9 +165,29 @@ __device__ __forceinline__ void expand_words(unsigned char* stage_base, int rows
   }
 }
 
+// fp32 scale -> three bf16 pieces with a = a1 + a2 + a3 up to 2^-26 |a| (each remainder is exact in fp32).
+__device__ __forceinline__ void split3(float a, uint32_t& h1, uint32_t& h2, uint32_t& h3) {
+  const __nv_bfloat16 b1 = __float2bfloat16_rn(a);
+  const float r1 = a - __bfloat162float(b1);
+  const __nv_bfloat16 b2 = __float2bfloat16_rn(r1);
+  const float r2 = r1 - __bfloat162float(b2);
+  const __nv_bfloat16 b3 = __float2bfloat16_rn(r2);
+  h1 = __bfloat16_as_ushort(b1); h2 = __bfloat16_as_ushort(b2); h3 = __bfloat16_as_ushort(b3);
+}
+// One row of the scale operands of a segment: eight bf16 (K columns 0..7; columns 8..15 read a shared
+// block of zeros).  Row of A': (a1, a1, a2, a2, a1, a3, 0, 0); row of B': (w1, w2, w1, w2, w3, w1, 0, 0):
+// their dot product is a1w1 + a1w2 + a2w1 + a2w2 + a1w3 + a3w1.
+template <bool IS_B>
+__device__ __forceinline__ uint4 scale_row(float v) {
+  uint32_t h1, h2, h3;
+  split3(v, h1, h2, h3);
+  if (IS_B) return make_uint4(h1 | (h2 << 16), h1 | (h2 << 16), h3 | (h1 << 16), 0u);
+  return make_uint4(h1 | (h1 << 16), h2 | (h2 << 16), h1 | (h3 << 16), 0u);
+}
+
 // K-major operand without swizzle: core matrices of 8 rows x 16 bytes stored contiguously
 // (128 bytes); `sbo` = byte distance between 8-row groups, `lbo` = byte distance between the two
-// 16-byte K-chunks of one K = 32 instruction.  Descriptor version 1, layout type 0.
+// 16-byte K-chunks of one instruction.  Descriptor version 1, layout type 0.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
   uint64_t d = 0;
   d |= static_cast<uint64_t>((addr >> 4) & 0x3FFF);
@@ -166,10 +196,12 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint3
   d |= static_cast<uint64_t>(1) << 46;
   return d;
 }
-// Instruction descriptor: fp32 accumulator, e4m3 x e4m3, both K-major, M = 128, N = TN.
-__host__ __device__ constexpr uint32_t instr_desc_f8(int n) {
-  return (1u << 4) | (0u << 7) | (0u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(TM >> 4) << 24);
+// Instruction descriptors: fp32 accumulator, both operands K-major, M = 128, N = n.
+__host__ __device__ constexpr uint32_t instr_desc(int n, uint32_t ab_format) {
+  return (1u << 4) | (ab_format << 7) | (ab_format << 10) | (static_cast<uint32_t>(n >> 3) << 17) |
+         (static_cast<uint32_t>(TM >> 4) << 24);
 }
+constexpr uint32_t kFmtE4M3 = 0, kFmtBF16 = 1;
 
 template <int TN>
 struct Smem {
@@ -177,12 +209,15 @@ struct Smem {
   static constexpr int B_WORD_BYTES = TN * 32;
   static constexpr int A_STAGE = WPS * A_WORD_BYTES;
   static constexpr int B_STAGE = WPS * B_WORD_BYTES;
+  static constexpr int SA_WORD_BYTES = TM * 16;           // scale pieces of one word slot: 8 bf16 per row
+  static constexpr int SB_WORD_BYTES = TN * 16;
   static constexpr int OFF_A = 0;
   static constexpr int OFF_B = OFF_A + STAGES * A_STAGE;
-  static constexpr int OFF_SA = OFF_B + STAGES * B_STAGE;               // [STAGES][WPS][TM] float
-  static constexpr int OFF_SW = OFF_SA + STAGES * WPS * TM * 4;         // [STAGES][WPS][TN] float
-  static constexpr int OFF_BAR = OFF_SW + STAGES * WPS * TN * 4;
-  static constexpr int NBUF = 512 / TN;                                 // TMEM accumulator buffers
+  static constexpr int OFF_SA = OFF_B + STAGES * B_STAGE;               // [STAGES][WPS][TM rows][16 bytes]
+  static constexpr int OFF_SB = OFF_SA + STAGES * WPS * SA_WORD_BYTES;  // [STAGES][WPS][TN rows][16 bytes]
+  static constexpr int OFF_ZERO = OFF_SB + STAGES * WPS * SB_WORD_BYTES;  // 128 rows x 16 bytes of zeros
+  static constexpr int OFF_BAR = OFF_ZERO + TM * 16;
+  static constexpr int NBUF = 512 / (2 * TN);                           // TMEM buffers: D and S side by side
   // barriers: full[STAGES], empty[STAGES], tfull[NBUF], tempty[NBUF], drain
   static constexpr int NBAR = 2 * STAGES + 2 * NBUF + 1;
   static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;                   // tmem base, abort flag
@@ -191,21 +226,20 @@ struct Smem {
   static constexpr int BYTES = USED > 120 * 1024 ? USED : 120 * 1024;
 };
 
-// What one producer thread has fetched for one stage: four K-words and their scales for its A row
-// and its B row.
-struct Fetched {
-  uint4 wa, wb;
-  float fa[WPS], fb[WPS];
+// One side (A or B) of the producer: this thread owns tile row `p` of that operand.
+struct Side {
+  const uint32_t* bits; const void* scales;
+  int64_t rows, ld_w, ld_s, G;
+  int32_t bf16, r;       // r: segments per group of this operand
 };
 
-// FAST: one K-word per segment, both operands with beta = 32 and fp32 scales -- the four scales of a
-// stage are then one 16-byte vector per row, like the four words.
-template <int TN, bool FAST>
+template <int TN>
 __global__ void __launch_bounds__(kThreads, 1)
 hbmm_umma_kernel(const Args g) {
   using S = Smem<TN>;
   constexpr int NBUF = S::NBUF;
   constexpr int HALF = TN / 2;                  // columns per epilogue warpgroup
+  constexpr int CH = HALF / 32;                 // 32-column chunks per epilogue warp
   extern __shared__ __align__(1024) unsigned char smem[];
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + S::OFF_BAR);
   uint64_t* empty = full + STAGES;
@@ -214,20 +248,21 @@ hbmm_umma_kernel(const Args g) {
   uint64_t* drain = tempty + NBUF;
   uint32_t* tmem_base_ptr = reinterpret_cast<uint32_t*>(smem + S::OFF_MISC);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + S::OFF_MISC + 4);
-  float* sA = reinterpret_cast<float*>(smem + S::OFF_SA);
-  float* sW = reinterpret_cast<float*>(smem + S::OFF_SW);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int64_t tiles_n = (g.N + TN - 1) / TN, tiles_m = (g.M + TM - 1) / TM;
   const int64_t n_tiles = tiles_m * tiles_n;
   const int64_t n_stages = (g.n_words + WPS - 1) / WPS;                 // per tile
   const int64_t n_segs = (g.n_words + g.seg_words - 1) / g.seg_words;   // per tile
+  // producer arrivals per stage: the four A warps, and as many B warps as the tile has rows for
+  constexpr int kBWarps = TN / 32 < 4 ? TN / 32 : 4;
 
   // ---- set-up
+  if (tid < TM) *reinterpret_cast<uint4*>(smem + S::OFF_ZERO + tid * 16) = make_uint4(0, 0, 0, 0);
   if (tid == 0) {
     for (int s = 0; s < STAGES; s++) {
-      mbar_init(&full[s], kProducerWarps);            // one arrival per producer warp
-      mbar_init(&empty[s], 1 + kEpilogueWarps);       // MMA commit + every epilogue warp (scales read)
+      mbar_init(&full[s], 4 + kBWarps);               // one arrival per working producer warp
+      mbar_init(&empty[s], 1);                        // MMA commit: the stage's bytes have been read
     }
     for (int b = 0; b < NBUF; b++) {
       mbar_init(&tfull[b], 1);                        // MMA commit
@@ -237,6 +272,7 @@ hbmm_umma_kernel(const Args g) {
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  fence_async_proxy();                                // the zero block is read by the tensor core
   if (warp == kMmaWarp) {
     tmem_alloc(tmem_base_ptr, 512);
     tmem_relinquish();
@@ -251,111 +287,75 @@ hbmm_umma_kernel(const Args g) {
   if (warp >= kFirstProducerWarp && warp < kMmaWarp) {
     // =========================== producers ===========================
     reg_dec<kRegsOther>();
-    const int p = tid - kFirstProducerWarp * 32;   // 0..127: A row p and B row p of the tile
-    const bool b_row = p < TN;
-    int64_t gst = 0;
-    bool ok = true;
-    if (FAST) {
-      // ---- one K-word per segment, fp32 scales: the four scales of a stage are one 16-byte vector
-      // like the four words.  All four loads of the next stage are in flight while this one is expanded.
-      const int64_t my_tiles = (n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x;
-      const int64_t total = my_tiles * n_stages;           // stages this CTA will produce
-      uint4 wa, wb, nwa, nwb;
-      float4 fa, fb, nfa, nfb;
-      auto fetch4 = [&](int64_t gs, uint4& xa, float4& ya, uint4& xb, float4& yb) {
-        const int64_t tile = blockIdx.x + (gs / n_stages) * gridDim.x, kw = (gs % n_stages) * WPS;
-        const int64_t m = (tile / tiles_n) * TM + p, n = (tile % tiles_n) * TN + p;
-        xa = make_uint4(0, 0, 0, 0); xb = make_uint4(0, 0, 0, 0);
-        ya = make_float4(0.f, 0.f, 0.f, 0.f); yb = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (m < g.M) {
-          if (kw < g.lda_w) xa = __ldg(reinterpret_cast<const uint4*>(g.a_bits + m * g.lda_w + kw));
-          if (kw < g.lda_s) ya = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(g.a_scales) + m * g.lda_s + kw));
-        }
-        if (b_row && n < g.N) {
-          if (kw < g.ldw_w) xb = __ldg(reinterpret_cast<const uint4*>(g.w_bits + n * g.ldw_w + kw));
-          if (kw < g.ldw_s) yb = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(g.w_scales) + n * g.ldw_s + kw));
-        }
-      };
-      if (total > 0) fetch4(0, wa, fa, wb, fb);
-      for (; gst < total; gst++) {
-        if (gst + 1 < total) fetch4(gst + 1, nwa, nfa, nwb, nfb);
-        const int s = static_cast<int>(gst % STAGES);
-        if (gst >= STAGES && !mbar_wait(&empty[s], static_cast<uint32_t>(((gst / STAGES) & 1) ^ 1), abort_flag, 1)) break;
-        expand_words(smem + S::OFF_A + s * S::A_STAGE, TM, p, wa);
-        float* sa_dst = sA + s * WPS * TM + p;
-        sa_dst[0] = fa.x; sa_dst[TM] = fa.y; sa_dst[2 * TM] = fa.z; sa_dst[3 * TM] = fa.w;
-        if (b_row) {
-          expand_words(smem + S::OFF_B + s * S::B_STAGE, TN, p, wb);
-          float* sw_dst = sW + s * WPS * TN + p;
-          sw_dst[0] = fb.x; sw_dst[TN] = fb.y; sw_dst[2 * TN] = fb.z; sw_dst[3 * TN] = fb.w;
-        }
-        fence_async_proxy();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&full[s]);
-        wa = nwa; wb = nwb; fa = nfa; fb = nfb;
-      }
-    } else
-    for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-      const int64_t m = (tile / tiles_n) * TM + p, n = (tile % tiles_n) * TN + p;
-      const bool a_in = m < g.M, b_in = b_row && n < g.N;
-      const uint32_t* a_ptr = g.a_bits + (a_in ? m : 0) * g.lda_w;
-      const uint32_t* b_ptr = g.w_bits + (b_in ? n : 0) * g.ldw_w;
-      const int64_t a_srow = (a_in ? m : 0) * g.lda_s, b_srow = (b_in ? n : 0) * g.ldw_s;
-      // running position of the next word to fetch: segment phase and the two group indices
-      int in_seg = 0, in_ga = 0, in_gw = 0;
-      int64_t ga = 0, gw = 0;
-      auto fetch = [&](int64_t st, Fetched& f) {
-        const int64_t kw = st * WPS;
-        f.wa = make_uint4(0, 0, 0, 0);
-        f.wb = make_uint4(0, 0, 0, 0);
-        if (a_in && kw < g.lda_w) f.wa = __ldg(reinterpret_cast<const uint4*>(a_ptr + kw));
-        if (b_in && kw < g.ldw_w) f.wb = __ldg(reinterpret_cast<const uint4*>(b_ptr + kw));
-        // first decide which scale every word needs (no loaded value is touched here) ...
-        int64_t ia[WPS], iw[WPS];
+    const bool is_b = warp >= kFirstProducerWarp + 4;
+    const int p = (tid - kFirstProducerWarp * 32) & 127;    // tile row of this thread's operand
+    const int rows = is_b ? TN : TM;
+    if (p < rows) {                                          // (whole warps: TN is a multiple of 32)
+      Side sd;
+      if (is_b) { sd.bits = g.w_bits; sd.scales = g.w_scales; sd.rows = g.N; sd.ld_w = g.ldw_w; sd.ld_s = g.ldw_s; sd.G = g.Gw; sd.bf16 = g.w_bf16; sd.r = g.rw; }
+      else      { sd.bits = g.a_bits; sd.scales = g.a_scales; sd.rows = g.M; sd.ld_w = g.lda_w; sd.ld_s = g.lda_s; sd.G = g.Ga; sd.bf16 = g.a_bf16; sd.r = g.ra; }
+      unsigned char* sign_base = smem + (is_b ? S::OFF_B : S::OFF_A);
+      const int sign_stage = is_b ? S::B_STAGE : S::A_STAGE;
+      unsigned char* sc_row = smem + (is_b ? S::OFF_SB : S::OFF_SA) + (p >> 3) * 128 + (p & 7) * 16;
+      const int sc_word = is_b ? S::SB_WORD_BYTES : S::SA_WORD_BYTES;
+      // fp32 scales with one group per segment: the four scales of a stage are one 16-byte vector
+      const bool vec_scales = !sd.bf16 && sd.r == 1 && g.seg_words == 1;
+      int64_t gst = 0;
+      bool ok = true;
+      for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const int64_t rix = (is_b ? (tile % tiles_n) * TN : (tile / tiles_n) * TM) + p;
+        const bool in = rix < sd.rows;
+        const uint32_t* bptr = sd.bits + (in ? rix : 0) * sd.ld_w;
+        const int64_t srow = (in ? rix : 0) * sd.ld_s;
+        int in_seg = 0, in_g = 0;      // position of the next word to fetch inside its segment / group
+        int64_t grp = 0;
+        auto fetch = [&](int64_t st, uint4& w, float (&f)[WPS]) {
+          const int64_t kw = st * WPS;
+          w = make_uint4(0, 0, 0, 0);
+          if (in && kw < sd.ld_w) w = __ldg(reinterpret_cast<const uint4*>(bptr + kw));
+          if (vec_scales) {
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (in && kw < sd.ld_s) v = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(sd.scales) + srow + kw));
+            f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;    // entries past the last group are stored zeros
+          } else {
+            // first decide which scale every word needs (no loaded value is touched here) ...
+            int64_t idx[WPS];
 #pragma unroll
-        for (int q = 0; q < WPS; q++) {
-          const bool live = kw + q < g.n_words;
-          ia[q] = (a_in && live && ga < g.Ga) ? a_srow + ga : -1;
-          iw[q] = (b_in && live && gw < g.Gw) ? b_srow + gw : -1;
-          if (++in_seg == g.seg_words) {           // next word starts a new segment
-            in_seg = 0;
-            if (++in_ga == g.ra) { in_ga = 0; ga++; }
-            if (++in_gw == g.rw) { in_gw = 0; gw++; }
+            for (int q = 0; q < WPS; q++) {
+              idx[q] = (in && kw + q < g.n_words && grp < sd.G) ? srow + grp : -1;
+              if (++in_seg == g.seg_words) { in_seg = 0; if (++in_g == sd.r) { in_g = 0; grp++; } }
+            }
+            // ... then issue the loads back to back
+#pragma unroll
+            for (int q = 0; q < WPS; q++) { f[q] = 0.0f; if (idx[q] >= 0) f[q] = load_scale(sd.scales, sd.bf16, idx[q]); }
           }
-        }
-        // ... then issue the loads back to back (repeated indices hit the same cache line)
+        };
+        uint4 w, nw;
+        float f[WPS], nf[WPS];
+        fetch(0, w, f);
+        for (int64_t st = 0; st < n_stages; st++, gst++) {
+          if (st + 1 < n_stages) fetch(st + 1, nw, nf);     // in flight while this stage is expanded
+          const int s = static_cast<int>(gst % STAGES);
+          if (gst >= STAGES && !mbar_wait(&empty[s], static_cast<uint32_t>(((gst / STAGES) & 1) ^ 1), abort_flag, 1)) { ok = false; break; }
+          expand_words(sign_base + s * sign_stage, rows, p, w);
 #pragma unroll
-        for (int q = 0; q < WPS; q++) {
-          f.fa[q] = 0.0f; f.fb[q] = 0.0f;
-          if (ia[q] >= 0) f.fa[q] = load_scale(g.a_scales, g.a_bf16, ia[q]);
-          if (iw[q] >= 0) f.fb[q] = load_scale(g.w_scales, g.w_bf16, iw[q]);
-        }
-      };
-      Fetched cur, nxt;
-      fetch(0, cur);
-      for (int64_t st = 0; st < n_stages; st++, gst++) {
-        if (st + 1 < n_stages) fetch(st + 1, nxt);     // in flight while this stage is expanded
-        const int s = static_cast<int>(gst % STAGES);
-        if (gst >= STAGES && !mbar_wait(&empty[s], static_cast<uint32_t>(((gst / STAGES) & 1) ^ 1), abort_flag, 1)) { ok = false; break; }
-        expand_words(smem + S::OFF_A + s * S::A_STAGE, TM, p, cur.wa);
+          for (int q = 0; q < WPS; q++)
+            *reinterpret_cast<uint4*>(sc_row + (s * WPS + q) * sc_word) = is_b ? scale_row<true>(f[q]) : scale_row<false>(f[q]);
+          fence_async_proxy();          // make the generic-proxy stores visible to the tensor core
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&full[s]);
+          w = nw;
 #pragma unroll
-        for (int q = 0; q < WPS; q++) sA[(s * WPS + q) * TM + p] = cur.fa[q];
-        if (b_row) {
-          expand_words(smem + S::OFF_B + s * S::B_STAGE, TN, p, cur.wb);
-#pragma unroll
-          for (int q = 0; q < WPS; q++) sW[(s * WPS + q) * TN + p] = cur.fb[q];
+          for (int q = 0; q < WPS; q++) f[q] = nf[q];
         }
-        fence_async_proxy();          // make the generic-proxy stores visible to the tensor core
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&full[s]);
-        cur = nxt;
       }
     }
   } else if (warp == kMmaWarp) {
     // =========================== MMA issuer ===========================
     reg_dec<kRegsOther>();
     if (lane == 0) {
-      constexpr uint32_t idesc = instr_desc_f8(TN);
+      constexpr uint32_t idesc_sign = instr_desc(TN, kFmtE4M3), idesc_scale = instr_desc(TN, kFmtBF16);
+      const uint32_t zero_addr = smem_u32(smem + S::OFF_ZERO);
       int64_t gst = 0, gseg = 0;
       bool ok = true;
       for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
@@ -370,15 +370,20 @@ hbmm_umma_kernel(const Args g) {
             const int64_t kw = st * WPS + q;
             if (kw >= g.n_words) break;
             const int buf = static_cast<int>(gseg % NBUF);
+            const uint32_t d_tmem = tmem_base + buf * 2 * TN;
             if (in_seg == 0 && gseg >= NBUF) {
               if (!mbar_wait(&tempty[buf], static_cast<uint32_t>(((gseg / NBUF) & 1) ^ 1), abort_flag, 3)) { ok = false; break; }
               tc_fence_after();
             }
-            umma_f8(tmem_base + buf * TN,
-                    smem_desc(a_addr + q * S::A_WORD_BYTES, TM * 16, 128),
-                    smem_desc(b_addr + q * S::B_WORD_BYTES, TN * 16, 128), idesc, in_seg != 0 ? 1u : 0u);
+            umma_f8(d_tmem, smem_desc(a_addr + q * S::A_WORD_BYTES, TM * 16, 128),
+                    smem_desc(b_addr + q * S::B_WORD_BYTES, TN * 16, 128), idesc_sign, in_seg != 0 ? 1u : 0u);
             if (++in_seg == g.seg_words || kw == g.n_words - 1) {
-              umma_commit(&tfull[buf]);     // segment complete: hand the accumulator to the epilogue
+              // scale product of the segment: K columns 0..7 from this word slot, 8..15 from the zero block
+              const uint32_t sa_addr = smem_u32(smem + S::OFF_SA + (s * WPS + q) * S::SA_WORD_BYTES);
+              const uint32_t sb_addr = smem_u32(smem + S::OFF_SB + (s * WPS + q) * S::SB_WORD_BYTES);
+              umma_bf16_overwrite(d_tmem + TN, smem_desc(sa_addr, zero_addr - sa_addr, 128),
+                                  smem_desc(sb_addr, zero_addr - sb_addr, 128), idesc_scale);
+              umma_commit(&tfull[buf]);     // segment complete: hand D and S to the epilogue
               gseg++;
               in_seg = 0;
             }
@@ -396,9 +401,9 @@ hbmm_umma_kernel(const Args g) {
     const int wg = warp >> 2;                       // column half
     const int row = (warp & 3) * 32 + lane;         // TMEM lane = tile row
     const uint32_t t_lane = static_cast<uint32_t>((warp & 3) * 32) << 16;
-    int64_t gseg = 0, gst_base = 0, released = 0;   // released: stages handed back to the producers so far
+    int64_t gseg = 0;
     bool ok = true;
-    for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, gst_base += n_stages) {
+    for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
       uint64_t acc[HALF / 2];                       // two fp32 outputs per register pair
 #pragma unroll
       for (int j = 0; j < HALF / 2; j++) acc[j] = 0ull;
@@ -406,36 +411,21 @@ hbmm_umma_kernel(const Args g) {
         const int buf = static_cast<int>(gseg % NBUF);
         if (!mbar_wait(&tfull[buf], static_cast<uint32_t>((gseg / NBUF) & 1), abort_flag, 5)) { ok = false; break; }
         tc_fence_after();
-        int64_t kw_last = (seg + 1) * g.seg_words - 1;        // the word that carries this segment's scales
-        if (kw_last > g.n_words - 1) kw_last = g.n_words - 1;
-        const int64_t st = gst_base + kw_last / WPS;
-        const int s = static_cast<int>(st % STAGES), q = static_cast<int>(kw_last % WPS);
-        const float sa = sA[(s * WPS + q) * TM + row];
-        const uint64_t sa2 = pack2(sa, sa);
-        const float* swp = sW + (s * WPS + q) * TN + wg * HALF;
-        uint32_t d[HALF / 32][32];
+        const uint32_t t_d = tmem_base + t_lane + buf * 2 * TN + wg * HALF, t_s = t_d + TN;
+        uint32_t d[32], sc[32];
 #pragma unroll
-        for (int c = 0; c < HALF / 32; c++) tmem_ld32(tmem_base + t_lane + buf * TN + wg * HALF + c * 32, d[c]);
-        tmem_ld_wait();
-#pragma unroll
-        for (int c = 0; c < HALF / 32; c++)
-#pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            const float4 sw = *reinterpret_cast<const float4*>(swp + c * 32 + j);
-            const uint64_t t0 = mul2(sa2, pack2(__uint_as_float(d[c][j + 0]), __uint_as_float(d[c][j + 1])));
-            const uint64_t t1 = mul2(sa2, pack2(__uint_as_float(d[c][j + 2]), __uint_as_float(d[c][j + 3])));
-            acc[(c * 32 + j) / 2] = fma2(t0, pack2(sw.x, sw.y), acc[(c * 32 + j) / 2]);
-            acc[(c * 32 + j) / 2 + 1] = fma2(t1, pack2(sw.z, sw.w), acc[(c * 32 + j) / 2 + 1]);
+        for (int c = 0; c < CH; c++) {
+          tmem_ld32(t_d + c * 32, d);
+          tmem_ld32(t_s + c * 32, sc);
+          tmem_ld_wait();
+          if (c == CH - 1) {                        // everything of this buffer is in registers: release it
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tempty[buf]);
           }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) {
-          mbar_arrive(&tempty[buf]);
-          // release every stage whose words are now all consumed (their scales will not be read again)
-          int64_t done_words = (seg + 1) * g.seg_words;
-          if (done_words > g.n_words) done_words = g.n_words;
-          const int64_t consumed = gst_base + ((done_words == g.n_words) ? n_stages : done_words / WPS);
-          for (; released < consumed; released++) mbar_arrive(&empty[released % STAGES]);
+#pragma unroll
+          for (int j = 0; j < 32; j += 2)
+            acc[(c * 32 + j) / 2] = fma2(pack2(sc[j], sc[j + 1]), pack2(d[j], d[j + 1]), acc[(c * 32 + j) / 2]);
         }
       }
       if (ok) {
@@ -456,7 +446,7 @@ hbmm_umma_kernel(const Args g) {
       }
     }
   } else {
-    reg_dec<kRegsOther>();   // warps 13..15: nothing to do but hand their registers over
+    reg_dec<kRegsOther>();   // warps 17..19: nothing to do but hand their registers over
   }
 
   // ---- teardown: everyone meets here (aborted threads too), then the allocating warp frees TMEM
@@ -468,13 +458,13 @@ hbmm_umma_kernel(const Args g) {
   }
 }
 
-template <int TN, bool FAST>
+template <int TN>
 cudaError_t launch_umma(const Args& g, cudaStream_t stream) {
   using S = Smem<TN>;
   static bool configured = false;
   static int sms = 0;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(hbmm_umma_kernel<TN, FAST>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::BYTES);
+    cudaError_t e = cudaFuncSetAttribute(hbmm_umma_kernel<TN>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::BYTES);
     if (e != cudaSuccess) return e;
     int dev = 0;
     cudaGetDevice(&dev);
@@ -483,7 +473,7 @@ cudaError_t launch_umma(const Args& g, cudaStream_t stream) {
   }
   const int64_t tiles = ((g.M + TM - 1) / TM) * ((g.N + TN - 1) / TN);
   const unsigned grid = static_cast<unsigned>(tiles < sms ? tiles : sms);   // one persistent CTA per SM
-  hbmm_umma_kernel<TN, FAST><<<grid, kThreads, S::BYTES, stream>>>(g);
+  hbmm_umma_kernel<TN><<<grid, kThreads, S::BYTES, stream>>>(g);
   return cudaGetLastError();
 }
 
@@ -516,9 +506,7 @@ cudaError_t launch_gemm_tensor(const PackedView& A, const PackedView& W, float* 
   g.rw = static_cast<int32_t>(w_one ? T : W.beta / seg);
   g.Ga = num_groups(A.K, A.beta);
   g.Gw = num_groups(W.K, W.beta);
-  const bool fast = g.seg_words == 1 && g.ra == 1 && g.rw == 1 && !g.a_bf16 && !g.w_bf16;
-  if (fast) return g.N <= 64 ? launch_umma<64, true>(g, stream) : launch_umma<128, true>(g, stream);
-  return g.N <= 64 ? launch_umma<64, false>(g, stream) : launch_umma<128, false>(g, stream);
+  return g.N <= 64 ? launch_umma<64>(g, stream) : launch_umma<128>(g, stream);
 }
 
 cudaError_t read_umma_error(int* code) {
