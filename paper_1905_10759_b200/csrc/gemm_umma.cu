@@ -41,8 +41,9 @@ constexpr int kProducerWarps = 8;                         // warpgroup 2 (A rows
 constexpr int kFirstProducerWarp = kEpilogueWarps;        // warps 8..15
 constexpr int kMmaWarp = kEpilogueWarps + kProducerWarps; // warp 16
 constexpr int kThreads = 20 * 32;                         // 640: five warpgroups
-constexpr int kRegsEpilogue = 144;                        // 256 x 144 + 384 x 64 = 61440 = 640 x 96, the CTA's register allocation at launch
-constexpr int kRegsOther = 64;
+constexpr int kRegsEpilogue = 144;                        // epilogue warps; the CTA's register allocation at launch is 640 x 96
+constexpr int kRegsProducer = 72;                         // 256 x 144 + 256 x 72 + 128 x 48 = 61440 = 640 x 96
+constexpr int kRegsIssuer = 48;
 constexpr int TM = 128;
 constexpr int WPS = 4;            // K-words per stage
 constexpr int STAGES = 4;
@@ -111,14 +112,11 @@ __device__ __forceinline__ void umma_f8(uint32_t d_tmem, uint64_t a_desc, uint64
       "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
-__device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t (&v)[32]) {
+__device__ __forceinline__ void tmem_ld16(uint32_t addr, uint32_t (&v)[16]) {
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
       : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
       : "r"(addr));
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
@@ -196,6 +194,11 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint3
   d |= static_cast<uint64_t>(1) << 46;
   return d;
 }
+// Same descriptor for a start address `delta`*16 bytes further on: only the low word changes (address
+// field up; for the scale operands `delta` also carries the matching decrease of the lbo field).
+__device__ __forceinline__ uint64_t desc_step(uint64_t d, uint32_t delta) {
+  return (d & 0xFFFFFFFF00000000ull) | static_cast<uint32_t>(static_cast<uint32_t>(d) + delta);
+}
 // Instruction descriptors: fp32 accumulator, both operands K-major, M = 128, N = n.
 __host__ __device__ constexpr uint32_t instr_desc(int n, uint32_t ab_format) {
   return (1u << 4) | (ab_format << 7) | (ab_format << 10) | (static_cast<uint32_t>(n >> 3) << 17) |
@@ -239,7 +242,6 @@ hbmm_umma_kernel(const Args g) {
   using S = Smem<TN>;
   constexpr int NBUF = S::NBUF;
   constexpr int HALF = TN / 2;                  // columns per epilogue warpgroup
-  constexpr int CH = HALF / 32;                 // 32-column chunks per epilogue warp
   extern __shared__ __align__(1024) unsigned char smem[];
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + S::OFF_BAR);
   uint64_t* empty = full + STAGES;
@@ -286,7 +288,7 @@ hbmm_umma_kernel(const Args g) {
   // accumulator rings simply continue across tiles (gst / gseg count stages / segments since launch).
   if (warp >= kFirstProducerWarp && warp < kMmaWarp) {
     // =========================== producers ===========================
-    reg_dec<kRegsOther>();
+    reg_dec<kRegsProducer>();
     const bool is_b = warp >= kFirstProducerWarp + 4;
     const int p = (tid - kFirstProducerWarp * 32) & 127;    // tile row of this thread's operand
     const int rows = is_b ? TN : TM;
@@ -352,43 +354,49 @@ hbmm_umma_kernel(const Args g) {
     }
   } else if (warp == kMmaWarp) {
     // =========================== MMA issuer ===========================
-    reg_dec<kRegsOther>();
+    reg_dec<kRegsIssuer>();
     if (lane == 0) {
       constexpr uint32_t idesc_sign = instr_desc(TN, kFmtE4M3), idesc_scale = instr_desc(TN, kFmtBF16);
+      // Descriptors of stage 0 / word 0; every other slot differs only by its start address (and, for
+      // the scale operands, by the distance to the zero block), so they are stepped with 32-bit adds
+      // of the low word: +bytes/16 in the address field, -bytes/16 in the lbo field (bits 16..29).
       const uint32_t zero_addr = smem_u32(smem + S::OFF_ZERO);
-      int64_t gst = 0, gseg = 0;
+      const uint32_t sa0 = smem_u32(smem + S::OFF_SA), sb0 = smem_u32(smem + S::OFF_SB);
+      const uint64_t da0 = smem_desc(smem_u32(smem + S::OFF_A), TM * 16, 128);
+      const uint64_t db0 = smem_desc(smem_u32(smem + S::OFF_B), TN * 16, 128);
+      const uint64_t dsa0 = smem_desc(sa0, zero_addr - sa0, 128), dsb0 = smem_desc(sb0, zero_addr - sb0, 128);
+      constexpr uint32_t kStepA = S::A_WORD_BYTES >> 4, kStepB = S::B_WORD_BYTES >> 4;
+      constexpr uint32_t kSa = S::SA_WORD_BYTES >> 4, kSb = S::SB_WORD_BYTES >> 4;
+      constexpr uint32_t kStepSA = kSa - (kSa << 16), kStepSB = kSb - (kSb << 16);   // modulo 2^32 on purpose
+      const uint32_t n_words = static_cast<uint32_t>(g.n_words), seg_words = static_cast<uint32_t>(g.seg_words);
+      uint32_t s = 0, full_par = 0;          // stage slot and the parity its "full" barrier completes with next
+      uint32_t buf = 0, tempty_par = 0;      // accumulator buffer; the first pass over the ring needs no wait
+      bool first_ring = true;
       bool ok = true;
       for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-        int64_t in_seg = 0;
-        for (int64_t st = 0; st < n_stages && ok; st++, gst++) {
-          const int s = static_cast<int>(gst % STAGES);
-          if (!mbar_wait(&full[s], static_cast<uint32_t>((gst / STAGES) & 1), abort_flag, 2)) { ok = false; break; }
+        uint32_t in_seg = 0;
+        for (uint32_t kw0 = 0; kw0 < n_words && ok; kw0 += WPS) {
+          if (!mbar_wait(&full[s], full_par, abort_flag, 2)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t a_addr = smem_u32(smem + S::OFF_A + s * S::A_STAGE);
-          const uint32_t b_addr = smem_u32(smem + S::OFF_B + s * S::B_STAGE);
-          for (int q = 0; q < WPS; q++) {
-            const int64_t kw = st * WPS + q;
-            if (kw >= g.n_words) break;
-            const int buf = static_cast<int>(gseg % NBUF);
+          const uint32_t slot = s * WPS;
+          const uint32_t nq = n_words - kw0 < WPS ? n_words - kw0 : WPS;
+          for (uint32_t q = 0; q < nq; q++) {
             const uint32_t d_tmem = tmem_base + buf * 2 * TN;
-            if (in_seg == 0 && gseg >= NBUF) {
-              if (!mbar_wait(&tempty[buf], static_cast<uint32_t>(((gseg / NBUF) & 1) ^ 1), abort_flag, 3)) { ok = false; break; }
+            if (in_seg == 0 && !first_ring) {
+              if (!mbar_wait(&tempty[buf], tempty_par, abort_flag, 3)) { ok = false; break; }
               tc_fence_after();
             }
-            umma_f8(d_tmem, smem_desc(a_addr + q * S::A_WORD_BYTES, TM * 16, 128),
-                    smem_desc(b_addr + q * S::B_WORD_BYTES, TN * 16, 128), idesc_sign, in_seg != 0 ? 1u : 0u);
-            if (++in_seg == g.seg_words || kw == g.n_words - 1) {
+            umma_f8(d_tmem, desc_step(da0, (slot + q) * kStepA), desc_step(db0, (slot + q) * kStepB), idesc_sign, in_seg);
+            if (++in_seg == seg_words || kw0 + q == n_words - 1) {
               // scale product of the segment: K columns 0..7 from this word slot, 8..15 from the zero block
-              const uint32_t sa_addr = smem_u32(smem + S::OFF_SA + (s * WPS + q) * S::SA_WORD_BYTES);
-              const uint32_t sb_addr = smem_u32(smem + S::OFF_SB + (s * WPS + q) * S::SB_WORD_BYTES);
-              umma_bf16_overwrite(d_tmem + TN, smem_desc(sa_addr, zero_addr - sa_addr, 128),
-                                  smem_desc(sb_addr, zero_addr - sb_addr, 128), idesc_scale);
+              umma_bf16_overwrite(d_tmem + TN, desc_step(dsa0, (slot + q) * kStepSA), desc_step(dsb0, (slot + q) * kStepSB), idesc_scale);
               umma_commit(&tfull[buf]);     // segment complete: hand D and S to the epilogue
-              gseg++;
               in_seg = 0;
+              if (++buf == NBUF) { buf = 0; if (first_ring) first_ring = false; else tempty_par ^= 1; }
             }
           }
           umma_commit(&empty[s]);           // stage's bytes are free once these MMAs have read them
+          if (++s == STAGES) { s = 0; full_par ^= 1; }
         }
       }
       umma_commit(drain);
@@ -412,20 +420,27 @@ hbmm_umma_kernel(const Args g) {
         if (!mbar_wait(&tfull[buf], static_cast<uint32_t>((gseg / NBUF) & 1), abort_flag, 5)) { ok = false; break; }
         tc_fence_after();
         const uint32_t t_d = tmem_base + t_lane + buf * 2 * TN + wg * HALF, t_s = t_d + TN;
-        uint32_t d[32], sc[32];
+        // 16-column pieces, double buffered: the loads of piece c+1 are in flight during the math of c
+        constexpr int PIECES = HALF / 16;
+        uint32_t d[2][16], sc[2][16];
+        tmem_ld16(t_d, d[0]);
+        tmem_ld16(t_s, sc[0]);
+        tmem_ld_wait();
 #pragma unroll
-        for (int c = 0; c < CH; c++) {
-          tmem_ld32(t_d + c * 32, d);
-          tmem_ld32(t_s + c * 32, sc);
-          tmem_ld_wait();
-          if (c == CH - 1) {                        // everything of this buffer is in registers: release it
+        for (int c = 0; c < PIECES; c++) {
+          if (c + 1 < PIECES) {
+            tmem_ld16(t_d + (c + 1) * 16, d[(c + 1) & 1]);
+            tmem_ld16(t_s + (c + 1) * 16, sc[(c + 1) & 1]);
+          }
+#pragma unroll
+          for (int j = 0; j < 16; j += 2)
+            acc[(c * 16 + j) / 2] = fma2(pack2(sc[c & 1][j], sc[c & 1][j + 1]), pack2(d[c & 1][j], d[c & 1][j + 1]), acc[(c * 16 + j) / 2]);
+          if (c + 1 < PIECES) tmem_ld_wait();
+          if (c == PIECES - 2) {                    // the last loads have landed: the buffer can be refilled
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&tempty[buf]);
           }
-#pragma unroll
-          for (int j = 0; j < 32; j += 2)
-            acc[(c * 32 + j) / 2] = fma2(pack2(sc[j], sc[j + 1]), pack2(d[j], d[j + 1]), acc[(c * 32 + j) / 2]);
         }
       }
       if (ok) {
@@ -446,7 +461,7 @@ hbmm_umma_kernel(const Args g) {
       }
     }
   } else {
-    reg_dec<kRegsOther>();   // warps 17..19: nothing to do but hand their registers over
+    reg_dec<kRegsIssuer>();   // warps 17..19: nothing to do but hand their registers over
   }
 
   // ---- teardown: everyone meets here (aborted threads too), then the allocating warp frees TMEM
