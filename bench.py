@@ -206,7 +206,8 @@ def kernel_breakdown(torch, hbmm, layers, iters: int):
         bits = L["ws"][: s.M * lw * 4].view(torch.int32).reshape(s.M, lw)
         scales = L["ws"][bits_bytes: bits_bytes + s.M * ls * 4].view(torch.float32).reshape(s.M, ls)
         A = hbmm.wrap_packed(bits, scales, s.K, BETA)
-        t_gemm = time_loop(torch, lambda: hbmm.gemm(A, L["W"], L["C"]), iters)
+        gws = torch.empty(max(hbmm.gemm_workspace_bytes(A, L["W"]), 16), dtype=torch.uint8, device=L["C"].device)
+        t_gemm = time_loop(torch, lambda: hbmm.gemm(A, L["W"], L["C"], gws), iters)
         out["hbmm_contraction"].append(t_gemm)
         out["front_end_pack"].append(max(t_conv - t_gemm, 0.0))
         t_convb = time_loop(torch, lambda: hbmm.conv_im2col(L["xb"], L["geom"], 1, hbmm.F32, L["W"], L["Cb"], L["ws"]), iters)

@@ -116,8 +116,11 @@ hbmm_status hbmm_operand_bytes(int64_t rows, int64_t K, int32_t beta, int32_t sc
 hbmm_status hbmm_quantize(const void *x, int32_t x_dtype, int64_t rows, int64_t K, int64_t ldx,
                           const hbmm_operand *out, void *stream);
 
-/* Bytes of scratch hbmm_gemm needs for these operands (currently 0 for every path; the query
- * exists so callers stay correct if a path grows a workspace).  bytes: host pointer. */
+/* Bytes of scratch hbmm_gemm wants for these operands (host pointer `bytes`).  The tensor-core
+ * contraction keeps the weight operand there, expanded once per call into the tile layout its
+ * kernel streams (about K bytes + K/2 bytes per weight row); 0 when no path needs scratch.
+ * hbmm_gemm still works without it (workspace NULL or too small): it then runs the
+ * integer-pipe path.  The workspace must be 16-byte aligned. */
 hbmm_status hbmm_gemm_workspace_bytes(const hbmm_operand *A, const hbmm_operand *W, size_t *bytes);
 
 /*
@@ -135,7 +138,8 @@ hbmm_status hbmm_gemm(const hbmm_operand *A, const hbmm_operand *W, float *C, in
                       void *workspace, size_t workspace_bytes, void *stream);
 
 /* Same as hbmm_gemm with the contraction kernel chosen by the caller (hbmm_path); a path that
- * cannot run these operands returns HBMM_ERR_UNSUPPORTED.  For measurement and tests. */
+ * cannot run these operands returns HBMM_ERR_UNSUPPORTED, HBMM_PATH_TENSOR without its workspace
+ * HBMM_ERR_WORKSPACE.  For measurement and tests. */
 hbmm_status hbmm_gemm_ex(const hbmm_operand *A, const hbmm_operand *W, float *C, int64_t ldc,
                          void *workspace, size_t workspace_bytes, int32_t path, void *stream);
 
@@ -148,8 +152,8 @@ hbmm_status hbmm_gemm_ex(const hbmm_operand *A, const hbmm_operand *W, float *C,
 hbmm_status hbmm_gemm_partials(const hbmm_operand *A, const hbmm_operand *W, int32_t *D,
                                int32_t path, void *stream);
 
-/* Scratch for hbmm_conv_im2col: the packed (or, for beta_a == 1, bf16 dense) im2col operand.
- * bytes: host pointer. */
+/* Scratch for hbmm_conv_im2col: the packed (or, for beta_a == 1, bf16 dense) im2col operand
+ * followed by the contraction's own workspace.  bytes: host pointer. */
 hbmm_status hbmm_conv_workspace_bytes(const hbmm_conv_geom *g, int32_t beta_a, int32_t a_scale_dtype,
                                       const hbmm_operand *W, size_t *bytes);
 
@@ -200,7 +204,7 @@ hbmm_status hbmm_conv_im2col_static(const void *x, int32_t x_dtype, const hbmm_c
 /*
  * Device-side health word of the tensor-core contraction.  Its kernels never spin without a
  * limit: a wait on a barrier that does not complete in time records a code (1 producer, 2/3/4
- * MMA issue, 5 epilogue), makes the kernel drain and return, and leaves the output undefined.
+ * MMA issue, 5 epilogue, 6 weight loader), makes the kernel drain and return, and leaves the output undefined.
  * This call copies the word back (it synchronises the device) and returns HBMM_ERR_TIMEOUT when
  * it is non-zero, HBMM_OK otherwise.  code: host pointer, may be NULL.
  */

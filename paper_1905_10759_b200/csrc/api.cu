@@ -60,8 +60,17 @@ hbmm_status check_c(const float* C, int64_t ldc, int64_t N) {
   return HBMM_OK;
 }
 
+// Workspace of the tensor-core contraction for these (validated, packed) operands, 0 when that path
+// cannot run them.
+size_t tensor_workspace(const PackedView& a, const PackedView& w) {
+  return gemm_tensor_supported(a, w) ? static_cast<size_t>(round_up(static_cast<int64_t>(gemm_tensor_workspace_bytes(a, w)), 256)) : 0;
+}
+inline bool workspace_ok(const void* ws, size_t have, size_t need) {
+  return need == 0 || (ws != nullptr && have >= need && (reinterpret_cast<uintptr_t>(ws) & 15u) == 0);
+}
+
 hbmm_status gemm_checked(const hbmm_operand* A, const hbmm_operand* W, float* C, int64_t ldc,
-                         int32_t path, cudaStream_t stream) {
+                         int32_t path, void* workspace, size_t workspace_bytes, cudaStream_t stream) {
   if (!A || !W) return HBMM_ERR_INVALID_ARG;
   if (W->beta == 1) return HBMM_ERR_UNSUPPORTED;  // the weight operand is always Hadamard-binary
   hbmm_status st = check_packed(W);
@@ -92,11 +101,15 @@ hbmm_status gemm_checked(const hbmm_operand* A, const hbmm_operand* W, float* C,
       break;
     case HBMM_PATH_TENSOR:
       if (!gemm_tensor_supported(a, w)) return HBMM_ERR_UNSUPPORTED;
-      e = launch_gemm_tensor(a, w, C, ldc, stream);
+      if (!workspace_ok(workspace, workspace_bytes, tensor_workspace(a, w))) return HBMM_ERR_WORKSPACE;
+      e = launch_gemm_tensor(a, w, C, ldc, workspace, stream);
       break;
     default:
-      if (gemm_tensor_supported(a, w)) e = launch_gemm_tensor(a, w, C, ldc, stream);
-      else e = launch_gemm_popc(a, w, C, ldc, stream);
+      // the tensor-core path needs its workspace; without one the integer-pipe path runs
+      if (gemm_tensor_supported(a, w) && workspace_ok(workspace, workspace_bytes, tensor_workspace(a, w)))
+        e = launch_gemm_tensor(a, w, C, ldc, workspace, stream);
+      else
+        e = launch_gemm_popc(a, w, C, ldc, stream);
       break;
   }
   return e == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
@@ -119,22 +132,31 @@ hbmm_status check_geom(const hbmm_conv_geom* g, ConvGeom* out) {
 
 struct ConvLayout {
   int64_t M, K, ld_words, ld_scales, ld_dense;
-  size_t bits_bytes, scales_bytes, total;
+  size_t bits_bytes, scales_bytes, operand_bytes, gemm_bytes, total;
 };
 
-ConvLayout conv_layout(const ConvGeom& g, int32_t beta_a, int32_t scale_dtype) {
+ConvLayout conv_layout(const ConvGeom& g, int32_t beta_a, int32_t scale_dtype, const hbmm_operand* W) {
   ConvLayout L{};
   L.M = static_cast<int64_t>(g.B) * g.Ho * g.Wo;
   L.K = static_cast<int64_t>(g.C) * g.kh * g.kw;
   if (beta_a == 1) {
     L.ld_dense = round_up(L.K, 8);
-    L.total = static_cast<size_t>(L.M) * L.ld_dense * 2;
+    L.operand_bytes = static_cast<size_t>(round_up(L.M * L.ld_dense * 2, 256));
+    L.total = L.operand_bytes;
   } else {
     L.ld_words = words_ld(L.K);
     L.ld_scales = scales_ld(L.K, beta_a, scale_dtype);
     L.bits_bytes = static_cast<size_t>(round_up(L.M * L.ld_words * 4, 256));
     L.scales_bytes = static_cast<size_t>(round_up(L.M * L.ld_scales * (scale_dtype == HBMM_BF16 ? 2 : 4), 256));
-    L.total = L.bits_bytes + L.scales_bytes;
+    L.operand_bytes = L.bits_bytes + L.scales_bytes;
+    // the contraction's own workspace follows the packed activation operand
+    PackedView a;
+    a.bits = nullptr; a.scales = nullptr; a.rows = L.M; a.K = L.K; a.ld_words = L.ld_words; a.ld_scales = L.ld_scales;
+    a.beta = beta_a; a.scale_bf16 = scale_dtype == HBMM_BF16;
+    hbmm_operand Aop{};
+    Aop.rows = L.M; Aop.K = L.K; Aop.beta = beta_a;
+    L.gemm_bytes = (W && W->K == L.K && segments_compatible(&Aop, W)) ? tensor_workspace(a, view_of(W)) : 0;
+    L.total = L.operand_bytes + L.gemm_bytes;
   }
   return L;
 }
@@ -171,19 +193,20 @@ hbmm_status hbmm_quantize(const void* x, int32_t x_dtype, int64_t rows, int64_t 
 hbmm_status hbmm_gemm_workspace_bytes(const hbmm_operand* A, const hbmm_operand* W, size_t* bytes) {
   if (!A || !W || !bytes) return HBMM_ERR_INVALID_ARG;
   *bytes = 0;
+  if (A->beta >= 2 && W->beta >= 2 && check_packed(A, false) == HBMM_OK && check_packed(W, false) == HBMM_OK &&
+      A->K == W->K && segments_compatible(A, W))
+    *bytes = tensor_workspace(view_of(A), view_of(W));
   return HBMM_OK;
 }
 
 hbmm_status hbmm_gemm(const hbmm_operand* A, const hbmm_operand* W, float* C, int64_t ldc, void* workspace,
                       size_t workspace_bytes, void* stream) {
-  (void)workspace; (void)workspace_bytes;
-  return gemm_checked(A, W, C, ldc, HBMM_PATH_AUTO, static_cast<cudaStream_t>(stream));
+  return gemm_checked(A, W, C, ldc, HBMM_PATH_AUTO, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
 }
 
 hbmm_status hbmm_gemm_ex(const hbmm_operand* A, const hbmm_operand* W, float* C, int64_t ldc, void* workspace,
                          size_t workspace_bytes, int32_t path, void* stream) {
-  (void)workspace; (void)workspace_bytes;
-  return gemm_checked(A, W, C, ldc, path, static_cast<cudaStream_t>(stream));
+  return gemm_checked(A, W, C, ldc, path, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
 }
 
 hbmm_status hbmm_gemm_partials(const hbmm_operand* A, const hbmm_operand* W, int32_t* D, int32_t path, void* stream) {
@@ -213,7 +236,8 @@ hbmm_status hbmm_conv_workspace_bytes(const hbmm_conv_geom* g, int32_t beta_a, i
   if (!bytes || !W || beta_a < 1 || !valid_dtype(a_scale_dtype)) return HBMM_ERR_INVALID_ARG;
   const int64_t K = static_cast<int64_t>(cg.C) * cg.kh * cg.kw;
   if (beta_a >= 2 && !beta_supported(K, beta_a)) return HBMM_ERR_UNSUPPORTED;
-  *bytes = conv_layout(cg, beta_a, a_scale_dtype).total;
+  if (check_packed(W, false) != HBMM_OK) return check_packed(W, false);
+  *bytes = conv_layout(cg, beta_a, a_scale_dtype, W).total;
   return HBMM_OK;
 }
 
@@ -225,7 +249,7 @@ hbmm_status hbmm_conv_im2col(const void* x, int32_t x_dtype, const hbmm_conv_geo
   if (st != HBMM_OK) return st;
   if (!x || !W || beta_a < 1 || !valid_dtype(x_dtype) || !valid_dtype(a_scale_dtype)) return HBMM_ERR_INVALID_ARG;
   if ((st = check_packed(W)) != HBMM_OK) return st;
-  const ConvLayout L = conv_layout(cg, beta_a, a_scale_dtype);
+  const ConvLayout L = conv_layout(cg, beta_a, a_scale_dtype, W);
   if (W->K != L.K) return HBMM_ERR_INVALID_ARG;
   if (beta_a >= 2 && !beta_supported(L.K, beta_a)) return HBMM_ERR_UNSUPPORTED;
   if ((st = check_c(C_out, ldc, W->rows)) != HBMM_OK) return st;
@@ -247,7 +271,7 @@ hbmm_status hbmm_conv_im2col(const void* x, int32_t x_dtype, const hbmm_conv_geo
                                a_scale_dtype == HBMM_BF16, s) != cudaSuccess)
       return HBMM_ERR_CUDA;
   }
-  return gemm_checked(&A, W, C_out, ldc, HBMM_PATH_AUTO, s);
+  return gemm_checked(&A, W, C_out, ldc, HBMM_PATH_AUTO, static_cast<char*>(workspace) + L.operand_bytes, L.gemm_bytes, s);
 }
 
 hbmm_status hbmm_last_device_error(int32_t* code) {

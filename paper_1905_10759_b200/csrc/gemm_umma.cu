@@ -20,9 +20,12 @@
 // walks the tiles of the output.
 //   warps 0-7   : epilogue (warp w reads TMEM lanes 32*(w%4).., warps 0-3 the left half of the
 //                 columns, warps 4-7 the right half); they take most of the register file
-//   warps 8-11  : A producers, warps 12-15 : B producers: packed words -> e4m3 bytes and scales ->
-//                 bf16 pieces, both in the UMMA K-major core-matrix layout (8 rows x 16 bytes contiguous)
-//   warp  16    : TMEM allocation and the single MMA-issuing thread (warps 17-19 only hand registers over)
+//   warps 8-11  : A producers: packed words -> e4m3 bytes and scales -> bf16 pieces, both in the UMMA
+//                 K-major core-matrix layout (8 rows x 16 bytes contiguous)
+//   warp  12    : TMEM allocation and the single MMA-issuing thread
+//   warp  13    : one thread streams the W operand: a small kernel has expanded W once per call into
+//                 the same stage layout in the workspace, so a stage of W is one contiguous bulk copy
+//                 (cp.async.bulk, completion counted on the stage's mbarrier) instead of per-tile work
 // A stage holds four K-words; stages and TMEM accumulator buffers are rings guarded by
 // mbarriers.  Every wait is bounded: when a limit expires the thread records an error code in
 // global memory, raises a CTA-wide abort flag that all other waits observe, and the kernel
@@ -37,16 +40,17 @@ __device__ int g_umma_error = 0;  // 0 = ok; otherwise the code of the first wai
 namespace {
 
 constexpr int kEpilogueWarps = 8;                         // warpgroups 0 and 1
-constexpr int kProducerWarps = 8;                         // warpgroup 2 (A rows) and warpgroup 3 (B rows)
-constexpr int kFirstProducerWarp = kEpilogueWarps;        // warps 8..15
-constexpr int kMmaWarp = kEpilogueWarps + kProducerWarps; // warp 16
-constexpr int kThreads = 20 * 32;                         // 640: five warpgroups
-constexpr int kRegsEpilogue = 144;                        // epilogue warps; the CTA's register allocation at launch is 640 x 96
-constexpr int kRegsProducer = 72;                         // 256 x 144 + 256 x 72 + 128 x 48 = 61440 = 640 x 96
-constexpr int kRegsIssuer = 48;
+constexpr int kProducerWarps = 4;                         // warpgroup 2: one A row per thread
+constexpr int kFirstProducerWarp = kEpilogueWarps;        // warps 8..11
+constexpr int kMmaWarp = kEpilogueWarps + kProducerWarps; // warp 12: TMEM allocation, MMA issue
+constexpr int kLoaderWarp = kMmaWarp + 1;                 // warp 13: bulk copies of the prepared W stages
+constexpr int kThreads = 16 * 32;                         // 512: four warpgroups (warps 14, 15 only hand registers over)
+constexpr int kRegsEpilogue = 208;                        // 256 x 208 + 128 x 64 + 128 x 32 = 64 K registers
+constexpr int kRegsProducer = 64;
+constexpr int kRegsIssuer = 32;
 constexpr int TM = 128;
 constexpr int WPS = 4;            // K-words per stage
-constexpr int STAGES = 4;
+constexpr int STAGES = 3;
 constexpr uint32_t kSpinLimit = 1u << 20;   // polls of a (hardware time-limited) try_wait
 
 struct Args {
@@ -59,6 +63,7 @@ struct Args {
   int64_t Ga, Gw;
   int64_t n_words;         // K / 32 (K is a multiple of 32 on this path)
   int64_t seg_words;       // K-words per segment
+  const unsigned char* w_prep;   // W expanded by prepare_w: [n tile][stage][Smem::B_STAGE bytes]
 };
 
 __device__ __forceinline__ float load_scale(const void* s, int bf16, int64_t idx) {
@@ -80,6 +85,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
                : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
+// The same on a precomputed shared-memory address (keeps the single-thread issue loops short).
+__device__ __forceinline__ bool mbar_try_wait_a(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void umma_commit_a(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
 // Bounded wait.  Returns false when the limit expired or another thread aborted.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int code) {
   for (uint32_t it = 0; it < kSpinLimit; it++) {
@@ -91,7 +106,27 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   return false;
 }
 
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("{\n\t.reg .b64 st;\n\tmbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n\t}" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// Asynchronous bulk copy global -> this CTA's shared memory (both 16-byte aligned, size a multiple of
+// 16); completion is counted in bytes on the mbarrier.  No multicast.
+__device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
 // ---- tcgen05 helpers
+__device__ __forceinline__ bool mbar_wait_a(uint32_t bar, uint32_t parity, volatile int* abort_flag, int code) {
+  if (mbar_try_wait_a(bar, parity)) return true;
+  for (uint32_t it = 0; it < kSpinLimit; it++) {
+    if (mbar_try_wait_a(bar, parity)) return true;
+    if (*abort_flag) return false;
+  }
+  atomicCAS(&g_umma_error, 0, code);
+  *abort_flag = 1;
+  return false;
+}
 __device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t cols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols));
 }
@@ -112,6 +147,16 @@ __device__ __forceinline__ void umma_f8(uint32_t d_tmem, uint64_t a_desc, uint64
       "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
+__device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(addr));
+}
 __device__ __forceinline__ void tmem_ld16(uint32_t addr, uint32_t (&v)[16]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
@@ -119,6 +164,8 @@ __device__ __forceinline__ void tmem_ld16(uint32_t addr, uint32_t (&v)[16]) {
         "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
       : "r"(addr));
 }
+__device__ __forceinline__ void tmem_ld_piece(uint32_t addr, uint32_t (&v)[32]) { tmem_ld32(addr, v); }
+__device__ __forceinline__ void tmem_ld_piece(uint32_t addr, uint32_t (&v)[16]) { tmem_ld16(addr, v); }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 template <int R> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(R)); }
 template <int R> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(R)); }
@@ -150,16 +197,21 @@ __device__ __forceinline__ void umma_bf16_overwrite(uint32_t d_tmem, uint64_t a_
 __device__ __forceinline__ uint32_t signs_lo(uint32_t v) { return (((v & 0x0Fu) * 0x10204080u) & 0x80808080u) ^ 0xB8B8B8B8u; }
 __device__ __forceinline__ uint32_t signs_hi(uint32_t v) { return (((v & 0xF0u) * 0x01020408u) & 0x80808080u) ^ 0xB8B8B8B8u; }
 
-// Four packed K-words of one tile row -> 4 x 32 e4m3 bytes in the UMMA core-matrix layout of a stage:
-// [word][K-half (16 bytes)][row / 8][row % 8][16 bytes].
-__device__ __forceinline__ void expand_words(unsigned char* stage_base, int rows, int row, const uint4& w4) {
+// Operand tiles in shared memory use the 128-byte-swizzled K-major layout of the tensor core: a row is
+// 128 contiguous bytes (the four K-words of a stage, 32 bytes each), rows follow each other, and the
+// 16-byte piece c of row r is stored at piece position c ^ (r % 8).  A tile starts on a 1024-byte
+// boundary; the instruction for word slot q reads from byte offset 32*q of the rows.
+__device__ __forceinline__ unsigned char* swz(unsigned char* tile, int row, int piece) {
+  return tile + row * 128 + ((piece ^ (row & 7)) << 4);
+}
+// Four packed K-words of one tile row -> 4 x 32 e4m3 bytes (pieces 0..7 of the row).
+__device__ __forceinline__ void expand_words(unsigned char* tile, int row, const uint4& w4) {
   const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
 #pragma unroll
   for (int q = 0; q < 4; q++) {
-    unsigned char* base = stage_base + q * rows * 32 + (row >> 3) * 128 + (row & 7) * 16;
     const uint32_t y0 = w[q] & 0xFF, y1 = (w[q] >> 8) & 0xFF, y2 = (w[q] >> 16) & 0xFF, y3 = w[q] >> 24;
-    *reinterpret_cast<uint4*>(base) = make_uint4(signs_lo(y0), signs_hi(y0), signs_lo(y1), signs_hi(y1));              // K bytes 0..15
-    *reinterpret_cast<uint4*>(base + rows * 16) = make_uint4(signs_lo(y2), signs_hi(y2), signs_lo(y3), signs_hi(y3));  // K bytes 16..31
+    *reinterpret_cast<uint4*>(swz(tile, row, 2 * q)) = make_uint4(signs_lo(y0), signs_hi(y0), signs_lo(y1), signs_hi(y1));      // K bytes 0..15
+    *reinterpret_cast<uint4*>(swz(tile, row, 2 * q + 1)) = make_uint4(signs_lo(y2), signs_hi(y2), signs_lo(y3), signs_hi(y3));  // K bytes 16..31
   }
 }
 
@@ -172,8 +224,8 @@ __device__ __forceinline__ void split3(float a, uint32_t& h1, uint32_t& h2, uint
   const __nv_bfloat16 b3 = __float2bfloat16_rn(r2);
   h1 = __bfloat16_as_ushort(b1); h2 = __bfloat16_as_ushort(b2); h3 = __bfloat16_as_ushort(b3);
 }
-// One row of the scale operands of a segment: eight bf16 (K columns 0..7; columns 8..15 read a shared
-// block of zeros).  Row of A': (a1, a1, a2, a2, a1, a3, 0, 0); row of B': (w1, w2, w1, w2, w3, w1, 0, 0):
+// One row of the scale operands of a segment: eight bf16 (K columns 0..7; columns 8..15 are a piece of
+// zeros next to it).  Row of A': (a1, a1, a2, a2, a1, a3, 0, 0); row of B': (w1, w2, w1, w2, w3, w1, 0, 0):
 // their dot product is a1w1 + a1w2 + a2w1 + a2w2 + a1w3 + a3w1.
 template <bool IS_B>
 __device__ __forceinline__ uint4 scale_row(float v) {
@@ -183,21 +235,17 @@ __device__ __forceinline__ uint4 scale_row(float v) {
   return make_uint4(h1 | (h1 << 16), h2 | (h2 << 16), h1 | (h3 << 16), 0u);
 }
 
-// K-major operand without swizzle: core matrices of 8 rows x 16 bytes stored contiguously
-// (128 bytes); `sbo` = byte distance between 8-row groups, `lbo` = byte distance between the two
-// 16-byte K-chunks of one instruction.  Descriptor version 1, layout type 0.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+// Shared-memory descriptor of a K-major, 128-byte-swizzled operand: start address, stride between
+// 8-row groups = 1024 bytes, descriptor version 1, layout type 2 (128-byte swizzle); the leading
+// offset is not used by this layout.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
   uint64_t d = 0;
   d |= static_cast<uint64_t>((addr >> 4) & 0x3FFF);
-  d |= static_cast<uint64_t>((lbo >> 4) & 0x3FFF) << 16;
-  d |= static_cast<uint64_t>((sbo >> 4) & 0x3FFF) << 32;
+  d |= static_cast<uint64_t>(1) << 16;
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;
   d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
   return d;
-}
-// Same descriptor for a start address `delta`*16 bytes further on: only the low word changes (address
-// field up; for the scale operands `delta` also carries the matching decrease of the lbo field).
-__device__ __forceinline__ uint64_t desc_step(uint64_t d, uint32_t delta) {
-  return (d & 0xFFFFFFFF00000000ull) | static_cast<uint32_t>(static_cast<uint32_t>(d) + delta);
 }
 // Instruction descriptors: fp32 accumulator, both operands K-major, M = 128, N = n.
 __host__ __device__ constexpr uint32_t instr_desc(int n, uint32_t ab_format) {
@@ -208,18 +256,14 @@ constexpr uint32_t kFmtE4M3 = 0, kFmtBF16 = 1;
 
 template <int TN>
 struct Smem {
-  static constexpr int A_WORD_BYTES = TM * 32;            // one K-word of the A tile, expanded
-  static constexpr int B_WORD_BYTES = TN * 32;
-  static constexpr int A_STAGE = WPS * A_WORD_BYTES;
-  static constexpr int B_STAGE = WPS * B_WORD_BYTES;
-  static constexpr int SA_WORD_BYTES = TM * 16;           // scale pieces of one word slot: 8 bf16 per row
-  static constexpr int SB_WORD_BYTES = TN * 16;
+  static constexpr int A_STAGE = TM * 128;                // sign bytes of the A tile: 128 rows x 4 words x 32 bytes
+  static constexpr int SA_STAGE = TM * 128;               // scale pieces: per word slot 16 bytes of pieces + 16 of zeros
+  static constexpr int B_SIGNS = TN * 128;
+  static constexpr int B_STAGE = 2 * B_SIGNS;             // signs then scale pieces: one bulk copy
   static constexpr int OFF_A = 0;
-  static constexpr int OFF_B = OFF_A + STAGES * A_STAGE;
-  static constexpr int OFF_SA = OFF_B + STAGES * B_STAGE;               // [STAGES][WPS][TM rows][16 bytes]
-  static constexpr int OFF_SB = OFF_SA + STAGES * WPS * SA_WORD_BYTES;  // [STAGES][WPS][TN rows][16 bytes]
-  static constexpr int OFF_ZERO = OFF_SB + STAGES * WPS * SB_WORD_BYTES;  // 128 rows x 16 bytes of zeros
-  static constexpr int OFF_BAR = OFF_ZERO + TM * 16;
+  static constexpr int OFF_SA = OFF_A + STAGES * A_STAGE;
+  static constexpr int OFF_B = OFF_SA + STAGES * SA_STAGE;
+  static constexpr int OFF_BAR = OFF_B + STAGES * B_STAGE;
   static constexpr int NBUF = 512 / (2 * TN);                           // TMEM buffers: D and S side by side
   // barriers: full[STAGES], empty[STAGES], tfull[NBUF], tempty[NBUF], drain
   static constexpr int NBAR = 2 * STAGES + 2 * NBUF + 1;
@@ -229,12 +273,32 @@ struct Smem {
   static constexpr int BYTES = USED > 120 * 1024 ? USED : 120 * 1024;
 };
 
-// One side (A or B) of the producer: this thread owns tile row `p` of that operand.
-struct Side {
-  const uint32_t* bits; const void* scales;
-  int64_t rows, ld_w, ld_s, G;
-  int32_t bf16, r;       // r: segments per group of this operand
-};
+// Expands the weight operand once per call into the stage layout the main kernel reads: for every
+// TN-row tile of W and every stage of four K-words, the e4m3 sign bytes followed by the bf16
+// scale pieces, exactly as they sit in shared memory.  One block per (stage, tile), one thread per row.
+template <int TN>
+__global__ void __launch_bounds__(TN)
+prepare_w_kernel(const Args g, unsigned char* __restrict__ out) {
+  using S = Smem<TN>;
+  const int p = threadIdx.x;
+  const int64_t st = blockIdx.x, tile_n = blockIdx.y;
+  const int64_t n_stages = (g.n_words + WPS - 1) / WPS;
+  const int64_t n = tile_n * TN + p;
+  const bool in = n < g.N;
+  const int64_t kw = st * WPS;
+  uint4 w = make_uint4(0, 0, 0, 0);
+  if (in && kw < g.ldw_w) w = __ldg(reinterpret_cast<const uint4*>(g.w_bits + n * g.ldw_w + kw));
+  unsigned char* base = out + (tile_n * n_stages + st) * S::B_STAGE;
+  expand_words(base, p, w);
+#pragma unroll
+  for (int q = 0; q < WPS; q++) {
+    float f = 0.0f;
+    const int64_t grp = ((kw + q) / g.seg_words) / g.rw;
+    if (in && kw + q < g.n_words && grp < g.Gw) f = load_scale(g.w_scales, g.w_bf16, n * g.ldw_s + grp);
+    *reinterpret_cast<uint4*>(swz(base + S::B_SIGNS, p, 2 * q)) = scale_row<true>(f);
+    *reinterpret_cast<uint4*>(swz(base + S::B_SIGNS, p, 2 * q + 1)) = make_uint4(0, 0, 0, 0);
+  }
+}
 
 template <int TN>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -256,14 +320,15 @@ hbmm_umma_kernel(const Args g) {
   const int64_t n_tiles = tiles_m * tiles_n;
   const int64_t n_stages = (g.n_words + WPS - 1) / WPS;                 // per tile
   const int64_t n_segs = (g.n_words + g.seg_words - 1) / g.seg_words;   // per tile
-  // producer arrivals per stage: the four A warps, and as many B warps as the tile has rows for
-  constexpr int kBWarps = TN / 32 < 4 ? TN / 32 : 4;
 
   // ---- set-up
-  if (tid < TM) *reinterpret_cast<uint4*>(smem + S::OFF_ZERO + tid * 16) = make_uint4(0, 0, 0, 0);
+  // the zero halves of the A scale rows never change: written once for every stage
+  if (tid < TM)
+    for (int s = 0; s < STAGES; s++)
+      for (int q = 0; q < WPS; q++) *reinterpret_cast<uint4*>(swz(smem + S::OFF_SA + s * S::SA_STAGE, tid, 2 * q + 1)) = make_uint4(0, 0, 0, 0);
   if (tid == 0) {
     for (int s = 0; s < STAGES; s++) {
-      mbar_init(&full[s], 4 + kBWarps);               // one arrival per working producer warp
+      mbar_init(&full[s], kProducerWarps + 1);        // the A producer warps + the loader's expect_tx arrival
       mbar_init(&empty[s], 1);                        // MMA commit: the stage's bytes have been read
     }
     for (int b = 0; b < NBUF; b++) {
@@ -274,7 +339,7 @@ hbmm_umma_kernel(const Args g) {
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  fence_async_proxy();                                // the zero block is read by the tensor core
+  fence_async_proxy();                                // those zeros are read by the tensor core
   if (warp == kMmaWarp) {
     tmem_alloc(tmem_base_ptr, 512);
     tmem_relinquish();
@@ -287,88 +352,94 @@ hbmm_umma_kernel(const Args g) {
   // The CTA is persistent: it walks tiles blockIdx.x, blockIdx.x + gridDim.x, ... and the stage and
   // accumulator rings simply continue across tiles (gst / gseg count stages / segments since launch).
   if (warp >= kFirstProducerWarp && warp < kMmaWarp) {
-    // =========================== producers ===========================
+    // =========================== A producers ===========================
     reg_dec<kRegsProducer>();
-    const bool is_b = warp >= kFirstProducerWarp + 4;
-    const int p = (tid - kFirstProducerWarp * 32) & 127;    // tile row of this thread's operand
-    const int rows = is_b ? TN : TM;
-    if (p < rows) {                                          // (whole warps: TN is a multiple of 32)
-      Side sd;
-      if (is_b) { sd.bits = g.w_bits; sd.scales = g.w_scales; sd.rows = g.N; sd.ld_w = g.ldw_w; sd.ld_s = g.ldw_s; sd.G = g.Gw; sd.bf16 = g.w_bf16; sd.r = g.rw; }
-      else      { sd.bits = g.a_bits; sd.scales = g.a_scales; sd.rows = g.M; sd.ld_w = g.lda_w; sd.ld_s = g.lda_s; sd.G = g.Ga; sd.bf16 = g.a_bf16; sd.r = g.ra; }
-      unsigned char* sign_base = smem + (is_b ? S::OFF_B : S::OFF_A);
-      const int sign_stage = is_b ? S::B_STAGE : S::A_STAGE;
-      unsigned char* sc_row = smem + (is_b ? S::OFF_SB : S::OFF_SA) + (p >> 3) * 128 + (p & 7) * 16;
-      const int sc_word = is_b ? S::SB_WORD_BYTES : S::SA_WORD_BYTES;
-      // fp32 scales with one group per segment: the four scales of a stage are one 16-byte vector
-      const bool vec_scales = !sd.bf16 && sd.r == 1 && g.seg_words == 1;
+    const int p = tid - kFirstProducerWarp * 32;             // tile row of this thread
+    // fp32 scales with one group per segment: the four scales of a stage are one 16-byte vector
+    const bool vec_scales = !g.a_bf16 && g.ra == 1 && g.seg_words == 1;
+    int64_t gst = 0;
+    bool ok = true;
+    for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      const int64_t m = (tile / tiles_n) * TM + p;
+      const bool in = m < g.M;
+      const uint32_t* bptr = g.a_bits + (in ? m : 0) * g.lda_w;
+      const int64_t srow = (in ? m : 0) * g.lda_s;
+      int in_seg = 0, in_g = 0;      // position of the next word to fetch inside its segment / group
+      int64_t grp = 0;
+      auto fetch = [&](int64_t st, uint4& w, float (&f)[WPS]) {
+        const int64_t kw = st * WPS;
+        w = make_uint4(0, 0, 0, 0);
+        if (in && kw < g.lda_w) w = __ldg(reinterpret_cast<const uint4*>(bptr + kw));
+        if (vec_scales) {
+          float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (in && kw < g.lda_s) v = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(g.a_scales) + srow + kw));
+          f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;    // entries past the last group are stored zeros
+        } else {
+          // first decide which scale every word needs (no loaded value is touched here) ...
+          int64_t idx[WPS];
+#pragma unroll
+          for (int q = 0; q < WPS; q++) {
+            idx[q] = (in && kw + q < g.n_words && grp < g.Ga) ? srow + grp : -1;
+            if (++in_seg == g.seg_words) { in_seg = 0; if (++in_g == g.ra) { in_g = 0; grp++; } }
+          }
+          // ... then issue the loads back to back
+#pragma unroll
+          for (int q = 0; q < WPS; q++) { f[q] = 0.0f; if (idx[q] >= 0) f[q] = load_scale(g.a_scales, g.a_bf16, idx[q]); }
+        }
+      };
+      uint4 w, nw;
+      float f[WPS], nf[WPS];
+      fetch(0, w, f);
+      for (int64_t st = 0; st < n_stages; st++, gst++) {
+        if (st + 1 < n_stages) fetch(st + 1, nw, nf);     // in flight while this stage is expanded
+        const int s = static_cast<int>(gst % STAGES);
+        if (gst >= STAGES && !mbar_wait(&empty[s], static_cast<uint32_t>(((gst / STAGES) & 1) ^ 1), abort_flag, 1)) { ok = false; break; }
+        expand_words(smem + S::OFF_A + s * S::A_STAGE, p, w);
+#pragma unroll
+        for (int q = 0; q < WPS; q++)
+          *reinterpret_cast<uint4*>(swz(smem + S::OFF_SA + s * S::SA_STAGE, p, 2 * q)) = scale_row<false>(f[q]);
+        fence_async_proxy();          // make the generic-proxy stores visible to the tensor core
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&full[s]);
+        w = nw;
+#pragma unroll
+        for (int q = 0; q < WPS; q++) f[q] = nf[q];
+      }
+    }
+  } else if (warp == kLoaderWarp) {
+    // =========================== W loader ===========================
+    reg_dec<kRegsIssuer>();
+    if (lane == 0) {
       int64_t gst = 0;
       bool ok = true;
       for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-        const int64_t rix = (is_b ? (tile % tiles_n) * TN : (tile / tiles_n) * TM) + p;
-        const bool in = rix < sd.rows;
-        const uint32_t* bptr = sd.bits + (in ? rix : 0) * sd.ld_w;
-        const int64_t srow = (in ? rix : 0) * sd.ld_s;
-        int in_seg = 0, in_g = 0;      // position of the next word to fetch inside its segment / group
-        int64_t grp = 0;
-        auto fetch = [&](int64_t st, uint4& w, float (&f)[WPS]) {
-          const int64_t kw = st * WPS;
-          w = make_uint4(0, 0, 0, 0);
-          if (in && kw < sd.ld_w) w = __ldg(reinterpret_cast<const uint4*>(bptr + kw));
-          if (vec_scales) {
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (in && kw < sd.ld_s) v = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(sd.scales) + srow + kw));
-            f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;    // entries past the last group are stored zeros
-          } else {
-            // first decide which scale every word needs (no loaded value is touched here) ...
-            int64_t idx[WPS];
-#pragma unroll
-            for (int q = 0; q < WPS; q++) {
-              idx[q] = (in && kw + q < g.n_words && grp < sd.G) ? srow + grp : -1;
-              if (++in_seg == g.seg_words) { in_seg = 0; if (++in_g == sd.r) { in_g = 0; grp++; } }
-            }
-            // ... then issue the loads back to back
-#pragma unroll
-            for (int q = 0; q < WPS; q++) { f[q] = 0.0f; if (idx[q] >= 0) f[q] = load_scale(sd.scales, sd.bf16, idx[q]); }
-          }
-        };
-        uint4 w, nw;
-        float f[WPS], nf[WPS];
-        fetch(0, w, f);
+        const unsigned char* src = g.w_prep + (tile % tiles_n) * n_stages * S::B_STAGE;
         for (int64_t st = 0; st < n_stages; st++, gst++) {
-          if (st + 1 < n_stages) fetch(st + 1, nw, nf);     // in flight while this stage is expanded
           const int s = static_cast<int>(gst % STAGES);
-          if (gst >= STAGES && !mbar_wait(&empty[s], static_cast<uint32_t>(((gst / STAGES) & 1) ^ 1), abort_flag, 1)) { ok = false; break; }
-          expand_words(sign_base + s * sign_stage, rows, p, w);
-#pragma unroll
-          for (int q = 0; q < WPS; q++)
-            *reinterpret_cast<uint4*>(sc_row + (s * WPS + q) * sc_word) = is_b ? scale_row<true>(f[q]) : scale_row<false>(f[q]);
-          fence_async_proxy();          // make the generic-proxy stores visible to the tensor core
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&full[s]);
-          w = nw;
-#pragma unroll
-          for (int q = 0; q < WPS; q++) f[q] = nf[q];
+          if (gst >= STAGES && !mbar_wait(&empty[s], static_cast<uint32_t>(((gst / STAGES) & 1) ^ 1), abort_flag, 6)) { ok = false; break; }
+          mbar_arrive_expect_tx(&full[s], S::B_STAGE);
+          bulk_copy_g2s(smem + S::OFF_B + s * S::B_STAGE, src + st * S::B_STAGE, S::B_STAGE, &full[s]);
         }
       }
     }
+    __syncwarp();
   } else if (warp == kMmaWarp) {
     // =========================== MMA issuer ===========================
     reg_dec<kRegsIssuer>();
     if (lane == 0) {
       constexpr uint32_t idesc_sign = instr_desc(TN, kFmtE4M3), idesc_scale = instr_desc(TN, kFmtBF16);
-      // Descriptors of stage 0 / word 0; every other slot differs only by its start address (and, for
-      // the scale operands, by the distance to the zero block), so they are stepped with 32-bit adds
-      // of the low word: +bytes/16 in the address field, -bytes/16 in the lbo field (bits 16..29).
-      const uint32_t zero_addr = smem_u32(smem + S::OFF_ZERO);
-      const uint32_t sa0 = smem_u32(smem + S::OFF_SA), sb0 = smem_u32(smem + S::OFF_SB);
-      const uint64_t da0 = smem_desc(smem_u32(smem + S::OFF_A), TM * 16, 128);
-      const uint64_t db0 = smem_desc(smem_u32(smem + S::OFF_B), TN * 16, 128);
-      const uint64_t dsa0 = smem_desc(sa0, zero_addr - sa0, 128), dsb0 = smem_desc(sb0, zero_addr - sb0, 128);
-      constexpr uint32_t kStepA = S::A_WORD_BYTES >> 4, kStepB = S::B_WORD_BYTES >> 4;
-      constexpr uint32_t kSa = S::SA_WORD_BYTES >> 4, kSb = S::SB_WORD_BYTES >> 4;
-      constexpr uint32_t kStepSA = kSa - (kSa << 16), kStepSB = kSb - (kSb << 16);   // modulo 2^32 on purpose
+      // Descriptors of stage 0 / word slot 0; every other slot differs only by its start address, so
+      // the low descriptor word is stepped by bytes/16.
+      const uint64_t da0 = smem_desc(smem_u32(smem + S::OFF_A)), db0 = smem_desc(smem_u32(smem + S::OFF_B));
+      const uint64_t dsa0 = smem_desc(smem_u32(smem + S::OFF_SA)), dsb0 = smem_desc(smem_u32(smem + S::OFF_B + S::B_SIGNS));
+      constexpr uint32_t kWord = 32 >> 4;                                   // next word slot: 32 bytes along the rows
+      constexpr uint32_t kStageA = S::A_STAGE >> 4, kStageSA = S::SA_STAGE >> 4, kStageB = S::B_STAGE >> 4;
       const uint32_t n_words = static_cast<uint32_t>(g.n_words), seg_words = static_cast<uint32_t>(g.seg_words);
+      const uint32_t full_a = smem_u32(full), empty_a = smem_u32(empty), tfull_a = smem_u32(tfull), tempty_a = smem_u32(tempty);
+      const uint32_t da_lo = static_cast<uint32_t>(da0), db_lo = static_cast<uint32_t>(db0);
+      const uint32_t dsa_lo = static_cast<uint32_t>(dsa0), dsb_lo = static_cast<uint32_t>(dsb0);
+      const uint64_t da_hi = da0 & 0xFFFFFFFF00000000ull, db_hi = db0 & 0xFFFFFFFF00000000ull;
+      const uint64_t dsa_hi = dsa0 & 0xFFFFFFFF00000000ull, dsb_hi = dsb0 & 0xFFFFFFFF00000000ull;
       uint32_t s = 0, full_par = 0;          // stage slot and the parity its "full" barrier completes with next
       uint32_t buf = 0, tempty_par = 0;      // accumulator buffer; the first pass over the ring needs no wait
       bool first_ring = true;
@@ -376,26 +447,29 @@ hbmm_umma_kernel(const Args g) {
       for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
         uint32_t in_seg = 0;
         for (uint32_t kw0 = 0; kw0 < n_words && ok; kw0 += WPS) {
-          if (!mbar_wait(&full[s], full_par, abort_flag, 2)) { ok = false; break; }
+          if (!mbar_wait_a(full_a + s * 8, full_par, abort_flag, 2)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t slot = s * WPS;
           const uint32_t nq = n_words - kw0 < WPS ? n_words - kw0 : WPS;
+          // low descriptor words of word slot 0 of this stage; the slots step by constants
+          uint32_t a_lo = da_lo + s * kStageA, b_lo = db_lo + s * kStageB;
+          uint32_t sa_lo = dsa_lo + s * kStageSA, sb_lo = dsb_lo + s * kStageB;
           for (uint32_t q = 0; q < nq; q++) {
-            const uint32_t d_tmem = tmem_base + buf * 2 * TN;
+            const uint32_t d_tmem = tmem_base + buf * (2 * TN);
             if (in_seg == 0 && !first_ring) {
-              if (!mbar_wait(&tempty[buf], tempty_par, abort_flag, 3)) { ok = false; break; }
+              if (!mbar_wait_a(tempty_a + buf * 8, tempty_par, abort_flag, 3)) { ok = false; break; }
               tc_fence_after();
             }
-            umma_f8(d_tmem, desc_step(da0, (slot + q) * kStepA), desc_step(db0, (slot + q) * kStepB), idesc_sign, in_seg);
+            umma_f8(d_tmem, da_hi | a_lo, db_hi | b_lo, idesc_sign, in_seg);
             if (++in_seg == seg_words || kw0 + q == n_words - 1) {
-              // scale product of the segment: K columns 0..7 from this word slot, 8..15 from the zero block
-              umma_bf16_overwrite(d_tmem + TN, desc_step(dsa0, (slot + q) * kStepSA), desc_step(dsb0, (slot + q) * kStepSB), idesc_scale);
-              umma_commit(&tfull[buf]);     // segment complete: hand D and S to the epilogue
+              // scale product of the segment (K columns 0..7 hold the pieces of this word slot, 8..15 zeros)
+              umma_bf16_overwrite(d_tmem + TN, dsa_hi | sa_lo, dsb_hi | sb_lo, idesc_scale);
+              umma_commit_a(tfull_a + buf * 8);   // segment complete: hand D and S to the epilogue
               in_seg = 0;
               if (++buf == NBUF) { buf = 0; if (first_ring) first_ring = false; else tempty_par ^= 1; }
             }
+            a_lo += kWord; b_lo += kWord; sa_lo += kWord; sb_lo += kWord;
           }
-          umma_commit(&empty[s]);           // stage's bytes are free once these MMAs have read them
+          umma_commit_a(empty_a + s * 8);     // stage's bytes are free once these MMAs have read them
           if (++s == STAGES) { s = 0; full_par ^= 1; }
         }
       }
@@ -409,41 +483,54 @@ hbmm_umma_kernel(const Args g) {
     const int wg = warp >> 2;                       // column half
     const int row = (warp & 3) * 32 + lane;         // TMEM lane = tile row
     const uint32_t t_lane = static_cast<uint32_t>((warp & 3) * 32) << 16;
-    int64_t gseg = 0;
+    // The warp's columns of a segment are read in two pieces (D and S of each), double buffered: while the
+    // FMAs of one piece run, the loads of the next piece -- of the next segment when this was the
+    // last one -- are in flight.  (tcgen05.wait::ld waits for every outstanding load, so two pieces
+    // are as deep as the pipeline can usefully go.)
+    constexpr int PIECES = 2, PW = HALF / 2;        // piece width: 32 columns for TN = 128, 16 for TN = 64
+    const int64_t my_tiles = blockIdx.x < n_tiles ? (n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    const int64_t total_segs = my_tiles * n_segs;
+    uint32_t d[2][PW], sc[2][PW];
+    uint64_t acc[HALF / 2];                         // two fp32 outputs per register pair
     bool ok = true;
-    for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-      uint64_t acc[HALF / 2];                       // two fp32 outputs per register pair
+    auto tmem_of = [&](int64_t gseg) { return tmem_base + t_lane + static_cast<uint32_t>(gseg % NBUF) * 2 * TN + wg * HALF; };
+    if (total_segs > 0) {
+      ok = mbar_wait(&tfull[0], 0, abort_flag, 5);
+      tc_fence_after();
+      if (ok) { tmem_ld_piece(tmem_of(0), d[0]); tmem_ld_piece(tmem_of(0) + TN, sc[0]); tmem_ld_wait(); }
+    }
+    int64_t tile = blockIdx.x, seg = 0;
+    for (int64_t gseg = 0; gseg < total_segs && ok; gseg++) {
+      if (seg == 0) {
 #pragma unroll
-      for (int j = 0; j < HALF / 2; j++) acc[j] = 0ull;
-      for (int64_t seg = 0; seg < n_segs; seg++, gseg++) {
-        const int buf = static_cast<int>(gseg % NBUF);
-        if (!mbar_wait(&tfull[buf], static_cast<uint32_t>((gseg / NBUF) & 1), abort_flag, 5)) { ok = false; break; }
-        tc_fence_after();
-        const uint32_t t_d = tmem_base + t_lane + buf * 2 * TN + wg * HALF, t_s = t_d + TN;
-        // 16-column pieces, double buffered: the loads of piece c+1 are in flight during the math of c
-        constexpr int PIECES = HALF / 16;
-        uint32_t d[2][16], sc[2][16];
-        tmem_ld16(t_d, d[0]);
-        tmem_ld16(t_s, sc[0]);
-        tmem_ld_wait();
+        for (int j = 0; j < HALF / 2; j++) acc[j] = 0ull;
+      }
 #pragma unroll
-        for (int c = 0; c < PIECES; c++) {
-          if (c + 1 < PIECES) {
-            tmem_ld16(t_d + (c + 1) * 16, d[(c + 1) & 1]);
-            tmem_ld16(t_s + (c + 1) * 16, sc[(c + 1) & 1]);
-          }
-#pragma unroll
-          for (int j = 0; j < 16; j += 2)
-            acc[(c * 16 + j) / 2] = fma2(pack2(sc[c & 1][j], sc[c & 1][j + 1]), pack2(d[c & 1][j], d[c & 1][j + 1]), acc[(c * 16 + j) / 2]);
-          if (c + 1 < PIECES) tmem_ld_wait();
-          if (c == PIECES - 2) {                    // the last loads have landed: the buffer can be refilled
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&tempty[buf]);
+      for (int c = 0; c < PIECES; c++) {
+        // piece c of this segment is in d[c & 1] / sc[c & 1]; start the loads of what comes next
+        if (c + 1 < PIECES) {
+          tmem_ld_piece(tmem_of(gseg) + (c + 1) * PW, d[(c + 1) & 1]);
+          tmem_ld_piece(tmem_of(gseg) + TN + (c + 1) * PW, sc[(c + 1) & 1]);
+        } else {
+          // every column of this segment is in registers: the buffer can be refilled
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&tempty[gseg % NBUF]);
+          if (gseg + 1 < total_segs) {
+            if (!mbar_wait(&tfull[(gseg + 1) % NBUF], static_cast<uint32_t>(((gseg + 1) / NBUF) & 1), abort_flag, 5)) { ok = false; break; }
+            tc_fence_after();
+            tmem_ld_piece(tmem_of(gseg + 1), d[(c + 1) & 1]);
+            tmem_ld_piece(tmem_of(gseg + 1) + TN, sc[(c + 1) & 1]);
           }
         }
+#pragma unroll
+        for (int j = 0; j < PW; j += 2)
+          acc[(c * PW + j) / 2] = fma2(pack2(sc[c & 1][j], sc[c & 1][j + 1]), pack2(d[c & 1][j], d[c & 1][j + 1]), acc[(c * PW + j) / 2]);
+        tmem_ld_wait();
       }
-      if (ok) {
+      if (!ok) break;
+      if (++seg == n_segs) {
+        seg = 0;
         const int64_t m = (tile / tiles_n) * TM + row, nb = (tile % tiles_n) * TN + wg * HALF;
         if (m < g.M) {
           float* dst = g.C + m * g.ldc + nb;
@@ -458,10 +545,11 @@ hbmm_umma_kernel(const Args g) {
                 if (nb + j + e < g.N) dst[j + e] = v[e];
           }
         }
+        tile += gridDim.x;
       }
     }
   } else {
-    reg_dec<kRegsIssuer>();   // warps 17..19: nothing to do but hand their registers over
+    reg_dec<kRegsIssuer>();   // warps 14, 15: nothing to do but hand their registers over
   }
 
   // ---- teardown: everyone meets here (aborted threads too), then the allocating warp frees TMEM
@@ -474,7 +562,13 @@ hbmm_umma_kernel(const Args g) {
 }
 
 template <int TN>
-cudaError_t launch_umma(const Args& g, cudaStream_t stream) {
+size_t prep_bytes(const Args& g) {
+  const int64_t tiles_n = (g.N + TN - 1) / TN, n_stages = (g.n_words + WPS - 1) / WPS;
+  return static_cast<size_t>(tiles_n * n_stages) * Smem<TN>::B_STAGE;
+}
+
+template <int TN>
+cudaError_t launch_umma(Args g, void* workspace, cudaStream_t stream) {
   using S = Smem<TN>;
   static bool configured = false;
   static int sms = 0;
@@ -486,24 +580,17 @@ cudaError_t launch_umma(const Args& g, cudaStream_t stream) {
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     configured = true;
   }
-  const int64_t tiles = ((g.M + TM - 1) / TM) * ((g.N + TN - 1) / TN);
+  const int64_t tiles_n = (g.N + TN - 1) / TN, n_stages = (g.n_words + WPS - 1) / WPS;
+  dim3 pgrid(static_cast<unsigned>(n_stages), static_cast<unsigned>(tiles_n));
+  prepare_w_kernel<TN><<<pgrid, TN, 0, stream>>>(g, static_cast<unsigned char*>(workspace));
+  g.w_prep = static_cast<const unsigned char*>(workspace);
+  const int64_t tiles = ((g.M + TM - 1) / TM) * tiles_n;
   const unsigned grid = static_cast<unsigned>(tiles < sms ? tiles : sms);   // one persistent CTA per SM
   hbmm_umma_kernel<TN><<<grid, kThreads, S::BYTES, stream>>>(g);
   return cudaGetLastError();
 }
 
-}  // namespace
-
-// K a multiple of 32 and segments of whole words (any number of them).
-bool gemm_tensor_supported(const PackedView& A, const PackedView& W) {
-  if (A.K % 32 != 0) return false;
-  const bool a_one = A.beta >= A.K, w_one = W.beta >= W.K;
-  if (!a_one && A.beta % 32 != 0) return false;
-  if (!w_one && W.beta % 32 != 0) return false;
-  return true;
-}
-
-cudaError_t launch_gemm_tensor(const PackedView& A, const PackedView& W, float* C, int64_t ldc, cudaStream_t stream) {
+Args make_args(const PackedView& A, const PackedView& W, float* C, int64_t ldc) {
   Args g;
   g.a_bits = A.bits; g.a_scales = A.scales; g.w_bits = W.bits; g.w_scales = W.scales; g.C = C;
   g.M = A.rows; g.N = W.rows; g.lda_w = A.ld_words; g.ldw_w = W.ld_words; g.lda_s = A.ld_scales; g.ldw_s = W.ld_scales;
@@ -521,7 +608,32 @@ cudaError_t launch_gemm_tensor(const PackedView& A, const PackedView& W, float* 
   g.rw = static_cast<int32_t>(w_one ? T : W.beta / seg);
   g.Ga = num_groups(A.K, A.beta);
   g.Gw = num_groups(W.K, W.beta);
-  return g.N <= 64 ? launch_umma<64>(g, stream) : launch_umma<128>(g, stream);
+  g.w_prep = nullptr;
+  return g;
+}
+
+}  // namespace
+
+// K a multiple of 32 and segments of whole words (any number of them).
+bool gemm_tensor_supported(const PackedView& A, const PackedView& W) {
+  if (A.K % 32 != 0) return false;
+  const bool a_one = A.beta >= A.K, w_one = W.beta >= W.K;
+  if (!a_one && A.beta % 32 != 0) return false;
+  if (!w_one && W.beta % 32 != 0) return false;
+  return true;
+}
+
+// Bytes of workspace the tensor path needs: the weight operand expanded into its stage layout.
+size_t gemm_tensor_workspace_bytes(const PackedView& A, const PackedView& W) {
+  const Args g = make_args(A, W, nullptr, 0);
+  return g.N <= 64 ? prep_bytes<64>(g) : prep_bytes<128>(g);
+}
+
+// workspace: device, 16-byte aligned, at least gemm_tensor_workspace_bytes.
+cudaError_t launch_gemm_tensor(const PackedView& A, const PackedView& W, float* C, int64_t ldc, void* workspace,
+                               cudaStream_t stream) {
+  const Args g = make_args(A, W, C, ldc);
+  return g.N <= 64 ? launch_umma<64>(g, workspace, stream) : launch_umma<128>(g, workspace, stream);
 }
 
 cudaError_t read_umma_error(int* code) {

@@ -52,7 +52,8 @@ cudaError_t launch_partials_b1(const PackedView& A, const PackedView& W, int32_t
 // read_umma_error copies the device-side error word (0 = no bounded wait ever expired); it synchronises.
 cudaError_t read_umma_error(int* code);
 bool gemm_tensor_supported(const PackedView& A, const PackedView& W);
-cudaError_t launch_gemm_tensor(const PackedView& A, const PackedView& W, float* C, int64_t ldc,
+size_t gemm_tensor_workspace_bytes(const PackedView& A, const PackedView& W);
+cudaError_t launch_gemm_tensor(const PackedView& A, const PackedView& W, float* C, int64_t ldc, void* workspace,
                                cudaStream_t stream);
 
 // Dense x packed contraction (HBWN).

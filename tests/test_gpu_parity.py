@@ -134,6 +134,12 @@ def _paths(hb):
     return [hb.PATH_POPC, hb.PATH_B1MMA, hb.PATH_TENSOR, hb.PATH_AUTO]
 
 
+def _gemm_ws(hb, A, W):
+    """Workspace of the contraction (the tensor-core path keeps its expanded weight operand there)."""
+    n = hb.gemm_workspace_bytes(A, W)
+    return torch.empty(max(n, 16), dtype=torch.uint8, device="cuda")
+
+
 @pytest.mark.parametrize("M,N,K,ba,bw,sdt", GEMM_CASES)
 def test_gemm_matches_oracle_on_every_path(hb, M, N, K, ba, bw, sdt):
     gu = _gu()
@@ -143,11 +149,12 @@ def test_gemm_matches_oracle_on_every_path(hb, M, N, K, ba, bw, sdt):
     W, dw, sw = gu.oracle_operand(w, bw, sdt)
     c_ref, absref = oracle.hbmm_from_quantized(da, sa, gu.eff_beta(ba, K), dw, sw, gu.eff_beta(bw, K))
     ran = 0
+    ws = _gemm_ws(hb, A, W)
     for path in _paths(hb):
         ldc = (N + 3) // 4 * 4 + 4
         C = torch.full((M, ldc), float("nan"), device="cuda")
         try:
-            hb.gemm_ex(A, W, C, path)
+            hb.gemm_ex(A, W, C, path, ws)
         except hb.HbmmError as e:
             assert e.status == hb.ERR_UNSUPPORTED and path not in (hb.PATH_POPC, hb.PATH_AUTO)
             continue
@@ -170,10 +177,11 @@ def test_unit_scales_give_exact_integers(hb, M, N, K, beta):
     A = hb.wrap_packed(gu.dev_bits(oracle.pack(sa, lw)), gu.scales_to_dev(np.ones((M, G)), hb.F32, ls), K, beta)
     W = hb.wrap_packed(gu.dev_bits(oracle.pack(sw, lw)), gu.scales_to_dev(np.ones((N, G)), hb.F32, ls), K, beta)
     ref = sa.astype(np.int32) @ sw.astype(np.int32).T
+    ws = _gemm_ws(hb, A, W)
     for path in _paths(hb):
         C = torch.empty((M, (N + 3) // 4 * 4), device="cuda")
         try:
-            hb.gemm_ex(A, W, C, path)
+            hb.gemm_ex(A, W, C, path, ws)
         except hb.HbmmError as e:
             assert e.status == hb.ERR_UNSUPPORTED
             continue
@@ -190,7 +198,7 @@ def test_quantize_then_gemm_end_to_end(hb):
         A = hb.quantize(torch.from_numpy(a).cuda(), hb.alloc_operand(M, K, 32, sdt))
         W = hb.quantize(torch.from_numpy(w).cuda(), hb.alloc_operand(N, K, 32, sdt))
         C = torch.empty((M, N), device="cuda")
-        hb.gemm(A, W, C)
+        hb.gemm(A, W, C, _gemm_ws(hb, A, W))
         c_ref, absref = oracle.hbmm(a, w, 32, 32, None)       # exact scales: the GPU's rounding is inside rtol
         gu.assert_close_rel_absref(C.cpu().numpy(), c_ref, absref, rtol)
 
@@ -278,3 +286,25 @@ def test_conv_im2col_matches_oracle(hb, B, C, H, W, N, kh, kw, st, pd, ba, bw, s
         _, _, lw, ls = hb.operand_bytes(M, K, ba, hb.F32)
         bits = ws[: M * lw * 4].view(torch.int32).reshape(M, lw)
         assert np.array_equal(gu.host_bits(bits), oracle.pack(sa, lw))
+
+
+def test_tensor_path_needs_its_workspace_and_auto_falls_back(hb):
+    """Without a workspace the tensor-core path is refused before any launch, and the automatic choice
+    runs the integer-pipe kernel instead; with one, both give the oracle's result."""
+    gu = _gu()
+    M, N, K = 96, 80, 256
+    a = inputs.normal((M, K), 77)
+    w = inputs.he_normal(N, K, 78)
+    A, da, sa = gu.oracle_operand(a, 32)
+    W, dw, sw = gu.oracle_operand(w, 32)
+    c_ref, absref = oracle.hbmm_from_quantized(da, sa, 32, dw, sw, 32)
+    assert hb.gemm_workspace_bytes(A, W) > 0
+    C = torch.empty((M, N), device="cuda")
+    with pytest.raises(hb.HbmmError) as e:
+        hb.gemm_ex(A, W, C, hb.PATH_TENSOR)
+    assert e.value.status == hb.ERR_WORKSPACE
+    hb.gemm(A, W, C)                                   # no workspace: integer-pipe path
+    gu.assert_close_rel_absref(C.cpu().numpy(), c_ref, absref, RTOL)
+    C.zero_()
+    hb.gemm(A, W, C, _gemm_ws(hb, A, W))
+    gu.assert_close_rel_absref(C.cpu().numpy(), c_ref, absref, RTOL)
