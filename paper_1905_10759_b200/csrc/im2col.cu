@@ -183,35 +183,41 @@ inline TilePlan make_plan(const ConvGeom& g, int sms) {
 template <typename T, typename Conv>
 __device__ __forceinline__ void stage_tile(T* tile, const void* __restrict__ x, int x_bf16, const ConvGeom& g,
                                            int64_t b, int c0, int cc, int yo0, const TilePlan& tp, Conv conv) {
-  // Work items are (staged row (c, r), block of 32 consecutive columns); a warp takes them eight at a
-  // time so that eight independent global loads are in flight before the first shared-memory store.
-  constexpr int BATCH = 8;
+  // A warp stages four tile rows (c, r) per pass, 64 columns of each at a time: the eight global
+  // loads of a pass are issued before the first shared-memory store, and all index arithmetic that
+  // needs a division is done once per row.
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
   const int y_base = yo0 * g.sh - g.ph;
-  const int xblocks = (tp.span + 31) / 32;
-  const int items = cc * tp.rows_in * xblocks;
-  for (int it0 = warp * BATCH; it0 < items; it0 += nwarps * BATCH) {
-    float v[BATCH];
-    int dst[BATCH];
+  const int rows_total = cc * tp.rows_in;
+  for (int row0 = warp * 4; row0 < rows_total; row0 += nwarps * 4) {
+    int64_t src[4];
+    bool rin[4];
 #pragma unroll
-    for (int u = 0; u < BATCH; u++) {
-      const int it = it0 + u;
-      v[u] = 0.0f;
-      dst[u] = -1;
-      if (it < items) {
-        const int row = it / xblocks, xx = (it - row * xblocks) * 32 + lane;
-        const int c = row / tp.rows_in, r = row - c * tp.rows_in;
-        const int y = y_base + r, xi = xx - g.pw;
-        if (xx < tp.span) {
-          dst[u] = row * tp.span + xx;
-          if (y >= 0 && y < g.H && xi >= 0 && xi < g.W)
-            v[u] = load_x(x, x_bf16, ((b * g.C + c0 + c) * static_cast<int64_t>(g.H) + y) * g.W + xi);
-        }
-      }
+    for (int u = 0; u < 4; u++) {
+      const int row = row0 + u;
+      const int c = row / tp.rows_in, r = row - c * tp.rows_in;
+      const int y = y_base + r;
+      rin[u] = row < rows_total && y >= 0 && y < g.H;
+      src[u] = ((b * g.C + c0 + c) * static_cast<int64_t>(g.H) + (rin[u] ? y : 0)) * g.W - g.pw;
     }
+    for (int xx0 = 0; xx0 < tp.span; xx0 += 64) {
+      float v[4][2];
 #pragma unroll
-    for (int u = 0; u < BATCH; u++)
-      if (dst[u] >= 0) tile[dst[u]] = conv(v[u]);
+      for (int u = 0; u < 4; u++)
+#pragma unroll
+        for (int h = 0; h < 2; h++) {
+          const int xx = xx0 + h * 32 + lane, xi = xx - g.pw;
+          v[u][h] = 0.0f;
+          if (rin[u] && xx < tp.span && xi >= 0 && xi < g.W) v[u][h] = load_x(x, x_bf16, src[u] + xx);
+        }
+#pragma unroll
+      for (int u = 0; u < 4; u++)
+#pragma unroll
+        for (int h = 0; h < 2; h++) {
+          const int xx = xx0 + h * 32 + lane;
+          if (row0 + u < rows_total && xx < tp.span) tile[(row0 + u) * tp.span + xx] = conv(v[u][h]);
+        }
+    }
   }
 }
 

@@ -110,6 +110,20 @@ def test_partials_bit_exact(hb, M, N, K, ba, bw):
     assert np.array_equal(D.cpu().numpy(), d_ref)
 
 
+@pytest.mark.parametrize("M,N,K,ba,bw", [(33, 17, 576, 128, 128), (20, 9, 1024, 256, 128), (6, 7, 77, 77, 77),
+                                         (40, 70, 640, 128, 640), (65, 66, 200, 128, 128)])
+def test_partials_bit_exact_on_the_b1_tensor_instruction(hb, M, N, K, ba, bw):
+    gu = _gu()
+    a = inputs.normal((M, K), 2100 + M + K)
+    w = inputs.normal((N, K), 3100 + N + K)
+    A, _, sa = gu.oracle_operand(a, ba)
+    W, _, sw = gu.oracle_operand(w, bw)
+    d_ref, _ = oracle.partials(sa, sw, gu.eff_beta(ba, K), gu.eff_beta(bw, K))
+    D = torch.full(d_ref.shape, -12345, dtype=torch.int32, device="cuda")
+    hb.gemm_partials(A, W, D, hb.PATH_B1MMA)
+    assert np.array_equal(D.cpu().numpy(), d_ref)
+
+
 # ------------------------------------------------------------------ packed x packed contraction
 GEMM_CASES = [
     # M, N, K, beta_a, beta_w, scale dtype
