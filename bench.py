@@ -120,13 +120,17 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+FALLBACK_BF16_TFLOPS = 1590.0
+
+
 def measured_peaks():
+    """(HBM GB/s, dense bf16 TFLOP/s burst, 'measured' | 'fallback')."""
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
         with open(p) as f:
             d = json.load(f)
-        return float(d["hbm_gbs"]), "measured"
-    return FALLBACK_HBM_GBS, "fallback"
+        return float(d["hbm_gbs"]), float(d["bf16_tflops"]), "measured"
+    return FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS, "fallback"
 
 
 # ----------------------------------------------------------------------------- workload
@@ -168,7 +172,8 @@ def run_step(hbmm, layers):
         hbmm.conv_im2col(L["xb"], L["geom"], 1, hbmm.F32, L["W"], L["Cb"], L["ws"])       # rows I, H
 
 
-LAUNCHES_PER_STEP = 4 * (2 + 2)  # per layer: gather+binarize, contraction; bf16 gather, HBWN contraction
+# per layer: gather+binarize, weight expansion, contraction; bf16 gather, weight pieces, HBWN contraction
+LAUNCHES_PER_STEP = 4 * (3 + 3)
 
 
 def run_step_e2e(hbmm, layers):
@@ -213,30 +218,38 @@ def kernel_breakdown(torch, hbmm, layers, iters: int):
         t_convb = time_loop(torch, lambda: hbmm.conv_im2col(L["xb"], L["geom"], 1, hbmm.F32, L["W"], L["Cb"], L["ws"]), iters)
         ld = (s.K + 7) // 8 * 8
         Ad = hbmm.wrap_dense(L["ws"][: s.M * ld * 2].view(torch.bfloat16).reshape(s.M, ld)[:, : s.K])
-        t_hbwn = time_loop(torch, lambda: hbmm.gemm(Ad, L["W"], L["Cb"]), iters)
+        hws = torch.empty(max(hbmm.gemm_workspace_bytes(Ad, L["W"]), 16), dtype=torch.uint8, device=L["C"].device)
+        t_hbwn = time_loop(torch, lambda: hbmm.gemm(Ad, L["W"], L["Cb"], hws), iters)
         out["hbwn_contraction"].append(t_hbwn)
         out["front_end_bf16"].append(max(t_convb - t_hbwn, 0.0))
     return out
 
 
-def roofline_for(kind: str, li: int, shape, ms: float, hbm_gbs: float, hbm_src: str):
-    """Roofline entry of one kernel launch (layer li) given its measured duration."""
+def roofline_for(kind: str, li: int, shape, ms: float, peaks):
+    """Roofline entry of one kernel launch (layer li) given its measured duration.
+
+    Both contractions run on the tensor cores (sign bits as +-1 e4m3 for HBMM, +-1 bf16 for HBWN), so
+    they are set against the dense tensor peak of their operand type: the measured bf16 GEMM peak, and
+    twice that for the 8-bit type (the nominal fp8 : bf16 ratio).  For HBMM the fraction of the
+    integer-pipe popcount roofline (one POPC per output and K-word at 16 / clk / SM) is given beside it."""
+    hbm_gbs, bf16_tflops, hbm_src = peaks
     M, N, K = shape.M, shape.N, shape.K
     G = -(-K // BETA)
     if kind == "hbmm_contraction":
         ops = 2.0 * M * N * K
-        # integer pipe: one 32-bit popcount per output and K-word; 64 binary ops per popcount
-        peak = SM_COUNT * POPC_PER_CLK_SM * SM_MAX_MHZ * 1e6 * 64 / 1e12
-        return {"kernel": "hbmm_contraction/%s" % shape.name, "bound": "alu", "achieved": ops / (ms * 1e-3) / 1e12,
-                "peak": peak, "unit": "TOP/s", "frac": ops / (ms * 1e-3) / 1e12 / peak, "traffic": None,
-                "peak_source": "148 SMs x 16 POPC/clk x 1965 MHz x 64 binary ops"}
+        peak = 2.0 * bf16_tflops
+        popc_peak = SM_COUNT * POPC_PER_CLK_SM * SM_MAX_MHZ * 1e6 * 64 / 1e12
+        ach = ops / (ms * 1e-3) / 1e12
+        return {"kernel": "hbmm_umma_kernel/%s" % shape.name, "bound": "tensor", "achieved": ach,
+                "peak": peak, "unit": "TFLOP/s", "frac": ach / peak, "traffic": None,
+                "peak_source": "2 x %s bf16 GEMM peak (e4m3 operands)" % hbm_src,
+                "frac_of_popcount_roofline": ach / popc_peak, "popcount_roofline_tops": popc_peak}
     if kind == "hbwn_contraction":
         ops = 2.0 * M * N * K
-        # fp32 pipe: one sign-selected add per multiply-accumulate
-        peak = SM_COUNT * FMA_PER_CLK_SM * SM_MAX_MHZ * 1e6 * 2 / 1e12
-        return {"kernel": "hbwn_contraction/%s" % shape.name, "bound": "alu", "achieved": ops / (ms * 1e-3) / 1e12,
-                "peak": peak, "unit": "TOP/s", "frac": ops / (ms * 1e-3) / 1e12 / peak, "traffic": None,
-                "peak_source": "148 SMs x 128 fp32 lanes/clk x 1965 MHz x 2 ops"}
+        ach = ops / (ms * 1e-3) / 1e12
+        return {"kernel": "hbwn_umma_kernel/%s" % shape.name, "bound": "tensor", "achieved": ach,
+                "peak": bf16_tflops, "unit": "TFLOP/s", "frac": ach / bf16_tflops, "traffic": None,
+                "peak_source": "%s bf16 GEMM peak" % hbm_src}
     if kind == "front_end_pack":
         x_bytes = 4.0 * shape.B * shape.C * shape.H * shape.W
         lw = ((K + 31) // 32 + 3) // 4 * 4
@@ -397,15 +410,16 @@ def run_ours(args):
 
     # per-kernel durations for the roofline entry (same buffers, same launch configuration)
     brk = kernel_breakdown(torch, hbmm, layers, max(5, min(args.steps, 20)))
-    hbm_gbs, hbm_src = measured_peaks()
+    peaks = measured_peaks()
+    hbm_gbs, _, hbm_src = peaks
     totals = {k: sum(v) for k, v in brk.items()}
     dominant = max(totals, key=totals.get)
     li = int(np.argmax(brk[dominant]))
-    roof = roofline_for(dominant, li, shapes[li], brk[dominant][li], hbm_gbs, hbm_src)
+    roof = roofline_for(dominant, li, shapes[li], brk[dominant][li], peaks)
     roof["share_of_step"] = totals[dominant] / sum(totals.values())
     kernels = {}
     for kind, times in brk.items():
-        kernels[kind] = [dict(layer=s.name, ms=round(t, 5), **{k: v for k, v in roofline_for(kind, i, s, t, hbm_gbs, hbm_src).items()
+        kernels[kind] = [dict(layer=s.name, ms=round(t, 5), **{k: v for k, v in roofline_for(kind, i, s, t, peaks).items()
                                                                 if k in ("bound", "achieved", "peak", "unit", "frac")})
                          for i, (s, t) in enumerate(zip(shapes, times))]
 
@@ -423,12 +437,13 @@ def run_ours(args):
     line = {
         "metric": "hbmm_effective_binary_tops", "value": aggregate(ops_step, world, ms_step), "unit": "TOPS",
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u32+f32",
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
         "config": {
             "workload": "resnet18_conv3x3_b64_hbmm+hbwn_beta32",
             "layers": [dict(name=s.name, M=s.M, N=s.N, K=s.K) for s in shapes],
             "beta_a": BETA, "beta_w": BETA, "scale_dtype": "f32", "hbwn_activation_dtype": "bf16",
+            "tensor_operands": "sign bits as +-1 e4m3 (HBMM) / +-1 bf16 (HBWN), exact; fp32 accumulate and scales",
             "batch_per_gpu": 64, "parallelism": "replicas(batch-sharded)x%d" % world,
             "l2": "per-step inputs+outputs+workspaces (~0.9 GB) exceed the 126 MB L2; no explicit flush",
         },

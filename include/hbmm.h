@@ -45,12 +45,17 @@ typedef enum {
 
 typedef enum { HBMM_F32 = 0, HBMM_BF16 = 1 } hbmm_dtype;
 
-/* Which contraction kernel hbmm_gemm_ex runs for two packed operands. */
+/* Which contraction kernel hbmm_gemm_ex runs.  First meaning: two packed operands (HBMM); second:
+ * dense activations x packed weights (HBWN, beta_a == 1). */
 typedef enum {
-  HBMM_PATH_AUTO = 0,   /* the fastest path that supports the operands                                 */
-  HBMM_PATH_POPC = 1,   /* XOR + __popc on the integer pipe, fp32 group-scale epilogue in registers    */
-  HBMM_PATH_B1MMA = 2,  /* legacy mma.sync b1 (xor.popc) tensor instruction, beta multiple of 128      */
-  HBMM_PATH_TENSOR = 3  /* sign bits expanded to +-1 e4m3 in shared memory, tcgen05 group dots in TMEM  */
+  HBMM_PATH_AUTO = 0,   /* the fastest path that supports the operands (and has its workspace)         */
+  HBMM_PATH_POPC = 1,   /* XOR + __popc on the integer pipe, fp32 group-scale epilogue in registers;
+                           HBWN: weight sign XOR-ed into fp32 activations on the fp32 pipe              */
+  HBMM_PATH_B1MMA = 2,  /* legacy warp-level mma.sync: b1 xor.popc, beta multiple of 128;
+                           HBWN: bf16 mma.sync with per-group partial sums (bf16 activations only)      */
+  HBMM_PATH_TENSOR = 3  /* tcgen05 with TMEM accumulators: sign bits expanded to +-1 e4m3, group dots
+                           scaled in the epilogue; HBWN: bf16 activations x weights written as three
+                           bf16 pieces +-d_i (delta = d1 + d2 + d3), one accumulation over all of K     */
 } hbmm_path;
 
 /*
@@ -117,10 +122,11 @@ hbmm_status hbmm_quantize(const void *x, int32_t x_dtype, int64_t rows, int64_t 
                           const hbmm_operand *out, void *stream);
 
 /* Bytes of scratch hbmm_gemm wants for these operands (host pointer `bytes`).  The tensor-core
- * contraction keeps the weight operand there, expanded once per call into the tile layout its
- * kernel streams (about K bytes + K/2 bytes per weight row); 0 when no path needs scratch.
- * hbmm_gemm still works without it (workspace NULL or too small): it then runs the
- * integer-pipe path.  The workspace must be 16-byte aligned. */
+ * contractions keep the weight operand there, expanded once per call into the tile layout their
+ * kernels stream (HBMM: about 1.5 K bytes per weight row; HBWN: 6 K bytes per weight row, three
+ * bf16 pieces); 0 when no path needs scratch.  hbmm_gemm still works without it (workspace NULL
+ * or too small): it then runs the integer-pipe path (HBMM) or the warp-level kernels (HBWN).
+ * The workspace must be 16-byte aligned. */
 hbmm_status hbmm_gemm_workspace_bytes(const hbmm_operand *A, const hbmm_operand *W, size_t *bytes);
 
 /*
@@ -202,9 +208,10 @@ hbmm_status hbmm_conv_im2col_static(const void *x, int32_t x_dtype, const hbmm_c
                                     float *C_out, int64_t ldc, void *stream);
 
 /*
- * Device-side health word of the tensor-core contraction.  Its kernels never spin without a
+ * Device-side health word of the tensor-core contractions.  Their kernels never spin without a
  * limit: a wait on a barrier that does not complete in time records a code (1 producer, 2/3/4
- * MMA issue, 5 epilogue, 6 weight loader), makes the kernel drain and return, and leaves the output undefined.
+ * MMA issue, 5 epilogue, 6 weight loader; 100 + the same codes for the HBWN kernel), makes the
+ * kernel drain and return, and leaves the output undefined.
  * This call copies the word back (it synchronises the device) and returns HBMM_ERR_TIMEOUT when
  * it is non-zero, HBMM_OK otherwise.  code: host pointer, may be NULL.
  */

@@ -65,6 +65,14 @@ hbmm_status check_c(const float* C, int64_t ldc, int64_t N) {
 size_t tensor_workspace(const PackedView& a, const PackedView& w) {
   return gemm_tensor_supported(a, w) ? static_cast<size_t>(round_up(static_cast<int64_t>(gemm_tensor_workspace_bytes(a, w)), 256)) : 0;
 }
+size_t hbwn_workspace(const DenseView& a, const PackedView& w) {
+  return hbwn_umma_supported(a, w) ? static_cast<size_t>(round_up(static_cast<int64_t>(hbwn_umma_workspace_bytes(a, w)), 256)) : 0;
+}
+DenseView dense_view_of(const hbmm_operand* A) {
+  DenseView dv;
+  dv.data = A->dense; dv.rows = A->rows; dv.K = A->K; dv.ld = A->ld_dense; dv.bf16 = A->dense_dtype == HBMM_BF16;
+  return dv;
+}
 inline bool workspace_ok(const void* ws, size_t have, size_t need) {
   return need == 0 || (ws != nullptr && have >= need && (reinterpret_cast<uintptr_t>(ws) & 15u) == 0);
 }
@@ -81,11 +89,28 @@ hbmm_status gemm_checked(const hbmm_operand* A, const hbmm_operand* W, float* C,
       return HBMM_ERR_INVALID_ARG;
     if (A->K != W->K) return HBMM_ERR_INVALID_ARG;
     if ((st = check_c(C, ldc, W->rows)) != HBMM_OK) return st;
-    if (path == HBMM_PATH_B1MMA) return HBMM_ERR_UNSUPPORTED;
-    DenseView dv;
-    dv.data = A->dense; dv.rows = A->rows; dv.K = A->K; dv.ld = A->ld_dense; dv.bf16 = A->dense_dtype == HBMM_BF16;
-    return launch_hbwn(dv, view_of(W), C, ldc, path == HBMM_PATH_TENSOR ? 1 : (path == HBMM_PATH_POPC ? 2 : 0), stream) == cudaSuccess
-               ? HBMM_OK : HBMM_ERR_CUDA;
+    const DenseView dv = dense_view_of(A);
+    const PackedView w = view_of(W);
+    const bool umma = hbwn_umma_supported(dv, w) && workspace_ok(workspace, workspace_bytes, hbwn_workspace(dv, w));
+    cudaError_t e;
+    switch (path) {
+      case HBMM_PATH_POPC: e = launch_hbwn_select(dv, w, C, ldc, stream); break;
+      case HBMM_PATH_B1MMA:
+        if (!hbwn_mma_supported(dv, w)) return HBMM_ERR_UNSUPPORTED;
+        e = launch_hbwn_mma(dv, w, C, ldc, stream);
+        break;
+      case HBMM_PATH_TENSOR:
+        if (!hbwn_umma_supported(dv, w)) return HBMM_ERR_UNSUPPORTED;
+        if (!umma) return HBMM_ERR_WORKSPACE;
+        e = launch_hbwn_umma(dv, w, C, ldc, workspace, stream);
+        break;
+      default:
+        if (umma) e = launch_hbwn_umma(dv, w, C, ldc, workspace, stream);
+        else if (hbwn_mma_supported(dv, w)) e = launch_hbwn_mma(dv, w, C, ldc, stream);
+        else e = launch_hbwn_select(dv, w, C, ldc, stream);
+        break;
+    }
+    return e == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
   }
   if ((st = check_packed(A)) != HBMM_OK) return st;
   if (A->K != W->K) return HBMM_ERR_INVALID_ARG;
@@ -142,7 +167,11 @@ ConvLayout conv_layout(const ConvGeom& g, int32_t beta_a, int32_t scale_dtype, c
   if (beta_a == 1) {
     L.ld_dense = round_up(L.K, 8);
     L.operand_bytes = static_cast<size_t>(round_up(L.M * L.ld_dense * 2, 256));
-    L.total = L.operand_bytes;
+    // the tensor-core contraction's prepared weight pieces follow the bf16 rows
+    DenseView a;
+    a.data = nullptr; a.rows = L.M; a.K = L.K; a.ld = L.ld_dense; a.bf16 = 1;
+    L.gemm_bytes = (W && W->K == L.K) ? hbwn_workspace(a, view_of(W)) : 0;
+    L.total = L.operand_bytes + L.gemm_bytes;
   } else {
     L.ld_words = words_ld(L.K);
     L.ld_scales = scales_ld(L.K, beta_a, scale_dtype);
@@ -196,6 +225,9 @@ hbmm_status hbmm_gemm_workspace_bytes(const hbmm_operand* A, const hbmm_operand*
   if (A->beta >= 2 && W->beta >= 2 && check_packed(A, false) == HBMM_OK && check_packed(W, false) == HBMM_OK &&
       A->K == W->K && segments_compatible(A, W))
     *bytes = tensor_workspace(view_of(A), view_of(W));
+  else if (A->beta == 1 && W->beta >= 2 && A->dense && A->rows > 0 && A->K == W->K && A->ld_dense >= A->K &&
+           valid_dtype(A->dense_dtype) && check_packed(W, false) == HBMM_OK)
+    *bytes = hbwn_workspace(dense_view_of(A), view_of(W));
   return HBMM_OK;
 }
 
@@ -276,7 +308,9 @@ hbmm_status hbmm_conv_im2col(const void* x, int32_t x_dtype, const hbmm_conv_geo
 
 hbmm_status hbmm_last_device_error(int32_t* code) {
   int c = 0;
-  if (read_umma_error(&c) != cudaSuccess) return HBMM_ERR_CUDA;
+  int c2 = 0;
+  if (read_gemm_umma_error(&c) != cudaSuccess || read_hbwn_umma_error(&c2) != cudaSuccess) return HBMM_ERR_CUDA;
+  if (c == 0 && c2 != 0) c = 100 + c2;    // codes of the HBWN kernel are reported as 100 + code
   if (code) *code = c;
   return c == 0 ? HBMM_OK : HBMM_ERR_TIMEOUT;
 }

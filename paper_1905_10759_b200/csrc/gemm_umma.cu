@@ -32,12 +32,12 @@
 // drains and frees its TMEM before returning.
 #include <cuda_bf16.h>
 #include "kernels.h"
+#include "umma_common.cuh"
 
 namespace hbmm {
-
-__device__ int g_umma_error = 0;  // 0 = ok; otherwise the code of the first wait that gave up
-
 namespace {
+
+using namespace umma;
 
 constexpr int kEpilogueWarps = 8;                         // warpgroups 0 and 1
 constexpr int kProducerWarps = 4;                         // warpgroup 2: one A row per thread
@@ -48,10 +48,8 @@ constexpr int kThreads = 16 * 32;                         // 512: four warpgroup
 constexpr int kRegsEpilogue = 208;                        // 256 x 208 + 128 x 64 + 128 x 32 = 64 K registers
 constexpr int kRegsProducer = 64;
 constexpr int kRegsIssuer = 32;
-constexpr int TM = 128;
 constexpr int WPS = 4;            // K-words per stage
 constexpr int STAGES = 3;
-constexpr uint32_t kSpinLimit = 1u << 20;   // polls of a (hardware time-limited) try_wait
 
 struct Args {
   const uint32_t* a_bits; const void* a_scales;
@@ -70,140 +68,11 @@ __device__ __forceinline__ float load_scale(const void* s, int bf16, int64_t idx
   if (bf16) return __uint_as_float(static_cast<uint32_t>(__ldg(reinterpret_cast<const unsigned short*>(s) + idx)) << 16);
   return __ldg(reinterpret_cast<const float*>(s) + idx);
 }
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-
-// ---- mbarrier helpers (shared::cta)
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("{\n\t.reg .b64 st;\n\tmbarrier.arrive.shared::cta.b64 st, [%0];\n\t}" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-               : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  return ok != 0;
-}
-// The same on a precomputed shared-memory address (keeps the single-thread issue loops short).
-__device__ __forceinline__ bool mbar_try_wait_a(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ void umma_commit_a(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// Bounded wait.  Returns false when the limit expired or another thread aborted.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int code) {
-  for (uint32_t it = 0; it < kSpinLimit; it++) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
-  }
-  atomicCAS(&g_umma_error, 0, code);
-  *abort_flag = 1;
-  return false;
-}
-
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("{\n\t.reg .b64 st;\n\tmbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n\t}" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-// Asynchronous bulk copy global -> this CTA's shared memory (both 16-byte aligned, size a multiple of
-// 16); completion is counted in bytes on the mbarrier.  No multicast.
-__device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
-}
-
-// ---- tcgen05 helpers
-__device__ __forceinline__ bool mbar_wait_a(uint32_t bar, uint32_t parity, volatile int* abort_flag, int code) {
-  if (mbar_try_wait_a(bar, parity)) return true;
-  for (uint32_t it = 0; it < kSpinLimit; it++) {
-    if (mbar_try_wait_a(bar, parity)) return true;
-    if (*abort_flag) return false;
-  }
-  atomicCAS(&g_umma_error, 0, code);
-  *abort_flag = 1;
-  return false;
-}
-__device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t cols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols));
-}
-__device__ __forceinline__ void tmem_relinquish() { asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::); }
-__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols));
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void umma_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-// D[tmem] (+)= A[smem desc] * B[smem desc]^T, 128 x N x 32, e4m3 operands, fp32 accumulate.
-__device__ __forceinline__ void umma_f8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t (&v)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-      : "r"(addr));
-}
-__device__ __forceinline__ void tmem_ld16(uint32_t addr, uint32_t (&v)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-      : "r"(addr));
-}
-__device__ __forceinline__ void tmem_ld_piece(uint32_t addr, uint32_t (&v)[32]) { tmem_ld32(addr, v); }
-__device__ __forceinline__ void tmem_ld_piece(uint32_t addr, uint32_t (&v)[16]) { tmem_ld16(addr, v); }
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-template <int R> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(R)); }
-template <int R> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(R)); }
-
-// Two fp32 lanes per instruction (halves the issue slots of the scale epilogue).
-__device__ __forceinline__ uint64_t pack2(uint32_t lo, uint32_t hi) {
-  uint64_t r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
-  return r;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
-  uint64_t r;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-  return r;
-}
-// D[tmem] = A[smem desc] * B[smem desc]^T, 128 x N x 16, bf16 operands, fp32 result (overwrites).
-__device__ __forceinline__ void umma_bf16_overwrite(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, 0, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc) : "memory");
-}
-
 // Four sign bits (in bits 0..3 or 4..7 of `v`, selected by the multiplier) -> four e4m3 bytes:
 // the multiply copies bit i to bit 8*i+7, the sign position of byte i; 0xB8 = -1.0, 0x38 = +1.0.
 __device__ __forceinline__ uint32_t signs_lo(uint32_t v) { return (((v & 0x0Fu) * 0x10204080u) & 0x80808080u) ^ 0xB8B8B8B8u; }
 __device__ __forceinline__ uint32_t signs_hi(uint32_t v) { return (((v & 0xF0u) * 0x01020408u) & 0x80808080u) ^ 0xB8B8B8B8u; }
 
-// Operand tiles in shared memory use the 128-byte-swizzled K-major layout of the tensor core: a row is
-// 128 contiguous bytes (the four K-words of a stage, 32 bytes each), rows follow each other, and the
-// 16-byte piece c of row r is stored at piece position c ^ (r % 8).  A tile starts on a 1024-byte
-// boundary; the instruction for word slot q reads from byte offset 32*q of the rows.
-__device__ __forceinline__ unsigned char* swz(unsigned char* tile, int row, int piece) {
-  return tile + row * 128 + ((piece ^ (row & 7)) << 4);
-}
 // Four packed K-words of one tile row -> 4 x 32 e4m3 bytes (pieces 0..7 of the row).
 __device__ __forceinline__ void expand_words(unsigned char* tile, int row, const uint4& w4) {
   const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
@@ -234,25 +103,6 @@ __device__ __forceinline__ uint4 scale_row(float v) {
   if (IS_B) return make_uint4(h1 | (h2 << 16), h1 | (h2 << 16), h3 | (h1 << 16), 0u);
   return make_uint4(h1 | (h1 << 16), h2 | (h2 << 16), h1 | (h3 << 16), 0u);
 }
-
-// Shared-memory descriptor of a K-major, 128-byte-swizzled operand: start address, stride between
-// 8-row groups = 1024 bytes, descriptor version 1, layout type 2 (128-byte swizzle); the leading
-// offset is not used by this layout.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
-  uint64_t d = 0;
-  d |= static_cast<uint64_t>((addr >> 4) & 0x3FFF);
-  d |= static_cast<uint64_t>(1) << 16;
-  d |= static_cast<uint64_t>(1024 >> 4) << 32;
-  d |= static_cast<uint64_t>(1) << 46;
-  d |= static_cast<uint64_t>(2) << 61;
-  return d;
-}
-// Instruction descriptors: fp32 accumulator, both operands K-major, M = 128, N = n.
-__host__ __device__ constexpr uint32_t instr_desc(int n, uint32_t ab_format) {
-  return (1u << 4) | (ab_format << 7) | (ab_format << 10) | (static_cast<uint32_t>(n >> 3) << 17) |
-         (static_cast<uint32_t>(TM >> 4) << 24);
-}
-constexpr uint32_t kFmtE4M3 = 0, kFmtBF16 = 1;
 
 template <int TN>
 struct Smem {
@@ -636,8 +486,8 @@ cudaError_t launch_gemm_tensor(const PackedView& A, const PackedView& W, float* 
   return g.N <= 64 ? launch_umma<64>(g, workspace, stream) : launch_umma<128>(g, workspace, stream);
 }
 
-cudaError_t read_umma_error(int* code) {
-  return cudaMemcpyFromSymbol(code, g_umma_error, sizeof(int));
+cudaError_t read_gemm_umma_error(int* code) {
+  return cudaMemcpyFromSymbol(code, umma::g_error_word, sizeof(int));
 }
 
 }  // namespace hbmm

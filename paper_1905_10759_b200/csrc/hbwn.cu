@@ -128,15 +128,4 @@ cudaError_t launch_hbwn_select(const DenseView& A, const PackedView& W, float* C
   return cudaGetLastError();
 }
 
-bool hbwn_mma_supported(const DenseView& A, const PackedView& W);
-cudaError_t launch_hbwn_mma(const DenseView& A, const PackedView& W, float* C, int64_t ldc, cudaStream_t stream);
-
-// kind: 0 = fastest available, 1 = tensor-core path (falls back when it cannot run the operands),
-// 2 = sign-select on the fp32 pipe.
-cudaError_t launch_hbwn(const DenseView& A, const PackedView& W, float* C, int64_t ldc, int kind,
-                        cudaStream_t stream) {
-  if (kind != 2 && hbwn_mma_supported(A, W)) return launch_hbwn_mma(A, W, C, ldc, stream);
-  return launch_hbwn_select(A, W, C, ldc, stream);
-}
-
 }  // namespace hbmm

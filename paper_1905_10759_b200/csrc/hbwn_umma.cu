@@ -1,0 +1,343 @@
+// HBWN contraction on the 5th-generation tensor cores: bf16 activations x Hadamard-binary weights,
+//   C[m,n] = sum_k A[m,k] * (deltaW[n, k/beta] * s(W[n,k])).
+// The binarized weight W~ = deltaW (.) Sign(W) (Eq. 2) is written as the sum of three bf16 matrices:
+// each fp32 group scale is split as delta = d1 + d2 + d3 (bf16 pieces, 24 significant bits together,
+// every remainder exact in fp32) and piece i of W~ is +-d_i.  A bf16 activation times a bf16 piece
+// is exact in fp32, so C = A W1^T + A W2^T + A W3^T accumulated in fp32 tensor memory reproduces the
+// per-group full-precision scaling to 2^-26 of each weight -- with no per-group epilogue at all: the
+// whole K walk of a tile is one accumulation in TMEM and the epilogue runs once per tile.
+// The three pieces of a 64-column tile are stacked along N, so one 128 x 192 x 16 MMA per K-step
+// forms all three products (the instruction costs about the same for any N <= 128, so stacking is
+// nearly three times cheaper than three accumulating MMAs); the epilogue adds the three column blocks.
+//
+// One persistent CTA per SM.  Stage = 64 K-elements: the A tile (128 rows x 128 bytes) arrives by
+// one tiled tensor copy (TMA, 128-byte swizzle, zeros past M and K), the three weight pieces of the
+// stage (192 rows) by one bulk copy from the workspace, where a small kernel has laid them out once
+// per call.  All operand tiles use the 128-byte-swizzled K-major layout.
+//   warps 0-3 : epilogue (TMEM lanes 32*w.., three blocks of TN columns, once per tile)
+//   warp  4   : one thread issues both copies of every stage
+//   warp  5   : TMEM allocation and the MMA-issuing thread
+// Waits are bounded as in the packed kernel (error word, CTA-wide abort flag, orderly teardown).
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include "kernels.h"
+#include "umma_common.cuh"
+
+namespace hbmm {
+namespace {
+
+using namespace umma;
+
+constexpr int kThreads = 6 * 32;
+constexpr int kLoaderWarp = 4, kMmaWarp = 5;
+constexpr int KB = 64;            // K elements per stage (128 bytes of bf16 per row)
+constexpr int STAGES = 5;
+
+struct Args {
+  const __nv_bfloat16* a; int64_t lda;
+  const uint32_t* w_bits; const void* w_scales; int64_t ldw_w, ldw_s; int32_t w_bf16;
+  float* C; int64_t ldc; int32_t c_vec;   // c_vec: rows of C allow 16-byte stores
+  int64_t M, N, K, Gw;
+  int64_t beta;                   // weight group length (>= K: one group per row)
+  const unsigned char* w_prep;    // [n tile][k block][3 pieces][TN rows x 128 bytes]
+};
+
+__device__ __forceinline__ float load_scale(const void* s, int bf16, int64_t idx) {
+  if (bf16) return __uint_as_float(static_cast<uint32_t>(__ldg(reinterpret_cast<const unsigned short*>(s) + idx)) << 16);
+  return __ldg(reinterpret_cast<const float*>(s) + idx);
+}
+
+template <int TN>
+struct Smem {
+  static constexpr int A_STAGE = TM * 128;
+  static constexpr int B_PIECE = TN * 128;
+  static constexpr int B_STAGE = 3 * B_PIECE;
+  static constexpr int OFF_A = 0;
+  static constexpr int OFF_B = OFF_A + STAGES * A_STAGE;
+  static constexpr int OFF_BAR = OFF_B + STAGES * B_STAGE;
+  static constexpr int NBAR = 2 * STAGES + 4 + 1;      // full, empty, tfull[2], tempty[2], drain
+  static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
+  static constexpr int USED = OFF_MISC + 16;
+  static constexpr int BYTES = USED > 120 * 1024 ? USED : 120 * 1024;   // one CTA per SM
+  static constexpr int NST = 3 * TN;                   // MMA N: the three pieces side by side
+  static constexpr int TMEM_COLS = 512;                // two accumulator buffers of NST columns
+  static_assert(NST <= 256 && NST % 16 == 0 && 2 * NST <= TMEM_COLS, "one MMA covers the stacked pieces");
+};
+
+// Writes the three bf16 pieces of W~ for one (column tile, k block): thread = (row, 16-byte piece of
+// 8 consecutive k).  Element k of row n: +-piece_i(deltaW[n, k / beta]), zero past K and past N.
+template <int TN>
+__global__ void __launch_bounds__(256)
+prepare_w_pieces_kernel(const Args g, unsigned char* __restrict__ out) {
+  using S = Smem<TN>;
+  const int64_t kb = blockIdx.x, tile_n = blockIdx.y;
+  const int64_t n_kb = (g.K + KB - 1) / KB;
+  unsigned char* base = out + (tile_n * n_kb + kb) * S::B_STAGE;
+  for (int item = threadIdx.x; item < TN * 8; item += 256) {
+    const int row = item >> 3, piece = item & 7;
+    const int64_t n = tile_n * TN + row, k0 = kb * KB + piece * 8;
+    uint32_t o[3][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}, {0, 0, 0, 0}};
+    if (n < g.N && k0 < g.K) {
+      const uint32_t word = __ldg(g.w_bits + n * g.ldw_w + (k0 >> 5));
+#pragma unroll
+      for (int e = 0; e < 8; e++) {
+        const int64_t k = k0 + e;
+        if (k < g.K) {
+          const int64_t grp = g.beta >= g.K ? 0 : k / g.beta;
+          const float d = load_scale(g.w_scales, g.w_bf16, n * g.ldw_s + grp);
+          const __nv_bfloat16 b1 = __float2bfloat16_rn(d);
+          const float r1 = d - __bfloat162float(b1);
+          const __nv_bfloat16 b2 = __float2bfloat16_rn(r1);
+          const __nv_bfloat16 b3 = __float2bfloat16_rn(r1 - __bfloat162float(b2));
+          const uint32_t neg = ((word >> (k & 31)) & 1u) ? 0u : 0x8000u;   // bit 0 <=> Sign = -1
+          const uint32_t h[3] = {__bfloat16_as_ushort(b1) ^ neg, __bfloat16_as_ushort(b2) ^ neg, __bfloat16_as_ushort(b3) ^ neg};
+#pragma unroll
+          for (int i = 0; i < 3; i++) o[i][e >> 1] |= h[i] << ((e & 1) * 16);
+        }
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 3; i++)
+      *reinterpret_cast<uint4*>(swz(base + i * S::B_PIECE, row, piece)) = make_uint4(o[i][0], o[i][1], o[i][2], o[i][3]);
+  }
+}
+
+template <int TN>
+__global__ void __launch_bounds__(kThreads, 1)
+hbwn_umma_kernel(const Args g, const __grid_constant__ CUtensorMap a_map) {
+  using S = Smem<TN>;
+  extern __shared__ __align__(1024) unsigned char smem[];
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + S::OFF_BAR);
+  uint64_t* empty = full + STAGES;
+  uint64_t* tfull = empty + STAGES;
+  uint64_t* tempty = tfull + 2;
+  uint64_t* drain = tempty + 2;
+  uint32_t* tmem_base_ptr = reinterpret_cast<uint32_t*>(smem + S::OFF_MISC);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + S::OFF_MISC + 4);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int64_t tiles_n = (g.N + TN - 1) / TN, tiles_m = (g.M + TM - 1) / TM;
+  const int64_t n_tiles = tiles_m * tiles_n;
+  const int64_t n_kb = (g.K + KB - 1) / KB;                 // stages per tile
+  const int64_t my_tiles = blockIdx.x < n_tiles ? (n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+  const int64_t total = my_tiles * n_kb;                    // stages this CTA walks
+
+  if (tid == 0) {
+    for (int s = 0; s < STAGES; s++) {
+      mbar_init(&full[s], 1);           // the loader's expect_tx arrival; the copies complete the bytes
+      mbar_init(&empty[s], 1);          // MMA commit
+    }
+    for (int b = 0; b < 2; b++) { mbar_init(&tfull[b], 1); mbar_init(&tempty[b], 4); }
+    mbar_init(drain, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == kMmaWarp) {
+    tmem_alloc(tmem_base_ptr, S::TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_base_ptr;
+
+  if (warp == kLoaderWarp) {
+    // =========================== loader ===========================
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&a_map) : "memory");
+      for (int64_t gs = 0; gs < total; gs++) {
+        const int s = static_cast<int>(gs % STAGES);
+        if (gs >= STAGES && !mbar_wait(&empty[s], static_cast<uint32_t>(((gs / STAGES) & 1) ^ 1), abort_flag, 1)) break;
+        const int64_t tile = blockIdx.x + (gs / n_kb) * gridDim.x, kb = gs % n_kb;
+        const unsigned char* src = g.w_prep + ((tile % tiles_n) * n_kb + kb) * S::B_STAGE;
+        mbar_arrive_expect_tx(&full[s], S::A_STAGE + S::B_STAGE);
+        // x = kb * 64 elements = a multiple of 128 bytes; rows past M and columns past K are zero-filled
+        tma_load_2d(smem + S::OFF_A + s * S::A_STAGE, &a_map, static_cast<int32_t>(kb * KB),
+                    static_cast<int32_t>((tile / tiles_n) * TM), &full[s]);
+        bulk_copy_g2s(smem + S::OFF_B + s * S::B_STAGE, src, S::B_STAGE, &full[s]);
+      }
+    }
+    __syncwarp();
+  } else if (warp == kMmaWarp) {
+    // =========================== MMA issuer ===========================
+    if (lane == 0) {
+      constexpr uint32_t idesc = instr_desc(S::NST, kFmtBF16);
+      const uint64_t da0 = smem_desc(smem_u32(smem + S::OFF_A)), db0 = smem_desc(smem_u32(smem + S::OFF_B));
+      const uint64_t da_hi = da0 & 0xFFFFFFFF00000000ull, db_hi = db0 & 0xFFFFFFFF00000000ull;
+      const uint32_t da_lo = static_cast<uint32_t>(da0), db_lo = static_cast<uint32_t>(db0);
+      const uint32_t full_a = smem_u32(full), empty_a = smem_u32(empty), tfull_a = smem_u32(tfull), tempty_a = smem_u32(tempty);
+      uint32_t s = 0, full_par = 0;
+      bool ok = true;
+      for (int64_t ti = 0; ti < my_tiles && ok; ti++) {
+        const uint32_t buf = static_cast<uint32_t>(ti & 1);
+        if (ti >= 2) {      // the epilogue must have drained this accumulator (used by tile ti - 2)
+          if (!mbar_wait_a(tempty_a + buf * 8, static_cast<uint32_t>(((ti >> 1) & 1) ^ 1), abort_flag, 3)) { ok = false; break; }
+          tc_fence_after();
+        }
+        const uint32_t d_tmem = tmem_base + buf * S::NST;
+        for (int64_t kb = 0; kb < n_kb; kb++) {
+          if (!mbar_wait_a(full_a + s * 8, full_par, abort_flag, 2)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_lo = da_lo + s * (S::A_STAGE >> 4), b_lo = db_lo + s * (S::B_STAGE >> 4);
+#pragma unroll
+          for (int ks = 0; ks < KB / 16; ks++)          // 16 K-elements = 32 bytes along the swizzled rows
+            umma_bf16(d_tmem, da_hi | (a_lo + ks * 2), db_hi | (b_lo + ks * 2), idesc, (kb | ks) != 0 ? 1u : 0u);
+          umma_commit_a(empty_a + s * 8);
+          if (++s == STAGES) { s = 0; full_par ^= 1; }
+        }
+        if (ok) umma_commit_a(tfull_a + buf * 8);
+      }
+      umma_commit(drain);
+      mbar_wait(drain, 0, abort_flag, 4);
+    }
+    __syncwarp();
+  } else if (warp < 4) {
+    // =========================== epilogue ===========================
+    const int row = warp * 32 + lane;
+    const uint32_t t_lane = static_cast<uint32_t>(warp * 32) << 16;
+    for (int64_t ti = 0; ti < my_tiles; ti++) {
+      const uint32_t buf = static_cast<uint32_t>(ti & 1);
+      if (!mbar_wait(&tfull[buf], static_cast<uint32_t>((ti >> 1) & 1), abort_flag, 5)) break;
+      tc_fence_after();
+      const int64_t tile = blockIdx.x + ti * gridDim.x;
+      const int64_t m = (tile / tiles_n) * TM + row, nb = (tile % tiles_n) * TN;
+      float* dst = g.C + m * g.ldc + nb;
+#pragma unroll
+      for (int c = 0; c < TN / 32; c++) {
+        uint32_t v1[32], v2[32], v3[32];
+        const uint32_t t_addr = tmem_base + t_lane + buf * S::NST + c * 32;
+        tmem_ld32(t_addr, v1);
+        tmem_ld32(t_addr + TN, v2);
+        tmem_ld32(t_addr + 2 * TN, v3);
+        tmem_ld_wait();
+        if (m < g.M) {
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            float o[4];
+#pragma unroll
+            for (int e = 0; e < 4; e++)      // smallest pieces first
+              o[e] = __uint_as_float(v1[j + e]) + (__uint_as_float(v2[j + e]) + __uint_as_float(v3[j + e]));
+            const int64_t n = nb + c * 32 + j;
+            if (g.c_vec && n + 3 < g.N)
+              *reinterpret_cast<float4*>(dst + c * 32 + j) = make_float4(o[0], o[1], o[2], o[3]);
+            else
+              for (int e = 0; e < 4; e++)
+                if (n + e < g.N) dst[c * 32 + j + e] = o[e];
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tempty[buf]);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == kMmaWarp) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, S::TMEM_COLS);
+  }
+}
+
+Args make_args(const DenseView& A, const PackedView& W, float* C, int64_t ldc) {
+  Args g;
+  g.a = reinterpret_cast<const __nv_bfloat16*>(A.data); g.lda = A.ld;
+  g.w_bits = W.bits; g.w_scales = W.scales; g.ldw_w = W.ld_words; g.ldw_s = W.ld_scales; g.w_bf16 = W.scale_bf16;
+  g.C = C; g.ldc = ldc;
+  g.c_vec = (reinterpret_cast<uintptr_t>(C) % 16 == 0 && ldc % 4 == 0) ? 1 : 0;
+  g.M = A.rows; g.N = W.rows; g.K = A.K;
+  g.Gw = num_groups(W.K, W.beta);
+  g.beta = W.beta;
+  g.w_prep = nullptr;
+  return g;
+}
+
+template <int TN>
+size_t prep_bytes(const Args& g) {
+  return static_cast<size_t>(((g.N + TN - 1) / TN) * ((g.K + KB - 1) / KB)) * Smem<TN>::B_STAGE;
+}
+
+// cuTensorMapEncodeTiled is a host-only driver routine; it is looked up through the runtime so the
+// library does not link against the driver.  nullptr when the driver does not offer it.
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+// Tensor map of the activation matrix: bf16 [M, K] with row pitch lda, boxes of 64 x 128 elements
+// (one 128-byte-swizzled stage tile), zeros outside the matrix.
+bool make_a_map(const Args& g, CUtensorMap* map) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(g.K), static_cast<cuuint64_t>(g.M)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(g.lda) * 2};
+  const cuuint32_t box[2] = {KB, TM};
+  const cuuint32_t elem[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(g.a), dims, strides, box, elem,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int TN>
+cudaError_t launch(Args g, void* workspace, cudaStream_t stream) {
+  using S = Smem<TN>;
+  CUtensorMap a_map;
+  if (!make_a_map(g, &a_map)) return cudaErrorNotSupported;
+  static bool configured = false;
+  static int sms = 0;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(hbwn_umma_kernel<TN>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::BYTES);
+    if (e != cudaSuccess) return e;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    configured = true;
+  }
+  const int64_t tiles_n = (g.N + TN - 1) / TN, n_kb = (g.K + KB - 1) / KB;
+  dim3 pgrid(static_cast<unsigned>(n_kb), static_cast<unsigned>(tiles_n));
+  prepare_w_pieces_kernel<TN><<<pgrid, 256, 0, stream>>>(g, static_cast<unsigned char*>(workspace));
+  g.w_prep = static_cast<const unsigned char*>(workspace);
+  const int64_t tiles = ((g.M + TM - 1) / TM) * tiles_n;
+  const unsigned grid = static_cast<unsigned>(tiles < sms ? tiles : sms);
+  hbwn_umma_kernel<TN><<<grid, kThreads, S::BYTES, stream>>>(g, a_map);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+// bf16 activations whose rows start on 16-byte boundaries (what a tensor map can describe: extents
+// below 2^32, pitch below 2^40 bytes); any weight group size.
+bool hbwn_umma_supported(const DenseView& A, const PackedView& W) {
+  (void)W;
+  return A.bf16 && reinterpret_cast<uintptr_t>(A.data) % 16 == 0 && (A.ld * 2) % 16 == 0 &&
+         A.rows < (int64_t{1} << 31) && A.K < (int64_t{1} << 31) && A.ld * 2 < (int64_t{1} << 40) &&
+         encode_tiled_fn() != nullptr;
+}
+
+size_t hbwn_umma_workspace_bytes(const DenseView& A, const PackedView& W) {
+  const Args g = make_args(A, W, nullptr, 0);
+  return prep_bytes<64>(g);
+}
+
+cudaError_t launch_hbwn_umma(const DenseView& A, const PackedView& W, float* C, int64_t ldc, void* workspace,
+                             cudaStream_t stream) {
+  const Args g = make_args(A, W, C, ldc);
+  return launch<64>(g, workspace, stream);
+}
+
+cudaError_t read_hbwn_umma_error(int* code) {
+  return cudaMemcpyFromSymbol(code, umma::g_error_word, sizeof(int));
+}
+
+}  // namespace hbmm

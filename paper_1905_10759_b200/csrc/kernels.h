@@ -49,17 +49,27 @@ cudaError_t launch_partials_b1(const PackedView& A, const PackedView& W, int32_t
                                cudaStream_t stream);
 
 // Packed x packed contraction with +-1 e4m3 operands on the tensor cores (tcgen05 / TMEM).
-// read_umma_error copies the device-side error word (0 = no bounded wait ever expired); it synchronises.
-cudaError_t read_umma_error(int* code);
+// read_*_umma_error copies a kernel family's device-side error word (0 = no bounded wait ever
+// expired); it synchronises.
+cudaError_t read_gemm_umma_error(int* code);
+cudaError_t read_hbwn_umma_error(int* code);
 bool gemm_tensor_supported(const PackedView& A, const PackedView& W);
 size_t gemm_tensor_workspace_bytes(const PackedView& A, const PackedView& W);
 cudaError_t launch_gemm_tensor(const PackedView& A, const PackedView& W, float* C, int64_t ldc, void* workspace,
                                cudaStream_t stream);
 
-// Dense x packed contraction (HBWN).
-// kind = 0: fastest available; 1: bf16 tensor-core path (falls back when unsupported); 2: sign-select.
-cudaError_t launch_hbwn(const DenseView& A, const PackedView& W, float* C, int64_t ldc, int kind,
-                        cudaStream_t stream);
+// Dense x packed contraction (HBWN), three kernels:
+//   select : sign bit XOR-ed into fp32 activations on the fp32 pipe (any dense dtype);
+//   mma    : legacy warp-level bf16 mma.sync with per-group partial sums (bf16 activations);
+//   umma   : tcgen05, weights as three stacked bf16 pieces prepared in a workspace (bf16 activations,
+//            16-byte aligned rows).
+cudaError_t launch_hbwn_select(const DenseView& A, const PackedView& W, float* C, int64_t ldc, cudaStream_t stream);
+bool hbwn_mma_supported(const DenseView& A, const PackedView& W);
+cudaError_t launch_hbwn_mma(const DenseView& A, const PackedView& W, float* C, int64_t ldc, cudaStream_t stream);
+bool hbwn_umma_supported(const DenseView& A, const PackedView& W);
+size_t hbwn_umma_workspace_bytes(const DenseView& A, const PackedView& W);
+cudaError_t launch_hbwn_umma(const DenseView& A, const PackedView& W, float* C, int64_t ldc, void* workspace,
+                             cudaStream_t stream);
 
 // im2col gather fused with Hadamard binarization (packed output), and bf16 dense gather.
 cudaError_t launch_im2col_quantize(const void* x, int x_bf16, const ConvGeom& g, int32_t beta,

@@ -243,10 +243,39 @@ def test_hbwn_matches_oracle(hb, M, N, K, bw, abf16):
         ad = ad.to(torch.bfloat16)
     rtol = _hbwn_rtol(gu, K, bw)
     assert rtol < RTOL_BF16
-    for path in (hb.PATH_AUTO, hb.PATH_TENSOR, hb.PATH_POPC):   # POPC selects the fp32 sign-select kernel
-        C = torch.full((M, (N + 3) // 4 * 4), float("nan"), device="cuda")
-        hb.gemm_ex(hb.wrap_dense(ad), W, C, path)
-        gu.assert_close_rel_absref(C.cpu().numpy()[:, :N], c_ref, absref, rtol, "hbwn path %d" % path)
+    A = hb.wrap_dense(ad)
+    ws = _gemm_ws(hb, A, W)
+    ran = 0
+    # TENSOR: tcgen05 kernel; B1MMA: warp-level bf16 mma.sync kernel; POPC: fp32 sign-select kernel
+    for path, wsp in ((hb.PATH_AUTO, ws), (hb.PATH_AUTO, None), (hb.PATH_TENSOR, ws), (hb.PATH_B1MMA, None),
+                      (hb.PATH_POPC, None)):
+        C = torch.full((M, (N + 3) // 4 * 4 + 4), float("nan"), device="cuda")
+        try:
+            hb.gemm_ex(A, W, C, path, wsp)
+        except hb.HbmmError as e:
+            # the two tensor-core kernels take bf16 activations whose rows start on 16-byte boundaries
+            assert e.status == hb.ERR_UNSUPPORTED and path in (hb.PATH_TENSOR, hb.PATH_B1MMA)
+            if path == hb.PATH_TENSOR:
+                assert not abf16 or K % 8 != 0
+            continue
+        ran += 1
+        out = C.cpu().numpy()
+        assert np.isnan(out[:, N:]).all()
+        gu.assert_close_rel_absref(out[:, :N], c_ref, absref, rtol, "hbwn path %d" % path)
+    assert ran >= (4 if abf16 and K % 8 == 0 else 3)
+
+
+def test_hbwn_tensor_path_needs_its_workspace(hb):
+    gu = _gu()
+    M, N, K = 64, 64, 128
+    _, a = inputs.as_bf16(inputs.normal((M, K), 61))
+    W, dw, sw = gu.oracle_operand(inputs.he_normal(N, K, 62), 32)
+    A = hb.wrap_dense(torch.from_numpy(a).cuda().to(torch.bfloat16))
+    assert hb.gemm_workspace_bytes(A, W) > 0
+    C = torch.empty((M, N), device="cuda")
+    with pytest.raises(hb.HbmmError) as e:
+        hb.gemm_ex(A, W, C, hb.PATH_TENSOR)
+    assert e.value.status == hb.ERR_WORKSPACE
 
 
 # ------------------------------------------------------------------ convolution front end
