@@ -157,6 +157,8 @@ hbmm_status check_geom(const hbmm_conv_geom* g, ConvGeom* out) {
 
 struct ConvLayout {
   int64_t M, K, ld_words, ld_scales, ld_dense;
+  bool implicit;     // beta_a == 1 only: NHWC copy + im2col-mode tensor copies instead of the im2col matrix
+  int32_t Cp;        // channel pitch of that copy
   size_t bits_bytes, scales_bytes, operand_bytes, gemm_bytes, total;
 };
 
@@ -164,7 +166,13 @@ ConvLayout conv_layout(const ConvGeom& g, int32_t beta_a, int32_t scale_dtype, c
   ConvLayout L{};
   L.M = static_cast<int64_t>(g.B) * g.Ho * g.Wo;
   L.K = static_cast<int64_t>(g.C) * g.kh * g.kw;
-  if (beta_a == 1) {
+  if (beta_a == 1 && W && W->K == L.K && hbwn_umma_conv_supported(g, view_of(W))) {
+    L.implicit = true;
+    L.Cp = static_cast<int32_t>(round_up(g.C, 8));
+    L.operand_bytes = static_cast<size_t>(round_up(static_cast<int64_t>(g.B) * g.H * g.W * L.Cp * 2, 256));
+    L.gemm_bytes = static_cast<size_t>(round_up(static_cast<int64_t>(hbwn_umma_conv_workspace_bytes(g, view_of(W))), 256));
+    L.total = L.operand_bytes + L.gemm_bytes;
+  } else if (beta_a == 1) {
     L.ld_dense = round_up(L.K, 8);
     L.operand_bytes = static_cast<size_t>(round_up(L.M * L.ld_dense * 2, 256));
     // the tensor-core contraction's prepared weight pieces follow the bf16 rows
@@ -290,6 +298,11 @@ hbmm_status hbmm_conv_im2col(const void* x, int32_t x_dtype, const hbmm_conv_geo
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   hbmm_operand A{};
   A.rows = L.M; A.K = L.K; A.beta = beta_a; A.scale_dtype = a_scale_dtype;
+  if (beta_a == 1 && L.implicit) {
+    if (launch_nchw_to_nhwc_bf16(x, x_dtype == HBMM_BF16, cg, workspace, L.Cp, s) != cudaSuccess) return HBMM_ERR_CUDA;
+    return launch_hbwn_umma_conv(workspace, L.Cp, cg, view_of(W), C_out, ldc, static_cast<char*>(workspace) + L.operand_bytes,
+                                 s) == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
+  }
   if (beta_a == 1) {
     if (launch_im2col_bf16(x, x_dtype == HBMM_BF16, cg, workspace, L.ld_dense, s) != cudaSuccess) return HBMM_ERR_CUDA;
     A.dense = workspace; A.ld_dense = L.ld_dense; A.dense_dtype = HBMM_BF16;

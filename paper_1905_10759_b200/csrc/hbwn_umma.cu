@@ -40,6 +40,14 @@ struct Args {
   int64_t M, N, K, Gw;
   int64_t beta;                   // weight group length (>= K: one group per row)
   const unsigned char* w_prep;    // [n tile][k block][3 pieces][TN rows x 128 bytes]
+  int64_t n_kb;                   // stages (K blocks of 64) per tile
+  // Convolution mode (conv != 0): A is the implicit im2col matrix of an NHWC bf16 image; K block
+  // kb = (filter tap, block of 64 channels), i.e. the K axis is walked tap-major.  Any one-to-one
+  // reordering of K leaves the product unchanged as long as both operands use it: the weight pieces
+  // are laid out in the same order, each element still scaled by the group of its original index
+  // k = c * taps + tap (channel slowest, Section 3.1.1).
+  int32_t conv, taps, kw, cblocks, Cin;
+  int32_t HoWo, Wo, sh, sw, ph, pw;
 };
 
 __device__ __forceinline__ float load_scale(const void* s, int bf16, int64_t idx) {
@@ -65,24 +73,29 @@ struct Smem {
 };
 
 // Writes the three bf16 pieces of W~ for one (column tile, k block): thread = (row, 16-byte piece of
-// 8 consecutive k).  Element k of row n: +-piece_i(deltaW[n, k / beta]), zero past K and past N.
+// 8 consecutive stage columns).  Stage column q of block kb is element k = kb * 64 + q of the weight
+// row (plain mode) or channel c = cb * 64 + q at filter tap t, k = c * taps + t (convolution mode,
+// kb = t * cblocks + cb).  The element is +-piece_i(deltaW[n, k / beta]); zero past K / C and past N.
 template <int TN>
 __global__ void __launch_bounds__(256)
 prepare_w_pieces_kernel(const Args g, unsigned char* __restrict__ out) {
   using S = Smem<TN>;
   const int64_t kb = blockIdx.x, tile_n = blockIdx.y;
-  const int64_t n_kb = (g.K + KB - 1) / KB;
-  unsigned char* base = out + (tile_n * n_kb + kb) * S::B_STAGE;
+  unsigned char* base = out + (tile_n * g.n_kb + kb) * S::B_STAGE;
+  const int64_t tap = g.conv ? kb / g.cblocks : 0;
+  const int64_t q0 = (g.conv ? kb - tap * g.cblocks : kb) * KB;     // first channel / element of the block
+  const int64_t q_end = g.conv ? g.Cin : g.K, k_mul = g.conv ? g.taps : 1;
   for (int item = threadIdx.x; item < TN * 8; item += 256) {
     const int row = item >> 3, piece = item & 7;
-    const int64_t n = tile_n * TN + row, k0 = kb * KB + piece * 8;
+    const int64_t n = tile_n * TN + row;
     uint32_t o[3][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}, {0, 0, 0, 0}};
-    if (n < g.N && k0 < g.K) {
-      const uint32_t word = __ldg(g.w_bits + n * g.ldw_w + (k0 >> 5));
+    if (n < g.N) {
 #pragma unroll
       for (int e = 0; e < 8; e++) {
-        const int64_t k = k0 + e;
-        if (k < g.K) {
+        const int64_t q = q0 + piece * 8 + e;
+        if (q < q_end) {
+          const int64_t k = q * k_mul + tap;
+          const uint32_t word = __ldg(g.w_bits + n * g.ldw_w + (k >> 5));
           const int64_t grp = g.beta >= g.K ? 0 : k / g.beta;
           const float d = load_scale(g.w_scales, g.w_bf16, n * g.ldw_s + grp);
           const __nv_bfloat16 b1 = __float2bfloat16_rn(d);
@@ -118,7 +131,7 @@ hbwn_umma_kernel(const Args g, const __grid_constant__ CUtensorMap a_map) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int64_t tiles_n = (g.N + TN - 1) / TN, tiles_m = (g.M + TM - 1) / TM;
   const int64_t n_tiles = tiles_m * tiles_n;
-  const int64_t n_kb = (g.K + KB - 1) / KB;                 // stages per tile
+  const int64_t n_kb = g.n_kb;                              // stages per tile
   const int64_t my_tiles = blockIdx.x < n_tiles ? (n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
   const int64_t total = my_tiles * n_kb;                    // stages this CTA walks
 
@@ -151,9 +164,20 @@ hbwn_umma_kernel(const Args g, const __grid_constant__ CUtensorMap a_map) {
         const int64_t tile = blockIdx.x + (gs / n_kb) * gridDim.x, kb = gs % n_kb;
         const unsigned char* src = g.w_prep + ((tile % tiles_n) * n_kb + kb) * S::B_STAGE;
         mbar_arrive_expect_tx(&full[s], S::A_STAGE + S::B_STAGE);
-        // x = kb * 64 elements = a multiple of 128 bytes; rows past M and columns past K are zero-filled
-        tma_load_2d(smem + S::OFF_A + s * S::A_STAGE, &a_map, static_cast<int32_t>(kb * KB),
-                    static_cast<int32_t>((tile / tiles_n) * TM), &full[s]);
+        const int64_t m0 = (tile / tiles_n) * TM;
+        if (g.conv) {
+          // 128 consecutive output pixels from (b, yo, xo), 64 channels from cb * 64 (a multiple of 128
+          // bytes), displaced by the filter tap; the halo and everything past the image arrive as zeros
+          const int32_t tap = static_cast<int32_t>(kb / g.cblocks), cb = static_cast<int32_t>(kb - tap * g.cblocks);
+          const int32_t fi = tap / g.kw, fj = tap - fi * g.kw;
+          const int32_t b = static_cast<int32_t>(m0 / g.HoWo), rem = static_cast<int32_t>(m0 - static_cast<int64_t>(b) * g.HoWo);
+          const int32_t yo = rem / g.Wo, xo = rem - yo * g.Wo;
+          tma_load_im2col_4d(smem + S::OFF_A + s * S::A_STAGE, &a_map, cb * KB, xo * g.sw - g.pw, yo * g.sh - g.ph, b,
+                             static_cast<uint16_t>(fj), static_cast<uint16_t>(fi), &full[s]);
+        } else {
+          // x = kb * 64 elements = a multiple of 128 bytes; rows past M and columns past K are zero-filled
+          tma_load_2d(smem + S::OFF_A + s * S::A_STAGE, &a_map, static_cast<int32_t>(kb * KB), static_cast<int32_t>(m0), &full[s]);
+        }
         bulk_copy_g2s(smem + S::OFF_B + s * S::B_STAGE, src, S::B_STAGE, &full[s]);
       }
     }
@@ -250,12 +274,15 @@ Args make_args(const DenseView& A, const PackedView& W, float* C, int64_t ldc) {
   g.Gw = num_groups(W.K, W.beta);
   g.beta = W.beta;
   g.w_prep = nullptr;
+  g.n_kb = (g.K + KB - 1) / KB;
+  g.conv = 0; g.taps = 1; g.kw = 1; g.cblocks = static_cast<int32_t>(g.n_kb); g.Cin = 0;
+  g.HoWo = 1; g.Wo = 1; g.sh = g.sw = 1; g.ph = g.pw = 0;
   return g;
 }
 
 template <int TN>
 size_t prep_bytes(const Args& g) {
-  return static_cast<size_t>(((g.N + TN - 1) / TN) * ((g.K + KB - 1) / KB)) * Smem<TN>::B_STAGE;
+  return static_cast<size_t>(((g.N + TN - 1) / TN) * g.n_kb) * Smem<TN>::B_STAGE;
 }
 
 // cuTensorMapEncodeTiled is a host-only driver routine; it is looked up through the runtime so the
@@ -289,11 +316,58 @@ bool make_a_map(const Args& g, CUtensorMap* map) {
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+using EncodeIm2colFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                    const int*, const int*, cuuint32_t, cuuint32_t, const cuuint32_t*, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeIm2colFn encode_im2col_fn() {
+  static EncodeIm2colFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeIm2colFn>(p);
+  }();
+  return fn;
+}
+
+// im2col tensor map of an NHWC bf16 image [B, H, W, Cp]: base pixels are the top-left input positions
+// of the filter windows (from -pad, stepping by the stride, Wo x Ho per image), 128 of them per copy
+// with 64 channels each; the filter tap is added by the copy instruction.
+bool make_conv_map(const void* x_nhwc, const ConvGeom& c, int Cp, CUtensorMap* map) {
+  EncodeIm2colFn fn = encode_im2col_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[4] = {static_cast<cuuint64_t>(c.C), static_cast<cuuint64_t>(c.W), static_cast<cuuint64_t>(c.H),
+                              static_cast<cuuint64_t>(c.B)};
+  const cuuint64_t strides[3] = {static_cast<cuuint64_t>(Cp) * 2, static_cast<cuuint64_t>(c.W) * Cp * 2,
+                                 static_cast<cuuint64_t>(c.H) * c.W * Cp * 2};
+  const int lower[2] = {-c.pw, -c.ph};
+  const int upper[2] = {c.pw - (c.kw - 1), c.ph - (c.kh - 1)};
+  const cuuint32_t elem[4] = {1, static_cast<cuuint32_t>(c.sw), static_cast<cuuint32_t>(c.sh), 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(x_nhwc), dims, strides, lower, upper, KB, TM, elem,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+Args make_conv_args(const ConvGeom& c, const PackedView& W, float* C, int64_t ldc) {
+  Args g;
+  g.a = nullptr; g.lda = 0;
+  g.w_bits = W.bits; g.w_scales = W.scales; g.ldw_w = W.ld_words; g.ldw_s = W.ld_scales; g.w_bf16 = W.scale_bf16;
+  g.C = C; g.ldc = ldc;
+  g.c_vec = (reinterpret_cast<uintptr_t>(C) % 16 == 0 && ldc % 4 == 0) ? 1 : 0;
+  g.M = static_cast<int64_t>(c.B) * c.Ho * c.Wo; g.N = W.rows; g.K = W.K;
+  g.Gw = num_groups(W.K, W.beta);
+  g.beta = W.beta;
+  g.w_prep = nullptr;
+  g.conv = 1; g.taps = c.kh * c.kw; g.kw = c.kw; g.cblocks = (c.C + KB - 1) / KB; g.Cin = c.C;
+  g.n_kb = static_cast<int64_t>(g.taps) * g.cblocks;
+  g.HoWo = c.Ho * c.Wo; g.Wo = c.Wo; g.sh = c.sh; g.sw = c.sw; g.ph = c.ph; g.pw = c.pw;
+  return g;
+}
+
 template <int TN>
-cudaError_t launch(Args g, void* workspace, cudaStream_t stream) {
+cudaError_t launch(Args g, const CUtensorMap& a_map, void* workspace, cudaStream_t stream) {
   using S = Smem<TN>;
-  CUtensorMap a_map;
-  if (!make_a_map(g, &a_map)) return cudaErrorNotSupported;
   static bool configured = false;
   static int sms = 0;
   if (!configured) {
@@ -304,7 +378,7 @@ cudaError_t launch(Args g, void* workspace, cudaStream_t stream) {
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     configured = true;
   }
-  const int64_t tiles_n = (g.N + TN - 1) / TN, n_kb = (g.K + KB - 1) / KB;
+  const int64_t tiles_n = (g.N + TN - 1) / TN, n_kb = g.n_kb;
   dim3 pgrid(static_cast<unsigned>(n_kb), static_cast<unsigned>(tiles_n));
   prepare_w_pieces_kernel<TN><<<pgrid, 256, 0, stream>>>(g, static_cast<unsigned char*>(workspace));
   g.w_prep = static_cast<const unsigned char*>(workspace);
@@ -333,7 +407,30 @@ size_t hbwn_umma_workspace_bytes(const DenseView& A, const PackedView& W) {
 cudaError_t launch_hbwn_umma(const DenseView& A, const PackedView& W, float* C, int64_t ldc, void* workspace,
                              cudaStream_t stream) {
   const Args g = make_args(A, W, C, ldc);
-  return launch<64>(g, workspace, stream);
+  CUtensorMap a_map;
+  if (!make_a_map(g, &a_map)) return cudaErrorNotSupported;
+  return launch<64>(g, a_map, workspace, stream);
+}
+
+// Implicit-GEMM convolution: whole 64-channel blocks (every tile row is then 128 bytes of real
+// channels), image extents and filter offsets inside what an im2col tensor map can describe.
+bool hbwn_umma_conv_supported(const ConvGeom& c, const PackedView& W) {
+  (void)W;
+  return c.C % KB == 0 && c.kh <= 16 && c.kw <= 16 && c.ph < 16 && c.pw < 16 && c.sh <= 8 && c.sw <= 8 &&
+         static_cast<int64_t>(c.Ho) * c.Wo < (int64_t{1} << 31) && encode_im2col_fn() != nullptr;
+}
+
+size_t hbwn_umma_conv_workspace_bytes(const ConvGeom& c, const PackedView& W) {
+  const Args g = make_conv_args(c, W, nullptr, 0);
+  return prep_bytes<64>(g);
+}
+
+cudaError_t launch_hbwn_umma_conv(const void* x_nhwc, int Cp, const ConvGeom& c, const PackedView& W, float* C, int64_t ldc,
+                                  void* workspace, cudaStream_t stream) {
+  const Args g = make_conv_args(c, W, C, ldc);
+  CUtensorMap a_map;
+  if (!make_conv_map(x_nhwc, c, Cp, &a_map)) return cudaErrorNotSupported;
+  return launch<64>(g, a_map, workspace, stream);
 }
 
 cudaError_t read_hbwn_umma_error(int* code) {

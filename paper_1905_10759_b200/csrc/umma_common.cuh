@@ -64,6 +64,16 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const void* tensor_map, i
   asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                ::"r"(smem_u32(dst)), "l"(tensor_map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
 }
+// im2col-mode tensor copy of an NHWC image: `pixels-per-column` consecutive base pixels starting at
+// (w, h, n) (walking W, then H, then N inside the map's bounding box), each displaced by the filter
+// offsets (w_off, h_off), `channels-per-pixel` channels from c.  c times the element size must be a
+// multiple of 16 bytes; pixels outside the image arrive as zeros.  No multicast.
+__device__ __forceinline__ void tma_load_im2col_4d(void* dst, const void* tensor_map, int32_t c, int32_t w, int32_t h, int32_t n,
+                                                   uint16_t w_off, uint16_t h_off, uint64_t* bar) {
+  asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6], {%7, %8};"
+               ::"r"(smem_u32(dst)), "l"(tensor_map), "r"(c), "r"(w), "r"(h), "r"(n), "r"(smem_u32(bar)), "h"(w_off), "h"(h_off)
+               : "memory");
+}
 
 // ---- tcgen05 helpers
 __device__ __forceinline__ bool mbar_wait_a(uint32_t bar, uint32_t parity, volatile int* abort_flag, int code) {

@@ -289,6 +289,13 @@ CONV_CASES = [
     (2, 24, 5, 5, 16, 1, 1, 1, 0, 32, 32, True, True),      # 1x1, bf16 input, K = 24 below a word
     (2, 64, 8, 8, 64, 3, 3, 1, 1, 1, 32, True, True),       # HBWN
     (2, 20, 7, 7, 33, 3, 3, 1, 1, 1, 32, False, False),     # HBWN from fp32 input (rounded to bf16 rows)
+    # HBWN with whole 64-channel blocks: no im2col matrix, tiles fetched by im2col-mode tensor copies
+    (3, 128, 7, 7, 72, 3, 3, 1, 1, 1, 32, True, False),     # two channel blocks, tiles span images, ragged M and N
+    (2, 64, 9, 9, 40, 3, 3, 2, 0, 1, 32, True, True),       # stride 2, no padding
+    (2, 64, 10, 10, 64, 3, 3, 2, 1, 1, 64, True, True),     # stride 2 with padding
+    (1, 64, 12, 12, 16, 1, 1, 1, 0, 1, 64, True, True),     # 1x1
+    (2, 64, 6, 6, 24, 5, 5, 1, 2, 1, 1600, True, True),     # 5x5, one weight group per row
+    (5, 192, 14, 14, 130, 3, 3, 1, 1, 1, 96, False, True),  # three blocks, several tiles per image, post-ReLU
 ]
 
 
