@@ -133,7 +133,6 @@ hbwn_umma_kernel(const Args g, const __grid_constant__ CUtensorMap a_map) {
   const int64_t n_tiles = tiles_m * tiles_n;
   const int64_t n_kb = g.n_kb;                              // stages per tile
   const int64_t my_tiles = blockIdx.x < n_tiles ? (n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
-  const int64_t total = my_tiles * n_kb;                    // stages this CTA walks
 
   if (tid == 0) {
     for (int s = 0; s < STAGES; s++) {
@@ -158,27 +157,40 @@ hbwn_umma_kernel(const Args g, const __grid_constant__ CUtensorMap a_map) {
     // =========================== loader ===========================
     if (lane == 0) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(&a_map) : "memory");
-      for (int64_t gs = 0; gs < total; gs++) {
-        const int s = static_cast<int>(gs % STAGES);
-        if (gs >= STAGES && !mbar_wait(&empty[s], static_cast<uint32_t>(((gs / STAGES) & 1) ^ 1), abort_flag, 1)) break;
-        const int64_t tile = blockIdx.x + (gs / n_kb) * gridDim.x, kb = gs % n_kb;
-        const unsigned char* src = g.w_prep + ((tile % tiles_n) * n_kb + kb) * S::B_STAGE;
-        mbar_arrive_expect_tx(&full[s], S::A_STAGE + S::B_STAGE);
-        const int64_t m0 = (tile / tiles_n) * TM;
+      // One thread feeds the whole CTA, so the loop carries its indices along instead of dividing:
+      // ring slot and round, K block -> (filter tap row, column, channel block).
+      int s = 0;
+      uint32_t round = 0;
+      bool ok = true;
+      for (int64_t ti = 0; ti < my_tiles && ok; ti++) {
+        const int64_t tile = blockIdx.x + ti * gridDim.x;
+        const int64_t tile_m = tile / tiles_n, tile_n = tile - tile_m * tiles_n;
+        const int64_t m0 = tile_m * TM;
+        const unsigned char* src = g.w_prep + tile_n * n_kb * S::B_STAGE;
+        int32_t b = 0, h0 = 0, w0 = 0;
         if (g.conv) {
-          // 128 consecutive output pixels from (b, yo, xo), 64 channels from cb * 64 (a multiple of 128
-          // bytes), displaced by the filter tap; the halo and everything past the image arrive as zeros
-          const int32_t tap = static_cast<int32_t>(kb / g.cblocks), cb = static_cast<int32_t>(kb - tap * g.cblocks);
-          const int32_t fi = tap / g.kw, fj = tap - fi * g.kw;
-          const int32_t b = static_cast<int32_t>(m0 / g.HoWo), rem = static_cast<int32_t>(m0 - static_cast<int64_t>(b) * g.HoWo);
+          // 128 consecutive output pixels from (b, yo, xo); the halo and everything past the image are zeros
+          b = static_cast<int32_t>(m0 / g.HoWo);
+          const int32_t rem = static_cast<int32_t>(m0 - static_cast<int64_t>(b) * g.HoWo);
           const int32_t yo = rem / g.Wo, xo = rem - yo * g.Wo;
-          tma_load_im2col_4d(smem + S::OFF_A + s * S::A_STAGE, &a_map, cb * KB, xo * g.sw - g.pw, yo * g.sh - g.ph, b,
-                             static_cast<uint16_t>(fj), static_cast<uint16_t>(fi), &full[s]);
-        } else {
-          // x = kb * 64 elements = a multiple of 128 bytes; rows past M and columns past K are zero-filled
-          tma_load_2d(smem + S::OFF_A + s * S::A_STAGE, &a_map, static_cast<int32_t>(kb * KB), static_cast<int32_t>(m0), &full[s]);
+          h0 = yo * g.sh - g.ph;
+          w0 = xo * g.sw - g.pw;
         }
-        bulk_copy_g2s(smem + S::OFF_B + s * S::B_STAGE, src, S::B_STAGE, &full[s]);
+        int32_t cb = 0, fi = 0, fj = 0;
+        for (int32_t kb = 0; kb < static_cast<int32_t>(n_kb); kb++) {
+          if (round > 0 && !mbar_wait(&empty[s], (round & 1) ^ 1, abort_flag, 1)) { ok = false; break; }
+          mbar_arrive_expect_tx(&full[s], S::A_STAGE + S::B_STAGE);
+          // the innermost coordinate (a channel or K offset, a multiple of 64 elements) is 128-byte aligned
+          if (g.conv)
+            tma_load_im2col_4d(smem + S::OFF_A + s * S::A_STAGE, &a_map, cb * KB, w0, h0, b, static_cast<uint16_t>(fj),
+                               static_cast<uint16_t>(fi), &full[s]);
+          else
+            tma_load_2d(smem + S::OFF_A + s * S::A_STAGE, &a_map, kb * KB, static_cast<int32_t>(m0), &full[s]);
+          bulk_copy_g2s(smem + S::OFF_B + s * S::B_STAGE, src, S::B_STAGE, &full[s]);
+          src += S::B_STAGE;
+          if (++cb == g.cblocks) { cb = 0; if (++fj == g.kw) { fj = 0; fi++; } }
+          if (++s == STAGES) { s = 0; round++; }
+        }
       }
     }
     __syncwarp();
