@@ -324,6 +324,9 @@ hbmm_status hbmm_last_device_error(int32_t* code) {
   int c2 = 0;
   if (read_gemm_umma_error(&c) != cudaSuccess || read_hbwn_umma_error(&c2) != cudaSuccess) return HBMM_ERR_CUDA;
   if (c == 0 && c2 != 0) c = 100 + c2;    // codes of the HBWN kernel are reported as 100 + code
+  int c3 = 0;
+  if (read_im2col_tma_error(&c3) != cudaSuccess) return HBMM_ERR_CUDA;
+  if (c == 0 && c3 != 0) c = 200 + c3;    // the packed front end's tile copy: 201
   if (code) *code = c;
   return c == 0 ? HBMM_OK : HBMM_ERR_TIMEOUT;
 }

@@ -18,9 +18,9 @@
 //   warp  4   : one thread issues both copies of every stage
 //   warp  5   : TMEM allocation and the MMA-issuing thread
 // Waits are bounded as in the packed kernel (error word, CTA-wide abort flag, orderly teardown).
-#include <cuda.h>
 #include <cuda_bf16.h>
 #include "kernels.h"
+#include "tensor_map.h"
 #include "umma_common.cuh"
 
 namespace hbmm {
@@ -297,23 +297,6 @@ size_t prep_bytes(const Args& g) {
   return static_cast<size_t>(((g.N + TN - 1) / TN) * g.n_kb) * Smem<TN>::B_STAGE;
 }
 
-// cuTensorMapEncodeTiled is a host-only driver routine; it is looked up through the runtime so the
-// library does not link against the driver.  nullptr when the driver does not offer it.
-using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-EncodeTiledFn encode_tiled_fn() {
-  static EncodeTiledFn fn = [] {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess)
-      p = nullptr;
-    return reinterpret_cast<EncodeTiledFn>(p);
-  }();
-  return fn;
-}
-
 // Tensor map of the activation matrix: bf16 [M, K] with row pitch lda, boxes of 64 x 128 elements
 // (one 128-byte-swizzled stage tile), zeros outside the matrix.
 bool make_a_map(const Args& g, CUtensorMap* map) {
@@ -326,21 +309,6 @@ bool make_a_map(const Args& g, CUtensorMap* map) {
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<__nv_bfloat16*>(g.a), dims, strides, box, elem,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-using EncodeIm2colFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                    const int*, const int*, cuuint32_t, cuuint32_t, const cuuint32_t*, CUtensorMapInterleave,
-                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-EncodeIm2colFn encode_im2col_fn() {
-  static EncodeIm2colFn fn = [] {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &p, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess)
-      p = nullptr;
-    return reinterpret_cast<EncodeIm2colFn>(p);
-  }();
-  return fn;
 }
 
 // im2col tensor map of an NHWC bf16 image [B, H, W, Cp]: base pixels are the top-left input positions

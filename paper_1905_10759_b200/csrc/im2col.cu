@@ -6,6 +6,7 @@
 // variant writes bf16 rows for the HBWN mode.
 #include <cuda_bf16.h>
 #include "kernels.h"
+#include "im2col_gather.cuh"
 
 namespace hbmm {
 namespace {
@@ -327,7 +328,11 @@ im2col_quantize_tiled_kernel(const void* __restrict__ x, int x_bf16, const ConvG
       const unsigned short* o = off + k_begin;
       uint32_t word = 0;
       float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-      if (nk == 32) {
+      if (cc == kTileCC && g.kh == 3 && g.kw == 3) {
+        gather_word_dispatch<3, 3>(w, base, tp.rows_in * tp.span, tp.span, word, s0);
+      } else if (cc == kTileCC && taps == 1) {
+        gather_word_dispatch<1, 1>(w, base, tp.rows_in * tp.span, tp.span, word, s0);
+      } else if (nk == 32) {
 #pragma unroll
         for (int e = 0; e < 32; e += 4) {
           const float v0 = base[o[e]], v1 = base[o[e + 1]], v2 = base[o[e + 2]], v3 = base[o[e + 3]];
@@ -373,6 +378,8 @@ cudaError_t launch_im2col_quantize(const void* x, int x_bf16, const ConvGeom& g,
   const int64_t M = static_cast<int64_t>(g.B) * g.Ho * g.Wo, K = static_cast<int64_t>(g.C) * g.kh * g.kw;
   const int64_t beta_eff = beta >= K ? K : beta;
   const int64_t G = num_groups(K, beta);
+  if (im2col_quantize_tma_supported(x, x_bf16, g, beta))
+    return launch_im2col_quantize_tma(x, g, bits, ld_words, scales, ld_scales, scale_bf16, stream);
   if (beta == 32 && beta < K && g.sw == 1) {
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);

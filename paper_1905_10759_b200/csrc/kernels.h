@@ -83,6 +83,11 @@ cudaError_t launch_hbwn_umma_conv(const void* x_nhwc, int Cp, const ConvGeom& g,
 cudaError_t launch_im2col_quantize(const void* x, int x_bf16, const ConvGeom& g, int32_t beta,
                                    uint32_t* bits, int64_t ld_words, void* scales, int64_t ld_scales,
                                    int scale_bf16, cudaStream_t stream);
+// The packed front end with its input tile staged by tensor copies (fp32 input, beta = 32).
+bool im2col_quantize_tma_supported(const void* x, int x_bf16, const ConvGeom& g, int32_t beta);
+cudaError_t launch_im2col_quantize_tma(const void* x, const ConvGeom& g, uint32_t* bits, int64_t ld_words, void* scales,
+                                       int64_t ld_scales, int scale_bf16, cudaStream_t stream);
+cudaError_t read_im2col_tma_error(int* code);
 cudaError_t launch_im2col_bf16(const void* x, int x_bf16, const ConvGeom& g, void* out, int64_t ld,
                                cudaStream_t stream);
 

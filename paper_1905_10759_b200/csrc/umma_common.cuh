@@ -64,6 +64,13 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const void* tensor_map, i
   asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                ::"r"(smem_u32(dst)), "l"(tensor_map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
 }
+// The same for a 4-D tensor (x innermost).  Loads may start at negative or out-of-range coordinates
+// (x still 16-byte aligned): whatever lies outside the tensor arrives as zeros.
+__device__ __forceinline__ void tma_load_4d(void* dst, const void* tensor_map, int32_t x, int32_t y, int32_t z, int32_t w,
+                                            uint64_t* bar) {
+  asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+               ::"r"(smem_u32(dst)), "l"(tensor_map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(smem_u32(bar)) : "memory");
+}
 // im2col-mode tensor copy of an NHWC image: `pixels-per-column` consecutive base pixels starting at
 // (w, h, n) (walking W, then H, then N inside the map's bounding box), each displaced by the filter
 // offsets (w_off, h_off), `channels-per-pixel` channels from c.  c times the element size must be a

@@ -289,6 +289,12 @@ CONV_CASES = [
     (2, 24, 5, 5, 16, 1, 1, 1, 0, 32, 32, True, True),      # 1x1, bf16 input, K = 24 below a word
     (2, 64, 8, 8, 64, 3, 3, 1, 1, 1, 32, True, True),       # HBWN
     (2, 20, 7, 7, 33, 3, 3, 1, 1, 1, 32, False, False),     # HBWN from fp32 input (rounded to bf16 rows)
+    # packed front end with the input tile staged by tensor copies (fp32 input, W % 4 == 0, stride 1 along x)
+    (2, 96, 20, 20, 40, 3, 3, 1, 1, 32, 32, True, False),   # several row blocks and channel ranges
+    (2, 40, 8, 8, 24, 5, 5, 1, 2, 32, 32, True, False),     # 5x5, last chunk of 8 channels
+    (1, 64, 12, 12, 16, 1, 1, 1, 0, 32, 32, True, False),   # 1x1
+    (3, 70, 16, 12, 33, 3, 3, 1, 0, 32, 64, True, False),   # no padding, ragged channels, beta_w = 64
+    (2, 64, 8, 8, 16, 3, 3, 1, 1, 32, 32, None, False),     # zeros of both signs in the input
     # HBWN with whole 64-channel blocks: no im2col matrix, tiles fetched by im2col-mode tensor copies
     (3, 128, 7, 7, 72, 3, 3, 1, 1, 1, 32, True, False),     # two channel blocks, tiles span images, ragged M and N
     (2, 64, 9, 9, 40, 3, 3, 2, 0, 1, 32, True, True),       # stride 2, no padding
@@ -303,7 +309,12 @@ CONV_CASES = [
 def test_conv_im2col_matches_oracle(hb, B, C, H, W, N, kh, kw, st, pd, ba, bw, signed, xbf16):
     gu = _gu()
     shape = inputs.ConvShape("t", B, C, H, W, N, kh, kw, st, pd)
-    x = inputs.conv_activation(shape, 8000 + C + H, signed=signed)
+    x = inputs.conv_activation(shape, 8000 + C + H, signed=bool(signed) or signed is None)
+    if signed is None:
+        # Sign(+0) = Sign(-0) = +1: plant zeros of both signs
+        flat = x.reshape(-1)
+        flat[::7] = 0.0
+        flat[3::11] = -0.0
     if xbf16 or ba == 1:
         _, xr = inputs.as_bf16(x)     # HBWN rows are bf16: the oracle sees the same rounded values
     else:
