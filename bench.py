@@ -138,9 +138,12 @@ def layer_ops(shapes):
     return [2.0 * s.M * s.N * s.K for s in shapes]
 
 
-def build_workload(torch, hbmm, inputs, rank: int, device):
-    """Device-resident inputs, weights (binarized once), outputs and workspaces for every layer."""
-    shapes = inputs.resnet18_convs(64)
+def build_workload(torch, hbmm, inputs, rank: int, device, only=None):
+    """Device-resident inputs, weights (binarized once), outputs and workspaces for every layer
+    (or for the one layer named by ``only``)."""
+    shapes = [s for s in inputs.resnet18_convs(64) if only is None or s.name == only]
+    if not shapes:
+        raise SystemExit("unknown layer %r" % only)
     off = rank_seed_offset(rank)
     layers = []
     for li, s in enumerate(shapes):
@@ -359,8 +362,16 @@ def run_ours(args):
         dist.barrier()
     from paper_1905_10759_b200 import hbmm, inputs
 
-    shapes, layers = build_workload(torch, hbmm, inputs, rank, device)
+    shapes, layers = build_workload(torch, hbmm, inputs, rank, device, args.profile_layer)
     ops_step = 2.0 * sum(layer_ops(shapes))        # HBMM + HBWN product of every layer
+    if args.profile_layer:
+        # a small, short run of one layer for profiler captures: no end-to-end leg, no breakdown, no CPU timing
+        for _ in range(max(args.warmup, 3) + args.steps):
+            run_step(hbmm, layers)
+        torch.cuda.synchronize()
+        assert hbmm.last_device_error() == 0
+        print(json.dumps({"profile_layer": args.profile_layer, "steps": args.steps, "launches_per_step": 6}))
+        return 0
 
     for _ in range(max(args.warmup, 3)):
         run_step(hbmm, layers)
@@ -438,7 +449,7 @@ def run_ours(args):
             "beta_a": BETA, "beta_w": BETA, "scale_dtype": "f32", "hbwn_activation_dtype": "bf16",
             "tensor_operands": "sign bits as +-1 e4m3 (HBMM) / +-1 bf16 (HBWN), exact; fp32 accumulate and scales",
             "batch_per_gpu": 64, "parallelism": "replicas(batch-sharded)x%d" % world,
-            "l2": "per-step inputs+outputs+workspaces (~0.9 GB) exceed the 126 MB L2; no explicit flush",
+            "l2": "per-step inputs+outputs+workspaces (~0.7 GB) exceed the 126 MB L2; no explicit flush",
         },
         "roofline": roof,
         "kernels": kernels,
@@ -463,6 +474,8 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--profile-layer", default=None,
+                    help="run only this layer (conv2_x .. conv5_x), few launches, no measurement: for profiler captures")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

@@ -6,11 +6,13 @@
 namespace hbmm {
 
 // One K-word: element e of word WORD is chunk-local k = 32 * WORD + e = (c, i, j) with
-// c = k / (KH * KW), read from a staged tile at base[c * cs + i * pitch + j].  Each element costs one
-// shared-memory load, one add of +0 (so that -0 counts as +0 and the sign bit alone decides
-// Sign(x): x >= 0 <=> bit clear), one funnel shift that collects the sign bit, and one add of |x|.
+// c = k / (KH * KW), read from a staged fp32 tile in shared memory at byte address
+// base + c * cs_bytes + i * pitch_bytes + 4 * j (one address per (c, i), the tap column as an
+// immediate).  Each element costs one shared-memory load, one add of +0 (so that -0 counts as +0 and
+// the sign bit alone decides Sign(x): x >= 0 <=> bit clear), one funnel shift that collects the sign
+// bit, and one add of |x|.  Returns the packed word (bit e = 1 <=> x >= 0) and the sum of |x|.
 template <int KH, int KW, int WORD>
-__device__ __forceinline__ void gather_word_static(const float* __restrict__ base, int cs, int pitch, uint32_t& word, float& sum) {
+__device__ __forceinline__ void gather_word_static(uint32_t base, uint32_t cs_bytes, uint32_t pitch_bytes, uint32_t& word, float& sum) {
   constexpr int T = KH * KW;
   uint32_t pat = 0;
   float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
@@ -20,21 +22,25 @@ __device__ __forceinline__ void gather_word_static(const float* __restrict__ bas
 #pragma unroll
     for (int u = 0; u < 4; u++) {
       const int k = 32 * WORD + e + u, c = k / T, t = k % T, i = t / KW, j = t % KW;
-      v[u] = base[c * cs + i * pitch + j] + 0.0f;
+      const uint32_t row = base + c * cs_bytes + i * pitch_bytes;
+      float x;
+      asm volatile("ld.shared.f32 %0, [%1];" : "=f"(x) : "r"(row + 4 * j));   // the constant folds into the load
+      v[u] = x + 0.0f;
       pat = __funnelshift_l(__float_as_uint(v[u]), pat, 1);     // pat = pat << 1 | sign bit
     }
     s0 += fabsf(v[0]); s1 += fabsf(v[1]); s2 += fabsf(v[2]); s3 += fabsf(v[3]);
   }
-  word = ~__brev(pat);                                            // element e at bit e, 1 <=> x >= 0
+  word = ~__brev(pat);                                            // element e at bit e
   sum = (s0 + s1) + (s2 + s3);
 }
 
 // w (warp-uniform) selects the word of the chunk: KH * KW words per 32 channels.
 template <int KH, int KW, int WORD = 0>
-__device__ __forceinline__ void gather_word_dispatch(int w, const float* __restrict__ base, int cs, int pitch, uint32_t& word, float& sum) {
+__device__ __forceinline__ void gather_word_dispatch(int w, uint32_t base, uint32_t cs_bytes, uint32_t pitch_bytes, uint32_t& word,
+                                                     float& sum) {
   if constexpr (WORD < KH * KW) {
-    if (w == WORD) gather_word_static<KH, KW, WORD>(base, cs, pitch, word, sum);
-    else gather_word_dispatch<KH, KW, WORD + 1>(w, base, cs, pitch, word, sum);
+    if (w == WORD) gather_word_static<KH, KW, WORD>(base, cs_bytes, pitch_bytes, word, sum);
+    else gather_word_dispatch<KH, KW, WORD + 1>(w, base, cs_bytes, pitch_bytes, word, sum);
   }
 }
 

@@ -1,11 +1,12 @@
 // Packed convolution front end (beta = 32, fp32 NCHW input) with the input tile staged by tensor
-// copies.  A block handles RB output rows of one image and a range of 32-channel chunks.  For every
+// copies.  A work item is RB output rows of one image and a range of 32-channel chunks.  For every
 // chunk one 4-D tensor copy brings [32 channels][rows_in input rows][pitch columns] into shared
 // memory, zero halo included (the copy starts left of and above the image where the padding asks
-// for it, and whatever lies outside the tensor arrives as zeros); the copy of the next chunk is in
-// flight while the current one is binarized.  One thread then produces one (output pixel, K-word):
-// the 32 lanes of a warp hold 32 consecutive pixels of the same word, so tile reads are consecutive.
-// Words and scales are collected in shared memory and leave the block as contiguous runs per row.
+// for it, and whatever lies outside the tensor arrives as zeros).  Two persistent CTAs per SM: a
+// loader thread keeps a ring of tile buffers full across chunks and items, twelve compute warps
+// binarize.  A warp-item is 32 consecutive pixels of one K-word, so tile reads are consecutive.
+// Words and scales of an item are collected in shared memory and leave as contiguous 16-byte runs.
+// Every wait is bounded (error word + CTA-wide abort flag, as in the tensor-core kernels).
 #include <cuda_bf16.h>
 #include "kernels.h"
 #include "tensor_map.h"
@@ -28,6 +29,7 @@ struct Plan {
   int splits;             // channel ranges (grid.y)
   int chunks_per_split;
   int n_chunks;           // ceil(C / 32)
+  int ring;               // tile buffers per CTA
 };
 
 __device__ __forceinline__ void store_scale(void* scales, int bf16, int64_t idx, float v) {
@@ -35,35 +37,55 @@ __device__ __forceinline__ void store_scale(void* scales, int bf16, int64_t idx,
   else reinterpret_cast<float*>(scales)[idx] = v;
 }
 
-__global__ void __launch_bounds__(256)
-im2col_quantize_tma_kernel(const __grid_constant__ CUtensorMap x_map, const ConvGeom g, const Plan tp,
+constexpr int kComputeWarps = 12;                    // 36 warp-items per chunk of 112..128 pixels: three rounds
+constexpr int kLoaderWarp = kComputeWarps;
+constexpr int kThreadsTma = (kComputeWarps + 1) * 32;
+constexpr int kMaxRing = 6;
+
+// Work item = (row block of one image, channel range).  A CTA is persistent: it walks items
+// blockIdx.x, blockIdx.x + gridDim.x, ... and the ring of tile buffers simply continues across items,
+// so the copies of the next item are in flight while the current one is binarized and written out.
+struct ItemCoords {
+  int32_t b, yo0, chunk_first, n_my;
+};
+__device__ __forceinline__ ItemCoords item_coords(int item, const Plan& tp) {
+  ItemCoords c;
+  const int rb = item / tp.splits, sp = item - rb * tp.splits;
+  c.b = rb / tp.yo_blocks;
+  c.yo0 = (rb - c.b * tp.yo_blocks) * tp.RB;
+  c.chunk_first = sp * tp.chunks_per_split;
+  c.n_my = (tp.n_chunks - c.chunk_first < tp.chunks_per_split) ? tp.n_chunks - c.chunk_first : tp.chunks_per_split;
+  return c;
+}
+
+__global__ void __launch_bounds__(kThreadsTma, 2)
+im2col_quantize_tma_kernel(const __grid_constant__ CUtensorMap x_map, const ConvGeom g, const Plan tp, int n_items, int ring,
                            uint32_t* __restrict__ bits, int64_t ld_words, void* __restrict__ scales, int64_t ld_scales,
                            int scale_bf16) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int taps = g.kh * g.kw;
   const int tile_elems = kCC * tp.rows_in * tp.pitch;           // floats per buffer; bytes are a multiple of 128
   const int max_pixels = tp.RB * g.Wo;
-  const int split_words = tp.chunks_per_split * taps;          // words this block produces per pixel (upper bound)
+  const int split_words = tp.chunks_per_split * taps;          // words an item produces per pixel (upper bound)
   const int ldo = split_words + 1;                             // odd-ish pitch: fewer bank conflicts on the column writes
-  float* tile0 = reinterpret_cast<float*>(smem_raw);                                   // two tile buffers
-  uint64_t* bar = reinterpret_cast<uint64_t*>(tile0 + 2 * tile_elems);                // two "tile landed" barriers
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(bar + 2);
-  uint32_t* out_bits = reinterpret_cast<uint32_t*>(bar + 4);                          // [max_pixels][ldo]
+  float* tile0 = reinterpret_cast<float*>(smem_raw);                                   // `ring` tile buffers
+  uint64_t* full = reinterpret_cast<uint64_t*>(tile0 + static_cast<size_t>(ring) * tile_elems);
+  uint64_t* empty = full + kMaxRing;
+  uint64_t* computed = empty + kMaxRing;                       // all compute warps are done with an item's chunks
+  uint64_t* written = computed + 1;                            // ... and with its write-out
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(written + 1);
+  uint32_t* out_bits = reinterpret_cast<uint32_t*>(written + 2);                      // [max_pixels][ldo]
   float* out_scale = reinterpret_cast<float*>(out_bits + max_pixels * ldo);           // same shape
-  unsigned short* off = reinterpret_cast<unsigned short*>(out_scale + max_pixels * ldo);
+  unsigned short* off = reinterpret_cast<unsigned short*>(out_scale + max_pixels * ldo);    // [32 * taps]
+  unsigned short* pixoff = off + (kCC * taps + 1) / 2 * 2;                                  // [max_pixels]
 
-  const int64_t b = blockIdx.x / tp.yo_blocks;
-  const int yo0 = static_cast<int>(blockIdx.x % tp.yo_blocks) * tp.RB;
-  const int rows = (g.Ho - yo0 < tp.RB) ? g.Ho - yo0 : tp.RB;
-  const int pixels = rows * g.Wo;
-  const int pix_pad = (pixels + 31) / 32 * 32;                 // keep a warp on one word
-  const int chunk_first = blockIdx.y * tp.chunks_per_split;
-  const int n_my = (tp.n_chunks - chunk_first < tp.chunks_per_split) ? tp.n_chunks - chunk_first : tp.chunks_per_split;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cs = tp.rows_in * tp.pitch;
 
   if (threadIdx.x == 0) {
-    mbar_init(&bar[0], 1);
-    mbar_init(&bar[1], 1);
+    for (int s = 0; s < kMaxRing; s++) { mbar_init(&full[s], 1); mbar_init(&empty[s], kComputeWarps); }
+    mbar_init(computed, kComputeWarps);
+    mbar_init(written, kComputeWarps);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -72,106 +94,167 @@ im2col_quantize_tma_kernel(const __grid_constant__ CUtensorMap x_map, const Conv
     const int c = k / taps, r = k - c * taps, i = r / g.kw, j = r - i * g.kw;
     off[k] = static_cast<unsigned short>(c * cs + i * tp.pitch + j);
   }
+  // pixel of an item -> tile offset of its first tap (channel 0, filter row 0, column 0)
+  for (int pix = threadIdx.x; pix < max_pixels; pix += blockDim.x) {
+    const int ry = pix / g.Wo, xo = pix - ry * g.Wo;
+    pixoff[pix] = static_cast<unsigned short>(ry * g.sh * tp.pitch + xo + tp.x0);
+  }
   __syncthreads();
 
-  const uint32_t tile_bytes = static_cast<uint32_t>(tile_elems) * 4;
-  auto issue = [&](int it) {
-    // x starts at -(x0 + pw), a multiple of 4 elements = 16 bytes; y may be negative too
-    fence_async_proxy();            // earlier reads of this buffer are ordered before the copy's writes
-    mbar_arrive_expect_tx(&bar[it & 1], tile_bytes);
-    tma_load_4d(tile0 + (it & 1) * tile_elems, &x_map, -(tp.x0 + g.pw), yo0 * g.sh - g.ph, (chunk_first + it) * kCC, static_cast<int32_t>(b),
-                &bar[it & 1]);
-  };
-  if (threadIdx.x == 0 && n_my > 0) issue(0);
-
-  int words_done = 0;                                          // words produced so far by this block
-  bool wrote_last = false;
-  for (int it = 0; it < n_my; it++) {
-    const int c0 = (chunk_first + it) * kCC;
-    const int cc = (g.C - c0 < kCC) ? g.C - c0 : kCC;
-    wrote_last = c0 + cc == g.C;
-    // the other buffer was last read in iteration it - 1, which ended with a block-wide barrier
-    if (threadIdx.x == 0 && it + 1 < n_my) issue(it + 1);
-    mbar_wait(&bar[it & 1], static_cast<uint32_t>((it >> 1) & 1), abort_flag, 1);   // bounded; on expiry the output is undefined
-    const float* t = tile0 + (it & 1) * tile_elems;
-    const int chunk_elems = cc * taps;
-    const int words = (chunk_elems + 31) / 32;
-    for (int idx = threadIdx.x; idx < pix_pad * words; idx += 256) {
-      const int w = idx / pix_pad, pix = idx - w * pix_pad;
-      if (pix >= pixels) continue;
-      const int ry = pix / g.Wo, xo = pix - ry * g.Wo;
-      const int k_begin = w * 32;
-      const int nk = (chunk_elems - k_begin < 32) ? chunk_elems - k_begin : 32;
-      const float* base = t + ry * g.sh * tp.pitch + xo + tp.x0;
-      uint32_t word = 0;
-      float sum = 0.f;
-      if (cc == kCC && g.kh == 3 && g.kw == 3) {
-        gather_word_dispatch<3, 3>(w, base, cs, tp.pitch, word, sum);
-      } else if (cc == kCC && taps == 1) {
-        gather_word_dispatch<1, 1>(w, base, cs, tp.pitch, word, sum);
-      } else {
-        const unsigned short* o = off + k_begin;
-        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-        int e = 0;
-        for (; e + 4 <= nk; e += 4) {
-          const float v0 = base[o[e]], v1 = base[o[e + 1]], v2 = base[o[e + 2]], v3 = base[o[e + 3]];
-          word |= (v0 >= 0.0f ? 1u : 0u) << e;
-          word |= (v1 >= 0.0f ? 1u : 0u) << (e + 1);
-          word |= (v2 >= 0.0f ? 1u : 0u) << (e + 2);
-          word |= (v3 >= 0.0f ? 1u : 0u) << (e + 3);
-          s0 += fabsf(v0); s1 += fabsf(v1); s2 += fabsf(v2); s3 += fabsf(v3);
+  if (warp == kLoaderWarp) {
+    // =========================== loader ===========================
+    if (lane == 0) {
+      const uint32_t tile_bytes = static_cast<uint32_t>(tile_elems) * 4;
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&x_map) : "memory");
+      int s = 0;
+      uint32_t round = 0;
+      int issued = 0;                                          // copies issued so far (for the abort path)
+      bool ok = true;
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+        const ItemCoords ic = item_coords(item, tp);
+        for (int it = 0; it < ic.n_my; it++) {
+          if (round > 0 && !mbar_wait(&empty[s], (round & 1) ^ 1, abort_flag, 1)) { ok = false; break; }
+          mbar_arrive_expect_tx(&full[s], tile_bytes);
+          // x starts at -(x0 + pw), a multiple of 4 elements = 16 bytes; y may be negative too; what lies
+          // outside the tensor (halo, channels past C) arrives as zeros
+          tma_load_4d(tile0 + static_cast<size_t>(s) * tile_elems, &x_map, -(tp.x0 + g.pw), ic.yo0 * g.sh - g.ph,
+                      (ic.chunk_first + it) * kCC, ic.b, &full[s]);
+          issued++;
+          if (++s == ring) { s = 0; round++; }
         }
-        for (; e < nk; e++) {
-          const float v = base[o[e]];
-          word |= (v >= 0.0f ? 1u : 0u) << e;
-          s0 += fabsf(v);
-        }
-        sum = (s0 + s1) + (s2 + s3);
       }
-      out_bits[pix * ldo + words_done + w] = word;
-      out_scale[pix * ldo + words_done + w] = sum / static_cast<float>(nk);
+      if (!ok) {
+        // aborted: let the copies already issued land before the CTA's shared memory goes away
+        const int pending = issued < ring ? issued : ring;
+        for (int q = 0; q < pending; q++) {
+          const int idx = issued - 1 - q, slot = idx % ring;
+          for (uint32_t spin = 0; spin < kSpinLimit; spin++)
+            if (mbar_try_wait(&full[slot], static_cast<uint32_t>((idx / ring) & 1))) break;
+        }
+      }
     }
-    words_done += words;
-    __syncthreads();
+    __syncwarp();
+    return;
   }
 
-  // contiguous runs: for each pixel the block's words, then (last range only) the zero padding
-  const int64_t word0 = static_cast<int64_t>(chunk_first) * kCC * taps / 32;
-  const int run_bits = wrote_last ? static_cast<int>(ld_words - word0) : words_done;
-  const int run_scale = wrote_last ? static_cast<int>(ld_scales - word0) : words_done;
-  const int64_t m_base = (b * g.Ho + yo0) * g.Wo;
-  if ((word0 & 3) == 0 && (run_bits & 3) == 0) {
-    const int q_per = run_bits >> 2;                         // 16-byte pieces per pixel
-    for (int idx = threadIdx.x; idx < pixels * q_per; idx += 256) {
-      const int pix = idx / q_per, w = (idx - pix * q_per) * 4;
-      const uint32_t* src = out_bits + pix * ldo + w;
-      uint4 o;
-      o.x = (w < words_done) ? src[0] : 0u; o.y = (w + 1 < words_done) ? src[1] : 0u;
-      o.z = (w + 2 < words_done) ? src[2] : 0u; o.w = (w + 3 < words_done) ? src[3] : 0u;
-      *reinterpret_cast<uint4*>(bits + (m_base + pix) * ld_words + word0 + w) = o;
+  // =========================== compute warps ===========================
+  int s = 0;
+  uint32_t round = 0, phase = 0;                               // ring position; parity of `computed` / `written`
+  for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+    const ItemCoords ic = item_coords(item, tp);
+    const int rows = (g.Ho - ic.yo0 < tp.RB) ? g.Ho - ic.yo0 : tp.RB;
+    const int pixels = rows * g.Wo;
+    const int pix_warps = (pixels + 31) / 32;                  // a warp stays on one word: 32 pixels x 1 word per warp-item
+    int words_done = 0;                                        // words produced so far for this item
+    bool wrote_last = false;
+    for (int it = 0; it < ic.n_my; it++) {
+      const int c0 = (ic.chunk_first + it) * kCC;
+      const int cc = (g.C - c0 < kCC) ? g.C - c0 : kCC;
+      wrote_last = c0 + cc == g.C;
+      if (!mbar_wait(&full[s], round & 1, abort_flag, 2)) return;
+      const float* t = tile0 + static_cast<size_t>(s) * tile_elems;
+      const int chunk_elems = cc * taps;
+      const int words = (chunk_elems + 31) / 32;
+      // warp-items (w, pw): word w of pixel group pw; walked with a stride of kComputeWarps, indices carried along
+      int pw = warp % pix_warps, w = warp / pix_warps;
+      const int dpw = kComputeWarps % pix_warps, dw = kComputeWarps / pix_warps;
+      const uint32_t t_addr = smem_u32(t);
+      for (; w < words; ) {
+        const int pix = pw * 32 + lane;
+        if (pix < pixels) {
+          const int k_begin = w * 32;
+          const int nk = (chunk_elems - k_begin < 32) ? chunk_elems - k_begin : 32;
+          const uint32_t po = pixoff[pix];                     // tile offset of the pixel's first tap, in elements
+          uint32_t word = 0;
+          float mean;
+          if (cc == kCC && g.kh == 3 && g.kw == 3) {
+            float sum;
+            gather_word_dispatch<3, 3>(w, t_addr + po * 4, cs * 4, tp.pitch * 4, word, sum);
+            mean = sum * 0.03125f;
+          } else if (cc == kCC && taps == 1) {
+            float sum;
+            gather_word_dispatch<1, 1>(w, t_addr + po * 4, cs * 4, tp.pitch * 4, word, sum);
+            mean = sum * 0.03125f;
+          } else {
+            const float* base = t + po;
+            const unsigned short* o = off + k_begin;
+            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+            int e = 0;
+            for (; e + 4 <= nk; e += 4) {
+              const float v0 = base[o[e]], v1 = base[o[e + 1]], v2 = base[o[e + 2]], v3 = base[o[e + 3]];
+              word |= (v0 >= 0.0f ? 1u : 0u) << e;
+              word |= (v1 >= 0.0f ? 1u : 0u) << (e + 1);
+              word |= (v2 >= 0.0f ? 1u : 0u) << (e + 2);
+              word |= (v3 >= 0.0f ? 1u : 0u) << (e + 3);
+              s0 += fabsf(v0); s1 += fabsf(v1); s2 += fabsf(v2); s3 += fabsf(v3);
+            }
+            for (; e < nk; e++) {
+              const float v = base[o[e]];
+              word |= (v >= 0.0f ? 1u : 0u) << e;
+              s0 += fabsf(v);
+            }
+            mean = ((s0 + s1) + (s2 + s3)) / static_cast<float>(nk);
+          }
+          out_bits[pix * ldo + words_done + w] = word;
+          out_scale[pix * ldo + words_done + w] = mean;
+        }
+        pw += dpw; w += dw;
+        if (pw >= pix_warps) { pw -= pix_warps; w++; }
+      }
+      words_done += words;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&empty[s]);                   // this warp is done with the tile
+      if (++s == ring) { s = 0; round++; }
     }
-  } else {
-    for (int idx = threadIdx.x; idx < pixels * run_bits; idx += 256) {
-      const int pix = idx / run_bits, w = idx - pix * run_bits;
-      bits[(m_base + pix) * ld_words + word0 + w] = (w < words_done) ? out_bits[pix * ldo + w] : 0u;
+    // every compute warp has produced its part of the item
+    __syncwarp();
+    if (lane == 0) mbar_arrive(computed);
+    if (!mbar_wait(computed, phase, abort_flag, 3)) return;
+
+    // contiguous runs: for each pixel the item's words, then (last range only) the zero padding
+    const int tid = threadIdx.x, nthr = kComputeWarps * 32;
+    const int64_t word0 = static_cast<int64_t>(ic.chunk_first) * kCC * taps / 32;
+    const int run_bits = wrote_last ? static_cast<int>(ld_words - word0) : words_done;
+    const int run_scale = wrote_last ? static_cast<int>(ld_scales - word0) : words_done;
+    const int64_t m_base = (static_cast<int64_t>(ic.b) * g.Ho + ic.yo0) * g.Wo;
+    if ((word0 & 3) == 0 && (run_bits & 3) == 0) {
+      const int q_per = run_bits >> 2;                         // 16-byte pieces per pixel
+      for (int idx = tid; idx < pixels * q_per; idx += nthr) {
+        const int pix = idx / q_per, w = (idx - pix * q_per) * 4;
+        const uint32_t* src = out_bits + pix * ldo + w;
+        uint4 o;
+        o.x = (w < words_done) ? src[0] : 0u; o.y = (w + 1 < words_done) ? src[1] : 0u;
+        o.z = (w + 2 < words_done) ? src[2] : 0u; o.w = (w + 3 < words_done) ? src[3] : 0u;
+        *reinterpret_cast<uint4*>(bits + (m_base + pix) * ld_words + word0 + w) = o;
+      }
+    } else {
+      for (int idx = tid; idx < pixels * run_bits; idx += nthr) {
+        const int pix = idx / run_bits, w = idx - pix * run_bits;
+        bits[(m_base + pix) * ld_words + word0 + w] = (w < words_done) ? out_bits[pix * ldo + w] : 0u;
+      }
     }
-  }
-  if (!scale_bf16 && (word0 & 3) == 0 && (run_scale & 3) == 0) {
-    const int q_per = run_scale >> 2;
-    float* sc = reinterpret_cast<float*>(scales);
-    for (int idx = threadIdx.x; idx < pixels * q_per; idx += 256) {
-      const int pix = idx / q_per, w = (idx - pix * q_per) * 4;
-      const float* src = out_scale + pix * ldo + w;
-      float4 o;
-      o.x = (w < words_done) ? src[0] : 0.f; o.y = (w + 1 < words_done) ? src[1] : 0.f;
-      o.z = (w + 2 < words_done) ? src[2] : 0.f; o.w = (w + 3 < words_done) ? src[3] : 0.f;
-      *reinterpret_cast<float4*>(sc + (m_base + pix) * ld_scales + word0 + w) = o;
+    if (!scale_bf16 && (word0 & 3) == 0 && (run_scale & 3) == 0) {
+      const int q_per = run_scale >> 2;
+      float* sc = reinterpret_cast<float*>(scales);
+      for (int idx = tid; idx < pixels * q_per; idx += nthr) {
+        const int pix = idx / q_per, w = (idx - pix * q_per) * 4;
+        const float* src = out_scale + pix * ldo + w;
+        float4 o;
+        o.x = (w < words_done) ? src[0] : 0.f; o.y = (w + 1 < words_done) ? src[1] : 0.f;
+        o.z = (w + 2 < words_done) ? src[2] : 0.f; o.w = (w + 3 < words_done) ? src[3] : 0.f;
+        *reinterpret_cast<float4*>(sc + (m_base + pix) * ld_scales + word0 + w) = o;
+      }
+    } else {
+      for (int idx = tid; idx < pixels * run_scale; idx += nthr) {
+        const int pix = idx / run_scale, w = idx - pix * run_scale;
+        store_scale(scales, scale_bf16, (m_base + pix) * ld_scales + word0 + w, (w < words_done) ? out_scale[pix * ldo + w] : 0.0f);
+      }
     }
-  } else {
-    for (int idx = threadIdx.x; idx < pixels * run_scale; idx += 256) {
-      const int pix = idx / run_scale, w = idx - pix * run_scale;
-      store_scale(scales, scale_bf16, (m_base + pix) * ld_scales + word0 + w, (w < words_done) ? out_scale[pix * ldo + w] : 0.0f);
-    }
+    // the staging arrays may be overwritten once every warp has read its part of them
+    __syncwarp();
+    if (lane == 0) mbar_arrive(written);
+    if (!mbar_wait(written, phase, abort_flag, 4)) return;
+    phase ^= 1;
   }
 }
 
@@ -195,10 +278,16 @@ bool make_plan(const ConvGeom& g, int sms, Plan* out, size_t* smem_bytes) {
   p.splits = (p.n_chunks + p.chunks_per_split - 1) / p.chunks_per_split;
   const int taps = g.kh * g.kw;
   const int64_t tile_elems = static_cast<int64_t>(kCC) * p.rows_in * p.pitch;
-  *smem_bytes = static_cast<size_t>(2 * tile_elems * 4 + 32 +
-                                    2LL * p.RB * g.Wo * (p.chunks_per_split * taps + 1) * 4 + static_cast<int64_t>(kCC) * taps * 2 + 16);
+  // everything but the tile ring: barriers, staging arrays of one item, offset table
+  const int64_t fixed = (2 * kMaxRing + 4) * 8 + 2LL * p.RB * g.Wo * (p.chunks_per_split * taps + 1) * 4 +
+                        static_cast<int64_t>(kCC) * taps * 2 + 2LL * p.RB * g.Wo + 32;
+  const int64_t budget = 100 * 1024;                           // two CTAs per SM: one computes while the other synchronises or writes
+  int64_t ring = (budget - fixed) / (tile_elems * 4);
+  if (ring > kMaxRing) ring = kMaxRing;
+  p.ring = static_cast<int>(ring);
+  *smem_bytes = static_cast<size_t>(ring * tile_elems * 4 + fixed);
   *out = p;
-  return p.pitch <= 256 && p.rows_in <= 256 && tile_elems < 65536 && *smem_bytes <= 200 * 1024;
+  return p.pitch <= 256 && p.rows_in <= 256 && tile_elems < 65536 && ring >= 2;
 }
 
 }  // namespace
@@ -233,14 +322,17 @@ cudaError_t launch_im2col_quantize_tma(const void* x, const ConvGeom& g, uint32_
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return cudaErrorNotSupported;
-  static size_t configured = 0;
-  if (smem > 48 * 1024 && smem > configured) {
-    cudaError_t e = cudaFuncSetAttribute(im2col_quantize_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(im2col_quantize_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 208 * 1024);
     if (e != cudaSuccess) return e;
-    configured = 200 * 1024;
+    configured = true;
   }
-  dim3 grid(static_cast<unsigned>(static_cast<int64_t>(g.B) * p.yo_blocks), static_cast<unsigned>(p.splits));
-  im2col_quantize_tma_kernel<<<grid, 256, smem, stream>>>(map, g, p, bits, ld_words, scales, ld_scales, scale_bf16);
+  const int64_t n_items = static_cast<int64_t>(g.B) * p.yo_blocks * p.splits;
+  if (n_items > (int64_t{1} << 30)) return cudaErrorNotSupported;
+  const unsigned grid = static_cast<unsigned>(n_items < 2 * sms ? n_items : 2 * sms);     // two persistent CTAs per SM
+  im2col_quantize_tma_kernel<<<grid, kThreadsTma, smem, stream>>>(map, g, p, static_cast<int>(n_items), p.ring, bits, ld_words,
+                                                                  scales, ld_scales, scale_bf16);
   return cudaGetLastError();
 }
 
