@@ -329,9 +329,9 @@ im2col_quantize_tiled_kernel(const void* __restrict__ x, int x_bf16, const ConvG
       uint32_t word = 0;
       float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
       if (cc == kTileCC && g.kh == 3 && g.kw == 3) {
-        gather_word_dispatch<3, 3>(w, static_cast<uint32_t>(__cvta_generic_to_shared(base)), tp.rows_in * tp.span * 4, tp.span * 4, word, s0);
+        gather_word_dispatch<3, 3>(w, static_cast<uint32_t>(__cvta_generic_to_shared(base)), tp.rows_in * tp.span * 4, tp.span * 4, 0u, word, s0);
       } else if (cc == kTileCC && taps == 1) {
-        gather_word_dispatch<1, 1>(w, static_cast<uint32_t>(__cvta_generic_to_shared(base)), tp.rows_in * tp.span * 4, tp.span * 4, word, s0);
+        gather_word_dispatch<1, 1>(w, static_cast<uint32_t>(__cvta_generic_to_shared(base)), tp.rows_in * tp.span * 4, tp.span * 4, 0u, word, s0);
       } else if (nk == 32) {
 #pragma unroll
         for (int e = 0; e < 32; e += 4) {

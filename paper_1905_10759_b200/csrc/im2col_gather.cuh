@@ -11,8 +11,11 @@ namespace hbmm {
 // immediate).  Each element costs one shared-memory load, one add of +0 (so that -0 counts as +0 and
 // the sign bit alone decides Sign(x): x >= 0 <=> bit clear), one funnel shift that collects the sign
 // bit, and one add of |x|.  Returns the packed word (bit e = 1 <=> x >= 0) and the sum of |x|.
-template <int KH, int KW, int WORD>
-__device__ __forceinline__ void gather_word_static(uint32_t base, uint32_t cs_bytes, uint32_t pitch_bytes, uint32_t& word, float& sum) {
+// MASKED: the tile has no zero halo; bit j of `mask` says that filter column j, bit 8 + i that filter
+// row i lies inside the image for this pixel, and taps outside are taken as 0 without being loaded.
+template <int KH, int KW, int WORD, bool MASKED>
+__device__ __forceinline__ void gather_word_static(uint32_t base, uint32_t cs_bytes, uint32_t pitch_bytes, uint32_t mask,
+                                                   uint32_t& word, float& sum) {
   constexpr int T = KH * KW;
   uint32_t pat = 0;
   float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
@@ -23,8 +26,9 @@ __device__ __forceinline__ void gather_word_static(uint32_t base, uint32_t cs_by
     for (int u = 0; u < 4; u++) {
       const int k = 32 * WORD + e + u, c = k / T, t = k % T, i = t / KW, j = t % KW;
       const uint32_t row = base + c * cs_bytes + i * pitch_bytes;
-      float x;
-      asm volatile("ld.shared.f32 %0, [%1];" : "=f"(x) : "r"(row + 4 * j));   // the constant folds into the load
+      float x = 0.0f;
+      if (!MASKED || ((mask >> j) & (mask >> (8 + i)) & 1u))
+        asm volatile("ld.shared.f32 %0, [%1];" : "=f"(x) : "r"(row + 4 * j));   // the constant folds into the load
       v[u] = x + 0.0f;
       pat = __funnelshift_l(__float_as_uint(v[u]), pat, 1);     // pat = pat << 1 | sign bit
     }
@@ -35,12 +39,12 @@ __device__ __forceinline__ void gather_word_static(uint32_t base, uint32_t cs_by
 }
 
 // w (warp-uniform) selects the word of the chunk: KH * KW words per 32 channels.
-template <int KH, int KW, int WORD = 0>
-__device__ __forceinline__ void gather_word_dispatch(int w, uint32_t base, uint32_t cs_bytes, uint32_t pitch_bytes, uint32_t& word,
-                                                     float& sum) {
+template <int KH, int KW, bool MASKED = false, int WORD = 0>
+__device__ __forceinline__ void gather_word_dispatch(int w, uint32_t base, uint32_t cs_bytes, uint32_t pitch_bytes, uint32_t mask,
+                                                     uint32_t& word, float& sum) {
   if constexpr (WORD < KH * KW) {
-    if (w == WORD) gather_word_static<KH, KW, WORD>(base, cs_bytes, pitch_bytes, word, sum);
-    else gather_word_dispatch<KH, KW, WORD + 1>(w, base, cs_bytes, pitch_bytes, word, sum);
+    if (w == WORD) gather_word_static<KH, KW, WORD, MASKED>(base, cs_bytes, pitch_bytes, mask, word, sum);
+    else gather_word_dispatch<KH, KW, MASKED, WORD + 1>(w, base, cs_bytes, pitch_bytes, mask, word, sum);
   }
 }
 

@@ -30,6 +30,8 @@ struct Plan {
   int chunks_per_split;
   int n_chunks;           // ceil(C / 32)
   int ring;               // tile buffers per CTA
+  int flat;               // 1: whole channel planes staged by one bulk copy per chunk, no halo (pitch = W, rows_in = H)
+  int tile_stride;        // floats between ring buffers (tile rounded up to 128 bytes)
 };
 
 __device__ __forceinline__ void store_scale(void* scales, int bf16, int64_t idx, float v) {
@@ -59,12 +61,13 @@ __device__ __forceinline__ ItemCoords item_coords(int item, const Plan& tp) {
 }
 
 __global__ void __launch_bounds__(kThreadsTma, 2)
-im2col_quantize_tma_kernel(const __grid_constant__ CUtensorMap x_map, const ConvGeom g, const Plan tp, int n_items, int ring,
+im2col_quantize_tma_kernel(const __grid_constant__ CUtensorMap x_map, const float* __restrict__ x, const ConvGeom g, const Plan tp,
+                           int n_items, int ring,
                            uint32_t* __restrict__ bits, int64_t ld_words, void* __restrict__ scales, int64_t ld_scales,
                            int scale_bf16) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int taps = g.kh * g.kw;
-  const int tile_elems = kCC * tp.rows_in * tp.pitch;           // floats per buffer; bytes are a multiple of 128
+  const int tile_elems = tp.tile_stride;                        // floats per ring buffer; bytes are a multiple of 128
   const int max_pixels = tp.RB * g.Wo;
   const int split_words = tp.chunks_per_split * taps;          // words an item produces per pixel (upper bound)
   const int ldo = split_words + 1;                             // odd-ish pitch: fewer bank conflicts on the column writes
@@ -77,7 +80,8 @@ im2col_quantize_tma_kernel(const __grid_constant__ CUtensorMap x_map, const Conv
   uint32_t* out_bits = reinterpret_cast<uint32_t*>(written + 2);                      // [max_pixels][ldo]
   float* out_scale = reinterpret_cast<float*>(out_bits + max_pixels * ldo);           // same shape
   unsigned short* off = reinterpret_cast<unsigned short*>(out_scale + max_pixels * ldo);    // [32 * taps]
-  unsigned short* pixoff = off + (kCC * taps + 1) / 2 * 2;                                  // [max_pixels]
+  short* pixoff = reinterpret_cast<short*>(off + (kCC * taps + 1) / 2 * 2);                 // [max_pixels]
+  unsigned short* pixmask = reinterpret_cast<unsigned short*>(pixoff + (max_pixels + 1) / 2 * 2);   // [max_pixels], flat mode
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cs = tp.rows_in * tp.pitch;
@@ -97,14 +101,26 @@ im2col_quantize_tma_kernel(const __grid_constant__ CUtensorMap x_map, const Conv
   // pixel of an item -> tile offset of its first tap (channel 0, filter row 0, column 0)
   for (int pix = threadIdx.x; pix < max_pixels; pix += blockDim.x) {
     const int ry = pix / g.Wo, xo = pix - ry * g.Wo;
-    pixoff[pix] = static_cast<unsigned short>(ry * g.sh * tp.pitch + xo + tp.x0);
+    if (!tp.flat) {
+      pixoff[pix] = static_cast<short>(ry * g.sh * tp.pitch + xo + tp.x0);
+      pixmask[pix] = 0;
+    } else {
+      // no halo: the offset of tap (0, 0) may point before the plane; the masks say which taps exist
+      const int y0 = ry * g.sh - g.ph, x0 = xo - g.pw;
+      pixoff[pix] = static_cast<short>(y0 * tp.pitch + x0);
+      unsigned m = 0;
+      for (int j = 0; j < g.kw; j++) if (x0 + j >= 0 && x0 + j < g.W) m |= 1u << j;
+      for (int i = 0; i < g.kh; i++) if (y0 + i >= 0 && y0 + i < g.H) m |= 1u << (8 + i);
+      pixmask[pix] = static_cast<unsigned short>(m);
+    }
   }
   __syncthreads();
 
   if (warp == kLoaderWarp) {
     // =========================== loader ===========================
     if (lane == 0) {
-      const uint32_t tile_bytes = static_cast<uint32_t>(tile_elems) * 4;
+      const uint32_t tile_bytes = static_cast<uint32_t>(kCC) * tp.rows_in * tp.pitch * 4;
+      const int64_t plane = static_cast<int64_t>(g.H) * g.W;
       asm volatile("prefetch.tensormap [%0];" ::"l"(&x_map) : "memory");
       int s = 0;
       uint32_t round = 0;
@@ -117,8 +133,12 @@ im2col_quantize_tma_kernel(const __grid_constant__ CUtensorMap x_map, const Conv
           mbar_arrive_expect_tx(&full[s], tile_bytes);
           // x starts at -(x0 + pw), a multiple of 4 elements = 16 bytes; y may be negative too; what lies
           // outside the tensor (halo, channels past C) arrives as zeros
-          tma_load_4d(tile0 + static_cast<size_t>(s) * tile_elems, &x_map, -(tp.x0 + g.pw), ic.yo0 * g.sh - g.ph,
-                      (ic.chunk_first + it) * kCC, ic.b, &full[s]);
+          if (tp.flat)   // 32 whole channel planes are one contiguous, 16-byte aligned run of the NCHW tensor
+            bulk_copy_g2s(tile0 + static_cast<size_t>(s) * tile_elems,
+                          x + (static_cast<int64_t>(ic.b) * g.C + (ic.chunk_first + it) * kCC) * plane, tile_bytes, &full[s]);
+          else
+            tma_load_4d(tile0 + static_cast<size_t>(s) * tile_elems, &x_map, -(tp.x0 + g.pw), ic.yo0 * g.sh - g.ph,
+                        (ic.chunk_first + it) * kCC, ic.b, &full[s]);
           issued++;
           if (++s == ring) { s = 0; round++; }
         }
@@ -164,16 +184,19 @@ im2col_quantize_tma_kernel(const __grid_constant__ CUtensorMap x_map, const Conv
         if (pix < pixels) {
           const int k_begin = w * 32;
           const int nk = (chunk_elems - k_begin < 32) ? chunk_elems - k_begin : 32;
-          const uint32_t po = pixoff[pix];                     // tile offset of the pixel's first tap, in elements
+          const int po = pixoff[pix];                          // tile offset of the pixel's first tap, in elements
+          const uint32_t pm = pixmask[pix];
           uint32_t word = 0;
           float mean;
           if (cc == kCC && g.kh == 3 && g.kw == 3) {
             float sum;
-            gather_word_dispatch<3, 3>(w, t_addr + po * 4, cs * 4, tp.pitch * 4, word, sum);
+            if (tp.flat) gather_word_dispatch<3, 3, true>(w, t_addr + po * 4, cs * 4, tp.pitch * 4, pm, word, sum);
+            else gather_word_dispatch<3, 3, false>(w, t_addr + po * 4, cs * 4, tp.pitch * 4, 0u, word, sum);
             mean = sum * 0.03125f;
           } else if (cc == kCC && taps == 1) {
             float sum;
-            gather_word_dispatch<1, 1>(w, t_addr + po * 4, cs * 4, tp.pitch * 4, word, sum);
+            if (tp.flat) gather_word_dispatch<1, 1, true>(w, t_addr + po * 4, cs * 4, tp.pitch * 4, pm, word, sum);
+            else gather_word_dispatch<1, 1, false>(w, t_addr + po * 4, cs * 4, tp.pitch * 4, 0u, word, sum);
             mean = sum * 0.03125f;
           } else {
             const float* base = t + po;
@@ -260,15 +283,23 @@ im2col_quantize_tma_kernel(const __grid_constant__ CUtensorMap x_map, const Conv
 
 inline int round_up4(int v) { return (v + 3) / 4 * 4; }
 
-bool make_plan(const ConvGeom& g, int sms, Plan* out, size_t* smem_bytes) {
+bool make_plan(const ConvGeom& g, int sms, bool flat, Plan* out, size_t* smem_bytes) {
   Plan p;
-  p.RB = 112 / g.Wo;
-  if (p.RB < 1) p.RB = 1;
-  if (p.RB > g.Ho) p.RB = g.Ho;
-  p.rows_in = (p.RB - 1) * g.sh + g.kh;
-  const int span = g.Wo - 1 + g.kw;                            // input columns the block's taps touch (stride 1 along x)
-  p.x0 = round_up4(g.pw) - g.pw;
-  p.pitch = round_up4(p.x0 + span);
+  p.flat = flat ? 1 : 0;
+  if (flat) {
+    p.RB = g.Ho;                                               // an item covers the whole image
+    p.rows_in = g.H;
+    p.x0 = 0;
+    p.pitch = g.W;
+  } else {
+    p.RB = 112 / g.Wo;
+    if (p.RB < 1) p.RB = 1;
+    if (p.RB > g.Ho) p.RB = g.Ho;
+    p.rows_in = (p.RB - 1) * g.sh + g.kh;
+    const int span = g.Wo - 1 + g.kw;                          // input columns the item's taps touch (stride 1 along x)
+    p.x0 = round_up4(g.pw) - g.pw;
+    p.pitch = round_up4(p.x0 + span);
+  }
   p.yo_blocks = (g.Ho + p.RB - 1) / p.RB;
   p.n_chunks = (g.C + kCC - 1) / kCC;
   const int64_t row_blocks = static_cast<int64_t>(g.B) * p.yo_blocks;
@@ -278,29 +309,40 @@ bool make_plan(const ConvGeom& g, int sms, Plan* out, size_t* smem_bytes) {
   p.splits = (p.n_chunks + p.chunks_per_split - 1) / p.chunks_per_split;
   const int taps = g.kh * g.kw;
   const int64_t tile_elems = static_cast<int64_t>(kCC) * p.rows_in * p.pitch;
-  // everything but the tile ring: barriers, staging arrays of one item, offset table
-  const int64_t fixed = (2 * kMaxRing + 4) * 8 + 2LL * p.RB * g.Wo * (p.chunks_per_split * taps + 1) * 4 +
-                        static_cast<int64_t>(kCC) * taps * 2 + 2LL * p.RB * g.Wo + 32;
+  p.tile_stride = static_cast<int>((tile_elems + 31) / 32 * 32);
+  const int64_t max_pixels = static_cast<int64_t>(p.RB) * g.Wo;
+  // everything but the tile ring: barriers, staging arrays of one item, offset / pixel tables
+  const int64_t fixed = (2 * kMaxRing + 4) * 8 + 2 * max_pixels * (p.chunks_per_split * taps + 1) * 4 +
+                        static_cast<int64_t>(kCC) * taps * 2 + 4 * max_pixels + 64;
   const int64_t budget = 100 * 1024;                           // two CTAs per SM: one computes while the other synchronises or writes
-  int64_t ring = (budget - fixed) / (tile_elems * 4);
+  int64_t ring = (budget - fixed) / (p.tile_stride * 4);
   if (ring > kMaxRing) ring = kMaxRing;
   p.ring = static_cast<int>(ring);
-  *smem_bytes = static_cast<size_t>(ring * tile_elems * 4 + fixed);
+  *smem_bytes = static_cast<size_t>(ring * p.tile_stride * 4 + fixed);
   *out = p;
-  return p.pitch <= 256 && p.rows_in <= 256 && tile_elems < 65536 && ring >= 2;
+  // offsets are 16-bit (signed for the pixel table)
+  return (flat || (p.pitch <= 256 && p.rows_in <= 256)) && tile_elems < 32768 && max_pixels < 32768 && ring >= 2;
+}
+
+// 0: not supported, 1: tensor-copy tiles with halo, 2: flat channel planes
+int tma_mode(const void* x, int x_bf16, const ConvGeom& g, int32_t beta) {
+  const int64_t K = static_cast<int64_t>(g.C) * g.kh * g.kw;
+  if (x_bf16 || beta != 32 || beta >= K || g.sw != 1 || reinterpret_cast<uintptr_t>(x) % 16 != 0) return 0;
+  Plan p;
+  size_t smem;
+  if (g.W % 4 == 0 && encode_tiled_fn() != nullptr && make_plan(g, 148, false, &p, &smem)) return 1;
+  // small images whose rows are not multiples of 16 bytes: whole planes, masked 3x3 / 1x1 gather
+  const bool filt = (g.kh == 3 && g.kw == 3) || (g.kh == 1 && g.kw == 1);
+  if (filt && g.C % kCC == 0 && (static_cast<int64_t>(g.C) * g.H * g.W) % 4 == 0 && make_plan(g, 148, true, &p, &smem)) return 2;
+  return 0;
 }
 
 }  // namespace
 
-// fp32 input whose rows start on 16-byte boundaries (a tensor map wants 16-byte strides), stride 1
-// along x, groups of exactly one K-word.
+// fp32 input, stride 1 along x, groups of exactly one K-word; rows that are multiples of 16 bytes (a
+// tensor map wants 16-byte strides), or small images with 3x3 / 1x1 filters and whole 32-channel chunks.
 bool im2col_quantize_tma_supported(const void* x, int x_bf16, const ConvGeom& g, int32_t beta) {
-  const int64_t K = static_cast<int64_t>(g.C) * g.kh * g.kw;
-  if (x_bf16 || beta != 32 || beta >= K || g.sw != 1 || g.W % 4 != 0 || reinterpret_cast<uintptr_t>(x) % 16 != 0) return false;
-  if (encode_tiled_fn() == nullptr) return false;
-  Plan p;
-  size_t smem;
-  return make_plan(g, 148, &p, &smem);
+  return tma_mode(x, x_bf16, g, beta) != 0;
 }
 
 cudaError_t launch_im2col_quantize_tma(const void* x, const ConvGeom& g, uint32_t* bits, int64_t ld_words, void* scales,
@@ -308,31 +350,34 @@ cudaError_t launch_im2col_quantize_tma(const void* x, const ConvGeom& g, uint32_
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int mode = tma_mode(x, 0, g, 32);
   Plan p;
   size_t smem;
-  if (!make_plan(g, sms, &p, &smem)) return cudaErrorNotSupported;
-  CUtensorMap map;
-  const cuuint64_t dims[4] = {static_cast<cuuint64_t>(g.W), static_cast<cuuint64_t>(g.H), static_cast<cuuint64_t>(g.C),
-                              static_cast<cuuint64_t>(g.B)};
-  const cuuint64_t strides[3] = {static_cast<cuuint64_t>(g.W) * 4, static_cast<cuuint64_t>(g.H) * g.W * 4,
-                                 static_cast<cuuint64_t>(g.C) * g.H * g.W * 4};
-  const cuuint32_t box[4] = {static_cast<cuuint32_t>(p.pitch), static_cast<cuuint32_t>(p.rows_in), kCC, 1};
-  const cuuint32_t elem[4] = {1, 1, 1, 1};
-  if (encode_tiled_fn()(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<void*>(x), dims, strides, box, elem,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-    return cudaErrorNotSupported;
+  if (mode == 0 || !make_plan(g, sms, mode == 2, &p, &smem)) return cudaErrorNotSupported;
+  CUtensorMap map{};
+  if (mode == 1) {
+    const cuuint64_t dims[4] = {static_cast<cuuint64_t>(g.W), static_cast<cuuint64_t>(g.H), static_cast<cuuint64_t>(g.C),
+                                static_cast<cuuint64_t>(g.B)};
+    const cuuint64_t strides[3] = {static_cast<cuuint64_t>(g.W) * 4, static_cast<cuuint64_t>(g.H) * g.W * 4,
+                                   static_cast<cuuint64_t>(g.C) * g.H * g.W * 4};
+    const cuuint32_t box[4] = {static_cast<cuuint32_t>(p.pitch), static_cast<cuuint32_t>(p.rows_in), kCC, 1};
+    const cuuint32_t elem[4] = {1, 1, 1, 1};
+    if (encode_tiled_fn()(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<void*>(x), dims, strides, box, elem,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaErrorNotSupported;
+  }
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(im2col_quantize_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 208 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(im2col_quantize_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 104 * 1024);
     if (e != cudaSuccess) return e;
     configured = true;
   }
   const int64_t n_items = static_cast<int64_t>(g.B) * p.yo_blocks * p.splits;
   if (n_items > (int64_t{1} << 30)) return cudaErrorNotSupported;
   const unsigned grid = static_cast<unsigned>(n_items < 2 * sms ? n_items : 2 * sms);     // two persistent CTAs per SM
-  im2col_quantize_tma_kernel<<<grid, kThreadsTma, smem, stream>>>(map, g, p, static_cast<int>(n_items), p.ring, bits, ld_words,
-                                                                  scales, ld_scales, scale_bf16);
+  im2col_quantize_tma_kernel<<<grid, kThreadsTma, smem, stream>>>(map, static_cast<const float*>(x), g, p, static_cast<int>(n_items),
+                                                                  p.ring, bits, ld_words, scales, ld_scales, scale_bf16);
   return cudaGetLastError();
 }
 

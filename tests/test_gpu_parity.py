@@ -295,6 +295,11 @@ CONV_CASES = [
     (1, 64, 12, 12, 16, 1, 1, 1, 0, 32, 32, True, False),   # 1x1
     (3, 70, 16, 12, 33, 3, 3, 1, 0, 32, 64, True, False),   # no padding, ragged channels, beta_w = 64
     (2, 64, 8, 8, 16, 3, 3, 1, 1, 32, 32, None, False),     # zeros of both signs in the input
+    # ... and with whole channel planes staged by bulk copies when rows are not multiples of 16 bytes
+    (2, 64, 7, 7, 24, 3, 3, 1, 1, 32, 32, True, False),
+    (3, 96, 14, 14, 40, 3, 3, 1, 1, 32, 32, True, False),
+    (2, 32, 9, 10, 16, 1, 1, 1, 0, 32, 32, True, False),
+    (2, 64, 7, 7, 24, 3, 3, 1, 0, 32, 32, None, False),     # no padding, zeros of both signs
     # HBWN with whole 64-channel blocks: no im2col matrix, tiles fetched by im2col-mode tensor copies
     (3, 128, 7, 7, 72, 3, 3, 1, 1, 1, 32, True, False),     # two channel blocks, tiles span images, ragged M and N
     (2, 64, 9, 9, 40, 3, 3, 2, 0, 1, 32, True, True),       # stride 2, no padding
