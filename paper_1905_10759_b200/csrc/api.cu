@@ -299,9 +299,8 @@ hbmm_status hbmm_conv_im2col(const void* x, int32_t x_dtype, const hbmm_conv_geo
   hbmm_operand A{};
   A.rows = L.M; A.K = L.K; A.beta = beta_a; A.scale_dtype = a_scale_dtype;
   if (beta_a == 1 && L.implicit) {
-    if (launch_nchw_to_nhwc_bf16(x, x_dtype == HBMM_BF16, cg, workspace, L.Cp, s) != cudaSuccess) return HBMM_ERR_CUDA;
-    return launch_hbwn_umma_conv(workspace, L.Cp, cg, view_of(W), C_out, ldc, static_cast<char*>(workspace) + L.operand_bytes,
-                                 s) == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
+    return launch_hbwn_umma_conv(x, x_dtype == HBMM_BF16, workspace, L.Cp, cg, view_of(W), C_out, ldc,
+                                 static_cast<char*>(workspace) + L.operand_bytes, s) == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
   }
   if (beta_a == 1) {
     if (launch_im2col_bf16(x, x_dtype == HBMM_BF16, cg, workspace, L.ld_dense, s) != cudaSuccess) return HBMM_ERR_CUDA;

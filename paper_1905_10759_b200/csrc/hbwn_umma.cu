@@ -21,6 +21,7 @@
 #include <cuda_bf16.h>
 #include "kernels.h"
 #include "tensor_map.h"
+#include "nhwc.cuh"
 #include "umma_common.cuh"
 
 namespace hbmm {
@@ -77,10 +78,8 @@ struct Smem {
 // row (plain mode) or channel c = cb * 64 + q at filter tap t, k = c * taps + t (convolution mode,
 // kb = t * cblocks + cb).  The element is +-piece_i(deltaW[n, k / beta]); zero past K / C and past N.
 template <int TN>
-__global__ void __launch_bounds__(256)
-prepare_w_pieces_kernel(const Args g, unsigned char* __restrict__ out) {
+__device__ __forceinline__ void prepare_w_pieces_block(const Args& g, unsigned char* __restrict__ out, int64_t kb, int64_t tile_n) {
   using S = Smem<TN>;
-  const int64_t kb = blockIdx.x, tile_n = blockIdx.y;
   unsigned char* base = out + (tile_n * g.n_kb + kb) * S::B_STAGE;
   const int64_t tap = g.conv ? kb / g.cblocks : 0;
   const int64_t q0 = (g.conv ? kb - tap * g.cblocks : kb) * KB;     // first channel / element of the block
@@ -112,6 +111,37 @@ prepare_w_pieces_kernel(const Args g, unsigned char* __restrict__ out) {
 #pragma unroll
     for (int i = 0; i < 3; i++)
       *reinterpret_cast<uint4*>(swz(base + i * S::B_PIECE, row, piece)) = make_uint4(o[i][0], o[i][1], o[i][2], o[i][3]);
+  }
+}
+
+template <int TN>
+__global__ void __launch_bounds__(256)
+prepare_w_pieces_kernel(const Args g, unsigned char* __restrict__ out) {
+  prepare_w_pieces_block<TN>(g, out, blockIdx.x, blockIdx.y);
+}
+
+// Convolution front end in one launch: the first `n_copy` blocks transpose the input to NHWC bf16, the
+// rest lay out the weight pieces.  The two jobs are independent, so the small weight job hides behind
+// the copy instead of costing a launch of its own.
+struct CopyArgs {
+  const void* x; int32_t x_bf16, C, Cp; int64_t HW; unsigned short* out;
+  int32_t gx, gy;          // pixel blocks and channel blocks per image
+  int64_t n_copy;
+};
+template <int TN>
+__global__ void __launch_bounds__(256)
+nhwc_and_pieces_kernel(const CopyArgs c, const Args g, unsigned char* __restrict__ w_out) {
+  __shared__ unsigned short tile[kNhwcCB][kNhwcPitch];
+  const int64_t blk = blockIdx.x;
+  if (blk < c.n_copy) {
+    const int64_t per_image = static_cast<int64_t>(c.gx) * c.gy;
+    const int64_t b = blk / per_image, r = blk - b * per_image;
+    const int cblock = static_cast<int>(r / c.gx);
+    nchw_to_nhwc_block(c.x, c.x_bf16, c.C, c.HW, c.Cp, c.out, b, cblock, r - static_cast<int64_t>(cblock) * c.gx, tile);
+  } else {
+    const int64_t j = blk - c.n_copy;
+    const int64_t tile_n = j / g.n_kb;
+    prepare_w_pieces_block<TN>(g, w_out, j - tile_n * g.n_kb, tile_n);
   }
 }
 
@@ -346,7 +376,7 @@ Args make_conv_args(const ConvGeom& c, const PackedView& W, float* C, int64_t ld
 }
 
 template <int TN>
-cudaError_t launch(Args g, const CUtensorMap& a_map, void* workspace, cudaStream_t stream) {
+cudaError_t launch(Args g, const CUtensorMap& a_map, void* workspace, cudaStream_t stream, const CopyArgs* copy = nullptr) {
   using S = Smem<TN>;
   static bool configured = false;
   static int sms = 0;
@@ -360,7 +390,13 @@ cudaError_t launch(Args g, const CUtensorMap& a_map, void* workspace, cudaStream
   }
   const int64_t tiles_n = (g.N + TN - 1) / TN, n_kb = g.n_kb;
   dim3 pgrid(static_cast<unsigned>(n_kb), static_cast<unsigned>(tiles_n));
-  prepare_w_pieces_kernel<TN><<<pgrid, 256, 0, stream>>>(g, static_cast<unsigned char*>(workspace));
+  if (copy) {
+    const int64_t blocks = copy->n_copy + n_kb * tiles_n;
+    if (blocks > 0x7fffffff) return cudaErrorNotSupported;
+    nhwc_and_pieces_kernel<TN><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(*copy, g, static_cast<unsigned char*>(workspace));
+  } else {
+    prepare_w_pieces_kernel<TN><<<pgrid, 256, 0, stream>>>(g, static_cast<unsigned char*>(workspace));
+  }
   g.w_prep = static_cast<const unsigned char*>(workspace);
   const int64_t tiles = ((g.M + TM - 1) / TM) * tiles_n;
   const unsigned grid = static_cast<unsigned>(tiles < sms ? tiles : sms);
@@ -405,12 +441,18 @@ size_t hbwn_umma_conv_workspace_bytes(const ConvGeom& c, const PackedView& W) {
   return prep_bytes<64>(g);
 }
 
-cudaError_t launch_hbwn_umma_conv(const void* x_nhwc, int Cp, const ConvGeom& c, const PackedView& W, float* C, int64_t ldc,
-                                  void* workspace, cudaStream_t stream) {
+cudaError_t launch_hbwn_umma_conv(const void* x, int x_bf16, void* x_nhwc, int Cp, const ConvGeom& c, const PackedView& W, float* C,
+                                  int64_t ldc, void* workspace, cudaStream_t stream) {
   const Args g = make_conv_args(c, W, C, ldc);
   CUtensorMap a_map;
   if (!make_conv_map(x_nhwc, c, Cp, &a_map)) return cudaErrorNotSupported;
-  return launch<64>(g, a_map, workspace, stream);
+  CopyArgs cp;
+  cp.x = x; cp.x_bf16 = x_bf16; cp.C = c.C; cp.Cp = Cp; cp.HW = static_cast<int64_t>(c.H) * c.W;
+  cp.out = static_cast<unsigned short*>(x_nhwc);
+  cp.gx = static_cast<int32_t>((cp.HW + kNhwcPB - 1) / kNhwcPB);
+  cp.gy = (Cp + kNhwcCB - 1) / kNhwcCB;
+  cp.n_copy = static_cast<int64_t>(cp.gx) * cp.gy * c.B;
+  return launch<64>(g, a_map, workspace, stream, &cp);
 }
 
 cudaError_t read_hbwn_umma_error(int* code) {

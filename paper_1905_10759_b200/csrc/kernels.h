@@ -71,13 +71,14 @@ size_t hbwn_umma_workspace_bytes(const DenseView& A, const PackedView& W);
 cudaError_t launch_hbwn_umma(const DenseView& A, const PackedView& W, float* C, int64_t ldc, void* workspace,
                              cudaStream_t stream);
 
-// HBWN convolution without the im2col matrix: NCHW -> NHWC bf16 copy (Cp = channels rounded up to 8),
-// then the tcgen05 kernel reads its activation tiles with im2col-mode tensor copies.
+// HBWN convolution without the im2col matrix: NCHW -> NHWC bf16 copy (Cp = channels rounded up to 8;
+// launch_hbwn_umma_conv does it in the same launch as the weight-piece layout), then the tcgen05 kernel
+// reads its activation tiles from x_nhwc with im2col-mode tensor copies.
 cudaError_t launch_nchw_to_nhwc_bf16(const void* x, int x_bf16, const ConvGeom& g, void* out, int Cp, cudaStream_t stream);
 bool hbwn_umma_conv_supported(const ConvGeom& g, const PackedView& W);
 size_t hbwn_umma_conv_workspace_bytes(const ConvGeom& g, const PackedView& W);
-cudaError_t launch_hbwn_umma_conv(const void* x_nhwc, int Cp, const ConvGeom& g, const PackedView& W, float* C, int64_t ldc,
-                                  void* workspace, cudaStream_t stream);
+cudaError_t launch_hbwn_umma_conv(const void* x, int x_bf16, void* x_nhwc, int Cp, const ConvGeom& g, const PackedView& W, float* C,
+                                  int64_t ldc, void* workspace, cudaStream_t stream);
 
 // im2col gather fused with Hadamard binarization (packed output), and bf16 dense gather.
 cudaError_t launch_im2col_quantize(const void* x, int x_bf16, const ConvGeom& g, int32_t beta,
