@@ -1,0 +1,137 @@
+"""GPU parity at full workload sizes, in the launch configuration the benchmark times: the library runs
+the whole problem, the CPU oracle recomputes sampled output rows one by one from the same seeded
+inputs (whole images for the convolutions, scattered rows for the matrix products)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1905_10759_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+RTOL = 1e-5
+BETA = 32
+
+
+@pytest.fixture(scope="module")
+def hb():
+    from paper_1905_10759_b200 import hbmm
+    yield hbmm
+    assert hbmm.last_device_error() == 0
+
+
+def _gu():
+    import gpu_util
+    return gpu_util
+
+
+def _sample_rows(M, n, seed):
+    """First and last rows, rows around 128-row tile borders, and random ones."""
+    rng = np.random.default_rng(seed)
+    fixed = [0, 1, 127, 128, 129, M // 2, M - 129, M - 128, M - 2, M - 1]
+    rows = set(r for r in fixed if 0 <= r < M)
+    while len(rows) < min(n, M):
+        rows.add(int(rng.integers(0, M)))
+    return np.array(sorted(rows))
+
+
+# ------------------------------------------------------------------ the benchmark's convolutions, batch 64
+@pytest.mark.parametrize("li", [0, 1, 2, 3])
+@pytest.mark.parametrize("signed", [False, True])
+def test_resnet_conv_hbmm_full_batch(hb, li, signed):
+    gu = _gu()
+    s = inputs.resnet18_convs(64)[li]
+    x = inputs.conv_activation(s, inputs.SEEDS["resnet_hbmm"][0] + li, signed=signed)
+    w = inputs.he_normal(s.N, s.K, inputs.SEEDS["resnet_hbmm"][1] + li)
+    Wop = hb.quantize(torch.from_numpy(w).cuda(), hb.alloc_operand(s.N, s.K, BETA, hb.F32))
+    geom = hb.make_geom(s.B, s.C, s.H, s.W, s.kh, s.kw, (s.stride, s.stride), (s.pad, s.pad))
+    ws = torch.empty(hb.conv_workspace_bytes(geom, BETA, hb.F32, Wop), dtype=torch.uint8, device="cuda")
+    C = torch.empty((s.M, s.N), device="cuda")
+    hb.conv_im2col(torch.from_numpy(x).cuda(), geom, BETA, hb.F32, Wop, C, ws)
+    torch.cuda.synchronize()
+    _, _, lw, ls = hb.operand_bytes(s.M, s.K, BETA, hb.F32)
+    bits = ws[: s.M * lw * 4].view(torch.int32).reshape(s.M, lw)
+    per_image = s.M // s.B
+    for b in (0, s.B // 2, s.B - 1):                       # whole images: first, middle, last
+        rows = oracle.im2col(x[b:b + 1], s.kh, s.kw, (s.stride, s.stride), (s.pad, s.pad))
+        da, sa = oracle.quantize(rows, BETA)
+        dw, sw = oracle.quantize(w, BETA)
+        c_ref, absref = oracle.hbmm_from_quantized(oracle.round_scales(da, "f32"), sa, BETA, oracle.round_scales(dw, "f32"), sw, BETA)
+        lo = b * per_image
+        assert np.array_equal(gu.host_bits(bits[lo: lo + per_image]), oracle.pack(sa, lw)), "packed activations of image %d" % b
+        gu.assert_close_rel_absref(C[lo: lo + per_image].cpu().numpy(), c_ref, absref, RTOL, "%s image %d" % (s.name, b))
+
+
+@pytest.mark.parametrize("li", [0, 1, 2, 3])
+def test_resnet_conv_hbwn_full_batch(hb, li):
+    gu = _gu()
+    s = inputs.resnet18_convs(64)[li]
+    x = inputs.conv_activation(s, inputs.SEEDS["resnet_hbwn"][0] + li, signed=(li % 2 == 1))
+    xb_bits, xb = inputs.as_bf16(x)
+    w = inputs.he_normal(s.N, s.K, inputs.SEEDS["resnet_hbmm"][1] + li)
+    Wop = hb.quantize(torch.from_numpy(w).cuda(), hb.alloc_operand(s.N, s.K, BETA, hb.F32))
+    geom = hb.make_geom(s.B, s.C, s.H, s.W, s.kh, s.kw, (s.stride, s.stride), (s.pad, s.pad))
+    ws = torch.empty(hb.conv_workspace_bytes(geom, 1, hb.F32, Wop), dtype=torch.uint8, device="cuda")
+    C = torch.empty((s.M, s.N), device="cuda")
+    xd = torch.from_numpy(xb_bits.view(np.int16)).view(torch.bfloat16).cuda()
+    hb.conv_im2col(xd, geom, 1, hb.F32, Wop, C, ws)
+    torch.cuda.synchronize()
+    dw, sw = oracle.quantize(w, BETA)
+    dw = oracle.round_scales(dw, "f32")
+    G = s.K // BETA
+    rtol = (BETA + G + 4) * 2 * gu.U
+    per_image = s.M // s.B
+    for b in (0, s.B // 2, s.B - 1):
+        rows = oracle.im2col(xb[b:b + 1], s.kh, s.kw, (s.stride, s.stride), (s.pad, s.pad))
+        c_ref, absref = oracle.hbwn_from_quantized(rows, dw, sw, BETA)
+        lo = b * per_image
+        gu.assert_close_rel_absref(C[lo: lo + per_image].cpu().numpy(), c_ref, absref, rtol, "%s image %d" % (s.name, b))
+
+
+# ------------------------------------------------------------------ square products and the FC stack
+@pytest.mark.parametrize("n,beta,sdt", [(4096, 32, 0), (4096, 128, 1), (8192, 64, 0)])
+def test_square_quantize_then_gemm_sampled_rows(hb, n, beta, sdt):
+    gu = _gu()
+    a = inputs.normal((n, n), inputs.SEEDS["square_sweep"][0] + n // 4096)
+    w = inputs.normal((n, n), inputs.SEEDS["square_sweep"][1] + n // 4096)
+    A = hb.quantize(torch.from_numpy(a).cuda(), hb.alloc_operand(n, n, beta, sdt))
+    W = hb.quantize(torch.from_numpy(w).cuda(), hb.alloc_operand(n, n, beta, sdt))
+    C = torch.empty((n, n), device="cuda")
+    ws = torch.empty(max(hb.gemm_workspace_bytes(A, W), 16), dtype=torch.uint8, device="cuda")
+    hb.gemm(A, W, C, ws)
+    torch.cuda.synchronize()
+    rows = _sample_rows(n, 24, n + beta)
+    # the oracle binarizes the same raw rows; stored scales are compared through the rounding the storage type applies
+    name = "f32" if sdt == hb.F32 else "bf16"
+    da, sa = oracle.quantize(a[rows], beta)
+    dw, sw = oracle.quantize(w, beta)
+    lw = A.bits.shape[1]
+    assert np.array_equal(gu.host_bits(A.bits[torch.from_numpy(rows).cuda()]), oracle.pack(sa, lw))
+    # products from the scales the GPU actually stored (isolates the contraction from the scale rounding)
+    G = n // beta
+    sa_gpu = A.scales[torch.from_numpy(rows).cuda()][:, :G].float().cpu().numpy().astype(np.float64)
+    sw_gpu = W.scales[:, :G].float().cpu().numpy().astype(np.float64)
+    tol_s = (int(np.ceil(np.log2(beta))) + 3) * gu.U + (2.0 ** -8 if name == "bf16" else 0.0)
+    assert np.all(np.abs(sa_gpu - da) <= tol_s * da + 1e-30)
+    c_ref, absref = oracle.hbmm_from_quantized(sa_gpu, sa, beta, sw_gpu, sw, beta)
+    gu.assert_close_rel_absref(C[torch.from_numpy(rows).cuda()].cpu().numpy(), c_ref, absref, RTOL, "square %d" % n)
+
+
+@pytest.mark.parametrize("batch", [1, 256])
+def test_alexnet_fc_stack(hb, batch):
+    gu = _gu()
+    beta = 64
+    for i, (K, N) in enumerate(inputs.ALEXNET_FC):
+        a = inputs.normal((batch, K), inputs.SEEDS["alexnet_fc"][0] + i)
+        w = inputs.he_normal(N, K, inputs.SEEDS["alexnet_fc"][1] + i)
+        A, da, sa = gu.oracle_operand(a, beta)
+        W, dw, sw = gu.oracle_operand(w, beta)
+        ldc = (N + 3) // 4 * 4
+        C = torch.empty((batch, ldc), device="cuda")
+        ws = torch.empty(max(hb.gemm_workspace_bytes(A, W), 16), dtype=torch.uint8, device="cuda")
+        hb.gemm(A, W, C, ws)
+        rows = _sample_rows(batch, 16, K + N)
+        c_ref, absref = oracle.hbmm_from_quantized(da[rows], sa[rows], beta, dw, sw, beta)
+        gu.assert_close_rel_absref(C[torch.from_numpy(rows).cuda()].cpu().numpy()[:, :N], c_ref, absref, RTOL,
+                                   "fc %dx%d batch %d" % (K, N, batch))
