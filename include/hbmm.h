@@ -53,9 +53,13 @@ typedef enum {
                            HBWN: weight sign XOR-ed into fp32 activations on the fp32 pipe              */
   HBMM_PATH_B1MMA = 2,  /* legacy warp-level mma.sync: b1 xor.popc, beta multiple of 128;
                            HBWN: bf16 mma.sync with per-group partial sums (bf16 activations only)      */
-  HBMM_PATH_TENSOR = 3  /* tcgen05 with TMEM accumulators: sign bits expanded to +-1 e4m3, group dots
+  HBMM_PATH_TENSOR = 3, /* tcgen05 with TMEM accumulators: sign bits expanded to +-1 e4m3, group dots
                            scaled in the epilogue; HBWN: bf16 activations x weights written as three
                            bf16 pieces +-d_i (delta = d1 + d2 + d3), one accumulation over all of K     */
+  HBMM_PATH_TENSOR_PREPARED = 4 /* HBMM_PATH_TENSOR, and the caller states that the workspace still holds
+                           the expanded weight operand an earlier HBMM_PATH_TENSOR / AUTO call with the
+                           same W, the same kind of A and this workspace left there (W unchanged
+                           since): the expansion kernel is skipped.  Results are undefined otherwise.  */
 } hbmm_path;
 
 /*

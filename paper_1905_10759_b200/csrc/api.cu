@@ -83,7 +83,9 @@ hbmm_status gemm_checked(const hbmm_operand* A, const hbmm_operand* W, float* C,
   if (W->beta == 1) return HBMM_ERR_UNSUPPORTED;  // the weight operand is always Hadamard-binary
   hbmm_status st = check_packed(W);
   if (st != HBMM_OK) return st;
-  if (path < HBMM_PATH_AUTO || path > HBMM_PATH_TENSOR) return HBMM_ERR_INVALID_ARG;
+  if (path < HBMM_PATH_AUTO || path > HBMM_PATH_TENSOR_PREPARED) return HBMM_ERR_INVALID_ARG;
+  const bool w_prepared = path == HBMM_PATH_TENSOR_PREPARED;
+  if (w_prepared) path = HBMM_PATH_TENSOR;
   if (A->beta == 1) {
     if (A->rows <= 0 || A->K <= 0 || !A->dense || A->ld_dense < A->K || !valid_dtype(A->dense_dtype))
       return HBMM_ERR_INVALID_ARG;
@@ -102,7 +104,7 @@ hbmm_status gemm_checked(const hbmm_operand* A, const hbmm_operand* W, float* C,
       case HBMM_PATH_TENSOR:
         if (!hbwn_umma_supported(dv, w)) return HBMM_ERR_UNSUPPORTED;
         if (!umma) return HBMM_ERR_WORKSPACE;
-        e = launch_hbwn_umma(dv, w, C, ldc, workspace, stream);
+        e = launch_hbwn_umma(dv, w, C, ldc, workspace, stream, w_prepared);
         break;
       default:
         if (umma) e = launch_hbwn_umma(dv, w, C, ldc, workspace, stream);
@@ -127,7 +129,7 @@ hbmm_status gemm_checked(const hbmm_operand* A, const hbmm_operand* W, float* C,
     case HBMM_PATH_TENSOR:
       if (!gemm_tensor_supported(a, w)) return HBMM_ERR_UNSUPPORTED;
       if (!workspace_ok(workspace, workspace_bytes, tensor_workspace(a, w))) return HBMM_ERR_WORKSPACE;
-      e = launch_gemm_tensor(a, w, C, ldc, workspace, stream);
+      e = launch_gemm_tensor(a, w, C, ldc, workspace, stream, w_prepared);
       break;
     default:
       // the tensor-core path needs its workspace; without one the integer-pipe path runs
@@ -311,6 +313,21 @@ hbmm_status hbmm_conv_im2col(const void* x, int32_t x_dtype, const hbmm_conv_geo
     A.ld_words = L.ld_words; A.ld_scales = L.ld_scales;
     hbmm_operand Aseg = A;
     if (!segments_compatible(&Aseg, W)) return HBMM_ERR_UNSUPPORTED;
+    // When the tensor-core contraction will run and the tensor-copy front end takes this input, the
+    // front end's launch also expands the weight operand (a few extra CTAs) and the contraction skips it.
+    const PackedView av = view_of(&A), wv = view_of(W);
+    void* gemm_ws = static_cast<char*>(workspace) + L.operand_bytes;
+    if (gemm_tensor_supported(av, wv) && L.gemm_bytes > 0 && L.gemm_bytes >= tensor_workspace(av, wv) &&
+        im2col_quantize_tma_supported(x, x_dtype == HBMM_BF16, cg, beta_a)) {
+      UmmaPrepJob job;
+      gemm_tensor_prep_job(av, wv, gemm_ws, &job);
+      if (job.n_stages * job.tiles_n <= 4096) {
+        if (launch_im2col_quantize_tma(x, cg, A.bits, A.ld_words, A.scales, A.ld_scales, a_scale_dtype == HBMM_BF16, s, &job) !=
+            cudaSuccess)
+          return HBMM_ERR_CUDA;
+        return launch_gemm_tensor(av, wv, C_out, ldc, gemm_ws, s, true) == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
+      }
+    }
     if (launch_im2col_quantize(x, x_dtype == HBMM_BF16, cg, beta_a, A.bits, A.ld_words, A.scales, A.ld_scales,
                                a_scale_dtype == HBMM_BF16, s) != cudaSuccess)
       return HBMM_ERR_CUDA;

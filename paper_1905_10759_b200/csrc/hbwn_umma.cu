@@ -376,7 +376,8 @@ Args make_conv_args(const ConvGeom& c, const PackedView& W, float* C, int64_t ld
 }
 
 template <int TN>
-cudaError_t launch(Args g, const CUtensorMap& a_map, void* workspace, cudaStream_t stream, const CopyArgs* copy = nullptr) {
+cudaError_t launch(Args g, const CUtensorMap& a_map, void* workspace, cudaStream_t stream, const CopyArgs* copy = nullptr,
+                   bool w_prepared = false) {
   using S = Smem<TN>;
   static bool configured = false;
   static int sms = 0;
@@ -394,7 +395,7 @@ cudaError_t launch(Args g, const CUtensorMap& a_map, void* workspace, cudaStream
     const int64_t blocks = copy->n_copy + n_kb * tiles_n;
     if (blocks > 0x7fffffff) return cudaErrorNotSupported;
     nhwc_and_pieces_kernel<TN><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(*copy, g, static_cast<unsigned char*>(workspace));
-  } else {
+  } else if (!w_prepared) {
     prepare_w_pieces_kernel<TN><<<pgrid, 256, 0, stream>>>(g, static_cast<unsigned char*>(workspace));
   }
   g.w_prep = static_cast<const unsigned char*>(workspace);
@@ -421,11 +422,11 @@ size_t hbwn_umma_workspace_bytes(const DenseView& A, const PackedView& W) {
 }
 
 cudaError_t launch_hbwn_umma(const DenseView& A, const PackedView& W, float* C, int64_t ldc, void* workspace,
-                             cudaStream_t stream) {
+                             cudaStream_t stream, bool w_prepared) {
   const Args g = make_args(A, W, C, ldc);
   CUtensorMap a_map;
   if (!make_a_map(g, &a_map)) return cudaErrorNotSupported;
-  return launch<64>(g, a_map, workspace, stream);
+  return launch<64>(g, a_map, workspace, stream, nullptr, w_prepared);
 }
 
 // Implicit-GEMM convolution: whole 64-channel blocks (every tile row is then 128 bytes of real

@@ -12,6 +12,7 @@
 #include "tensor_map.h"
 #include "umma_common.cuh"
 #include "im2col_gather.cuh"
+#include "gemm_umma_prep.cuh"
 
 namespace hbmm {
 namespace {
@@ -62,9 +63,18 @@ __device__ __forceinline__ ItemCoords item_coords(int item, const Plan& tp) {
 
 __global__ void __launch_bounds__(kThreadsTma, 2)
 im2col_quantize_tma_kernel(const __grid_constant__ CUtensorMap x_map, const float* __restrict__ x, const ConvGeom g, const Plan tp,
-                           int n_items, int ring,
+                           const __grid_constant__ UmmaPrepJob prep, int n_prep, int n_items, int ring,
                            uint32_t* __restrict__ bits, int64_t ld_words, void* __restrict__ scales, int64_t ld_scales,
                            int scale_bf16) {
+  // The first n_prep CTAs expand the weight operand of the contraction that follows (one task each:
+  // a stage of one column tile, one thread per weight row); they are scheduled first and leave at once.
+  if (static_cast<int>(blockIdx.x) < n_prep) {
+    const int st = blockIdx.x % prep.n_stages, tile_n = blockIdx.x / prep.n_stages;
+    if (prep.tn == 64) { if (threadIdx.x < 64) umma_prep::prepare_w_task<64>(prep.g, prep.out, st, tile_n, threadIdx.x); }
+    else if (threadIdx.x < 128) umma_prep::prepare_w_task<128>(prep.g, prep.out, st, tile_n, threadIdx.x);
+    return;
+  }
+  const int cta = blockIdx.x - n_prep, n_ctas = gridDim.x - n_prep;      // the persistent CTAs of the front end
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int taps = g.kh * g.kw;
   const int tile_elems = tp.tile_stride;                        // floats per ring buffer; bytes are a multiple of 128
@@ -126,7 +136,7 @@ im2col_quantize_tma_kernel(const __grid_constant__ CUtensorMap x_map, const floa
       uint32_t round = 0;
       int issued = 0;                                          // copies issued so far (for the abort path)
       bool ok = true;
-      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+      for (int item = cta; item < n_items && ok; item += n_ctas) {
         const ItemCoords ic = item_coords(item, tp);
         for (int it = 0; it < ic.n_my; it++) {
           if (round > 0 && !mbar_wait(&empty[s], (round & 1) ^ 1, abort_flag, 1)) { ok = false; break; }
@@ -160,7 +170,7 @@ im2col_quantize_tma_kernel(const __grid_constant__ CUtensorMap x_map, const floa
   // =========================== compute warps ===========================
   int s = 0;
   uint32_t round = 0, phase = 0;                               // ring position; parity of `computed` / `written`
-  for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+  for (int item = cta; item < n_items; item += n_ctas) {
     const ItemCoords ic = item_coords(item, tp);
     const int rows = (g.Ho - ic.yo0 < tp.RB) ? g.Ho - ic.yo0 : tp.RB;
     const int pixels = rows * g.Wo;
@@ -346,7 +356,7 @@ bool im2col_quantize_tma_supported(const void* x, int x_bf16, const ConvGeom& g,
 }
 
 cudaError_t launch_im2col_quantize_tma(const void* x, const ConvGeom& g, uint32_t* bits, int64_t ld_words, void* scales,
-                                       int64_t ld_scales, int scale_bf16, cudaStream_t stream) {
+                                       int64_t ld_scales, int scale_bf16, cudaStream_t stream, const UmmaPrepJob* prep) {
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -376,8 +386,16 @@ cudaError_t launch_im2col_quantize_tma(const void* x, const ConvGeom& g, uint32_
   const int64_t n_items = static_cast<int64_t>(g.B) * p.yo_blocks * p.splits;
   if (n_items > (int64_t{1} << 30)) return cudaErrorNotSupported;
   const unsigned grid = static_cast<unsigned>(n_items < 2 * sms ? n_items : 2 * sms);     // two persistent CTAs per SM
-  im2col_quantize_tma_kernel<<<grid, kThreadsTma, smem, stream>>>(map, static_cast<const float*>(x), g, p, static_cast<int>(n_items),
-                                                                  p.ring, bits, ld_words, scales, ld_scales, scale_bf16);
+  UmmaPrepJob job{};
+  int n_prep = 0;
+  if (prep) {
+    job = *prep;
+    n_prep = job.n_stages * job.tiles_n;
+    if (n_prep > 4096) return cudaErrorNotSupported;       // the caller expands large weight operands on its own
+  }
+  im2col_quantize_tma_kernel<<<grid + n_prep, kThreadsTma, smem, stream>>>(map, static_cast<const float*>(x), g, p, job, n_prep,
+                                                                           static_cast<int>(n_items), p.ring, bits, ld_words,
+                                                                           scales, ld_scales, scale_bf16);
   return cudaGetLastError();
 }
 

@@ -48,6 +48,26 @@ cudaError_t launch_gemm_b1(const PackedView& A, const PackedView& W, float* C, i
 cudaError_t launch_partials_b1(const PackedView& A, const PackedView& W, int32_t* D,
                                cudaStream_t stream);
 
+// Argument block of the tcgen05 HBMM kernel and of its weight-expansion routine.
+struct UmmaArgs {
+  const uint32_t* a_bits; const void* a_scales;
+  const uint32_t* w_bits; const void* w_scales;
+  float* C;
+  int64_t M, N, lda_w, ldw_w, lda_s, ldw_s, ldc;
+  int32_t a_bf16, w_bf16;
+  int32_t ra, rw;          // A group = segment / ra, W group = segment / rw
+  int64_t Ga, Gw;
+  int64_t n_words;         // K / 32 (K is a multiple of 32 on this path)
+  int64_t seg_words;       // K-words per segment
+  const unsigned char* w_prep;   // W expanded into [n tile][stage][stage bytes]
+};
+// The weight expansion as a job another kernel can run: n_stages x tiles_n tasks of tn threads each.
+struct UmmaPrepJob {
+  UmmaArgs g;
+  unsigned char* out;
+  int32_t tn, n_stages, tiles_n;
+};
+
 // Packed x packed contraction with +-1 e4m3 operands on the tensor cores (tcgen05 / TMEM).
 // read_*_umma_error copies a kernel family's device-side error word (0 = no bounded wait ever
 // expired); it synchronises.
@@ -55,8 +75,11 @@ cudaError_t read_gemm_umma_error(int* code);
 cudaError_t read_hbwn_umma_error(int* code);
 bool gemm_tensor_supported(const PackedView& A, const PackedView& W);
 size_t gemm_tensor_workspace_bytes(const PackedView& A, const PackedView& W);
+// w_prepared: the workspace already holds the expanded weight operand of exactly these operands (a
+// front-end kernel ran gemm_tensor_prep_job's tasks earlier on the same stream).
 cudaError_t launch_gemm_tensor(const PackedView& A, const PackedView& W, float* C, int64_t ldc, void* workspace,
-                               cudaStream_t stream);
+                               cudaStream_t stream, bool w_prepared = false);
+void gemm_tensor_prep_job(const PackedView& A, const PackedView& W, void* workspace, UmmaPrepJob* job);
 
 // Dense x packed contraction (HBWN), three kernels:
 //   select : sign bit XOR-ed into fp32 activations on the fp32 pipe (any dense dtype);
@@ -69,7 +92,7 @@ cudaError_t launch_hbwn_mma(const DenseView& A, const PackedView& W, float* C, i
 bool hbwn_umma_supported(const DenseView& A, const PackedView& W);
 size_t hbwn_umma_workspace_bytes(const DenseView& A, const PackedView& W);
 cudaError_t launch_hbwn_umma(const DenseView& A, const PackedView& W, float* C, int64_t ldc, void* workspace,
-                             cudaStream_t stream);
+                             cudaStream_t stream, bool w_prepared = false);
 
 // HBWN convolution without the im2col matrix: NCHW -> NHWC bf16 copy (Cp = channels rounded up to 8;
 // launch_hbwn_umma_conv does it in the same launch as the weight-piece layout), then the tcgen05 kernel
@@ -86,8 +109,9 @@ cudaError_t launch_im2col_quantize(const void* x, int x_bf16, const ConvGeom& g,
                                    int scale_bf16, cudaStream_t stream);
 // The packed front end with its input tile staged by tensor copies (fp32 input, beta = 32).
 bool im2col_quantize_tma_supported(const void* x, int x_bf16, const ConvGeom& g, int32_t beta);
+// prep (optional): weight-expansion tasks of the contraction that follows, run by extra CTAs of the launch.
 cudaError_t launch_im2col_quantize_tma(const void* x, const ConvGeom& g, uint32_t* bits, int64_t ld_words, void* scales,
-                                       int64_t ld_scales, int scale_bf16, cudaStream_t stream);
+                                       int64_t ld_scales, int scale_bf16, cudaStream_t stream, const UmmaPrepJob* prep = nullptr);
 cudaError_t read_im2col_tma_error(int* code);
 cudaError_t launch_im2col_bf16(const void* x, int x_bf16, const ConvGeom& g, void* out, int64_t ld,
                                cudaStream_t stream);

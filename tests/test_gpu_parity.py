@@ -374,3 +374,33 @@ def test_tensor_path_needs_its_workspace_and_auto_falls_back(hb):
     C.zero_()
     hb.gemm(A, W, C, _gemm_ws(hb, A, W))
     gu.assert_close_rel_absref(C.cpu().numpy(), c_ref, absref, RTOL)
+
+
+def test_prepared_weights_path_repeats_the_tensor_path_bit_for_bit(hb):
+    """HBMM_PATH_TENSOR_PREPARED skips the weight expansion and reuses what the previous call left in the
+    workspace: same kernel, same operands, so the results are identical."""
+    gu = _gu()
+    M, N, K = 300, 136, 640
+    a = inputs.normal((M, K), 91)
+    w = inputs.he_normal(N, K, 92)
+    A, da, sa = gu.oracle_operand(a, 32)
+    W, dw, sw = gu.oracle_operand(w, 64)
+    ws = _gemm_ws(hb, A, W)
+    C1 = torch.empty((M, N), device="cuda")
+    C2 = torch.full((M, N), float("nan"), device="cuda")
+    hb.gemm_ex(A, W, C1, hb.PATH_TENSOR, ws)
+    hb.gemm_ex(A, W, C2, hb.PATH_TENSOR_PREPARED, ws)
+    assert torch.equal(C1, C2)
+    with pytest.raises(hb.HbmmError) as e:
+        hb.gemm_ex(A, W, C2, hb.PATH_TENSOR_PREPARED)
+    assert e.value.status == hb.ERR_WORKSPACE
+    # dense activations (HBWN)
+    _, ab = inputs.as_bf16(a)
+    Ad = hb.wrap_dense(torch.from_numpy(ab).cuda().to(torch.bfloat16))
+    wsd = _gemm_ws(hb, Ad, W)
+    hb.gemm_ex(Ad, W, C1, hb.PATH_TENSOR, wsd)
+    C2.fill_(float("nan"))
+    hb.gemm_ex(Ad, W, C2, hb.PATH_TENSOR_PREPARED, wsd)
+    assert torch.equal(C1, C2)
+    c_ref, absref = oracle.hbwn_from_quantized(ab, dw, sw, 64)
+    gu.assert_close_rel_absref(C2.cpu().numpy(), c_ref, absref, _hbwn_rtol(gu, K, 64))
