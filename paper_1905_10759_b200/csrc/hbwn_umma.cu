@@ -89,19 +89,26 @@ __device__ __forceinline__ void prepare_w_pieces_block(const Args& g, unsigned c
     const int64_t n = tile_n * TN + row;
     uint32_t o[3][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}, {0, 0, 0, 0}};
     if (n < g.N) {
+      // all sixteen loads of the piece are issued before the first use
+      uint32_t word[8];
+      float d[8];
+      bool valid[8];
 #pragma unroll
       for (int e = 0; e < 8; e++) {
         const int64_t q = q0 + piece * 8 + e;
-        if (q < q_end) {
-          const int64_t k = q * k_mul + tap;
-          const uint32_t word = __ldg(g.w_bits + n * g.ldw_w + (k >> 5));
-          const int64_t grp = g.beta >= g.K ? 0 : k / g.beta;
-          const float d = load_scale(g.w_scales, g.w_bf16, n * g.ldw_s + grp);
-          const __nv_bfloat16 b1 = __float2bfloat16_rn(d);
-          const float r1 = d - __bfloat162float(b1);
+        valid[e] = q < q_end;
+        const int64_t k = valid[e] ? q * k_mul + tap : 0;
+        word[e] = __ldg(g.w_bits + n * g.ldw_w + (k >> 5)) >> (k & 31);
+        d[e] = load_scale(g.w_scales, g.w_bf16, n * g.ldw_s + (g.beta >= g.K ? 0 : k / g.beta));
+      }
+#pragma unroll
+      for (int e = 0; e < 8; e++) {
+        if (valid[e]) {
+          const __nv_bfloat16 b1 = __float2bfloat16_rn(d[e]);
+          const float r1 = d[e] - __bfloat162float(b1);
           const __nv_bfloat16 b2 = __float2bfloat16_rn(r1);
           const __nv_bfloat16 b3 = __float2bfloat16_rn(r1 - __bfloat162float(b2));
-          const uint32_t neg = ((word >> (k & 31)) & 1u) ? 0u : 0x8000u;   // bit 0 <=> Sign = -1
+          const uint32_t neg = (word[e] & 1u) ? 0u : 0x8000u;   // bit 0 <=> Sign = -1
           const uint32_t h[3] = {__bfloat16_as_ushort(b1) ^ neg, __bfloat16_as_ushort(b2) ^ neg, __bfloat16_as_ushort(b3) ^ neg};
 #pragma unroll
           for (int i = 0; i < 3; i++) o[i][e >> 1] |= h[i] << ((e & 1) * 16);
