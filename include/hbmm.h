@@ -56,10 +56,22 @@ typedef enum {
   HBMM_PATH_TENSOR = 3, /* tcgen05 with TMEM accumulators: sign bits expanded to +-1 e4m3, group dots
                            scaled in the epilogue; HBWN: bf16 activations x weights written as three
                            bf16 pieces +-d_i (delta = d1 + d2 + d3), one accumulation over all of K     */
-  HBMM_PATH_TENSOR_PREPARED = 4 /* HBMM_PATH_TENSOR, and the caller states that the workspace still holds
+  HBMM_PATH_TENSOR_PREPARED = 4, /* HBMM_PATH_TENSOR, and the caller states that the workspace still holds
                            the expanded weight operand an earlier HBMM_PATH_TENSOR / AUTO call with the
                            same W, the same kind of A and this workspace left there (W unchanged
                            since): the expansion kernel is skipped.  Results are undefined otherwise.  */
+  HBMM_PATH_FOLDED = 5, /* tcgen05, both operands packed: every group scale, times a power of two chosen
+                           per row, is split into two fp16 pieces (22 significant bits) and folded into
+                           the +-1 elements, so that Eq. 7's sum over groups is one fp32 accumulation of
+                           exact fp16 x fp16 products with no per-group step; the powers of two are
+                           divided out once per output.  Scales more than 2^17 below their row's
+                           largest lose relative accuracy (absolute error at most 2^-39 of that
+                           largest scale).  The K products are summed one by one in fp32, so
+                           the error follows sum_k |A~[m,k]| |W~[n,k]| (a few 2^-24 of it) instead of
+                           vanishing where group dots cancel.  What HBMM_PATH_AUTO picks when it has
+                           the workspace and the finer grouping has at most 128 elements per group.   */
+  HBMM_PATH_FOLDED_PREPARED = 6 /* HBMM_PATH_FOLDED with the expanded weights of an earlier
+                           HBMM_PATH_FOLDED / AUTO call reused, as HBMM_PATH_TENSOR_PREPARED          */
 } hbmm_path;
 
 /*
@@ -127,8 +139,8 @@ hbmm_status hbmm_quantize(const void *x, int32_t x_dtype, int64_t rows, int64_t 
 
 /* Bytes of scratch hbmm_gemm wants for these operands (host pointer `bytes`).  The tensor-core
  * contractions keep the weight operand there, expanded once per call into the tile layout their
- * kernels stream (HBMM: about 1.5 K bytes per weight row; HBWN: 6 K bytes per weight row, three
- * bf16 pieces); 0 when no path needs scratch.  hbmm_gemm still works without it (workspace NULL
+ * kernels stream (HBMM: 4 K bytes per weight row, two fp16 pieces; HBWN: 6 K bytes per weight row,
+ * three bf16 pieces); 0 when no path needs scratch.  hbmm_gemm still works without it (workspace NULL
  * or too small): it then runs the integer-pipe path (HBMM) or the warp-level kernels (HBWN).
  * The workspace must be 16-byte aligned. */
 hbmm_status hbmm_gemm_workspace_bytes(const hbmm_operand *A, const hbmm_operand *W, size_t *bytes);
@@ -214,7 +226,8 @@ hbmm_status hbmm_conv_im2col_static(const void *x, int32_t x_dtype, const hbmm_c
 /*
  * Device-side health word of the tensor-core contractions.  Their kernels never spin without a
  * limit: a wait on a barrier that does not complete in time records a code (1 producer, 2/3/4
- * MMA issue, 5 epilogue, 6 weight loader; 100 + the same codes for the HBWN kernel), makes the
+ * MMA issue, 5 epilogue, 6 weight loader; 100 + the same codes for the HBWN kernel, 200 + for the
+ * packed convolution front end, 300 + for the folded-scale HBMM kernel), makes the
  * kernel drain and return, and leaves the output undefined.
  * This call copies the word back (it synchronises the device) and returns HBMM_ERR_TIMEOUT when
  * it is non-zero, HBMM_OK otherwise.  code: host pointer, may be NULL.

@@ -65,6 +65,23 @@ hbmm_status check_c(const float* C, int64_t ldc, int64_t N) {
 size_t tensor_workspace(const PackedView& a, const PackedView& w) {
   return gemm_tensor_supported(a, w) ? static_cast<size_t>(round_up(static_cast<int64_t>(gemm_tensor_workspace_bytes(a, w)), 256)) : 0;
 }
+size_t fold_workspace(const PackedView& a, const PackedView& w) {
+  return gemm_fold_supported(a, w) ? static_cast<size_t>(round_up(static_cast<int64_t>(gemm_fold_workspace_bytes(a, w)), 256)) : 0;
+}
+// Which tensor-core kernel the automatic choice takes.  The folded-scale kernel sums the K individual
+// products in fp32, so its error follows sum_k |A~||W~| rather than sum_g |deltaA deltaW D_g|; the two drift
+// apart as groups grow (for a group of n random signs |D| is about sqrt(n)).  Up to 128 elements per
+// group it stays well inside 1e-5 of the latter and is the faster kernel; beyond that the e4m3 kernel,
+// whose integer group dots are exact and whose per-group step has become rare, is both.
+bool prefer_fold(const PackedView& a, const PackedView& w) {
+  const int64_t ba = a.beta >= a.K ? a.K : a.beta, bw = w.beta >= w.K ? w.K : w.beta;
+  return gemm_fold_supported(a, w) && (ba < bw ? ba : bw) <= 128;
+}
+// What hbmm_gemm_workspace_bytes reports for two packed operands: enough for either tensor-core kernel.
+size_t packed_workspace(const PackedView& a, const PackedView& w) {
+  const size_t t = tensor_workspace(a, w), f = fold_workspace(a, w);
+  return t > f ? t : f;
+}
 size_t hbwn_workspace(const DenseView& a, const PackedView& w) {
   return hbwn_umma_supported(a, w) ? static_cast<size_t>(round_up(static_cast<int64_t>(hbwn_umma_workspace_bytes(a, w)), 256)) : 0;
 }
@@ -83,9 +100,10 @@ hbmm_status gemm_checked(const hbmm_operand* A, const hbmm_operand* W, float* C,
   if (W->beta == 1) return HBMM_ERR_UNSUPPORTED;  // the weight operand is always Hadamard-binary
   hbmm_status st = check_packed(W);
   if (st != HBMM_OK) return st;
-  if (path < HBMM_PATH_AUTO || path > HBMM_PATH_TENSOR_PREPARED) return HBMM_ERR_INVALID_ARG;
-  const bool w_prepared = path == HBMM_PATH_TENSOR_PREPARED;
-  if (w_prepared) path = HBMM_PATH_TENSOR;
+  if (path < HBMM_PATH_AUTO || path > HBMM_PATH_FOLDED_PREPARED) return HBMM_ERR_INVALID_ARG;
+  const bool w_prepared = path == HBMM_PATH_TENSOR_PREPARED || path == HBMM_PATH_FOLDED_PREPARED;
+  if (path == HBMM_PATH_TENSOR_PREPARED) path = HBMM_PATH_TENSOR;
+  if (path == HBMM_PATH_FOLDED_PREPARED) path = HBMM_PATH_FOLDED;
   if (A->beta == 1) {
     if (A->rows <= 0 || A->K <= 0 || !A->dense || A->ld_dense < A->K || !valid_dtype(A->dense_dtype))
       return HBMM_ERR_INVALID_ARG;
@@ -101,6 +119,7 @@ hbmm_status gemm_checked(const hbmm_operand* A, const hbmm_operand* W, float* C,
         if (!hbwn_mma_supported(dv, w)) return HBMM_ERR_UNSUPPORTED;
         e = launch_hbwn_mma(dv, w, C, ldc, stream);
         break;
+      case HBMM_PATH_FOLDED: return HBMM_ERR_UNSUPPORTED;   // dense activations have no group scales to fold
       case HBMM_PATH_TENSOR:
         if (!hbwn_umma_supported(dv, w)) return HBMM_ERR_UNSUPPORTED;
         if (!umma) return HBMM_ERR_WORKSPACE;
@@ -131,9 +150,16 @@ hbmm_status gemm_checked(const hbmm_operand* A, const hbmm_operand* W, float* C,
       if (!workspace_ok(workspace, workspace_bytes, tensor_workspace(a, w))) return HBMM_ERR_WORKSPACE;
       e = launch_gemm_tensor(a, w, C, ldc, workspace, stream, w_prepared);
       break;
+    case HBMM_PATH_FOLDED:
+      if (!gemm_fold_supported(a, w)) return HBMM_ERR_UNSUPPORTED;
+      if (!workspace_ok(workspace, workspace_bytes, fold_workspace(a, w))) return HBMM_ERR_WORKSPACE;
+      e = launch_gemm_fold(a, w, C, ldc, workspace, stream, w_prepared);
+      break;
     default:
-      // the tensor-core path needs its workspace; without one the integer-pipe path runs
-      if (gemm_tensor_supported(a, w) && workspace_ok(workspace, workspace_bytes, tensor_workspace(a, w)))
+      // the tensor-core paths need their workspace; without one the integer-pipe path runs
+      if (prefer_fold(a, w) && workspace_ok(workspace, workspace_bytes, fold_workspace(a, w)))
+        e = launch_gemm_fold(a, w, C, ldc, workspace, stream);
+      else if (gemm_tensor_supported(a, w) && workspace_ok(workspace, workspace_bytes, tensor_workspace(a, w)))
         e = launch_gemm_tensor(a, w, C, ldc, workspace, stream);
       else
         e = launch_gemm_popc(a, w, C, ldc, stream);
@@ -194,7 +220,7 @@ ConvLayout conv_layout(const ConvGeom& g, int32_t beta_a, int32_t scale_dtype, c
     a.beta = beta_a; a.scale_bf16 = scale_dtype == HBMM_BF16;
     hbmm_operand Aop{};
     Aop.rows = L.M; Aop.K = L.K; Aop.beta = beta_a;
-    L.gemm_bytes = (W && W->K == L.K && segments_compatible(&Aop, W)) ? tensor_workspace(a, view_of(W)) : 0;
+    L.gemm_bytes = (W && W->K == L.K && segments_compatible(&Aop, W)) ? packed_workspace(a, view_of(W)) : 0;
     L.total = L.operand_bytes + L.gemm_bytes;
   }
   return L;
@@ -234,7 +260,7 @@ hbmm_status hbmm_gemm_workspace_bytes(const hbmm_operand* A, const hbmm_operand*
   *bytes = 0;
   if (A->beta >= 2 && W->beta >= 2 && check_packed(A, false) == HBMM_OK && check_packed(W, false) == HBMM_OK &&
       A->K == W->K && segments_compatible(A, W))
-    *bytes = tensor_workspace(view_of(A), view_of(W));
+    *bytes = packed_workspace(view_of(A), view_of(W));
   else if (A->beta == 1 && W->beta >= 2 && A->dense && A->rows > 0 && A->K == W->K && A->ld_dense >= A->K &&
            valid_dtype(A->dense_dtype) && check_packed(W, false) == HBMM_OK)
     *bytes = hbwn_workspace(dense_view_of(A), view_of(W));
@@ -317,15 +343,15 @@ hbmm_status hbmm_conv_im2col(const void* x, int32_t x_dtype, const hbmm_conv_geo
     // front end's launch also expands the weight operand (a few extra CTAs) and the contraction skips it.
     const PackedView av = view_of(&A), wv = view_of(W);
     void* gemm_ws = static_cast<char*>(workspace) + L.operand_bytes;
-    if (gemm_tensor_supported(av, wv) && L.gemm_bytes > 0 && L.gemm_bytes >= tensor_workspace(av, wv) &&
+    if (prefer_fold(av, wv) && L.gemm_bytes > 0 && L.gemm_bytes >= fold_workspace(av, wv) &&
         im2col_quantize_tma_supported(x, x_dtype == HBMM_BF16, cg, beta_a)) {
-      UmmaPrepJob job;
-      gemm_tensor_prep_job(av, wv, gemm_ws, &job);
+      UmmaPrepJob job{};
+      gemm_fold_prep_job(av, wv, gemm_ws, &job);
       if (job.n_stages * job.tiles_n <= 4096) {
         if (launch_im2col_quantize_tma(x, cg, A.bits, A.ld_words, A.scales, A.ld_scales, a_scale_dtype == HBMM_BF16, s, &job) !=
             cudaSuccess)
           return HBMM_ERR_CUDA;
-        return launch_gemm_tensor(av, wv, C_out, ldc, gemm_ws, s, true) == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
+        return launch_gemm_fold(av, wv, C_out, ldc, gemm_ws, s, true) == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
       }
     }
     if (launch_im2col_quantize(x, x_dtype == HBMM_BF16, cg, beta_a, A.bits, A.ld_words, A.scales, A.ld_scales,
@@ -343,6 +369,9 @@ hbmm_status hbmm_last_device_error(int32_t* code) {
   int c3 = 0;
   if (read_im2col_tma_error(&c3) != cudaSuccess) return HBMM_ERR_CUDA;
   if (c == 0 && c3 != 0) c = 200 + c3;    // the packed front end's tile copy: 201
+  int c4 = 0;
+  if (read_gemm_fold_error(&c4) != cudaSuccess) return HBMM_ERR_CUDA;
+  if (c == 0 && c4 != 0) c = 300 + c4;    // the folded-scale HBMM kernel: 301..306
   if (code) *code = c;
   return c == 0 ? HBMM_OK : HBMM_ERR_TIMEOUT;
 }

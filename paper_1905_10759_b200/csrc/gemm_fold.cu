@@ -1,0 +1,427 @@
+// HBMM contraction of two packed operands on the 5th-generation tensor cores with the group scales
+// folded into the operands (tcgen05 / TMEM).
+//
+// Section 4.2, Eq. 7 computes  C[m,n] = sum_g deltaA[m,g] deltaW[n,g] D_g[m,n]  with D_g the signed +-1 dot
+// of group g.  That is the plain product of the Hadamard-product operands A~ = deltaA (.) Sign(A) and
+// W~ = deltaW (.) Sign(W) (Eq. 2 / Eq. 4).  Here each operand is expanded on the fly into two fp16
+// matrices whose sum carries its fp32 group scales to 22 bits (see gemm_fold_prep.cuh), every fp16 x fp16
+// product is exact in the fp32 accumulator, and the four cross products
+//     A1 W1^T + A1 W2^T + A2 W1^T + A2 W2^T
+// are one accumulation in tensor memory over the whole of K: the two weight pieces of a column tile are
+// stacked along N, so per 16 K-elements two MMAs of 128 x 2TN x 16 (A1 and A2 against [W1; W2]) do all four.
+// There is no per-group step; the epilogue runs once per tile, adds the two column blocks and divides
+// the rows' and columns' powers of two out again (exact).  Compared with forming D_g and the scale
+// product per group this trades 4x the tensor work for the removal of the per-group TMEM round trip
+// that bounded the e4m3 kernel.
+//
+// CTA tile = 128 rows x TN columns; one persistent CTA per SM walks the tiles of the output.
+//   warps 0-3   : epilogue, once per tile (TMEM lanes 32*w ..)
+//   warps 4-11  : A producers: thread = (tile row, stage parity); packed words + group scales -> the
+//                 64 elements of both fp16 pieces in the 128-byte-swizzled K-major layout, with the
+//                 global loads issued several stages ahead
+//   warps 14-17 : scouts: one thread per tile row finds the row's largest scale (the power of two that
+//                 normalises the row) a few tiles ahead of everyone else
+//   warp  12    : TMEM allocation and the single MMA-issuing thread
+//   warp  13    : one thread streams the prepared W stages (cp.async.bulk, completion on the stage's
+//                 mbarrier); W is expanded once per call (or once per weight tensor) into a workspace
+// A stage holds 64 K-elements (two packed words).  Stages and the two TMEM accumulators are mbarrier
+// rings.  Every wait is bounded: on expiry the thread records a code, raises a CTA-wide abort flag
+// that all other waits observe, and the kernel drains and frees its TMEM before returning.
+#include <cuda_fp16.h>
+#include "kernels.h"
+#include "umma_common.cuh"
+#include "gemm_fold_prep.cuh"
+
+namespace hbmm {
+namespace {
+
+using namespace umma;
+using namespace fold;
+
+constexpr int kEpilogueWarps = 4;
+constexpr int kProducerWarps = 8;
+constexpr int kFirstProducerWarp = kEpilogueWarps;
+constexpr int kMmaWarp = kEpilogueWarps + kProducerWarps;   // 12
+constexpr int kLoaderWarp = kMmaWarp + 1;                   // 13
+constexpr int kFirstScoutWarp = kLoaderWarp + 1;            // 14..17
+constexpr int kScoutWarps = 4;
+constexpr int kThreads = (kFirstScoutWarp + kScoutWarps) * 32;
+constexpr int kDepth = 4;     // stages of packed words + scales each producer thread keeps in flight
+
+template <int TN>
+__global__ void __launch_bounds__(TN)
+prepare_w_fold_kernel(const Args g, unsigned char* __restrict__ out, float* __restrict__ w_down) {
+  prepare_w_task<TN>(g, out, w_down, blockIdx.x, blockIdx.y, threadIdx.x);
+}
+
+// Walks the stages a producer thread owns (every second stage of the CTA's stream of tiles) and keeps
+// the row pointers of the tile it is in.
+struct StageCursor {
+  int64_t ti, st;            // tile (in this CTA's sequence) and stage inside it
+  const uint32_t* bptr;      // packed words of this thread's row
+  int64_t srow;              // first scale of the row
+  bool in;                   // the row exists
+};
+
+template <int TN>
+__global__ void __launch_bounds__(kThreads, 1)
+hbmm_fold_kernel(const Args g) {
+  using S = Smem<TN>;
+  constexpr int STAGES = S::STAGES;
+  extern __shared__ __align__(1024) unsigned char smem[];
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + S::OFF_BAR);
+  uint64_t* empty = full + STAGES;
+  uint64_t* tfull = empty + STAGES;
+  uint64_t* tempty = tfull + 2;
+  uint64_t* drain = tempty + 2;
+  uint64_t* rowfull = drain + 1;                 // the scouts have stored a tile's row factors
+  uint64_t* rowempty = rowfull + kRowSlots;      // the epilogue has read them
+  float* rowup = reinterpret_cast<float*>(smem + S::OFF_ROWF);
+  float* rowdown = rowup + kRowSlots * TM;
+  float* colf = reinterpret_cast<float*>(smem + S::OFF_COLF);
+  uint32_t* tmem_base_ptr = reinterpret_cast<uint32_t*>(smem + S::OFF_MISC);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + S::OFF_MISC + 4);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int64_t tiles_n = (g.N + TN - 1) / TN, tiles_m = (g.M + TM - 1) / TM;
+  const int64_t n_tiles = tiles_m * tiles_n;
+  const int64_t n_stages = (g.n_words + WPS - 1) / WPS;      // per tile
+  const int64_t my_tiles = blockIdx.x < n_tiles ? (n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+
+  if (tid == 0) {
+    for (int s = 0; s < STAGES; s++) {
+      mbar_init(&full[s], kProducerWarps / 2 + 1);  // the four producer warps of the stage + the loader's expect_tx arrival
+      mbar_init(&empty[s], 1);                      // MMA commit: the stage's bytes have been read
+    }
+    for (int b = 0; b < 2; b++) { mbar_init(&tfull[b], 1); mbar_init(&tempty[b], kEpilogueWarps); }
+    mbar_init(drain, 1);
+    for (int r = 0; r < kRowSlots; r++) { mbar_init(&rowfull[r], kScoutWarps); mbar_init(&rowempty[r], kEpilogueWarps); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == kMmaWarp) {
+    tmem_alloc(tmem_base_ptr, S::TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_base_ptr;
+
+  // The CTA is persistent: it walks tiles blockIdx.x, blockIdx.x + gridDim.x, ... and the stage ring
+  // simply continues across tiles (gst counts stages since launch).
+  if (warp >= kFirstProducerWarp && warp < kMmaWarp) {
+    // =========================== A producers ===========================
+    // Thread = (tile row p, parity q): it expands both words of every stage whose number since launch
+    // has parity q.  Packed words and scales are loaded kDepth of its stages (2 kDepth stages of the
+    // CTA) ahead, across tile boundaries, so that no global-memory latency is left in the stage loop.
+    const int pt = tid - kFirstProducerWarp * 32;
+    const int q = pt >> 7;
+    const int p = pt & (TM - 1);
+    const uint32_t n_words = static_cast<uint32_t>(g.n_words), gw = static_cast<uint32_t>(g.a_gw);
+    const bool vec_scales = !g.a_bf16 && gw == 1;      // one fp32 scale per word: a stage's two scales are one 8-byte load
+    const int64_t total = my_tiles * n_stages;
+    auto set_tile = [&](StageCursor& c) {
+      const int64_t tile = blockIdx.x + c.ti * gridDim.x;
+      const int64_t m = (tile / tiles_n) * TM + p;
+      c.in = c.ti < my_tiles && m < g.M;
+      c.bptr = g.a_bits + (c.in ? m : 0) * g.lda_w;
+      c.srow = (c.in ? m : 0) * g.lda_s;
+    };
+    auto advance = [&](StageCursor& c) {
+      c.st += 2;
+      if (c.st >= n_stages) {
+        do { c.st -= n_stages; c.ti++; } while (c.st >= n_stages);
+        set_tile(c);
+      }
+    };
+    auto fetch = [&](const StageCursor& c, uint2& w, float& s0, float& s1) {
+      w = make_uint2(0u, 0u);
+      s0 = s1 = 0.0f;
+      const uint32_t wi = static_cast<uint32_t>(c.st) * WPS;
+      if (c.in && wi < n_words) {
+        w = __ldg(reinterpret_cast<const uint2*>(c.bptr + wi));      // the row is padded with zero words to a multiple of four
+        if (vec_scales) {
+          const float2 v = __ldg(reinterpret_cast<const float2*>(reinterpret_cast<const float*>(g.a_scales) + c.srow + wi));
+          s0 = v.x;
+          s1 = v.y;                                                    // past the last group: a stored zero
+        } else {
+          s0 = load_scale(g.a_scales, g.a_bf16, c.srow + wi / gw);
+          if (wi + 1 < n_words) s1 = load_scale(g.a_scales, g.a_bf16, c.srow + (wi + 1) / gw);
+        }
+      }
+    };
+    StageCursor pf, cur;
+    pf.ti = 0; pf.st = q;
+    if (pf.st >= n_stages) { do { pf.st -= n_stages; pf.ti++; } while (pf.st >= n_stages); }
+    set_tile(pf);
+    cur = pf;
+    uint2 w[kDepth];
+    float s0[kDepth], s1[kDepth];
+#pragma unroll
+    for (int u = 0; u < kDepth; u++) { fetch(pf, w[u], s0[u], s1[u]); advance(pf); }
+    int64_t up_tile = -1;
+    float up = 0.0f;
+    bool ok = true;
+    for (int64_t gst = q; gst < total && ok; gst += 2 * kDepth) {
+#pragma unroll
+      for (int u = 0; u < kDepth; u++) {
+        const int64_t my = gst + 2 * u;
+        if (my < total && ok) {
+          if (cur.ti != up_tile) {
+            // the row's power of two comes from the scouts, who run ahead of the tile being filled
+            const int slot = static_cast<int>(cur.ti & (kRowSlots - 1));
+            if (!mbar_wait(&rowfull[slot], static_cast<uint32_t>((cur.ti / kRowSlots) & 1), abort_flag, 7)) { ok = false; }
+            up = rowup[slot * TM + p];
+            up_tile = cur.ti;
+          }
+          const int s = static_cast<int>(my % STAGES);
+          if (ok && my >= STAGES && !mbar_wait(&empty[s], static_cast<uint32_t>(((my / STAGES) & 1) ^ 1), abort_flag, 1)) ok = false;
+          if (ok) {
+            unsigned char* a1 = smem + S::OFF_A + s * S::A_STAGE;
+            expand_word(a1, a1 + S::A_PIECE, p, 0, w[u].x, s0[u] * up);
+            expand_word(a1, a1 + S::A_PIECE, p, 1, w[u].y, s1[u] * up);
+            fence_async_proxy();          // make the generic-proxy stores visible to the tensor core
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&full[s]);
+            fetch(pf, w[u], s0[u], s1[u]);  // this register slot is free again: load kDepth of my stages ahead
+            advance(pf);
+            advance(cur);
+          }
+        }
+      }
+    }
+  } else if (warp >= kFirstScoutWarp) {
+    // =========================== scouts ===========================
+    // One thread per tile row finds the row's largest scale and stores the two powers of two, up to
+    // kRowSlots tiles ahead of the epilogue.
+    const int p = tid - kFirstScoutWarp * 32;
+    for (int64_t ti = 0; ti < my_tiles; ti++) {
+      const int slot = static_cast<int>(ti & (kRowSlots - 1));
+      if (ti >= kRowSlots && !mbar_wait(&rowempty[slot], static_cast<uint32_t>(((ti / kRowSlots) & 1) ^ 1), abort_flag, 8)) break;
+      const int64_t tile = blockIdx.x + ti * gridDim.x;
+      const int64_t m = (tile / tiles_n) * TM + p;
+      float up = 0.0f, down = 1.0f;
+      if (m < g.M) norm_factors(row_max_scale(g.a_scales, g.a_bf16, m * g.lda_s, g.lda_s), up, down);
+      rowup[slot * TM + p] = up;
+      rowdown[slot * TM + p] = down;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&rowfull[slot]);
+    }
+  } else if (warp == kLoaderWarp) {
+    // =========================== W loader ===========================
+    if (lane == 0) {
+      int64_t gst = 0;
+      bool ok = true;
+      for (int64_t ti = 0; ti < my_tiles && ok; ti++) {
+        const int64_t tile = blockIdx.x + ti * gridDim.x;
+        const unsigned char* src = g.w_prep + (tile % tiles_n) * n_stages * S::B_STAGE;
+        for (int64_t st = 0; st < n_stages; st++, gst++) {
+          const int s = static_cast<int>(gst % STAGES);
+          if (gst >= STAGES && !mbar_wait(&empty[s], static_cast<uint32_t>(((gst / STAGES) & 1) ^ 1), abort_flag, 6)) { ok = false; break; }
+          mbar_arrive_expect_tx(&full[s], S::B_STAGE);
+          bulk_copy_g2s(smem + S::OFF_B + s * S::B_STAGE, src + st * S::B_STAGE, S::B_STAGE, &full[s]);
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == kMmaWarp) {
+    // =========================== MMA issuer ===========================
+    // The whole warp walks the loop so that ring indices and descriptors stay warp-uniform values; one
+    // lane issues the MMAs and commits.
+    {
+      constexpr uint32_t idesc = instr_desc(S::NST, kFmtF16);
+      const uint64_t da0 = smem_desc(smem_u32(smem + S::OFF_A)), db0 = smem_desc(smem_u32(smem + S::OFF_B));
+      const uint64_t da_hi = da0 & 0xFFFFFFFF00000000ull, db_hi = db0 & 0xFFFFFFFF00000000ull;
+      const uint32_t da_lo = static_cast<uint32_t>(da0), db_lo = static_cast<uint32_t>(db0);
+      const uint32_t full_a = smem_u32(full), empty_a = smem_u32(empty), tfull_a = smem_u32(tfull), tempty_a = smem_u32(tempty);
+      const bool leader = lane == 0;
+      const uint32_t n_st = static_cast<uint32_t>(n_stages);
+      uint32_t s = 0, full_par = 0;
+      bool ok = true;
+      for (int64_t ti = 0; ti < my_tiles && ok; ti++) {
+        const uint32_t buf = static_cast<uint32_t>(ti & 1);
+        if (ti >= 2) {      // the epilogue must have drained this accumulator (used by tile ti - 2)
+          if (!mbar_wait_a(tempty_a + buf * 8, static_cast<uint32_t>(((ti >> 1) & 1) ^ 1), abort_flag, 3)) { ok = false; break; }
+          tc_fence_after();
+        }
+        const uint32_t d_tmem = tmem_base + buf * S::NST;
+        for (uint32_t st = 0; st < n_st; st++) {
+          if (!mbar_wait_a(full_a + s * 8, full_par, abort_flag, 2)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a1_lo = da_lo + s * (S::A_STAGE >> 4), a2_lo = a1_lo + (S::A_PIECE >> 4);
+          const uint32_t b_lo = db_lo + s * (S::B_STAGE >> 4);
+          if (leader) {
+#pragma unroll
+            for (int ks = 0; ks < KB / 16; ks++) {        // 16 K-elements = 32 bytes along the swizzled rows
+              umma_bf16(d_tmem, da_hi | (a1_lo + ks * 2), db_hi | (b_lo + ks * 2), idesc, (st | ks) != 0 ? 1u : 0u);
+              umma_bf16(d_tmem, da_hi | (a2_lo + ks * 2), db_hi | (b_lo + ks * 2), idesc, 1u);
+            }
+            umma_commit_a(empty_a + s * 8);     // the stage's bytes are free once these MMAs have read them
+          }
+          __syncwarp();
+          if (++s == STAGES) { s = 0; full_par ^= 1; }
+        }
+        if (ok && leader) umma_commit_a(tfull_a + buf * 8);
+        __syncwarp();
+      }
+      if (leader) {
+        umma_commit(drain);
+        mbar_wait(drain, 0, abort_flag, 4);   // every MMA has retired before TMEM is released
+      }
+    }
+    __syncwarp();
+  } else if (warp < kEpilogueWarps) {
+    // =========================== epilogue ===========================
+    const int row = warp * 32 + lane;               // TMEM lane = tile row
+    const uint32_t t_lane = static_cast<uint32_t>(warp * 32) << 16;
+    for (int64_t ti = 0; ti < my_tiles; ti++) {
+      const uint32_t buf = static_cast<uint32_t>(ti & 1);
+      const int slot = static_cast<int>(ti & (kRowSlots - 1));
+      const int64_t tile = blockIdx.x + ti * gridDim.x;
+      const int64_t m = (tile / tiles_n) * TM + row, nb = (tile % tiles_n) * TN;
+      // the tile's column factors go through shared memory (one copy per warp, so no warp waits for
+      // another): requested before the wait for the accumulator, read back as broadcasts
+      float fcol[TN / 32];
+#pragma unroll
+      for (int i = 0; i < TN / 32; i++) fcol[i] = __ldg(g.w_down + nb + i * 32 + lane);   // w_down holds a whole number of tiles
+      if (!mbar_wait(&tfull[buf], static_cast<uint32_t>((ti >> 1) & 1), abort_flag, 5)) break;
+      if (!mbar_wait(&rowfull[slot], static_cast<uint32_t>((ti / kRowSlots) & 1), abort_flag, 5)) break;   // long complete
+      tc_fence_after();
+      const float fa = rowdown[slot * TM + row];
+      float* cf = colf + warp * TN;
+#pragma unroll
+      for (int i = 0; i < TN / 32; i++) cf[i * 32 + lane] = fcol[i];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&rowempty[slot]);
+      float* dst = g.C + m * g.ldc + nb;
+#pragma unroll
+      for (int c = 0; c < TN / 32; c++) {
+        uint32_t v1[32], v2[32];
+        const uint32_t t_addr = tmem_base + t_lane + buf * S::NST + c * 32;
+        tmem_ld32(t_addr, v1);
+        tmem_ld32(t_addr + TN, v2);
+        tmem_ld_wait();
+        if (m < g.M) {
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            const float4 fw = *reinterpret_cast<const float4*>(cf + c * 32 + j);
+            float o[4];
+#pragma unroll
+            for (int e = 0; e < 4; e++) o[e] = (__uint_as_float(v1[j + e]) + __uint_as_float(v2[j + e])) * fa;
+            o[0] *= fw.x; o[1] *= fw.y; o[2] *= fw.z; o[3] *= fw.w;
+            const int64_t n = nb + c * 32 + j;
+            if (n + 3 < g.N) *reinterpret_cast<float4*>(dst + c * 32 + j) = make_float4(o[0], o[1], o[2], o[3]);
+            else
+              for (int e = 0; e < 4; e++)
+                if (n + e < g.N) dst[c * 32 + j + e] = o[e];
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();          // also: every lane is done with the warp's column factors
+      if (lane == 0) mbar_arrive(&tempty[buf]);
+    }
+  }
+
+  // ---- teardown: everyone meets here (aborted threads too), then the allocating warp frees TMEM
+  tc_fence_before();
+  __syncthreads();
+  if (warp == kMmaWarp) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, S::TMEM_COLS);
+  }
+}
+
+Args make_args(const PackedView& A, const PackedView& W, float* C, int64_t ldc) {
+  Args g;
+  g.a_bits = A.bits; g.a_scales = A.scales; g.w_bits = W.bits; g.w_scales = W.scales; g.C = C;
+  g.M = A.rows; g.N = W.rows; g.lda_w = A.ld_words; g.ldw_w = W.ld_words; g.lda_s = A.ld_scales; g.ldw_s = W.ld_scales;
+  g.ldc = ldc; g.a_bf16 = A.scale_bf16; g.w_bf16 = W.scale_bf16;
+  g.n_words = A.K / 32;
+  g.a_gw = A.beta >= A.K ? g.n_words : A.beta / 32;
+  g.w_gw = W.beta >= W.K ? g.n_words : W.beta / 32;
+  g.w_prep = nullptr;
+  g.w_down = nullptr;
+  return g;
+}
+
+template <int TN>
+size_t stage_bytes(const Args& g) {
+  const int64_t tiles_n = (g.N + TN - 1) / TN, n_stages = (g.n_words + WPS - 1) / WPS;
+  return static_cast<size_t>(tiles_n * n_stages) * Smem<TN>::B_STAGE;
+}
+template <int TN>
+size_t prep_bytes(const Args& g) {
+  return stage_bytes<TN>(g) + static_cast<size_t>((g.N + TN - 1) / TN) * TN * sizeof(float);
+}
+
+template <int TN>
+cudaError_t launch_fold(Args g, void* workspace, cudaStream_t stream, bool w_prepared) {
+  using S = Smem<TN>;
+  static bool configured = false;
+  static int sms = 0;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(hbmm_fold_kernel<TN>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::BYTES);
+    if (e != cudaSuccess) return e;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    configured = true;
+  }
+  const int64_t tiles_n = (g.N + TN - 1) / TN, n_stages = (g.n_words + WPS - 1) / WPS;
+  unsigned char* stages = static_cast<unsigned char*>(workspace);
+  float* down = reinterpret_cast<float*>(stages + stage_bytes<TN>(g));
+  if (!w_prepared) {
+    dim3 pgrid(static_cast<unsigned>((n_stages + kPrepStages - 1) / kPrepStages), static_cast<unsigned>(tiles_n));
+    prepare_w_fold_kernel<TN><<<pgrid, TN, 0, stream>>>(g, stages, down);
+  }
+  g.w_prep = stages;
+  g.w_down = down;
+  const int64_t tiles = ((g.M + TM - 1) / TM) * tiles_n;
+  const unsigned grid = static_cast<unsigned>(tiles < sms ? tiles : sms);   // one persistent CTA per SM
+  hbmm_fold_kernel<TN><<<grid, kThreads, S::BYTES, stream>>>(g);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+// K a multiple of 32 and scale groups of whole words (or one group per row).
+bool gemm_fold_supported(const PackedView& A, const PackedView& W) {
+  if (A.K % 32 != 0 || A.K / 32 >= (int64_t{1} << 31)) return false;
+  const bool a_one = A.beta >= A.K, w_one = W.beta >= W.K;
+  if (!a_one && A.beta % 32 != 0) return false;
+  if (!w_one && W.beta % 32 != 0) return false;
+  return true;
+}
+
+// Bytes of workspace: the weight operand as fp16 piece tiles (4 bytes per element) + one float per row.
+size_t gemm_fold_workspace_bytes(const PackedView& A, const PackedView& W) {
+  const Args g = make_args(A, W, nullptr, 0);
+  return g.N <= 64 ? prep_bytes<64>(g) : prep_bytes<128>(g);
+}
+
+// workspace: device, 16-byte aligned, at least gemm_fold_workspace_bytes.
+cudaError_t launch_gemm_fold(const PackedView& A, const PackedView& W, float* C, int64_t ldc, void* workspace,
+                             cudaStream_t stream, bool w_prepared) {
+  const Args g = make_args(A, W, C, ldc);
+  return g.N <= 64 ? launch_fold<64>(g, workspace, stream, w_prepared) : launch_fold<128>(g, workspace, stream, w_prepared);
+}
+
+// The weight expansion of launch_gemm_fold(A, W, ..., workspace) as a job for another kernel.
+void gemm_fold_prep_job(const PackedView& A, const PackedView& W, void* workspace, UmmaPrepJob* job) {
+  job->f = make_args(A, W, nullptr, 0);
+  job->folded = 1;
+  job->out = static_cast<unsigned char*>(workspace);
+  job->tn = job->f.N <= 64 ? 64 : 128;
+  const int64_t n_stages = (job->f.n_words + WPS - 1) / WPS;
+  job->n_stages = static_cast<int32_t>((n_stages + kPrepStages - 1) / kPrepStages);    // tasks per column tile
+  job->tiles_n = static_cast<int32_t>((job->f.N + job->tn - 1) / job->tn);
+  job->out_down = reinterpret_cast<float*>(job->out + (job->tn == 64 ? stage_bytes<64>(job->f) : stage_bytes<128>(job->f)));
+}
+
+cudaError_t read_gemm_fold_error(int* code) {
+  return cudaMemcpyFromSymbol(code, umma::g_error_word, sizeof(int));
+}
+
+}  // namespace hbmm

@@ -1,0 +1,163 @@
+// Pieces of the folded-scale tcgen05 HBMM kernel that other translation units need: the shared-memory
+// stage layout, the routine that turns packed words + group scales into fp16 operand tiles, and the
+// weight-expansion task (the packed convolution front end runs it in a few extra CTAs of its launch).
+//
+// Folded scales.  A Hadamard-binary operand X~ = delta (.) Sign(X) (Eq. 2 / Eq. 4) is written as the sum of
+// two fp16 matrices X1 + X2: the group scale, multiplied by a power of two 2^u chosen per row so that the
+// row's largest scale lies in [2^14, 2^15), is split as delta * 2^u = d1 + d2 with d1 = fp16(delta * 2^u) and
+// d2 = fp16(delta * 2^u - d1) (the remainder is exact in fp32), and element k of piece i is +-d_i.  d1 + d2
+// carries 22 significant bits of every scale that is within 2^-17 of its row's largest (below that d2
+// becomes subnormal and the error is at most 2^-39 of the row's largest scale).  fp16 x fp16 products are
+// exact in fp32, so A~ W~^T = (A1 + A2)(W1 + W2)^T accumulated in fp32 reproduces Eq. 7's per-group
+// full-precision scaling with no per-group step at all; the powers of two are divided out once per output.
+#pragma once
+#include <cuda_fp16.h>
+#include <cstdint>
+#include "kernels.h"
+#include "umma_common.cuh"
+
+namespace hbmm {
+namespace fold {
+
+using namespace umma;
+using Args = FoldArgs;
+
+constexpr int KB = 64;            // K elements per stage: one 128-byte row of fp16
+constexpr int WPS = 2;            // packed K-words per stage
+constexpr int kRowSlots = 8;      // ring of per-tile row factors (scouts -> producers and epilogue)
+
+template <int TN>
+struct Smem {
+  static constexpr int STAGES = TN == 64 ? 4 : 3;
+  static constexpr int A_PIECE = TM * 128;                // one fp16 piece of the A tile: 128 rows x 64 elements
+  static constexpr int A_STAGE = 2 * A_PIECE;
+  static constexpr int B_PIECE = TN * 128;
+  static constexpr int B_STAGE = 2 * B_PIECE;             // W1 rows then W2 rows: one MMA of N = 2 TN reads both
+  static constexpr int OFF_A = 0;
+  static constexpr int OFF_B = OFF_A + STAGES * A_STAGE;
+  static constexpr int OFF_ROWF = OFF_B + STAGES * B_STAGE;
+  static constexpr int OFF_COLF = OFF_ROWF + 2 * kRowSlots * TM * 4;  // per slot and row: normalising power of two and its inverse
+  static constexpr int OFF_BAR = OFF_COLF + 4 * TN * 4;               // the tile's column factors, one copy per epilogue warp
+  static constexpr int NBAR = 2 * STAGES + 4 + 1 + 2 * kRowSlots;     // full, empty, tfull[2], tempty[2], drain, rowfull, rowempty
+  static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
+  static constexpr int BYTES = OFF_MISC + 16;
+  static constexpr int NST = 2 * TN;                      // MMA N
+  static constexpr int TMEM_COLS = 2 * NST;               // two accumulators
+  static_assert(BYTES > 120 * 1024, "one CTA per SM: it owns the tensor memory it allocates");
+  static_assert(NST <= 256 && NST % 16 == 0, "one MMA covers both weight pieces");
+};
+
+__device__ __forceinline__ float load_scale(const void* s, int bf16, int64_t idx) {
+  if (bf16) return __uint_as_float(static_cast<uint32_t>(__ldg(reinterpret_cast<const unsigned short*>(s) + idx)) << 16);
+  return __ldg(reinterpret_cast<const float*>(s) + idx);
+}
+
+// Largest scale of one operand row.  Rows are 16-byte vectors (the leading dimension is a multiple of 4
+// fp32 / 8 bf16 entries) and entries past the last group are stored zeros.  Scales are >= 0, so their bit
+// patterns order like the values.
+__device__ __forceinline__ float row_max_scale(const void* s, int bf16, int64_t row_off, int64_t ld) {
+  uint32_t mx = 0;
+  if (bf16) {
+    const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned short*>(s) + row_off);
+#pragma unroll 4
+    for (int64_t i = 0; i < ld / 8; i++) {
+      const uint4 v = __ldg(p + i);
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int e = 0; e < 4; e++) { mx = max(mx, w[e] << 16); mx = max(mx, w[e] & 0xFFFF0000u); }
+    }
+  } else {
+    const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(s) + row_off);
+#pragma unroll 4
+    for (int64_t i = 0; i < ld / 4; i++) {
+      const uint4 v = __ldg(p + i);
+      mx = max(max(mx, v.x), max(v.y, max(v.z, v.w)));
+    }
+  }
+  return __uint_as_float(mx);
+}
+
+// Powers of two for a row whose largest scale is mx: mx * up lies in [2^14, 2^15), down = 1 / up.
+// Rows whose scales are all below 2^-100 (an all-zero row included) are treated as if their largest
+// were 2^-100, which keeps both factors normal numbers.
+__device__ __forceinline__ void norm_factors(float mx, float& up, float& down) {
+  uint32_t e = (__float_as_uint(mx) >> 23) & 0xFFu;      // biased exponent
+  e = e < 27u ? 27u : e;
+  up = __uint_as_float((268u - e) << 23);                // 2^(14 - (e - 127))
+  down = __uint_as_float((e - 14u) << 23);               // 2^((e - 127) - 14)
+}
+
+// One packed K-word of tile row `row` -> its 32 elements in both fp16 pieces.  `scaled` is the word's
+// group scale times the row's power of two (0 for words past K or rows past the operand: +-0).
+// Word slot q of the stage fills the 16-byte chunks 4q .. 4q+3 of the 128-byte row; 32-bit position j of
+// the slot holds the elements of bits j (low half) and j + 16 (high half).  Both operands use this
+// order, and a dot product does not depend on the order of its terms.  Bit 1 <=> +1, bit 0 <=> -1: the
+// inverted bit is moved onto the fp16 sign.
+__device__ __forceinline__ void expand_word(unsigned char* piece1, unsigned char* piece2, int row, int q, uint32_t word, float scaled) {
+  const __half d1 = __float2half_rn(scaled);
+  const __half d2 = __float2half_rn(scaled - __half2float(d1));
+  const uint32_t h1 = static_cast<uint32_t>(__half_as_ushort(d1)) * 0x10001u;
+  const uint32_t h2 = static_cast<uint32_t>(__half_as_ushort(d2)) * 0x10001u;
+  const uint32_t nw = ~word;
+#pragma unroll
+  for (int c = 0; c < 4; c++) {
+    uint32_t m[4];
+#pragma unroll
+    for (int i = 0; i < 4; i++) m[i] = (nw << (15 - (4 * c + i))) & 0x80008000u;
+    *reinterpret_cast<uint4*>(swz(piece1, row, 4 * q + c)) = make_uint4(m[0] ^ h1, m[1] ^ h1, m[2] ^ h1, m[3] ^ h1);
+    *reinterpret_cast<uint4*>(swz(piece2, row, 4 * q + c)) = make_uint4(m[0] ^ h2, m[1] ^ h2, m[2] ^ h2, m[3] ^ h2);
+  }
+}
+
+// Expands kPrepStages consecutive stages of one column tile of the weight operand into the stage layout
+// the main kernel streams: rows 0 .. TN-1 piece 1, rows TN .. 2TN-1 piece 2, exactly as they sit in
+// shared memory.  The task of the first stages also stores the rows' inverse powers of two.
+// p = row of the tile, one thread per row (it scans its row's scales once per task).
+constexpr int kPrepStages = 8;
+template <int TN>
+__device__ __forceinline__ void prepare_w_task(const Args& g, unsigned char* __restrict__ out, float* __restrict__ w_down,
+                                               int64_t chunk, int64_t tile_n, int p) {
+  using S = Smem<TN>;
+  const int64_t n_stages = (g.n_words + WPS - 1) / WPS;
+  const int64_t n = tile_n * TN + p;
+  const bool in = n < g.N;
+  float up = 0.0f, down = 1.0f;
+  if (in) norm_factors(row_max_scale(g.w_scales, g.w_bf16, n * g.ldw_s, g.ldw_s), up, down);
+  if (chunk == 0) w_down[n] = down;
+  const int64_t st0 = chunk * kPrepStages;
+  const int64_t st1 = st0 + kPrepStages < n_stages ? st0 + kPrepStages : n_stages;
+  const bool vec_scales = !g.w_bf16 && g.w_gw == 1;
+  // the words (and, one fp32 scale per word, the scales) of four stages are two 16-byte loads each
+  for (int64_t st = st0; st < st1; st += 4) {
+    uint32_t word[8];
+    float sc[8];
+#pragma unroll
+    for (int h = 0; h < 2; h++) {
+      const int64_t wi = st * WPS + 4 * h;
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (in && wi < g.ldw_w) v = __ldg(reinterpret_cast<const uint4*>(g.w_bits + n * g.ldw_w + wi));   // zero words pad the row
+      word[4 * h] = v.x; word[4 * h + 1] = v.y; word[4 * h + 2] = v.z; word[4 * h + 3] = v.w;
+      if (vec_scales) {
+        float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (in && wi < g.ldw_s) f = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(g.w_scales) + n * g.ldw_s + wi));
+        sc[4 * h] = f.x; sc[4 * h + 1] = f.y; sc[4 * h + 2] = f.z; sc[4 * h + 3] = f.w;                  // stored zeros past the last group
+      } else {
+#pragma unroll
+        for (int e = 0; e < 4; e++)
+          sc[4 * h + e] = (in && wi + e < g.n_words) ? load_scale(g.w_scales, g.w_bf16, n * g.ldw_s + (wi + e) / g.w_gw) : 0.0f;
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < 8; e++) {
+      const int64_t sst = st + e / WPS;
+      if (sst < st1) {
+        unsigned char* base = out + (tile_n * n_stages + sst) * S::B_STAGE;
+        const bool valid = st * WPS + e < g.n_words;
+        expand_word(base, base + S::B_PIECE, p, e % WPS, valid ? word[e] : 0u, valid ? sc[e] * up : 0.0f);
+      }
+    }
+  }
+}
+
+}  // namespace fold
+}  // namespace hbmm

@@ -396,6 +396,8 @@ cudaError_t launch_gemm_tensor(const PackedView& A, const PackedView& W, float* 
 // The weight expansion of launch_gemm_tensor(A, W, ..., workspace) as a job for another kernel.
 void gemm_tensor_prep_job(const PackedView& A, const PackedView& W, void* workspace, UmmaPrepJob* job) {
   job->g = make_args(A, W, nullptr, 0);
+  job->folded = 0;
+  job->out_down = nullptr;
   job->out = static_cast<unsigned char*>(workspace);
   job->tn = job->g.N <= 64 ? 64 : 128;
   job->n_stages = static_cast<int32_t>((job->g.n_words + WPS - 1) / WPS);

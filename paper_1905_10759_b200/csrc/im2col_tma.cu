@@ -13,6 +13,7 @@
 #include "umma_common.cuh"
 #include "im2col_gather.cuh"
 #include "gemm_umma_prep.cuh"
+#include "gemm_fold_prep.cuh"
 
 namespace hbmm {
 namespace {
@@ -70,8 +71,13 @@ im2col_quantize_tma_kernel(const __grid_constant__ CUtensorMap x_map, const floa
   // a stage of one column tile, one thread per weight row); they are scheduled first and leave at once.
   if (static_cast<int>(blockIdx.x) < n_prep) {
     const int st = blockIdx.x % prep.n_stages, tile_n = blockIdx.x / prep.n_stages;
-    if (prep.tn == 64) { if (threadIdx.x < 64) umma_prep::prepare_w_task<64>(prep.g, prep.out, st, tile_n, threadIdx.x); }
-    else if (threadIdx.x < 128) umma_prep::prepare_w_task<128>(prep.g, prep.out, st, tile_n, threadIdx.x);
+    if (prep.folded) {
+      if (prep.tn == 64) { if (threadIdx.x < 64) fold::prepare_w_task<64>(prep.f, prep.out, prep.out_down, st, tile_n, threadIdx.x); }
+      else if (threadIdx.x < 128) fold::prepare_w_task<128>(prep.f, prep.out, prep.out_down, st, tile_n, threadIdx.x);
+    } else {
+      if (prep.tn == 64) { if (threadIdx.x < 64) umma_prep::prepare_w_task<64>(prep.g, prep.out, st, tile_n, threadIdx.x); }
+      else if (threadIdx.x < 128) umma_prep::prepare_w_task<128>(prep.g, prep.out, st, tile_n, threadIdx.x);
+    }
     return;
   }
   const int cta = blockIdx.x - n_prep, n_ctas = gridDim.x - n_prep;      // the persistent CTAs of the front end

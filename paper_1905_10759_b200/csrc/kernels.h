@@ -61,10 +61,27 @@ struct UmmaArgs {
   int64_t seg_words;       // K-words per segment
   const unsigned char* w_prep;   // W expanded into [n tile][stage][stage bytes]
 };
-// The weight expansion as a job another kernel can run: n_stages x tiles_n tasks of tn threads each.
+// Argument block of the folded-scale tcgen05 HBMM kernel (group scales carried by fp16 operand pieces).
+struct FoldArgs {
+  const uint32_t* a_bits; const void* a_scales;
+  const uint32_t* w_bits; const void* w_scales;
+  float* C;
+  int64_t M, N, lda_w, ldw_w, lda_s, ldw_s, ldc;
+  int32_t a_bf16, w_bf16;
+  int64_t n_words;         // K / 32 (K is a multiple of 32 on this path)
+  int64_t a_gw, w_gw;      // K-words per scale group of A / W (n_words: one group per row)
+  const unsigned char* w_prep;   // W expanded into [n tile][stage][stage bytes]
+  const float* w_down;           // per weight row: the power of two that undoes its normalisation
+};
+// The weight expansion as a job another kernel can run: n_stages x tiles_n tasks of tn threads each
+// (n_stages counts tasks per column tile: single stages of the e4m3 layout, runs of stages of the folded one).
+// folded == 0: the e4m3 kernel's layout (g); folded == 1: the folded-scale kernel's layout (f, out_down).
 struct UmmaPrepJob {
   UmmaArgs g;
+  FoldArgs f;
   unsigned char* out;
+  float* out_down;
+  int32_t folded;
   int32_t tn, n_stages, tiles_n;
 };
 
@@ -80,6 +97,15 @@ size_t gemm_tensor_workspace_bytes(const PackedView& A, const PackedView& W);
 cudaError_t launch_gemm_tensor(const PackedView& A, const PackedView& W, float* C, int64_t ldc, void* workspace,
                                cudaStream_t stream, bool w_prepared = false);
 void gemm_tensor_prep_job(const PackedView& A, const PackedView& W, void* workspace, UmmaPrepJob* job);
+
+// Packed x packed contraction with the group scales folded into two fp16 pieces per operand (tcgen05 /
+// TMEM, one accumulation over all of K, no per-group step).  Same operand support as the e4m3 kernel.
+cudaError_t read_gemm_fold_error(int* code);
+bool gemm_fold_supported(const PackedView& A, const PackedView& W);
+size_t gemm_fold_workspace_bytes(const PackedView& A, const PackedView& W);
+cudaError_t launch_gemm_fold(const PackedView& A, const PackedView& W, float* C, int64_t ldc, void* workspace,
+                             cudaStream_t stream, bool w_prepared = false);
+void gemm_fold_prep_job(const PackedView& A, const PackedView& W, void* workspace, UmmaPrepJob* job);
 
 // Dense x packed contraction (HBWN), three kernels:
 //   select : sign bit XOR-ed into fp32 activations on the fp32 pipe (any dense dtype);

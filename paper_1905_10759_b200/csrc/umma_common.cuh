@@ -150,7 +150,8 @@ __device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
   asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
   return r;
 }
-// D[tmem] (+)= A[smem desc] * B[smem desc]^T, 128 x N x 16, bf16 operands, fp32 accumulate.
+// D[tmem] (+)= A[smem desc] * B[smem desc]^T, 128 x N x 16, bf16 (or, by the instruction descriptor, fp16)
+// operands, fp32 accumulate.
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
@@ -195,7 +196,8 @@ __host__ __device__ constexpr uint32_t instr_desc(int n, uint32_t ab_format) {
   return (1u << 4) | (ab_format << 7) | (ab_format << 10) | (static_cast<uint32_t>(n >> 3) << 17) |
          (static_cast<uint32_t>(TM >> 4) << 24);
 }
-constexpr uint32_t kFmtE4M3 = 0, kFmtBF16 = 1;
+constexpr uint32_t kFmtE4M3 = 0, kFmtBF16 = 1;   // kind::f8f6f4 / kind::f16 operand codes
+constexpr uint32_t kFmtF16 = 0;                  // kind::f16 with fp16 operands
 
 
 }  // namespace umma

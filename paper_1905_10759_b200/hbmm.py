@@ -26,7 +26,7 @@ _lib = ctypes.CDLL(LIB_PATH)
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(7)
 F32, BF16 = 0, 1
-PATH_AUTO, PATH_POPC, PATH_B1MMA, PATH_TENSOR, PATH_TENSOR_PREPARED = 0, 1, 2, 3, 4
+PATH_AUTO, PATH_POPC, PATH_B1MMA, PATH_TENSOR, PATH_TENSOR_PREPARED, PATH_FOLDED, PATH_FOLDED_PREPARED = 0, 1, 2, 3, 4, 5, 6
 
 EXPORTS = [
     "hbmm_operand_bytes", "hbmm_quantize", "hbmm_gemm_workspace_bytes", "hbmm_gemm", "hbmm_gemm_ex",

@@ -40,10 +40,25 @@ def eff_beta(beta: int, K: int) -> int:
     return K if beta >= K else beta
 
 
-def assert_close_rel_absref(c_gpu: np.ndarray, c_ref: np.ndarray, absref: np.ndarray, rtol: float, what=""):
+def elementwise_magnitude(da: np.ndarray, beta_a: int, dw: np.ndarray, beta_w: int, K: int) -> np.ndarray:
+    """F[m,n] = sum_k |A~[m,k]| |W~[n,k]| = sum_k deltaA[m, k/beta_a] deltaW[n, k/beta_w]: the magnitude of the
+    K individual products.  A kernel that accumulates those products in fp32 (instead of cancelling the
+    +-1 terms of a group in integers first) cannot be closer than a few 2^-24 F where the group dots vanish."""
+    ea = np.repeat(np.asarray(da, dtype=np.float64), beta_a, axis=1)[:, :K]
+    ew = np.repeat(np.asarray(dw, dtype=np.float64), beta_w, axis=1)[:, :K]
+    return ea @ ew.T
+
+
+# Absolute floor of the folded-scale kernel's bound, in units of 2^-24 F (see elementwise_magnitude).
+FOLDED_FLOOR_ULPS = 4.0
+
+
+def assert_close_rel_absref(c_gpu: np.ndarray, c_ref: np.ndarray, absref: np.ndarray, rtol: float, what="", floor=None):
     err = np.abs(c_gpu.astype(np.float64) - c_ref)
     # the second term is the rounding floor of the oracle's own double-precision sum
     bound = rtol * absref + 1e-12 * max(1.0, float(absref.max()))
+    if floor is not None:
+        bound = bound + floor
     bad = err > bound
     if bad.any():
         i = np.unravel_index(np.argmax(err / bound), err.shape)

@@ -145,7 +145,7 @@ GEMM_CASES = [
 
 
 def _paths(hb):
-    return [hb.PATH_POPC, hb.PATH_B1MMA, hb.PATH_TENSOR, hb.PATH_AUTO]
+    return [hb.PATH_POPC, hb.PATH_B1MMA, hb.PATH_TENSOR, hb.PATH_FOLDED, hb.PATH_AUTO]
 
 
 def _gemm_ws(hb, A, W):
@@ -162,6 +162,9 @@ def test_gemm_matches_oracle_on_every_path(hb, M, N, K, ba, bw, sdt):
     A, da, sa = gu.oracle_operand(a, ba, sdt)
     W, dw, sw = gu.oracle_operand(w, bw, sdt)
     c_ref, absref = oracle.hbmm_from_quantized(da, sa, gu.eff_beta(ba, K), dw, sw, gu.eff_beta(bw, K))
+    # the folded-scale kernel (what AUTO runs when it has the workspace) sums the individual products in
+    # fp32: where every group dot is zero the magnitude reference is zero and a few ulps of F remain
+    floor = gu.FOLDED_FLOOR_ULPS * gu.U * gu.elementwise_magnitude(da, gu.eff_beta(ba, K), dw, gu.eff_beta(bw, K), K)
     ran = 0
     ws = _gemm_ws(hb, A, W)
     for path in _paths(hb):
@@ -175,7 +178,8 @@ def test_gemm_matches_oracle_on_every_path(hb, M, N, K, ba, bw, sdt):
         ran += 1
         out = C.cpu().numpy()
         assert np.isnan(out[:, N:]).all()          # nothing written beyond column N
-        gu.assert_close_rel_absref(out[:, :N], c_ref, absref, RTOL, "path %d" % path)
+        gu.assert_close_rel_absref(out[:, :N], c_ref, absref, RTOL, "path %d" % path,
+                                   floor if path in (hb.PATH_FOLDED, hb.PATH_AUTO) else None)
     assert ran >= 2
 
 
@@ -330,6 +334,7 @@ def test_conv_im2col_matches_oracle(hb, B, C, H, W, N, kh, kw, st, pd, ba, bw, s
     w = inputs.he_normal(N, K, 9000 + N)
     Wop, dw, sw = gu.oracle_operand(w, bw)
     a_rows = oracle.im2col(xr, kh, kw, (st, st), (pd, pd))
+    floor = None
     if ba == 1:
         c_ref, absref = oracle.hbwn_from_quantized(a_rows, dw, sw, gu.eff_beta(bw, K))
         rtol = _hbwn_rtol(gu, K, bw)
@@ -337,6 +342,8 @@ def test_conv_im2col_matches_oracle(hb, B, C, H, W, N, kh, kw, st, pd, ba, bw, s
         da, sa = oracle.quantize(a_rows, gu.eff_beta(ba, K))
         c_ref, absref = oracle.hbmm_from_quantized(da, sa, gu.eff_beta(ba, K), dw, sw, gu.eff_beta(bw, K))
         rtol = RTOL
+        # the contraction that follows the front end is the folded-scale kernel when K is whole words
+        floor = gu.FOLDED_FLOOR_ULPS * gu.U * gu.elementwise_magnitude(da, gu.eff_beta(ba, K), dw, gu.eff_beta(bw, K), K)
     geom = hb.make_geom(B, C, H, W, kh, kw, (st, st), (pd, pd))
     xd = torch.from_numpy(x).cuda()
     if xbf16:
@@ -346,7 +353,7 @@ def test_conv_im2col_matches_oracle(hb, B, C, H, W, N, kh, kw, st, pd, ba, bw, s
     M = c_ref.shape[0]
     Cout = torch.full((M, (N + 3) // 4 * 4), float("nan"), device="cuda")
     hb.conv_im2col(xd, geom, ba, hb.F32, Wop, Cout, ws)
-    gu.assert_close_rel_absref(Cout.cpu().numpy()[:, :N], c_ref, absref, rtol)
+    gu.assert_close_rel_absref(Cout.cpu().numpy()[:, :N], c_ref, absref, rtol, "", floor if ba > 1 else None)
     if ba > 1:
         # the packed activation operand left in the workspace: bits exact
         _, _, lw, ls = hb.operand_bytes(M, K, ba, hb.F32)
@@ -394,6 +401,11 @@ def test_prepared_weights_path_repeats_the_tensor_path_bit_for_bit(hb):
     with pytest.raises(hb.HbmmError) as e:
         hb.gemm_ex(A, W, C2, hb.PATH_TENSOR_PREPARED)
     assert e.value.status == hb.ERR_WORKSPACE
+    # the folded-scale kernel
+    C2.fill_(float("nan"))
+    hb.gemm_ex(A, W, C1, hb.PATH_FOLDED, ws)
+    hb.gemm_ex(A, W, C2, hb.PATH_FOLDED_PREPARED, ws)
+    assert torch.equal(C1, C2)
     # dense activations (HBWN)
     _, ab = inputs.as_bf16(a)
     Ad = hb.wrap_dense(torch.from_numpy(ab).cuda().to(torch.bfloat16))
@@ -404,3 +416,40 @@ def test_prepared_weights_path_repeats_the_tensor_path_bit_for_bit(hb):
     assert torch.equal(C1, C2)
     c_ref, absref = oracle.hbwn_from_quantized(ab, dw, sw, 64)
     gu.assert_close_rel_absref(C2.cpu().numpy(), c_ref, absref, _hbwn_rtol(gu, K, 64))
+
+
+@pytest.mark.parametrize("spread", [0, 8, 16])
+def test_folded_path_keeps_the_tolerance_when_group_scales_differ_by_orders_of_magnitude(hb, spread):
+    """The folded-scale kernel normalises every row by a power of two and carries each group scale in two
+    fp16 pieces; scales up to 2^17 below the largest of their row keep 22 significant bits.  Rows whose
+    groups differ by up to 2^spread, rows that are zero, and very large / very small rows must all
+    stay inside the 1e-5 bound."""
+    gu = _gu()
+    M, N, K, beta = 140, 72, 640, 32
+    rng = np.random.default_rng(300 + spread)
+    a = inputs.normal((M, K), 301 + spread)
+    w = inputs.he_normal(N, K, 302 + spread)
+    G = K // beta
+    for x in (a, w):
+        f = np.exp2(rng.integers(-spread, 1, size=(x.shape[0], G))).astype(np.float32)
+        x *= np.repeat(f, beta, axis=1)
+    a[3] = 0.0                       # an all-zero row
+    a[5] *= np.float32(2.0 ** 60)    # rows far from 1: the normalisation is per row
+    a[7] *= np.float32(2.0 ** -60)
+    w[2] *= np.float32(2.0 ** 40)
+    w[9] *= np.float32(2.0 ** -50)
+    A, da, sa = gu.oracle_operand(a, beta)
+    W, dw, sw = gu.oracle_operand(w, beta)
+    c_ref, absref = oracle.hbmm_from_quantized(da, sa, beta, dw, sw, beta)
+    C = torch.full((M, N), float("nan"), device="cuda")
+    hb.gemm_ex(A, W, C, hb.PATH_FOLDED, _gemm_ws(hb, A, W))
+    out = C.cpu().numpy()
+    assert np.all(out[3] == 0.0)
+    floor = gu.FOLDED_FLOOR_ULPS * gu.U * gu.elementwise_magnitude(da, beta, dw, beta, K)
+    # compared block by block, so that the floor of the bound follows each block's own magnitude
+    rows_n = np.array([r for r in range(M) if r not in (3, 5, 7)])
+    cols_n = np.array([c for c in range(N) if c not in (2, 9)])
+    for rows in (rows_n, np.array([5]), np.array([7])):
+        for cols in (cols_n, np.array([2]), np.array([9])):
+            ix = np.ix_(rows, cols)
+            gu.assert_close_rel_absref(out[ix], c_ref[ix], absref[ix], RTOL, "folded, spread 2^%d" % spread, floor[ix])
