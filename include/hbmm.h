@@ -86,8 +86,10 @@ typedef enum {
  *                [g*beta, min((g+1)*beta, K)) (a tail group is averaged over its own length);
  *                entries g >= ceil(K/beta) are zero.  ld_scales is a multiple of 4 (fp32) or 8
  *                (bf16); 16-byte aligned.  bf16 scales are the fp32 scale rounded to nearest even.
- *       Supported beta: multiples of 32, and any beta >= K (one group per row, the XNOR-Net case
- *       of Section 5).  Sub-word beta (2..16) returns HBMM_ERR_UNSUPPORTED.
+ *       Supported beta: multiples of 32; the sub-word powers of two 2, 4, 8 and 16 (the settings of
+ *       the paper's experiments, Section 5; a word then holds 32 / beta groups); and any beta >= K
+ *       (one group per row, the XNOR-Net case of Section 5).  Anything else returns
+ *       HBMM_ERR_UNSUPPORTED.
  *   beta == 1 : the tensor stays at full precision (X~ = X; the paper's first/last layers and the
  *       HBWN mode).  `dense` [rows, ld_dense] of dense_dtype is used, bits/scales are ignored.
  */

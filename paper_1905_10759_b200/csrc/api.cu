@@ -20,8 +20,11 @@ inline int64_t scales_ld(int64_t K, int32_t beta, int32_t dtype) {
   return round_up(num_groups(K, beta), dtype == HBMM_BF16 ? 8 : 4);
 }
 
-// beta values the packed kernels implement: whole words per group, or one group per row.
-inline bool beta_supported(int64_t K, int32_t beta) { return beta >= 2 && (beta % 32 == 0 || beta >= K); }
+// beta values the packed kernels implement: whole words per group, one group per row, or the sub-word
+// powers of two (the settings of the paper's experiments).
+inline bool beta_supported(int64_t K, int32_t beta) {
+  return beta >= 2 && (beta % 32 == 0 || beta >= K || beta == 2 || beta == 4 || beta == 8 || beta == 16);
+}
 
 hbmm_status check_packed(const hbmm_operand* op, bool need_buffers = true) {
   if (!op) return HBMM_ERR_INVALID_ARG;
@@ -140,7 +143,7 @@ hbmm_status gemm_checked(const hbmm_operand* A, const hbmm_operand* W, float* C,
   const PackedView a = view_of(A), w = view_of(W);
   cudaError_t e;
   switch (path) {
-    case HBMM_PATH_POPC: e = launch_gemm_popc(a, w, C, ldc, stream); break;
+    case HBMM_PATH_POPC: e = gemm_subword(a, w) ? launch_gemm_popc_sub(a, w, C, ldc, stream) : launch_gemm_popc(a, w, C, ldc, stream); break;
     case HBMM_PATH_B1MMA:
       if (!gemm_b1_supported(a, w)) return HBMM_ERR_UNSUPPORTED;
       e = launch_gemm_b1(a, w, C, ldc, stream);
@@ -162,7 +165,7 @@ hbmm_status gemm_checked(const hbmm_operand* A, const hbmm_operand* W, float* C,
       else if (gemm_tensor_supported(a, w) && workspace_ok(workspace, workspace_bytes, tensor_workspace(a, w)))
         e = launch_gemm_tensor(a, w, C, ldc, workspace, stream);
       else
-        e = launch_gemm_popc(a, w, C, ldc, stream);
+        e = gemm_subword(a, w) ? launch_gemm_popc_sub(a, w, C, ldc, stream) : launch_gemm_popc(a, w, C, ldc, stream);
       break;
   }
   return e == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
@@ -286,7 +289,8 @@ hbmm_status hbmm_gemm_partials(const hbmm_operand* A, const hbmm_operand* W, int
   const PackedView a = view_of(A), w = view_of(W);
   cudaError_t e;
   if (path == HBMM_PATH_AUTO || path == HBMM_PATH_POPC) {
-    e = launch_partials_popc(a, w, D, static_cast<cudaStream_t>(stream));
+    e = gemm_subword(a, w) ? launch_partials_popc_sub(a, w, D, static_cast<cudaStream_t>(stream))
+                           : launch_partials_popc(a, w, D, static_cast<cudaStream_t>(stream));
   } else if (path == HBMM_PATH_B1MMA) {
     if (!gemm_b1_supported(a, w)) return HBMM_ERR_UNSUPPORTED;
     e = launch_partials_b1(a, w, D, static_cast<cudaStream_t>(stream));

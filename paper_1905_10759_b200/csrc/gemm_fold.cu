@@ -46,7 +46,8 @@ constexpr int kLoaderWarp = kMmaWarp + 1;                   // 13
 constexpr int kFirstScoutWarp = kLoaderWarp + 1;            // 14..17
 constexpr int kScoutWarps = 4;
 constexpr int kThreads = (kFirstScoutWarp + kScoutWarps) * 32;
-constexpr int kDepth = 4;     // stages of packed words + scales each producer thread keeps in flight
+// Stages of packed words + scales each producer thread keeps in flight; fewer when a word has many scales.
+template <int SUBW> struct DepthFor { static constexpr int value = SUBW == 1 ? 4 : (SUBW <= 4 ? 2 : 1); };
 
 template <int TN>
 __global__ void __launch_bounds__(TN)
@@ -63,10 +64,12 @@ struct StageCursor {
   bool in;                   // the row exists
 };
 
-template <int TN>
+// ASUB: scale groups per packed word of A (1: groups of whole words; 2 .. 16: beta_a = 16 .. 2).
+template <int TN, int ASUB>
 __global__ void __launch_bounds__(kThreads, 1)
 hbmm_fold_kernel(const Args g) {
   using S = Smem<TN>;
+  constexpr int kDepth = DepthFor<ASUB>::value;
   constexpr int STAGES = S::STAGES;
   extern __shared__ __align__(1024) unsigned char smem[];
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + S::OFF_BAR);
@@ -119,7 +122,7 @@ hbmm_fold_kernel(const Args g) {
     const int q = pt >> 7;
     const int p = pt & (TM - 1);
     const uint32_t n_words = static_cast<uint32_t>(g.n_words), gw = static_cast<uint32_t>(g.a_gw);
-    const bool vec_scales = !g.a_bf16 && gw == 1;      // one fp32 scale per word: a stage's two scales are one 8-byte load
+    const bool vec_scales = ASUB == 1 && !g.a_bf16 && gw == 1;      // one fp32 scale per word: a stage's two scales are one 8-byte load
     const int64_t total = my_tiles * n_stages;
     auto set_tile = [&](StageCursor& c) {
       const int64_t tile = blockIdx.x + c.ti * gridDim.x;
@@ -135,19 +138,33 @@ hbmm_fold_kernel(const Args g) {
         set_tile(c);
       }
     };
-    auto fetch = [&](const StageCursor& c, uint2& w, float& s0, float& s1) {
+    // raw scales of the stage's two words: sc[0 .. ASUB) of the first, sc[ASUB .. 2 ASUB) of the second
+    auto fetch = [&](const StageCursor& c, uint2& w, float (&sc)[2 * ASUB]) {
       w = make_uint2(0u, 0u);
-      s0 = s1 = 0.0f;
+#pragma unroll
+      for (int i = 0; i < 2 * ASUB; i++) sc[i] = 0.0f;
       const uint32_t wi = static_cast<uint32_t>(c.st) * WPS;
       if (c.in && wi < n_words) {
         w = __ldg(reinterpret_cast<const uint2*>(c.bptr + wi));      // the row is padded with zero words to a multiple of four
-        if (vec_scales) {
+        if (ASUB > 1) {
+          // K is a multiple of 32 here, so every word has all its ASUB groups
+          float lo[ASUB], hi[ASUB];
+          load_scaled<(ASUB > 1 ? ASUB : 2)>(g.a_scales, g.a_bf16, c.srow + static_cast<int64_t>(wi) * ASUB, 1.0f,
+                                             reinterpret_cast<float(&)[(ASUB > 1 ? ASUB : 2)]>(lo));
+#pragma unroll
+          for (int i = 0; i < ASUB; i++) { sc[i] = lo[i]; hi[i] = 0.0f; }
+          if (wi + 1 < n_words)
+            load_scaled<(ASUB > 1 ? ASUB : 2)>(g.a_scales, g.a_bf16, c.srow + static_cast<int64_t>(wi + 1) * ASUB, 1.0f,
+                                               reinterpret_cast<float(&)[(ASUB > 1 ? ASUB : 2)]>(hi));
+#pragma unroll
+          for (int i = 0; i < ASUB; i++) sc[ASUB + i] = hi[i];
+        } else if (vec_scales) {
           const float2 v = __ldg(reinterpret_cast<const float2*>(reinterpret_cast<const float*>(g.a_scales) + c.srow + wi));
-          s0 = v.x;
-          s1 = v.y;                                                    // past the last group: a stored zero
+          sc[0] = v.x;
+          sc[ASUB] = v.y;                                              // past the last group: a stored zero
         } else {
-          s0 = load_scale(g.a_scales, g.a_bf16, c.srow + wi / gw);
-          if (wi + 1 < n_words) s1 = load_scale(g.a_scales, g.a_bf16, c.srow + (wi + 1) / gw);
+          sc[0] = load_scale(g.a_scales, g.a_bf16, c.srow + wi / gw);
+          if (wi + 1 < n_words) sc[ASUB] = load_scale(g.a_scales, g.a_bf16, c.srow + (wi + 1) / gw);
         }
       }
     };
@@ -157,9 +174,9 @@ hbmm_fold_kernel(const Args g) {
     set_tile(pf);
     cur = pf;
     uint2 w[kDepth];
-    float s0[kDepth], s1[kDepth];
+    float sc[kDepth][2 * ASUB];
 #pragma unroll
-    for (int u = 0; u < kDepth; u++) { fetch(pf, w[u], s0[u], s1[u]); advance(pf); }
+    for (int u = 0; u < kDepth; u++) { fetch(pf, w[u], sc[u]); advance(pf); }
     int64_t up_tile = -1;
     float up = 0.0f;
     bool ok = true;
@@ -179,12 +196,21 @@ hbmm_fold_kernel(const Args g) {
           if (ok && my >= STAGES && !mbar_wait(&empty[s], static_cast<uint32_t>(((my / STAGES) & 1) ^ 1), abort_flag, 1)) ok = false;
           if (ok) {
             unsigned char* a1 = smem + S::OFF_A + s * S::A_STAGE;
-            expand_word(a1, a1 + S::A_PIECE, p, 0, w[u].x, s0[u] * up);
-            expand_word(a1, a1 + S::A_PIECE, p, 1, w[u].y, s1[u] * up);
+            if (ASUB == 1) {
+              expand_word(a1, a1 + S::A_PIECE, p, 0, w[u].x, sc[u][0] * up);
+              expand_word(a1, a1 + S::A_PIECE, p, 1, w[u].y, sc[u][ASUB] * up);
+            } else {
+              constexpr int SB = ASUB > 1 ? ASUB : 2;
+              float lo[SB], hi[SB];
+#pragma unroll
+              for (int i = 0; i < ASUB; i++) { lo[i] = sc[u][i] * up; hi[i] = sc[u][ASUB + i] * up; }
+              expand_word_sub<SB>(a1, a1 + S::A_PIECE, p, 0, w[u].x, lo);
+              expand_word_sub<SB>(a1, a1 + S::A_PIECE, p, 1, w[u].y, hi);
+            }
             fence_async_proxy();          // make the generic-proxy stores visible to the tensor core
             __syncwarp();
             if (lane == 0) mbar_arrive(&full[s]);
-            fetch(pf, w[u], s0[u], s1[u]);  // this register slot is free again: load kDepth of my stages ahead
+            fetch(pf, w[u], sc[u]);         // this register slot is free again: load kDepth of my stages ahead
             advance(pf);
             advance(cur);
           }
@@ -339,8 +365,11 @@ Args make_args(const PackedView& A, const PackedView& W, float* C, int64_t ldc) 
   g.M = A.rows; g.N = W.rows; g.lda_w = A.ld_words; g.ldw_w = W.ld_words; g.lda_s = A.ld_scales; g.ldw_s = W.ld_scales;
   g.ldc = ldc; g.a_bf16 = A.scale_bf16; g.w_bf16 = W.scale_bf16;
   g.n_words = A.K / 32;
-  g.a_gw = A.beta >= A.K ? g.n_words : A.beta / 32;
-  g.w_gw = W.beta >= W.K ? g.n_words : W.beta / 32;
+  const bool a_subword = A.beta < 32 && A.beta < A.K, w_subword = W.beta < 32 && W.beta < W.K;
+  g.a_sub = a_subword ? 32 / A.beta : 1;
+  g.w_sub = w_subword ? 32 / W.beta : 1;
+  g.a_gw = A.beta >= A.K ? g.n_words : (a_subword ? 1 : A.beta / 32);
+  g.w_gw = W.beta >= W.K ? g.n_words : (w_subword ? 1 : W.beta / 32);
   g.w_prep = nullptr;
   g.w_down = nullptr;
   return g;
@@ -356,13 +385,13 @@ size_t prep_bytes(const Args& g) {
   return stage_bytes<TN>(g) + static_cast<size_t>((g.N + TN - 1) / TN) * TN * sizeof(float);
 }
 
-template <int TN>
+template <int TN, int ASUB>
 cudaError_t launch_fold(Args g, void* workspace, cudaStream_t stream, bool w_prepared) {
   using S = Smem<TN>;
   static bool configured = false;
   static int sms = 0;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(hbmm_fold_kernel<TN>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::BYTES);
+    cudaError_t e = cudaFuncSetAttribute(hbmm_fold_kernel<TN, ASUB>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::BYTES);
     if (e != cudaSuccess) return e;
     int dev = 0;
     cudaGetDevice(&dev);
@@ -380,19 +409,30 @@ cudaError_t launch_fold(Args g, void* workspace, cudaStream_t stream, bool w_pre
   g.w_down = down;
   const int64_t tiles = ((g.M + TM - 1) / TM) * tiles_n;
   const unsigned grid = static_cast<unsigned>(tiles < sms ? tiles : sms);   // one persistent CTA per SM
-  hbmm_fold_kernel<TN><<<grid, kThreads, S::BYTES, stream>>>(g);
+  hbmm_fold_kernel<TN, ASUB><<<grid, kThreads, S::BYTES, stream>>>(g);
   return cudaGetLastError();
+}
+
+template <int TN>
+cudaError_t launch_fold_tn(const Args& g, void* workspace, cudaStream_t stream, bool w_prepared) {
+  switch (g.a_sub) {
+    case 2: return launch_fold<TN, 2>(g, workspace, stream, w_prepared);
+    case 4: return launch_fold<TN, 4>(g, workspace, stream, w_prepared);
+    case 8: return launch_fold<TN, 8>(g, workspace, stream, w_prepared);
+    case 16: return launch_fold<TN, 16>(g, workspace, stream, w_prepared);
+    default: return launch_fold<TN, 1>(g, workspace, stream, w_prepared);
+  }
 }
 
 }  // namespace
 
-// K a multiple of 32 and scale groups of whole words (or one group per row).
+// K a multiple of 32; scale groups of whole words, one group per row, or the sub-word groups 2, 4, 8, 16.
 bool gemm_fold_supported(const PackedView& A, const PackedView& W) {
   if (A.K % 32 != 0 || A.K / 32 >= (int64_t{1} << 31)) return false;
-  const bool a_one = A.beta >= A.K, w_one = W.beta >= W.K;
-  if (!a_one && A.beta % 32 != 0) return false;
-  if (!w_one && W.beta % 32 != 0) return false;
-  return true;
+  auto ok = [](const PackedView& v) {
+    return v.beta >= v.K || v.beta % 32 == 0 || v.beta == 2 || v.beta == 4 || v.beta == 8 || v.beta == 16;
+  };
+  return ok(A) && ok(W);
 }
 
 // Bytes of workspace: the weight operand as fp16 piece tiles (4 bytes per element) + one float per row.
@@ -405,7 +445,7 @@ size_t gemm_fold_workspace_bytes(const PackedView& A, const PackedView& W) {
 cudaError_t launch_gemm_fold(const PackedView& A, const PackedView& W, float* C, int64_t ldc, void* workspace,
                              cudaStream_t stream, bool w_prepared) {
   const Args g = make_args(A, W, C, ldc);
-  return g.N <= 64 ? launch_fold<64>(g, workspace, stream, w_prepared) : launch_fold<128>(g, workspace, stream, w_prepared);
+  return g.N <= 64 ? launch_fold_tn<64>(g, workspace, stream, w_prepared) : launch_fold_tn<128>(g, workspace, stream, w_prepared);
 }
 
 // The weight expansion of launch_gemm_fold(A, W, ..., workspace) as a job for another kernel.

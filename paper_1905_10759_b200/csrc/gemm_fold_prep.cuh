@@ -109,6 +109,78 @@ __device__ __forceinline__ void expand_word(unsigned char* piece1, unsigned char
   }
 }
 
+// The same for sub-word groups (beta = 32 / SUB = 2 .. 16, the settings of the paper's experiments): the
+// word has SUB scales, group i covering bits [i * beta, (i + 1) * beta).  Position j holds bits j and j + 16,
+// i.e. groups j / beta and j / beta + SUB / 2, so there are SUB / 2 distinct pairs of fp16 values per piece.
+template <int SUB>
+__device__ __forceinline__ void expand_word_sub(unsigned char* piece1, unsigned char* piece2, int row, int q, uint32_t word,
+                                                const float (&scaled)[SUB]) {
+  static_assert(SUB == 2 || SUB == 4 || SUB == 8 || SUB == 16, "beta = 16, 8, 4, 2");
+  constexpr int BETA = 32 / SUB, HALF = SUB / 2;
+  uint32_t h1[HALF], h2[HALF];
+#pragma unroll
+  for (int t = 0; t < HALF; t++) {
+    const __half2 d1 = __floats2half2_rn(scaled[t], scaled[t + HALF]);          // low half: group t, high half: group t + SUB/2
+    const float2 back = __half22float2(d1);
+    const __half2 d2 = __floats2half2_rn(scaled[t] - back.x, scaled[t + HALF] - back.y);
+    h1[t] = *reinterpret_cast<const uint32_t*>(&d1);
+    h2[t] = *reinterpret_cast<const uint32_t*>(&d2);
+  }
+  const uint32_t nw = ~word;
+#pragma unroll
+  for (int c = 0; c < 4; c++) {
+    uint32_t m[4], o1[4], o2[4];
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+      const int j = 4 * c + i;
+      m[i] = (nw << (15 - j)) & 0x80008000u;
+      o1[i] = m[i] ^ h1[j / BETA];
+      o2[i] = m[i] ^ h2[j / BETA];
+    }
+    *reinterpret_cast<uint4*>(swz(piece1, row, 4 * q + c)) = make_uint4(o1[0], o1[1], o1[2], o1[3]);
+    *reinterpret_cast<uint4*>(swz(piece2, row, 4 * q + c)) = make_uint4(o2[0], o2[1], o2[2], o2[3]);
+  }
+}
+
+// SUB scales of one word (index of the first one given), times the row's power of two.
+template <int SUB>
+__device__ __forceinline__ void load_scaled(const void* s, int bf16, int64_t idx, float up, float (&out)[SUB]) {
+  if (!bf16) {
+    const float* p = reinterpret_cast<const float*>(s) + idx;       // idx is a multiple of SUB: vectors stay aligned
+    if (SUB == 2) {
+      const float2 v = __ldg(reinterpret_cast<const float2*>(p));
+      out[0] = v.x * up; out[1] = v.y * up;
+    } else {
+#pragma unroll
+      for (int i = 0; i < SUB / 4; i++) {
+        const float4 v = __ldg(reinterpret_cast<const float4*>(p) + i);
+        out[4 * i] = v.x * up; out[4 * i + 1] = v.y * up; out[4 * i + 2] = v.z * up; out[4 * i + 3] = v.w * up;
+      }
+    }
+  } else {
+    const uint32_t* p = reinterpret_cast<const uint32_t*>(reinterpret_cast<const unsigned short*>(s) + idx);
+#pragma unroll
+    for (int i = 0; i < SUB / 2; i++) {
+      const uint32_t v = __ldg(p + i);
+      out[2 * i] = __uint_as_float(v << 16) * up;
+      out[2 * i + 1] = __uint_as_float(v & 0xFFFF0000u) * up;
+    }
+  }
+}
+
+// One word of a weight row with a run-time number of groups per word.
+__device__ __forceinline__ void expand_weight_word(unsigned char* p1, unsigned char* p2, int row, int q, uint32_t word, const void* scales,
+                                                   int bf16, int64_t idx, int sub, float up, bool valid) {
+  if (!valid) { expand_word(p1, p2, row, q, 0u, 0.0f); return; }
+  switch (sub) {
+    case 2: { float sc[2]; load_scaled<2>(scales, bf16, idx, up, sc); expand_word_sub<2>(p1, p2, row, q, word, sc); break; }
+    case 4: { float sc[4]; load_scaled<4>(scales, bf16, idx, up, sc); expand_word_sub<4>(p1, p2, row, q, word, sc); break; }
+    case 8: { float sc[8]; load_scaled<8>(scales, bf16, idx, up, sc); expand_word_sub<8>(p1, p2, row, q, word, sc); break; }
+    case 16: { float sc[16]; load_scaled<16>(scales, bf16, idx, up, sc); expand_word_sub<16>(p1, p2, row, q, word, sc); break; }
+    default: expand_word(p1, p2, row, q, word, load_scale(scales, bf16, idx) * up); break;
+  }
+}
+
 // Expands kPrepStages consecutive stages of one column tile of the weight operand into the stage layout
 // the main kernel streams: rows 0 .. TN-1 piece 1, rows TN .. 2TN-1 piece 2, exactly as they sit in
 // shared memory.  The task of the first stages also stores the rows' inverse powers of two.
@@ -126,35 +198,15 @@ __device__ __forceinline__ void prepare_w_task(const Args& g, unsigned char* __r
   if (chunk == 0) w_down[n] = down;
   const int64_t st0 = chunk * kPrepStages;
   const int64_t st1 = st0 + kPrepStages < n_stages ? st0 + kPrepStages : n_stages;
-  const bool vec_scales = !g.w_bf16 && g.w_gw == 1;
-  // the words (and, one fp32 scale per word, the scales) of four stages are two 16-byte loads each
-  for (int64_t st = st0; st < st1; st += 4) {
-    uint32_t word[8];
-    float sc[8];
+  for (int64_t st = st0; st < st1; st++) {
+    unsigned char* base = out + (tile_n * n_stages + st) * S::B_STAGE;
 #pragma unroll
-    for (int h = 0; h < 2; h++) {
-      const int64_t wi = st * WPS + 4 * h;
-      uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (in && wi < g.ldw_w) v = __ldg(reinterpret_cast<const uint4*>(g.w_bits + n * g.ldw_w + wi));   // zero words pad the row
-      word[4 * h] = v.x; word[4 * h + 1] = v.y; word[4 * h + 2] = v.z; word[4 * h + 3] = v.w;
-      if (vec_scales) {
-        float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (in && wi < g.ldw_s) f = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(g.w_scales) + n * g.ldw_s + wi));
-        sc[4 * h] = f.x; sc[4 * h + 1] = f.y; sc[4 * h + 2] = f.z; sc[4 * h + 3] = f.w;                  // stored zeros past the last group
-      } else {
-#pragma unroll
-        for (int e = 0; e < 4; e++)
-          sc[4 * h + e] = (in && wi + e < g.n_words) ? load_scale(g.w_scales, g.w_bf16, n * g.ldw_s + (wi + e) / g.w_gw) : 0.0f;
-      }
-    }
-#pragma unroll
-    for (int e = 0; e < 8; e++) {
-      const int64_t sst = st + e / WPS;
-      if (sst < st1) {
-        unsigned char* base = out + (tile_n * n_stages + sst) * S::B_STAGE;
-        const bool valid = st * WPS + e < g.n_words;
-        expand_word(base, base + S::B_PIECE, p, e % WPS, valid ? word[e] : 0u, valid ? sc[e] * up : 0.0f);
-      }
+    for (int q = 0; q < WPS; q++) {
+      const int64_t wi = st * WPS + q;
+      const bool valid = in && wi < g.n_words;
+      const uint32_t word = valid ? __ldg(g.w_bits + n * g.ldw_w + wi) : 0u;
+      const int64_t idx = n * g.ldw_s + (g.w_sub > 1 ? wi * g.w_sub : wi / g.w_gw);
+      expand_weight_word(base, base + S::B_PIECE, p, q, word, g.w_scales, g.w_bf16, idx, g.w_sub, up, valid);
     }
   }
 }

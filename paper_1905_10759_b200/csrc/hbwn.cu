@@ -30,11 +30,14 @@ struct HbwnArgs {
 };
 
 // 64 x 64 tile, 4 x 4 outputs per thread, one K-word (32 elements) per stage.
+// SUB: weight scale groups per K-word (1: groups of whole words; 2 .. 16: beta_w = 16 .. 2, the group
+// sizes of the paper's experiments -- the partial sum is then folded into the output inside the word).
+template <int SUB>
 __global__ void __launch_bounds__(kThreads)
 hbwn_select_kernel(const HbwnArgs g) {
   __shared__ __align__(16) float As[2][32][64 + 4];  // k-major
   __shared__ uint32_t Ws[2][64];
-  __shared__ float WsS[2][64];
+  __shared__ float WsS[2][64][SUB];
   const int t = threadIdx.x, tx = t & 15, ty = t >> 4;
   const int64_t m0 = static_cast<int64_t>(blockIdx.y) * 64, n0 = static_cast<int64_t>(blockIdx.x) * 64;
   float acc[4][4], part[4][4];
@@ -47,7 +50,7 @@ hbwn_select_kernel(const HbwnArgs g) {
   const int srow = t >> 2, sk = (t & 3) * 8;
   float pa[8];
   uint32_t pw = 0;
-  float ps = 0.0f;
+  float ps[SUB];
   auto prefetch = [&](int64_t kw) {
     const int64_t m = m0 + srow;
 #pragma unroll
@@ -58,14 +61,21 @@ hbwn_select_kernel(const HbwnArgs g) {
     if (t < 64) {
       const int64_t n = n0 + t;
       pw = (n < g.N) ? __ldg(g.w_bits + n * g.ldw_w + kw) : 0u;
-      const int64_t grp = kw / g.group_words;
-      ps = (n < g.N && grp < g.Gw) ? load_scale(g.w_scales, g.w_bf16, n * g.ldw_s + grp) : 0.0f;
+#pragma unroll
+      for (int u = 0; u < SUB; u++) {
+        const int64_t grp = SUB > 1 ? kw * SUB + u : kw / g.group_words;
+        ps[u] = (n < g.N && grp < g.Gw) ? load_scale(g.w_scales, g.w_bf16, n * g.ldw_s + grp) : 0.0f;
+      }
     }
   };
   auto stage = [&](int buf) {
 #pragma unroll
     for (int e = 0; e < 8; e++) As[buf][sk + e][srow] = pa[e];
-    if (t < 64) { Ws[buf][t] = pw; WsS[buf][t] = ps; }
+    if (t < 64) {
+      Ws[buf][t] = pw;
+#pragma unroll
+      for (int u = 0; u < SUB; u++) WsS[buf][t][u] = ps[u];
+    }
   };
   prefetch(0);
   stage(0);
@@ -86,12 +96,20 @@ hbwn_select_kernel(const HbwnArgs g) {
 #pragma unroll
         for (int i = 0; i < 4; i++) part[i][j] += __uint_as_float(__float_as_uint(a[i]) ^ flip);
       }
+      if (SUB > 1 && (k + 1) % (32 / SUB) == 0) {      // a sub-word group ends here
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+          const float s = WsS[buf][tx * 4 + j][k / (32 / SUB)];
+#pragma unroll
+          for (int i = 0; i < 4; i++) { acc[i][j] = fmaf(s, part[i][j], acc[i][j]); part[i][j] = 0.0f; }
+        }
+      }
     }
-    const bool group_end = ((kw + 1) % g.group_words == 0) || (kw + 1 == g.n_words);
+    const bool group_end = SUB == 1 && (((kw + 1) % g.group_words == 0) || (kw + 1 == g.n_words));
     if (group_end) {
 #pragma unroll
       for (int j = 0; j < 4; j++) {
-        const float s = WsS[buf][tx * 4 + j];
+        const float s = WsS[buf][tx * 4 + j][0];
 #pragma unroll
         for (int i = 0; i < 4; i++) { acc[i][j] = fmaf(s, part[i][j], acc[i][j]); part[i][j] = 0.0f; }
       }
@@ -122,9 +140,16 @@ cudaError_t launch_hbwn_select(const DenseView& A, const PackedView& W, float* C
   g.C = C; g.ldc = ldc; g.M = A.rows; g.N = W.rows; g.K = A.K;
   g.n_words = (A.K + 31) / 32;
   g.Gw = num_groups(W.K, W.beta);
-  g.group_words = W.beta >= W.K ? g.n_words : W.beta / 32;
+  const bool subword = W.beta < 32 && W.beta < W.K;
+  g.group_words = W.beta >= W.K ? g.n_words : (subword ? 1 : W.beta / 32);
   dim3 grid(static_cast<unsigned>((g.N + 63) / 64), static_cast<unsigned>((g.M + 63) / 64));
-  hbwn_select_kernel<<<grid, kThreads, 0, stream>>>(g);
+  switch (subword ? 32 / W.beta : 1) {
+    case 2: hbwn_select_kernel<2><<<grid, kThreads, 0, stream>>>(g); break;
+    case 4: hbwn_select_kernel<4><<<grid, kThreads, 0, stream>>>(g); break;
+    case 8: hbwn_select_kernel<8><<<grid, kThreads, 0, stream>>>(g); break;
+    case 16: hbwn_select_kernel<16><<<grid, kThreads, 0, stream>>>(g); break;
+    default: hbwn_select_kernel<1><<<grid, kThreads, 0, stream>>>(g); break;
+  }
   return cudaGetLastError();
 }
 

@@ -256,6 +256,7 @@ bool hbwn_mma_supported(const DenseView& A, const PackedView& W) {
   if (!A.bf16) return false;
   if (reinterpret_cast<uintptr_t>(A.data) % 16 != 0 || (A.ld * 2) % 16 != 0) return false;
   if (W.beta >= W.K) return true;
+  if (W.beta % 32 != 0) return false;       // sub-word groups: the tcgen05 and the sign-select kernels take them
   const int64_t gw = W.beta / 32;
   return gw == 1 || gw % 2 == 0;
 }

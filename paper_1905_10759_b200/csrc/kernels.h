@@ -41,6 +41,11 @@ cudaError_t launch_gemm_popc(const PackedView& A, const PackedView& W, float* C,
 cudaError_t launch_partials_popc(const PackedView& A, const PackedView& W, int32_t* D,
                                  cudaStream_t stream);
 
+// The same for sub-word segments (the finer grouping is 2, 4, 8 or 16 elements): masked popcounts inside a word.
+bool gemm_subword(const PackedView& A, const PackedView& W);
+cudaError_t launch_gemm_popc_sub(const PackedView& A, const PackedView& W, float* C, int64_t ldc, cudaStream_t stream);
+cudaError_t launch_partials_popc_sub(const PackedView& A, const PackedView& W, int32_t* D, cudaStream_t stream);
+
 // Packed x packed contraction on the legacy b1 tensor instruction (segment multiple of 128 bits).
 bool gemm_b1_supported(const PackedView& A, const PackedView& W);
 cudaError_t launch_gemm_b1(const PackedView& A, const PackedView& W, float* C, int64_t ldc,
@@ -70,6 +75,7 @@ struct FoldArgs {
   int32_t a_bf16, w_bf16;
   int64_t n_words;         // K / 32 (K is a multiple of 32 on this path)
   int64_t a_gw, w_gw;      // K-words per scale group of A / W (n_words: one group per row)
+  int32_t a_sub, w_sub;    // scale groups per K-word: 1, or 32 / beta for the sub-word groups beta = 2 .. 16
   const unsigned char* w_prep;   // W expanded into [n tile][stage][stage bytes]
   const float* w_down;           // per weight row: the power of two that undoes its normalisation
 };

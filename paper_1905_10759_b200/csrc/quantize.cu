@@ -117,6 +117,87 @@ quantize_small_beta(const void* __restrict__ x, int64_t rows, int64_t K, int64_t
   }
 }
 
+// Sub-word groups (beta = 2, 4, 8 or 16 < K): the paper's own settings (Section 5 uses beta 2 .. 16).
+// Same warp item as above (32 lanes x EPT consecutive elements of one row); a group lies inside one
+// thread's elements (beta <= EPT) or inside beta / EPT neighbouring lanes, so its sum is a pairwise tree
+// in registers followed by at most two shuffle steps.  Scales leave as EPT / beta consecutive values
+// per thread, i.e. contiguous across the warp.
+template <bool BF16, int BETA>
+__global__ void __launch_bounds__(kThreads)
+quantize_subword(const void* __restrict__ x, int64_t rows, int64_t K, int64_t ldx, bool vec_ok,
+                 uint32_t* __restrict__ bits, int64_t ld_words, void* __restrict__ scales, int64_t ld_scales,
+                 int scale_bf16, int64_t G) {
+  using L = In<BF16>;
+  constexpr int EPT = L::EPT;
+  constexpr int LPW = 32 / EPT;
+  constexpr int WPW = EPT;
+  constexpr int GPT = EPT >= BETA ? EPT / BETA : 1;     // groups per thread
+  constexpr int LPG = EPT >= BETA ? 1 : BETA / EPT;     // lanes per group
+  const int lane = threadIdx.x & 31;
+  const int64_t chunks = (ld_words + WPW - 1) / WPW;
+  const int64_t items = rows * chunks;
+  const int64_t warp0 = (static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x) >> 5;
+  const int64_t nwarps = (static_cast<int64_t>(gridDim.x) * kThreads) >> 5;
+  for (int64_t it = warp0; it < items; it += nwarps) {
+    const int64_t row = it / chunks, chunk = it - row * chunks;
+    const int64_t k0 = (chunk * WPW * 32) + lane * EPT;
+    float v[EPT];
+    uint32_t sb = 0;
+    if (vec_ok && k0 + EPT <= K) {
+      const typename L::Vec* p = reinterpret_cast<const typename L::Vec*>(
+          reinterpret_cast<const char*>(x) + (row * ldx + k0) * (BF16 ? 2 : 4));
+      L::unpack(__ldg(p), v);
+#pragma unroll
+      for (int e = 0; e < EPT; e++) sb |= (v[e] >= 0.0f ? 1u : 0u) << e;
+    } else {
+#pragma unroll
+      for (int e = 0; e < EPT; e++) {
+        const bool in = k0 + e < K;
+        v[e] = in ? L::scalar(x, row * ldx + k0 + e) : 0.0f;      // absent columns: value 0, sign bit 0
+        sb |= ((in && v[e] >= 0.0f) ? 1u : 0u) << e;
+      }
+    }
+    uint32_t word = sb << (EPT * (lane % LPW));
+#pragma unroll
+    for (int off = 1; off < LPW; off <<= 1) word |= __shfl_xor_sync(0xffffffffu, word, off);
+    const int64_t wi = chunk * WPW + lane / LPW;
+    if ((lane % LPW) == 0 && wi < ld_words) bits[row * ld_words + wi] = word;
+    // group sums of |x|
+#pragma unroll
+    for (int e = 0; e < EPT; e++) v[e] = fabsf(v[e]);
+    constexpr int SPAN = EPT >= BETA ? BETA : EPT;     // elements of one group inside a thread
+#pragma unroll
+    for (int w = 1; w < SPAN; w <<= 1)
+#pragma unroll
+      for (int e = 0; e < EPT; e += 2 * w) v[e] += v[e + w];
+#pragma unroll
+    for (int off = 1; off < LPG; off <<= 1) v[0] += __shfl_xor_sync(0xffffffffu, v[0], off);
+    if ((lane % LPG) == 0) {
+#pragma unroll
+      for (int i = 0; i < GPT; i++) {
+        const int64_t g = k0 / BETA + i;
+        if (g < G) {
+          const int64_t cnt = (K - g * BETA < BETA) ? (K - g * BETA) : BETA;
+          store_scale(scales, scale_bf16, row * ld_scales + g, v[i * SPAN] / static_cast<float>(cnt));
+          if (g == G - 1)
+            for (int64_t z = G; z < ld_scales; z++) store_scale(scales, scale_bf16, row * ld_scales + z, 0.0f);
+        }
+      }
+    }
+  }
+}
+
+template <bool BF16>
+void launch_subword(int beta, unsigned blocks, cudaStream_t stream, const void* x, int64_t rows, int64_t K, int64_t ldx, bool vec_ok,
+                    uint32_t* bits, int64_t ld_words, void* scales, int64_t ld_scales, int scale_bf16, int64_t G) {
+  switch (beta) {
+    case 2: quantize_subword<BF16, 2><<<blocks, kThreads, 0, stream>>>(x, rows, K, ldx, vec_ok, bits, ld_words, scales, ld_scales, scale_bf16, G); break;
+    case 4: quantize_subword<BF16, 4><<<blocks, kThreads, 0, stream>>>(x, rows, K, ldx, vec_ok, bits, ld_words, scales, ld_scales, scale_bf16, G); break;
+    case 8: quantize_subword<BF16, 8><<<blocks, kThreads, 0, stream>>>(x, rows, K, ldx, vec_ok, bits, ld_words, scales, ld_scales, scale_bf16, G); break;
+    default: quantize_subword<BF16, 16><<<blocks, kThreads, 0, stream>>>(x, rows, K, ldx, vec_ok, bits, ld_words, scales, ld_scales, scale_bf16, G); break;
+  }
+}
+
 // General path: beta any multiple of 32, or one group per row (beta >= K).  One block per row;
 // the per-word |x| sums are kept in shared memory and each group is then summed by one warp
 // (lane-strided partial sums followed by a shuffle tree).
@@ -184,6 +265,18 @@ cudaError_t launch_quantize(const void* x, int x_bf16, int64_t rows, int64_t K, 
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (!one_group && beta < 32) {
+    if (beta != 2 && beta != 4 && beta != 8 && beta != 16) return cudaErrorInvalidValue;
+    const int64_t chunks = (ld_words + wpw - 1) / wpw;
+    const int64_t items = rows * chunks;
+    int64_t blocks = (items + (kThreads / 32) - 1) / (kThreads / 32);
+    const int64_t cap = static_cast<int64_t>(sms) * 16;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    if (x_bf16) launch_subword<true>(beta, static_cast<unsigned>(blocks), stream, x, rows, K, ldx, vec_ok, bits, ld_words, scales, ld_scales, scale_bf16, G);
+    else launch_subword<false>(beta, static_cast<unsigned>(blocks), stream, x, rows, K, ldx, vec_ok, bits, ld_words, scales, ld_scales, scale_bf16, G);
+    return cudaGetLastError();
+  }
   if (!one_group && pow2 && beta_words <= wpw) {
     const int64_t chunks = (ld_words + wpw - 1) / wpw;
     const int64_t items = rows * chunks;

@@ -100,7 +100,7 @@ def test_host_validation_rejects_before_launch(hb):
     assert gemm(A, W, cptr=ctypes.c_void_p(0x3004)) == hb.ERR_ALIGNMENT          # C not 16-byte aligned
     assert gemm(A, W, ldc=6) == hb.ERR_ALIGNMENT                                 # ldc % 4
     assert gemm(A, W, cptr=None) == hb.ERR_INVALID_ARG
-    assert gemm(_fake_packed(hb, 8, 64, 16), W) == hb.ERR_UNSUPPORTED            # sub-word beta
+    assert gemm(_fake_packed(hb, 8, 64, 12), W) == hb.ERR_UNSUPPORTED            # sub-word beta that is no power of two
     assert gemm(_fake_packed(hb, 8, 64, 32, bits=0x1004), W) == hb.ERR_ALIGNMENT
     assert gemm(_fake_packed(hb, 8, 64, 32, lw=2), W) == hb.ERR_ALIGNMENT        # ld_words % 4
     assert gemm(_fake_packed(hb, 8, 64, 32, lw=1), W) == hb.ERR_INVALID_ARG      # ld_words too small
@@ -121,8 +121,8 @@ def test_host_validation_rejects_before_launch(hb):
     assert lib.hbmm_quantize(x, 0, 9, 64, 64, ctypes.byref(q.desc), None) == hb.ERR_INVALID_ARG   # rows mismatch
     assert lib.hbmm_quantize(None, 0, 8, 64, 64, ctypes.byref(q.desc), None) == hb.ERR_INVALID_ARG
     assert lib.hbmm_quantize(x, 5, 8, 64, 64, ctypes.byref(q.desc), None) == hb.ERR_INVALID_ARG
-    q16 = _fake_packed(hb, 8, 64, 8)
-    assert lib.hbmm_quantize(x, 0, 8, 64, 64, ctypes.byref(q16.desc), None) == hb.ERR_UNSUPPORTED
+    q24 = _fake_packed(hb, 8, 64, 24)
+    assert lib.hbmm_quantize(x, 0, 8, 64, 64, ctypes.byref(q24.desc), None) == hb.ERR_UNSUPPORTED
 
     g = hb.make_geom(2, 4, 8, 8, 3, 3, (1, 1), (1, 1))
     Wc = _fake_packed(hb, 4, 36, 36)
@@ -137,4 +137,4 @@ def test_host_validation_rejects_before_launch(hb):
     assert call(g, _fake_packed(hb, 4, 40, 40), ws, n.value) == hb.ERR_INVALID_ARG    # K != C*kh*kw
     bad = hb.make_geom(2, 4, 2, 2, 5, 5, (1, 1), (0, 0))
     assert call(bad, Wc, ws, n.value) == hb.ERR_INVALID_ARG                           # filter larger than image
-    assert call(g, Wc, ws, n.value, beta_a=8) == hb.ERR_UNSUPPORTED
+    assert call(g, Wc, ws, n.value, beta_a=12) == hb.ERR_UNSUPPORTED

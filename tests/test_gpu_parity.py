@@ -43,6 +43,17 @@ QUANT_CASES = [
     (20, 333, 32, True, 1, 8),
     (11, 2048, 256, True, 0, 0),
     (1, 1, 32, False, 0, 0),
+    # sub-word groups, the settings of the paper's experiments (Section 5: beta 2 .. 16)
+    (64, 576, 16, False, 0, 0),
+    (37, 100, 8, False, 0, 0),     # ragged K: 100 = 12 * 8 + 4, tail group of four
+    (33, 333, 4, False, 1, 0),     # tail group of one element, bf16 scales
+    (20, 576, 2, False, 0, 0),
+    (5, 45, 2, False, 0, 3),       # unaligned rows -> scalar loads, odd K
+    (130, 1000, 16, True, 0, 0),   # bf16 input: eight elements per thread
+    (16, 264, 8, True, 1, 0),
+    (9, 77, 4, True, 0, 8),
+    (12, 512, 2, True, 0, 0),
+    (4, 8, 16, False, 0, 0),       # beta >= K: one group per row
 ]
 
 
@@ -94,7 +105,9 @@ def test_quantize_signs_of_special_values(hb):
 
 # ------------------------------------------------------------------ integer partials (bit exact)
 PARTIAL_CASES = [(33, 17, 256, 32, 32), (20, 9, 100, 32, 64), (8, 8, 576, 128, 32), (5, 6, 333, 333, 32),
-                 (4, 3, 384, 96, 96), (6, 7, 77, 77, 77), (3, 5, 1024, 256, 64)]
+                 (4, 3, 384, 96, 96), (6, 7, 77, 77, 77), (3, 5, 1024, 256, 64),
+                 # sub-word segments: masked popcounts inside a word
+                 (9, 7, 256, 16, 16), (6, 5, 100, 4, 4), (5, 4, 77, 2, 16), (4, 6, 128, 8, 64), (3, 3, 45, 45, 2)]
 
 
 @pytest.mark.parametrize("M,N,K,ba,bw", PARTIAL_CASES)
@@ -141,6 +154,15 @@ GEMM_CASES = [
     (40, 1000, 4096, 64, 64, 0),     # FC-style ragged N = 1000
     (1, 1000, 4096, 64, 64, 0),      # batch 1
     (3, 5, 31, 32, 32, 0),           # K below one word
+    # sub-word groups (beta 2 .. 16, Section 5), alone and mixed as in the paper's tables (beta_a <= beta_w)
+    (200, 72, 576, 16, 16, 0),
+    (130, 140, 1152, 4, 4, 0),
+    (70, 64, 256, 2, 16, 0),
+    (65, 33, 320, 8, 64, 0),         # sub-word activations against word-multiple weight groups
+    (40, 50, 384, 2, 2, 1),          # bf16 scales
+    (33, 40, 100, 4, 8, 0),          # K no multiple of 32: integer-pipe path only
+    (50, 60, 320, 320, 16, 0),       # one group per row against beta 16
+    (300, 130, 640, 32, 8, 0),       # finer weight groups
 ]
 
 
@@ -222,7 +244,8 @@ def test_quantize_then_gemm_end_to_end(hb):
 
 
 # ------------------------------------------------------------------ HBWN (beta_a = 1)
-HBWN_CASES = [(256, 64, 576, 32, True), (100, 130, 1152, 32, True), (65, 70, 100, 32, True), (40, 33, 576, 64, False),
+HBWN_CASES = [(130, 72, 576, 16, True), (65, 40, 320, 4, True), (40, 33, 100, 2, False), (70, 130, 256, 8, True),   # sub-word weight groups
+              (256, 64, 576, 32, True), (100, 130, 1152, 32, True), (65, 70, 100, 32, True), (40, 33, 576, 64, False),
               (30, 40, 333, 333, True), (129, 256, 2304, 32, True), (8, 16, 64, 32, False), (300, 64, 576, 64, True),
               (130, 200, 672, 128, True), (70, 50, 96, 64, True), (257, 129, 1160, 1160, True), (33, 64, 40, 32, True),
               (64, 72, 384, 96, True)]
@@ -285,6 +308,11 @@ def test_hbwn_tensor_path_needs_its_workspace(hb):
 # ------------------------------------------------------------------ convolution front end
 CONV_CASES = [
     # B, C, H, W, N, kh, kw, stride, pad, beta_a, beta_w, signed, x bf16
+    # sub-word groups (Section 5: beta_a / beta_w such as 2/16, 4/4, 1/4)
+    (2, 64, 8, 8, 64, 3, 3, 1, 1, 16, 16, True, False),
+    (2, 32, 6, 6, 16, 3, 3, 1, 1, 2, 16, True, False),
+    (2, 20, 7, 7, 33, 3, 3, 1, 1, 4, 4, True, False),       # K = 180: no whole words, integer-pipe contraction
+    (2, 64, 8, 8, 64, 3, 3, 1, 1, 1, 4, True, True),        # HBWN with beta_w = 4
     (2, 64, 8, 8, 64, 3, 3, 1, 1, 32, 32, True, False),
     (2, 64, 8, 8, 64, 3, 3, 1, 1, 32, 32, False, False),    # post-ReLU: every sign bit is 1
     (3, 32, 7, 9, 40, 3, 3, 1, 1, 64, 32, True, False),
