@@ -74,8 +74,48 @@ __device__ __forceinline__ void load_signs_abs(const void* x, int64_t row_off, i
   asum = v[0];
 }
 
+// Loads only (no reduction): the EPT elements starting at column k0 of a row; columns >= K read as 0 with
+// the `in` mask cleared, so that several loads can be issued before the first one is used.
+template <bool BF16>
+__device__ __forceinline__ void load_elems(const void* x, int64_t row_off, int64_t k0, int64_t K, bool vec_ok,
+                                           float (&v)[In<BF16>::EPT], uint32_t& in_mask) {
+  using L = In<BF16>;
+  constexpr int EPT = L::EPT;
+  if (vec_ok && k0 + EPT <= K) {
+    const typename L::Vec* p = reinterpret_cast<const typename L::Vec*>(
+        reinterpret_cast<const char*>(x) + (row_off + k0) * (BF16 ? 2 : 4));
+    L::unpack(__ldg(p), v);
+    in_mask = (1u << EPT) - 1u;
+  } else {
+    in_mask = 0;
+#pragma unroll
+    for (int e = 0; e < EPT; e++) {
+      const bool in = k0 + e < K;
+      v[e] = in ? L::scalar(x, row_off + k0 + e) : 0.0f;
+      in_mask |= (in ? 1u : 0u) << e;
+    }
+  }
+}
+template <int EPT>
+__device__ __forceinline__ void signs_and_abs_sum(float (&v)[EPT], uint32_t in_mask, uint32_t& sbits, float& asum) {
+  sbits = 0;
+#pragma unroll
+  for (int e = 0; e < EPT; e++) sbits |= (v[e] >= 0.0f ? 1u : 0u) << e;
+  sbits &= in_mask;
+#pragma unroll
+  for (int e = 0; e < EPT; e++) v[e] = fabsf(v[e]);
+#pragma unroll
+  for (int w = 1; w < EPT; w <<= 1)
+#pragma unroll
+    for (int e = 0; e < EPT; e += 2 * w) v[e] += v[e + w];
+  asum = v[0];
+}
+
 // Fast path: beta/32 is a power of two no larger than the words one warp covers.
-// One warp item = WPW consecutive words of one row.
+// One warp item = WPW consecutive words of one row; a warp takes kUnroll items per trip and issues all
+// their loads before it touches the first value (the kernel is a pure stream: what limits it is the
+// number of bytes in flight).
+constexpr int kUnroll = 4;
 template <bool BF16>
 __global__ void __launch_bounds__(kThreads)
 quantize_small_beta(const void* __restrict__ x, int64_t rows, int64_t K, int64_t ldx, bool vec_ok,
@@ -90,31 +130,136 @@ quantize_small_beta(const void* __restrict__ x, int64_t rows, int64_t K, int64_t
   const int64_t warp0 = (static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x) >> 5;
   const int64_t nwarps = (static_cast<int64_t>(gridDim.x) * kThreads) >> 5;
   const int64_t beta = static_cast<int64_t>(beta_words) * 32;
-  for (int64_t it = warp0; it < items; it += nwarps) {
-    const int64_t row = it / chunks, chunk = it - row * chunks;
-    const int64_t k0 = (chunk * WPW * 32) + lane * EPT;
-    uint32_t sb;
-    float s;
-    load_signs_abs<BF16>(x, row * ldx, k0, K, vec_ok, sb, s);
-    uint32_t word = sb << (EPT * (lane % LPW));
+  const int bw_shift = __ffs(beta_words) - 1;                 // beta_words is a power of two on this path
+  // (row, chunk) of the next item are carried along instead of divided out of the item number
+  const int64_t step_rows = nwarps / chunks, step_chunks = nwarps - step_rows * chunks;
+  int64_t nrow = warp0 / chunks, nchunk = warp0 - nrow * chunks;
+  for (int64_t it0 = warp0; it0 < items; it0 += nwarps * kUnroll) {
+    float v[kUnroll][EPT];
+    uint32_t in_mask[kUnroll];
+    int64_t row[kUnroll], chunk[kUnroll];
 #pragma unroll
-    for (int off = 1; off < LPW; off <<= 1) {
-      word |= __shfl_xor_sync(0xffffffffu, word, off);
-      s += __shfl_xor_sync(0xffffffffu, s, off);
+    for (int u = 0; u < kUnroll; u++) {
+      const int64_t it = it0 + u * nwarps;
+      row[u] = nrow;
+      chunk[u] = nchunk;
+      nrow += step_rows;
+      nchunk += step_chunks;
+      if (nchunk >= chunks) { nchunk -= chunks; nrow++; }
+      in_mask[u] = 0;
+      if (it < items) load_elems<BF16>(x, row[u] * ldx, (chunk[u] * WPW * 32) + lane * EPT, K, vec_ok, v[u], in_mask[u]);
     }
-    for (int off = LPW; off < LPW * beta_words; off <<= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
-    const int64_t wi = chunk * WPW + lane / LPW;
-    if ((lane % LPW) == 0 && wi < ld_words) bits[row * ld_words + wi] = word;
-    if ((lane % (LPW * beta_words)) == 0) {
-      const int64_t g = wi / beta_words;
-      if (g < G) {
-        const int64_t cnt = (K - g * beta < beta) ? (K - g * beta) : beta;
-        store_scale(scales, scale_bf16, row * ld_scales + g, s / static_cast<float>(cnt));
-        if (g == G - 1)
-          for (int64_t z = G; z < ld_scales; z++) store_scale(scales, scale_bf16, row * ld_scales + z, 0.0f);
+#pragma unroll
+    for (int u = 0; u < kUnroll; u++) {
+      if (it0 + u * nwarps >= items) break;
+      uint32_t sb;
+      float s;
+      signs_and_abs_sum<EPT>(v[u], in_mask[u], sb, s);
+      uint32_t word = sb << (EPT * (lane % LPW));
+#pragma unroll
+      for (int off = 1; off < LPW; off <<= 1) {
+        word |= __shfl_xor_sync(0xffffffffu, word, off);
+        s += __shfl_xor_sync(0xffffffffu, s, off);
+      }
+      for (int off = LPW; off < LPW * beta_words; off <<= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+      const int64_t wi = chunk[u] * WPW + lane / LPW;
+      if ((lane % LPW) == 0 && wi < ld_words) bits[row[u] * ld_words + wi] = word;
+      if ((lane % (LPW * beta_words)) == 0) {
+        const int64_t g = wi >> bw_shift;
+        if (g < G) {
+          const int64_t cnt = (K - g * beta < beta) ? (K - g * beta) : beta;
+          store_scale(scales, scale_bf16, row[u] * ld_scales + g, s / static_cast<float>(cnt));
+          if (g == G - 1)
+            for (int64_t z = G; z < ld_scales; z++) store_scale(scales, scale_bf16, row[u] * ld_scales + z, 0.0f);
+        }
       }
     }
   }
+}
+
+// Stream path: rows without padding (ldx == K), K a multiple of 32 and of beta, beta a power of two from
+// 2 to 512.  The tensor is then one contiguous run of elements whose words and groups never straddle a
+// row, and the kernel is written for instructions per element: a lane owns 16 consecutive elements
+// (64 bytes of fp32, 32 of bf16), so a packed word is two lanes and a beta = 32 group sum one shuffle.
+// Sign(x) = +1 for x >= 0 including -0: adding +0.0 turns -0 into +0, after which the IEEE sign bit
+// decides; it is shifted into the lane's 16-bit sign field with one funnel shift per element.
+template <bool BF16, int BETA>
+__global__ void __launch_bounds__(kThreads)
+quantize_stream(const void* __restrict__ x, int64_t total_words, uint32_t n_words, uint32_t* __restrict__ bits, int64_t ld_words,
+                void* __restrict__ scales, int64_t ld_scales, int scale_bf16, uint32_t G) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp0 = (static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x) >> 5;
+  const int64_t nwarps = (static_cast<int64_t>(gridDim.x) * kThreads) >> 5;
+  const int64_t items = (total_words + 15) / 16;                  // 16 words = 512 elements per warp and trip
+  for (int64_t it = warp0; it < items; it += nwarps) {
+    const int64_t fw = it * 16 + (lane >> 1);                      // this lane's word, counted over the whole tensor
+    const bool live = fw < total_words;
+    float v[16];
+    if (live) {
+      if (BF16) {
+        const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned short*>(x) + fw * 32 + (lane & 1) * 16);
+        const uint4 a = __ldg(p), b = __ldg(p + 1);
+        In<true>::unpack(a, v);
+        In<true>::unpack(b, v + 8);
+      } else {
+        const float4* p = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(x) + fw * 32 + (lane & 1) * 16);
+        const float4 a = __ldg(p), b = __ldg(p + 1), c = __ldg(p + 2), d = __ldg(p + 3);
+        In<false>::unpack(a, v); In<false>::unpack(b, v + 4); In<false>::unpack(c, v + 8); In<false>::unpack(d, v + 12);
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < 16; e++) v[e] = 0.0f;
+    }
+    uint32_t neg = 0;                                             // bit e set <=> element e is negative
+#pragma unroll
+    for (int e = 15; e >= 0; e--) neg = __funnelshift_l(__float_as_uint(v[e] + 0.0f), neg, 1);
+    const uint32_t sb = ~neg & 0xFFFFu;
+    const uint32_t other = __shfl_xor_sync(0xffffffffu, sb, 1);
+    const uint32_t row = static_cast<uint32_t>(fw / n_words), wi = static_cast<uint32_t>(fw - static_cast<int64_t>(row) * n_words);
+    if (live && (lane & 1) == 0) {
+      uint32_t* brow = bits + static_cast<int64_t>(row) * ld_words;
+      brow[wi] = sb | (other << 16);
+      if (wi == 0) {                                              // the row's zero padding
+        for (int64_t z = n_words; z < ld_words; z++) brow[z] = 0u;
+        for (int64_t z = G; z < ld_scales; z++) store_scale(scales, scale_bf16, static_cast<int64_t>(row) * ld_scales + z, 0.0f);
+      }
+    }
+    // pairwise sums of |x|: after the level of width w, v[e] (e a multiple of 2w) holds the sum of 2w elements
+#pragma unroll
+    for (int e = 0; e < 16; e++) v[e] = fabsf(v[e]);
+    constexpr int IN_LANE = BETA < 16 ? BETA : 16;
+#pragma unroll
+    for (int w = 1; w < IN_LANE; w <<= 1)
+#pragma unroll
+      for (int e = 0; e < 16; e += 2 * w) v[e] += v[e + w];
+    constexpr float inv = 1.0f / static_cast<float>(BETA);        // beta is a power of two: the same as dividing
+    if constexpr (BETA <= 16) {
+      constexpr int GPL = 16 / BETA;                              // groups per lane, consecutive in the scale row
+      const int64_t g0 = static_cast<int64_t>(row) * ld_scales + (wi * 32u + (lane & 1) * 16u) / BETA;
+      if (live) {
+#pragma unroll
+        for (int i = 0; i < GPL; i++) store_scale(scales, scale_bf16, g0 + i, v[i * BETA] * inv);
+      }
+    } else {
+      constexpr int LANES = BETA / 16;                            // lanes per group
+      float sum = v[0];
+#pragma unroll
+      for (int off = 1; off < LANES; off <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+      if (live && (lane % LANES) == 0)
+        store_scale(scales, scale_bf16, static_cast<int64_t>(row) * ld_scales + wi / (BETA / 32), sum * inv);
+    }
+  }
+}
+
+template <bool BF16>
+bool launch_stream(int beta, unsigned blocks, cudaStream_t stream, const void* x, int64_t total_words, uint32_t n_words, uint32_t* bits,
+                   int64_t ld_words, void* scales, int64_t ld_scales, int scale_bf16, uint32_t G) {
+#define HBMM_QS(B) case B: quantize_stream<BF16, B><<<blocks, kThreads, 0, stream>>>(x, total_words, n_words, bits, ld_words, scales, ld_scales, scale_bf16, G); return true;
+  switch (beta) {
+    HBMM_QS(2) HBMM_QS(4) HBMM_QS(8) HBMM_QS(16) HBMM_QS(32) HBMM_QS(64) HBMM_QS(128) HBMM_QS(256) HBMM_QS(512)
+    default: return false;
+  }
+#undef HBMM_QS
 }
 
 // Sub-word groups (beta = 2, 4, 8 or 16 < K): the paper's own settings (Section 5 uses beta 2 .. 16).
@@ -138,8 +283,13 @@ quantize_subword(const void* __restrict__ x, int64_t rows, int64_t K, int64_t ld
   const int64_t items = rows * chunks;
   const int64_t warp0 = (static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x) >> 5;
   const int64_t nwarps = (static_cast<int64_t>(gridDim.x) * kThreads) >> 5;
+  const int64_t step_rows = nwarps / chunks, step_chunks = nwarps - step_rows * chunks;
+  int64_t nrow = warp0 / chunks, nchunk = warp0 - nrow * chunks;
   for (int64_t it = warp0; it < items; it += nwarps) {
-    const int64_t row = it / chunks, chunk = it - row * chunks;
+    const int64_t row = nrow, chunk = nchunk;
+    nrow += step_rows;
+    nchunk += step_chunks;
+    if (nchunk >= chunks) { nchunk -= chunks; nrow++; }
     const int64_t k0 = (chunk * WPW * 32) + lane * EPT;
     float v[EPT];
     uint32_t sb = 0;
@@ -265,6 +415,17 @@ cudaError_t launch_quantize(const void* x, int x_bf16, int64_t rows, int64_t K, 
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (!one_group && vec_ok && ldx == K && K % 32 == 0 && K % beta == 0 && K / 32 < (int64_t{1} << 31) && rows < (int64_t{1} << 31)) {
+    const int64_t total_words = rows * (K / 32);
+    int64_t blocks = ((total_words + 15) / 16 + (kThreads / 32) - 1) / (kThreads / 32);
+    const int64_t cap = static_cast<int64_t>(sms) * 16;
+    if (blocks > cap) blocks = cap;
+    const bool ok = x_bf16 ? launch_stream<true>(beta, static_cast<unsigned>(blocks), stream, x, total_words, static_cast<uint32_t>(K / 32), bits,
+                                                 ld_words, scales, ld_scales, scale_bf16, static_cast<uint32_t>(G))
+                           : launch_stream<false>(beta, static_cast<unsigned>(blocks), stream, x, total_words, static_cast<uint32_t>(K / 32), bits,
+                                                  ld_words, scales, ld_scales, scale_bf16, static_cast<uint32_t>(G));
+    if (ok) return cudaGetLastError();
+  }
   if (!one_group && beta < 32) {
     if (beta != 2 && beta != 4 && beta != 8 && beta != 16) return cudaErrorInvalidValue;
     const int64_t chunks = (ld_words + wpw - 1) / wpw;
