@@ -228,6 +228,37 @@ def kernel_breakdown(torch, hbmm, layers, iters: int):
     return out
 
 
+def side_measurements(torch, hbmm, peaks, iters: int):
+    """Rows of the hot path that the convolution step only runs in fused form, timed on their own on the
+    conv3_x matrix view (M = 50176, K = 1152, N = 128; 231 MB of fp32 input, larger than L2):
+    hbmm_quantize alone (HBM bound), and the folded-scale contraction at the sub-word group sizes of the
+    paper's experiments.  Reported beside the step, not part of it."""
+    hbm_gbs, bf16_tflops, _ = peaks
+    M, N, K = 50176, 128, 1152
+    g = torch.Generator(device="cuda")
+    g.manual_seed(19160)
+    a = torch.randn((M, K), device="cuda", generator=g)
+    w = torch.randn((N, K), device="cuda", generator=g) * (2.0 / K) ** 0.5
+    out = []
+    for beta in (32, 4):
+        A = hbmm.alloc_operand(M, K, beta, hbmm.F32)
+        ms = time_loop(torch, lambda: hbmm.quantize(a, A), iters)
+        by = 4.0 * M * K + A.bits.numel() * 4.0 + A.scales.numel() * 4.0
+        out.append({"kernel": "hbmm_quantize/beta%d" % beta, "shape": [M, K], "ms": round(ms, 5), "bound": "hbm",
+                    "achieved": by / (ms * 1e-3) / 1e9, "peak": hbm_gbs, "unit": "GB/s", "frac": by / (ms * 1e-3) / 1e9 / hbm_gbs})
+    for ba, bw in ((16, 16), (4, 4), (2, 16)):
+        A = hbmm.quantize(a, hbmm.alloc_operand(M, K, ba, hbmm.F32))
+        W = hbmm.quantize(w, hbmm.alloc_operand(N, K, bw, hbmm.F32))
+        ws = torch.empty(max(hbmm.gemm_workspace_bytes(A, W), 16), dtype=torch.uint8, device="cuda")
+        C = torch.empty((M, N), device="cuda")
+        hbmm.gemm_ex(A, W, C, hbmm.PATH_FOLDED, ws)
+        ms = time_loop(torch, lambda: hbmm.gemm_ex(A, W, C, hbmm.PATH_FOLDED_PREPARED, ws), iters)
+        ach = 2.0 * M * N * K / (ms * 1e-3) / 1e12
+        out.append({"kernel": "hbmm_fold_kernel/beta_a%d_beta_w%d" % (ba, bw), "shape": [M, N, K], "ms": round(ms, 5), "bound": "tensor",
+                    "achieved": ach, "peak": bf16_tflops, "unit": "TFLOP/s", "frac": ach / bf16_tflops})
+    return out
+
+
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
 # (same kernels, same workload); entries are dropped when a kernel changes after its capture.
 NCU_DRAM_BYTES = {
@@ -449,7 +480,9 @@ def run_ours(args):
         return 0
 
     base = None
+    side = None
     if world == 1:
+        side = side_measurements(torch, hbmm, peaks, max(5, min(args.steps, 20)))
         base, _, _ = cpu_baseline(shapes, 12.0)
 
     line = {
@@ -467,6 +500,7 @@ def run_ours(args):
         },
         "roofline": roof,
         "kernels": kernels,
+        "other_rows": side,
         "e2e": {"value": aggregate(ops_step, world, ms_e2e), "unit": "TOPS", "ms_per_step": ms_e2e,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": LAUNCHES_PER_STEP * args.steps,

@@ -69,7 +69,10 @@ typedef enum {
                            largest scale).  The K products are summed one by one in fp32, so
                            the error follows sum_k |A~[m,k]| |W~[n,k]| (a few 2^-24 of it) instead of
                            vanishing where group dots cancel.  What HBMM_PATH_AUTO picks when it has
-                           the workspace and the finer grouping has at most 128 elements per group.   */
+                           the workspace and the finer grouping has at most 128 elements per group.
+                           HBWN: bf16 activations x weights written as TWO bf16 pieces (the group
+                           scale to 2^-17 instead of 2^-26; activations carry 2^-9), 128-column
+                           tiles; what HBMM_PATH_AUTO picks for dense bf16 activations.              */
   HBMM_PATH_FOLDED_PREPARED = 6 /* HBMM_PATH_FOLDED with the expanded weights of an earlier
                            HBMM_PATH_FOLDED / AUTO call reused, as HBMM_PATH_TENSOR_PREPARED          */
 } hbmm_path;

@@ -122,11 +122,11 @@ hbmm_status gemm_checked(const hbmm_operand* A, const hbmm_operand* W, float* C,
         if (!hbwn_mma_supported(dv, w)) return HBMM_ERR_UNSUPPORTED;
         e = launch_hbwn_mma(dv, w, C, ldc, stream);
         break;
-      case HBMM_PATH_FOLDED: return HBMM_ERR_UNSUPPORTED;   // dense activations have no group scales to fold
-      case HBMM_PATH_TENSOR:
+      case HBMM_PATH_FOLDED:      // two bf16 pieces per weight (group scale to 2^-17)
+      case HBMM_PATH_TENSOR:      // three (2^-26)
         if (!hbwn_umma_supported(dv, w)) return HBMM_ERR_UNSUPPORTED;
         if (!umma) return HBMM_ERR_WORKSPACE;
-        e = launch_hbwn_umma(dv, w, C, ldc, workspace, stream, w_prepared);
+        e = launch_hbwn_umma(dv, w, C, ldc, workspace, stream, w_prepared, path == HBMM_PATH_TENSOR);
         break;
       default:
         if (umma) e = launch_hbwn_umma(dv, w, C, ldc, workspace, stream);

@@ -7,14 +7,17 @@
 // per-group full-precision scaling to 2^-26 of each weight -- with no per-group epilogue at all: the
 // whole K walk of a tile is one accumulation in TMEM and the epilogue runs once per tile.
 // The three pieces of a 64-column tile are stacked along N, so one 128 x 192 x 16 MMA per K-step
-// forms all three products (the instruction costs about the same for any N <= 128, so stacking is
-// nearly three times cheaper than three accumulating MMAs); the epilogue adds the three column blocks.
+// forms all three products; the epilogue adds the three column blocks.
+// The default variant keeps two pieces (delta = d1 + d2 to 2^-17, still far finer than the 2^-9 of a bf16
+// activation) and 128-column tiles: one 128 x 256 x 16 MMA per K-step.  The kernel is bound by
+// shared-memory traffic (operand reads of the tensor core plus the copies that fill the stages), and that
+// variant moves 24 KB instead of 40 KB per 128 x 128 outputs and K-step.
 //
 // One persistent CTA per SM.  Stage = 64 K-elements: the A tile (128 rows x 128 bytes) arrives by
 // one tiled tensor copy (TMA, 128-byte swizzle, zeros past M and K), the three weight pieces of the
 // stage (192 rows) by one bulk copy from the workspace, where a small kernel has laid them out once
 // per call.  All operand tiles use the 128-byte-swizzled K-major layout.
-//   warps 0-3 : epilogue (TMEM lanes 32*w.., three blocks of TN columns, once per tile)
+//   warps 0-3 : epilogue (TMEM lanes 32*w.., one block of TN columns per piece, once per tile)
 //   warp  4   : one thread issues both copies of every stage
 //   warp  5   : TMEM allocation and the MMA-issuing thread
 // Waits are bounded as in the packed kernel (error word, CTA-wide abort flag, orderly teardown).
@@ -32,7 +35,6 @@ using namespace umma;
 constexpr int kThreads = 6 * 32;
 constexpr int kLoaderWarp = 4, kMmaWarp = 5;
 constexpr int KB = 64;            // K elements per stage (128 bytes of bf16 per row)
-constexpr int STAGES = 5;
 
 struct Args {
   const __nv_bfloat16* a; int64_t lda;
@@ -56,30 +58,39 @@ __device__ __forceinline__ float load_scale(const void* s, int bf16, int64_t idx
   return __ldg(reinterpret_cast<const float*>(s) + idx);
 }
 
-template <int TN>
+// TN: columns of the CTA tile.  NP: bf16 pieces per weight -- 3 carry the fp32 group scale to 2^-26 (64-column
+// tiles: 192 stacked rows per MMA), 2 carry it to 2^-17 (128-column tiles: 256 stacked rows per MMA, which
+// moves 40 % fewer shared-memory bytes per output, the resource that bounds this kernel).
+template <int TN, int NP>
 struct Smem {
   static constexpr int A_STAGE = TM * 128;
   static constexpr int B_PIECE = TN * 128;
-  static constexpr int B_STAGE = 3 * B_PIECE;
+  static constexpr int B_STAGE = NP * B_PIECE;
+  static constexpr int STAGES = (200 * 1024) / (A_STAGE + B_STAGE);
   static constexpr int OFF_A = 0;
   static constexpr int OFF_B = OFF_A + STAGES * A_STAGE;
   static constexpr int OFF_BAR = OFF_B + STAGES * B_STAGE;
-  static constexpr int NBAR = 2 * STAGES + 4 + 1;      // full, empty, tfull[2], tempty[2], drain
+  static constexpr int NBAR = 2 * STAGES + 4 + 2;      // full, empty, tfull[2], tempty[2], drain, wfull
   static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
   static constexpr int USED = OFF_MISC + 16;
   static constexpr int BYTES = USED > 120 * 1024 ? USED : 120 * 1024;   // one CTA per SM
-  static constexpr int NST = 3 * TN;                   // MMA N: the three pieces side by side
+  static constexpr int NST = NP * TN;                  // MMA N: the pieces side by side
   static constexpr int TMEM_COLS = 512;                // two accumulator buffers of NST columns
+  // Resident mode (one column tile whose weight pieces fit beside the activation ring): the pieces of all
+  // K blocks are copied into shared memory once per CTA and only activation tiles stream afterwards.
+  static constexpr int RES_STAGES = 4;
+  static constexpr int RES_OFF_B = RES_STAGES * A_STAGE;
+  static constexpr int RES_MAX_B = 225 * 1024 - RES_OFF_B - 512;        // bytes of weight pieces that fit
   static_assert(NST <= 256 && NST % 16 == 0 && 2 * NST <= TMEM_COLS, "one MMA covers the stacked pieces");
 };
 
-// Writes the three bf16 pieces of W~ for one (column tile, k block): thread = (row, 16-byte piece of
+// Writes the NP bf16 pieces of W~ for one (column tile, k block): thread = (row, 16-byte piece of
 // 8 consecutive stage columns).  Stage column q of block kb is element k = kb * 64 + q of the weight
 // row (plain mode) or channel c = cb * 64 + q at filter tap t, k = c * taps + t (convolution mode,
 // kb = t * cblocks + cb).  The element is +-piece_i(deltaW[n, k / beta]); zero past K / C and past N.
-template <int TN>
+template <int TN, int NP>
 __device__ __forceinline__ void prepare_w_pieces_block(const Args& g, unsigned char* __restrict__ out, int64_t kb, int64_t tile_n) {
-  using S = Smem<TN>;
+  using S = Smem<TN, NP>;
   unsigned char* base = out + (tile_n * g.n_kb + kb) * S::B_STAGE;
   const int64_t tap = g.conv ? kb / g.cblocks : 0;
   const int64_t q0 = (g.conv ? kb - tap * g.cblocks : kb) * KB;     // first channel / element of the block
@@ -111,20 +122,20 @@ __device__ __forceinline__ void prepare_w_pieces_block(const Args& g, unsigned c
           const uint32_t neg = (word[e] & 1u) ? 0u : 0x8000u;   // bit 0 <=> Sign = -1
           const uint32_t h[3] = {__bfloat16_as_ushort(b1) ^ neg, __bfloat16_as_ushort(b2) ^ neg, __bfloat16_as_ushort(b3) ^ neg};
 #pragma unroll
-          for (int i = 0; i < 3; i++) o[i][e >> 1] |= h[i] << ((e & 1) * 16);
+          for (int i = 0; i < NP; i++) o[i][e >> 1] |= h[i] << ((e & 1) * 16);
         }
       }
     }
 #pragma unroll
-    for (int i = 0; i < 3; i++)
+    for (int i = 0; i < NP; i++)
       *reinterpret_cast<uint4*>(swz(base + i * S::B_PIECE, row, piece)) = make_uint4(o[i][0], o[i][1], o[i][2], o[i][3]);
   }
 }
 
-template <int TN>
+template <int TN, int NP>
 __global__ void __launch_bounds__(256)
 prepare_w_pieces_kernel(const Args g, unsigned char* __restrict__ out) {
-  prepare_w_pieces_block<TN>(g, out, blockIdx.x, blockIdx.y);
+  prepare_w_pieces_block<TN, NP>(g, out, blockIdx.x, blockIdx.y);
 }
 
 // Convolution front end in one launch: the first `n_copy` blocks transpose the input to NHWC bf16, the
@@ -135,7 +146,7 @@ struct CopyArgs {
   int32_t gx, gy;          // pixel blocks and channel blocks per image
   int64_t n_copy;
 };
-template <int TN>
+template <int TN, int NP>
 __global__ void __launch_bounds__(256)
 nhwc_and_pieces_kernel(const CopyArgs c, const Args g, unsigned char* __restrict__ w_out) {
   __shared__ unsigned short tile[kNhwcCB][kNhwcPitch];
@@ -148,22 +159,27 @@ nhwc_and_pieces_kernel(const CopyArgs c, const Args g, unsigned char* __restrict
   } else {
     const int64_t j = blk - c.n_copy;
     const int64_t tile_n = j / g.n_kb;
-    prepare_w_pieces_block<TN>(g, w_out, j - tile_n * g.n_kb, tile_n);
+    prepare_w_pieces_block<TN, NP>(g, w_out, j - tile_n * g.n_kb, tile_n);
   }
 }
 
-template <int TN>
+template <int TN, int NP, bool RES>
 __global__ void __launch_bounds__(kThreads, 1)
 hbwn_umma_kernel(const Args g, const __grid_constant__ CUtensorMap a_map) {
-  using S = Smem<TN>;
+  using S = Smem<TN, NP>;
+  constexpr int STAGES = RES ? S::RES_STAGES : S::STAGES;
   extern __shared__ __align__(1024) unsigned char smem[];
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem + S::OFF_BAR);
+  // resident mode: [activation ring][all weight pieces][barriers]; streaming mode: the static layout of Smem
+  const int off_b = RES ? S::RES_OFF_B : S::OFF_B;
+  const int off_bar = RES ? S::RES_OFF_B + static_cast<int>(g.n_kb) * S::B_STAGE : S::OFF_BAR;
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + off_bar);
   uint64_t* empty = full + STAGES;
   uint64_t* tfull = empty + STAGES;
   uint64_t* tempty = tfull + 2;
   uint64_t* drain = tempty + 2;
-  uint32_t* tmem_base_ptr = reinterpret_cast<uint32_t*>(smem + S::OFF_MISC);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + S::OFF_MISC + 4);
+  uint64_t* wfull = drain + 1;                            // resident mode: all weight pieces have arrived
+  uint32_t* tmem_base_ptr = reinterpret_cast<uint32_t*>(wfull + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_base_ptr + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int64_t tiles_n = (g.N + TN - 1) / TN, tiles_m = (g.M + TM - 1) / TM;
@@ -178,6 +194,7 @@ hbwn_umma_kernel(const Args g, const __grid_constant__ CUtensorMap a_map) {
     }
     for (int b = 0; b < 2; b++) { mbar_init(&tfull[b], 1); mbar_init(&tempty[b], 4); }
     mbar_init(drain, 1);
+    mbar_init(wfull, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -199,6 +216,12 @@ hbwn_umma_kernel(const Args g, const __grid_constant__ CUtensorMap a_map) {
       int s = 0;
       uint32_t round = 0;
       bool ok = true;
+      if (RES && my_tiles > 0) {
+        // one column tile: its weight pieces are the same for every row tile of this CTA
+        mbar_arrive_expect_tx(wfull, static_cast<uint32_t>(n_kb) * S::B_STAGE);
+        for (int64_t kb = 0; kb < n_kb; kb++)
+          bulk_copy_g2s(smem + off_b + kb * S::B_STAGE, g.w_prep + kb * S::B_STAGE, S::B_STAGE, wfull);
+      }
       for (int64_t ti = 0; ti < my_tiles && ok; ti++) {
         const int64_t tile = blockIdx.x + ti * gridDim.x;
         const int64_t tile_m = tile / tiles_n, tile_n = tile - tile_m * tiles_n;
@@ -216,14 +239,14 @@ hbwn_umma_kernel(const Args g, const __grid_constant__ CUtensorMap a_map) {
         int32_t cb = 0, fi = 0, fj = 0;
         for (int32_t kb = 0; kb < static_cast<int32_t>(n_kb); kb++) {
           if (round > 0 && !mbar_wait(&empty[s], (round & 1) ^ 1, abort_flag, 1)) { ok = false; break; }
-          mbar_arrive_expect_tx(&full[s], S::A_STAGE + S::B_STAGE);
+          mbar_arrive_expect_tx(&full[s], RES ? S::A_STAGE : S::A_STAGE + S::B_STAGE);
           // the innermost coordinate (a channel or K offset, a multiple of 64 elements) is 128-byte aligned
           if (g.conv)
             tma_load_im2col_4d(smem + S::OFF_A + s * S::A_STAGE, &a_map, cb * KB, w0, h0, b, static_cast<uint16_t>(fj),
                                static_cast<uint16_t>(fi), &full[s]);
           else
             tma_load_2d(smem + S::OFF_A + s * S::A_STAGE, &a_map, kb * KB, static_cast<int32_t>(m0), &full[s]);
-          bulk_copy_g2s(smem + S::OFF_B + s * S::B_STAGE, src, S::B_STAGE, &full[s]);
+          if (!RES) bulk_copy_g2s(smem + off_b + s * S::B_STAGE, src, S::B_STAGE, &full[s]);
           src += S::B_STAGE;
           if (++cb == g.cblocks) { cb = 0; if (++fj == g.kw) { fj = 0; fi++; } }
           if (++s == STAGES) { s = 0; round++; }
@@ -235,12 +258,13 @@ hbwn_umma_kernel(const Args g, const __grid_constant__ CUtensorMap a_map) {
     // =========================== MMA issuer ===========================
     if (lane == 0) {
       constexpr uint32_t idesc = instr_desc(S::NST, kFmtBF16);
-      const uint64_t da0 = smem_desc(smem_u32(smem + S::OFF_A)), db0 = smem_desc(smem_u32(smem + S::OFF_B));
+      const uint64_t da0 = smem_desc(smem_u32(smem + S::OFF_A)), db0 = smem_desc(smem_u32(smem + off_b));
       const uint64_t da_hi = da0 & 0xFFFFFFFF00000000ull, db_hi = db0 & 0xFFFFFFFF00000000ull;
       const uint32_t da_lo = static_cast<uint32_t>(da0), db_lo = static_cast<uint32_t>(db0);
       const uint32_t full_a = smem_u32(full), empty_a = smem_u32(empty), tfull_a = smem_u32(tfull), tempty_a = smem_u32(tempty);
       uint32_t s = 0, full_par = 0;
       bool ok = true;
+      if (RES && my_tiles > 0) ok = mbar_wait(wfull, 0, abort_flag, 6);
       for (int64_t ti = 0; ti < my_tiles && ok; ti++) {
         const uint32_t buf = static_cast<uint32_t>(ti & 1);
         if (ti >= 2) {      // the epilogue must have drained this accumulator (used by tile ti - 2)
@@ -251,7 +275,8 @@ hbwn_umma_kernel(const Args g, const __grid_constant__ CUtensorMap a_map) {
         for (int64_t kb = 0; kb < n_kb; kb++) {
           if (!mbar_wait_a(full_a + s * 8, full_par, abort_flag, 2)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t a_lo = da_lo + s * (S::A_STAGE >> 4), b_lo = db_lo + s * (S::B_STAGE >> 4);
+          const uint32_t a_lo = da_lo + s * (S::A_STAGE >> 4);
+          const uint32_t b_lo = db_lo + (RES ? static_cast<uint32_t>(kb) : s) * (S::B_STAGE >> 4);
 #pragma unroll
           for (int ks = 0; ks < KB / 16; ks++)          // 16 K-elements = 32 bytes along the swizzled rows
             umma_bf16(d_tmem, da_hi | (a_lo + ks * 2), db_hi | (b_lo + ks * 2), idesc, (kb | ks) != 0 ? 1u : 0u);
@@ -277,19 +302,22 @@ hbwn_umma_kernel(const Args g, const __grid_constant__ CUtensorMap a_map) {
       float* dst = g.C + m * g.ldc + nb;
 #pragma unroll
       for (int c = 0; c < TN / 32; c++) {
-        uint32_t v1[32], v2[32], v3[32];
+        uint32_t v[NP][32];
         const uint32_t t_addr = tmem_base + t_lane + buf * S::NST + c * 32;
-        tmem_ld32(t_addr, v1);
-        tmem_ld32(t_addr + TN, v2);
-        tmem_ld32(t_addr + 2 * TN, v3);
+#pragma unroll
+        for (int i = 0; i < NP; i++) tmem_ld32(t_addr + i * TN, v[i]);
         tmem_ld_wait();
         if (m < g.M) {
 #pragma unroll
           for (int j = 0; j < 32; j += 4) {
             float o[4];
 #pragma unroll
-            for (int e = 0; e < 4; e++)      // smallest pieces first
-              o[e] = __uint_as_float(v1[j + e]) + (__uint_as_float(v2[j + e]) + __uint_as_float(v3[j + e]));
+            for (int e = 0; e < 4; e++) {    // smallest pieces first
+              float acc = __uint_as_float(v[NP - 1][j + e]);
+#pragma unroll
+              for (int i = NP - 2; i >= 0; i--) acc += __uint_as_float(v[i][j + e]);
+              o[e] = acc;
+            }
             const int64_t n = nb + c * 32 + j;
             if (g.c_vec && n + 3 < g.N)
               *reinterpret_cast<float4*>(dst + c * 32 + j) = make_float4(o[0], o[1], o[2], o[3]);
@@ -329,9 +357,9 @@ Args make_args(const DenseView& A, const PackedView& W, float* C, int64_t ldc) {
   return g;
 }
 
-template <int TN>
+template <int TN, int NP>
 size_t prep_bytes(const Args& g) {
-  return static_cast<size_t>(((g.N + TN - 1) / TN) * g.n_kb) * Smem<TN>::B_STAGE;
+  return static_cast<size_t>(((g.N + TN - 1) / TN) * g.n_kb) * Smem<TN, NP>::B_STAGE;
 }
 
 // Tensor map of the activation matrix: bf16 [M, K] with row pitch lda, boxes of 64 x 128 elements
@@ -382,14 +410,17 @@ Args make_conv_args(const ConvGeom& c, const PackedView& W, float* C, int64_t ld
   return g;
 }
 
-template <int TN>
+template <int TN, int NP>
 cudaError_t launch(Args g, const CUtensorMap& a_map, void* workspace, cudaStream_t stream, const CopyArgs* copy = nullptr,
                    bool w_prepared = false) {
-  using S = Smem<TN>;
+  using S = Smem<TN, NP>;
+  constexpr int kResBytes = 225 * 1024;
   static bool configured = false;
   static int sms = 0;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(hbwn_umma_kernel<TN>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::BYTES);
+    cudaError_t e = cudaFuncSetAttribute(hbwn_umma_kernel<TN, NP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::BYTES);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(hbwn_umma_kernel<TN, NP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kResBytes);
     if (e != cudaSuccess) return e;
     int dev = 0;
     cudaGetDevice(&dev);
@@ -401,15 +432,27 @@ cudaError_t launch(Args g, const CUtensorMap& a_map, void* workspace, cudaStream
   if (copy) {
     const int64_t blocks = copy->n_copy + n_kb * tiles_n;
     if (blocks > 0x7fffffff) return cudaErrorNotSupported;
-    nhwc_and_pieces_kernel<TN><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(*copy, g, static_cast<unsigned char*>(workspace));
+    nhwc_and_pieces_kernel<TN, NP><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(*copy, g, static_cast<unsigned char*>(workspace));
   } else if (!w_prepared) {
-    prepare_w_pieces_kernel<TN><<<pgrid, 256, 0, stream>>>(g, static_cast<unsigned char*>(workspace));
+    prepare_w_pieces_kernel<TN, NP><<<pgrid, 256, 0, stream>>>(g, static_cast<unsigned char*>(workspace));
   }
   g.w_prep = static_cast<const unsigned char*>(workspace);
   const int64_t tiles = ((g.M + TM - 1) / TM) * tiles_n;
   const unsigned grid = static_cast<unsigned>(tiles < sms ? tiles : sms);
-  hbwn_umma_kernel<TN><<<grid, kThreads, S::BYTES, stream>>>(g, a_map);
+  // a single column tile whose pieces fit beside the activation ring stays resident in shared memory
+  if (tiles_n == 1 && n_kb * S::B_STAGE <= S::RES_MAX_B && tiles > sms)
+    hbwn_umma_kernel<TN, NP, true><<<grid, kThreads, kResBytes, stream>>>(g, a_map);
+  else
+    hbwn_umma_kernel<TN, NP, false><<<grid, kThreads, S::BYTES, stream>>>(g, a_map);
   return cudaGetLastError();
+}
+
+// exact: three pieces, 64-column tiles.  Otherwise two pieces: 128-column tiles when there are more than 64 columns.
+cudaError_t launch_any(const Args& g, const CUtensorMap& a_map, void* workspace, cudaStream_t stream, const CopyArgs* copy, bool w_prepared,
+                       bool exact) {
+  if (exact) return launch<64, 3>(g, a_map, workspace, stream, copy, w_prepared);
+  if (g.N <= 64) return launch<64, 2>(g, a_map, workspace, stream, copy, w_prepared);
+  return launch<128, 2>(g, a_map, workspace, stream, copy, w_prepared);
 }
 
 }  // namespace
@@ -423,17 +466,19 @@ bool hbwn_umma_supported(const DenseView& A, const PackedView& W) {
          encode_tiled_fn() != nullptr;
 }
 
+// enough for either piece count (the three-piece layout is the larger one)
 size_t hbwn_umma_workspace_bytes(const DenseView& A, const PackedView& W) {
   const Args g = make_args(A, W, nullptr, 0);
-  return prep_bytes<64>(g);
+  const size_t a = prep_bytes<64, 3>(g), b = prep_bytes<128, 2>(g);
+  return a > b ? a : b;
 }
 
 cudaError_t launch_hbwn_umma(const DenseView& A, const PackedView& W, float* C, int64_t ldc, void* workspace,
-                             cudaStream_t stream, bool w_prepared) {
+                             cudaStream_t stream, bool w_prepared, bool exact) {
   const Args g = make_args(A, W, C, ldc);
   CUtensorMap a_map;
   if (!make_a_map(g, &a_map)) return cudaErrorNotSupported;
-  return launch<64>(g, a_map, workspace, stream, nullptr, w_prepared);
+  return launch_any(g, a_map, workspace, stream, nullptr, w_prepared, exact);
 }
 
 // Implicit-GEMM convolution: whole 64-channel blocks (every tile row is then 128 bytes of real
@@ -446,7 +491,8 @@ bool hbwn_umma_conv_supported(const ConvGeom& c, const PackedView& W) {
 
 size_t hbwn_umma_conv_workspace_bytes(const ConvGeom& c, const PackedView& W) {
   const Args g = make_conv_args(c, W, nullptr, 0);
-  return prep_bytes<64>(g);
+  const size_t a = prep_bytes<64, 2>(g), b = prep_bytes<128, 2>(g);
+  return a > b ? a : b;
 }
 
 cudaError_t launch_hbwn_umma_conv(const void* x, int x_bf16, void* x_nhwc, int Cp, const ConvGeom& c, const PackedView& W, float* C,
@@ -460,7 +506,7 @@ cudaError_t launch_hbwn_umma_conv(const void* x, int x_bf16, void* x_nhwc, int C
   cp.gx = static_cast<int32_t>((cp.HW + kNhwcPB - 1) / kNhwcPB);
   cp.gy = (Cp + kNhwcCB - 1) / kNhwcCB;
   cp.n_copy = static_cast<int64_t>(cp.gx) * cp.gy * c.B;
-  return launch<64>(g, a_map, workspace, stream, &cp);
+  return launch_any(g, a_map, workspace, stream, &cp, false, false);
 }
 
 cudaError_t read_hbwn_umma_error(int* code) {

@@ -123,8 +123,9 @@ bool hbwn_mma_supported(const DenseView& A, const PackedView& W);
 cudaError_t launch_hbwn_mma(const DenseView& A, const PackedView& W, float* C, int64_t ldc, cudaStream_t stream);
 bool hbwn_umma_supported(const DenseView& A, const PackedView& W);
 size_t hbwn_umma_workspace_bytes(const DenseView& A, const PackedView& W);
+// exact: three bf16 pieces per weight (group scale to 2^-26); otherwise two (2^-17), the faster layout.
 cudaError_t launch_hbwn_umma(const DenseView& A, const PackedView& W, float* C, int64_t ldc, void* workspace,
-                             cudaStream_t stream, bool w_prepared = false);
+                             cudaStream_t stream, bool w_prepared = false, bool exact = false);
 
 // HBWN convolution without the im2col matrix: NCHW -> NHWC bf16 copy (Cp = channels rounded up to 8;
 // launch_hbwn_umma_conv does it in the same launch as the weight-piece layout), then the tcgen05 kernel

@@ -80,7 +80,7 @@ def test_resnet_conv_hbwn_full_batch(hb, li):
     dw, sw = oracle.quantize(w, BETA)
     dw = oracle.round_scales(dw, "f32")
     G = s.K // BETA
-    rtol = (BETA + G + 4) * 2 * gu.U
+    rtol = (BETA + G + 4) * 2 * gu.U + 2.0 ** -18     # fp32 sums + the weight scale carried by two bf16 pieces
     per_image = s.M // s.B
     for b in (0, s.B // 2, s.B - 1):
         rows = oracle.im2col(xb[b:b + 1], s.kh, s.kw, (s.stride, s.stride), (s.pad, s.pad))

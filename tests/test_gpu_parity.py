@@ -251,9 +251,12 @@ HBWN_CASES = [(130, 72, 576, 16, True), (65, 40, 320, 4, True), (40, 33, 100, 2,
               (64, 72, 384, 96, True)]
 
 
-def _hbwn_rtol(gu, K, beta_w):
+def _hbwn_rtol(gu, K, beta_w, two_pieces=False):
     be = gu.eff_beta(beta_w, K)
-    return (be + -(-K // be) + 4) * 2 * gu.U       # sequential fp32 sums inside and across groups, x2 margin
+    rtol = (be + -(-K // be) + 4) * 2 * gu.U       # sequential fp32 sums inside and across groups, x2 margin
+    if two_pieces:
+        rtol += 2.0 ** -18                         # the default tensor-core kernel carries the weight scale in two bf16 pieces
+    return rtol
 
 
 @pytest.mark.parametrize("M,N,K,bw,abf16", HBWN_CASES)
@@ -269,27 +272,30 @@ def test_hbwn_matches_oracle(hb, M, N, K, bw, abf16):
     if abf16:
         ad = ad.to(torch.bfloat16)
     rtol = _hbwn_rtol(gu, K, bw)
-    assert rtol < RTOL_BF16
+    rtol2 = _hbwn_rtol(gu, K, bw, True)
+    assert rtol2 < RTOL_BF16
     A = hb.wrap_dense(ad)
     ws = _gemm_ws(hb, A, W)
     ran = 0
-    # TENSOR: tcgen05 kernel; B1MMA: warp-level bf16 mma.sync kernel; POPC: fp32 sign-select kernel
-    for path, wsp in ((hb.PATH_AUTO, ws), (hb.PATH_AUTO, None), (hb.PATH_TENSOR, ws), (hb.PATH_B1MMA, None),
+    # TENSOR: tcgen05 kernel, three weight pieces; FOLDED (and AUTO with a workspace): two pieces;
+    # B1MMA: warp-level bf16 mma.sync kernel; POPC: fp32 sign-select kernel
+    for path, wsp in ((hb.PATH_AUTO, ws), (hb.PATH_AUTO, None), (hb.PATH_TENSOR, ws), (hb.PATH_FOLDED, ws), (hb.PATH_B1MMA, None),
                       (hb.PATH_POPC, None)):
         C = torch.full((M, (N + 3) // 4 * 4 + 4), float("nan"), device="cuda")
         try:
             hb.gemm_ex(A, W, C, path, wsp)
         except hb.HbmmError as e:
             # the two tensor-core kernels take bf16 activations whose rows start on 16-byte boundaries
-            assert e.status == hb.ERR_UNSUPPORTED and path in (hb.PATH_TENSOR, hb.PATH_B1MMA)
-            if path == hb.PATH_TENSOR:
+            assert e.status == hb.ERR_UNSUPPORTED and path in (hb.PATH_TENSOR, hb.PATH_FOLDED, hb.PATH_B1MMA)
+            if path in (hb.PATH_TENSOR, hb.PATH_FOLDED):
                 assert not abf16 or K % 8 != 0
             continue
         ran += 1
         out = C.cpu().numpy()
         assert np.isnan(out[:, N:]).all()
-        gu.assert_close_rel_absref(out[:, :N], c_ref, absref, rtol, "hbwn path %d" % path)
-    assert ran >= (4 if abf16 and K % 8 == 0 else 3)
+        two = wsp is not None and path in (hb.PATH_AUTO, hb.PATH_FOLDED)
+        gu.assert_close_rel_absref(out[:, :N], c_ref, absref, rtol2 if two else rtol, "hbwn path %d" % path)
+    assert ran >= (4 if abf16 and K % 8 == 0 else 2)
 
 
 def test_hbwn_tensor_path_needs_its_workspace(hb):
@@ -365,7 +371,7 @@ def test_conv_im2col_matches_oracle(hb, B, C, H, W, N, kh, kw, st, pd, ba, bw, s
     floor = None
     if ba == 1:
         c_ref, absref = oracle.hbwn_from_quantized(a_rows, dw, sw, gu.eff_beta(bw, K))
-        rtol = _hbwn_rtol(gu, K, bw)
+        rtol = _hbwn_rtol(gu, K, bw, True)
     else:
         da, sa = oracle.quantize(a_rows, gu.eff_beta(ba, K))
         c_ref, absref = oracle.hbmm_from_quantized(da, sa, gu.eff_beta(ba, K), dw, sw, gu.eff_beta(bw, K))
@@ -444,6 +450,11 @@ def test_prepared_weights_path_repeats_the_tensor_path_bit_for_bit(hb):
     assert torch.equal(C1, C2)
     c_ref, absref = oracle.hbwn_from_quantized(ab, dw, sw, 64)
     gu.assert_close_rel_absref(C2.cpu().numpy(), c_ref, absref, _hbwn_rtol(gu, K, 64))
+    hb.gemm_ex(Ad, W, C1, hb.PATH_FOLDED, wsd)
+    C2.fill_(float("nan"))
+    hb.gemm_ex(Ad, W, C2, hb.PATH_FOLDED_PREPARED, wsd)
+    assert torch.equal(C1, C2)
+    gu.assert_close_rel_absref(C2.cpu().numpy(), c_ref, absref, _hbwn_rtol(gu, K, 64, True))
 
 
 @pytest.mark.parametrize("spread", [0, 8, 16])
