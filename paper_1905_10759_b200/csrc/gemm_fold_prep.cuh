@@ -181,11 +181,11 @@ __device__ __forceinline__ void expand_weight_word(unsigned char* p1, unsigned c
   }
 }
 
-// Expands kPrepStages consecutive stages of one column tile of the weight operand into the stage layout
+// Expands kPrepStages consecutive stages (short tasks: many of them run side by side) of one column tile of the weight operand into the stage layout
 // the main kernel streams: rows 0 .. TN-1 piece 1, rows TN .. 2TN-1 piece 2, exactly as they sit in
 // shared memory.  The task of the first stages also stores the rows' inverse powers of two.
 // p = row of the tile, one thread per row (it scans its row's scales once per task).
-constexpr int kPrepStages = 8;
+constexpr int kPrepStages = 2;
 template <int TN>
 __device__ __forceinline__ void prepare_w_task(const Args& g, unsigned char* __restrict__ out, float* __restrict__ w_down,
                                                int64_t chunk, int64_t tile_n, int p) {
