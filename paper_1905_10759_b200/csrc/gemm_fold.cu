@@ -31,6 +31,7 @@
 #include "kernels.h"
 #include "umma_common.cuh"
 #include "gemm_fold_prep.cuh"
+#include "pdl.cuh"
 
 namespace hbmm {
 namespace {
@@ -91,6 +92,7 @@ hbmm_fold_kernel(const Args g) {
   const int64_t n_stages = (g.n_words + WPS - 1) / WPS;      // per tile
   const int64_t my_tiles = blockIdx.x < n_tiles ? (n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
 
+  pdl_launch_dependents();      // the next kernel of the stream may start its own set-up
   if (tid == 0) {
     for (int s = 0; s < STAGES; s++) {
       mbar_init(&full[s], kProducerWarps / 2 + 1);  // the four producer warps of the stage + the loader's expect_tx arrival
@@ -106,6 +108,7 @@ hbmm_fold_kernel(const Args g) {
     tmem_alloc(tmem_base_ptr, S::TMEM_COLS);
     tmem_relinquish();
   }
+  pdl_wait();                   // everything before this line touched no global memory
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -409,8 +412,7 @@ cudaError_t launch_fold(Args g, void* workspace, cudaStream_t stream, bool w_pre
   g.w_down = down;
   const int64_t tiles = ((g.M + TM - 1) / TM) * tiles_n;
   const unsigned grid = static_cast<unsigned>(tiles < sms ? tiles : sms);   // one persistent CTA per SM
-  hbmm_fold_kernel<TN, ASUB><<<grid, kThreads, S::BYTES, stream>>>(g);
-  return cudaGetLastError();
+  return launch_pdl(hbmm_fold_kernel<TN, ASUB>, dim3(grid), dim3(kThreads), S::BYTES, stream, g);
 }
 
 template <int TN>

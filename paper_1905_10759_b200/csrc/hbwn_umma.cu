@@ -26,6 +26,7 @@
 #include "tensor_map.h"
 #include "nhwc.cuh"
 #include "umma_common.cuh"
+#include "pdl.cuh"
 
 namespace hbmm {
 namespace {
@@ -151,6 +152,8 @@ __global__ void __launch_bounds__(256)
 nhwc_and_pieces_kernel(const CopyArgs c, const Args g, unsigned char* __restrict__ w_out) {
   __shared__ unsigned short tile[kNhwcCB][kNhwcPitch];
   const int64_t blk = blockIdx.x;
+  pdl_launch_dependents();
+  pdl_wait();                   // the workspace may still be in use by the kernel before this one
   if (blk < c.n_copy) {
     const int64_t per_image = static_cast<int64_t>(c.gx) * c.gy;
     const int64_t b = blk / per_image, r = blk - b * per_image;
@@ -187,6 +190,7 @@ hbwn_umma_kernel(const Args g, const __grid_constant__ CUtensorMap a_map) {
   const int64_t n_kb = g.n_kb;                              // stages per tile
   const int64_t my_tiles = blockIdx.x < n_tiles ? (n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
 
+  pdl_launch_dependents();      // the next kernel of the stream may start its own set-up
   if (tid == 0) {
     for (int s = 0; s < STAGES; s++) {
       mbar_init(&full[s], 1);           // the loader's expect_tx arrival; the copies complete the bytes
@@ -202,6 +206,7 @@ hbwn_umma_kernel(const Args g, const __grid_constant__ CUtensorMap a_map) {
     tmem_alloc(tmem_base_ptr, S::TMEM_COLS);
     tmem_relinquish();
   }
+  pdl_wait();                   // everything before this line touched no global memory
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -432,7 +437,9 @@ cudaError_t launch(Args g, const CUtensorMap& a_map, void* workspace, cudaStream
   if (copy) {
     const int64_t blocks = copy->n_copy + n_kb * tiles_n;
     if (blocks > 0x7fffffff) return cudaErrorNotSupported;
-    nhwc_and_pieces_kernel<TN, NP><<<static_cast<unsigned>(blocks), 256, 0, stream>>>(*copy, g, static_cast<unsigned char*>(workspace));
+    const cudaError_t e = launch_pdl(nhwc_and_pieces_kernel<TN, NP>, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, stream, *copy, g,
+                                     static_cast<unsigned char*>(workspace));
+    if (e != cudaSuccess) return e;
   } else if (!w_prepared) {
     prepare_w_pieces_kernel<TN, NP><<<pgrid, 256, 0, stream>>>(g, static_cast<unsigned char*>(workspace));
   }
@@ -441,10 +448,8 @@ cudaError_t launch(Args g, const CUtensorMap& a_map, void* workspace, cudaStream
   const unsigned grid = static_cast<unsigned>(tiles < sms ? tiles : sms);
   // a single column tile whose pieces fit beside the activation ring stays resident in shared memory
   if (tiles_n == 1 && n_kb * S::B_STAGE <= S::RES_MAX_B && tiles > sms)
-    hbwn_umma_kernel<TN, NP, true><<<grid, kThreads, kResBytes, stream>>>(g, a_map);
-  else
-    hbwn_umma_kernel<TN, NP, false><<<grid, kThreads, S::BYTES, stream>>>(g, a_map);
-  return cudaGetLastError();
+    return launch_pdl(hbwn_umma_kernel<TN, NP, true>, dim3(grid), dim3(kThreads), kResBytes, stream, g, a_map);
+  return launch_pdl(hbwn_umma_kernel<TN, NP, false>, dim3(grid), dim3(kThreads), S::BYTES, stream, g, a_map);
 }
 
 // exact: three pieces, 64-column tiles.  Otherwise two pieces: 128-column tiles when there are more than 64 columns.

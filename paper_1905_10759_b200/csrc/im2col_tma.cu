@@ -14,6 +14,7 @@
 #include "im2col_gather.cuh"
 #include "gemm_umma_prep.cuh"
 #include "gemm_fold_prep.cuh"
+#include "pdl.cuh"
 
 namespace hbmm {
 namespace {
@@ -67,9 +68,11 @@ im2col_quantize_tma_kernel(const __grid_constant__ CUtensorMap x_map, const floa
                            const __grid_constant__ UmmaPrepJob prep, int n_prep, int n_items, int ring,
                            uint32_t* __restrict__ bits, int64_t ld_words, void* __restrict__ scales, int64_t ld_scales,
                            int scale_bf16) {
+  pdl_launch_dependents();      // the next kernel of the stream may start its own set-up
   // The first n_prep CTAs expand the weight operand of the contraction that follows (one task each:
   // a stage of one column tile, one thread per weight row); they are scheduled first and leave at once.
   if (static_cast<int>(blockIdx.x) < n_prep) {
+    pdl_wait();                 // the workspace may still be read by the kernel before this one
     const int st = blockIdx.x % prep.n_stages, tile_n = blockIdx.x / prep.n_stages;
     if (prep.folded) {
       if (prep.tn == 64) { if (threadIdx.x < 64) fold::prepare_w_task<64>(prep.f, prep.out, prep.out_down, st, tile_n, threadIdx.x); }
@@ -130,6 +133,7 @@ im2col_quantize_tma_kernel(const __grid_constant__ CUtensorMap x_map, const floa
       pixmask[pix] = static_cast<unsigned short>(m);
     }
   }
+  pdl_wait();                   // the tables above live in shared memory; global memory is touched from here on
   __syncthreads();
 
   if (warp == kLoaderWarp) {
@@ -399,10 +403,8 @@ cudaError_t launch_im2col_quantize_tma(const void* x, const ConvGeom& g, uint32_
     n_prep = job.n_stages * job.tiles_n;
     if (n_prep > 4096) return cudaErrorNotSupported;       // the caller expands large weight operands on its own
   }
-  im2col_quantize_tma_kernel<<<grid + n_prep, kThreadsTma, smem, stream>>>(map, static_cast<const float*>(x), g, p, job, n_prep,
-                                                                           static_cast<int>(n_items), p.ring, bits, ld_words,
-                                                                           scales, ld_scales, scale_bf16);
-  return cudaGetLastError();
+  return launch_pdl(im2col_quantize_tma_kernel, dim3(grid + n_prep), dim3(kThreadsTma), smem, stream, map, static_cast<const float*>(x), g, p,
+                    job, n_prep, static_cast<int>(n_items), p.ring, bits, ld_words, scales, ld_scales, scale_bf16);
 }
 
 cudaError_t read_im2col_tma_error(int* code) {
