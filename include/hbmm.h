@@ -201,6 +201,22 @@ hbmm_status hbmm_conv_im2col(const void *x, int32_t x_dtype, const hbmm_conv_geo
                              void *stream);
 
 /*
+ * hbmm_conv_im2col with flags.  HBMM_CONV_WEIGHTS_PREPARED: the caller states that the part of `workspace`
+ * that holds the expanded weight operand (the tile layout the tensor-core contraction streams; Section 4.2:
+ * weights are fixed at inference time) was filled by an earlier hbmm_conv_im2col / hbmm_conv_im2col_ex
+ * call with the same W, geometry, beta_a, scale type and workspace, and that nothing has written it since.
+ * The call then skips the expansion; the activation part of the workspace is rewritten by every call
+ * either way.  Results are undefined when the statement is false.  Paths that keep no expanded weights
+ * ignore the flag.  Unknown flag bits: HBMM_ERR_INVALID_ARG.  Everything else as hbmm_conv_im2col
+ * (which is this call with flags = 0).
+ */
+#define HBMM_CONV_WEIGHTS_PREPARED 1u
+hbmm_status hbmm_conv_im2col_ex(const void *x, int32_t x_dtype, const hbmm_conv_geom *g,
+                                int32_t beta_a, int32_t a_scale_dtype, const hbmm_operand *W,
+                                float *C_out, int64_t ldc, void *workspace, size_t workspace_bytes,
+                                uint32_t flags, void *stream);
+
+/*
  * hbmm_conv_im2col for callers that cannot allocate device memory.  (No counterpart in the
  * paper: this is a deployment convenience, not part of the method.)
  *

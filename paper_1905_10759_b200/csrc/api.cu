@@ -316,6 +316,15 @@ hbmm_status hbmm_conv_workspace_bytes(const hbmm_conv_geom* g, int32_t beta_a, i
 hbmm_status hbmm_conv_im2col(const void* x, int32_t x_dtype, const hbmm_conv_geom* g, int32_t beta_a,
                              int32_t a_scale_dtype, const hbmm_operand* W, float* C_out, int64_t ldc,
                              void* workspace, size_t workspace_bytes, void* stream) {
+  return hbmm_conv_im2col_ex(x, x_dtype, g, beta_a, a_scale_dtype, W, C_out, ldc, workspace, workspace_bytes, 0u, stream);
+}
+
+hbmm_status hbmm_conv_im2col_ex(const void* x, int32_t x_dtype, const hbmm_conv_geom* g, int32_t beta_a,
+                                int32_t a_scale_dtype, const hbmm_operand* W, float* C_out, int64_t ldc,
+                                void* workspace, size_t workspace_bytes, uint32_t flags, void* stream) {
+  if (flags & ~static_cast<uint32_t>(HBMM_CONV_WEIGHTS_PREPARED)) return HBMM_ERR_INVALID_ARG;
+  // honoured on the two tensor-copy paths below; every other path expands the weights again (still correct)
+  const bool w_prepared = (flags & HBMM_CONV_WEIGHTS_PREPARED) != 0;
   ConvGeom cg;
   hbmm_status st = check_geom(g, &cg);
   if (st != HBMM_OK) return st;
@@ -332,7 +341,7 @@ hbmm_status hbmm_conv_im2col(const void* x, int32_t x_dtype, const hbmm_conv_geo
   A.rows = L.M; A.K = L.K; A.beta = beta_a; A.scale_dtype = a_scale_dtype;
   if (beta_a == 1 && L.implicit) {
     return launch_hbwn_umma_conv(x, x_dtype == HBMM_BF16, workspace, L.Cp, cg, view_of(W), C_out, ldc,
-                                 static_cast<char*>(workspace) + L.operand_bytes, s) == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
+                                 static_cast<char*>(workspace) + L.operand_bytes, s, w_prepared) == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
   }
   if (beta_a == 1) {
     if (launch_im2col_bf16(x, x_dtype == HBMM_BF16, cg, workspace, L.ld_dense, s) != cudaSuccess) return HBMM_ERR_CUDA;
@@ -352,8 +361,8 @@ hbmm_status hbmm_conv_im2col(const void* x, int32_t x_dtype, const hbmm_conv_geo
       UmmaPrepJob job{};
       gemm_fold_prep_job(av, wv, gemm_ws, &job);
       if (job.n_stages * job.tiles_n <= 4096) {
-        if (launch_im2col_quantize_tma(x, cg, A.bits, A.ld_words, A.scales, A.ld_scales, a_scale_dtype == HBMM_BF16, s, &job) !=
-            cudaSuccess)
+        if (launch_im2col_quantize_tma(x, cg, A.bits, A.ld_words, A.scales, A.ld_scales, a_scale_dtype == HBMM_BF16, s,
+                                       w_prepared ? nullptr : &job) != cudaSuccess)
           return HBMM_ERR_CUDA;
         return launch_gemm_fold(av, wv, C_out, ldc, gemm_ws, s, true) == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
       }

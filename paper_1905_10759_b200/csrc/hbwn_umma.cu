@@ -435,7 +435,7 @@ cudaError_t launch(Args g, const CUtensorMap& a_map, void* workspace, cudaStream
   const int64_t tiles_n = (g.N + TN - 1) / TN, n_kb = g.n_kb;
   dim3 pgrid(static_cast<unsigned>(n_kb), static_cast<unsigned>(tiles_n));
   if (copy) {
-    const int64_t blocks = copy->n_copy + n_kb * tiles_n;
+    const int64_t blocks = copy->n_copy + (w_prepared ? 0 : n_kb * tiles_n);     // prepared weights: the copy blocks only
     if (blocks > 0x7fffffff) return cudaErrorNotSupported;
     const cudaError_t e = launch_pdl(nhwc_and_pieces_kernel<TN, NP>, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, stream, *copy, g,
                                      static_cast<unsigned char*>(workspace));
@@ -501,7 +501,7 @@ size_t hbwn_umma_conv_workspace_bytes(const ConvGeom& c, const PackedView& W) {
 }
 
 cudaError_t launch_hbwn_umma_conv(const void* x, int x_bf16, void* x_nhwc, int Cp, const ConvGeom& c, const PackedView& W, float* C,
-                                  int64_t ldc, void* workspace, cudaStream_t stream) {
+                                  int64_t ldc, void* workspace, cudaStream_t stream, bool w_prepared) {
   const Args g = make_conv_args(c, W, C, ldc);
   CUtensorMap a_map;
   if (!make_conv_map(x_nhwc, c, Cp, &a_map)) return cudaErrorNotSupported;
@@ -511,7 +511,7 @@ cudaError_t launch_hbwn_umma_conv(const void* x, int x_bf16, void* x_nhwc, int C
   cp.gx = static_cast<int32_t>((cp.HW + kNhwcPB - 1) / kNhwcPB);
   cp.gy = (Cp + kNhwcCB - 1) / kNhwcCB;
   cp.n_copy = static_cast<int64_t>(cp.gx) * cp.gy * c.B;
-  return launch_any(g, a_map, workspace, stream, &cp, false, false);
+  return launch_any(g, a_map, workspace, stream, &cp, w_prepared, false);
 }
 
 cudaError_t read_hbwn_umma_error(int* code) {

@@ -133,8 +133,9 @@ cudaError_t launch_hbwn_umma(const DenseView& A, const PackedView& W, float* C, 
 cudaError_t launch_nchw_to_nhwc_bf16(const void* x, int x_bf16, const ConvGeom& g, void* out, int Cp, cudaStream_t stream);
 bool hbwn_umma_conv_supported(const ConvGeom& g, const PackedView& W);
 size_t hbwn_umma_conv_workspace_bytes(const ConvGeom& g, const PackedView& W);
+// w_prepared: the workspace still holds the weight pieces an earlier call with the same W and geometry laid out.
 cudaError_t launch_hbwn_umma_conv(const void* x, int x_bf16, void* x_nhwc, int Cp, const ConvGeom& g, const PackedView& W, float* C,
-                                  int64_t ldc, void* workspace, cudaStream_t stream);
+                                  int64_t ldc, void* workspace, cudaStream_t stream, bool w_prepared = false);
 
 // im2col gather fused with Hadamard binarization (packed output), and bf16 dense gather.
 cudaError_t launch_im2col_quantize(const void* x, int x_bf16, const ConvGeom& g, int32_t beta,

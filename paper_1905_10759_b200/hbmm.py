@@ -31,7 +31,7 @@ PATH_AUTO, PATH_POPC, PATH_B1MMA, PATH_TENSOR, PATH_TENSOR_PREPARED, PATH_FOLDED
 EXPORTS = [
     "hbmm_operand_bytes", "hbmm_quantize", "hbmm_gemm_workspace_bytes", "hbmm_gemm", "hbmm_gemm_ex",
     "hbmm_gemm_partials", "hbmm_conv_workspace_bytes", "hbmm_conv_im2col", "hbmm_status_string",
-    "hbmm_version", "hbmm_conv_im2col_static", "hbmm_last_device_error",
+    "hbmm_version", "hbmm_conv_im2col_static", "hbmm_last_device_error", "hbmm_conv_im2col_ex",
 ]
 STATIC_SCRATCH_BYTES = 32 << 20
 
@@ -63,6 +63,9 @@ _lib.hbmm_gemm_partials.argtypes = [_P(hbmm_operand), _P(hbmm_operand), _vp, _i3
 _lib.hbmm_conv_workspace_bytes.argtypes = [_P(hbmm_conv_geom), _i32, _i32, _P(hbmm_operand), _P(_sz)]
 _lib.hbmm_conv_im2col.argtypes = [_vp, _i32, _P(hbmm_conv_geom), _i32, _i32, _P(hbmm_operand), _vp, _i64,
                                   _vp, _sz, _vp]
+_lib.hbmm_conv_im2col_ex.argtypes = [_vp, _i32, _P(hbmm_conv_geom), _i32, _i32, _P(hbmm_operand), _vp, _i64,
+                                     _vp, _sz, ctypes.c_uint32, _vp]
+_lib.hbmm_conv_im2col_ex.restype = _i32
 _lib.hbmm_conv_im2col_static.argtypes = [_vp, _i32, _P(hbmm_conv_geom), _i32, _i32, _P(hbmm_operand), _vp, _i64, _vp]
 _lib.hbmm_conv_im2col_static.restype = _i32
 _lib.hbmm_last_device_error.argtypes = [_P(_i32)]
@@ -219,11 +222,20 @@ def conv_workspace_bytes(geom: hbmm_conv_geom, beta_a: int, a_scale_dtype: int, 
     return n.value
 
 
+CONV_WEIGHTS_PREPARED = 1
+
+
 def conv_im2col(x: torch.Tensor, geom: hbmm_conv_geom, beta_a: int, a_scale_dtype: int, W: Operand,
-                C_out: torch.Tensor, workspace: torch.Tensor, stream=None):
-    """hbmm_conv_im2col: x NCHW contiguous; C_out fp32 [B*Ho*Wo, N]."""
+                C_out: torch.Tensor, workspace: torch.Tensor, stream=None, flags: int = 0):
+    """hbmm_conv_im2col (flags == 0) / hbmm_conv_im2col_ex: x NCHW contiguous; C_out fp32 [B*Ho*Wo, N]."""
     if not x.is_contiguous():
         raise ValueError("x must be a contiguous NCHW tensor")
+    if flags:
+        _check(_lib.hbmm_conv_im2col_ex(_dev_ptr(x), _dtype_code(x.dtype), ctypes.byref(geom), beta_a, a_scale_dtype,
+                                        ctypes.byref(W.desc), _dev_ptr(C_out), C_out.stride(0), _dev_ptr(workspace),
+                                        workspace.numel() * workspace.element_size(), flags, _stream(stream)),
+               "hbmm_conv_im2col_ex")
+        return C_out
     _check(_lib.hbmm_conv_im2col(_dev_ptr(x), _dtype_code(x.dtype), ctypes.byref(geom), beta_a, a_scale_dtype,
                                  ctypes.byref(W.desc), _dev_ptr(C_out), C_out.stride(0), _dev_ptr(workspace),
                                  workspace.numel() * workspace.element_size(), _stream(stream)), "hbmm_conv_im2col")

@@ -138,3 +138,4 @@ def test_host_validation_rejects_before_launch(hb):
     bad = hb.make_geom(2, 4, 2, 2, 5, 5, (1, 1), (0, 0))
     assert call(bad, Wc, ws, n.value) == hb.ERR_INVALID_ARG                           # filter larger than image
     assert call(g, Wc, ws, n.value, beta_a=12) == hb.ERR_UNSUPPORTED
+    assert lib.hbmm_conv_im2col_ex(x, 0, ctypes.byref(g), 36, 0, ctypes.byref(Wc.desc), c, 4, ws, n.value, 2, None) == hb.ERR_INVALID_ARG  # unknown flag

@@ -492,3 +492,29 @@ def test_folded_path_keeps_the_tolerance_when_group_scales_differ_by_orders_of_m
         for cols in (cols_n, np.array([2]), np.array([9])):
             ix = np.ix_(rows, cols)
             gu.assert_close_rel_absref(out[ix], c_ref[ix], absref[ix], RTOL, "folded, spread 2^%d" % spread, floor[ix])
+
+
+@pytest.mark.parametrize("beta_a,xbf16,C,H", [(32, False, 64, 12), (1, True, 64, 8), (32, False, 96, 7), (16, False, 32, 6)])
+def test_conv_with_prepared_weights_repeats_the_plain_call_bit_for_bit(hb, beta_a, xbf16, C, H):
+    """HBMM_CONV_WEIGHTS_PREPARED skips the weight expansion and reuses what an earlier call left in the
+    workspace; a second batch through the same workspace must give exactly what the plain call gives."""
+    shape = inputs.ConvShape("t", 3, C, H, H, 72, 3, 3, 1, 1)
+    K = C * 9
+    w = inputs.he_normal(72, K, 511)
+    Wop = hb.quantize(torch.from_numpy(w).cuda(), hb.alloc_operand(72, K, 32))
+    geom = hb.make_geom(3, C, H, H, 3, 3, (1, 1), (1, 1))
+    ws = torch.empty(hb.conv_workspace_bytes(geom, beta_a, hb.F32, Wop), dtype=torch.uint8, device="cuda")
+    ws2 = torch.empty_like(ws)
+    outs = []
+    for seed in (512, 513):
+        x = torch.from_numpy(inputs.conv_activation(shape, seed, signed=True)).cuda()
+        if xbf16:
+            x = x.to(torch.bfloat16)
+        plain = torch.full((shape.M, 72), float("nan"), device="cuda")
+        hb.conv_im2col(x, geom, beta_a, hb.F32, Wop, plain, ws2)
+        fast = torch.full((shape.M, 72), float("nan"), device="cuda")
+        # first batch fills the workspace, every later one states that the weights are still there
+        hb.conv_im2col(x, geom, beta_a, hb.F32, Wop, fast, ws, flags=hb.CONV_WEIGHTS_PREPARED if outs else 0)
+        assert torch.equal(plain, fast)
+        outs.append(fast)
+    assert not torch.equal(outs[0], outs[1])
