@@ -135,3 +135,31 @@ def test_alexnet_fc_stack(hb, batch):
         c_ref, absref = oracle.hbmm_from_quantized(da[rows], sa[rows], beta, dw, sw, beta)
         gu.assert_close_rel_absref(C[torch.from_numpy(rows).cuda()].cpu().numpy()[:, :N], c_ref, absref, RTOL,
                                    "fc %dx%d batch %d" % (K, N, batch))
+
+
+@pytest.mark.parametrize("ba,bw", [(16, 16), (4, 4), (2, 16)])
+def test_subword_groups_on_the_conv3_matrix_sampled_rows(hb, ba, bw):
+    """The paper's own group sizes (Section 5: beta_a / beta_w = 2 .. 16, mixed) at a benchmark shape
+    (M = 50176, N = 128, K = 1152), through hbmm_quantize and the automatic contraction path."""
+    gu = _gu()
+    M, N, K = 50176, 128, 1152
+    a = inputs.normal((M, K), inputs.SEEDS["resnet_hbmm"][0] + 40 + ba)
+    w = inputs.he_normal(N, K, inputs.SEEDS["resnet_hbmm"][1] + 40 + bw)
+    A = hb.quantize(torch.from_numpy(a).cuda(), hb.alloc_operand(M, K, ba, hb.F32))
+    W = hb.quantize(torch.from_numpy(w).cuda(), hb.alloc_operand(N, K, bw, hb.F32))
+    C = torch.empty((M, N), device="cuda")
+    ws = torch.empty(max(hb.gemm_workspace_bytes(A, W), 16), dtype=torch.uint8, device="cuda")
+    hb.gemm(A, W, C, ws)
+    torch.cuda.synchronize()
+    rows = _sample_rows(M, 48, M + ba)
+    rows_d = torch.from_numpy(rows).cuda()
+    da, sa = oracle.quantize(a[rows], ba)
+    dw, sw = oracle.quantize(w, bw)
+    assert np.array_equal(gu.host_bits(A.bits[rows_d]), oracle.pack(sa, A.bits.shape[1]))
+    # products from the scales the GPU stored (they are checked against the oracle's to their own bound)
+    sa_gpu = A.scales[rows_d][:, : K // ba].float().cpu().numpy().astype(np.float64)
+    sw_gpu = W.scales[:, : K // bw].float().cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(sa_gpu - da) <= 8 * gu.U * da + 1e-30) and np.all(np.abs(sw_gpu - dw) <= 8 * gu.U * dw + 1e-30)
+    c_ref, absref = oracle.hbmm_from_quantized(sa_gpu, sa, ba, sw_gpu, sw, bw)
+    floor = gu.FOLDED_FLOOR_ULPS * gu.U * gu.elementwise_magnitude(sa_gpu, ba, sw_gpu, bw, K)
+    gu.assert_close_rel_absref(C[rows_d].cpu().numpy(), c_ref, absref, RTOL, "conv3 matrix beta %d/%d" % (ba, bw), floor)
