@@ -86,6 +86,18 @@ def quantize(x: np.ndarray, beta: int) -> Tuple[np.ndarray, np.ndarray]:
     return delta, sign
 
 
+def binarize_backward(x: np.ndarray, gy: np.ndarray, beta: int) -> np.ndarray:
+    """dC/dX from dC/dX~ for X~ = delta (.) Sign(X) (Eq. 6 with the straight-through estimator of Eq. 5):
+    float64 [rows, K]."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    gy = np.ascontiguousarray(gy, dtype=np.float32)
+    assert x.shape == gy.shape
+    rows, K = x.shape
+    gx = np.empty((rows, K), dtype=np.float64)
+    _L().oracle_binarize_backward(_ptr(x), _ptr(gy), _i64(rows), _i64(K), _i64(K), _i64(K), _i64(beta), _ptr(gx))
+    return gx
+
+
 def round_scales(delta: np.ndarray, scale_dtype: Optional[str]) -> np.ndarray:
     """Value of the scale tensor after storage: None = exact, 'f32', or 'bf16' (RNE of the fp32 value)."""
     out = np.array(delta, dtype=np.float64, order="C", copy=True)

@@ -65,6 +65,43 @@ void oracle_quantize(const float *x, int64_t rows, int64_t K, int64_t ldx, int64
     }
 }
 
+/*
+ * Gradient through the Hadamard binarization X~ = delta (.) Sign(X) (Section 3.1.3, Eq. 6, with the
+ * straight-through estimator of Eq. 5 for dSign/dx).  gy = dC/dX~ (incoming), gx = dC/dX (result).
+ * For element i of group g (n_g elements, s = Sign(x)):
+ *   gx[i] = (1/n_g) * s_i * sum_{j in g} gy[j] * s_j        (delta depends on every |x_j| of the group)
+ *         + delta_g * gy[i] * [ |x_i| <= 1 ]                 (Eq. 5: the estimator passes |x| <= 1)
+ * Readings: the printed sum runs j = beta*floor(i/beta) .. beta*(floor(i/beta)+1), one index too many,
+ * as in Eq. 1 / Eq. 3: it is taken over the beta elements of the group; a tail group uses its own
+ * length, as in oracle_quantize; the paper's "delta_{l,i}, the absolute value of the binarized weight"
+ * is the group scale.  Taken in the paper's order: first the group sum, then the two terms.
+ */
+void oracle_binarize_backward(const float *x, const float *gy, int64_t rows, int64_t K, int64_t ldx,
+                              int64_t ldg, int64_t beta, double *gx)
+{
+    int64_t G = n_groups(K, beta);
+    #pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; r++) {
+        for (int64_t g = 0; g < G; g++) {
+            int64_t k0 = g * beta, k1 = k0 + beta;
+            if (k1 > K) k1 = K;
+            double n = (double)(k1 - k0), abs_sum = 0.0, gs = 0.0;
+            for (int64_t k = k0; k < k1; k++) {
+                double v = (double)x[r * ldx + k];
+                abs_sum += fabs(v);
+                gs += (double)gy[r * ldg + k] * (v >= 0.0 ? 1.0 : -1.0);
+            }
+            double delta = abs_sum / n;
+            for (int64_t k = k0; k < k1; k++) {
+                double v = (double)x[r * ldx + k];
+                double sgn = v >= 0.0 ? 1.0 : -1.0;
+                double ste = fabs(v) <= 1.0 ? 1.0 : 0.0;
+                gx[r * K + k] = sgn * gs / n + delta * (double)gy[r * ldg + k] * ste;
+            }
+        }
+    }
+}
+
 /* Storage rounding of the "full precision" scale tensor: fp32 (the paper's 32-bit
  * full precision, Section 4.1) -- value after round-to-nearest-even to float. */
 void oracle_round_f32(double *v, int64_t n)

@@ -315,3 +315,72 @@ def test_conv_hbmm_binarizes_im2col_rows_along_k():
     cols = torch.nn.functional.unfold(torch.from_numpy(x), 3, padding=1).permute(0, 2, 1).reshape(-1, 36).numpy()
     ref = _np_hadamard(cols, 4) @ _np_hadamard(w2d, 12).T
     np.testing.assert_allclose(c, ref, rtol=0, atol=1e-12)
+
+
+# ---------------------------------------------------------------- gradient through the binarization (Eq. 5, Eq. 6)
+def _hadamard_objective(x64, gy64, beta):
+    """sum(gy * (delta (.) Sign(x))) in exact rational arithmetic is overkill here: float64 with values that
+    are small dyadic rationals keeps every step exact."""
+    rows, K = x64.shape
+    total = 0.0
+    for r in range(rows):
+        for k0 in range(0, K, beta):
+            seg = x64[r, k0:k0 + beta]
+            d = np.abs(seg).sum() / len(seg)
+            total += float((gy64[r, k0:k0 + beta] * d * np.where(seg >= 0, 1.0, -1.0)).sum())
+    return total
+
+
+def test_binarize_backward_hand_example():
+    """x = (0.5, -2), gy = (1, 3), beta = 2: s = (+1, -1), delta = 1.25, sum gy*s = -2.
+    First term (1/2) s_i (-2) = (-1, +1); estimator term delta*gy_i*[|x_i| <= 1] = (1.25, 0)."""
+    gx = oracle.binarize_backward(np.array([[0.5, -2.0]], np.float32), np.array([[1.0, 3.0]], np.float32), 2)
+    assert np.array_equal(gx, np.array([[0.25, 1.0]]))
+
+
+@pytest.mark.parametrize("K,beta", [(12, 4), (10, 4), (9, 2), (16, 16), (7, 1), (5, 8)])
+def test_binarize_backward_first_term_is_the_exact_derivative_with_signs_held(K, beta):
+    """Away from |x| <= 1 the estimator term vanishes, and delta (.) Sign(x) is piecewise linear in x: a
+    finite difference that does not cross zero gives dC/dx exactly (dyadic inputs: no rounding at all).
+    Pins the group sum, its 1/n_g factor (tail group included), both sign factors and the row layout."""
+    rng = np.random.default_rng(700 + K + beta)
+    x = (rng.integers(9, 40, size=(3, K)) / 8.0 * rng.choice([-1.0, 1.0], size=(3, K))).astype(np.float32)   # 1.125 <= |x| < 5
+    gy = (rng.integers(-16, 17, size=(3, K)) / 4.0).astype(np.float32)
+    gx = oracle.binarize_backward(x, gy, beta)
+    x64, gy64 = x.astype(np.float64), gy.astype(np.float64)
+    f0 = _hadamard_objective(x64, gy64, beta)
+    h = 2.0 ** -6
+    for r in range(3):
+        for i in range(K):
+            xp = x64.copy()
+            xp[r, i] += h * (1.0 if xp[r, i] > 0 else -1.0)          # away from zero
+            fd = (_hadamard_objective(xp, gy64, beta) - f0) / h * (1.0 if x64[r, i] > 0 else -1.0)
+            assert abs(fd - gx[r, i]) < 1e-9, (r, i, fd, gx[r, i])
+
+
+def test_binarize_backward_estimator_term_and_its_threshold():
+    """Eq. 5: the straight-through term delta_g * gy_i is added exactly where |x_i| <= 1 (inclusive)."""
+    x = np.array([[1.0, -1.0, 1.0000001, -0.25, 0.0, 3.0, -1.5, 0.75]], np.float32)
+    gy = np.array([[2.0, -3.0, 5.0, 7.0, -1.0, 4.0, 0.5, 8.0]], np.float32)
+    beta = 4
+    gx = oracle.binarize_backward(x, gy, beta)
+    x64 = x.astype(np.float64)
+    s = np.where(x64 >= 0, 1.0, -1.0)                                  # Sign(0) = +1
+    for g in range(2):
+        sl = slice(4 * g, 4 * g + 4)
+        delta = np.abs(x64[0, sl]).mean()
+        first = s[0, sl] * (gy[0, sl].astype(np.float64) * s[0, sl]).sum() / 4.0
+        ste = gx[0, sl] - first
+        expect = np.where(np.abs(x64[0, sl]) <= 1.0, delta * gy[0, sl], 0.0)
+        np.testing.assert_allclose(ste, expect, rtol=0, atol=1e-12)
+    assert gx[0, 2] - (s[0, 2] * (gy[0, :4] * s[0, :4]).sum() / 4.0) == 0.0     # 1.0000001 > 1: no estimator term
+
+
+def test_binarize_backward_beta_one():
+    """beta = 1: delta = |x| and X~ = X, so Eq. 6 gives gy_i * (1 + |x_i| [|x_i| <= 1])."""
+    rng = np.random.default_rng(71)
+    x = rng.standard_normal((4, 9)).astype(np.float32)
+    gy = rng.standard_normal((4, 9)).astype(np.float32)
+    gx = oracle.binarize_backward(x, gy, 1)
+    x64, g64 = x.astype(np.float64), gy.astype(np.float64)
+    np.testing.assert_allclose(gx, g64 * (1.0 + np.abs(x64) * (np.abs(x64) <= 1.0)), rtol=0, atol=1e-15)
