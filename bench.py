@@ -273,7 +273,8 @@ def kernel_breakdown(torch, hbmm, layers, iters: int):
 def side_measurements(torch, hbmm, peaks, iters: int):
     """Rows of the hot path that the convolution step only runs in fused form, timed on their own on the
     conv3_x matrix view (M = 50176, K = 1152, N = 128; 231 MB of fp32 input, larger than L2):
-    hbmm_quantize alone (HBM bound), and the folded-scale contraction at the sub-word group sizes of the
+    hbmm_quantize alone (HBM bound), the gradient through the binarization (Eq. 6, HBM bound: 8 bytes read
+    and 4 written per element), and the folded-scale contraction at the sub-word group sizes of the
     paper's experiments.  Reported beside the step, not part of it."""
     hbm_gbs, bf16_tflops, _ = peaks
     M, N, K = 50176, 128, 1152
@@ -287,6 +288,13 @@ def side_measurements(torch, hbmm, peaks, iters: int):
         ms = time_loop(torch, lambda: hbmm.quantize(a, A), iters)
         by = 4.0 * M * K + A.bits.numel() * 4.0 + A.scales.numel() * 4.0
         out.append({"kernel": "hbmm_quantize/beta%d" % beta, "shape": [M, K], "ms": round(ms, 5), "bound": "hbm",
+                    "achieved": by / (ms * 1e-3) / 1e9, "peak": hbm_gbs, "unit": "GB/s", "frac": by / (ms * 1e-3) / 1e9 / hbm_gbs})
+    gy = torch.randn((M, K), device="cuda", generator=g)
+    gx = torch.empty_like(a)
+    for beta in (4, 32):
+        ms = time_loop(torch, lambda: hbmm.binarize_backward(a, gy, beta, gx), iters)
+        by = 12.0 * M * K
+        out.append({"kernel": "hbmm_binarize_backward/beta%d" % beta, "shape": [M, K], "ms": round(ms, 5), "bound": "hbm",
                     "achieved": by / (ms * 1e-3) / 1e9, "peak": hbm_gbs, "unit": "GB/s", "frac": by / (ms * 1e-3) / 1e9 / hbm_gbs})
     for ba, bw in ((16, 16), (4, 4), (2, 16)):
         A = hbmm.quantize(a, hbmm.alloc_operand(M, K, ba, hbmm.F32))

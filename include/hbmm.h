@@ -142,6 +142,22 @@ hbmm_status hbmm_operand_bytes(int64_t rows, int64_t K, int32_t beta, int32_t sc
 hbmm_status hbmm_quantize(const void *x, int32_t x_dtype, int64_t rows, int64_t K, int64_t ldx,
                           const hbmm_operand *out, void *stream);
 
+/*
+ * Training side: gradient through the Hadamard binarization X~ = delta (.) Sign(X) (Section 3.1.3).
+ * Given gy = dC/dX~ it returns gx = dC/dX by Eq. 6, with the straight-through estimator of Eq. 5 for the
+ * derivative of Sign:
+ *     gx[r,i] = (1/n_g) Sign(x_i) sum_{j in group(i)} gy[r,j] Sign(x_j)  +  delta_g gy[r,i] [|x_i| <= 1],
+ * group(i) the run of beta consecutive row elements that holds i (a tail group uses its own length n_g),
+ * delta_g its mean |x|, Sign(0) = +1.  beta >= 1 (any value; beta >= K: one group per row; beta = 1: X~ = X).
+ * x, gy, gx: device fp32 [rows, ld*], ld* >= K, 4-byte aligned (16-byte aligned unpadded rows take the
+ * streaming kernel).  gx may not alias x or gy.  The re-binarization of the weights that every training
+ * step needs (Algorithm 1) is hbmm_quantize.
+ * Errors: INVALID_ARG, ALIGNMENT, CUDA.
+ */
+hbmm_status hbmm_binarize_backward(const float *x, int64_t ldx, const float *gy, int64_t ldg,
+                                   int64_t rows, int64_t K, int32_t beta, float *gx, int64_t ldo,
+                                   void *stream);
+
 /* Bytes of scratch hbmm_gemm wants for these operands (host pointer `bytes`).  The tensor-core
  * contractions keep the weight operand there, expanded once per call into the tile layout their
  * kernels stream (HBMM: 4 K bytes per weight row, two fp16 pieces; HBWN: 6 K bytes per weight row,

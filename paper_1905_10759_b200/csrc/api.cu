@@ -258,6 +258,15 @@ hbmm_status hbmm_quantize(const void* x, int32_t x_dtype, int64_t rows, int64_t 
   return e == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
 }
 
+hbmm_status hbmm_binarize_backward(const float* x, int64_t ldx, const float* gy, int64_t ldg, int64_t rows, int64_t K,
+                                   int32_t beta, float* gx, int64_t ldo, void* stream) {
+  if (!x || !gy || !gx || rows <= 0 || K <= 0 || beta < 1 || ldx < K || ldg < K || ldo < K) return HBMM_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(x) % 4 != 0 || reinterpret_cast<uintptr_t>(gy) % 4 != 0 || reinterpret_cast<uintptr_t>(gx) % 4 != 0)
+    return HBMM_ERR_ALIGNMENT;
+  return launch_binarize_backward(x, ldx, gy, ldg, rows, K, beta, gx, ldo, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? HBMM_OK : HBMM_ERR_CUDA;
+}
+
 hbmm_status hbmm_gemm_workspace_bytes(const hbmm_operand* A, const hbmm_operand* W, size_t* bytes) {
   if (!A || !W || !bytes) return HBMM_ERR_INVALID_ARG;
   *bytes = 0;

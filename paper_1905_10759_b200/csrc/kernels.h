@@ -35,6 +35,10 @@ cudaError_t launch_quantize(const void* x, int x_bf16, int64_t rows, int64_t K, 
                             uint32_t* bits, int64_t ld_words, void* scales, int64_t ld_scales,
                             int scale_bf16, int32_t beta, cudaStream_t stream);
 
+// Gradient through the Hadamard binarization (Eq. 6 with the straight-through estimator of Eq. 5).
+cudaError_t launch_binarize_backward(const float* x, int64_t ldx, const float* gy, int64_t ldg, int64_t rows, int64_t K, int32_t beta,
+                                     float* gx, int64_t ldo, cudaStream_t stream);
+
 // Packed x packed contraction on the integer pipe (XOR + POPC).
 cudaError_t launch_gemm_popc(const PackedView& A, const PackedView& W, float* C, int64_t ldc,
                              cudaStream_t stream);

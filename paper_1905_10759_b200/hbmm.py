@@ -32,6 +32,7 @@ EXPORTS = [
     "hbmm_operand_bytes", "hbmm_quantize", "hbmm_gemm_workspace_bytes", "hbmm_gemm", "hbmm_gemm_ex",
     "hbmm_gemm_partials", "hbmm_conv_workspace_bytes", "hbmm_conv_im2col", "hbmm_status_string",
     "hbmm_version", "hbmm_conv_im2col_static", "hbmm_last_device_error", "hbmm_conv_im2col_ex",
+    "hbmm_binarize_backward",
 ]
 STATIC_SCRATCH_BYTES = 32 << 20
 
@@ -223,6 +224,22 @@ def conv_workspace_bytes(geom: hbmm_conv_geom, beta_a: int, a_scale_dtype: int, 
 
 
 CONV_WEIGHTS_PREPARED = 1
+
+_lib.hbmm_binarize_backward.argtypes = [_vp, _i64, _vp, _i64, _i64, _i64, _i32, _vp, _i64, _vp]
+_lib.hbmm_binarize_backward.restype = _i32
+
+
+def binarize_backward(x: torch.Tensor, gy: torch.Tensor, beta: int, gx: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """hbmm_binarize_backward: x, gy fp32 [rows, K] (row stride >= K, unit column stride); returns gx = dC/dX."""
+    if x.dtype != torch.float32 or gy.dtype != torch.float32 or x.shape != gy.shape or x.dim() != 2:
+        raise ValueError("x and gy must be fp32 matrices of one shape")
+    if x.stride(1) != 1 or gy.stride(1) != 1:
+        raise ValueError("rows must be contiguous")
+    if gx is None:
+        gx = torch.empty(x.shape, dtype=torch.float32, device=x.device)
+    _check(_lib.hbmm_binarize_backward(_dev_ptr(x), x.stride(0), _dev_ptr(gy), gy.stride(0), x.shape[0], x.shape[1], beta,
+                                       _dev_ptr(gx), gx.stride(0), _stream(stream)), "hbmm_binarize_backward")
+    return gx
 
 
 def conv_im2col(x: torch.Tensor, geom: hbmm_conv_geom, beta_a: int, a_scale_dtype: int, W: Operand,

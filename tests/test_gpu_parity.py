@@ -518,3 +518,41 @@ def test_conv_with_prepared_weights_repeats_the_plain_call_bit_for_bit(hb, beta_
         assert torch.equal(plain, fast)
         outs.append(fast)
     assert not torch.equal(outs[0], outs[1])
+
+
+# ------------------------------------------------------------------ gradient through the binarization (Eq. 5, Eq. 6)
+BACKWARD_CASES = [
+    # rows, K, beta, row padding of the inputs
+    (64, 576, 2, 0), (33, 1152, 4, 0), (20, 256, 8, 0), (17, 512, 16, 0), (130, 576, 32, 0), (9, 1024, 128, 0), (40, 100, 1, 0),
+    (7, 333, 4, 0),      # ragged K: tail group of one element -> general kernel
+    (12, 96, 96, 0),     # one group per row
+    (5, 45, 7, 3),       # odd everything, padded rows
+    (16, 128, 256, 0),   # beta > K
+]
+
+
+@pytest.mark.parametrize("rows,K,beta,pad", BACKWARD_CASES)
+def test_binarize_backward_matches_oracle(hb, rows, K, beta, pad):
+    gu = _gu()
+    x = inputs.normal((rows, K), 9100 + rows + K)
+    gy = inputs.normal((rows, K), 9200 + rows + beta)
+    x[0, :4] = [1.0, -1.0, 0.0, -0.0]                       # estimator threshold (inclusive) and Sign(+-0) = +1
+    ref = oracle.binarize_backward(x, gy, beta)
+    xd = torch.zeros((rows, K + pad)); xd[:, :K] = torch.from_numpy(x)
+    gd = torch.zeros((rows, K + pad)); gd[:, :K] = torch.from_numpy(gy)
+    out = torch.full((rows, K + pad), float("nan"), device="cuda")
+    hb.binarize_backward(xd.cuda()[:, :K], gd.cuda()[:, :K], beta, out[:, :K])
+    got = out.cpu().numpy()
+    assert np.isnan(got[:, K:]).all()
+    # both terms are fp32 trees over at most beta elements followed by one multiply and one add
+    be = gu.eff_beta(beta, K)
+    G = -(-K // be)
+    x64, g64 = x.astype(np.float64), gy.astype(np.float64)
+    mag = np.empty_like(x64)
+    for g in range(G):
+        sl = slice(g * be, min((g + 1) * be, K))
+        n = sl.stop - sl.start
+        mag[:, sl] = np.abs(g64[:, sl]).sum(axis=1, keepdims=True) / n + np.abs(x64[:, sl]).mean(axis=1, keepdims=True) * np.abs(g64[:, sl])
+    tol = (int(np.ceil(np.log2(max(be, 2)))) + int(np.ceil(be / 32)) + 4) * gu.U
+    err = np.abs(got[:, :K].astype(np.float64) - ref)
+    assert (err <= tol * mag + 1e-30).all(), float((err / (mag + 1e-30)).max() / gu.U)
