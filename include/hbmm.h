@@ -187,6 +187,25 @@ hbmm_status hbmm_gemm_ex(const hbmm_operand *A, const hbmm_operand *W, float *C,
                          void *workspace, size_t workspace_bytes, int32_t path, void *stream);
 
 /*
+ * Product fused with the next layer's binarization (the layer order of Section 5 is batch normalisation ->
+ * binarize -> product, so the consumer of C is a binarizer): inside the contraction's epilogue every output
+ * goes through a per-column affine map  z[m,n] = bn_scale[n] * C[m,n] + bn_shift[n]  (a batch normalisation
+ * folded to inference form; either pointer may be NULL: 1 and 0) and each row of z is Hadamard-binarized along
+ * n with group next->beta (Eq. 3-4).  Only the packed result is written: the fp32 product never reaches
+ * memory (4 bytes per output become 1 + 32/beta bits).  `next`: host descriptor of a packed operand with
+ * rows = A.rows, K = W.rows, buffers sized by hbmm_operand_bytes; filled like hbmm_quantize fills its output,
+ * zero padding included.  It is what a following fully connected layer or 1 x 1 convolution reads as its A.
+ * Runs on the folded-scale tensor-core kernel only: A and W packed with K a multiple of 32 and activation
+ * groups of whole words; next->beta one of 2, 4, 8, 16, 32, 64, 128, at most 64 when W has at most 64 rows,
+ * and smaller than W.rows; workspace as hbmm_gemm_workspace_bytes(A, W) reports.  bn_scale / bn_shift:
+ * device fp32 [W.rows].  Where z is within rounding of zero the sign follows the fp32 value the kernel
+ * computed.  Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, WORKSPACE, CUDA.
+ */
+hbmm_status hbmm_gemm_binarize_next(const hbmm_operand *A, const hbmm_operand *W, const float *bn_scale,
+                                    const float *bn_shift, const hbmm_operand *next, void *workspace,
+                                    size_t workspace_bytes, void *stream);
+
+/*
  * The integer term of Eq. 7 on its own: D[m,n,t] = signed +-1 dot product of K-segment t
  * (segment length min(beta_a, beta_w); T = ceil(K / segment) segments), int32, device
  * [M, N, T] contiguous.  Both operands packed.  Meant for checking the popcount path

@@ -289,6 +289,29 @@ hbmm_status hbmm_gemm_ex(const hbmm_operand* A, const hbmm_operand* W, float* C,
   return gemm_checked(A, W, C, ldc, path, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
 }
 
+hbmm_status hbmm_gemm_binarize_next(const hbmm_operand* A, const hbmm_operand* W, const float* bn_scale, const float* bn_shift,
+                                    const hbmm_operand* next, void* workspace, size_t workspace_bytes, void* stream) {
+  hbmm_status st;
+  if (!A || !W || !next) return HBMM_ERR_INVALID_ARG;
+  if (A->beta == 1 || W->beta == 1) return HBMM_ERR_UNSUPPORTED;       // both operands packed
+  if ((st = check_packed(A)) != HBMM_OK) return st;
+  if ((st = check_packed(W)) != HBMM_OK) return st;
+  if (A->K != W->K) return HBMM_ERR_INVALID_ARG;
+  if (next->rows != A->rows || next->K != W->rows) return HBMM_ERR_INVALID_ARG;
+  if ((st = check_packed(next)) != HBMM_OK) return st;
+  if ((bn_scale && reinterpret_cast<uintptr_t>(bn_scale) % 4 != 0) || (bn_shift && reinterpret_cast<uintptr_t>(bn_shift) % 4 != 0))
+    return HBMM_ERR_ALIGNMENT;
+  const PackedView a = view_of(A), w = view_of(W);
+  const bool a_subword = A->beta < 32 && A->beta < A->K;
+  if (!gemm_fold_supported(a, w) || a_subword || next->beta >= next->K || !gemm_fold_next_supported(W->rows, next->beta))
+    return HBMM_ERR_UNSUPPORTED;
+  if (!workspace_ok(workspace, workspace_bytes, fold_workspace(a, w))) return HBMM_ERR_WORKSPACE;
+  FoldNext nx;
+  nx.bn_scale = bn_scale; nx.bn_shift = bn_shift; nx.bits = next->bits; nx.scales = next->scales;
+  nx.ld_words = next->ld_words; nx.ld_scales = next->ld_scales; nx.scale_bf16 = next->scale_dtype == HBMM_BF16; nx.beta = next->beta;
+  return launch_gemm_fold(a, w, nullptr, 0, workspace, static_cast<cudaStream_t>(stream), false, &nx) == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
+}
+
 hbmm_status hbmm_gemm_partials(const hbmm_operand* A, const hbmm_operand* W, int32_t* D, int32_t path, void* stream) {
   hbmm_status st;
   if ((st = check_packed(A)) != HBMM_OK) return st;

@@ -27,6 +27,7 @@
 // A stage holds 64 K-elements (two packed words).  Stages and the two TMEM accumulators are mbarrier
 // rings.  Every wait is bounded: on expiry the thread records a code, raises a CTA-wide abort flag
 // that all other waits observe, and the kernel drains and frees its TMEM before returning.
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include "kernels.h"
 #include "umma_common.cuh"
@@ -56,6 +57,50 @@ prepare_w_fold_kernel(const Args g, unsigned char* __restrict__ out, float* __re
   prepare_w_task<TN>(g, out, w_down, blockIdx.x, blockIdx.y, threadIdx.x);
 }
 
+__device__ __forceinline__ void store_next_scale(void* s, int bf16, int64_t idx, float v) {
+  if (bf16) reinterpret_cast<__nv_bfloat16*>(s)[idx] = __float2bfloat16_rn(v);
+  else reinterpret_cast<float*>(s)[idx] = v;
+}
+
+// Fused epilogue: 32 consecutive columns of one row of z (columns n0 .. n0 + 31, `valid` of them inside the
+// output) become one packed word (bit e = 1 <=> z[e] >= 0, -0 counting as +0; bits of absent columns 0) and
+// the scales of the groups that end inside the chunk (mean |z| over the group's columns inside the output).
+// BETA > 32: the chunk's |z| sum is added to `carry`, and the group is closed by its last chunk.
+template <int BETA>
+__device__ __forceinline__ void emit_next_chunk(const float (&z)[32], int valid, int64_t n0, int64_t N, uint32_t* bits_row, void* scales,
+                                                int bf16, int64_t srow, int64_t ld_scales, float& carry) {
+  uint32_t neg = 0;
+#pragma unroll
+  for (int e = 31; e >= 0; e--) neg = __funnelshift_l(__float_as_uint(z[e] + 0.0f), neg, 1);
+  const uint32_t vmask = valid >= 32 ? 0xFFFFFFFFu : (valid <= 0 ? 0u : ((1u << valid) - 1u));
+  bits_row[n0 >> 5] = ~neg & vmask;
+  float a[16];                                            // pairwise tree of |z|, first level formed on the fly
+#pragma unroll
+  for (int e = 0; e < 16; e++)
+    a[e] = (2 * e < valid ? fabsf(z[2 * e]) : 0.0f) + (2 * e + 1 < valid ? fabsf(z[2 * e + 1]) : 0.0f);
+  constexpr int SPAN = (BETA < 32 ? BETA : 32) / 2;       // pairs per group inside the chunk
+#pragma unroll
+  for (int w = 1; w < SPAN; w <<= 1)
+#pragma unroll
+    for (int e = 0; e < 16; e += 2 * w) a[e] += a[e + w];
+  if constexpr (BETA <= 32) {
+#pragma unroll
+    for (int gi = 0; gi < 32 / BETA; gi++) {
+      const int64_t gidx = n0 / BETA + gi;
+      const int cnt = valid - gi * BETA < BETA ? valid - gi * BETA : BETA;
+      if (gidx < ld_scales) store_next_scale(scales, bf16, srow + gidx, cnt > 0 ? a[gi * SPAN] / static_cast<float>(cnt) : 0.0f);
+    }
+  } else {
+    carry += a[0];
+    if ((n0 + 32) % BETA == 0) {
+      const int64_t g0 = n0 + 32 - BETA, gidx = g0 / BETA;
+      const int64_t cnt = N - g0 < BETA ? N - g0 : BETA;
+      if (gidx < ld_scales) store_next_scale(scales, bf16, srow + gidx, cnt > 0 ? carry / static_cast<float>(cnt) : 0.0f);
+      carry = 0.0f;
+    }
+  }
+}
+
 // Walks the stages a producer thread owns (every second stage of the CTA's stream of tiles) and keeps
 // the row pointers of the tile it is in.
 struct StageCursor {
@@ -66,7 +111,8 @@ struct StageCursor {
 };
 
 // ASUB: scale groups per packed word of A (1: groups of whole words; 2 .. 16: beta_a = 16 .. 2).
-template <int TN, int ASUB>
+// FUSE: the epilogue binarizes the (affinely mapped) output rows for the next layer instead of storing them.
+template <int TN, int ASUB, bool FUSE>
 __global__ void __launch_bounds__(kThreads, 1)
 hbmm_fold_kernel(const Args g) {
   using S = Smem<TN>;
@@ -311,19 +357,31 @@ hbmm_fold_kernel(const Args g) {
       const int64_t m = (tile / tiles_n) * TM + row, nb = (tile % tiles_n) * TN;
       // the tile's column factors go through shared memory (one copy per warp, so no warp waits for
       // another): requested before the wait for the accumulator, read back as broadcasts
-      float fcol[TN / 32];
+      float fcol[TN / 32], fsc[TN / 32], fsh[TN / 32];
 #pragma unroll
-      for (int i = 0; i < TN / 32; i++) fcol[i] = __ldg(g.w_down + nb + i * 32 + lane);   // w_down holds a whole number of tiles
+      for (int i = 0; i < TN / 32; i++) {
+        const int64_t n = nb + i * 32 + lane;
+        fcol[i] = __ldg(g.w_down + n);                                                     // w_down holds a whole number of tiles
+        fsc[i] = (FUSE && g.bn_scale && n < g.N) ? __ldg(g.bn_scale + n) : 1.0f;
+        fsh[i] = (FUSE && g.bn_shift && n < g.N) ? __ldg(g.bn_shift + n) : 0.0f;
+      }
       if (!mbar_wait(&tfull[buf], static_cast<uint32_t>((ti >> 1) & 1), abort_flag, 5)) break;
       if (!mbar_wait(&rowfull[slot], static_cast<uint32_t>((ti / kRowSlots) & 1), abort_flag, 5)) break;   // long complete
       tc_fence_after();
       const float fa = rowdown[slot * TM + row];
-      float* cf = colf + warp * TN;
+      float* cf = colf + warp * (3 * TN);
 #pragma unroll
-      for (int i = 0; i < TN / 32; i++) cf[i * 32 + lane] = fcol[i];
+      for (int i = 0; i < TN / 32; i++) {
+        cf[i * 32 + lane] = fcol[i];
+        if (FUSE) {
+          cf[TN + i * 32 + lane] = fsc[i];
+          cf[2 * TN + i * 32 + lane] = fsh[i];
+        }
+      }
       __syncwarp();
       if (lane == 0) mbar_arrive(&rowempty[slot]);
       float* dst = g.C + m * g.ldc + nb;
+      float carry = 0.0f;                                   // |z| sum of a group wider than a 32-column chunk
 #pragma unroll
       for (int c = 0; c < TN / 32; c++) {
         uint32_t v1[32], v2[32];
@@ -331,7 +389,40 @@ hbmm_fold_kernel(const Args g) {
         tmem_ld32(t_addr, v1);
         tmem_ld32(t_addr + TN, v2);
         tmem_ld_wait();
-        if (m < g.M) {
+        if constexpr (FUSE) {
+          if (m < g.M) {
+          // affine map per column, then the row is binarized for the next layer: packed word + group scales
+          float z[32];
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            const float4 fw = *reinterpret_cast<const float4*>(cf + c * 32 + j);
+            const float4 bs = *reinterpret_cast<const float4*>(cf + TN + c * 32 + j);
+            const float4 bh = *reinterpret_cast<const float4*>(cf + 2 * TN + c * 32 + j);
+            const float w4[4] = {fw.x, fw.y, fw.z, fw.w}, s4[4] = {bs.x, bs.y, bs.z, bs.w}, h4[4] = {bh.x, bh.y, bh.z, bh.w};
+#pragma unroll
+            for (int e = 0; e < 4; e++)
+              z[j + e] = fmaf((__uint_as_float(v1[j + e]) + __uint_as_float(v2[j + e])) * fa * w4[e], s4[e], h4[e]);
+          }
+          const int64_t n0 = nb + c * 32;
+          const int valid = g.N - n0 >= 32 ? 32 : static_cast<int>(g.N - n0 > 0 ? g.N - n0 : 0);
+          uint32_t* brow = g.nx_bits + m * g.nx_ld_words;
+          const int64_t srow = m * g.nx_ld_scales;
+          switch (g.nx_beta) {
+            case 2: emit_next_chunk<2>(z, valid, n0, g.N, brow, g.nx_scales, g.nx_bf16, srow, g.nx_ld_scales, carry); break;
+            case 4: emit_next_chunk<4>(z, valid, n0, g.N, brow, g.nx_scales, g.nx_bf16, srow, g.nx_ld_scales, carry); break;
+            case 8: emit_next_chunk<8>(z, valid, n0, g.N, brow, g.nx_scales, g.nx_bf16, srow, g.nx_ld_scales, carry); break;
+            case 16: emit_next_chunk<16>(z, valid, n0, g.N, brow, g.nx_scales, g.nx_bf16, srow, g.nx_ld_scales, carry); break;
+            case 32: emit_next_chunk<32>(z, valid, n0, g.N, brow, g.nx_scales, g.nx_bf16, srow, g.nx_ld_scales, carry); break;
+            case 64: emit_next_chunk<64>(z, valid, n0, g.N, brow, g.nx_scales, g.nx_bf16, srow, g.nx_ld_scales, carry); break;
+            default: emit_next_chunk<128>(z, valid, n0, g.N, brow, g.nx_scales, g.nx_bf16, srow, g.nx_ld_scales, carry); break;
+          }
+          if (c == TN / 32 - 1 && nb + TN >= g.N) {
+            // last column tile: the row's zero padding past what the tiles cover
+            for (int64_t wz = (nb + TN) >> 5; wz < g.nx_ld_words; wz++) brow[wz] = 0u;
+            for (int64_t sz = (nb + TN) / g.nx_beta; sz < g.nx_ld_scales; sz++) store_next_scale(g.nx_scales, g.nx_bf16, srow + sz, 0.0f);
+          }
+          }
+        } else if (m < g.M) {
 #pragma unroll
           for (int j = 0; j < 32; j += 4) {
             const float4 fw = *reinterpret_cast<const float4*>(cf + c * 32 + j);
@@ -375,6 +466,9 @@ Args make_args(const PackedView& A, const PackedView& W, float* C, int64_t ldc) 
   g.w_gw = W.beta >= W.K ? g.n_words : (w_subword ? 1 : W.beta / 32);
   g.w_prep = nullptr;
   g.w_down = nullptr;
+  g.fuse = 0; g.nx_bf16 = 0; g.nx_beta = 32; g.nx_pad = 0;
+  g.bn_scale = nullptr; g.bn_shift = nullptr; g.nx_bits = nullptr; g.nx_scales = nullptr;
+  g.nx_ld_words = 0; g.nx_ld_scales = 0;
   return g;
 }
 
@@ -388,13 +482,13 @@ size_t prep_bytes(const Args& g) {
   return stage_bytes<TN>(g) + static_cast<size_t>((g.N + TN - 1) / TN) * TN * sizeof(float);
 }
 
-template <int TN, int ASUB>
+template <int TN, int ASUB, bool FUSE = false>
 cudaError_t launch_fold(Args g, void* workspace, cudaStream_t stream, bool w_prepared) {
   using S = Smem<TN>;
   static bool configured = false;
   static int sms = 0;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(hbmm_fold_kernel<TN, ASUB>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::BYTES);
+    cudaError_t e = cudaFuncSetAttribute(hbmm_fold_kernel<TN, ASUB, FUSE>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::BYTES);
     if (e != cudaSuccess) return e;
     int dev = 0;
     cudaGetDevice(&dev);
@@ -412,11 +506,15 @@ cudaError_t launch_fold(Args g, void* workspace, cudaStream_t stream, bool w_pre
   g.w_down = down;
   const int64_t tiles = ((g.M + TM - 1) / TM) * tiles_n;
   const unsigned grid = static_cast<unsigned>(tiles < sms ? tiles : sms);   // one persistent CTA per SM
-  return launch_pdl(hbmm_fold_kernel<TN, ASUB>, dim3(grid), dim3(kThreads), S::BYTES, stream, g);
+  return launch_pdl(hbmm_fold_kernel<TN, ASUB, FUSE>, dim3(grid), dim3(kThreads), S::BYTES, stream, g);
 }
 
 template <int TN>
 cudaError_t launch_fold_tn(const Args& g, void* workspace, cudaStream_t stream, bool w_prepared) {
+  if (g.fuse) {      // the fused epilogue is built for activation groups of whole words
+    if (g.a_sub != 1) return cudaErrorNotSupported;
+    return launch_fold<TN, 1, true>(g, workspace, stream, w_prepared);
+  }
   switch (g.a_sub) {
     case 2: return launch_fold<TN, 2>(g, workspace, stream, w_prepared);
     case 4: return launch_fold<TN, 4>(g, workspace, stream, w_prepared);
@@ -444,9 +542,21 @@ size_t gemm_fold_workspace_bytes(const PackedView& A, const PackedView& W) {
 }
 
 // workspace: device, 16-byte aligned, at least gemm_fold_workspace_bytes.
+// The fused epilogue closes a group inside one thread's row of a tile: the group must divide the tile width.
+bool gemm_fold_next_supported(int64_t N, int32_t beta_next) {
+  const int tn = N <= 64 ? 64 : 128;
+  return (beta_next == 2 || beta_next == 4 || beta_next == 8 || beta_next == 16 || beta_next == 32 || beta_next == 64 ||
+          beta_next == 128) && beta_next <= tn;
+}
+
 cudaError_t launch_gemm_fold(const PackedView& A, const PackedView& W, float* C, int64_t ldc, void* workspace,
-                             cudaStream_t stream, bool w_prepared) {
-  const Args g = make_args(A, W, C, ldc);
+                             cudaStream_t stream, bool w_prepared, const FoldNext* next) {
+  Args g = make_args(A, W, C, ldc);
+  if (next) {
+    g.fuse = 1; g.nx_bf16 = next->scale_bf16; g.nx_beta = next->beta;
+    g.bn_scale = next->bn_scale; g.bn_shift = next->bn_shift; g.nx_bits = next->bits; g.nx_scales = next->scales;
+    g.nx_ld_words = next->ld_words; g.nx_ld_scales = next->ld_scales;
+  }
   return g.N <= 64 ? launch_fold_tn<64>(g, workspace, stream, w_prepared) : launch_fold_tn<128>(g, workspace, stream, w_prepared);
 }
 

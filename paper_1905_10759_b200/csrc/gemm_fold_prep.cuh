@@ -37,7 +37,7 @@ struct Smem {
   static constexpr int OFF_B = OFF_A + STAGES * A_STAGE;
   static constexpr int OFF_ROWF = OFF_B + STAGES * B_STAGE;
   static constexpr int OFF_COLF = OFF_ROWF + 2 * kRowSlots * TM * 4;  // per slot and row: normalising power of two and its inverse
-  static constexpr int OFF_BAR = OFF_COLF + 4 * TN * 4;               // the tile's column factors, one copy per epilogue warp
+  static constexpr int OFF_BAR = OFF_COLF + 3 * 4 * TN * 4;           // the tile's column factors (power of two, affine scale and shift), one copy per epilogue warp
   static constexpr int NBAR = 2 * STAGES + 4 + 1 + 2 * kRowSlots;     // full, empty, tfull[2], tempty[2], drain, rowfull, rowempty
   static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
   static constexpr int BYTES = OFF_MISC + 16;

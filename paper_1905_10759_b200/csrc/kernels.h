@@ -82,6 +82,19 @@ struct FoldArgs {
   int32_t a_sub, w_sub;    // scale groups per K-word: 1, or 32 / beta for the sub-word groups beta = 2 .. 16
   const unsigned char* w_prep;   // W expanded into [n tile][stage][stage bytes]
   const float* w_down;           // per weight row: the power of two that undoes its normalisation
+  // Fused epilogue (fuse != 0): z = bn_scale[n] * C + bn_shift[n] is Hadamard-binarized along n for the next
+  // layer and only its packed form is written (C is ignored).
+  int32_t fuse, nx_bf16, nx_beta, nx_pad;
+  const float* bn_scale; const float* bn_shift;      // per column; null = 1 / 0
+  uint32_t* nx_bits; void* nx_scales;
+  int64_t nx_ld_words, nx_ld_scales;
+};
+// Where the fused epilogue of the folded kernel writes the next layer's operand.
+struct FoldNext {
+  const float* bn_scale; const float* bn_shift;
+  uint32_t* bits; void* scales;
+  int64_t ld_words, ld_scales;
+  int32_t scale_bf16, beta;
 };
 // The weight expansion as a job another kernel can run: n_stages x tiles_n tasks of tn threads each
 // (n_stages counts tasks per column tile: single stages of the e4m3 layout, runs of stages of the folded one).
@@ -114,7 +127,9 @@ cudaError_t read_gemm_fold_error(int* code);
 bool gemm_fold_supported(const PackedView& A, const PackedView& W);
 size_t gemm_fold_workspace_bytes(const PackedView& A, const PackedView& W);
 cudaError_t launch_gemm_fold(const PackedView& A, const PackedView& W, float* C, int64_t ldc, void* workspace,
-                             cudaStream_t stream, bool w_prepared = false);
+                             cudaStream_t stream, bool w_prepared = false, const FoldNext* next = nullptr);
+// Group sizes the fused epilogue can emit for an output of N columns.
+bool gemm_fold_next_supported(int64_t N, int32_t beta_next);
 void gemm_fold_prep_job(const PackedView& A, const PackedView& W, void* workspace, UmmaPrepJob* job);
 
 // Dense x packed contraction (HBWN), three kernels:

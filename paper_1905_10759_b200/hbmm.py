@@ -32,7 +32,7 @@ EXPORTS = [
     "hbmm_operand_bytes", "hbmm_quantize", "hbmm_gemm_workspace_bytes", "hbmm_gemm", "hbmm_gemm_ex",
     "hbmm_gemm_partials", "hbmm_conv_workspace_bytes", "hbmm_conv_im2col", "hbmm_status_string",
     "hbmm_version", "hbmm_conv_im2col_static", "hbmm_last_device_error", "hbmm_conv_im2col_ex",
-    "hbmm_binarize_backward",
+    "hbmm_binarize_backward", "hbmm_gemm_binarize_next",
 ]
 STATIC_SCRATCH_BYTES = 32 << 20
 
@@ -227,6 +227,22 @@ CONV_WEIGHTS_PREPARED = 1
 
 _lib.hbmm_binarize_backward.argtypes = [_vp, _i64, _vp, _i64, _i64, _i64, _i32, _vp, _i64, _vp]
 _lib.hbmm_binarize_backward.restype = _i32
+
+
+_lib.hbmm_gemm_binarize_next.argtypes = [_P(hbmm_operand), _P(hbmm_operand), _vp, _vp, _P(hbmm_operand), _vp, _sz, _vp]
+_lib.hbmm_gemm_binarize_next.restype = _i32
+
+
+def gemm_binarize_next(A: "Operand", W: "Operand", nxt: "Operand", workspace: torch.Tensor, bn_scale: Optional[torch.Tensor] = None,
+                       bn_shift: Optional[torch.Tensor] = None, stream=None) -> "Operand":
+    """hbmm_gemm_binarize_next: the product's rows, after an optional per-column affine map, leave the kernel
+    already binarized for the next layer (bits and scales of `nxt`); the fp32 product is never stored."""
+    _check(_lib.hbmm_gemm_binarize_next(ctypes.byref(A.desc), ctypes.byref(W.desc),
+                                        _dev_ptr(bn_scale) if bn_scale is not None else None,
+                                        _dev_ptr(bn_shift) if bn_shift is not None else None, ctypes.byref(nxt.desc),
+                                        _dev_ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)),
+           "hbmm_gemm_binarize_next")
+    return nxt
 
 
 def binarize_backward(x: torch.Tensor, gy: torch.Tensor, beta: int, gx: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:

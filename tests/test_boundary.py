@@ -139,6 +139,11 @@ def test_host_validation_rejects_before_launch(hb):
     assert call(bad, Wc, ws, n.value) == hb.ERR_INVALID_ARG                           # filter larger than image
     assert call(g, Wc, ws, n.value, beta_a=12) == hb.ERR_UNSUPPORTED
     assert lib.hbmm_conv_im2col_ex(x, 0, ctypes.byref(g), 36, 0, ctypes.byref(Wc.desc), c, 4, ws, n.value, 2, None) == hb.ERR_INVALID_ARG  # unknown flag
+    fz = lib.hbmm_gemm_binarize_next
+    nx = _fake_packed(hb, 8, 4, 2)
+    assert fz(ctypes.byref(A.desc), ctypes.byref(W.desc), None, None, ctypes.byref(nx.desc), None, 0, None) == hb.ERR_WORKSPACE
+    assert fz(ctypes.byref(A.desc), ctypes.byref(W.desc), None, None, ctypes.byref(_fake_packed(hb, 8, 5, 2).desc), None, 0, None) == hb.ERR_INVALID_ARG   # K of next != rows of W
+    assert fz(ctypes.byref(A.desc), ctypes.byref(W.desc), None, None, ctypes.byref(_fake_packed(hb, 8, 4, 4).desc), None, 0, None) == hb.ERR_UNSUPPORTED   # group as long as the row
     bw = lib.hbmm_binarize_backward
     assert bw(x, 64, x, 64, 8, 64, 4, c, 32, None) == hb.ERR_INVALID_ARG          # output rows shorter than K
     assert bw(x, 64, x, 64, 8, 64, 0, c, 64, None) == hb.ERR_INVALID_ARG          # beta < 1

@@ -556,3 +556,62 @@ def test_binarize_backward_matches_oracle(hb, rows, K, beta, pad):
     tol = (int(np.ceil(np.log2(max(be, 2)))) + int(np.ceil(be / 32)) + 4) * gu.U
     err = np.abs(got[:, :K].astype(np.float64) - ref)
     assert (err <= tol * mag + 1e-30).all(), float((err / (mag + 1e-30)).max() / gu.U)
+
+
+# ------------------------------------------------------------------ product fused with the next layer's binarization
+FUSED_CASES = [
+    # M, N, K, beta_a, beta_w, beta_next, next scale dtype, affine map?
+    (200, 128, 576, 32, 32, 32, 0, True),
+    (130, 1000, 1024, 64, 64, 64, 0, True),     # ragged N: tail group of 40 columns, absent columns in the last tile
+    (70, 64, 256, 32, 32, 4, 0, True),          # narrow tile
+    (65, 200, 320, 32, 128, 128, 0, False),     # group as wide as the tile
+    (40, 72, 384, 32, 32, 16, 1, True),         # bf16 scales, two column tiles with a ragged second one
+    (300, 130, 640, 32, 32, 2, 0, True),
+    (129, 256, 2304, 32, 32, 8, 0, False),
+]
+
+
+@pytest.mark.parametrize("M,N,K,ba,bw,bn,sdt,affine", FUSED_CASES)
+def test_gemm_binarize_next_matches_oracle(hb, M, N, K, ba, bw, bn, sdt, affine):
+    """hbmm_gemm_binarize_next against the composition of the pinned oracle steps: product, affine map,
+    binarization of its rows.  Signs are compared where z is outside the product's own error band (inside it
+    the fp32 value the kernel computed decides, as the header says); scales to the band's mean plus the
+    rounding of a pairwise fp32 tree."""
+    gu = _gu()
+    a = inputs.normal((M, K), 9300 + M + K)
+    w = inputs.he_normal(N, K, 9400 + N + K)
+    A, da, sa = gu.oracle_operand(a, ba)
+    W, dw, sw = gu.oracle_operand(w, bw)
+    c_ref, absref = oracle.hbmm_from_quantized(da, sa, gu.eff_beta(ba, K), dw, sw, gu.eff_beta(bw, K))
+    fine = gu.elementwise_magnitude(da, gu.eff_beta(ba, K), dw, gu.eff_beta(bw, K), K)
+    rng = np.random.default_rng(M + N)
+    bs = (rng.uniform(0.5, 2.0, N) * rng.choice([-1.0, 1.0], N)).astype(np.float32) if affine else np.ones(N, np.float32)
+    bh = (0.3 * rng.standard_normal(N)).astype(np.float32) if affine else np.zeros(N, np.float32)
+    z_ref = c_ref * bs.astype(np.float64) + bh.astype(np.float64)
+    band = np.abs(bs) * (RTOL * absref + gu.FOLDED_FLOOR_ULPS * gu.U * fine) + 4 * gu.U * (np.abs(c_ref * bs) + np.abs(bh)) + 1e-30
+    nxt = hb.alloc_operand(M, N, bn, sdt)
+    nxt.bits.fill_(-1)
+    nxt.scales.fill_(float("nan"))
+    ws = _gemm_ws(hb, A, W)
+    hb.gemm_binarize_next(A, W, nxt, ws, torch.from_numpy(bs).cuda() if affine else None, torch.from_numpy(bh).cuda() if affine else None)
+    torch.cuda.synchronize()
+    bits = gu.host_bits(nxt.bits)
+    lw = bits.shape[1]
+    got_sign = ((bits[:, np.arange(N) // 32] >> (np.arange(N) % 32).astype(np.uint32)) & 1).astype(np.int8) * 2 - 1
+    want_sign = np.where(z_ref >= 0, 1, -1)
+    decided = np.abs(z_ref) > band
+    assert (got_sign[decided] == want_sign[decided]).all()
+    assert decided.mean() > 0.99
+    # zero padding: bits past N and words past ceil(N / 32)
+    full = np.zeros((M, lw * 32), dtype=np.int8)
+    full[:, :N] = (got_sign > 0)
+    assert np.array_equal(bits, oracle.pack(np.where(full > 0, 1, -1).astype(np.int8)[:, :N], lw))
+    G = -(-N // bn)
+    sc = nxt.scales.float().cpu().numpy().astype(np.float64)
+    assert np.all(sc[:, G:] == 0.0)
+    tree = (int(np.ceil(np.log2(bn))) + 3) * gu.U + (2.0 ** -8 if sdt == hb.BF16 else 0.0)
+    for g in range(G):
+        sl = slice(g * bn, min((g + 1) * bn, N))
+        want = np.abs(z_ref[:, sl]).mean(axis=1)
+        tol = band[:, sl].mean(axis=1) + tree * want
+        assert (np.abs(sc[:, g] - want) <= tol).all(), g
