@@ -306,6 +306,25 @@ def side_measurements(torch, hbmm, peaks, iters: int):
         ach = 2.0 * M * N * K / (ms * 1e-3) / 1e12
         out.append({"kernel": "hbmm_fold_kernel/beta_a%d_beta_w%d" % (ba, bw), "shape": [M, N, K], "ms": round(ms, 5), "bound": "tensor",
                     "achieved": ach, "peak": bf16_tflops, "unit": "TFLOP/s", "frac": ach / bf16_tflops})
+    # AlexNet-style fully connected layer at batch 256 (4096 -> 4096, beta 64): product + binarization of its
+    # rows for the next layer, as two calls (fp32 product stored, then hbmm_quantize) and fused in the epilogue
+    Mf, Kf, Nf, bf = 256, 4096, 4096, 64
+    af = torch.randn((Mf, Kf), device="cuda", generator=g)
+    wf = torch.randn((Nf, Kf), device="cuda", generator=g) * (2.0 / Kf) ** 0.5
+    Af = hbmm.quantize(af, hbmm.alloc_operand(Mf, Kf, bf, hbmm.F32))
+    Wf = hbmm.quantize(wf, hbmm.alloc_operand(Nf, Kf, bf, hbmm.F32))
+    wsf = torch.empty(max(hbmm.gemm_workspace_bytes(Af, Wf), 16), dtype=torch.uint8, device="cuda")
+    Cf = torch.empty((Mf, Nf), device="cuda")
+    nxt = hbmm.alloc_operand(Mf, Nf, bf, hbmm.F32)
+
+    def two_calls():
+        hbmm.gemm(Af, Wf, Cf, wsf)
+        hbmm.quantize(Cf, nxt)
+
+    ms2 = time_loop(torch, two_calls, iters)
+    ms1 = time_loop(torch, lambda: hbmm.gemm_binarize_next(Af, Wf, nxt, wsf), iters)
+    out.append({"kernel": "fc_4096x4096_b256_beta64: hbmm_gemm + hbmm_quantize", "shape": [Mf, Nf, Kf], "ms": round(ms2, 5)})
+    out.append({"kernel": "fc_4096x4096_b256_beta64: hbmm_gemm_binarize_next", "shape": [Mf, Nf, Kf], "ms": round(ms1, 5)})
     return out
 
 
