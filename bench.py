@@ -331,8 +331,8 @@ def side_measurements(torch, hbmm, peaks, iters: int):
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
 # (same kernels, same workload); entries are dropped when a kernel changes after its capture.
 NCU_DRAM_BYTES = {
-    ("hbmm_contraction", "conv2_x"): 32.372e6 + 1.853e6,     # profiles/hbmm_fold_kernel_conv2_x.md
-    ("front_end_pack", "conv2_x"): 51.512e6 + 3.521e6,       # profiles/im2col_quantize_tma_kernel_conv2_x.md
+    ("hbmm_contraction", "conv2_x"): 32.373e6 + 2.103e6,     # profiles/hbmm_fold_kernel_conv2_x.md
+    ("front_end_pack", "conv2_x"): 51.511e6 + 2.524e6,       # profiles/im2col_quantize_tma_kernel_conv2_x.md
 }
 
 
