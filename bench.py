@@ -91,7 +91,15 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.rows.append((time.time(), line.strip()))
 
-    def stop(self, t0: float, t1: float):
+    def wait_ready(self, rows: int = 2, timeout: float = 5.0):
+        """nvidia-smi needs a moment to start: block until it has delivered a few samples."""
+        t = time.time()
+        while self.proc is not None and len(self.rows) < rows and time.time() - t < timeout:
+            time.sleep(0.02)
+
+    def stop(self, t0: float, t1: float, t_end: float = None):
+        """Samples inside [t0, t1] (the timed region); when that short region caught fewer than three, the
+        samples of the legs that follow it under the same load (up to t_end) are used and `window` says so."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         time.sleep(0.15)
@@ -100,6 +108,11 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
+        window = "timed region"
+        inside = sum(1 for ts, _ in self.rows if t0 <= ts <= t1 + 0.1)
+        if inside < 3 and t_end is not None:
+            t1 = t_end
+            window = "timed region and the legs after it (weight-expansion step, end-to-end leg)"
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for ts, line in self.rows:
@@ -117,7 +130,7 @@ class ClockSampler:
                 if v.lower().startswith("active"):
                     reasons.add(n)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm), "window": window}
 
 
 FALLBACK_BF16_TFLOPS = 1590.0
@@ -502,7 +515,7 @@ def run_ours(args):
 
     sampler = ClockSampler(local_rank)
     sampler.start()
-    time.sleep(0.3)
+    sampler.wait_ready()
     barrier()
     t0 = time.time()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -513,7 +526,6 @@ def run_ours(args):
     barrier()
     t1 = time.time()
     ms_step = e0.elapsed_time(e1) / args.steps
-    clocks = sampler.stop(t0, t1)
     ms_step = max_over_ranks(ms_step, world, device)
     # the same step with the weight expansion repeated by every call (plain hbmm_conv_im2col), for comparison
     barrier()
@@ -539,6 +551,7 @@ def run_ours(args):
     e1.record()
     barrier()
     ms_e2e = max_over_ranks(e0.elapsed_time(e1) / args.steps, world, device)
+    clocks = sampler.stop(t0, t1, time.time())
     h2d = sum(L["x_host"].numel() * 4 + L["xb_host"].numel() * 2 for L in layers)
     d2h = sum(L["C_host"].numel() * 4 + L["Cb_host"].numel() * 4 for L in layers)
 

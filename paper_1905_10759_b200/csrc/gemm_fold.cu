@@ -485,15 +485,13 @@ size_t prep_bytes(const Args& g) {
 template <int TN, int ASUB, bool FUSE = false>
 cudaError_t launch_fold(Args g, void* workspace, cudaStream_t stream, bool w_prepared) {
   using S = Smem<TN>;
-  static bool configured = false;
-  static int sms = 0;
-  if (!configured) {
+  static DeviceOnce configured;
+  int dev = 0, sms = 0;
+  if (current_device(&dev, &sms) != cudaSuccess) return cudaErrorInvalidDevice;
+  if (configured.pending(dev)) {
     cudaError_t e = cudaFuncSetAttribute(hbmm_fold_kernel<TN, ASUB, FUSE>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::BYTES);
     if (e != cudaSuccess) return e;
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    configured = true;
+    configured.mark(dev);
   }
   const int64_t tiles_n = (g.N + TN - 1) / TN, n_stages = (g.n_words + WPS - 1) / WPS;
   unsigned char* stages = static_cast<unsigned char*>(workspace);

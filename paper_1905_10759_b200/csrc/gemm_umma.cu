@@ -327,15 +327,13 @@ size_t prep_bytes(const Args& g) {
 template <int TN>
 cudaError_t launch_umma(Args g, void* workspace, cudaStream_t stream, bool w_prepared) {
   using S = Smem<TN>;
-  static bool configured = false;
-  static int sms = 0;
-  if (!configured) {
+  static DeviceOnce configured;
+  int dev = 0, sms = 0;
+  if (current_device(&dev, &sms) != cudaSuccess) return cudaErrorInvalidDevice;
+  if (configured.pending(dev)) {
     cudaError_t e = cudaFuncSetAttribute(hbmm_umma_kernel<TN>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::BYTES);
     if (e != cudaSuccess) return e;
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    configured = true;
+    configured.mark(dev);
   }
   const int64_t tiles_n = (g.N + TN - 1) / TN, n_stages = (g.n_words + WPS - 1) / WPS;
   dim3 pgrid(static_cast<unsigned>(n_stages), static_cast<unsigned>(tiles_n));

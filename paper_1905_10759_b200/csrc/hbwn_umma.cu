@@ -420,17 +420,15 @@ cudaError_t launch(Args g, const CUtensorMap& a_map, void* workspace, cudaStream
                    bool w_prepared = false) {
   using S = Smem<TN, NP>;
   constexpr int kResBytes = 225 * 1024;
-  static bool configured = false;
-  static int sms = 0;
-  if (!configured) {
+  static DeviceOnce configured;
+  int dev = 0, sms = 0;
+  if (current_device(&dev, &sms) != cudaSuccess) return cudaErrorInvalidDevice;
+  if (configured.pending(dev)) {
     cudaError_t e = cudaFuncSetAttribute(hbwn_umma_kernel<TN, NP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::BYTES);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(hbwn_umma_kernel<TN, NP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kResBytes);
     if (e != cudaSuccess) return e;
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    configured = true;
+    configured.mark(dev);
   }
   const int64_t tiles_n = (g.N + TN - 1) / TN, n_kb = g.n_kb;
   dim3 pgrid(static_cast<unsigned>(n_kb), static_cast<unsigned>(tiles_n));

@@ -387,11 +387,11 @@ cudaError_t launch_im2col_quantize_tma(const void* x, const ConvGeom& g, uint32_
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return cudaErrorNotSupported;
   }
-  static bool configured = false;
-  if (!configured) {
+  static DeviceOnce configured;
+  if (configured.pending(dev)) {
     cudaError_t e = cudaFuncSetAttribute(im2col_quantize_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 104 * 1024);
     if (e != cudaSuccess) return e;
-    configured = true;
+    configured.mark(dev);
   }
   const int64_t n_items = static_cast<int64_t>(g.B) * p.yo_blocks * p.splits;
   if (n_items > (int64_t{1} << 30)) return cudaErrorNotSupported;

@@ -1,11 +1,26 @@
 // Internal launcher interface between the C-ABI layer (api.cu) and the kernel files.
 // Host-only declarations; every launcher enqueues on `stream` and returns the launch status.
 #pragma once
+#include <atomic>
 #include <cstddef>
 #include <cstdint>
 #include <cuda_runtime.h>
 
 namespace hbmm {
+
+// A kernel's opt-in shared-memory size is a per-device attribute, so "already configured" is kept per device
+// (one process may drive several GPUs); setting it twice is harmless, hence no lock.
+struct DeviceOnce {
+  std::atomic<uint64_t> mask{0};
+  bool pending(int dev) const { return dev < 0 || dev >= 64 || !((mask.load(std::memory_order_acquire) >> dev) & 1u); }
+  void mark(int dev) { if (dev >= 0 && dev < 64) mask.fetch_or(uint64_t{1} << dev, std::memory_order_release); }
+};
+// Current device and its multiprocessor count.
+inline cudaError_t current_device(int* dev, int* sms) {
+  cudaError_t e = cudaGetDevice(dev);
+  if (e != cudaSuccess) return e;
+  return cudaDeviceGetAttribute(sms, cudaDevAttrMultiProcessorCount, *dev);
+}
 
 // Device-side view of one packed Hadamard-binary operand (validated by the caller).
 struct PackedView {
