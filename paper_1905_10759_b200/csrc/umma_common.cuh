@@ -52,12 +52,12 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t by
   asm volatile("{\n\t.reg .b64 st;\n\tmbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n\t}" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
 // Asynchronous bulk copy global -> this CTA's shared memory (both 16-byte aligned, size a multiple of
-// 16); completion is counted in bytes on the mbarrier.  No multicast.
+// 16); completion is counted in bytes on the mbarrier.  The copy targets this CTA alone.
 __device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
-// Tiled 2-D tensor copy global -> this CTA's shared memory through a tensor map (no multicast).
+// Tiled 2-D tensor copy global -> this CTA's shared memory through a tensor map (this CTA alone).
 // x (innermost coordinate) times the element size must be a multiple of 16 bytes; rows and columns
 // outside the tensor arrive as zeros and still count towards the transaction bytes.
 __device__ __forceinline__ void tma_load_2d(void* dst, const void* tensor_map, int32_t x, int32_t y, uint64_t* bar) {
@@ -74,7 +74,7 @@ __device__ __forceinline__ void tma_load_4d(void* dst, const void* tensor_map, i
 // im2col-mode tensor copy of an NHWC image: `pixels-per-column` consecutive base pixels starting at
 // (w, h, n) (walking W, then H, then N inside the map's bounding box), each displaced by the filter
 // offsets (w_off, h_off), `channels-per-pixel` channels from c.  c times the element size must be a
-// multiple of 16 bytes; pixels outside the image arrive as zeros.  No multicast.
+// multiple of 16 bytes; pixels outside the image arrive as zeros.  This CTA alone.
 __device__ __forceinline__ void tma_load_im2col_4d(void* dst, const void* tensor_map, int32_t c, int32_t w, int32_t h, int32_t n,
                                                    uint16_t w_off, uint16_t h_off, uint64_t* bar) {
   asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6], {%7, %8};"
