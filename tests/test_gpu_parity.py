@@ -615,3 +615,32 @@ def test_gemm_binarize_next_matches_oracle(hb, M, N, K, ba, bw, bn, sdt, affine)
         want = np.abs(z_ref[:, sl]).mean(axis=1)
         tol = band[:, sl].mean(axis=1) + tree * want
         assert (np.abs(sc[:, g] - want) <= tol).all(), g
+
+
+@pytest.mark.parametrize("beta_a,xbf16", [(32, False), (1, True)])
+def test_back_to_back_calls_on_one_workspace_do_not_disturb_each_other(hb, beta_a, xbf16):
+    """The kernels of a convolution call are launched so that their set-up may overlap the tail of the kernel
+    before them.  A second call that reuses the workspace right behind the first must still wait for it:
+    the results of a burst of calls equal those of calls separated by device synchronisation."""
+    shape = inputs.ConvShape("t", 8, 64, 28, 28, 72, 3, 3, 1, 1)
+    K = 64 * 9
+    Wop = hb.quantize(torch.from_numpy(inputs.he_normal(72, K, 611)).cuda(), hb.alloc_operand(72, K, 32))
+    geom = hb.make_geom(8, 64, 28, 28, 3, 3, (1, 1), (1, 1))
+    ws = torch.empty(hb.conv_workspace_bytes(geom, beta_a, hb.F32, Wop), dtype=torch.uint8, device="cuda")
+    xs = []
+    for seed in range(4):
+        x = torch.from_numpy(inputs.conv_activation(shape, 620 + seed, signed=True)).cuda()
+        xs.append(x.to(torch.bfloat16) if xbf16 else x)
+    calm = []
+    for x in xs:
+        out = torch.empty((shape.M, 72), device="cuda")
+        hb.conv_im2col(x, geom, beta_a, hb.F32, Wop, out, ws)
+        torch.cuda.synchronize()
+        calm.append(out)
+    burst = [torch.empty((shape.M, 72), device="cuda") for _ in xs]
+    for _ in range(3):
+        for x, out in zip(xs, burst):
+            hb.conv_im2col(x, geom, beta_a, hb.F32, Wop, out, ws)
+    torch.cuda.synchronize()
+    for a, b in zip(calm, burst):
+        assert torch.equal(a, b)
