@@ -644,3 +644,36 @@ def test_back_to_back_calls_on_one_workspace_do_not_disturb_each_other(hb, beta_
     torch.cuda.synchronize()
     for a, b in zip(calm, burst):
         assert torch.equal(a, b)
+
+
+def test_two_products_on_two_streams_equal_their_serial_results(hb):
+    """HBMM and HBWN calls that share no buffer may run on different streams at the same time (the schedule
+    the benchmark times): the library keeps no scratch of its own between them, so the results are those of
+    the calls made one after the other."""
+    shapes = [inputs.ConvShape("a", 16, 64, 28, 28, 128, 3, 3, 1, 1), inputs.ConvShape("b", 16, 128, 14, 14, 256, 3, 3, 1, 1)]
+    jobs = []
+    for i, s in enumerate(shapes):
+        K = s.C * 9
+        Wop = hb.quantize(torch.from_numpy(inputs.he_normal(s.N, K, 700 + i)).cuda(), hb.alloc_operand(s.N, K, 32))
+        geom = hb.make_geom(s.B, s.C, s.H, s.W, 3, 3, (1, 1), (1, 1))
+        x = torch.from_numpy(inputs.conv_activation(s, 710 + i, signed=True)).cuda()
+        for beta_a, xin in ((32, x), (1, x.to(torch.bfloat16))):
+            ws = torch.empty(hb.conv_workspace_bytes(geom, beta_a, hb.F32, Wop), dtype=torch.uint8, device="cuda")
+            jobs.append(dict(x=xin, geom=geom, beta_a=beta_a, W=Wop, ws=ws, M=s.M, N=s.N))
+    calm = []
+    for j in jobs:
+        out = torch.empty((j["M"], j["N"]), device="cuda")
+        hb.conv_im2col(j["x"], j["geom"], j["beta_a"], hb.F32, j["W"], out, j["ws"])
+        torch.cuda.synchronize()
+        calm.append(out)
+    outs = [torch.empty_like(c) for c in calm]
+    streams = {32: torch.cuda.Stream(), 1: torch.cuda.Stream()}
+    torch.cuda.synchronize()
+    for _ in range(5):
+        for j, out in zip(jobs, outs):
+            with torch.cuda.stream(streams[j["beta_a"]]):
+                hb.conv_im2col(j["x"], j["geom"], j["beta_a"], hb.F32, j["W"], out, j["ws"])
+    torch.cuda.synchronize()
+    assert hb.last_device_error() == 0
+    for a, b in zip(calm, outs):
+        assert torch.equal(a, b)
