@@ -250,3 +250,45 @@ def conv_im2col(x, w2d, kh, kw, stride, pad, beta_a: int, beta_w: int,
     if beta_a == 1:
         return hbwn(a, w2d, beta_w, scale_dtype)
     return hbmm(a, w2d, beta_a, beta_w, scale_dtype)
+
+
+def binarize_map(x: np.ndarray, beta_a: int) -> np.ndarray:
+    """Eq. 3-4 as printed: an NCHW activation map binarized in runs of ``beta_a`` neighbours along each row of the
+    map (the width axis; the paper asks beta_a <= width, a larger value is taken as the width; a tail run has its
+    own length).  Returns A~ = delta (.) Sign(A) as float64 NCHW."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    B, C, H, W = x.shape
+    b = min(int(beta_a), W)
+    if b == 1:
+        return widen(x.reshape(B * C * H, W)).reshape(B, C, H, W)
+    delta, sign = quantize(x.reshape(B * C * H, W), b)
+    return dequant(delta, sign, b).reshape(B, C, H, W)
+
+
+def im2col_f64(xt: np.ndarray, kh: int, kw: int, stride=(1, 1), pad=(0, 0)) -> np.ndarray:
+    """The gather of ``im2col`` on a float64 map: rows m = (b, yo, xo), columns k = (c, i, j), c slowest; zero outside
+    the image."""
+    xt = np.asarray(xt, dtype=np.float64)
+    B, C, H, W = xt.shape
+    Ho = (H + 2 * pad[0] - kh) // stride[0] + 1
+    Wo = (W + 2 * pad[1] - kw) // stride[1] + 1
+    xp = np.zeros((B, C, H + 2 * pad[0], W + 2 * pad[1]), dtype=np.float64)
+    xp[:, :, pad[0]:pad[0] + H, pad[1]:pad[1] + W] = xt
+    cols = np.empty((B, Ho, Wo, C, kh, kw), dtype=np.float64)
+    for i in range(kh):
+        for j in range(kw):
+            win = xp[:, :, i:i + stride[0] * (Ho - 1) + 1:stride[0], j:j + stride[1] * (Wo - 1) + 1:stride[1]]
+            cols[:, :, :, :, i, j] = win.transpose(0, 2, 3, 1)
+    return cols.reshape(B * Ho * Wo, C * kh * kw)
+
+
+def conv_map_binarized(x: np.ndarray, w2d: np.ndarray, kh: int, kw: int, stride, pad, beta_a: int, beta_w: int):
+    """Convolution of Eq. 3's A~ (``binarize_map``) with W~ (Eq. 1-2 on Reshape(W, (filters, -1))): the activation
+    is binarized on the map, before the gather, so an im2col row mixes scales of several map groups.  Returns
+    ``(C, absref)`` like ``hbmm``: float64 [B*Ho*Wo, filters] and the same sum over absolute values."""
+    at = im2col_f64(binarize_map(x, beta_a), kh, kw, stride, pad)
+    w2d = np.ascontiguousarray(w2d, dtype=np.float32)
+    bw = min(int(beta_w), w2d.shape[1])
+    dw, sw = quantize(w2d, bw)
+    wt = dequant(dw, sw, bw)
+    return matmul_nt(at, wt), matmul_nt(np.abs(at), np.abs(wt))

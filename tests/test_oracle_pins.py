@@ -384,3 +384,97 @@ def test_binarize_backward_beta_one():
     gx = oracle.binarize_backward(x, gy, 1)
     x64, g64 = x.astype(np.float64), gy.astype(np.float64)
     np.testing.assert_allclose(gx, g64 * (1.0 + np.abs(x64) * (np.abs(x64) <= 1.0)), rtol=0, atol=1e-15)
+
+
+# ---------------------------------------------------------------- Eq. 3 as printed: groups along the rows of the activation map
+def test_binarize_map_hand_example():
+    """A 2 x 4 map with beta_a = 2, worked by hand: (1,-3) -> delta 2; (0,2) -> delta 1 with Sign(0) = +1;
+    (-.5,-.5) -> delta .5; (4,-2) -> delta 3."""
+    x = np.array([[[[1.0, -3.0, 0.0, 2.0], [-0.5, -0.5, 4.0, -2.0]]]], dtype=np.float32)
+    want = np.array([[[[2.0, -2.0, 1.0, 1.0], [-0.5, -0.5, 3.0, -3.0]]]])
+    assert np.array_equal(oracle.binarize_map(x, 2), want)
+
+
+def test_binarize_map_groups_run_along_the_width_only():
+    """Each (batch, channel, height) line is binarized on its own: permuting lines permutes the result, the group
+    sums of |A~| equal those of |A| (delta is the mean), and a tail run of one element is kept as it is."""
+    rng = np.random.default_rng(31)
+    x = rng.standard_normal((2, 3, 4, 7)).astype(np.float32)
+    got = oracle.binarize_map(x, 3)
+    perm = rng.permutation(4)
+    assert np.array_equal(oracle.binarize_map(x[:, :, perm, :], 3), got[:, :, perm, :])
+    assert np.array_equal(oracle.binarize_map(x.transpose(1, 0, 2, 3).copy(), 3), got.transpose(1, 0, 2, 3))
+    for g0 in (0, 3):
+        np.testing.assert_allclose(np.abs(got[..., g0:g0 + 3]).sum(-1), np.abs(x[..., g0:g0 + 3].astype(np.float64)).sum(-1), rtol=1e-15)
+        assert np.all(np.abs(got[..., g0:g0 + 3]) == np.abs(got[..., g0:g0 + 1]))        # one magnitude per group
+    assert np.array_equal(got[..., 6], x[..., 6].astype(np.float64))                      # tail group of length 1
+    assert np.array_equal(np.signbit(got), np.signbit(x) & (x != 0))
+    assert np.array_equal(oracle.binarize_map(x, 1), x.astype(np.float64))                # beta_a = 1: full precision
+    assert np.array_equal(oracle.binarize_map(x, 64), oracle.binarize_map(x, 7))          # beta_a above the width: one group per line
+
+
+def test_conv_of_map_binarized_activations_brute_force():
+    """Direct convolution, written as plain loops, of a map binarized by plain loops with filters binarized by plain
+    loops: strided, padded, width not a multiple of beta_a."""
+    rng = np.random.default_rng(32)
+    B, C, H, W, F, kh, kw, st, pd, ba, bw = 2, 2, 5, 6, 3, 3, 3, 2, 1, 4, 6
+    x = (rng.integers(-8, 9, size=(B, C, H, W)) / 4.0).astype(np.float32)
+    w4 = (rng.integers(-8, 9, size=(F, C, kh, kw)) / 8.0).astype(np.float32)
+    at = np.zeros((B, C, H, W))
+    for b in range(B):
+        for c in range(C):
+            for y in range(H):
+                for x0 in range(0, W, ba):
+                    seg = x[b, c, y, x0:x0 + ba].astype(np.float64)
+                    d = sum(abs(v) for v in seg) / len(seg)
+                    for t, v in enumerate(seg):
+                        at[b, c, y, x0 + t] = d if v >= 0 else -d
+    w2d = w4.reshape(F, -1)
+    wt = np.zeros(w2d.shape)
+    for f in range(F):
+        for k0 in range(0, w2d.shape[1], bw):
+            seg = w2d[f, k0:k0 + bw].astype(np.float64)
+            d = sum(abs(v) for v in seg) / len(seg)
+            for t, v in enumerate(seg):
+                wt[f, k0 + t] = d if v >= 0 else -d
+    wt4 = wt.reshape(F, C, kh, kw)
+    Ho, Wo = (H + 2 * pd - kh) // st + 1, (W + 2 * pd - kw) // st + 1
+    ref = np.zeros((B * Ho * Wo, F))
+    for b in range(B):
+        for yo in range(Ho):
+            for xo in range(Wo):
+                for f in range(F):
+                    acc = 0.0
+                    for c in range(C):
+                        for i in range(kh):
+                            for j in range(kw):
+                                y, xx = yo * st + i - pd, xo * st + j - pd
+                                if 0 <= y < H and 0 <= xx < W:
+                                    acc += at[b, c, y, xx] * wt4[f, c, i, j]
+                    ref[(b * Ho + yo) * Wo + xo, f] = acc
+    got, absref = oracle.conv_map_binarized(x, w2d, kh, kw, (st, st), (pd, pd), ba, bw)
+    np.testing.assert_allclose(got, ref, rtol=0, atol=1e-12)
+    assert np.all(absref >= np.abs(got) - 1e-12)
+
+
+def test_conv_of_map_binarized_activations_special_cases():
+    """beta_a = 1 is the HBWN convolution; and a map whose magnitudes are constant along every group is its own
+    binarization, so the result is again the HBWN convolution of the map itself."""
+    rng = np.random.default_rng(33)
+    x = rng.standard_normal((2, 3, 6, 8)).astype(np.float32)
+    w2d = rng.standard_normal((4, 27)).astype(np.float32)
+    a, _ = oracle.conv_map_binarized(x, w2d, 3, 3, (1, 1), (1, 1), 1, 9)
+    b, _ = oracle.conv_im2col(x, w2d, 3, 3, (1, 1), (1, 1), 1, 9)
+    np.testing.assert_allclose(a, b, rtol=0, atol=1e-12)
+    mags = np.repeat(rng.integers(1, 9, size=(2, 3, 6, 2)) / 8.0, 4, axis=-1)
+    xs = (mags * np.where(rng.standard_normal((2, 3, 6, 8)) >= 0, 1.0, -1.0)).astype(np.float32)
+    a, _ = oracle.conv_map_binarized(xs, w2d, 3, 3, (1, 1), (1, 1), 4, 9)
+    b, _ = oracle.conv_im2col(xs, w2d, 3, 3, (1, 1), (1, 1), 1, 9)
+    np.testing.assert_allclose(a, b, rtol=0, atol=1e-12)
+
+
+def test_im2col_f64_matches_the_float_gather():
+    rng = np.random.default_rng(34)
+    x = rng.standard_normal((2, 3, 7, 5)).astype(np.float32)
+    for kh, kw, st, pd in ((3, 3, (1, 1), (1, 1)), (3, 3, (2, 2), (0, 0)), (1, 1, (1, 1), (0, 0)), (5, 3, (1, 2), (2, 1))):
+        assert np.array_equal(oracle.im2col_f64(x.astype(np.float64), kh, kw, st, pd), oracle.im2col(x, kh, kw, st, pd).astype(np.float64))
