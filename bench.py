@@ -338,6 +338,14 @@ def side_measurements(torch, hbmm, peaks, iters: int):
         by = 12.0 * M * K
         out.append({"kernel": "hbmm_binarize_backward/beta%d" % beta, "shape": [M, K], "ms": round(ms, 5), "bound": "hbm",
                     "achieved": by / (ms * 1e-3) / 1e9, "peak": hbm_gbs, "unit": "GB/s", "frac": by / (ms * 1e-3) / 1e9 / hbm_gbs})
+    # Eq. 3 on a conv2_x-shaped activation map (256 x 64 x 56 x 56 fp32, beyond L2): lines of 56, groups of 8
+    amap = torch.randn((256 * 64 * 56, 56), device="cuda", generator=g)
+    for odt, name, ob in ((hbmm.BF16, "bf16", 2.0), (hbmm.F32, "f32", 4.0)):
+        om = torch.empty(amap.shape, device="cuda", dtype=torch.bfloat16 if odt == hbmm.BF16 else torch.float32)
+        ms = time_loop(torch, lambda: hbmm.binarize_dense(amap, 8, odt, om), iters)
+        by = (4.0 + ob) * amap.numel()
+        out.append({"kernel": "hbmm_binarize_dense/beta8_%s" % name, "shape": list(amap.shape), "ms": round(ms, 5), "bound": "hbm",
+                    "achieved": by / (ms * 1e-3) / 1e9, "peak": hbm_gbs, "unit": "GB/s", "frac": by / (ms * 1e-3) / 1e9 / hbm_gbs})
     for ba, bw in ((16, 16), (4, 4), (2, 16)):
         A = hbmm.quantize(a, hbmm.alloc_operand(M, K, ba, hbmm.F32))
         W = hbmm.quantize(w, hbmm.alloc_operand(N, K, bw, hbmm.F32))

@@ -158,6 +158,22 @@ hbmm_status hbmm_binarize_backward(const float *x, int64_t ldx, const float *gy,
                                    int64_t rows, int64_t K, int32_t beta, float *gx, int64_t ldo,
                                    void *stream);
 
+/*
+ * The binarized tensor itself, dense: out[r,k] = delta_g Sign(x[r,k]) (Eq. 2; Eq. 3-4), g the run of beta
+ * consecutive row elements that holds k (a tail run uses its own length), delta_g its mean |x| in fp32,
+ * Sign(0) = +1.  beta >= 1 (any value; beta >= K: one group per row; beta = 1: out = x).
+ * Called on an NCHW activation map viewed as [batch*channels*height, width] with beta = beta_a <= width it is
+ * Eq. 3 as printed -- groups of beta_a neighbours along a row of the map, before the convolution -- and
+ * hbmm_conv_im2col with beta_a = 1 on its output is the convolution of Eq. 3's A~ with W~.  (hbmm_conv_im2col
+ * with beta_a >= 2 groups along K of the im2col row instead, the form Eq. 7 is stated for.)
+ * x: device fp32 [rows, ldx], ldx >= K, 4-byte aligned.  out: device [rows, ldo] of out_dtype (HBMM_F32 or
+ * HBMM_BF16, round to nearest even), ldo >= K, aligned to its element; may not alias x.  16-byte aligned
+ * unpadded rows with a power-of-two beta <= 128 dividing K take the streaming kernel.
+ * Errors: INVALID_ARG, ALIGNMENT, CUDA.
+ */
+hbmm_status hbmm_binarize_dense(const float *x, int64_t ldx, int64_t rows, int64_t K, int32_t beta,
+                                void *out, int32_t out_dtype, int64_t ldo, void *stream);
+
 /* Bytes of scratch hbmm_gemm wants for these operands (host pointer `bytes`).  The tensor-core
  * contractions keep the weight operand there, expanded once per call into the tile layout their
  * kernels stream (HBMM: 4 K bytes per weight row, two fp16 pieces; HBWN: 6 K bytes per weight row,

@@ -267,6 +267,15 @@ hbmm_status hbmm_binarize_backward(const float* x, int64_t ldx, const float* gy,
              ? HBMM_OK : HBMM_ERR_CUDA;
 }
 
+hbmm_status hbmm_binarize_dense(const float* x, int64_t ldx, int64_t rows, int64_t K, int32_t beta, void* out, int32_t out_dtype,
+                                int64_t ldo, void* stream) {
+  if (!x || !out || rows <= 0 || K <= 0 || beta < 1 || ldx < K || ldo < K || !valid_dtype(out_dtype)) return HBMM_ERR_INVALID_ARG;
+  const uintptr_t out_align = out_dtype == HBMM_BF16 ? 2 : 4;
+  if (reinterpret_cast<uintptr_t>(x) % 4 != 0 || reinterpret_cast<uintptr_t>(out) % out_align != 0) return HBMM_ERR_ALIGNMENT;
+  return launch_binarize_dense(x, ldx, rows, K, beta, out, out_dtype == HBMM_BF16, ldo, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? HBMM_OK : HBMM_ERR_CUDA;
+}
+
 hbmm_status hbmm_gemm_workspace_bytes(const hbmm_operand* A, const hbmm_operand* W, size_t* bytes) {
   if (!A || !W || !bytes) return HBMM_ERR_INVALID_ARG;
   *bytes = 0;

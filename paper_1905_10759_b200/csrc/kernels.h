@@ -54,6 +54,10 @@ cudaError_t launch_quantize(const void* x, int x_bf16, int64_t rows, int64_t K, 
 cudaError_t launch_binarize_backward(const float* x, int64_t ldx, const float* gy, int64_t ldg, int64_t rows, int64_t K, int32_t beta,
                                      float* gx, int64_t ldo, cudaStream_t stream);
 
+// The binarized tensor written out dense, fp32 or bf16 (Eq. 2; Eq. 3-4 on an activation map's rows).
+cudaError_t launch_binarize_dense(const float* x, int64_t ldx, int64_t rows, int64_t K, int32_t beta, void* out, bool out_bf16,
+                                  int64_t ldo, cudaStream_t stream);
+
 // Packed x packed contraction on the integer pipe (XOR + POPC).
 cudaError_t launch_gemm_popc(const PackedView& A, const PackedView& W, float* C, int64_t ldc,
                              cudaStream_t stream);

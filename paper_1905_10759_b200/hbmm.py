@@ -32,7 +32,7 @@ EXPORTS = [
     "hbmm_operand_bytes", "hbmm_quantize", "hbmm_gemm_workspace_bytes", "hbmm_gemm", "hbmm_gemm_ex",
     "hbmm_gemm_partials", "hbmm_conv_workspace_bytes", "hbmm_conv_im2col", "hbmm_status_string",
     "hbmm_version", "hbmm_conv_im2col_static", "hbmm_last_device_error", "hbmm_conv_im2col_ex",
-    "hbmm_binarize_backward", "hbmm_gemm_binarize_next",
+    "hbmm_binarize_backward", "hbmm_gemm_binarize_next", "hbmm_binarize_dense",
 ]
 STATIC_SCRATCH_BYTES = 32 << 20
 
@@ -227,6 +227,8 @@ CONV_WEIGHTS_PREPARED = 1
 
 _lib.hbmm_binarize_backward.argtypes = [_vp, _i64, _vp, _i64, _i64, _i64, _i32, _vp, _i64, _vp]
 _lib.hbmm_binarize_backward.restype = _i32
+_lib.hbmm_binarize_dense.argtypes = [_vp, _i64, _i64, _i64, _i32, _vp, _i32, _i64, _vp]
+_lib.hbmm_binarize_dense.restype = _i32
 
 
 _lib.hbmm_gemm_binarize_next.argtypes = [_P(hbmm_operand), _P(hbmm_operand), _vp, _vp, _P(hbmm_operand), _vp, _sz, _vp]
@@ -256,6 +258,29 @@ def binarize_backward(x: torch.Tensor, gy: torch.Tensor, beta: int, gx: Optional
     _check(_lib.hbmm_binarize_backward(_dev_ptr(x), x.stride(0), _dev_ptr(gy), gy.stride(0), x.shape[0], x.shape[1], beta,
                                        _dev_ptr(gx), gx.stride(0), _stream(stream)), "hbmm_binarize_backward")
     return gx
+
+
+def binarize_dense(x: torch.Tensor, beta: int, out_dtype: int = F32, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """hbmm_binarize_dense: x fp32 [rows, K] (row stride >= K, unit column stride); returns delta (.) Sign(x) as fp32 or bf16."""
+    if x.dtype != torch.float32 or x.dim() != 2 or x.stride(1) != 1:
+        raise ValueError("x must be an fp32 matrix with contiguous rows")
+    tdt = torch.bfloat16 if out_dtype == BF16 else torch.float32
+    if out is None:
+        out = torch.empty(x.shape, dtype=tdt, device=x.device)
+    if out.dtype != tdt or out.shape != x.shape or out.stride(1) != 1:
+        raise ValueError("out must match x's shape and the requested type")
+    _check(_lib.hbmm_binarize_dense(_dev_ptr(x), x.stride(0), x.shape[0], x.shape[1], beta, _dev_ptr(out), out_dtype, out.stride(0),
+                                    _stream(stream)), "hbmm_binarize_dense")
+    return out
+
+
+def binarize_map(x: torch.Tensor, beta_a: int, out_dtype: int = F32, stream=None) -> torch.Tensor:
+    """Eq. 3-4 on a contiguous NCHW activation map: groups of beta_a neighbours along each map row.  Argument
+    marshalling only: the map is passed to hbmm_binarize_dense as [batch*channels*height, width]."""
+    if x.dim() != 4 or not x.is_contiguous():
+        raise ValueError("x must be a contiguous NCHW tensor")
+    B, C, H, W = x.shape
+    return binarize_dense(x.view(B * C * H, W), beta_a, out_dtype, stream=stream).view(B, C, H, W)
 
 
 def conv_im2col(x: torch.Tensor, geom: hbmm_conv_geom, beta_a: int, a_scale_dtype: int, W: Operand,

@@ -149,3 +149,10 @@ def test_host_validation_rejects_before_launch(hb):
     assert bw(x, 64, x, 64, 8, 64, 0, c, 64, None) == hb.ERR_INVALID_ARG          # beta < 1
     assert bw(None, 64, x, 64, 8, 64, 4, c, 64, None) == hb.ERR_INVALID_ARG
     assert bw(ctypes.c_void_p(0x5002), 64, x, 64, 8, 64, 4, c, 64, None) == hb.ERR_ALIGNMENT
+    bd = lib.hbmm_binarize_dense
+    assert bd(x, 64, 8, 64, 4, c, hb.F32, 32, None) == hb.ERR_INVALID_ARG            # output rows shorter than K
+    assert bd(x, 64, 8, 64, 0, c, hb.F32, 64, None) == hb.ERR_INVALID_ARG            # beta < 1
+    assert bd(x, 64, 8, 64, 4, c, 7, 64, None) == hb.ERR_INVALID_ARG                 # unknown output type
+    assert bd(x, 64, 8, 64, 4, None, hb.F32, 64, None) == hb.ERR_INVALID_ARG
+    assert bd(x, 64, 8, 64, 4, ctypes.c_void_p(0x5002), hb.F32, 64, None) == hb.ERR_ALIGNMENT
+    assert bd(x, 64, 8, 64, 4, ctypes.c_void_p(0x5001), hb.BF16, 64, None) == hb.ERR_ALIGNMENT

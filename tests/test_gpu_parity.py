@@ -677,3 +677,79 @@ def test_two_products_on_two_streams_equal_their_serial_results(hb):
     assert hb.last_device_error() == 0
     for a, b in zip(calm, outs):
         assert torch.equal(a, b)
+
+
+# ------------------------------------------------------------------ Eq. 3 as printed: the binarized tensor written out dense
+DENSE_CASES = [
+    # rows, K, beta, row padding
+    (64, 576, 2, 0), (33, 1152, 4, 0), (20, 256, 8, 0), (17, 512, 16, 0), (130, 576, 32, 0), (9, 1024, 128, 0), (40, 100, 1, 0),
+    (7, 333, 4, 0),      # ragged K: tail group of one element -> general kernel
+    (1000, 56, 8, 0),    # a 56-wide map line, 7 groups of 8
+    (1000, 28, 16, 0),   # tail group of 12
+    (300, 7, 4, 0),      # conv5-sized map line
+    (5, 45, 7, 3),       # odd everything, padded rows
+    (16, 128, 256, 0),   # beta > K
+]
+
+
+@pytest.mark.parametrize("rows,K,beta,pad", DENSE_CASES)
+def test_binarize_dense_matches_oracle(hb, rows, K, beta, pad):
+    gu = _gu()
+    x = inputs.normal((rows, K), 9300 + rows + K)
+    x[0, :4] = [1.0, -1.0, 0.0, -0.0]                       # Sign(+-0) = +1
+    be = gu.eff_beta(beta, K)
+    delta, sign = oracle.quantize(x, be)
+    ref = oracle.dequant(delta, sign, be)
+    xd = torch.zeros((rows, K + pad)); xd[:, :K] = torch.from_numpy(x)
+    xg = xd.cuda()[:, :K]
+    out = torch.full((rows, K + pad), float("nan"), device="cuda")
+    hb.binarize_dense(xg, beta, hb.F32, out[:, :K])
+    got = out.cpu().numpy()
+    assert np.isnan(got[:, K:]).all()
+    got = got[:, :K]
+    assert np.array_equal(np.signbit(got), sign < 0)                          # signs are bit-exact, zeros positive
+    # the scale is an fp32 tree over at most beta non-negative terms and one multiply
+    tol = (int(np.ceil(np.log2(max(be, 2)))) + int(np.ceil(be / 32)) + 2) * gu.U
+    assert (np.abs(np.abs(got.astype(np.float64)) - np.abs(ref)) <= tol * np.abs(ref)).all()
+    # bf16 output: the same fp32 values rounded to nearest even
+    outb = torch.full((rows, K + pad), float("nan"), device="cuda", dtype=torch.bfloat16)
+    hb.binarize_dense(xg, beta, hb.BF16, outb[:, :K])
+    assert torch.isnan(outb[:, K:]).all()
+    assert torch.equal(outb[:, :K], out[:, :K].to(torch.bfloat16))
+
+
+MAP_CONV_CASES = [
+    # B, C, H, W, filters, stride, beta_a, beta_w
+    (4, 64, 28, 28, 72, 1, 4, 32),
+    (2, 64, 56, 56, 64, 1, 8, 32),
+    (3, 128, 14, 14, 130, 2, 16, 64),      # tail group of 14 along the map line, strided
+    (2, 32, 9, 11, 40, 1, 3, 32),          # odd width, groups of three
+]
+
+
+@pytest.mark.parametrize("B,C,H,W,F,st,ba,bw", MAP_CONV_CASES)
+def test_convolution_of_the_map_binarized_as_in_eq3(hb, B, C, H, W, F, st, ba, bw):
+    """Eq. 3 groups the activations along the rows of the map, before the gather.  The path: hbmm_binarize_dense
+    on the map (bf16 out), then hbmm_conv_im2col with beta_a = 1 on it.  The activation values are A~ rounded
+    to bf16 (2^-9 relative, as for any bf16 activation of the HBWN path); the rest is the HBWN tolerance."""
+    gu = _gu()
+    shape = inputs.ConvShape("t", B, C, H, W, F, 3, 3, st, 1)
+    K = C * 9
+    x = inputs.conv_activation(shape, 9400 + C + W, signed=True)
+    w = inputs.he_normal(F, K, 9500 + F)
+    ref, absref = oracle.conv_map_binarized(x, w, 3, 3, (st, st), (1, 1), ba, bw)
+    Wop = hb.quantize(torch.from_numpy(w).cuda(), hb.alloc_operand(F, K, bw))
+    geom = hb.make_geom(B, C, H, W, 3, 3, (st, st), (1, 1))
+    at = hb.binarize_map(torch.from_numpy(x).cuda(), ba, hb.BF16)
+    ws = torch.empty(hb.conv_workspace_bytes(geom, 1, hb.F32, Wop), dtype=torch.uint8, device="cuda")
+    out = torch.full((shape.M, (F + 3) // 4 * 4), float("nan"), device="cuda")
+    hb.conv_im2col(at, geom, 1, hb.F32, Wop, out, ws)
+    torch.cuda.synchronize()
+    assert hb.last_device_error() == 0
+    rtol = 2.0 ** -9 + _hbwn_rtol(gu, K, bw, True)
+    gu.assert_close_rel_absref(out.cpu().numpy()[:, :F], ref, absref, rtol, "eq3 conv")
+    # and the map itself against the oracle: signs exact, magnitudes to bf16 rounding
+    a64 = oracle.binarize_map(x, ba)
+    ag = at.float().cpu().numpy()
+    assert np.array_equal(np.signbit(ag), a64 < 0)
+    assert (np.abs(np.abs(ag) - np.abs(a64)) <= 2.0 ** -8 * np.abs(a64)).all()
