@@ -4,10 +4,10 @@
 // width this is Eq. 3 as printed: groups of beta_a neighbours along a map row, before any convolution.
 // A pure stream: 4 bytes read and 4 (fp32) or 2 (bf16) written per element, HBM bound.
 //
-// Fast kernel (unpadded fp32 rows, K a multiple of beta, beta a power of two up to 128, element count a multiple of 4 / 8):
-// the tensor is one contiguous run whose groups never straddle a row; a lane owns four (fp32 out) or eight
-// (bf16 out) consecutive elements -- 16-byte loads, one 16-byte store -- and a group is a run inside one
-// lane or several neighbouring lanes whose |x| sums meet in an xor-shuffle tree.
+// Fast kernel (unpadded fp32 rows, K a multiple of beta, beta a power of two up to 128, element count a multiple of 4):
+// the tensor is one contiguous run whose groups never straddle a row; a lane owns four consecutive elements
+// (one 16-byte load, one 16- or 8-byte store) and a group is a run inside one lane or several neighbouring
+// lanes whose |x| sums meet in an xor-shuffle tree.
 // General kernel (any beta >= 1, any K, padded rows): one thread per (row, group), two passes over the group.
 #include <cstdint>
 #include <cuda_bf16.h>
@@ -30,13 +30,15 @@ __device__ __forceinline__ uint32_t bf16_pair(float lo, float hi) {
   const __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&p);
 }
-__device__ __forceinline__ void store_run(__nv_bfloat16* out, int64_t i, const float (&o)[8]) {
-  reinterpret_cast<uint4*>(out)[i] = make_uint4(bf16_pair(o[0], o[1]), bf16_pair(o[2], o[3]), bf16_pair(o[4], o[5]), bf16_pair(o[6], o[7]));
+__device__ __forceinline__ void store_run(__nv_bfloat16* out, int64_t i, const float (&o)[4]) {
+  reinterpret_cast<uint2*>(out)[i] = make_uint2(bf16_pair(o[0], o[1]), bf16_pair(o[2], o[3]));
 }
 __device__ __forceinline__ void store1(float* out, int64_t i, float v) { out[i] = v; }
 __device__ __forceinline__ void store1(__nv_bfloat16* out, int64_t i, float v) { out[i] = __float2bfloat16_rn(v); }
 
-// E = elements per lane: 4 for fp32 output, 8 for bf16 output (so that every store is 16 bytes wide).
+// E = consecutive elements per lane.  Four, for either output type: a warp's 16-byte loads then cover one
+// contiguous 512-byte run.  (Eight per lane, which makes the bf16 store 16 bytes wide too, leaves every load
+// instruction touching half of each 32-byte sector and measured 13 % slower.)
 template <int BETA, int E, typename OUT>
 __global__ void __launch_bounds__(kThreads)
 binarize_dense_stream(const float4* __restrict__ x, OUT* __restrict__ out, int64_t n_items) {
@@ -99,7 +101,7 @@ binarize_dense_general(const float* __restrict__ x, int64_t ldx, int64_t rows, i
 template <typename OUT>
 cudaError_t launch_typed(const float* x, int64_t ldx, int64_t rows, int64_t K, int64_t beff, OUT* out, int64_t ldo, int sms,
                          cudaStream_t stream) {
-  constexpr int E = sizeof(OUT) == 2 ? 8 : 4;            // elements per lane: 16-byte stores
+  constexpr int E = 4;                                   // elements per lane
   const bool aligned = reinterpret_cast<uintptr_t>(x) % 16 == 0 && reinterpret_cast<uintptr_t>(out) % 16 == 0;
   const bool pow2 = (beff & (beff - 1)) == 0;
   const int64_t cap = static_cast<int64_t>(sms) * 32;
