@@ -163,3 +163,32 @@ def test_subword_groups_on_the_conv3_matrix_sampled_rows(hb, ba, bw):
     c_ref, absref = oracle.hbmm_from_quantized(sa_gpu, sa, ba, sw_gpu, sw, bw)
     floor = gu.FOLDED_FLOOR_ULPS * gu.U * gu.elementwise_magnitude(sa_gpu, ba, sw_gpu, bw, K)
     gu.assert_close_rel_absref(C[rows_d].cpu().numpy(), c_ref, absref, RTOL, "conv3 matrix beta %d/%d" % (ba, bw), floor)
+
+
+# ------------------------------------------------------------------ Eq. 3 grouping (along map rows) at the benchmark's sizes
+@pytest.mark.parametrize("li,beta_a", [(0, 8), (2, 2), (3, 4)])
+def test_resnet_conv_of_map_binarized_activations_full_batch(hb, li, beta_a):
+    """hbmm_binarize_dense on the whole batch-64 map (bf16 out), then the HBWN convolution; the oracle redoes
+    three whole images.  conv5_x with beta_a = 4: lines of 7, a tail run of 3 in every line."""
+    gu = _gu()
+    s = inputs.resnet18_convs(64)[li]
+    x = inputs.conv_activation(s, inputs.SEEDS["resnet_hbwn"][0] + 40 + li, signed=True)
+    w = inputs.he_normal(s.N, s.K, inputs.SEEDS["resnet_hbmm"][1] + li)
+    Wop = hb.quantize(torch.from_numpy(w).cuda(), hb.alloc_operand(s.N, s.K, BETA, hb.F32))
+    geom = hb.make_geom(s.B, s.C, s.H, s.W, s.kh, s.kw, (s.stride, s.stride), (s.pad, s.pad))
+    ws = torch.empty(hb.conv_workspace_bytes(geom, 1, hb.F32, Wop), dtype=torch.uint8, device="cuda")
+    C = torch.empty((s.M, s.N), device="cuda")
+    at = hb.binarize_map(torch.from_numpy(x).cuda(), beta_a, hb.BF16)
+    hb.conv_im2col(at, geom, 1, hb.F32, Wop, C, ws)
+    torch.cuda.synchronize()
+    G = s.K // BETA
+    rtol = 2.0 ** -9 + (BETA + G + 4) * 2 * gu.U + 2.0 ** -18     # A~ rounded to bf16; fp32 sums; two-piece weight scales
+    per_image = s.M // s.B
+    for b in (0, s.B // 2, s.B - 1):
+        a64 = oracle.binarize_map(x[b:b + 1], beta_a)
+        ag = at[b:b + 1].float().cpu().numpy()
+        assert np.array_equal(np.signbit(ag), a64 < 0)
+        assert (np.abs(np.abs(ag) - np.abs(a64)) <= 2.0 ** -8 * np.abs(a64)).all()
+        c_ref, absref = oracle.conv_map_binarized(x[b:b + 1], w, s.kh, s.kw, (s.stride, s.stride), (s.pad, s.pad), beta_a, BETA)
+        lo = b * per_image
+        gu.assert_close_rel_absref(C[lo: lo + per_image].cpu().numpy(), c_ref, absref, rtol, "%s image %d" % (s.name, b))
