@@ -375,6 +375,25 @@ def side_measurements(torch, hbmm, peaks, iters: int):
     ms1 = time_loop(torch, lambda: hbmm.gemm_binarize_next(Af, Wf, nxt, wsf), iters)
     out.append({"kernel": "fc_4096x4096_b256_beta64: hbmm_gemm + hbmm_quantize", "shape": [Mf, Nf, Kf], "ms": round(ms2, 5)})
     out.append({"kernel": "fc_4096x4096_b256_beta64: hbmm_gemm_binarize_next", "shape": [Mf, Nf, Kf], "ms": round(ms1, 5)})
+    # conv2_x with the activations grouped along map rows (Eq. 3 as printed): binarize the map, then the HBWN convolution
+    Bc, Cc, Hc, Nc = 64, 64, 56, 64
+    xm = torch.randn((Bc, Cc, Hc, Hc), device="cuda", generator=g)
+    wc = torch.randn((Nc, Cc * 9), device="cuda", generator=g) * (2.0 / (Cc * 9)) ** 0.5
+    Wc = hbmm.quantize(wc, hbmm.alloc_operand(Nc, Cc * 9, BETA, hbmm.F32))
+    geom = hbmm.make_geom(Bc, Cc, Hc, Hc, 3, 3, (1, 1), (1, 1))
+    wsc = torch.empty(hbmm.conv_workspace_bytes(geom, 1, hbmm.F32, Wc), dtype=torch.uint8, device="cuda")
+    Cc_out = torch.empty((Bc * Hc * Hc, Nc), device="cuda")
+    am = torch.empty((Bc * Cc * Hc, Hc), device="cuda", dtype=torch.bfloat16)
+
+    def eq3_conv(flags):
+        hbmm.binarize_dense(xm.view(Bc * Cc * Hc, Hc), 8, hbmm.BF16, am)
+        hbmm.conv_im2col(am.view(Bc, Cc, Hc, Hc), geom, 1, hbmm.F32, Wc, Cc_out, wsc, flags=flags)
+
+    eq3_conv(0)
+    ms3 = time_loop(torch, lambda: eq3_conv(hbmm.CONV_WEIGHTS_PREPARED), iters)
+    ach = 2.0 * Bc * Hc * Hc * Nc * Cc * 9 / (ms3 * 1e-3) / 1e12
+    out.append({"kernel": "conv2_x_eq3_grouping_beta_a8: hbmm_binarize_dense + hbmm_conv_im2col(beta_a=1)", "shape": [Bc * Hc * Hc, Nc, Cc * 9],
+                "ms": round(ms3, 5), "bound": "tensor", "achieved": ach, "peak": bf16_tflops, "unit": "TFLOP/s", "frac": ach / bf16_tflops})
     return out
 
 
