@@ -617,6 +617,9 @@ def run_ours(args):
     barrier()
     ms_e2e = max_over_ranks(e0.elapsed_time(e1) / args.steps, world, device)
     clocks = sampler.stop(t0, t1, time.time())
+    err = hbmm.last_device_error()
+    if err != 0:
+        raise RuntimeError("a kernel reported device error %d during the timed steps: the numbers are void" % err)
     h2d = sum(L["x_host"].numel() * 4 + L["xb_host"].numel() * 2 for L in layers)
     d2h = sum(L["C_host"].numel() * 4 + L["Cb_host"].numel() * 4 for L in layers)
 
