@@ -5,8 +5,10 @@ One step = one pass of the whole path over one synthetic batch: for each of the 
 3x3 convolution shapes at batch 64, the convolution as HBMM (im2col gather + Hadamard
 binarization + packed contraction, beta_a = beta_w = 32, fp32 scales) and the same convolution
 in HBWN mode (bf16 activations x Hadamard-binary weights, beta_w = 32).  Weights are binarized
-once outside the timed region.  The metric is effective binary TOPS = 2*M*N*K summed over the
-eight products / step time.
+once outside the timed region.  The eight calls of a step share no buffer; the timed schedule
+runs the four HBMM calls on one stream and the four HBWN calls on a second one, joined every
+step (the one-stream time is reported beside it).  The metric is effective binary TOPS =
+2*M*N*K summed over the eight products / step time.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
