@@ -70,6 +70,9 @@ typedef enum {
                            the error follows sum_k |A~[m,k]| |W~[n,k]| (a few 2^-24 of it) instead of
                            vanishing where group dots cancel.  What HBMM_PATH_AUTO picks when it has
                            the workspace and the finer grouping has at most 128 elements per group.
+                           Callers that need Eq. 7's exact cancellation inside a group (integer
+                           group dots, error relative to sum_g |dA dW D_g| alone) pass
+                           HBMM_PATH_TENSOR.
                            HBWN: bf16 activations x weights written as TWO bf16 pieces (the group
                            scale to 2^-17 instead of 2^-26; activations carry 2^-9), 128-column
                            tiles; what HBMM_PATH_AUTO picks for dense bf16 activations.              */
@@ -284,7 +287,11 @@ hbmm_status hbmm_conv_im2col_ex(const void *x, int32_t x_dtype, const hbmm_conv_
  * launched (this includes every realistic beta_a == 1 problem, whose bf16 row matrix is large).
  *
  * The first call on each device looks up the array's device address (the device must be
- * current); make that first call outside any stream capture.  All calls on a device share the
+ * current); make that first call outside any stream capture, and at start-up: with CUDA's lazy
+ * module loading it can be the call that brings the array into device memory, so it is the one
+ * call that may synchronise and that can fail for lack of memory (HBMM_ERR_CUDA) when another
+ * allocator has already taken the whole device.  Devices with an index of 64 or more are not
+ * served (HBMM_ERR_CUDA).  All calls on a device share the
  * one array: it keeps whatever the last call left, which is harmless because each call rewrites
  * all of the region it reads (nothing has to start at zero), but two calls whose kernels can
  * overlap on the GPU (different streams, or different host threads on different streams) race
@@ -296,15 +303,49 @@ hbmm_status hbmm_conv_im2col_static(const void *x, int32_t x_dtype, const hbmm_c
                                     float *C_out, int64_t ldc, void *stream);
 
 /*
- * Device-side health word of the tensor-core contractions.  Their kernels never spin without a
- * limit: a wait on a barrier that does not complete in time records a code (1 producer, 2/3/4
- * MMA issue, 5 epilogue, 6 weight loader; 100 + the same codes for the HBWN kernel, 200 + for the
- * packed convolution front end, 300 + for the folded-scale HBMM kernel), makes the
- * kernel drain and return, and leaves the output undefined.
- * This call copies the word back (it synchronises the device) and returns HBMM_ERR_TIMEOUT when
- * it is non-zero, HBMM_OK otherwise.  code: host pointer, may be NULL.
+ * Device-side health word of the kernels that wait on barriers (the tensor-core contractions and the
+ * packed convolution front end).  Their kernels never spin without a limit: a wait that does not
+ * complete within the limit records a code, makes the kernel drain what it has in flight, free its
+ * tensor memory and return, and leaves the output of that launch undefined.  Codes: 1 producer / tile
+ * loader waiting for a free stage, 2 / 3 the MMA issuer waiting for a stage / for an accumulator, 4 the
+ * final drain of the tensor core, 5 epilogue, 6 weight loader, 7 producer waiting for the row factors,
+ * 8 the warps that compute them, 9 the self-test of hbmm_debug_expire_wait; reported as they are for
+ * the e4m3 HBMM kernel, 100 + code for the HBWN kernel, 200 + code for the packed convolution front end
+ * (201 loader, 202-204 compute warps), 300 + code for the folded-scale HBMM kernel.
+ * Lifetime: one word per kernel family and process, holding the FIRST code recorded since it was last
+ * cleared; nothing but hbmm_clear_device_error resets it, so after one expiry every later query reports
+ * HBMM_ERR_TIMEOUT, whichever call it follows, until the word is cleared.
+ * hbmm_last_device_error copies the words back (it synchronises the device) and returns
+ * HBMM_ERR_TIMEOUT when one is non-zero, HBMM_OK otherwise.  code: host pointer, may be NULL.
+ * hbmm_clear_device_error zeroes them (it synchronises too).
  */
 hbmm_status hbmm_last_device_error(int32_t *code);
+hbmm_status hbmm_clear_device_error(void);
+
+/*
+ * Test hooks for the bounded waits; not for production use.  (Section 4 of the paper has no counterpart:
+ * they exist so that the failure path can be exercised without starving a real kernel.)
+ * hbmm_debug_set_wait_limit: number of polls after which a device-side wait gives up, for every kernel
+ * family, on the current device; 0 restores the default (2^20).  Synchronises.  Errors: INVALID_ARG, CUDA.
+ * hbmm_debug_expire_wait: launches one tiny block on `stream` in which a single thread waits, with the
+ * library's bounded wait, on a barrier that nobody will ever arrive at and that guards nothing (no copy and
+ * no tensor-core work is in flight).  The wait runs out after the limit in force, code 309 is recorded and
+ * the kernel returns normally.  Lower the limit first: with the default the launch takes about a second.
+ */
+hbmm_status hbmm_debug_set_wait_limit(uint32_t polls);
+hbmm_status hbmm_debug_expire_wait(void *stream);
+
+/*
+ * Measurement aid: a register-only arithmetic loop that times the issue rate of one unit -- kind 0: 32-bit
+ * population counts (each fed by an XOR, the inner step of Eq. 7's XNOR/popcount form), 1: fp32 additions
+ * (the inner step of the sign-select form of the dense x packed product), 2: fp32 fused multiply-adds.
+ * Launches `blocks` blocks of 1024 threads on `stream`; each thread runs `iters` iterations of eight
+ * independent operations.  *ops (host, may be NULL) receives the operations per launch; the caller times
+ * the launch.  sink: device, at least blocks * 1024 words (the loop's results are never stored in
+ * practice).  Errors: INVALID_ARG, CUDA.
+ */
+hbmm_status hbmm_bench_alu_rate(int32_t kind, int32_t blocks, int32_t iters, uint32_t *sink, int64_t *ops,
+                                void *stream);
 
 /* Static, NUL-terminated description of a status code (host). */
 const char *hbmm_status_string(int32_t status);

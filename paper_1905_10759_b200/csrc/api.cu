@@ -418,16 +418,42 @@ hbmm_status hbmm_conv_im2col_ex(const void* x, int32_t x_dtype, const hbmm_conv_
 hbmm_status hbmm_last_device_error(int32_t* code) {
   int c = 0;
   int c2 = 0;
-  if (read_gemm_umma_error(&c) != cudaSuccess || read_hbwn_umma_error(&c2) != cudaSuccess) return HBMM_ERR_CUDA;
+  if (gemm_umma_health(kHealthRead, &c) != cudaSuccess || hbwn_umma_health(kHealthRead, &c2) != cudaSuccess) return HBMM_ERR_CUDA;
   if (c == 0 && c2 != 0) c = 100 + c2;    // codes of the HBWN kernel are reported as 100 + code
   int c3 = 0;
-  if (read_im2col_tma_error(&c3) != cudaSuccess) return HBMM_ERR_CUDA;
-  if (c == 0 && c3 != 0) c = 200 + c3;    // the packed front end's tile copy: 201
+  if (im2col_tma_health(kHealthRead, &c3) != cudaSuccess) return HBMM_ERR_CUDA;
+  if (c == 0 && c3 != 0) c = 200 + c3;    // the packed front end: 201..204
   int c4 = 0;
-  if (read_gemm_fold_error(&c4) != cudaSuccess) return HBMM_ERR_CUDA;
-  if (c == 0 && c4 != 0) c = 300 + c4;    // the folded-scale HBMM kernel: 301..306
+  if (gemm_fold_health(kHealthRead, &c4) != cudaSuccess) return HBMM_ERR_CUDA;
+  if (c == 0 && c4 != 0) c = 300 + c4;    // the folded-scale HBMM kernel: 301..309
   if (code) *code = c;
   return c == 0 ? HBMM_OK : HBMM_ERR_TIMEOUT;
+}
+
+hbmm_status hbmm_clear_device_error(void) {
+  int unused = 0;
+  if (gemm_umma_health(kHealthClear, &unused) != cudaSuccess || hbwn_umma_health(kHealthClear, &unused) != cudaSuccess ||
+      im2col_tma_health(kHealthClear, &unused) != cudaSuccess || gemm_fold_health(kHealthClear, &unused) != cudaSuccess)
+    return HBMM_ERR_CUDA;
+  return HBMM_OK;
+}
+
+hbmm_status hbmm_debug_set_wait_limit(uint32_t polls) {
+  int v = static_cast<int>(polls);
+  if (polls > 0x7FFFFFFFu) return HBMM_ERR_INVALID_ARG;
+  if (gemm_umma_health(kHealthSetSpinLimit, &v) != cudaSuccess || hbwn_umma_health(kHealthSetSpinLimit, &v) != cudaSuccess ||
+      im2col_tma_health(kHealthSetSpinLimit, &v) != cudaSuccess || gemm_fold_health(kHealthSetSpinLimit, &v) != cudaSuccess)
+    return HBMM_ERR_CUDA;
+  return HBMM_OK;
+}
+
+hbmm_status hbmm_debug_expire_wait(void* stream) {
+  return launch_wait_expiry_selftest(static_cast<cudaStream_t>(stream)) == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
+}
+
+hbmm_status hbmm_bench_alu_rate(int32_t kind, int32_t blocks, int32_t iters, uint32_t* sink, int64_t* ops, void* stream) {
+  if (kind < 0 || kind > 2 || blocks <= 0 || iters <= 0 || !sink) return HBMM_ERR_INVALID_ARG;
+  return launch_alu_rate(kind, blocks, iters, sink, ops, static_cast<cudaStream_t>(stream)) == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
 }
 
 const char* hbmm_status_string(int32_t status) {

@@ -298,6 +298,17 @@ hbmm_fold_kernel(const Args g) {
           bulk_copy_g2s(smem + S::OFF_B + s * S::B_STAGE, src + st * S::B_STAGE, S::B_STAGE, &full[s]);
         }
       }
+      if (!ok || *abort_flag) {
+        // aborted: the copies already issued (at most one per stage) must land before the CTA's shared memory
+        // goes away.  Their barriers also count producer arrivals that may never come, so each wait is a
+        // short bounded one that ignores the abort flag: it ends when the phase completes or after a time
+        // that is long next to a copy.
+        const int64_t pending = gst < STAGES ? gst : STAGES;
+        for (int64_t q = 1; q <= pending; q++) {
+          const int64_t idx = gst - q;
+          mbar_wait_quiet(&full[idx % STAGES], static_cast<uint32_t>((idx / STAGES) & 1), kDrainPolls);
+        }
+      }
     }
     __syncwarp();
   } else if (warp == kMmaWarp) {
@@ -341,8 +352,14 @@ hbmm_fold_kernel(const Args g) {
         __syncwarp();
       }
       if (leader) {
+        // every MMA issued so far has retired before TMEM is released -- also after an abort, so this wait
+        // does not look at the abort flag (the commit arrives once the tensor core is done, whatever the
+        // other warps do)
         umma_commit(drain);
-        mbar_wait(drain, 0, abort_flag, 4);   // every MMA has retired before TMEM is released
+        if (!mbar_wait_quiet(drain, 0, g_spin_limit < kDrainPolls ? kDrainPolls : g_spin_limit)) {
+          atomicCAS(&g_error_word, 0, 4);
+          *abort_flag = 1;
+        }
       }
     }
     __syncwarp();
@@ -451,6 +468,25 @@ hbmm_fold_kernel(const Args g) {
     tc_fence_after();
     tmem_dealloc(tmem_base, S::TMEM_COLS);
   }
+}
+
+// Test only: thread 0 waits, with the bounded wait every role of the kernel above uses, on a barrier that
+// nobody arrives at and that guards nothing (no copy, no MMA in flight).  The wait runs out after the
+// limit in force, records code 9 and raises the abort flag, which the other threads then see.
+__global__ void wait_expiry_selftest_kernel(int* saw_abort) {
+  __shared__ uint64_t bar;
+  __shared__ int flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  volatile int* abort_flag = &flag;
+  bool done = true;
+  if (threadIdx.x == 0) done = mbar_wait(&bar, 0, abort_flag, 9);
+  __syncthreads();
+  if (threadIdx.x == 1 && saw_abort) *saw_abort = (*abort_flag != 0 && done) ? 1 : 0;
 }
 
 Args make_args(const PackedView& A, const PackedView& W, float* C, int64_t ldc) {
@@ -570,8 +606,18 @@ void gemm_fold_prep_job(const PackedView& A, const PackedView& W, void* workspac
   job->out_down = reinterpret_cast<float*>(job->out + (job->tn == 64 ? stage_bytes<64>(job->f) : stage_bytes<128>(job->f)));
 }
 
-cudaError_t read_gemm_fold_error(int* code) {
-  return cudaMemcpyFromSymbol(code, umma::g_error_word, sizeof(int));
+cudaError_t launch_wait_expiry_selftest(cudaStream_t stream) {
+  wait_expiry_selftest_kernel<<<1, 32, 0, stream>>>(nullptr);
+  return cudaGetLastError();
+}
+
+cudaError_t gemm_fold_health(int op, int* value) {
+  switch (op) {
+    case kHealthRead: return umma::read_error_word(value);
+    case kHealthClear: return umma::clear_error_word();
+    case kHealthSetSpinLimit: return umma::set_spin_limit(static_cast<uint32_t>(*value));
+    default: return cudaErrorInvalidValue;
+  }
 }
 
 }  // namespace hbmm

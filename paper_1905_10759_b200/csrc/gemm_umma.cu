@@ -178,6 +178,16 @@ hbmm_umma_kernel(const Args g) {
           bulk_copy_g2s(smem + S::OFF_B + s * S::B_STAGE, src + st * S::B_STAGE, S::B_STAGE, &full[s]);
         }
       }
+      if (!ok || *abort_flag) {
+        // aborted: the copies already issued (at most one per stage) must land before the CTA's shared memory
+        // goes away.  Their barriers also count producer arrivals that may never come, so each wait is a
+        // short bounded one that ignores the abort flag.
+        const int64_t pending = gst < STAGES ? gst : STAGES;
+        for (int64_t q = 1; q <= pending; q++) {
+          const int64_t idx = gst - q;
+          mbar_wait_quiet(&full[idx % STAGES], static_cast<uint32_t>((idx / STAGES) & 1), kDrainPolls);
+        }
+      }
     }
     __syncwarp();
   } else if (warp == kMmaWarp) {
@@ -230,8 +240,13 @@ hbmm_umma_kernel(const Args g) {
           if (++s == STAGES) { s = 0; full_par ^= 1; }
         }
       }
+      // every MMA issued so far has retired before TMEM is released -- also after an abort, so this wait does
+      // not look at the abort flag
       umma_commit(drain);
-      mbar_wait(drain, 0, abort_flag, 4);   // every MMA has retired before TMEM is released
+      if (!mbar_wait_quiet(drain, 0, g_spin_limit < kDrainPolls ? kDrainPolls : g_spin_limit)) {
+        atomicCAS(&g_error_word, 0, 4);
+        *abort_flag = 1;
+      }
     }
     __syncwarp();
   } else if (warp < kEpilogueWarps) {
@@ -402,8 +417,13 @@ void gemm_tensor_prep_job(const PackedView& A, const PackedView& W, void* worksp
   job->tiles_n = static_cast<int32_t>((job->g.N + job->tn - 1) / job->tn);
 }
 
-cudaError_t read_gemm_umma_error(int* code) {
-  return cudaMemcpyFromSymbol(code, umma::g_error_word, sizeof(int));
+cudaError_t gemm_umma_health(int op, int* value) {
+  switch (op) {
+    case kHealthRead: return umma::read_error_word(value);
+    case kHealthClear: return umma::clear_error_word();
+    case kHealthSetSpinLimit: return umma::set_spin_limit(static_cast<uint32_t>(*value));
+    default: return cudaErrorInvalidValue;
+  }
 }
 
 }  // namespace hbmm

@@ -220,6 +220,7 @@ hbwn_umma_kernel(const Args g, const __grid_constant__ CUtensorMap a_map) {
       // ring slot and round, K block -> (filter tap row, column, channel block).
       int s = 0;
       uint32_t round = 0;
+      int64_t issued = 0;                                       // stages handed to the copy engine so far
       bool ok = true;
       if (RES && my_tiles > 0) {
         // one column tile: its weight pieces are the same for every row tile of this CTA
@@ -253,8 +254,19 @@ hbwn_umma_kernel(const Args g, const __grid_constant__ CUtensorMap a_map) {
             tma_load_2d(smem + S::OFF_A + s * S::A_STAGE, &a_map, kb * KB, static_cast<int32_t>(m0), &full[s]);
           if (!RES) bulk_copy_g2s(smem + off_b + s * S::B_STAGE, src, S::B_STAGE, &full[s]);
           src += S::B_STAGE;
+          issued++;
           if (++cb == g.cblocks) { cb = 0; if (++fj == g.kw) { fj = 0; fi++; } }
           if (++s == STAGES) { s = 0; round++; }
+        }
+      }
+      if (!ok || *abort_flag) {
+        // aborted: the copies already issued must land before the CTA's shared memory goes away (their
+        // barriers count nothing but this thread's arrival and the bytes, so each wait ends with its copy)
+        if (RES && my_tiles > 0) mbar_wait_quiet(wfull, 0, kDrainPolls);
+        const int64_t pending = issued < STAGES ? issued : STAGES;
+        for (int64_t q = 1; q <= pending; q++) {
+          const int64_t idx = issued - q;
+          mbar_wait_quiet(&full[idx % STAGES], static_cast<uint32_t>((idx / STAGES) & 1), kDrainPolls);
         }
       }
     }
@@ -290,8 +302,13 @@ hbwn_umma_kernel(const Args g, const __grid_constant__ CUtensorMap a_map) {
         }
         if (ok) umma_commit_a(tfull_a + buf * 8);
       }
+      // every MMA issued so far has retired before TMEM is released -- also after an abort, so this wait does
+      // not look at the abort flag
       umma_commit(drain);
-      mbar_wait(drain, 0, abort_flag, 4);
+      if (!mbar_wait_quiet(drain, 0, g_spin_limit < kDrainPolls ? kDrainPolls : g_spin_limit)) {
+        atomicCAS(&g_error_word, 0, 4);
+        *abort_flag = 1;
+      }
     }
     __syncwarp();
   } else if (warp < 4) {
@@ -512,8 +529,13 @@ cudaError_t launch_hbwn_umma_conv(const void* x, int x_bf16, void* x_nhwc, int C
   return launch_any(g, a_map, workspace, stream, &cp, w_prepared, false);
 }
 
-cudaError_t read_hbwn_umma_error(int* code) {
-  return cudaMemcpyFromSymbol(code, umma::g_error_word, sizeof(int));
+cudaError_t hbwn_umma_health(int op, int* value) {
+  switch (op) {
+    case kHealthRead: return umma::read_error_word(value);
+    case kHealthClear: return umma::clear_error_word();
+    case kHealthSetSpinLimit: return umma::set_spin_limit(static_cast<uint32_t>(*value));
+    default: return cudaErrorInvalidValue;
+  }
 }
 
 }  // namespace hbmm

@@ -390,11 +390,11 @@ cudaError_t launch_im2col_quantize(const void* x, int x_bf16, const ConvGeom& g,
                         2 * static_cast<size_t>(tp.RB) * g.Wo * (tp.chunks_per_split * taps + 1) * 4 +
                         static_cast<size_t>(kTileCC) * taps * 2 + 16;
     if (smem <= 160 * 1024 && static_cast<int64_t>(kTileCC) * tp.rows_in * tp.span < 65536) {
-      static size_t configured = 0;
-      if (smem > 48 * 1024 && smem > configured) {
+      static DeviceOnce configured;            // the opt-in shared-memory size is a per-device attribute
+      if (smem > 48 * 1024 && configured.pending(dev)) {
         if (cudaFuncSetAttribute(im2col_quantize_tiled_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  160 * 1024) != cudaSuccess) return cudaGetLastError();
-        configured = 160 * 1024;
+        configured.mark(dev);
       }
       dim3 grid(static_cast<unsigned>(static_cast<int64_t>(g.B) * tp.yo_blocks), static_cast<unsigned>(tp.splits));
       im2col_quantize_tiled_kernel<<<grid, 256, smem, stream>>>(x, x_bf16, g, tp, K, G, (K + 31) / 32, bits, ld_words,

@@ -168,8 +168,7 @@ im2col_quantize_tma_kernel(const __grid_constant__ CUtensorMap x_map, const floa
         const int pending = issued < ring ? issued : ring;
         for (int q = 0; q < pending; q++) {
           const int idx = issued - 1 - q, slot = idx % ring;
-          for (uint32_t spin = 0; spin < kSpinLimit; spin++)
-            if (mbar_try_wait(&full[slot], static_cast<uint32_t>((idx / ring) & 1))) break;
+          mbar_wait_quiet(&full[slot], static_cast<uint32_t>((idx / ring) & 1), kDrainPolls);
         }
       }
     }
@@ -350,10 +349,12 @@ int tma_mode(const void* x, int x_bf16, const ConvGeom& g, int32_t beta) {
   if (x_bf16 || beta != 32 || beta >= K || g.sw != 1 || reinterpret_cast<uintptr_t>(x) % 16 != 0) return 0;
   Plan p;
   size_t smem;
-  if (g.W % 4 == 0 && encode_tiled_fn() != nullptr && make_plan(g, 148, false, &p, &smem)) return 1;
+  int dev = 0, sms = 0;
+  if (current_device(&dev, &sms) != cudaSuccess) return 0;       // the plan's channel split follows the device's SM count
+  if (g.W % 4 == 0 && encode_tiled_fn() != nullptr && make_plan(g, sms, false, &p, &smem)) return 1;
   // small images whose rows are not multiples of 16 bytes: whole planes, masked 3x3 / 1x1 gather
   const bool filt = (g.kh == 3 && g.kw == 3) || (g.kh == 1 && g.kw == 1);
-  if (filt && g.C % kCC == 0 && (static_cast<int64_t>(g.C) * g.H * g.W) % 4 == 0 && make_plan(g, 148, true, &p, &smem)) return 2;
+  if (filt && g.C % kCC == 0 && (static_cast<int64_t>(g.C) * g.H * g.W) % 4 == 0 && make_plan(g, sms, true, &p, &smem)) return 2;
   return 0;
 }
 
@@ -407,8 +408,13 @@ cudaError_t launch_im2col_quantize_tma(const void* x, const ConvGeom& g, uint32_
                     job, n_prep, static_cast<int>(n_items), p.ring, bits, ld_words, scales, ld_scales, scale_bf16);
 }
 
-cudaError_t read_im2col_tma_error(int* code) {
-  return cudaMemcpyFromSymbol(code, umma::g_error_word, sizeof(int));
+cudaError_t im2col_tma_health(int op, int* value) {
+  switch (op) {
+    case kHealthRead: return umma::read_error_word(value);
+    case kHealthClear: return umma::clear_error_word();
+    case kHealthSetSpinLimit: return umma::set_spin_limit(static_cast<uint32_t>(*value));
+    default: return cudaErrorInvalidValue;
+  }
 }
 
 }  // namespace hbmm

@@ -128,10 +128,12 @@ struct UmmaPrepJob {
 };
 
 // Packed x packed contraction with +-1 e4m3 operands on the tensor cores (tcgen05 / TMEM).
-// read_*_umma_error copies a kernel family's device-side error word (0 = no bounded wait ever
-// expired); it synchronises.
-cudaError_t read_gemm_umma_error(int* code);
-cudaError_t read_hbwn_umma_error(int* code);
+// *_health: the device-side error word of a kernel family (0 = no bounded wait has expired since it was
+// last cleared) and the poll limit of its waits.  Read copies the word to *value, Clear zeroes it,
+// SetSpinLimit stores *value polls (0 = the default).  All three synchronise with the device.
+enum HealthOp { kHealthRead = 0, kHealthClear = 1, kHealthSetSpinLimit = 2 };
+cudaError_t gemm_umma_health(int op, int* value);
+cudaError_t hbwn_umma_health(int op, int* value);
 bool gemm_tensor_supported(const PackedView& A, const PackedView& W);
 size_t gemm_tensor_workspace_bytes(const PackedView& A, const PackedView& W);
 // w_prepared: the workspace already holds the expanded weight operand of exactly these operands (a
@@ -142,7 +144,9 @@ void gemm_tensor_prep_job(const PackedView& A, const PackedView& W, void* worksp
 
 // Packed x packed contraction with the group scales folded into two fp16 pieces per operand (tcgen05 /
 // TMEM, one accumulation over all of K, no per-group step).  Same operand support as the e4m3 kernel.
-cudaError_t read_gemm_fold_error(int* code);
+cudaError_t gemm_fold_health(int op, int* value);
+// Test only: one thread waits on a barrier nobody arrives at, with the family's bounded wait (code 9).
+cudaError_t launch_wait_expiry_selftest(cudaStream_t stream);
 bool gemm_fold_supported(const PackedView& A, const PackedView& W);
 size_t gemm_fold_workspace_bytes(const PackedView& A, const PackedView& W);
 cudaError_t launch_gemm_fold(const PackedView& A, const PackedView& W, float* C, int64_t ldc, void* workspace,
@@ -184,7 +188,12 @@ bool im2col_quantize_tma_supported(const void* x, int x_bf16, const ConvGeom& g,
 // prep (optional): weight-expansion tasks of the contraction that follows, run by extra CTAs of the launch.
 cudaError_t launch_im2col_quantize_tma(const void* x, const ConvGeom& g, uint32_t* bits, int64_t ld_words, void* scales,
                                        int64_t ld_scales, int scale_bf16, cudaStream_t stream, const UmmaPrepJob* prep = nullptr);
-cudaError_t read_im2col_tma_error(int* code);
+cudaError_t im2col_tma_health(int op, int* value);
+// Register-only arithmetic loop for measuring a unit's issue rate (kind 0: XOR + POPC, 1: fp32 add, 2: fp32
+// fused multiply-add): blocks x 1024 threads, iters x 8 operations each; *ops = operations per launch.
+// sink: device, at least blocks * 1024 words (never written in practice).
+cudaError_t launch_alu_rate(int kind, int blocks, int iters, uint32_t* sink, int64_t* ops, cudaStream_t stream);
+
 cudaError_t launch_im2col_bf16(const void* x, int x_bf16, const ConvGeom& g, void* out, int64_t ld,
                                cudaStream_t stream);
 

@@ -8,8 +8,12 @@
 namespace hbmm {
 namespace umma {
 
-static __device__ int g_error_word = 0;    // 0 = ok; otherwise the code of the first wait that gave up
+static __device__ int g_error_word = 0;    // 0 = ok; otherwise the code of the first wait that gave up (kept until cleared)
 constexpr uint32_t kSpinLimit = 1u << 20;   // polls of a (hardware time-limited) try_wait
+static __device__ uint32_t g_spin_limit = kSpinLimit;   // the limit in force: the default unless a test lowered it
+// Teardown waits -- for asynchronous work that has already been issued and only needs to land -- ignore the
+// abort flag and use this many polls: far longer than a copy or an MMA batch takes, short next to kSpinLimit.
+constexpr uint32_t kDrainPolls = 1u << 14;
 constexpr int TM = 128;                     // rows of every UMMA tile (= TMEM lanes)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
@@ -39,12 +43,21 @@ __device__ __forceinline__ void umma_commit_a(uint32_t bar) {
 }
 // Bounded wait.  Returns false when the limit expired or another thread aborted.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int code) {
-  for (uint32_t it = 0; it < kSpinLimit; it++) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint32_t limit = g_spin_limit;             // read on the slow path only
+  for (uint32_t it = 0; it < limit; it++) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
   }
   atomicCAS(&g_error_word, 0, code);
   *abort_flag = 1;
+  return false;
+}
+// Bounded wait that does not look at the abort flag and records nothing: used on the way out, where work
+// already handed to the copy engine or the tensor core must finish before shared or tensor memory goes away.
+__device__ __forceinline__ bool mbar_wait_quiet(uint64_t* bar, uint32_t parity, uint32_t polls) {
+  for (uint32_t it = 0; it < polls; it++)
+    if (mbar_try_wait(bar, parity)) return true;
   return false;
 }
 
@@ -85,7 +98,8 @@ __device__ __forceinline__ void tma_load_im2col_4d(void* dst, const void* tensor
 // ---- tcgen05 helpers
 __device__ __forceinline__ bool mbar_wait_a(uint32_t bar, uint32_t parity, volatile int* abort_flag, int code) {
   if (mbar_try_wait_a(bar, parity)) return true;
-  for (uint32_t it = 0; it < kSpinLimit; it++) {
+  const uint32_t limit = g_spin_limit;
+  for (uint32_t it = 0; it < limit; it++) {
     if (mbar_try_wait_a(bar, parity)) return true;
     if (*abort_flag) return false;
   }
@@ -199,6 +213,17 @@ __host__ __device__ constexpr uint32_t instr_desc(int n, uint32_t ab_format) {
 constexpr uint32_t kFmtE4M3 = 0, kFmtBF16 = 1;   // kind::f8f6f4 / kind::f16 operand codes
 constexpr uint32_t kFmtF16 = 0;                  // kind::f16 with fp16 operands
 
+// Host side of this translation unit's health word and spin limit (each file that includes this header has
+// its own copies, hence internal linkage).  All three synchronise with the device.
+static inline cudaError_t read_error_word(int* code) { return cudaMemcpyFromSymbol(code, g_error_word, sizeof(int)); }
+static inline cudaError_t clear_error_word() {
+  const int zero = 0;
+  return cudaMemcpyToSymbol(g_error_word, &zero, sizeof(int));
+}
+static inline cudaError_t set_spin_limit(uint32_t polls) {     // 0 restores the default
+  const uint32_t v = polls == 0 ? kSpinLimit : polls;
+  return cudaMemcpyToSymbol(g_spin_limit, &v, sizeof(uint32_t));
+}
 
 }  // namespace umma
 }  // namespace hbmm

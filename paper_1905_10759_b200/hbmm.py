@@ -33,6 +33,7 @@ EXPORTS = [
     "hbmm_gemm_partials", "hbmm_conv_workspace_bytes", "hbmm_conv_im2col", "hbmm_status_string",
     "hbmm_version", "hbmm_conv_im2col_static", "hbmm_last_device_error", "hbmm_conv_im2col_ex",
     "hbmm_binarize_backward", "hbmm_gemm_binarize_next", "hbmm_binarize_dense",
+    "hbmm_clear_device_error", "hbmm_debug_set_wait_limit", "hbmm_debug_expire_wait", "hbmm_bench_alu_rate",
 ]
 STATIC_SCRATCH_BYTES = 32 << 20
 
@@ -320,3 +321,40 @@ def last_device_error() -> int:
     if st not in (OK, ERR_TIMEOUT):
         raise HbmmError(st, "hbmm_last_device_error")
     return int(code.value)
+
+
+_lib.hbmm_clear_device_error.argtypes = []
+_lib.hbmm_clear_device_error.restype = _i32
+_lib.hbmm_debug_set_wait_limit.argtypes = [ctypes.c_uint32]
+_lib.hbmm_debug_set_wait_limit.restype = _i32
+_lib.hbmm_debug_expire_wait.argtypes = [_vp]
+_lib.hbmm_debug_expire_wait.restype = _i32
+_lib.hbmm_bench_alu_rate.argtypes = [_i32, _i32, _i32, _vp, _P(_i64), _vp]
+_lib.hbmm_bench_alu_rate.restype = _i32
+
+
+def clear_device_error() -> None:
+    """hbmm_clear_device_error: zero the device-side health words (synchronises)."""
+    _check(_lib.hbmm_clear_device_error(), "hbmm_clear_device_error")
+
+
+def debug_set_wait_limit(polls: int) -> None:
+    """hbmm_debug_set_wait_limit: polls before a device-side wait gives up; 0 restores the default."""
+    _check(_lib.hbmm_debug_set_wait_limit(polls), "hbmm_debug_set_wait_limit")
+
+
+def debug_expire_wait(stream=None) -> None:
+    """hbmm_debug_expire_wait: one thread waits on a barrier nobody arrives at until the limit runs out."""
+    _check(_lib.hbmm_debug_expire_wait(_stream(stream)), "hbmm_debug_expire_wait")
+
+
+ALU_POPC, ALU_FADD, ALU_FFMA = 0, 1, 2
+
+
+def bench_alu_rate(kind: int, blocks: int, iters: int, sink: torch.Tensor, stream=None) -> int:
+    """hbmm_bench_alu_rate: enqueue the register-only loop; returns the operations one launch performs."""
+    if sink.numel() * sink.element_size() < blocks * 1024 * 4:
+        raise ValueError("sink too small")
+    ops = _i64(0)
+    _check(_lib.hbmm_bench_alu_rate(kind, blocks, iters, _dev_ptr(sink), ctypes.byref(ops), _stream(stream)), "hbmm_bench_alu_rate")
+    return int(ops.value)

@@ -1,6 +1,8 @@
 """GPU parity at full workload sizes, in the launch configuration the benchmark times: the library runs
 the whole problem, the CPU oracle recomputes sampled output rows one by one from the same seeded
 inputs (whole images for the convolutions, scattered rows for the matrix products)."""
+import functools
+
 import numpy as np
 import pytest
 import torch
@@ -90,11 +92,20 @@ def test_resnet_conv_hbwn_full_batch(hb, li):
 
 
 # ------------------------------------------------------------------ square products and the FC stack
-@pytest.mark.parametrize("n,beta,sdt", [(4096, 32, 0), (4096, 128, 1), (8192, 64, 0)])
+@functools.lru_cache(maxsize=1)
+def _square_inputs(n):
+    """Raw inputs of one square size, shared by its six (group size, scale storage) combinations."""
+    return (inputs.normal((n, n), inputs.SEEDS["square_sweep"][0] + n // 4096),
+            inputs.normal((n, n), inputs.SEEDS["square_sweep"][1] + n // 4096))
+
+
+# the whole sweep of the square configuration: two sizes x three group sizes x two scale storage types
+@pytest.mark.parametrize("sdt", [0, 1], ids=["f32scales", "bf16scales"])
+@pytest.mark.parametrize("beta", [32, 64, 128])
+@pytest.mark.parametrize("n", [4096, 8192])
 def test_square_quantize_then_gemm_sampled_rows(hb, n, beta, sdt):
     gu = _gu()
-    a = inputs.normal((n, n), inputs.SEEDS["square_sweep"][0] + n // 4096)
-    w = inputs.normal((n, n), inputs.SEEDS["square_sweep"][1] + n // 4096)
+    a, w = _square_inputs(n)
     A = hb.quantize(torch.from_numpy(a).cuda(), hb.alloc_operand(n, n, beta, sdt))
     W = hb.quantize(torch.from_numpy(w).cuda(), hb.alloc_operand(n, n, beta, sdt))
     C = torch.empty((n, n), device="cuda")
@@ -161,8 +172,8 @@ def test_subword_groups_on_the_conv3_matrix_sampled_rows(hb, ba, bw):
     sw_gpu = W.scales[:, : K // bw].float().cpu().numpy().astype(np.float64)
     assert np.all(np.abs(sa_gpu - da) <= 8 * gu.U * da + 1e-30) and np.all(np.abs(sw_gpu - dw) <= 8 * gu.U * dw + 1e-30)
     c_ref, absref = oracle.hbmm_from_quantized(sa_gpu, sa, ba, sw_gpu, sw, bw)
-    floor = gu.FOLDED_FLOOR_ULPS * gu.U * gu.elementwise_magnitude(sa_gpu, ba, sw_gpu, bw, K)
-    gu.assert_close_rel_absref(C[rows_d].cpu().numpy(), c_ref, absref, RTOL, "conv3 matrix beta %d/%d" % (ba, bw), floor)
+    # no absolute floor: at this size no output's group dots all cancel, so 1e-5 R alone must hold
+    gu.assert_close_rel_absref(C[rows_d].cpu().numpy(), c_ref, absref, RTOL, "conv3 matrix beta %d/%d" % (ba, bw))
 
 
 # ------------------------------------------------------------------ Eq. 3 grouping (along map rows) at the benchmark's sizes

@@ -38,8 +38,29 @@ def test_static_scratch_matches_workspace_entry_point_twice(hb):
     second = inputs.ConvShape("b", 2, 32, 9, 7, 40)          # smaller: sits on top of the first call's leftovers
     for shape, seed, beta in ((first, 31, 32), (second, 47, 64)):
         out, ref = _both(hb, shape, seed, beta)
+        # the same kernels on the same inputs, only the scratch differs: the tolerance of the other GPU tests
+        # (1e-5 relative) holds with room to spare, because the two results are bit-identical
         scale = np.abs(ref).max()
         np.testing.assert_allclose(out, ref, rtol=1e-5, atol=1e-5 * scale)
+        assert np.array_equal(out, ref)
+
+
+def test_static_entry_point_leaves_device_memory_as_it_found_it(hb):
+    """After the first call on a device (which may load the part of the library that holds the array) further
+    calls must not change the amount of free device memory: the entry point allocates and frees nothing."""
+    shape = inputs.ConvShape("c", 2, 64, 12, 12, 48)
+    x = torch.from_numpy(inputs.conv_activation(shape, 53, signed=True)).cuda()
+    W = hb.quantize(torch.from_numpy(inputs.he_normal(shape.N, shape.K, 54)).cuda(), hb.alloc_operand(shape.N, shape.K, 32))
+    geom = hb.make_geom(shape.B, shape.C, shape.H, shape.W, 3, 3, (1, 1), (1, 1))
+    out = torch.empty((shape.M, shape.N), device="cuda")
+    hb.conv_im2col_static(x, geom, 32, hb.F32, W, out)
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    for _ in range(3):
+        hb.conv_im2col_static(x, geom, 32, hb.F32, W, out)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
 
 
 def test_static_scratch_rejects_problems_that_do_not_fit(hb):
