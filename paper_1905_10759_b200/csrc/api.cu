@@ -97,6 +97,12 @@ inline bool workspace_ok(const void* ws, size_t have, size_t need) {
   return need == 0 || (ws != nullptr && have >= need && (reinterpret_cast<uintptr_t>(ws) & 15u) == 0);
 }
 
+// The integer-pipe contraction that fits the operands: matrix-vector shaped, sub-word segments, or tiled.
+cudaError_t popc_any(const PackedView& a, const PackedView& w, float* C, int64_t ldc, cudaStream_t stream) {
+  if (gemv_popc_supported(a, w)) return launch_gemv_popc(a, w, C, ldc, stream);
+  return gemm_subword(a, w) ? launch_gemm_popc_sub(a, w, C, ldc, stream) : launch_gemm_popc(a, w, C, ldc, stream);
+}
+
 hbmm_status gemm_checked(const hbmm_operand* A, const hbmm_operand* W, float* C, int64_t ldc,
                          int32_t path, void* workspace, size_t workspace_bytes, cudaStream_t stream) {
   if (!A || !W) return HBMM_ERR_INVALID_ARG;
@@ -143,7 +149,7 @@ hbmm_status gemm_checked(const hbmm_operand* A, const hbmm_operand* W, float* C,
   const PackedView a = view_of(A), w = view_of(W);
   cudaError_t e;
   switch (path) {
-    case HBMM_PATH_POPC: e = gemm_subword(a, w) ? launch_gemm_popc_sub(a, w, C, ldc, stream) : launch_gemm_popc(a, w, C, ldc, stream); break;
+    case HBMM_PATH_POPC: e = popc_any(a, w, C, ldc, stream); break;
     case HBMM_PATH_B1MMA:
       if (!gemm_b1_supported(a, w)) return HBMM_ERR_UNSUPPORTED;
       e = launch_gemm_b1(a, w, C, ldc, stream);
@@ -159,13 +165,16 @@ hbmm_status gemm_checked(const hbmm_operand* A, const hbmm_operand* W, float* C,
       e = launch_gemm_fold(a, w, C, ldc, workspace, stream, w_prepared);
       break;
     default:
+      // a handful of activation rows: reading the packed weights once beats any tile kernel (and the expanded
+      // weight operand of the tensor-core paths is 32 times larger than the packed one)
+      if (gemv_popc_supported(a, w)) e = launch_gemv_popc(a, w, C, ldc, stream);
       // the tensor-core paths need their workspace; without one the integer-pipe path runs
-      if (prefer_fold(a, w) && workspace_ok(workspace, workspace_bytes, fold_workspace(a, w)))
+      else if (prefer_fold(a, w) && workspace_ok(workspace, workspace_bytes, fold_workspace(a, w)))
         e = launch_gemm_fold(a, w, C, ldc, workspace, stream);
       else if (gemm_tensor_supported(a, w) && workspace_ok(workspace, workspace_bytes, tensor_workspace(a, w)))
         e = launch_gemm_tensor(a, w, C, ldc, workspace, stream);
       else
-        e = gemm_subword(a, w) ? launch_gemm_popc_sub(a, w, C, ldc, stream) : launch_gemm_popc(a, w, C, ldc, stream);
+        e = popc_any(a, w, C, ldc, stream);
       break;
   }
   return e == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;

@@ -64,6 +64,11 @@ cudaError_t launch_gemm_popc(const PackedView& A, const PackedView& W, float* C,
 cudaError_t launch_partials_popc(const PackedView& A, const PackedView& W, int32_t* D,
                                  cudaStream_t stream);
 
+// The same for at most eight activation rows (batch 1 .. 8 of a fully connected layer): one warp per weight
+// row, bound by reading the packed weights once.  Segments of 32, 64 or 128 elements.
+bool gemv_popc_supported(const PackedView& A, const PackedView& W);
+cudaError_t launch_gemv_popc(const PackedView& A, const PackedView& W, float* C, int64_t ldc, cudaStream_t stream);
+
 // The same for sub-word segments (the finer grouping is 2, 4, 8 or 16 elements): masked popcounts inside a word.
 bool gemm_subword(const PackedView& A, const PackedView& W);
 cudaError_t launch_gemm_popc_sub(const PackedView& A, const PackedView& W, float* C, int64_t ldc, cudaStream_t stream);

@@ -154,6 +154,12 @@ GEMM_CASES = [
     (40, 1000, 4096, 64, 64, 0),     # FC-style ragged N = 1000
     (1, 1000, 4096, 64, 64, 0),      # batch 1
     (3, 5, 31, 32, 32, 0),           # K below one word
+    # at most eight activation rows: the matrix-vector kernel (one warp per weight row)
+    (7, 129, 333, 32, 32, 0),        # ragged K: tail segment of 13 bits
+    (8, 130, 576, 128, 32, 0),       # mixed groups, 576 = 4 * 128 + 64
+    (5, 64, 320, 320, 64, 0),        # one activation group per row
+    (2, 33, 200, 64, 64, 1),         # bf16 scales, tail segment of 8 bits
+    (4, 1000, 9216, 64, 64, 0),      # the first fully connected layer's depth
     # sub-word groups (beta 2 .. 16, Section 5), alone and mixed as in the paper's tables (beta_a <= beta_w)
     (200, 72, 576, 16, 16, 0),
     (130, 140, 1152, 4, 4, 0),
