@@ -34,12 +34,15 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 BETA = 32
-SM_COUNT = 148
-SM_MAX_MHZ = 1965.0
-# Unit counts of one SM (per clock): 16 POPC results, 128 fp32 FMA lanes.
-POPC_PER_CLK_SM = 16
-FMA_PER_CLK_SM = 128
+# Planning figures used only when the arithmetic-rate loops could not be timed (they always are on a GPU):
+# 16 population counts and 128 fp32 additions per clock and multiprocessor.
+PLAN_POPC_PER_CLK_SM = 16
+PLAN_FADD_PER_CLK_SM = 128
 FALLBACK_HBM_GBS = 6650.0
+L2_BYTES = 126e6
+PAPER_CONTEXT = ("paper, Section 4.2 / Fig. 5: xHBNN is approximately 10x faster than a full-precision (32-bit) matrix "
+                 "multiply on square matrices at beta = 16, on an Intel Xeon Gold 6128 CPU (3.40 GHz, 19.25 MB cache); "
+                 "no absolute times are given")
 
 
 # ----------------------------------------------------------------------------- distributed plumbing
@@ -286,35 +289,128 @@ def time_loop(torch, fn, iters: int) -> float:
     return e0.elapsed_time(e1) / iters
 
 
-def kernel_breakdown(torch, hbmm, layers, iters: int):
-    """Per-kernel average launch durations on the bench's own buffers and launch configuration.
-    The packed activation operand of each layer is rebuilt in its workspace by the front end, then
-    the contraction kernel is timed alone through hbmm_gemm_ex on exactly that operand; the front end
-    (with the weight expansion its launch carries) is the rest of the convolution call."""
-    out = {"hbmm_contraction": [], "hbwn_conv": [], "front_end_pack": []}
-    for L in layers:
-        s = L["shape"]
-        PREP = hbmm.CONV_WEIGHTS_PREPARED      # the timed step reuses the expanded weights the warm-up left in the workspaces
-        t_conv = time_loop(torch, lambda: hbmm.conv_im2col(L["x"], L["geom"], BETA, hbmm.F32, L["W"], L["C"], L["ws"], flags=PREP), iters)
-        _, _, lw, ls = hbmm.operand_bytes(s.M, s.K, BETA, hbmm.F32)
-        bits_bytes = (s.M * lw * 4 + 255) // 256 * 256
-        bits = L["ws"][: s.M * lw * 4].view(torch.int32).reshape(s.M, lw)
-        scales = L["ws"][bits_bytes: bits_bytes + s.M * ls * 4].view(torch.float32).reshape(s.M, ls)
-        A = hbmm.wrap_packed(bits, scales, s.K, BETA)
-        gws = torch.empty(max(hbmm.gemm_workspace_bytes(A, L["W"]), 16), dtype=torch.uint8, device=L["C"].device)
-        # the contraction kernel alone: the weight expansion is part of the front end's launch in the
-        # convolution call, so it is left in the workspace once and skipped here
-        hbmm.gemm(A, L["W"], L["C"], gws)
-        t_gemm = time_loop(torch, lambda: hbmm.gemm_ex(A, L["W"], L["C"], hbmm.PATH_FOLDED_PREPARED, gws), iters)
-        out["hbmm_contraction"].append(t_gemm)
-        out["front_end_pack"].append(max(t_conv - t_gemm, 1e-3))
-        # HBWN: one call = NCHW -> NHWC bf16 copy, weight pieces, implicit-GEMM contraction (no im2col matrix)
-        t_convb = time_loop(torch, lambda: hbmm.conv_im2col(L["xb"], L["geom"], 1, hbmm.F32, L["W"], L["Cb"], L["wsb"], flags=PREP), iters)
-        out["hbwn_conv"].append(t_convb)
+def time_rotating(torch, fns, rounds: int) -> float:
+    """Average milliseconds per call of a list of equivalent calls on different buffer sets, walked in turn, so
+    that a call finds none of its operands in L2 (the sets together exceed it)."""
+    for fn in fns:
+        fn()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(rounds):
+        for fn in fns:
+            fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / (rounds * len(fns))
+
+
+def time_graph(torch, fns, rounds: int, replays: int = 5) -> float:
+    """Average milliseconds per call with the calls captured in a CUDA graph (`rounds` passes over `fns`) and
+    the graph replayed: for kernels of a few microseconds, whose back-to-back issue from Python (about 10 us
+    per call) would otherwise be what is timed.  The library enqueues on the capturing stream and neither
+    allocates nor synchronises, so its calls can be captured."""
+    for fn in fns:
+        fn()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for _ in range(rounds):
+            for fn in fns:
+                fn()
+    graph.replay()
+    return time_loop(torch, graph.replay, replays) / (rounds * len(fns))
+
+
+def measure_alu_rates(torch, hbmm, clock_reader):
+    """Issue rates of the units the two ALU rooflines are built on, from the library's register-only loops:
+    32-bit population counts per second and fp32 additions per second over the whole GPU, with the SM clock
+    seen while they ran.  `at_max_clock` scales the measured rate by max clock / observed clock."""
+    props = torch.cuda.get_device_properties(torch.cuda.current_device())
+    sms = props.multi_processor_count
+    blocks = sms * 2                       # two blocks of 1024 threads fill a multiprocessor
+    sink = torch.empty(blocks * 1024, dtype=torch.int32, device="cuda")
+    out = {"sm_count": sms}
+    for name, kind, iters in (("popc", hbmm.ALU_POPC, 1 << 15), ("fadd", hbmm.ALU_FADD, 1 << 17), ("ffma", hbmm.ALU_FFMA, 1 << 17)):
+        ops = hbmm.bench_alu_rate(kind, blocks, iters, sink)          # warm-up
+        for _ in range(2):
+            hbmm.bench_alu_rate(kind, blocks, iters, sink)
+        best = None
+        mhz = []
+        for _ in range(5):
+            ms = time_loop(torch, lambda: hbmm.bench_alu_rate(kind, blocks, iters, sink), 2)
+            best = ms if best is None else min(best, ms)
+            c = clock_reader()
+            if c:
+                mhz.append(c)
+        rate = ops / (best * 1e-3)
+        sm_mhz = statistics.median(mhz) if mhz else None
+        out[name] = {"ops_per_s": rate, "ms_per_launch": best, "ops_per_launch": ops,
+                     "per_clk_per_sm": rate / (sms * sm_mhz * 1e6) if sm_mhz else None, "sm_mhz": sm_mhz}
     return out
 
 
-def side_measurements(torch, hbmm, peaks, iters: int):
+def read_sm_clock(index: int):
+    """(current, max) SM clock in MHz from nvidia-smi, or None."""
+    try:
+        o = subprocess.run(["nvidia-smi", "-i", str(index), "--query-gpu=clocks.sm,clocks.max.sm", "--format=csv,noheader,nounits"],
+                           capture_output=True, text=True, timeout=10).stdout.strip().split(",")
+        return float(o[0]), float(o[1])
+    except Exception:
+        return None
+
+
+def kernel_breakdown(torch, hbmm, layers, rounds: int):
+    """Per-kernel average launch durations in the launch configuration of the step, L2-cold: every call of a
+    family walks a ring of buffer sets (input, workspace, output) that together exceed L2, as in the step,
+    where ~0.7 GB pass between two uses of a buffer.  Three timings per layer: the packed front end alone
+    (hbmm_conv_im2col_ex with HBMM_CONV_PACK_ONLY: gather + binarize + pack), the HBMM contraction alone
+    (hbmm_gemm_ex on the packed operand a front end left in the set's workspace, expanded weights reused),
+    and the whole HBWN convolution call (layout copy + contraction: one call, two launches)."""
+    out = {"hbmm_contraction": [], "hbwn_conv": [], "front_end_pack": [], "hbmm_conv_call": [], "sets": []}
+    PREP = hbmm.CONV_WEIGHTS_PREPARED
+    for L in layers:
+        s = L["shape"]
+        bb, sb, lw, ls = hbmm.operand_bytes(s.M, s.K, BETA, hbmm.F32)
+        x_bytes = L["x"].numel() * 4
+        c_bytes = s.M * s.N * 4
+        per_set = min(x_bytes + bb + sb, bb + sb + c_bytes, L["xb"].numel() * 2 + c_bytes)
+        n_sets = max(2, min(32, int(2 * L2_BYTES / per_set) + 1))
+        xs = [L["x"]] + [L["x"].clone() for _ in range(n_sets - 1)]
+        xbs = [L["xb"]] + [L["xb"].clone() for _ in range(n_sets - 1)]
+        wss = [L["ws"]] + [torch.empty_like(L["ws"]) for _ in range(n_sets - 1)]
+        wsbs = [L["wsb"]] + [torch.empty_like(L["wsb"]) for _ in range(n_sets - 1)]
+        Cs = [L["C"]] + [torch.empty_like(L["C"]) for _ in range(n_sets - 1)]
+        for i in range(n_sets):          # every set's workspace gets its own expanded weights and packed operand
+            hbmm.conv_im2col(xs[i], L["geom"], BETA, hbmm.F32, L["W"], Cs[i], wss[i])
+            hbmm.conv_im2col(xbs[i], L["geom"], 1, hbmm.F32, L["W"], Cs[i], wsbs[i])
+        bits_off = (bb + 255) // 256 * 256
+        ops_pk = []
+        for i in range(n_sets):
+            bits = wss[i][:bb].view(torch.int32).reshape(s.M, lw)
+            scales = wss[i][bits_off: bits_off + sb].view(torch.float32).reshape(s.M, ls)
+            ops_pk.append(hbmm.wrap_packed(bits, scales, s.K, BETA))
+        gws_off = (bits_off + sb + 255) // 256 * 256
+        gws = [wss[i][gws_off:] for i in range(n_sets)]
+        t_front = time_rotating(torch, [
+            (lambda i=i: hbmm.conv_im2col(xs[i], L["geom"], BETA, hbmm.F32, L["W"], None, wss[i], flags=PREP | hbmm.CONV_PACK_ONLY))
+            for i in range(n_sets)], rounds)
+        t_gemm = time_rotating(torch, [
+            (lambda i=i: hbmm.gemm_ex(ops_pk[i], L["W"], Cs[i], hbmm.PATH_FOLDED_PREPARED, gws[i])) for i in range(n_sets)], rounds)
+        t_call = time_rotating(torch, [
+            (lambda i=i: hbmm.conv_im2col(xs[i], L["geom"], BETA, hbmm.F32, L["W"], Cs[i], wss[i], flags=PREP)) for i in range(n_sets)], rounds)
+        t_hbwn = time_rotating(torch, [
+            (lambda i=i: hbmm.conv_im2col(xbs[i], L["geom"], 1, hbmm.F32, L["W"], Cs[i], wsbs[i], flags=PREP)) for i in range(n_sets)], rounds)
+        out["front_end_pack"].append(t_front)
+        out["hbmm_contraction"].append(t_gemm)
+        out["hbmm_conv_call"].append(t_call)
+        out["hbwn_conv"].append(t_hbwn)
+        out["sets"].append(n_sets)
+        del xs, xbs, wss, wsbs, Cs, ops_pk, gws
+    return out
+
+
+def side_measurements(torch, hbmm, inputs, peaks, iters: int):
     """Rows of the hot path that the convolution step only runs in fused form, timed on their own on the
     conv3_x matrix view (M = 50176, K = 1152, N = 128; 231 MB of fp32 input, larger than L2):
     hbmm_quantize alone (HBM bound), the gradient through the binarization (Eq. 6, HBM bound: 8 bytes read
@@ -396,6 +492,36 @@ def side_measurements(torch, hbmm, peaks, iters: int):
     ach = 2.0 * Bc * Hc * Hc * Nc * Cc * 9 / (ms3 * 1e-3) / 1e12
     out.append({"kernel": "conv2_x_eq3_grouping_beta_a8: hbmm_binarize_dense + hbmm_conv_im2col(beta_a=1)", "shape": [Bc * Hc * Hc, Nc, Cc * 9],
                 "ms": round(ms3, 5), "bound": "tensor", "achieved": ach, "peak": bf16_tflops, "unit": "TFLOP/s", "frac": ach / bf16_tflops})
+    del xm, am, Cc_out, amap, a, gy, gx
+    # Exact-scale variants on the four convolution matrices (seeded device-generated operands of the same shapes):
+    # HBMM with integer group dots and a per-group fp32 scale step (HBMM_PATH_TENSOR) beside the default
+    # folded-scale kernel, and HBWN on the dense bf16 im2col matrix with three bf16 weight pieces (scales to 2^-26,
+    # HBMM_PATH_TENSOR) beside two pieces (HBMM_PATH_FOLDED).
+    for sh in inputs.resnet18_convs(64):
+        a = torch.randn((sh.M, sh.K), device="cuda", generator=g)
+        w = torch.randn((sh.N, sh.K), device="cuda", generator=g) * (2.0 / sh.K) ** 0.5
+        A = hbmm.quantize(a, hbmm.alloc_operand(sh.M, sh.K, BETA, hbmm.F32))
+        W = hbmm.quantize(w, hbmm.alloc_operand(sh.N, sh.K, BETA, hbmm.F32))
+        C = torch.empty((sh.M, sh.N), device="cuda")
+        ws = torch.empty(max(hbmm.gemm_workspace_bytes(A, W), 16), dtype=torch.uint8, device="cuda")
+        ops = 2.0 * sh.M * sh.N * sh.K
+        for label, first, again in (("hbmm_umma_kernel (e4m3 operands, per-group fp32 scale step)", hbmm.PATH_TENSOR, hbmm.PATH_TENSOR_PREPARED),
+                                    ("hbmm_fold_kernel (default)", hbmm.PATH_FOLDED, hbmm.PATH_FOLDED_PREPARED),
+                                    ("gemm_popc_kernel (integer pipe, no workspace)", hbmm.PATH_POPC, hbmm.PATH_POPC)):
+            hbmm.gemm_ex(A, W, C, first, ws)
+            ms = time_loop(torch, lambda: hbmm.gemm_ex(A, W, C, again, ws), iters)
+            out.append({"kernel": "%s/%s" % (label, sh.name), "shape": [sh.M, sh.N, sh.K], "ms": round(ms, 5),
+                        "tops": ops / (ms * 1e-3) / 1e12, "timing": "L2-warm loop on one operand set"})
+        Ad = hbmm.wrap_dense(a.to(torch.bfloat16))
+        wsd = torch.empty(max(hbmm.gemm_workspace_bytes(Ad, W), 16), dtype=torch.uint8, device="cuda")
+        for label, first, again in (("hbwn_umma_kernel, three weight pieces (dense bf16 rows)", hbmm.PATH_TENSOR, hbmm.PATH_TENSOR_PREPARED),
+                                    ("hbwn_umma_kernel, two weight pieces (dense bf16 rows)", hbmm.PATH_FOLDED, hbmm.PATH_FOLDED_PREPARED),
+                                    ("hbwn_select_kernel (fp32 sign-select, no workspace)", hbmm.PATH_POPC, hbmm.PATH_POPC)):
+            hbmm.gemm_ex(Ad, W, C, first, wsd)
+            ms = time_loop(torch, lambda: hbmm.gemm_ex(Ad, W, C, again, wsd), iters if first != hbmm.PATH_POPC else max(2, iters // 4))
+            out.append({"kernel": "%s/%s" % (label, sh.name), "shape": [sh.M, sh.N, sh.K], "ms": round(ms, 5),
+                        "tflops": ops / (ms * 1e-3) / 1e12, "timing": "L2-warm loop on one operand set"})
+        del a, A, C, ws, Ad, wsd
     return out
 
 
@@ -403,45 +529,278 @@ def side_measurements(torch, hbmm, peaks, iters: int):
 # (same kernels, same workload); entries are dropped when a kernel changes after its capture.
 NCU_DRAM_BYTES = {
     ("hbmm_contraction", "conv2_x"): 32.373e6 + 2.103e6,     # profiles/hbmm_fold_kernel_conv2_x.md
-    ("front_end_pack", "conv2_x"): 51.511e6 + 2.524e6,       # profiles/im2col_quantize_tma_kernel_conv2_x.md
 }
 
 
-def roofline_for(kind: str, li: int, shape, ms: float, peaks):
+def hbmm_bytes(M, N, K, beta, scale_bytes=4):
+    """Algorithmic bytes of a packed x packed product: both packed operands once, the fp32 result once."""
+    G = -(-K // beta)
+    return M * K / 8.0 + M * G * scale_bytes + N * K / 8.0 + N * G * scale_bytes + 4.0 * M * N
+
+
+def popc_hbm_roofline(M, N, K, beta, scale_bytes, rates, hbm_gbs):
+    """Seconds: the larger of the bytes at the HBM copy bandwidth and one population count per output and
+    K-word at the measured population-count rate (and at that rate scaled to the maximum SM clock)."""
+    t_hbm = hbmm_bytes(M, N, K, beta, scale_bytes) / (hbm_gbs * 1e9)
+    words = M * N * float(-(-K // 32))
+    t_popc = words / rates["popc"]["ops_per_s"]
+    t_popc_max = words / rates["popc"]["ops_per_s_at_max_clock"]
+    return {"t_hbm_us": t_hbm * 1e6, "t_popc_us": t_popc * 1e6, "t_roof_us": max(t_hbm, t_popc) * 1e6,
+            "t_roof_us_at_max_clock": max(t_hbm, t_popc_max) * 1e6, "bound": "hbm" if t_hbm > t_popc else "popc"}
+
+
+def roofline_for(kind: str, li: int, shape, ms: float, peaks, rates):
     """Roofline entry of one kernel launch (layer li) given its measured duration.
 
     Both contractions run on the tensor cores (HBMM: two fp16 pieces per operand carrying sign and group
     scale; HBWN: bf16 activations x two bf16 weight pieces), so they are set against the measured dense
     16-bit GEMM peak.  `achieved` counts the ALGORITHMIC operations 2 M N K; the HBMM kernel issues four
-    times that on the tensor pipe (2 x 2 pieces), the HBWN kernel twice.  For HBMM the fraction of
-    the integer-pipe popcount roofline (one POPC per output and K-word at 16 / clk / SM) is given beside it."""
+    times that on the tensor pipe (2 x 2 pieces), the HBWN kernel twice.  Beside it: the fraction of the
+    popcount / HBM roofline for HBMM (one population count per output and K-word at the MEASURED rate of the
+    integer pipe, or the algorithmic bytes at the HBM copy bandwidth, whichever is slower) and of the fp32-add
+    / HBM roofline for HBWN (one addition per output and K-element at the measured rate)."""
     hbm_gbs, bf16_tflops, hbm_src = peaks
     M, N, K = shape.M, shape.N, shape.K
     G = -(-K // BETA)
     if kind == "hbmm_contraction":
         ops = 2.0 * M * N * K
-        peak = bf16_tflops
-        popc_peak = SM_COUNT * POPC_PER_CLK_SM * SM_MAX_MHZ * 1e6 * 64 / 1e12
         ach = ops / (ms * 1e-3) / 1e12
+        rf = popc_hbm_roofline(M, N, K, BETA, 4, rates, hbm_gbs)
         return {"kernel": "hbmm_fold_kernel/%s" % shape.name, "bound": "tensor", "achieved": ach,
-                "peak": peak, "unit": "TFLOP/s", "frac": ach / peak, "traffic": None,
+                "peak": bf16_tflops, "unit": "TFLOP/s", "frac": ach / bf16_tflops, "traffic": None,
                 "peak_source": "%s bf16 GEMM peak (fp16 operands, same rate)" % hbm_src,
                 "tensor_pipe_work_factor": 4,
-                "frac_of_popcount_roofline": ach / popc_peak, "popcount_roofline_tops": popc_peak}
+                "frac_of_popcount_hbm_roofline": rf["t_roof_us"] / (ms * 1e3),
+                "frac_of_popcount_hbm_roofline_at_max_clock": rf["t_roof_us_at_max_clock"] / (ms * 1e3),
+                "popcount_hbm_roofline": rf, "timing": "L2-cold (ring of buffer sets larger than L2), weights already expanded"}
     if kind == "hbwn_conv":
         # the whole HBWN call (layout copy + weight pieces + contraction) set against the contraction's flops
         ops = 2.0 * M * N * K
         ach = ops / (ms * 1e-3) / 1e12
+        by = 2.0 * shape.B * shape.C * shape.H * shape.W + N * K / 8.0 + 4.0 * N * G + 4.0 * M * N
+        t_roof = max(by / (hbm_gbs * 1e9), M * N * float(K) / rates["fadd"]["ops_per_s"])
         return {"kernel": "hbwn_umma_kernel(im2col tensor copies)/%s" % shape.name, "bound": "tensor", "achieved": ach,
                 "peak": bf16_tflops, "unit": "TFLOP/s", "frac": ach / bf16_tflops, "traffic": None,
-                "peak_source": "%s bf16 GEMM peak" % hbm_src}
+                "peak_source": "%s bf16 GEMM peak" % hbm_src, "tensor_pipe_work_factor": 2,
+                "frac_of_fp32_add_hbm_roofline": t_roof / (ms * 1e-3), "timing": "L2-cold, whole call (layout copy + contraction)"}
     x_bytes = 4.0 * shape.B * shape.C * shape.H * shape.W
     lw = ((K + 31) // 32 + 3) // 4 * 4
     ls = (G + 3) // 4 * 4
     by = x_bytes + M * lw * 4.0 + M * ls * 4.0
+    if kind == "hbmm_conv_call":
+        by += N * K / 8.0 + 4.0 * N * G + 4.0 * M * N - (M * lw * 4.0 + M * ls * 4.0)   # the packed operand is internal to the call
+        rf = popc_hbm_roofline(M, N, K, BETA, 4, rates, hbm_gbs)
+        t_roof = max(by / (hbm_gbs * 1e9), rf["t_popc_us"] * 1e-6)
+        ach = 2.0 * M * N * K / (ms * 1e-3) / 1e12
+        return {"kernel": "hbmm_conv_im2col/%s" % shape.name, "bound": "tensor", "achieved": ach, "peak": bf16_tflops,
+                "unit": "TFLOP/s", "frac": ach / bf16_tflops, "traffic": None,
+                "frac_of_popcount_hbm_roofline": t_roof / (ms * 1e-3), "timing": "L2-cold, whole call (front end + contraction)"}
     return {"kernel": "%s/%s" % (kind, shape.name), "bound": "hbm", "achieved": by / (ms * 1e-3) / 1e9,
             "peak": hbm_gbs, "unit": "GB/s", "frac": by / (ms * 1e-3) / 1e9 / hbm_gbs, "traffic": None,
-            "peak_source": "%s HBM copy bandwidth" % hbm_src}
+            "peak_source": "%s HBM copy bandwidth" % hbm_src, "timing": "L2-cold, front end alone (HBMM_CONV_PACK_ONLY)"}
+
+
+# ----------------------------------------------------------------------------- the five configurations, one by one
+def cublas_context(torch, M, N, K, iters):
+    """torch.matmul of the same shape in fp32 (TF32 off: the analogue of the paper's full-precision multiply)
+    and in bf16, milliseconds per call; library GEMMs, timed for context only."""
+    old = torch.backends.cuda.matmul.allow_tf32
+    torch.backends.cuda.matmul.allow_tf32 = False
+    try:
+        a = torch.randn((M, K), device="cuda")
+        w = torch.randn((N, K), device="cuda")
+        c = torch.empty((M, N), device="cuda")
+        for _ in range(2):
+            torch.matmul(a, w.t(), out=c)
+        ms32 = time_loop(torch, lambda: torch.matmul(a, w.t(), out=c), iters)
+        ab, wb = a.to(torch.bfloat16), w.to(torch.bfloat16)
+        cb = torch.empty((M, N), device="cuda", dtype=torch.bfloat16)
+        for _ in range(2):
+            torch.matmul(ab, wb.t(), out=cb)
+        msb = time_loop(torch, lambda: torch.matmul(ab, wb.t(), out=cb), iters)
+    finally:
+        torch.backends.cuda.matmul.allow_tf32 = old
+    return {"fp32_ms": round(ms32, 5), "bf16_ms": round(msb, 5),
+            "fp32_tflops": 2.0 * M * N * K / (ms32 * 1e-3) / 1e12, "bf16_tflops": 2.0 * M * N * K / (msb * 1e-3) / 1e12}
+
+
+def oracle_row_sample(oracle, a_rows, w, beta_a, beta_w, M, hbwn=False):
+    """The CPU checker as it stands on a row sample of the shape: seconds for the sample and the time for all M
+    rows extrapolated by rows (labelled as such)."""
+    t0 = time.perf_counter()
+    if hbwn:
+        oracle.hbwn(a_rows, w, beta_w, "f32")
+    else:
+        oracle.hbmm(a_rows, w, beta_a, beta_w, "f32")
+    dt = time.perf_counter() - t0
+    r = a_rows.shape[0]
+    return {"sample_rows": r, "sample_s": round(dt, 4), "full_ms_row_extrapolated": dt * 1e3 * M / r, "cores": oracle.num_threads()}
+
+
+def sample_rows_for(M, N, K, budget_macs=1.2e9):
+    return int(max(1, min(M, budget_macs / (float(N) * K))))
+
+
+def product_row(torch, hbmm, name, M, N, K, beta, sdt, a_dev, w_dev, rates, peaks, iters, with_quantize=True):
+    """One packed x packed product of a configuration: hbmm_quantize of the activation matrix alone, hbmm_gemm
+    alone on the packed operands (weights expanded once, outside the timing), against the popcount / HBM
+    roofline.  Products whose operands and result fit L2 are timed over a ring of operand / result sets."""
+    hbm_gbs, bf16_tflops, _ = peaks
+    sb = 4 if sdt == hbmm.F32 else 2
+    W = hbmm.quantize(w_dev, hbmm.alloc_operand(N, K, beta, sdt))
+    row = {"name": name, "M": M, "N": N, "K": K, "beta": beta, "scale_dtype": "f32" if sdt == hbmm.F32 else "bf16"}
+    by = hbmm_bytes(M, N, K, beta, sb)
+    n_sets = max(1, min(16, int(2 * L2_BYTES / by) + 1)) if by < 2 * L2_BYTES else 1
+    As = [hbmm.quantize(a_dev, hbmm.alloc_operand(M, K, beta, sdt)) for _ in range(n_sets)]
+    Cs = [torch.empty((M, (N + 3) // 4 * 4), device="cuda") for _ in range(n_sets)]
+    nws = max(hbmm.gemm_workspace_bytes(As[0], W), 16)
+    wss = [torch.empty(nws, dtype=torch.uint8, device="cuda") for _ in range(n_sets)]
+    gemv = M <= 8
+    if gemv:
+        # a handful of rows: the matrix-vector kernel reads the packed weights; its ring rotates weight copies too
+        Ws = [W] + [hbmm.quantize(w_dev, hbmm.alloc_operand(N, K, beta, sdt)) for _ in range(n_sets - 1)]
+        fns = [(lambda i=i: hbmm.gemm(As[i], Ws[i], Cs[i], wss[i])) for i in range(n_sets)]
+        path = "gemv_popc_kernel"
+    else:
+        for i in range(n_sets):
+            hbmm.gemm(As[i], W, Cs[i], wss[i])                 # leaves the expanded weights in each workspace
+        auto_folded = min(beta, K) <= 128
+        prepared = hbmm.PATH_FOLDED_PREPARED if auto_folded else hbmm.PATH_TENSOR_PREPARED
+        fns = [(lambda i=i: hbmm.gemm_ex(As[i], W, Cs[i], prepared, wss[i])) for i in range(n_sets)]
+        path = "hbmm_fold_kernel" if auto_folded else "hbmm_umma_kernel"
+    small = 2.0 * M * N * K < 4e9                      # a few microseconds of work: time inside a CUDA graph
+    ms = time_graph(torch, fns, max(2, 40 // n_sets)) if small else time_rotating(torch, fns, max(2, iters // n_sets))
+    rf = popc_hbm_roofline(M, N, K, beta, sb, rates, hbm_gbs)
+    row.update({"kernel": path, "hbmm_gemm_ms": round(ms, 5), "tops": 2.0 * M * N * K / (ms * 1e-3) / 1e12,
+                "gbs": by / (ms * 1e-3) / 1e9, "roofline_bound": rf["bound"], "t_roof_us": round(rf["t_roof_us"], 3),
+                "frac_of_popcount_hbm_roofline": rf["t_roof_us"] / (ms * 1e3),
+                "frac_of_popcount_hbm_roofline_at_max_clock": rf["t_roof_us_at_max_clock"] / (ms * 1e3),
+                "frac_of_bf16_tensor_peak": 2.0 * M * N * K / (ms * 1e-3) / 1e12 / bf16_tflops, "buffer_sets": n_sets,
+                "timing": "CUDA graph replay" if small else "stream of launches"})
+    if with_quantize:
+        qs = [hbmm.alloc_operand(M, K, beta, sdt) for _ in range(n_sets)]
+        x_copies = [a_dev] + [a_dev.clone() for _ in range(n_sets - 1)] if 4.0 * M * K < 2 * L2_BYTES else [a_dev] * n_sets
+        qfns = [(lambda i=i: hbmm.quantize(x_copies[i], qs[i])) for i in range(n_sets)]
+        msq = time_graph(torch, qfns, max(2, 40 // n_sets)) if 4.0 * M * K < 64e6 else time_rotating(torch, qfns, max(2, iters // n_sets))
+        G = -(-K // beta)
+        byq = 4.0 * M * K + M * K / 8.0 + M * G * sb
+        row.update({"hbmm_quantize_ms": round(msq, 5), "quantize_gbs": byq / (msq * 1e-3) / 1e9,
+                    "quantize_frac_of_hbm": byq / (msq * 1e-3) / 1e9 / hbm_gbs})
+    return row
+
+
+def config_rows(torch, hbmm, inputs, layers, brk, rates, peaks, iters):
+    """Every configuration of the workload list on its own: the 256-cube, the square sweep (two sizes x three
+    group sizes x two scale storage types), the four convolution shapes as HBMM and as HBWN (from the kernel
+    breakdown), and the fully connected stack at batch 256 and batch 1.  Each row: time, effective binary
+    TOPS, algorithmic GB/s, fraction of its roofline, a library GEMM of the same shape in fp32 and bf16, and
+    the CPU checker on a row sample of the same shape."""
+    import oracle
+    oracle.build()
+    rows = []
+    hbm_gbs, bf16_tflops, _ = peaks
+    # --- 256-cube
+    a = inputs.normal((256, 256), inputs.SEEDS["square256"][0])
+    w = inputs.normal((256, 256), inputs.SEEDS["square256"][1])
+    r = product_row(torch, hbmm, "square256", 256, 256, 256, 32, hbmm.F32, torch.from_numpy(a).cuda(), torch.from_numpy(w).cuda(),
+                    rates, peaks, 200)
+    r["note"] = "0.1 us of roofline time: launch latency decides"
+    r["cublas"] = cublas_context(torch, 256, 256, 256, 100)
+    r["oracle"] = oracle_row_sample(oracle, a, w, 32, 32, 256)
+    rows.append(r)
+    # --- square sweep
+    for n in (4096, 8192):
+        a = inputs.normal((n, n), inputs.SEEDS["square_sweep"][0] + n // 4096)
+        w = inputs.normal((n, n), inputs.SEEDS["square_sweep"][1] + n // 4096)
+        ad, wd = torch.from_numpy(a).cuda(), torch.from_numpy(w).cuda()
+        cub = cublas_context(torch, n, n, n, 5 if n == 4096 else 3)
+        sr = sample_rows_for(n, n, n)
+        orc = {}
+        for beta in (32, 64, 128):
+            orc[beta] = oracle_row_sample(oracle, a[:sr], w, beta, beta, n)
+            for sdt in (hbmm.F32, hbmm.BF16):
+                r = product_row(torch, hbmm, "square%d" % n, n, n, n, beta, sdt, ad, wd, rates, peaks, 10 if n == 4096 else 4)
+                r["cublas"] = cub
+                r["oracle"] = orc[beta]
+                rows.append(r)
+        del ad, wd
+    # --- the convolution shapes, from the breakdown of the timed step's calls
+    for i, L in enumerate(layers):
+        sh = L["shape"]
+        cub = cublas_context(torch, sh.M, sh.N, sh.K, 10)
+        sr = sample_rows_for(sh.M, sh.N, sh.K, 6e8)
+        b = max(1, -(-sr // (sh.M // sh.B)))
+        sub = inputs.ConvShape(sh.name, b, sh.C, sh.H, sh.W, sh.N)
+        xa = oracle.im2col(inputs.conv_activation(sub, inputs.SEEDS["resnet_hbmm"][0] + i), sh.kh, sh.kw, (1, 1), (1, 1))[:sr]
+        wh = inputs.he_normal(sh.N, sh.K, inputs.SEEDS["resnet_hbmm"][1] + i)
+        rf = popc_hbm_roofline(sh.M, sh.N, sh.K, BETA, 4, rates, hbm_gbs)
+        ms = brk["hbmm_contraction"][i]
+        rows.append({"name": "resnet18_%s_hbmm" % sh.name, "M": sh.M, "N": sh.N, "K": sh.K, "beta": BETA, "scale_dtype": "f32",
+                     "kernel": "hbmm_fold_kernel", "hbmm_gemm_ms": round(ms, 5), "tops": 2.0 * sh.M * sh.N * sh.K / (ms * 1e-3) / 1e12,
+                     "gbs": hbmm_bytes(sh.M, sh.N, sh.K, BETA) / (ms * 1e-3) / 1e9, "roofline_bound": rf["bound"],
+                     "t_roof_us": round(rf["t_roof_us"], 3), "frac_of_popcount_hbm_roofline": rf["t_roof_us"] / (ms * 1e3),
+                     "frac_of_popcount_hbm_roofline_at_max_clock": rf["t_roof_us_at_max_clock"] / (ms * 1e3),
+                     "front_end_ms": round(brk["front_end_pack"][i], 5), "conv_call_ms": round(brk["hbmm_conv_call"][i], 5),
+                     "conv_call_frac_of_popcount_hbm_roofline": roofline_for("hbmm_conv_call", i, sh, brk["hbmm_conv_call"][i], peaks, rates)["frac_of_popcount_hbm_roofline"],
+                     "cublas": cub, "oracle": oracle_row_sample(oracle, xa, wh, BETA, BETA, sh.M)})
+        _, xab = inputs.as_bf16(xa)
+        msb = brk["hbwn_conv"][i]
+        rows.append({"name": "resnet18_%s_hbwn" % sh.name, "M": sh.M, "N": sh.N, "K": sh.K, "beta_w": BETA, "activation_dtype": "bf16",
+                     "kernel": "nhwc copy + hbwn_umma_kernel", "conv_call_ms": round(msb, 5),
+                     "tops": 2.0 * sh.M * sh.N * sh.K / (msb * 1e-3) / 1e12,
+                     "frac_of_fp32_add_hbm_roofline": roofline_for("hbwn_conv", i, sh, msb, peaks, rates)["frac_of_fp32_add_hbm_roofline"],
+                     "frac_of_bf16_tensor_peak": 2.0 * sh.M * sh.N * sh.K / (msb * 1e-3) / 1e12 / bf16_tflops,
+                     "cublas": cub, "oracle": oracle_row_sample(oracle, xab, wh, 1, BETA, sh.M, hbwn=True)})
+    # --- fully connected stack, scale groups of 64
+    for batch in (256, 1):
+        stack = []
+        for i, (K, N) in enumerate(inputs.ALEXNET_FC):
+            a = inputs.normal((batch, K), inputs.SEEDS["alexnet_fc"][0] + i)
+            w = inputs.he_normal(N, K, inputs.SEEDS["alexnet_fc"][1] + i)
+            ad, wd = torch.from_numpy(a).cuda(), torch.from_numpy(w).cuda()
+            r = product_row(torch, hbmm, "alexnet_fc%d_b%d" % (6 + i, batch), batch, N, K, 64, hbmm.F32, ad, wd, rates, peaks, 60)
+            r["cublas"] = cublas_context(torch, batch, N, K, 30)
+            r["oracle"] = oracle_row_sample(oracle, a[:sample_rows_for(batch, N, K)], w, 64, 64, batch)
+            rows.append(r)
+            A = hbmm.quantize(ad, hbmm.alloc_operand(batch, K, 64, hbmm.F32))
+            W = hbmm.quantize(wd, hbmm.alloc_operand(N, K, 64, hbmm.F32))
+            ws = torch.empty(max(hbmm.gemm_workspace_bytes(A, W), 16), dtype=torch.uint8, device="cuda")
+            C = torch.empty((batch, (N + 3) // 4 * 4), device="cuda")
+            hbmm.gemm(A, W, C, ws)
+            stack.append((A, W, C, ws))
+
+        def run_stack():
+            for A, W, C, ws in stack:
+                if batch <= 8:
+                    hbmm.gemm(A, W, C, ws)
+                else:
+                    hbmm.gemm_ex(A, W, C, hbmm.PATH_FOLDED_PREPARED, ws)
+
+        # the three launches as one CUDA graph, so that they run back to back on the device
+        warm = time_graph(torch, [run_stack], 20)
+        one = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(one):
+            run_stack()
+        flush = torch.empty(int(2 * L2_BYTES) // 4, dtype=torch.float32, device="cuda")
+        cold = []
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for _ in range(20):
+            flush.zero_()                                   # evicts the weights from L2
+            e0.record()
+            one.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            cold.append(e0.elapsed_time(e1))
+        by = sum(hbmm_bytes(batch, N, K, 64) for K, N in inputs.ALEXNET_FC)
+        ops = sum(2.0 * batch * N * K for K, N in inputs.ALEXNET_FC)
+        t_roof = sum(popc_hbm_roofline(batch, N, K, 64, 4, rates, hbm_gbs)["t_roof_us"] for K, N in inputs.ALEXNET_FC)
+        rows.append({"name": "alexnet_fc_stack_b%d" % batch, "launches": 3, "warm_l2_ms": round(warm, 5),
+                     "cold_l2_ms_median": round(statistics.median(cold), 5), "cold_l2_ms_min": round(min(cold), 5),
+                     "tops_warm": ops / (warm * 1e-3) / 1e12, "gbs_cold": by / (statistics.median(cold) * 1e-3) / 1e9,
+                     "t_roof_us": round(t_roof, 3), "frac_of_popcount_hbm_roofline_cold": t_roof / (statistics.median(cold) * 1e3),
+                     "note": "three hbmm_gemm launches back to back in one CUDA graph; products are not chained (each layer has its own seeded input)"})
+        del stack
+    return rows
 
 
 # ----------------------------------------------------------------------------- CPU checker timing
@@ -575,17 +934,22 @@ def run_ours(args):
     sampler = ClockSampler(local_rank)
     sampler.start()
     sampler.wait_ready()
-    barrier()
-    t0 = time.time()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(args.steps):
-        step2(hbmm, layers, PREP)
-    e1.record()
-    barrier()
+    # The timed region (exactly `steps` steps between a barrier + synchronize on both sides) is repeated
+    # kRepeats times; the reported step time is the median region, the spread is reported beside it.
+    kRepeats = 5
+    regions = []
+    t0 = time.time()
+    for _ in range(kRepeats):
+        barrier()
+        e0.record()
+        for _ in range(args.steps):
+            step2(hbmm, layers, PREP)
+        e1.record()
+        barrier()
+        regions.append(max_over_ranks(e0.elapsed_time(e1) / args.steps, world, device))
     t1 = time.time()
-    ms_step = e0.elapsed_time(e1) / args.steps
-    ms_step = max_over_ranks(ms_step, world, device)
+    ms_step = statistics.median(regions)
     # the same step with all eight calls on one stream
     barrier()
     e0.record()
@@ -625,21 +989,36 @@ def run_ours(args):
     h2d = sum(L["x_host"].numel() * 4 + L["xb_host"].numel() * 2 for L in layers)
     d2h = sum(L["C_host"].numel() * 4 + L["Cb_host"].numel() * 4 for L in layers)
 
-    # per-kernel durations for the roofline entry (same buffers, same launch configuration)
-    brk = kernel_breakdown(torch, hbmm, layers, max(5, min(args.steps, 20)))
+    # measured issue rates of the integer and fp32 pipes: the denominators of the ALU rooflines
+    rates = measure_alu_rates(torch, hbmm, lambda: (read_sm_clock(local_rank) or (None,))[0])
+    ck = read_sm_clock(local_rank)
+    sm_max = ck[1] if ck else None
+    for k in ("popc", "fadd", "ffma"):
+        r = rates[k]
+        scale = (sm_max / r["sm_mhz"]) if (sm_max and r["sm_mhz"]) else 1.0
+        r["ops_per_s_at_max_clock"] = r["ops_per_s"] * scale
+    rates["sm_max_mhz"] = sm_max
+    rates["popcount_roofline_tops"] = rates["popc"]["ops_per_s"] * 64 / 1e12         # 32 binary MACs = 64 ops per count
+    rates["planning_figures"] = {"popc_per_clk_per_sm": PLAN_POPC_PER_CLK_SM, "fadd_per_clk_per_sm": PLAN_FADD_PER_CLK_SM}
+
+    # per-kernel durations for the roofline entry (launch configuration of the step, L2-cold)
+    brk = kernel_breakdown(torch, hbmm, layers, 3 if args.steps < 50 else 6)
     peaks = measured_peaks()
     hbm_gbs, _, hbm_src = peaks
-    totals = {k: sum(v) for k, v in brk.items()}
+    families = ("hbmm_contraction", "hbwn_conv", "front_end_pack")       # these three add up to the step's kernels
+    totals = {k: sum(brk[k]) for k in families}
     dominant = max(totals, key=totals.get)
     li = int(np.argmax(brk[dominant]))
-    roof = roofline_for(dominant, li, shapes[li], brk[dominant][li], peaks)
+    roof = roofline_for(dominant, li, shapes[li], brk[dominant][li], peaks, rates)
     roof["traffic"] = NCU_DRAM_BYTES.get((dominant, shapes[li].name))
     roof["share_of_step"] = totals[dominant] / sum(totals.values())
     kernels = {}
-    for kind, times in brk.items():
-        kernels[kind] = [dict(layer=s.name, ms=round(t, 5), **{k: v for k, v in roofline_for(kind, i, s, t, peaks).items()
-                                                                if k in ("bound", "achieved", "peak", "unit", "frac")})
-                         for i, (s, t) in enumerate(zip(shapes, times))]
+    keep = ("bound", "achieved", "peak", "unit", "frac", "frac_of_popcount_hbm_roofline", "frac_of_popcount_hbm_roofline_at_max_clock",
+            "frac_of_fp32_add_hbm_roofline", "timing")
+    for kind in families + ("hbmm_conv_call",):
+        kernels[kind] = [dict(layer=s.name, ms=round(t, 5), **{k: v for k, v in roofline_for(kind, i, s, t, peaks, rates).items() if k in keep})
+                         for i, (s, t) in enumerate(zip(shapes, brk[kind]))]
+    kernels["buffer_sets_per_layer"] = brk["sets"]
 
     if rank != 0:
         if world > 1:
@@ -650,13 +1029,20 @@ def run_ours(args):
 
     base = None
     side = None
+    configs = None
     if world == 1:
-        side = side_measurements(torch, hbmm, peaks, max(5, min(args.steps, 20)))
+        configs = config_rows(torch, hbmm, inputs, layers, brk, rates, peaks, 10)
+        side = side_measurements(torch, hbmm, inputs, peaks, max(5, min(args.steps, 20)))
         base, _, _ = cpu_baseline(shapes, 12.0)
+        err = hbmm.last_device_error()
+        if err != 0:
+            raise RuntimeError("a kernel reported device error %d during the side measurements: the numbers are void" % err)
 
     line = {
         "metric": "hbmm_effective_binary_tops", "value": aggregate(ops_step, world, ms_step), "unit": "TOPS",
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_step,
+        "timed_regions": {"count": len(regions), "steps_each": args.steps, "ms_per_step_median": ms_step,
+                          "ms_per_step_min": min(regions), "ms_per_step_max": max(regions)},
         "ms_per_step_one_stream": ms_step_one_stream,
         "ms_per_step_expanding_weights_every_call": ms_step_expand,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
@@ -675,10 +1061,14 @@ def run_ours(args):
         },
         "roofline": roof,
         "kernels": kernels,
+        "measured_alu_rates": rates,
+        "configs": configs,
+        "context": {"paper": PAPER_CONTEXT,
+                    "cublas": "each row of `configs` carries torch.matmul of the same shape in fp32 (TF32 off) and in bf16"},
         "other_rows": side,
         "e2e": {"value": aggregate(ops_step, world, ms_e2e), "unit": "TOPS", "ms_per_step": ms_e2e,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-        "gpu_launches": LAUNCHES_PER_STEP * args.steps,
+        "gpu_launches": LAUNCHES_PER_STEP * args.steps * len(regions), "gpu_launches_per_step": LAUNCHES_PER_STEP,
         "clocks": clocks,
     }
     if base is not None:

@@ -261,10 +261,20 @@ hbmm_status hbmm_conv_im2col(const void *x, int32_t x_dtype, const hbmm_conv_geo
  * call with the same W, geometry, beta_a, scale type and workspace, and that nothing has written it since.
  * The call then skips the expansion; the activation part of the workspace is rewritten by every call
  * either way.  Results are undefined when the statement is false.  Paths that keep no expanded weights
- * ignore the flag.  Unknown flag bits: HBMM_ERR_INVALID_ARG.  Everything else as hbmm_conv_im2col
- * (which is this call with flags = 0).
+ * ignore the flag.
+ * HBMM_CONV_PACK_ONLY (beta_a >= 2 only, otherwise HBMM_ERR_INVALID_ARG): the call stops once the packed
+ * activation operand -- bits [M, ld_words] at the start of the workspace, then, from the next 256-byte
+ * boundary, scales [M, ld_scales], both as hbmm_operand_bytes(M, C*kh*kw, beta_a, a_scale_dtype) lays
+ * them out -- has been written (gather + Hadamard binarization + packing, Eq. 3-4 on the im2col row);
+ * no product is formed and C_out / ldc are ignored (C_out may be NULL).  For callers that multiply one
+ * packed activation operand by several weight tensors through hbmm_gemm, and for timing the front end on
+ * its own.  On the paths that expand the weights in the front end's launch the expansion still runs unless
+ * HBMM_CONV_WEIGHTS_PREPARED is given too.
+ * Unknown flag bits: HBMM_ERR_INVALID_ARG.  Everything else as hbmm_conv_im2col (which is this call with
+ * flags = 0).
  */
 #define HBMM_CONV_WEIGHTS_PREPARED 1u
+#define HBMM_CONV_PACK_ONLY 2u
 hbmm_status hbmm_conv_im2col_ex(const void *x, int32_t x_dtype, const hbmm_conv_geom *g,
                                 int32_t beta_a, int32_t a_scale_dtype, const hbmm_operand *W,
                                 float *C_out, int64_t ldc, void *workspace, size_t workspace_bytes,

@@ -372,7 +372,9 @@ hbmm_status hbmm_conv_im2col(const void* x, int32_t x_dtype, const hbmm_conv_geo
 hbmm_status hbmm_conv_im2col_ex(const void* x, int32_t x_dtype, const hbmm_conv_geom* g, int32_t beta_a,
                                 int32_t a_scale_dtype, const hbmm_operand* W, float* C_out, int64_t ldc,
                                 void* workspace, size_t workspace_bytes, uint32_t flags, void* stream) {
-  if (flags & ~static_cast<uint32_t>(HBMM_CONV_WEIGHTS_PREPARED)) return HBMM_ERR_INVALID_ARG;
+  if (flags & ~static_cast<uint32_t>(HBMM_CONV_WEIGHTS_PREPARED | HBMM_CONV_PACK_ONLY)) return HBMM_ERR_INVALID_ARG;
+  const bool pack_only = (flags & HBMM_CONV_PACK_ONLY) != 0;
+  if (pack_only && beta_a < 2) return HBMM_ERR_INVALID_ARG;     // only a packed activation operand can be left behind
   // honoured on the two tensor-copy paths below; every other path expands the weights again (still correct)
   const bool w_prepared = (flags & HBMM_CONV_WEIGHTS_PREPARED) != 0;
   ConvGeom cg;
@@ -383,7 +385,7 @@ hbmm_status hbmm_conv_im2col_ex(const void* x, int32_t x_dtype, const hbmm_conv_
   const ConvLayout L = conv_layout(cg, beta_a, a_scale_dtype, W);
   if (W->K != L.K) return HBMM_ERR_INVALID_ARG;
   if (beta_a >= 2 && !beta_supported(L.K, beta_a)) return HBMM_ERR_UNSUPPORTED;
-  if ((st = check_c(C_out, ldc, W->rows)) != HBMM_OK) return st;
+  if (!pack_only && (st = check_c(C_out, ldc, W->rows)) != HBMM_OK) return st;
   if (!workspace || workspace_bytes < L.total) return HBMM_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return HBMM_ERR_ALIGNMENT;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -414,12 +416,14 @@ hbmm_status hbmm_conv_im2col_ex(const void* x, int32_t x_dtype, const hbmm_conv_
         if (launch_im2col_quantize_tma(x, cg, A.bits, A.ld_words, A.scales, A.ld_scales, a_scale_dtype == HBMM_BF16, s,
                                        w_prepared ? nullptr : &job) != cudaSuccess)
           return HBMM_ERR_CUDA;
+        if (pack_only) return HBMM_OK;
         return launch_gemm_fold(av, wv, C_out, ldc, gemm_ws, s, true) == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
       }
     }
     if (launch_im2col_quantize(x, x_dtype == HBMM_BF16, cg, beta_a, A.bits, A.ld_words, A.scales, A.ld_scales,
                                a_scale_dtype == HBMM_BF16, s) != cudaSuccess)
       return HBMM_ERR_CUDA;
+    if (pack_only) return HBMM_OK;
   }
   return gemm_checked(&A, W, C_out, ldc, HBMM_PATH_AUTO, static_cast<char*>(workspace) + L.operand_bytes, L.gemm_bytes, s);
 }

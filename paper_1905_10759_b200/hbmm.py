@@ -225,6 +225,7 @@ def conv_workspace_bytes(geom: hbmm_conv_geom, beta_a: int, a_scale_dtype: int, 
 
 
 CONV_WEIGHTS_PREPARED = 1
+CONV_PACK_ONLY = 2
 
 _lib.hbmm_binarize_backward.argtypes = [_vp, _i64, _vp, _i64, _i64, _i64, _i32, _vp, _i64, _vp]
 _lib.hbmm_binarize_backward.restype = _i32
@@ -291,8 +292,8 @@ def conv_im2col(x: torch.Tensor, geom: hbmm_conv_geom, beta_a: int, a_scale_dtyp
         raise ValueError("x must be a contiguous NCHW tensor")
     if flags:
         _check(_lib.hbmm_conv_im2col_ex(_dev_ptr(x), _dtype_code(x.dtype), ctypes.byref(geom), beta_a, a_scale_dtype,
-                                        ctypes.byref(W.desc), _dev_ptr(C_out), C_out.stride(0), _dev_ptr(workspace),
-                                        workspace.numel() * workspace.element_size(), flags, _stream(stream)),
+                                        ctypes.byref(W.desc), _dev_ptr(C_out), 0 if C_out is None else C_out.stride(0),
+                                        _dev_ptr(workspace), workspace.numel() * workspace.element_size(), flags, _stream(stream)),
                "hbmm_conv_im2col_ex")
         return C_out
     _check(_lib.hbmm_conv_im2col(_dev_ptr(x), _dtype_code(x.dtype), ctypes.byref(geom), beta_a, a_scale_dtype,

@@ -138,7 +138,9 @@ def test_host_validation_rejects_before_launch(hb):
     bad = hb.make_geom(2, 4, 2, 2, 5, 5, (1, 1), (0, 0))
     assert call(bad, Wc, ws, n.value) == hb.ERR_INVALID_ARG                           # filter larger than image
     assert call(g, Wc, ws, n.value, beta_a=12) == hb.ERR_UNSUPPORTED
-    assert lib.hbmm_conv_im2col_ex(x, 0, ctypes.byref(g), 36, 0, ctypes.byref(Wc.desc), c, 4, ws, n.value, 2, None) == hb.ERR_INVALID_ARG  # unknown flag
+    assert lib.hbmm_conv_im2col_ex(x, 0, ctypes.byref(g), 36, 0, ctypes.byref(Wc.desc), c, 4, ws, n.value, 4, None) == hb.ERR_INVALID_ARG  # unknown flag
+    assert lib.hbmm_conv_im2col_ex(x, 0, ctypes.byref(g), 1, 0, ctypes.byref(Wc.desc), c, 4, ws, n.value, hb.CONV_PACK_ONLY,
+                                   None) == hb.ERR_INVALID_ARG             # only a packed operand can be left behind
     fz = lib.hbmm_gemm_binarize_next
     nx = _fake_packed(hb, 8, 4, 2)
     assert fz(ctypes.byref(A.desc), ctypes.byref(W.desc), None, None, ctypes.byref(nx.desc), None, 0, None) == hb.ERR_WORKSPACE

@@ -528,6 +528,43 @@ def test_conv_with_prepared_weights_repeats_the_plain_call_bit_for_bit(hb, beta_
     assert not torch.equal(outs[0], outs[1])
 
 
+@pytest.mark.parametrize("C,H,beta_a", [(64, 12, 32), (96, 7, 32), (32, 6, 16), (40, 9, 64)])
+def test_conv_pack_only_leaves_the_operand_the_contraction_would_read(hb, C, H, beta_a):
+    """HBMM_CONV_PACK_ONLY stops after the front end: the packed activation operand in the workspace equals the
+    oracle's binarization of the im2col rows, and hbmm_gemm on it repeats the one-call convolution bit for bit."""
+    gu = _gu()
+    shape = inputs.ConvShape("t", 2, C, H, H, 72, 3, 3, 1, 1)
+    K = C * 9
+    x = inputs.conv_activation(shape, 640 + C, signed=True)
+    Wop = hb.quantize(torch.from_numpy(inputs.he_normal(72, K, 641)).cuda(), hb.alloc_operand(72, K, 32))
+    geom = hb.make_geom(2, C, H, H, 3, 3, (1, 1), (1, 1))
+    ws = torch.empty(hb.conv_workspace_bytes(geom, beta_a, hb.F32, Wop), dtype=torch.uint8, device="cuda")
+    ws.fill_(0xAB)
+    xd = torch.from_numpy(x).cuda()
+    hb.conv_im2col(xd, geom, beta_a, hb.F32, Wop, None, ws, flags=hb.CONV_PACK_ONLY)
+    M = shape.M
+    bb, sb, lw, ls = hb.operand_bytes(M, K, beta_a, hb.F32)
+    bits = ws[:bb].view(torch.int32).reshape(M, lw)
+    off = (bb + 255) // 256 * 256
+    scales = ws[off: off + sb].view(torch.float32).reshape(M, ls)
+    da, sa = oracle.quantize(oracle.im2col(x, 3, 3, (1, 1), (1, 1)), beta_a)
+    assert np.array_equal(gu.host_bits(bits), oracle.pack(sa, lw))
+    G = da.shape[1]
+    sc = scales.cpu().numpy().astype(np.float64)
+    assert np.all(sc[:, G:] == 0.0)
+    np.testing.assert_allclose(sc[:, :G], da, rtol=(int(np.ceil(np.log2(beta_a))) + 3) * gu.U, atol=0)
+    A = hb.wrap_packed(bits, scales, K, beta_a)
+    two = torch.empty((M, 72), device="cuda")
+    hb.gemm(A, Wop, two, _gemm_ws(hb, A, Wop))
+    one = torch.empty((M, 72), device="cuda")
+    ws2 = torch.empty_like(ws)
+    hb.conv_im2col(xd, geom, beta_a, hb.F32, Wop, one, ws2)
+    assert torch.equal(one, two)
+    with pytest.raises(hb.HbmmError) as e:      # a dense activation operand is never left behind
+        hb.conv_im2col(xd.to(torch.bfloat16), geom, 1, hb.F32, Wop, None, ws, flags=hb.CONV_PACK_ONLY)
+    assert e.value.status == hb.ERR_INVALID_ARG
+
+
 # ------------------------------------------------------------------ gradient through the binarization (Eq. 5, Eq. 6)
 BACKWARD_CASES = [
     # rows, K, beta, row padding of the inputs
