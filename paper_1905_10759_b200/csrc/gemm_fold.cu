@@ -7,29 +7,32 @@
 // matrices whose sum carries its fp32 group scales to 22 bits (see gemm_fold_prep.cuh), every fp16 x fp16
 // product is exact in the fp32 accumulator, and the cross products
 //     A1 W1^T + A1 W2^T + A2 W1^T
-// are one accumulation in tensor memory over the whole of K: the two weight pieces of a column tile are
-// stacked along N, so per 16 K-elements one MMA of 128 x 2TN x 16 (A1 against [W1; W2]) and one of
-// 128 x TN x 16 (A2 against W1) do all three.  The fourth product A2 W2^T is left out: both second pieces are
+// are one accumulation in tensor memory over the whole of K: per 16 K-elements three MMAs of 128 x TN x 16
+// (A1 against W1, A2 against W1, A1 against W2) add into the same TN accumulator columns (the 64-column tile
+// forms A1 W1 and A1 W2 with one MMA of 128 columns instead and adds the blocks in the epilogue).  The fourth product A2 W2^T is left out: both second pieces are
 // constant inside a scale group and at most 2^-11 of the first, so it equals sum_g (a2_g w2_g) D_g, at
 // most 2^-22 of sum_g |deltaA deltaW D_g| -- forty times below the 1e-5 the result is held to.
-// There is no per-group step; the epilogue runs once per tile, adds the two column blocks and divides
-// the rows' and columns' powers of two out again (exact).  Compared with forming D_g and the scale
+// There is no per-group step; the epilogue runs once per tile and divides the rows' and columns' powers of
+// two out again (exact).  Compared with forming D_g and the scale
 // product per group this trades 3x the tensor work for the removal of the per-group TMEM round trip
 // that bounded the e4m3 kernel.
 //
 // CTA tile = 128 rows x TN columns; one persistent CTA per SM walks the tiles of the output.
 //   warps 0-3   : epilogue, once per tile (TMEM lanes 32*w ..)
 //   warps 4-11  : A producers: thread = (tile row, stage parity); packed words + group scales -> the
-//                 64 elements of both fp16 pieces in the 128-byte-swizzled K-major layout, with the
-//                 global loads issued several stages ahead
+//                 64 elements of both fp16 pieces, written from registers straight into TENSOR memory (the
+//                 MMA takes its A operand from there: the activation operand never passes through shared
+//                 memory, whose bandwidth bounded the kernel while it did), with the global loads issued
+//                 several stages ahead
 //   warps 14-17 : scouts: one thread per tile row finds the row's largest scale (the power of two that
 //                 normalises the row) a few tiles ahead of everyone else
 //   warp  12    : TMEM allocation and the single MMA-issuing thread
 //   warp  13    : one thread streams the prepared W stages (cp.async.bulk, completion on the stage's
 //                 mbarrier); W is expanded once per call (or once per weight tensor) into a workspace
-// A stage holds 64 K-elements (two packed words).  Stages and the two TMEM accumulators are mbarrier
-// rings.  Every wait is bounded: on expiry the thread records a code, raises a CTA-wide abort flag
-// that all other waits observe, and the kernel drains and frees its TMEM before returning.
+// A stage holds 64 K-elements (two packed words): 64 TMEM columns of A pieces and the W stage in shared
+// memory.  Tensor memory: two accumulators of TN columns, the rest is the ring of A stages.  Stages and the
+// accumulators are mbarrier rings.  Every wait is bounded: on expiry the thread records a code, raises a
+// CTA-wide abort flag that all other waits observe, and the kernel drains and frees its TMEM before returning.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include "kernels.h"
@@ -173,6 +176,7 @@ hbmm_fold_kernel(const Args g) {
     const int pt = tid - kFirstProducerWarp * 32;
     const int q = pt >> 7;
     const int p = pt & (TM - 1);
+    const uint32_t t_lane = static_cast<uint32_t>((warp & 3) * 32) << 16;     // this warp's quarter of the TMEM lanes = its tile rows
     const uint32_t n_words = static_cast<uint32_t>(g.n_words), gw = static_cast<uint32_t>(g.a_gw);
     const bool vec_scales = ASUB == 1 && !g.a_bf16 && gw == 1;      // one fp32 scale per word: a stage's two scales are one 8-byte load
     const int64_t total = my_tiles * n_stages;
@@ -246,20 +250,28 @@ hbmm_fold_kernel(const Args g) {
           }
           const int s = static_cast<int>(my % STAGES);
           if (ok && my >= STAGES && !mbar_wait(&empty[s], static_cast<uint32_t>(((my / STAGES) & 1) ^ 1), abort_flag, 1)) ok = false;
+          ok = __all_sync(0xFFFFFFFFu, ok);      // the tensor-memory stores below are warp-wide: all lanes or none
           if (ok) {
-            unsigned char* a1 = smem + S::OFF_A + s * S::A_STAGE;
-            if (ASUB == 1) {
-              expand_word(a1, a1 + S::A_PIECE, p, 0, w[u].x, sc[u][0] * up);
-              expand_word(a1, a1 + S::A_PIECE, p, 1, w[u].y, sc[u][ASUB] * up);
-            } else {
-              constexpr int SB = ASUB > 1 ? ASUB : 2;
-              float lo[SB], hi[SB];
+            // stage s: columns [0, 32) piece 1, [32, 64) piece 2; word slot q in columns 16 q .. 16 q + 15 of its piece
+            const uint32_t a_col = tmem_base + t_lane + S::A_BASE + static_cast<uint32_t>(s) * S::A_COLS;
 #pragma unroll
-              for (int i = 0; i < ASUB; i++) { lo[i] = sc[u][i] * up; hi[i] = sc[u][ASUB + i] * up; }
-              expand_word_sub<SB>(a1, a1 + S::A_PIECE, p, 0, w[u].x, lo);
-              expand_word_sub<SB>(a1, a1 + S::A_PIECE, p, 1, w[u].y, hi);
+            for (int qw = 0; qw < WPS; qw++) {
+              uint32_t p1[16], p2[16];
+              const uint32_t word = qw == 0 ? w[u].x : w[u].y;
+              if (ASUB == 1) {
+                expand_word_regs(word, sc[u][qw * ASUB] * up, p1, p2);
+              } else {
+                constexpr int SB = ASUB > 1 ? ASUB : 2;
+                float sw[SB];
+#pragma unroll
+                for (int i = 0; i < ASUB; i++) sw[i] = sc[u][qw * ASUB + i] * up;
+                expand_word_sub_regs<SB>(word, sw, p1, p2);
+              }
+              tmem_st16(a_col + qw * 16, p1);
+              tmem_st16(a_col + KB / 2 + qw * 16, p2);
             }
-            fence_async_proxy();          // make the generic-proxy stores visible to the tensor core
+            tmem_st_wait();               // the pieces are in tensor memory ...
+            tc_fence_before();            // ... before the arrival that lets the MMA read them
             __syncwarp();
             if (lane == 0) mbar_arrive(&full[s]);
             fetch(pf, w[u], sc[u]);         // this register slot is free again: load kDepth of my stages ahead
@@ -319,11 +331,11 @@ hbmm_fold_kernel(const Args g) {
     // The whole warp walks the loop so that ring indices and descriptors stay warp-uniform values; one
     // lane issues the MMAs and commits.
     {
-      constexpr uint32_t idesc = instr_desc(S::NST, kFmtF16);     // A1 against [W1; W2]: both column blocks
-      constexpr uint32_t idesc_w1 = instr_desc(TN, kFmtF16);      // A2 against W1 alone: the first column block
-      const uint64_t da0 = smem_desc(smem_u32(smem + S::OFF_A)), db0 = smem_desc(smem_u32(smem + S::OFF_B));
-      const uint64_t da_hi = da0 & 0xFFFFFFFF00000000ull, db_hi = db0 & 0xFFFFFFFF00000000ull;
-      const uint32_t da_lo = static_cast<uint32_t>(da0), db_lo = static_cast<uint32_t>(db0);
+      constexpr uint32_t idesc = instr_desc(TN, kFmtF16);
+      constexpr uint32_t idesc2 = instr_desc(2 * TN, kFmtF16);     // stacked: both weight pieces in one instruction
+      const uint64_t db0 = smem_desc(smem_u32(smem + S::OFF_B));
+      const uint64_t db_hi = db0 & 0xFFFFFFFF00000000ull;
+      const uint32_t db_lo = static_cast<uint32_t>(db0);
       const uint32_t full_a = smem_u32(full), empty_a = smem_u32(empty), tfull_a = smem_u32(tfull), tempty_a = smem_u32(tempty);
       const bool leader = lane == 0;
       const uint32_t n_st = static_cast<uint32_t>(n_stages);
@@ -335,19 +347,25 @@ hbmm_fold_kernel(const Args g) {
           if (!mbar_wait_a(tempty_a + buf * 8, static_cast<uint32_t>(((ti >> 1) & 1) ^ 1), abort_flag, 3)) { ok = false; break; }
           tc_fence_after();
         }
-        const uint32_t d_tmem = tmem_base + buf * S::NST;
+        const uint32_t d_tmem = tmem_base + buf * S::ACC_COLS;
         for (uint32_t st = 0; st < n_st; st++) {
           if (!mbar_wait_a(full_a + s * 8, full_par, abort_flag, 2)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t a1_lo = da_lo + s * (S::A_STAGE >> 4), a2_lo = a1_lo + (S::A_PIECE >> 4);
-          const uint32_t b_lo = db_lo + s * (S::B_STAGE >> 4);
+          const uint32_t a1 = tmem_base + S::A_BASE + s * S::A_COLS, a2 = a1 + KB / 2;
+          const uint32_t b1_lo = db_lo + s * (S::B_STAGE >> 4), b2_lo = b1_lo + (S::B_PIECE >> 4);
           if (leader) {
 #pragma unroll
-            for (int ks = 0; ks < KB / 16; ks++) {        // 16 K-elements = 32 bytes along the swizzled rows
-              umma_bf16(d_tmem, da_hi | (a1_lo + ks * 2), db_hi | (b_lo + ks * 2), idesc, (st | ks) != 0 ? 1u : 0u);
-              umma_bf16(d_tmem, da_hi | (a2_lo + ks * 2), db_hi | (b_lo + ks * 2), idesc_w1, 1u);
+            for (int ks = 0; ks < KB / 16; ks++) {        // 16 K-elements = 8 TMEM columns of A, 32 bytes along the swizzled rows of W
+              if constexpr (S::STACKED) {
+                umma_f16_ts(d_tmem, a1 + ks * 8, db_hi | (b1_lo + ks * 2), idesc2, (st | ks) != 0 ? 1u : 0u);   // A1 [W1; W2]
+                umma_f16_ts(d_tmem, a2 + ks * 8, db_hi | (b1_lo + ks * 2), idesc, 1u);                           // A2 W1
+              } else {
+                umma_f16_ts(d_tmem, a1 + ks * 8, db_hi | (b1_lo + ks * 2), idesc, (st | ks) != 0 ? 1u : 0u);
+                umma_f16_ts(d_tmem, a2 + ks * 8, db_hi | (b1_lo + ks * 2), idesc, 1u);
+                umma_f16_ts(d_tmem, a1 + ks * 8, db_hi | (b2_lo + ks * 2), idesc, 1u);
+              }
             }
-            umma_commit_a(empty_a + s * 8);     // the stage's bytes are free once these MMAs have read them
+            umma_commit_a(empty_a + s * 8);     // the stage (TMEM columns and W bytes) is free once these MMAs have read it
           }
           __syncwarp();
           if (++s == STAGES) { s = 0; full_par ^= 1; }
@@ -405,11 +423,18 @@ hbmm_fold_kernel(const Args g) {
       float carry = 0.0f;                                   // |z| sum of a group wider than a 32-column chunk
 #pragma unroll
       for (int c = 0; c < TN / 32; c++) {
-        uint32_t v1[32], v2[32];
-        const uint32_t t_addr = tmem_base + t_lane + buf * S::NST + c * 32;
+        uint32_t v1[32];
+        const uint32_t t_addr = tmem_base + t_lane + buf * S::ACC_COLS + c * 32;
         tmem_ld32(t_addr, v1);
-        tmem_ld32(t_addr + TN, v2);
-        tmem_ld_wait();
+        if constexpr (S::STACKED) {      // the A1 W2 block sits TN columns further on
+          uint32_t v2[32];
+          tmem_ld32(t_addr + TN, v2);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; j++) v1[j] = __float_as_uint(__uint_as_float(v1[j]) + __uint_as_float(v2[j]));
+        } else {
+          tmem_ld_wait();
+        }
         if constexpr (FUSE) {
           if (m < g.M) {
           // affine map per column, then the row is binarized for the next layer: packed word + group scales
@@ -422,7 +447,7 @@ hbmm_fold_kernel(const Args g) {
             const float w4[4] = {fw.x, fw.y, fw.z, fw.w}, s4[4] = {bs.x, bs.y, bs.z, bs.w}, h4[4] = {bh.x, bh.y, bh.z, bh.w};
 #pragma unroll
             for (int e = 0; e < 4; e++)
-              z[j + e] = fmaf((__uint_as_float(v1[j + e]) + __uint_as_float(v2[j + e])) * fa * w4[e], s4[e], h4[e]);
+              z[j + e] = fmaf(__uint_as_float(v1[j + e]) * fa * w4[e], s4[e], h4[e]);
           }
           const int64_t n0 = nb + c * 32;
           const int valid = g.N - n0 >= 32 ? 32 : static_cast<int>(g.N - n0 > 0 ? g.N - n0 : 0);
@@ -449,7 +474,7 @@ hbmm_fold_kernel(const Args g) {
             const float4 fw = *reinterpret_cast<const float4*>(cf + c * 32 + j);
             float o[4];
 #pragma unroll
-            for (int e = 0; e < 4; e++) o[e] = (__uint_as_float(v1[j + e]) + __uint_as_float(v2[j + e])) * fa;
+            for (int e = 0; e < 4; e++) o[e] = __uint_as_float(v1[j + e]) * fa;
             o[0] *= fw.x; o[1] *= fw.y; o[2] *= fw.z; o[3] *= fw.w;
             const int64_t n = nb + c * 32 + j;
             if (n + 3 < g.N) *reinterpret_cast<float4*>(dst + c * 32 + j) = make_float4(o[0], o[1], o[2], o[3]);

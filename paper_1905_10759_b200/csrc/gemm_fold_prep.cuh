@@ -26,25 +26,34 @@ constexpr int KB = 64;            // K elements per stage: one 128-byte row of f
 constexpr int WPS = 2;            // packed K-words per stage
 constexpr int kRowSlots = 8;      // ring of per-tile row factors (scouts -> producers and epilogue)
 
+// The weight stages live in shared memory (streamed from the prepared workspace by bulk copies); the
+// activation pieces live in TENSOR memory: the producers write them there straight from registers and the
+// MMA reads its A operand from there, so the activation operand never touches shared memory.
 template <int TN>
 struct Smem {
-  static constexpr int STAGES = TN == 64 ? 4 : 3;
-  static constexpr int A_PIECE = TM * 128;                // one fp16 piece of the A tile: 128 rows x 64 elements
-  static constexpr int A_STAGE = 2 * A_PIECE;
+  static constexpr int A_COLS = 2 * (KB / 2);             // TMEM columns of one A stage: two pieces x 64 fp16 (two per 32-bit column)
+  // A tensor-core instruction costs about the same for 64 and for 128 columns, so the narrow tile stacks
+  // the two weight pieces along N: one MMA of 2 TN columns forms A1 W1 and A1 W2 side by side (the epilogue
+  // adds the two blocks) and a second one of TN columns adds A2 W1.  The wide tile has no room for a
+  // 256-column accumulator pair beside the A ring and adds all three products into the same TN columns.
+  static constexpr bool STACKED = TN == 64;
+  static constexpr int ACC_COLS = STACKED ? 2 * TN : TN;  // one fp32 accumulator
+  static constexpr int STAGES = (512 - 2 * ACC_COLS) / A_COLS;        // 4: the rest of the 512 columns
+  static constexpr int A_BASE = 2 * ACC_COLS;             // first TMEM column of the A ring
+  static constexpr int TMEM_COLS = 512;
   static constexpr int B_PIECE = TN * 128;
-  static constexpr int B_STAGE = 2 * B_PIECE;             // W1 rows then W2 rows: one MMA of N = 2 TN reads both
-  static constexpr int OFF_A = 0;
-  static constexpr int OFF_B = OFF_A + STAGES * A_STAGE;
+  static constexpr int B_STAGE = 2 * B_PIECE;             // W1 rows then W2 rows
+  static constexpr int OFF_B = 0;
   static constexpr int OFF_ROWF = OFF_B + STAGES * B_STAGE;
   static constexpr int OFF_COLF = OFF_ROWF + 2 * kRowSlots * TM * 4;  // per slot and row: normalising power of two and its inverse
   static constexpr int OFF_BAR = OFF_COLF + 3 * 4 * TN * 4;           // the tile's column factors (power of two, affine scale and shift), one copy per epilogue warp
   static constexpr int NBAR = 2 * STAGES + 4 + 1 + 2 * kRowSlots;     // full, empty, tfull[2], tempty[2], drain, rowfull, rowempty
   static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
-  static constexpr int BYTES = OFF_MISC + 16;
-  static constexpr int NST = 2 * TN;                      // MMA N
-  static constexpr int TMEM_COLS = 2 * NST;               // two accumulators
-  static_assert(BYTES > 120 * 1024, "one CTA per SM: it owns the tensor memory it allocates");
-  static_assert(NST <= 256 && NST % 16 == 0, "one MMA covers both weight pieces");
+  static constexpr int USED = OFF_MISC + 16;
+  // more than half of an SM's shared memory is requested whatever is used: one CTA per SM, which owns all 512
+  // columns of tensor memory
+  static constexpr int BYTES = USED > 120 * 1024 ? USED : 120 * 1024;
+  static_assert(STAGES >= 3 && A_BASE + STAGES * A_COLS <= 512, "accumulators and the A ring share 512 columns");
 };
 
 __device__ __forceinline__ float load_scale(const void* s, int bf16, int64_t idx) {
@@ -106,6 +115,44 @@ __device__ __forceinline__ void expand_word(unsigned char* piece1, unsigned char
     for (int i = 0; i < 4; i++) m[i] = (nw << (15 - (4 * c + i))) & 0x80008000u;
     *reinterpret_cast<uint4*>(swz(piece1, row, 4 * q + c)) = make_uint4(m[0] ^ h1, m[1] ^ h1, m[2] ^ h1, m[3] ^ h1);
     *reinterpret_cast<uint4*>(swz(piece2, row, 4 * q + c)) = make_uint4(m[0] ^ h2, m[1] ^ h2, m[2] ^ h2, m[3] ^ h2);
+  }
+}
+
+// The same 32 elements as 16 + 16 register values (one per 32-bit column of tensor memory): column j of the
+// word's 16 columns holds the elements of bits j (low half) and j + 16 (high half), exactly the pairs
+// expand_word stores at 32-bit position j.
+__device__ __forceinline__ void expand_word_regs(uint32_t word, float scaled, uint32_t (&p1)[16], uint32_t (&p2)[16]) {
+  const __half d1 = __float2half_rn(scaled);
+  const __half d2 = __float2half_rn(scaled - __half2float(d1));
+  const uint32_t h1 = static_cast<uint32_t>(__half_as_ushort(d1)) * 0x10001u;
+  const uint32_t h2 = static_cast<uint32_t>(__half_as_ushort(d2)) * 0x10001u;
+  const uint32_t nw = ~word;
+#pragma unroll
+  for (int j = 0; j < 16; j++) {
+    const uint32_t m = (nw << (15 - j)) & 0x80008000u;
+    p1[j] = m ^ h1;
+    p2[j] = m ^ h2;
+  }
+}
+template <int SUB>
+__device__ __forceinline__ void expand_word_sub_regs(uint32_t word, const float (&scaled)[SUB], uint32_t (&p1)[16], uint32_t (&p2)[16]) {
+  static_assert(SUB == 2 || SUB == 4 || SUB == 8 || SUB == 16, "beta = 16, 8, 4, 2");
+  constexpr int BETA = 32 / SUB, HALF = SUB / 2;
+  uint32_t h1[HALF], h2[HALF];
+#pragma unroll
+  for (int t = 0; t < HALF; t++) {
+    const __half2 d1 = __floats2half2_rn(scaled[t], scaled[t + HALF]);          // low half: group t, high half: group t + SUB/2
+    const float2 back = __half22float2(d1);
+    const __half2 d2 = __floats2half2_rn(scaled[t] - back.x, scaled[t + HALF] - back.y);
+    h1[t] = *reinterpret_cast<const uint32_t*>(&d1);
+    h2[t] = *reinterpret_cast<const uint32_t*>(&d2);
+  }
+  const uint32_t nw = ~word;
+#pragma unroll
+  for (int j = 0; j < 16; j++) {
+    const uint32_t m = (nw << (15 - j)) & 0x80008000u;
+    p1[j] = m ^ h1[j / BETA];
+    p2[j] = m ^ h2[j / BETA];
   }
 }
 
