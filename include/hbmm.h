@@ -219,10 +219,57 @@ hbmm_status hbmm_gemm_ex(const hbmm_operand *A, const hbmm_operand *W, float *C,
  * and smaller than W.rows; workspace as hbmm_gemm_workspace_bytes(A, W) reports.  bn_scale / bn_shift:
  * device fp32 [W.rows].  Where z is within rounding of zero the sign follows the fp32 value the kernel
  * computed.  Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, WORKSPACE, CUDA.
+ * (hbmm_gemm_fused with HBMM_OUT_PACKED, no activation, both operands packed.)
  */
 hbmm_status hbmm_gemm_binarize_next(const hbmm_operand *A, const hbmm_operand *W, const float *bn_scale,
                                     const float *bn_shift, const hbmm_operand *next, void *workspace,
                                     size_t workspace_bytes, void *stream);
+
+/*
+ * What may happen to a product before it leaves the contraction kernel -- the rest of the paper's layer (Section 5:
+ * batch normalisation -> binarization -> convolution -> activation -> pooling, then the next block's batch
+ * normalisation and binarization), applied in the epilogue while the outputs are in registers:
+ *     y = activation(C)                    HBMM_ACT_NONE, or HBMM_ACT_RELU: max(0, C)
+ *     z[m,n] = bn_scale[n] * y + bn_shift[n]   the NEXT block's batch normalisation folded to inference form
+ *                                              (device fp32 [N]; either pointer may be NULL: 1 and 0)
+ * and then one of
+ *   HBMM_OUT_DENSE : z stored as out[m * ld_out + n], out_dtype HBMM_F32 or HBMM_BF16 (round to nearest even),
+ *                    ld_out >= N, out aligned to its element (16-byte aligned rows take vector stores).  For a
+ *                    convolution the rows are output pixels, so this is the NHWC activation tensor of the next
+ *                    layer: a dense-activation (beta_a = 1) convolution reads it directly when it is given
+ *                    HBMM_CONV_INPUT_NHWC, with no layout copy and no fp32 round trip.
+ *   HBMM_OUT_PACKED: every row of z is Hadamard-binarized along n with group next->beta (Eq. 3-4) and only the
+ *                    packed result is written (4 bytes per output become 1 + 32/beta bits).  `next`: host
+ *                    descriptor of a packed operand with rows = M, K = N, buffers sized by hbmm_operand_bytes;
+ *                    filled like hbmm_quantize fills its output, zero padding included.  It is what a following
+ *                    fully connected layer or 1 x 1 convolution reads as its A.  next->beta one of 2, 4, 8, 16, 32,
+ *                    64, 128, at most 64 when the product has at most 64 columns, and smaller than N.  Where z
+ *                    is within rounding of zero the sign follows the fp32 value the kernel computed.
+ * Pooling is not part of the chain.  The fp32 product itself is never stored.
+ */
+typedef enum { HBMM_ACT_NONE = 0, HBMM_ACT_RELU = 1 } hbmm_activation;
+typedef enum { HBMM_OUT_DENSE = 1, HBMM_OUT_PACKED = 2 } hbmm_out_kind;
+typedef struct {
+  int32_t activation;        /* hbmm_activation */
+  int32_t out_kind;          /* hbmm_out_kind */
+  const float *bn_scale;     /* device fp32 [N] or NULL */
+  const float *bn_shift;     /* device fp32 [N] or NULL */
+  void *out;                 /* HBMM_OUT_DENSE: device [M, ld_out] */
+  int64_t ld_out;
+  int32_t out_dtype;         /* hbmm_dtype */
+  int32_t reserved;
+  const hbmm_operand *next;  /* HBMM_OUT_PACKED: host descriptor, device buffers */
+} hbmm_epilogue;
+
+/*
+ * hbmm_gemm with the epilogue chain above instead of the fp32 store.  A packed (scale groups of whole K-words,
+ * or one group per row; K a multiple of 32): the folded-scale tensor-core kernel; A dense bf16 with rows on
+ * 16-byte boundaries (beta_a = 1): the tensor-core HBWN kernel.  workspace as hbmm_gemm_workspace_bytes(A, W)
+ * reports (required).  ep: host struct, read before the call returns.
+ * Errors: INVALID_ARG, UNSUPPORTED (operands outside the above, next->beta), ALIGNMENT, WORKSPACE, CUDA.
+ */
+hbmm_status hbmm_gemm_fused(const hbmm_operand *A, const hbmm_operand *W, const hbmm_epilogue *ep, void *workspace,
+                            size_t workspace_bytes, void *stream);
 
 /*
  * The integer term of Eq. 7 on its own: D[m,n,t] = signed +-1 dot product of K-segment t
@@ -275,10 +322,26 @@ hbmm_status hbmm_conv_im2col(const void *x, int32_t x_dtype, const hbmm_conv_geo
  */
 #define HBMM_CONV_WEIGHTS_PREPARED 1u
 #define HBMM_CONV_PACK_ONLY 2u
+/* beta_a == 1 only: x is an NHWC bf16 tensor [B, H, W, C] (16-byte aligned, C a multiple of 64) instead of NCHW --
+ * what HBMM_OUT_DENSE of the layer before wrote.  The layout copy of the dense-activation path is skipped.
+ * Otherwise HBMM_ERR_INVALID_ARG (beta_a, dtype) / HBMM_ERR_UNSUPPORTED (channel count) / HBMM_ERR_ALIGNMENT. */
+#define HBMM_CONV_INPUT_NHWC 4u
 hbmm_status hbmm_conv_im2col_ex(const void *x, int32_t x_dtype, const hbmm_conv_geom *g,
                                 int32_t beta_a, int32_t a_scale_dtype, const hbmm_operand *W,
                                 float *C_out, int64_t ldc, void *workspace, size_t workspace_bytes,
                                 uint32_t flags, void *stream);
+
+/*
+ * hbmm_conv_im2col_ex with the epilogue chain of hbmm_epilogue instead of the fp32 NHWC store: the convolution,
+ * the activation that follows it, the next block's folded batch normalisation, and the form the next layer
+ * reads (dense NHWC bf16 / fp32, or rows binarized along the output channels).  beta_a >= 2: K = C*kh*kw a
+ * multiple of 32 and activation groups of whole K-words (or one group per row); beta_a == 1: C a multiple of
+ * 64.  Flags as hbmm_conv_im2col_ex except HBMM_CONV_PACK_ONLY.  Workspace as hbmm_conv_workspace_bytes.
+ * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, WORKSPACE, CUDA.
+ */
+hbmm_status hbmm_conv_im2col_fused(const void *x, int32_t x_dtype, const hbmm_conv_geom *g, int32_t beta_a,
+                                   int32_t a_scale_dtype, const hbmm_operand *W, const hbmm_epilogue *ep,
+                                   void *workspace, size_t workspace_bytes, uint32_t flags, void *stream);
 
 /*
  * hbmm_conv_im2col for callers that cannot allocate device memory.  (No counterpart in the

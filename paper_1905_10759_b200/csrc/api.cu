@@ -238,6 +238,37 @@ ConvLayout conv_layout(const ConvGeom& g, int32_t beta_a, int32_t scale_dtype, c
   return L;
 }
 
+// Validates a caller's epilogue description for an M x N product and translates it for the kernels.
+hbmm_status make_epilogue(const hbmm_epilogue* ep, int64_t M, int64_t N, EpiArgs* out) {
+  EpiArgs e = plain_epilogue();
+  if (ep->activation != HBMM_ACT_NONE && ep->activation != HBMM_ACT_RELU) return HBMM_ERR_INVALID_ARG;
+  if ((ep->bn_scale && reinterpret_cast<uintptr_t>(ep->bn_scale) % 4 != 0) || (ep->bn_shift && reinterpret_cast<uintptr_t>(ep->bn_shift) % 4 != 0))
+    return HBMM_ERR_ALIGNMENT;
+  e.act = ep->activation == HBMM_ACT_RELU ? 1 : 0;
+  e.bn_scale = ep->bn_scale; e.bn_shift = ep->bn_shift;
+  if (ep->out_kind == HBMM_OUT_DENSE) {
+    if (!ep->out || !valid_dtype(ep->out_dtype) || ep->ld_out < N) return HBMM_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(ep->out) % (ep->out_dtype == HBMM_BF16 ? 2 : 4) != 0) return HBMM_ERR_ALIGNMENT;
+    e.mode = kEpiDense; e.out = ep->out; e.out_bf16 = ep->out_dtype == HBMM_BF16; e.ld_out = ep->ld_out;
+  } else if (ep->out_kind == HBMM_OUT_PACKED) {
+    const hbmm_operand* nx = ep->next;
+    if (!nx || nx->rows != M || nx->K != N) return HBMM_ERR_INVALID_ARG;
+    const hbmm_status st = check_packed(nx);
+    if (st != HBMM_OK) return st;
+    if (nx->beta >= nx->K) return HBMM_ERR_UNSUPPORTED;
+    e.mode = kEpiPacked; e.nx_bits = nx->bits; e.nx_scales = nx->scales; e.nx_ld_words = nx->ld_words; e.nx_ld_scales = nx->ld_scales;
+    e.nx_bf16 = nx->scale_dtype == HBMM_BF16; e.nx_beta = nx->beta;
+  } else {
+    return HBMM_ERR_INVALID_ARG;
+  }
+  *out = e;
+  return HBMM_OK;
+}
+
+hbmm_status conv_checked(const void* x, int32_t x_dtype, const hbmm_conv_geom* g, int32_t beta_a, int32_t a_scale_dtype,
+                         const hbmm_operand* W, float* C_out, int64_t ldc, const hbmm_epilogue* ep, void* workspace,
+                         size_t workspace_bytes, uint32_t flags, void* stream);
+
 }  // namespace
 
 extern "C" {
@@ -307,27 +338,41 @@ hbmm_status hbmm_gemm_ex(const hbmm_operand* A, const hbmm_operand* W, float* C,
   return gemm_checked(A, W, C, ldc, path, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
 }
 
-hbmm_status hbmm_gemm_binarize_next(const hbmm_operand* A, const hbmm_operand* W, const float* bn_scale, const float* bn_shift,
-                                    const hbmm_operand* next, void* workspace, size_t workspace_bytes, void* stream) {
+hbmm_status hbmm_gemm_fused(const hbmm_operand* A, const hbmm_operand* W, const hbmm_epilogue* ep, void* workspace,
+                            size_t workspace_bytes, void* stream) {
   hbmm_status st;
-  if (!A || !W || !next) return HBMM_ERR_INVALID_ARG;
-  if (A->beta == 1 || W->beta == 1) return HBMM_ERR_UNSUPPORTED;       // both operands packed
-  if ((st = check_packed(A)) != HBMM_OK) return st;
+  if (!A || !W || !ep) return HBMM_ERR_INVALID_ARG;
+  if (W->beta == 1) return HBMM_ERR_UNSUPPORTED;                       // the weight operand is always Hadamard-binary
   if ((st = check_packed(W)) != HBMM_OK) return st;
   if (A->K != W->K) return HBMM_ERR_INVALID_ARG;
-  if (next->rows != A->rows || next->K != W->rows) return HBMM_ERR_INVALID_ARG;
-  if ((st = check_packed(next)) != HBMM_OK) return st;
-  if ((bn_scale && reinterpret_cast<uintptr_t>(bn_scale) % 4 != 0) || (bn_shift && reinterpret_cast<uintptr_t>(bn_shift) % 4 != 0))
-    return HBMM_ERR_ALIGNMENT;
-  const PackedView a = view_of(A), w = view_of(W);
+  EpiArgs e;
+  if ((st = make_epilogue(ep, A->rows, W->rows, &e)) != HBMM_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const PackedView w = view_of(W);
+  if (A->beta == 1) {
+    if (A->rows <= 0 || A->K <= 0 || !A->dense || A->ld_dense < A->K || !valid_dtype(A->dense_dtype)) return HBMM_ERR_INVALID_ARG;
+    const DenseView dv = dense_view_of(A);
+    if (!hbwn_umma_supported(dv, w)) return HBMM_ERR_UNSUPPORTED;     // bf16 rows on 16-byte boundaries
+    if (e.mode == kEpiPacked && !gemm_fold_next_supported(W->rows, e.nx_beta)) return HBMM_ERR_UNSUPPORTED;
+    if (!workspace_ok(workspace, workspace_bytes, hbwn_workspace(dv, w))) return HBMM_ERR_WORKSPACE;
+    return launch_hbwn_umma(dv, w, nullptr, 0, workspace, s, false, false, &e) == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
+  }
+  if ((st = check_packed(A)) != HBMM_OK) return st;
+  const PackedView a = view_of(A);
   const bool a_subword = A->beta < 32 && A->beta < A->K;
-  if (!gemm_fold_supported(a, w) || a_subword || next->beta >= next->K || !gemm_fold_next_supported(W->rows, next->beta))
-    return HBMM_ERR_UNSUPPORTED;
+  if (!segments_compatible(A, W) || !gemm_fold_supported(a, w) || a_subword) return HBMM_ERR_UNSUPPORTED;
+  if (e.mode == kEpiPacked && !gemm_fold_next_supported(W->rows, e.nx_beta)) return HBMM_ERR_UNSUPPORTED;
   if (!workspace_ok(workspace, workspace_bytes, fold_workspace(a, w))) return HBMM_ERR_WORKSPACE;
-  FoldNext nx;
-  nx.bn_scale = bn_scale; nx.bn_shift = bn_shift; nx.bits = next->bits; nx.scales = next->scales;
-  nx.ld_words = next->ld_words; nx.ld_scales = next->ld_scales; nx.scale_bf16 = next->scale_dtype == HBMM_BF16; nx.beta = next->beta;
-  return launch_gemm_fold(a, w, nullptr, 0, workspace, static_cast<cudaStream_t>(stream), false, &nx) == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
+  return launch_gemm_fold(a, w, nullptr, 0, workspace, s, false, &e) == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
+}
+
+hbmm_status hbmm_gemm_binarize_next(const hbmm_operand* A, const hbmm_operand* W, const float* bn_scale, const float* bn_shift,
+                                    const hbmm_operand* next, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!A || !W || !next) return HBMM_ERR_INVALID_ARG;
+  if (A->beta == 1 || W->beta == 1) return HBMM_ERR_UNSUPPORTED;       // both operands packed
+  hbmm_epilogue ep{};
+  ep.activation = HBMM_ACT_NONE; ep.out_kind = HBMM_OUT_PACKED; ep.bn_scale = bn_scale; ep.bn_shift = bn_shift; ep.next = next;
+  return hbmm_gemm_fused(A, W, &ep, workspace, workspace_bytes, stream);
 }
 
 hbmm_status hbmm_gemm_partials(const hbmm_operand* A, const hbmm_operand* W, int32_t* D, int32_t path, void* stream) {
@@ -372,8 +417,26 @@ hbmm_status hbmm_conv_im2col(const void* x, int32_t x_dtype, const hbmm_conv_geo
 hbmm_status hbmm_conv_im2col_ex(const void* x, int32_t x_dtype, const hbmm_conv_geom* g, int32_t beta_a,
                                 int32_t a_scale_dtype, const hbmm_operand* W, float* C_out, int64_t ldc,
                                 void* workspace, size_t workspace_bytes, uint32_t flags, void* stream) {
-  if (flags & ~static_cast<uint32_t>(HBMM_CONV_WEIGHTS_PREPARED | HBMM_CONV_PACK_ONLY)) return HBMM_ERR_INVALID_ARG;
+  return conv_checked(x, x_dtype, g, beta_a, a_scale_dtype, W, C_out, ldc, nullptr, workspace, workspace_bytes, flags, stream);
+}
+
+hbmm_status hbmm_conv_im2col_fused(const void* x, int32_t x_dtype, const hbmm_conv_geom* g, int32_t beta_a,
+                                   int32_t a_scale_dtype, const hbmm_operand* W, const hbmm_epilogue* ep,
+                                   void* workspace, size_t workspace_bytes, uint32_t flags, void* stream) {
+  if (!ep || (flags & HBMM_CONV_PACK_ONLY)) return HBMM_ERR_INVALID_ARG;
+  return conv_checked(x, x_dtype, g, beta_a, a_scale_dtype, W, nullptr, 0, ep, workspace, workspace_bytes, flags, stream);
+}
+
+}  // extern "C"
+
+namespace {
+
+hbmm_status conv_checked(const void* x, int32_t x_dtype, const hbmm_conv_geom* g, int32_t beta_a, int32_t a_scale_dtype,
+                         const hbmm_operand* W, float* C_out, int64_t ldc, const hbmm_epilogue* ep, void* workspace,
+                         size_t workspace_bytes, uint32_t flags, void* stream) {
+  if (flags & ~static_cast<uint32_t>(HBMM_CONV_WEIGHTS_PREPARED | HBMM_CONV_PACK_ONLY | HBMM_CONV_INPUT_NHWC)) return HBMM_ERR_INVALID_ARG;
   const bool pack_only = (flags & HBMM_CONV_PACK_ONLY) != 0;
+  const bool input_nhwc = (flags & HBMM_CONV_INPUT_NHWC) != 0;
   if (pack_only && beta_a < 2) return HBMM_ERR_INVALID_ARG;     // only a packed activation operand can be left behind
   // honoured on the two tensor-copy paths below; every other path expands the weights again (still correct)
   const bool w_prepared = (flags & HBMM_CONV_WEIGHTS_PREPARED) != 0;
@@ -385,7 +448,20 @@ hbmm_status hbmm_conv_im2col_ex(const void* x, int32_t x_dtype, const hbmm_conv_
   const ConvLayout L = conv_layout(cg, beta_a, a_scale_dtype, W);
   if (W->K != L.K) return HBMM_ERR_INVALID_ARG;
   if (beta_a >= 2 && !beta_supported(L.K, beta_a)) return HBMM_ERR_UNSUPPORTED;
-  if (!pack_only && (st = check_c(C_out, ldc, W->rows)) != HBMM_OK) return st;
+  EpiArgs epi = plain_epilogue();
+  if (ep) {
+    if ((st = make_epilogue(ep, L.M, W->rows, &epi)) != HBMM_OK) return st;
+    if (epi.mode == kEpiPacked && !gemm_fold_next_supported(W->rows, epi.nx_beta)) return HBMM_ERR_UNSUPPORTED;
+  } else if (!pack_only && (st = check_c(C_out, ldc, W->rows)) != HBMM_OK) {
+    return st;
+  }
+  if (input_nhwc) {
+    // an NHWC bf16 image (what a dense-output epilogue of the layer before wrote): the dense-activation
+    // tensor-core path reads it as it is
+    if (beta_a != 1 || x_dtype != HBMM_BF16) return HBMM_ERR_INVALID_ARG;
+    if (!L.implicit || L.Cp != cg.C) return HBMM_ERR_UNSUPPORTED;
+    if (reinterpret_cast<uintptr_t>(x) % 16 != 0) return HBMM_ERR_ALIGNMENT;
+  }
   if (!workspace || workspace_bytes < L.total) return HBMM_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return HBMM_ERR_ALIGNMENT;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -393,9 +469,11 @@ hbmm_status hbmm_conv_im2col_ex(const void* x, int32_t x_dtype, const hbmm_conv_
   A.rows = L.M; A.K = L.K; A.beta = beta_a; A.scale_dtype = a_scale_dtype;
   if (beta_a == 1 && L.implicit) {
     return launch_hbwn_umma_conv(x, x_dtype == HBMM_BF16, workspace, L.Cp, cg, view_of(W), C_out, ldc,
-                                 static_cast<char*>(workspace) + L.operand_bytes, s, w_prepared) == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
+                                 static_cast<char*>(workspace) + L.operand_bytes, s, w_prepared, ep ? &epi : nullptr,
+                                 input_nhwc) == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
   }
   if (beta_a == 1) {
+    if (ep) return HBMM_ERR_UNSUPPORTED;       // the epilogue chain needs the implicit tensor-core path (whole 64-channel blocks)
     if (launch_im2col_bf16(x, x_dtype == HBMM_BF16, cg, workspace, L.ld_dense, s) != cudaSuccess) return HBMM_ERR_CUDA;
     A.dense = workspace; A.ld_dense = L.ld_dense; A.dense_dtype = HBMM_BF16;
   } else {
@@ -408,7 +486,12 @@ hbmm_status hbmm_conv_im2col_ex(const void* x, int32_t x_dtype, const hbmm_conv_
     // front end's launch also expands the weight operand (a few extra CTAs) and the contraction skips it.
     const PackedView av = view_of(&A), wv = view_of(W);
     void* gemm_ws = static_cast<char*>(workspace) + L.operand_bytes;
-    if (prefer_fold(av, wv) && L.gemm_bytes > 0 && L.gemm_bytes >= fold_workspace(av, wv) &&
+    if (ep) {
+      // the epilogue chain lives in the folded-scale kernel: activation groups of whole words, K in whole words
+      const bool a_subword = beta_a < 32 && beta_a < L.K;
+      if (!gemm_fold_supported(av, wv) || a_subword || L.gemm_bytes < fold_workspace(av, wv)) return HBMM_ERR_UNSUPPORTED;
+    }
+    if ((ep || prefer_fold(av, wv)) && L.gemm_bytes > 0 && L.gemm_bytes >= fold_workspace(av, wv) &&
         im2col_quantize_tma_supported(x, x_dtype == HBMM_BF16, cg, beta_a)) {
       UmmaPrepJob job{};
       gemm_fold_prep_job(av, wv, gemm_ws, &job);
@@ -417,16 +500,22 @@ hbmm_status hbmm_conv_im2col_ex(const void* x, int32_t x_dtype, const hbmm_conv_
                                        w_prepared ? nullptr : &job) != cudaSuccess)
           return HBMM_ERR_CUDA;
         if (pack_only) return HBMM_OK;
-        return launch_gemm_fold(av, wv, C_out, ldc, gemm_ws, s, true) == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
+        return launch_gemm_fold(av, wv, C_out, ldc, gemm_ws, s, true, ep ? &epi : nullptr) == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
       }
     }
     if (launch_im2col_quantize(x, x_dtype == HBMM_BF16, cg, beta_a, A.bits, A.ld_words, A.scales, A.ld_scales,
                                a_scale_dtype == HBMM_BF16, s) != cudaSuccess)
       return HBMM_ERR_CUDA;
     if (pack_only) return HBMM_OK;
+    if (ep)
+      return launch_gemm_fold(av, wv, nullptr, 0, gemm_ws, s, w_prepared, &epi) == cudaSuccess ? HBMM_OK : HBMM_ERR_CUDA;
   }
   return gemm_checked(&A, W, C_out, ldc, HBMM_PATH_AUTO, static_cast<char*>(workspace) + L.operand_bytes, L.gemm_bytes, s);
 }
+
+}  // namespace
+
+extern "C" {
 
 hbmm_status hbmm_last_device_error(int32_t* code) {
   int c = 0;

@@ -38,6 +38,7 @@
 #include "kernels.h"
 #include "umma_common.cuh"
 #include "gemm_fold_prep.cuh"
+#include "epilogue.cuh"
 #include "pdl.cuh"
 
 namespace hbmm {
@@ -63,50 +64,6 @@ prepare_w_fold_kernel(const Args g, unsigned char* __restrict__ out, float* __re
   prepare_w_task<TN>(g, out, w_down, blockIdx.x, blockIdx.y, threadIdx.x);
 }
 
-__device__ __forceinline__ void store_next_scale(void* s, int bf16, int64_t idx, float v) {
-  if (bf16) reinterpret_cast<__nv_bfloat16*>(s)[idx] = __float2bfloat16_rn(v);
-  else reinterpret_cast<float*>(s)[idx] = v;
-}
-
-// Fused epilogue: 32 consecutive columns of one row of z (columns n0 .. n0 + 31, `valid` of them inside the
-// output) become one packed word (bit e = 1 <=> z[e] >= 0, -0 counting as +0; bits of absent columns 0) and
-// the scales of the groups that end inside the chunk (mean |z| over the group's columns inside the output).
-// BETA > 32: the chunk's |z| sum is added to `carry`, and the group is closed by its last chunk.
-template <int BETA>
-__device__ __forceinline__ void emit_next_chunk(const float (&z)[32], int valid, int64_t n0, int64_t N, uint32_t* bits_row, void* scales,
-                                                int bf16, int64_t srow, int64_t ld_scales, float& carry) {
-  uint32_t neg = 0;
-#pragma unroll
-  for (int e = 31; e >= 0; e--) neg = __funnelshift_l(__float_as_uint(z[e] + 0.0f), neg, 1);
-  const uint32_t vmask = valid >= 32 ? 0xFFFFFFFFu : (valid <= 0 ? 0u : ((1u << valid) - 1u));
-  bits_row[n0 >> 5] = ~neg & vmask;
-  float a[16];                                            // pairwise tree of |z|, first level formed on the fly
-#pragma unroll
-  for (int e = 0; e < 16; e++)
-    a[e] = (2 * e < valid ? fabsf(z[2 * e]) : 0.0f) + (2 * e + 1 < valid ? fabsf(z[2 * e + 1]) : 0.0f);
-  constexpr int SPAN = (BETA < 32 ? BETA : 32) / 2;       // pairs per group inside the chunk
-#pragma unroll
-  for (int w = 1; w < SPAN; w <<= 1)
-#pragma unroll
-    for (int e = 0; e < 16; e += 2 * w) a[e] += a[e + w];
-  if constexpr (BETA <= 32) {
-#pragma unroll
-    for (int gi = 0; gi < 32 / BETA; gi++) {
-      const int64_t gidx = n0 / BETA + gi;
-      const int cnt = valid - gi * BETA < BETA ? valid - gi * BETA : BETA;
-      if (gidx < ld_scales) store_next_scale(scales, bf16, srow + gidx, cnt > 0 ? a[gi * SPAN] / static_cast<float>(cnt) : 0.0f);
-    }
-  } else {
-    carry += a[0];
-    if ((n0 + 32) % BETA == 0) {
-      const int64_t g0 = n0 + 32 - BETA, gidx = g0 / BETA;
-      const int64_t cnt = N - g0 < BETA ? N - g0 : BETA;
-      if (gidx < ld_scales) store_next_scale(scales, bf16, srow + gidx, cnt > 0 ? carry / static_cast<float>(cnt) : 0.0f);
-      carry = 0.0f;
-    }
-  }
-}
-
 // Walks the stages a producer thread owns (every second stage of the CTA's stream of tiles) and keeps
 // the row pointers of the tile it is in.
 struct StageCursor {
@@ -117,7 +74,8 @@ struct StageCursor {
 };
 
 // ASUB: scale groups per packed word of A (1: groups of whole words; 2 .. 16: beta_a = 16 .. 2).
-// FUSE: the epilogue binarizes the (affinely mapped) output rows for the next layer instead of storing them.
+// FUSE: the epilogue runs the activation / affine map / dense or binarized output chain of epilogue.cuh instead of
+// storing the product as fp32.
 template <int TN, int ASUB, bool FUSE>
 __global__ void __launch_bounds__(kThreads, 1)
 hbmm_fold_kernel(const Args g) {
@@ -401,8 +359,8 @@ hbmm_fold_kernel(const Args g) {
       for (int i = 0; i < TN / 32; i++) {
         const int64_t n = nb + i * 32 + lane;
         fcol[i] = __ldg(g.w_down + n);                                                     // w_down holds a whole number of tiles
-        fsc[i] = (FUSE && g.bn_scale && n < g.N) ? __ldg(g.bn_scale + n) : 1.0f;
-        fsh[i] = (FUSE && g.bn_shift && n < g.N) ? __ldg(g.bn_shift + n) : 0.0f;
+        fsc[i] = (FUSE && g.ep.bn_scale && n < g.N) ? __ldg(g.ep.bn_scale + n) : 1.0f;
+        fsh[i] = (FUSE && g.ep.bn_shift && n < g.N) ? __ldg(g.ep.bn_shift + n) : 0.0f;
       }
       if (!mbar_wait(&tfull[buf], static_cast<uint32_t>((ti >> 1) & 1), abort_flag, 5)) break;
       if (!mbar_wait(&rowfull[slot], static_cast<uint32_t>((ti / kRowSlots) & 1), abort_flag, 5)) break;   // long complete
@@ -437,36 +395,22 @@ hbmm_fold_kernel(const Args g) {
         }
         if constexpr (FUSE) {
           if (m < g.M) {
-          // affine map per column, then the row is binarized for the next layer: packed word + group scales
-          float z[32];
+            // the product of the chunk's 32 columns, then activation, affine map and dense or binarized output
+            float cv[32], fs[32], fh[32];
 #pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            const float4 fw = *reinterpret_cast<const float4*>(cf + c * 32 + j);
-            const float4 bs = *reinterpret_cast<const float4*>(cf + TN + c * 32 + j);
-            const float4 bh = *reinterpret_cast<const float4*>(cf + 2 * TN + c * 32 + j);
-            const float w4[4] = {fw.x, fw.y, fw.z, fw.w}, s4[4] = {bs.x, bs.y, bs.z, bs.w}, h4[4] = {bh.x, bh.y, bh.z, bh.w};
+            for (int j = 0; j < 32; j += 4) {
+              const float4 fw = *reinterpret_cast<const float4*>(cf + c * 32 + j);
+              const float4 bs = *reinterpret_cast<const float4*>(cf + TN + c * 32 + j);
+              const float4 bh = *reinterpret_cast<const float4*>(cf + 2 * TN + c * 32 + j);
+              const float w4[4] = {fw.x, fw.y, fw.z, fw.w}, s4[4] = {bs.x, bs.y, bs.z, bs.w}, h4[4] = {bh.x, bh.y, bh.z, bh.w};
 #pragma unroll
-            for (int e = 0; e < 4; e++)
-              z[j + e] = fmaf(__uint_as_float(v1[j + e]) * fa * w4[e], s4[e], h4[e]);
-          }
-          const int64_t n0 = nb + c * 32;
-          const int valid = g.N - n0 >= 32 ? 32 : static_cast<int>(g.N - n0 > 0 ? g.N - n0 : 0);
-          uint32_t* brow = g.nx_bits + m * g.nx_ld_words;
-          const int64_t srow = m * g.nx_ld_scales;
-          switch (g.nx_beta) {
-            case 2: emit_next_chunk<2>(z, valid, n0, g.N, brow, g.nx_scales, g.nx_bf16, srow, g.nx_ld_scales, carry); break;
-            case 4: emit_next_chunk<4>(z, valid, n0, g.N, brow, g.nx_scales, g.nx_bf16, srow, g.nx_ld_scales, carry); break;
-            case 8: emit_next_chunk<8>(z, valid, n0, g.N, brow, g.nx_scales, g.nx_bf16, srow, g.nx_ld_scales, carry); break;
-            case 16: emit_next_chunk<16>(z, valid, n0, g.N, brow, g.nx_scales, g.nx_bf16, srow, g.nx_ld_scales, carry); break;
-            case 32: emit_next_chunk<32>(z, valid, n0, g.N, brow, g.nx_scales, g.nx_bf16, srow, g.nx_ld_scales, carry); break;
-            case 64: emit_next_chunk<64>(z, valid, n0, g.N, brow, g.nx_scales, g.nx_bf16, srow, g.nx_ld_scales, carry); break;
-            default: emit_next_chunk<128>(z, valid, n0, g.N, brow, g.nx_scales, g.nx_bf16, srow, g.nx_ld_scales, carry); break;
-          }
-          if (c == TN / 32 - 1 && nb + TN >= g.N) {
-            // last column tile: the row's zero padding past what the tiles cover
-            for (int64_t wz = (nb + TN) >> 5; wz < g.nx_ld_words; wz++) brow[wz] = 0u;
-            for (int64_t sz = (nb + TN) / g.nx_beta; sz < g.nx_ld_scales; sz++) store_next_scale(g.nx_scales, g.nx_bf16, srow + sz, 0.0f);
-          }
+              for (int e = 0; e < 4; e++) {
+                cv[j + e] = __uint_as_float(v1[j + e]) * fa * w4[e];
+                fs[j + e] = s4[e];
+                fh[j + e] = h4[e];
+              }
+            }
+            epi::finish_chunk(g.ep, cv, fs, fh, m, nb + c * 32, g.N, c == TN / 32 - 1, nb + TN, carry);
           }
         } else if (m < g.M) {
 #pragma unroll
@@ -531,9 +475,7 @@ Args make_args(const PackedView& A, const PackedView& W, float* C, int64_t ldc) 
   g.w_gw = W.beta >= W.K ? g.n_words : (w_subword ? 1 : W.beta / 32);
   g.w_prep = nullptr;
   g.w_down = nullptr;
-  g.fuse = 0; g.nx_bf16 = 0; g.nx_beta = 32; g.nx_pad = 0;
-  g.bn_scale = nullptr; g.bn_shift = nullptr; g.nx_bits = nullptr; g.nx_scales = nullptr;
-  g.nx_ld_words = 0; g.nx_ld_scales = 0;
+  g.ep = plain_epilogue();
   return g;
 }
 
@@ -574,7 +516,7 @@ cudaError_t launch_fold(Args g, void* workspace, cudaStream_t stream, bool w_pre
 
 template <int TN>
 cudaError_t launch_fold_tn(const Args& g, void* workspace, cudaStream_t stream, bool w_prepared) {
-  if (g.fuse) {      // the fused epilogue is built for activation groups of whole words
+  if (g.ep.mode != kEpiPlain) {      // the fused epilogue is built for activation groups of whole words
     if (g.a_sub != 1) return cudaErrorNotSupported;
     return launch_fold<TN, 1, true>(g, workspace, stream, w_prepared);
   }
@@ -613,13 +555,9 @@ bool gemm_fold_next_supported(int64_t N, int32_t beta_next) {
 }
 
 cudaError_t launch_gemm_fold(const PackedView& A, const PackedView& W, float* C, int64_t ldc, void* workspace,
-                             cudaStream_t stream, bool w_prepared, const FoldNext* next) {
+                             cudaStream_t stream, bool w_prepared, const EpiArgs* ep) {
   Args g = make_args(A, W, C, ldc);
-  if (next) {
-    g.fuse = 1; g.nx_bf16 = next->scale_bf16; g.nx_beta = next->beta;
-    g.bn_scale = next->bn_scale; g.bn_shift = next->bn_shift; g.nx_bits = next->bits; g.nx_scales = next->scales;
-    g.nx_ld_words = next->ld_words; g.nx_ld_scales = next->ld_scales;
-  }
+  if (ep) g.ep = *ep;
   return g.N <= 64 ? launch_fold_tn<64>(g, workspace, stream, w_prepared) : launch_fold_tn<128>(g, workspace, stream, w_prepared);
 }
 

@@ -26,6 +26,7 @@
 #include "tensor_map.h"
 #include "nhwc.cuh"
 #include "umma_common.cuh"
+#include "epilogue.cuh"
 #include "pdl.cuh"
 
 namespace hbmm {
@@ -52,6 +53,7 @@ struct Args {
   // k = c * taps + tap (channel slowest, Section 3.1.1).
   int32_t conv, taps, kw, cblocks, Cin;
   int32_t HoWo, Wo, sh, sw, ph, pw;
+  EpiArgs ep;                     // what the epilogue does with a finished tile (plain: store C as fp32)
 };
 
 __device__ __forceinline__ float load_scale(const void* s, int bf16, int64_t idx) {
@@ -322,6 +324,7 @@ hbwn_umma_kernel(const Args g, const __grid_constant__ CUtensorMap a_map) {
       const int64_t tile = blockIdx.x + ti * gridDim.x;
       const int64_t m = (tile / tiles_n) * TM + row, nb = (tile % tiles_n) * TN;
       float* dst = g.C + m * g.ldc + nb;
+      float carry = 0.0f;                                   // |z| sum of a next-layer group wider than a 32-column chunk
 #pragma unroll
       for (int c = 0; c < TN / 32; c++) {
         uint32_t v[NP][32];
@@ -329,7 +332,21 @@ hbwn_umma_kernel(const Args g, const __grid_constant__ CUtensorMap a_map) {
 #pragma unroll
         for (int i = 0; i < NP; i++) tmem_ld32(t_addr + i * TN, v[i]);
         tmem_ld_wait();
-        if (m < g.M) {
+        if (m < g.M && g.ep.mode != kEpiPlain) {
+          // activation, affine map, then a dense (fp32 / bf16) or binarized row instead of the fp32 product
+          float cv[32], fs[32], fh[32];
+#pragma unroll
+          for (int e = 0; e < 32; e++) {
+            float acc = __uint_as_float(v[NP - 1][e]);
+#pragma unroll
+            for (int i = NP - 2; i >= 0; i--) acc += __uint_as_float(v[i][e]);
+            cv[e] = acc;
+            const int64_t n = nb + c * 32 + e;
+            fs[e] = (g.ep.bn_scale && n < g.N) ? __ldg(g.ep.bn_scale + n) : 1.0f;
+            fh[e] = (g.ep.bn_shift && n < g.N) ? __ldg(g.ep.bn_shift + n) : 0.0f;
+          }
+          epi::finish_chunk(g.ep, cv, fs, fh, m, nb + c * 32, g.N, c == TN / 32 - 1, nb + TN, carry);
+        } else if (m < g.M) {
 #pragma unroll
           for (int j = 0; j < 32; j += 4) {
             float o[4];
@@ -376,6 +393,7 @@ Args make_args(const DenseView& A, const PackedView& W, float* C, int64_t ldc) {
   g.n_kb = (g.K + KB - 1) / KB;
   g.conv = 0; g.taps = 1; g.kw = 1; g.cblocks = static_cast<int32_t>(g.n_kb); g.Cin = 0;
   g.HoWo = 1; g.Wo = 1; g.sh = g.sw = 1; g.ph = g.pw = 0;
+  g.ep = plain_epilogue();
   return g;
 }
 
@@ -429,6 +447,7 @@ Args make_conv_args(const ConvGeom& c, const PackedView& W, float* C, int64_t ld
   g.conv = 1; g.taps = c.kh * c.kw; g.kw = c.kw; g.cblocks = (c.C + KB - 1) / KB; g.Cin = c.C;
   g.n_kb = static_cast<int64_t>(g.taps) * g.cblocks;
   g.HoWo = c.Ho * c.Wo; g.Wo = c.Wo; g.sh = c.sh; g.sw = c.sw; g.ph = c.ph; g.pw = c.pw;
+  g.ep = plain_epilogue();
   return g;
 }
 
@@ -494,8 +513,9 @@ size_t hbwn_umma_workspace_bytes(const DenseView& A, const PackedView& W) {
 }
 
 cudaError_t launch_hbwn_umma(const DenseView& A, const PackedView& W, float* C, int64_t ldc, void* workspace,
-                             cudaStream_t stream, bool w_prepared, bool exact) {
-  const Args g = make_args(A, W, C, ldc);
+                             cudaStream_t stream, bool w_prepared, bool exact, const EpiArgs* ep) {
+  Args g = make_args(A, W, C, ldc);
+  if (ep) g.ep = *ep;
   CUtensorMap a_map;
   if (!make_a_map(g, &a_map)) return cudaErrorNotSupported;
   return launch_any(g, a_map, workspace, stream, nullptr, w_prepared, exact);
@@ -516,9 +536,16 @@ size_t hbwn_umma_conv_workspace_bytes(const ConvGeom& c, const PackedView& W) {
 }
 
 cudaError_t launch_hbwn_umma_conv(const void* x, int x_bf16, void* x_nhwc, int Cp, const ConvGeom& c, const PackedView& W, float* C,
-                                  int64_t ldc, void* workspace, cudaStream_t stream, bool w_prepared) {
-  const Args g = make_conv_args(c, W, C, ldc);
+                                  int64_t ldc, void* workspace, cudaStream_t stream, bool w_prepared, const EpiArgs* ep,
+                                  bool input_is_nhwc) {
+  Args g = make_conv_args(c, W, C, ldc);
+  if (ep) g.ep = *ep;
   CUtensorMap a_map;
+  if (input_is_nhwc) {
+    // the caller's tensor already is the NHWC bf16 image the tensor copies read (channel pitch Cp): no layout copy
+    if (!make_conv_map(x, c, Cp, &a_map)) return cudaErrorNotSupported;
+    return launch_any(g, a_map, workspace, stream, nullptr, w_prepared, false);
+  }
   if (!make_conv_map(x_nhwc, c, Cp, &a_map)) return cudaErrorNotSupported;
   CopyArgs cp;
   cp.x = x; cp.x_bf16 = x_bf16; cp.C = c.C; cp.Cp = Cp; cp.HW = static_cast<int64_t>(c.H) * c.W;

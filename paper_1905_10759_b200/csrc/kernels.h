@@ -81,6 +81,22 @@ cudaError_t launch_gemm_b1(const PackedView& A, const PackedView& W, float* C, i
 cudaError_t launch_partials_b1(const PackedView& A, const PackedView& W, int32_t* D,
                                cudaStream_t stream);
 
+// What a tensor-core contraction does with a finished product tile besides storing it as fp32 (the chain of the
+// paper's layer order, Section 5: convolution -> activation -> batch normalisation -> binarization of the next block):
+//   y = act(C), z = bn_scale[n] * y + bn_shift[n], then z stored dense (fp32 or bf16, [M, ld_out]) or each row of z
+//   Hadamard-binarized along n (Eq. 3-4) and only its packed form stored.
+enum EpiMode : int32_t { kEpiPlain = 0, kEpiDense = 1, kEpiPacked = 2 };
+struct EpiArgs {
+  int32_t mode;             // EpiMode
+  int32_t act;              // 0 none, 1 max(0, .)
+  const float* bn_scale; const float* bn_shift;      // device, per column; null = 1 / 0
+  void* out; int32_t out_bf16; int64_t ld_out;       // dense
+  uint32_t* nx_bits; void* nx_scales;                // packed: the next layer's operand (rows = M, K = N)
+  int64_t nx_ld_words, nx_ld_scales;
+  int32_t nx_bf16, nx_beta;
+};
+inline EpiArgs plain_epilogue() { EpiArgs e{}; e.mode = kEpiPlain; e.nx_beta = 32; return e; }
+
 // Argument block of the tcgen05 HBMM kernel and of its weight-expansion routine.
 struct UmmaArgs {
   const uint32_t* a_bits; const void* a_scales;
@@ -106,19 +122,7 @@ struct FoldArgs {
   int32_t a_sub, w_sub;    // scale groups per K-word: 1, or 32 / beta for the sub-word groups beta = 2 .. 16
   const unsigned char* w_prep;   // W expanded into [n tile][stage][stage bytes]
   const float* w_down;           // per weight row: the power of two that undoes its normalisation
-  // Fused epilogue (fuse != 0): z = bn_scale[n] * C + bn_shift[n] is Hadamard-binarized along n for the next
-  // layer and only its packed form is written (C is ignored).
-  int32_t fuse, nx_bf16, nx_beta, nx_pad;
-  const float* bn_scale; const float* bn_shift;      // per column; null = 1 / 0
-  uint32_t* nx_bits; void* nx_scales;
-  int64_t nx_ld_words, nx_ld_scales;
-};
-// Where the fused epilogue of the folded kernel writes the next layer's operand.
-struct FoldNext {
-  const float* bn_scale; const float* bn_shift;
-  uint32_t* bits; void* scales;
-  int64_t ld_words, ld_scales;
-  int32_t scale_bf16, beta;
+  EpiArgs ep;                    // what the epilogue does with a finished tile (ep.mode == kEpiPlain: store C as fp32)
 };
 // The weight expansion as a job another kernel can run: n_stages x tiles_n tasks of tn threads each
 // (n_stages counts tasks per column tile: single stages of the e4m3 layout, runs of stages of the folded one).
@@ -155,7 +159,7 @@ cudaError_t launch_wait_expiry_selftest(cudaStream_t stream);
 bool gemm_fold_supported(const PackedView& A, const PackedView& W);
 size_t gemm_fold_workspace_bytes(const PackedView& A, const PackedView& W);
 cudaError_t launch_gemm_fold(const PackedView& A, const PackedView& W, float* C, int64_t ldc, void* workspace,
-                             cudaStream_t stream, bool w_prepared = false, const FoldNext* next = nullptr);
+                             cudaStream_t stream, bool w_prepared = false, const EpiArgs* ep = nullptr);
 // Group sizes the fused epilogue can emit for an output of N columns.
 bool gemm_fold_next_supported(int64_t N, int32_t beta_next);
 void gemm_fold_prep_job(const PackedView& A, const PackedView& W, void* workspace, UmmaPrepJob* job);
@@ -172,7 +176,7 @@ bool hbwn_umma_supported(const DenseView& A, const PackedView& W);
 size_t hbwn_umma_workspace_bytes(const DenseView& A, const PackedView& W);
 // exact: three bf16 pieces per weight (group scale to 2^-26); otherwise two (2^-17), the faster layout.
 cudaError_t launch_hbwn_umma(const DenseView& A, const PackedView& W, float* C, int64_t ldc, void* workspace,
-                             cudaStream_t stream, bool w_prepared = false, bool exact = false);
+                             cudaStream_t stream, bool w_prepared = false, bool exact = false, const EpiArgs* ep = nullptr);
 
 // HBWN convolution without the im2col matrix: NCHW -> NHWC bf16 copy (Cp = channels rounded up to 8;
 // launch_hbwn_umma_conv does it in the same launch as the weight-piece layout), then the tcgen05 kernel
@@ -181,8 +185,11 @@ cudaError_t launch_nchw_to_nhwc_bf16(const void* x, int x_bf16, const ConvGeom& 
 bool hbwn_umma_conv_supported(const ConvGeom& g, const PackedView& W);
 size_t hbwn_umma_conv_workspace_bytes(const ConvGeom& g, const PackedView& W);
 // w_prepared: the workspace still holds the weight pieces an earlier call with the same W and geometry laid out.
+// ep (optional): epilogue chain instead of the fp32 store.  input_is_nhwc: x already is an NHWC bf16 image with
+// channel pitch Cp (16-byte aligned), so the layout copy is skipped and x_nhwc is not used.
 cudaError_t launch_hbwn_umma_conv(const void* x, int x_bf16, void* x_nhwc, int Cp, const ConvGeom& g, const PackedView& W, float* C,
-                                  int64_t ldc, void* workspace, cudaStream_t stream, bool w_prepared = false);
+                                  int64_t ldc, void* workspace, cudaStream_t stream, bool w_prepared = false,
+                                  const EpiArgs* ep = nullptr, bool input_is_nhwc = false);
 
 // im2col gather fused with Hadamard binarization (packed output), and bf16 dense gather.
 cudaError_t launch_im2col_quantize(const void* x, int x_bf16, const ConvGeom& g, int32_t beta,

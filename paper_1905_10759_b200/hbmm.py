@@ -34,6 +34,7 @@ EXPORTS = [
     "hbmm_version", "hbmm_conv_im2col_static", "hbmm_last_device_error", "hbmm_conv_im2col_ex",
     "hbmm_binarize_backward", "hbmm_gemm_binarize_next", "hbmm_binarize_dense",
     "hbmm_clear_device_error", "hbmm_debug_set_wait_limit", "hbmm_debug_expire_wait", "hbmm_bench_alu_rate",
+    "hbmm_gemm_fused", "hbmm_conv_im2col_fused",
 ]
 STATIC_SCRATCH_BYTES = 32 << 20
 
@@ -226,6 +227,9 @@ def conv_workspace_bytes(geom: hbmm_conv_geom, beta_a: int, a_scale_dtype: int, 
 
 CONV_WEIGHTS_PREPARED = 1
 CONV_PACK_ONLY = 2
+CONV_INPUT_NHWC = 4
+ACT_NONE, ACT_RELU = 0, 1
+OUT_DENSE, OUT_PACKED = 1, 2
 
 _lib.hbmm_binarize_backward.argtypes = [_vp, _i64, _vp, _i64, _i64, _i64, _i32, _vp, _i64, _vp]
 _lib.hbmm_binarize_backward.restype = _i32
@@ -359,3 +363,56 @@ def bench_alu_rate(kind: int, blocks: int, iters: int, sink: torch.Tensor, strea
     ops = _i64(0)
     _check(_lib.hbmm_bench_alu_rate(kind, blocks, iters, _dev_ptr(sink), ctypes.byref(ops), _stream(stream)), "hbmm_bench_alu_rate")
     return int(ops.value)
+
+
+class hbmm_epilogue(ctypes.Structure):
+    _fields_ = [
+        ("activation", ctypes.c_int32), ("out_kind", ctypes.c_int32),
+        ("bn_scale", ctypes.c_void_p), ("bn_shift", ctypes.c_void_p),
+        ("out", ctypes.c_void_p), ("ld_out", ctypes.c_int64),
+        ("out_dtype", ctypes.c_int32), ("reserved", ctypes.c_int32),
+        ("next", ctypes.POINTER(hbmm_operand)),
+    ]
+
+
+_lib.hbmm_gemm_fused.argtypes = [_P(hbmm_operand), _P(hbmm_operand), _P(hbmm_epilogue), _vp, _sz, _vp]
+_lib.hbmm_gemm_fused.restype = _i32
+_lib.hbmm_conv_im2col_fused.argtypes = [_vp, _i32, _P(hbmm_conv_geom), _i32, _i32, _P(hbmm_operand), _P(hbmm_epilogue), _vp, _sz,
+                                        ctypes.c_uint32, _vp]
+_lib.hbmm_conv_im2col_fused.restype = _i32
+
+
+def make_epilogue(activation: int = ACT_NONE, bn_scale: Optional[torch.Tensor] = None, bn_shift: Optional[torch.Tensor] = None,
+                  out: Optional[torch.Tensor] = None, nxt: Optional[Operand] = None) -> hbmm_epilogue:
+    """Fills an hbmm_epilogue: `out` (a dense [M, N] fp32 / bf16 device tensor with contiguous rows) selects
+    HBMM_OUT_DENSE, `nxt` (a packed operand) HBMM_OUT_PACKED.  Marshalling only."""
+    ep = hbmm_epilogue()
+    ep.activation = activation
+    ep.bn_scale = _dev_ptr(bn_scale) if bn_scale is not None else None
+    ep.bn_shift = _dev_ptr(bn_shift) if bn_shift is not None else None
+    if (out is None) == (nxt is None):
+        raise ValueError("exactly one of out / nxt")
+    if out is not None:
+        ep.out_kind = OUT_DENSE
+        ep.out, ep.ld_out, ep.out_dtype = out.data_ptr(), out.stride(0), _dtype_code(out.dtype)
+    else:
+        ep.out_kind = OUT_PACKED
+        ep.next = ctypes.pointer(nxt.desc)
+    ep._keep_alive = (bn_scale, bn_shift, out, nxt)      # the struct holds raw pointers: keep their owners alive with it
+    return ep
+
+
+def gemm_fused(A: Operand, W: Operand, ep: hbmm_epilogue, workspace: torch.Tensor, stream=None) -> None:
+    """hbmm_gemm_fused: the product goes through activation, affine map and dense / binarized output in the epilogue."""
+    _check(_lib.hbmm_gemm_fused(ctypes.byref(A.desc), ctypes.byref(W.desc), ctypes.byref(ep), _dev_ptr(workspace),
+                                workspace.numel() * workspace.element_size(), _stream(stream)), "hbmm_gemm_fused")
+
+
+def conv_im2col_fused(x: torch.Tensor, geom: hbmm_conv_geom, beta_a: int, a_scale_dtype: int, W: Operand, ep: hbmm_epilogue,
+                      workspace: torch.Tensor, stream=None, flags: int = 0) -> None:
+    """hbmm_conv_im2col_fused: x NCHW contiguous (or NHWC bf16 with CONV_INPUT_NHWC)."""
+    if not x.is_contiguous():
+        raise ValueError("x must be contiguous")
+    _check(_lib.hbmm_conv_im2col_fused(_dev_ptr(x), _dtype_code(x.dtype), ctypes.byref(geom), beta_a, a_scale_dtype,
+                                       ctypes.byref(W.desc), ctypes.byref(ep), _dev_ptr(workspace),
+                                       workspace.numel() * workspace.element_size(), flags, _stream(stream)), "hbmm_conv_im2col_fused")

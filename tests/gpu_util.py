@@ -116,3 +116,29 @@ def signs_of_words(bits: np.ndarray, K: int) -> np.ndarray:
     Plain numpy bit unpacking, independent of the library and of the oracle's packer."""
     b = np.unpackbits(np.ascontiguousarray(bits).view(np.uint8), axis=1, bitorder="little")[:, :K]
     return b.astype(np.float32) * 2.0 - 1.0
+
+
+def check_next_operand(nxt, z_ref: np.ndarray, band: np.ndarray, bn: int, bf16_scales: bool):
+    """A packed operand written by a fused epilogue against the reference rows z_ref (double): signs where |z| is
+    outside the product's own error band (inside it the fp32 value the kernel computed decides), more than 99 %
+    of them decided; exact zero padding; every group scale to the band's mean over the group plus the rounding
+    of a pairwise fp32 tree (and of bf16 storage)."""
+    import oracle
+    M, N = z_ref.shape
+    bits = host_bits(nxt.bits)
+    lw = bits.shape[1]
+    got_sign = ((bits[:, np.arange(N) // 32] >> (np.arange(N) % 32).astype(np.uint32)) & 1).astype(np.int8) * 2 - 1
+    want_sign = np.where(z_ref >= 0, 1, -1)
+    decided = np.abs(z_ref) > band
+    assert (got_sign[decided] == want_sign[decided]).all()
+    assert decided.mean() > 0.99
+    assert np.array_equal(bits, oracle.pack(got_sign.astype(np.int8), lw))       # bits past N and words past ceil(N / 32) are zero
+    G = -(-N // bn)
+    sc = nxt.scales.float().cpu().numpy().astype(np.float64)
+    assert np.all(sc[:, G:] == 0.0)
+    tree = (int(np.ceil(np.log2(bn))) + 3) * U + (2.0 ** -8 if bf16_scales else 0.0)
+    for g in range(G):
+        sl = slice(g * bn, min((g + 1) * bn, N))
+        want = np.abs(z_ref[:, sl]).mean(axis=1)
+        tol = band[:, sl].mean(axis=1) + tree * want
+        assert (np.abs(sc[:, g] - want) <= tol).all(), g

@@ -203,3 +203,46 @@ def test_resnet_conv_of_map_binarized_activations_full_batch(hb, li, beta_a):
         c_ref, absref = oracle.conv_map_binarized(x[b:b + 1], w, s.kh, s.kw, (s.stride, s.stride), (s.pad, s.pad), beta_a, BETA)
         lo = b * per_image
         gu.assert_close_rel_absref(C[lo: lo + per_image].cpu().numpy(), c_ref, absref, rtol, "%s image %d" % (s.name, b))
+
+
+# ------------------------------------------------------------------ two layers chained through the epilogue, batch 64
+def test_conv3_chain_through_the_epilogue_full_batch(hb):
+    """conv3_x -> ReLU -> the next block's batch-norm map -> NHWC bf16 (all in the first contraction's epilogue), then a
+    second conv3_x that reads that tensor directly (HBMM_CONV_INPUT_NHWC).  Three whole images are redone by the
+    oracle: layer 1 from the raw input, layer 2 from exactly the values layer 1 stored."""
+    gu = _gu()
+    s = inputs.resnet18_convs(64)[1]
+    B, C, H, N = s.B, s.C, s.H, s.N
+    x = inputs.conv_activation(s, inputs.SEEDS["resnet_hbwn"][0] + 70, signed=True)
+    xb_bits, xb = inputs.as_bf16(x)
+    w1 = inputs.he_normal(N, s.K, inputs.SEEDS["resnet_hbmm"][1] + 70)
+    w2 = inputs.he_normal(N, N * 9, inputs.SEEDS["resnet_hbmm"][1] + 71)
+    W1 = hb.quantize(torch.from_numpy(w1).cuda(), hb.alloc_operand(N, s.K, BETA, hb.F32))
+    W2 = hb.quantize(torch.from_numpy(w2).cuda(), hb.alloc_operand(N, N * 9, BETA, hb.F32))
+    rng = np.random.default_rng(70)
+    bs = rng.uniform(0.5, 2.0, N).astype(np.float32)
+    bh = (0.2 * rng.standard_normal(N)).astype(np.float32)
+    geom = hb.make_geom(B, C, H, H, 3, 3, (1, 1), (1, 1))
+    ws1 = torch.empty(hb.conv_workspace_bytes(geom, 1, hb.F32, W1), dtype=torch.uint8, device="cuda")
+    ws2 = torch.empty(hb.conv_workspace_bytes(geom, 1, hb.F32, W2), dtype=torch.uint8, device="cuda")
+    z = torch.empty((s.M, N), device="cuda", dtype=torch.bfloat16)
+    ep = hb.make_epilogue(hb.ACT_RELU, torch.from_numpy(bs).cuda(), torch.from_numpy(bh).cuda(), out=z)
+    xd = torch.from_numpy(xb_bits.view(np.int16)).view(torch.bfloat16).cuda()
+    hb.conv_im2col_fused(xd, geom, 1, hb.F32, W1, ep, ws1)
+    out = torch.empty((s.M, N), device="cuda")
+    hb.conv_im2col(z.view(B, H, H, N), geom, 1, hb.F32, W2, out, ws2, flags=hb.CONV_INPUT_NHWC)
+    torch.cuda.synchronize()
+    G = s.K // BETA
+    rtol = (BETA + G + 4) * 2 * gu.U + 2.0 ** -18
+    per_image = s.M // B
+    for b in (0, B // 2, B - 1):
+        lo = b * per_image
+        c1, abs1 = oracle.conv_im2col(xb[b:b + 1], w1, 3, 3, (1, 1), (1, 1), 1, BETA)
+        y1 = np.maximum(c1, 0.0)
+        z_ref = y1 * bs.astype(np.float64) + bh.astype(np.float64)
+        z_gpu = z[lo: lo + per_image].float().cpu().numpy()
+        bound = np.abs(bs) * rtol * abs1 + 4 * gu.U * (np.abs(y1 * bs) + np.abs(bh)) + 2.0 ** -8 * np.abs(z_ref) + 1e-30
+        assert (np.abs(z_gpu - z_ref) <= bound).all(), "layer 1, image %d" % b
+        z_img = np.ascontiguousarray(z_gpu.reshape(1, H, H, N).transpose(0, 3, 1, 2))
+        c2, abs2 = oracle.conv_im2col(z_img, w2, 3, 3, (1, 1), (1, 1), 1, BETA)
+        gu.assert_close_rel_absref(out[lo: lo + per_image].cpu().numpy(), c2, abs2, rtol, "layer 2, image %d" % b)

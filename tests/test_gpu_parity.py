@@ -640,26 +640,169 @@ def test_gemm_binarize_next_matches_oracle(hb, M, N, K, ba, bw, bn, sdt, affine)
     ws = _gemm_ws(hb, A, W)
     hb.gemm_binarize_next(A, W, nxt, ws, torch.from_numpy(bs).cuda() if affine else None, torch.from_numpy(bh).cuda() if affine else None)
     torch.cuda.synchronize()
-    bits = gu.host_bits(nxt.bits)
-    lw = bits.shape[1]
-    got_sign = ((bits[:, np.arange(N) // 32] >> (np.arange(N) % 32).astype(np.uint32)) & 1).astype(np.int8) * 2 - 1
-    want_sign = np.where(z_ref >= 0, 1, -1)
-    decided = np.abs(z_ref) > band
-    assert (got_sign[decided] == want_sign[decided]).all()
-    assert decided.mean() > 0.99
-    # zero padding: bits past N and words past ceil(N / 32)
-    full = np.zeros((M, lw * 32), dtype=np.int8)
-    full[:, :N] = (got_sign > 0)
-    assert np.array_equal(bits, oracle.pack(np.where(full > 0, 1, -1).astype(np.int8)[:, :N], lw))
-    G = -(-N // bn)
-    sc = nxt.scales.float().cpu().numpy().astype(np.float64)
-    assert np.all(sc[:, G:] == 0.0)
-    tree = (int(np.ceil(np.log2(bn))) + 3) * gu.U + (2.0 ** -8 if sdt == hb.BF16 else 0.0)
-    for g in range(G):
-        sl = slice(g * bn, min((g + 1) * bn, N))
-        want = np.abs(z_ref[:, sl]).mean(axis=1)
-        tol = band[:, sl].mean(axis=1) + tree * want
-        assert (np.abs(sc[:, g] - want) <= tol).all(), g
+    gu.check_next_operand(nxt, z_ref, band, bn, sdt == hb.BF16)
+
+
+# ------------------------------------------------------------------ the rest of the layer in the epilogue (Section 5's order)
+FUSED_DENSE_CASES = [
+    # M, N, K, beta_a (1 = dense bf16 activations), beta_w, ReLU?, affine?, bf16 output?
+    (200, 128, 576, 32, 32, True, True, True),
+    (130, 1000, 1024, 64, 64, False, True, False),    # ragged N, fp32 out
+    (70, 64, 256, 32, 32, True, False, True),         # narrow tile
+    (65, 200, 320, 32, 128, True, True, False),
+    (300, 130, 640, 1, 32, True, True, True),         # HBWN kernel, ragged N: scalar bf16 stores at the edge
+    (129, 256, 1152, 1, 32, False, True, False),
+    (40, 64, 128, 1, 64, True, False, True),
+]
+
+
+@pytest.mark.parametrize("M,N,K,ba,bw,relu,affine,obf16", FUSED_DENSE_CASES)
+def test_gemm_fused_dense_output_matches_oracle(hb, M, N, K, ba, bw, relu, affine, obf16):
+    """hbmm_gemm_fused with a dense output: product -> activation -> per-column affine map -> fp32 or bf16 rows,
+    against the same chain applied to the oracle's product in double.  The bound is the product's own tolerance
+    carried through the map plus the fp32 arithmetic of the map (and half a bf16 ulp for bf16 rows)."""
+    gu = _gu()
+    a = inputs.normal((M, K), 9600 + M + K)
+    w = inputs.he_normal(N, K, 9700 + N + K)
+    W, dw, sw = gu.oracle_operand(w, bw)
+    if ba == 1:
+        _, a = inputs.as_bf16(a)
+        A = hb.wrap_dense(torch.from_numpy(a).cuda().to(torch.bfloat16))
+        c_ref, absref = oracle.hbwn_from_quantized(a, dw, sw, gu.eff_beta(bw, K))
+        tol_c = _hbwn_rtol(gu, K, bw, True) * absref
+    else:
+        A, da, sa = gu.oracle_operand(a, ba)
+        c_ref, absref = oracle.hbmm_from_quantized(da, sa, gu.eff_beta(ba, K), dw, sw, gu.eff_beta(bw, K))
+        fine = gu.elementwise_magnitude(da, gu.eff_beta(ba, K), dw, gu.eff_beta(bw, K), K)
+        tol_c = RTOL * absref + gu.FOLDED_FLOOR_ULPS * gu.U * fine
+    rng = np.random.default_rng(M + N)
+    bs = (rng.uniform(0.5, 2.0, N) * rng.choice([-1.0, 1.0], N)).astype(np.float32) if affine else np.ones(N, np.float32)
+    bh = (0.3 * rng.standard_normal(N)).astype(np.float32) if affine else np.zeros(N, np.float32)
+    y_ref = np.maximum(c_ref, 0.0) if relu else c_ref
+    z_ref = y_ref * bs.astype(np.float64) + bh.astype(np.float64)
+    bound = np.abs(bs) * tol_c + 4 * gu.U * (np.abs(y_ref * bs) + np.abs(bh)) + 1e-30
+    if obf16:
+        bound = bound + 2.0 ** -8 * np.abs(z_ref)
+    ld = (N + 7) // 8 * 8 + 8
+    out = torch.full((M, ld), float("nan"), device="cuda", dtype=torch.bfloat16 if obf16 else torch.float32)
+    ep = hb.make_epilogue(hb.ACT_RELU if relu else hb.ACT_NONE, torch.from_numpy(bs).cuda() if affine else None,
+                          torch.from_numpy(bh).cuda() if affine else None, out=out[:, :N])
+    hb.gemm_fused(A, W, ep, _gemm_ws(hb, A, W))
+    got = out.float().cpu().numpy().astype(np.float64)
+    assert np.isnan(got[:, N:]).all()                  # nothing written beyond column N
+    err = np.abs(got[:, :N] - z_ref)
+    assert (err <= bound).all(), float((err / bound).max())
+
+
+def test_gemm_fused_packed_output_after_relu_from_dense_activations(hb):
+    """HBWN product -> ReLU -> affine map -> rows binarized for the next layer, in the tensor-core HBWN kernel."""
+    gu = _gu()
+    M, N, K, bw, bn = 200, 136, 576, 32, 32
+    _, a = inputs.as_bf16(inputs.normal((M, K), 9801))
+    w = inputs.he_normal(N, K, 9802)
+    W, dw, sw = gu.oracle_operand(w, bw)
+    A = hb.wrap_dense(torch.from_numpy(a).cuda().to(torch.bfloat16))
+    c_ref, absref = oracle.hbwn_from_quantized(a, dw, sw, bw)
+    rng = np.random.default_rng(5)
+    bs = rng.uniform(0.5, 2.0, N).astype(np.float32)
+    bh = (-0.4 + 0.2 * rng.standard_normal(N)).astype(np.float32)       # shifts the rectified values around zero
+    y_ref = np.maximum(c_ref, 0.0)
+    z_ref = y_ref * bs.astype(np.float64) + bh.astype(np.float64)
+    band = np.abs(bs) * _hbwn_rtol(gu, K, bw, True) * absref + 4 * gu.U * (np.abs(y_ref * bs) + np.abs(bh)) + 1e-30
+    nxt = hb.alloc_operand(M, N, bn, hb.F32)
+    nxt.bits.fill_(-1)
+    nxt.scales.fill_(float("nan"))
+    ep = hb.make_epilogue(hb.ACT_RELU, torch.from_numpy(bs).cuda(), torch.from_numpy(bh).cuda(), nxt=nxt)
+    hb.gemm_fused(A, W, ep, _gemm_ws(hb, A, W))
+    torch.cuda.synchronize()
+    gu.check_next_operand(nxt, z_ref, band, bn, False)
+
+
+def _nhwc_to_nchw(z, B, Ho, Wo):
+    return np.ascontiguousarray(z.reshape(B, Ho, Wo, -1).transpose(0, 3, 1, 2))
+
+
+@pytest.mark.parametrize("B,C,H,F1,F2", [(3, 64, 12, 64, 72), (2, 128, 7, 128, 40)])
+def test_two_dense_activation_convolutions_chained_through_the_epilogue(hb, B, C, H, F1, F2):
+    """Layer 1: convolution (bf16 activations x Hadamard-binary weights) -> ReLU -> the next block's batch-norm map ->
+    NHWC bf16, written by the epilogue.  Layer 2 reads that tensor as it is (HBMM_CONV_INPUT_NHWC).  Layer 1 is held to
+    the composed oracle (product tolerance carried through the map, half a bf16 ulp); layer 2 to the oracle's
+    convolution of exactly the values layer 1 stored."""
+    gu = _gu()
+    s1 = inputs.ConvShape("l1", B, C, H, H, F1)
+    x = inputs.conv_activation(s1, 9900 + C, signed=True)
+    _, xb = inputs.as_bf16(x)
+    w1 = inputs.he_normal(F1, C * 9, 9901)
+    w2 = inputs.he_normal(F2, F1 * 9, 9902)
+    W1 = hb.quantize(torch.from_numpy(w1).cuda(), hb.alloc_operand(F1, C * 9, 32))
+    W2 = hb.quantize(torch.from_numpy(w2).cuda(), hb.alloc_operand(F2, F1 * 9, 32))
+    rng = np.random.default_rng(C)
+    bs = rng.uniform(0.5, 2.0, F1).astype(np.float32)
+    bh = (0.2 * rng.standard_normal(F1)).astype(np.float32)
+    g1 = hb.make_geom(B, C, H, H, 3, 3, (1, 1), (1, 1))
+    g2 = hb.make_geom(B, F1, H, H, 3, 3, (1, 1), (1, 1))
+    ws1 = torch.empty(hb.conv_workspace_bytes(g1, 1, hb.F32, W1), dtype=torch.uint8, device="cuda")
+    ws2 = torch.empty(hb.conv_workspace_bytes(g2, 1, hb.F32, W2), dtype=torch.uint8, device="cuda")
+    M = B * H * H
+    z = torch.full((M, F1), float("nan"), device="cuda", dtype=torch.bfloat16)
+    ep = hb.make_epilogue(hb.ACT_RELU, torch.from_numpy(bs).cuda(), torch.from_numpy(bh).cuda(), out=z)
+    hb.conv_im2col_fused(torch.from_numpy(xb).cuda().to(torch.bfloat16), g1, 1, hb.F32, W1, ep, ws1)
+    out = torch.full((M, (F2 + 3) // 4 * 4), float("nan"), device="cuda")
+    hb.conv_im2col(z.view(B, H, H, F1), g2, 1, hb.F32, W2, out, ws2, flags=hb.CONV_INPUT_NHWC)
+    torch.cuda.synchronize()
+    # layer 1
+    c1, abs1 = oracle.conv_im2col(xb, w1, 3, 3, (1, 1), (1, 1), 1, 32)
+    y1 = np.maximum(c1, 0.0)
+    z_ref = y1 * bs.astype(np.float64) + bh.astype(np.float64)
+    z_gpu = z.float().cpu().numpy()
+    bound = np.abs(bs) * _hbwn_rtol(gu, C * 9, 32, True) * abs1 + 4 * gu.U * (np.abs(y1 * bs) + np.abs(bh)) + 2.0 ** -8 * np.abs(z_ref) + 1e-30
+    assert (np.abs(z_gpu - z_ref) <= bound).all()
+    # layer 2 from the stored values
+    c2, abs2 = oracle.conv_im2col(_nhwc_to_nchw(z_gpu, B, H, H), w2, 3, 3, (1, 1), (1, 1), 1, 32)
+    gu.assert_close_rel_absref(out.cpu().numpy()[:, :F2], c2, abs2, _hbwn_rtol(gu, F1 * 9, 32, True), "layer 2")
+
+
+def test_packed_convolution_feeding_a_pointwise_layer_through_the_epilogue(hb):
+    """Layer 1: 3 x 3 convolution as HBMM (beta_a = beta_w = 32) -> ReLU -> batch-norm map -> rows binarized along the
+    output channels by the epilogue (the fp32 product never stored).  Layer 2: a 1 x 1 convolution = hbmm_gemm on that
+    packed operand.  Layer 1 is checked like hbmm_gemm_binarize_next; layer 2 against the oracle's product of the
+    operand layer 1 actually wrote."""
+    gu = _gu()
+    B, C, H, F1, F2, bn = 2, 64, 12, 128, 96, 32
+    s1 = inputs.ConvShape("l1", B, C, H, H, F1)
+    x = inputs.conv_activation(s1, 9950, signed=True)
+    w1 = inputs.he_normal(F1, C * 9, 9951)
+    w2 = inputs.he_normal(F2, F1, 9952)
+    W1, dw1, sw1 = gu.oracle_operand(w1, 32)
+    W2, dw2, sw2 = gu.oracle_operand(w2, bn)
+    rng = np.random.default_rng(11)
+    bs = rng.uniform(0.5, 2.0, F1).astype(np.float32)
+    bh = (-0.3 + 0.2 * rng.standard_normal(F1)).astype(np.float32)
+    g1 = hb.make_geom(B, C, H, H, 3, 3, (1, 1), (1, 1))
+    ws1 = torch.empty(hb.conv_workspace_bytes(g1, 32, hb.F32, W1), dtype=torch.uint8, device="cuda")
+    M = B * H * H
+    nxt = hb.alloc_operand(M, F1, bn, hb.F32)
+    nxt.bits.fill_(-1)
+    nxt.scales.fill_(float("nan"))
+    ep = hb.make_epilogue(hb.ACT_RELU, torch.from_numpy(bs).cuda(), torch.from_numpy(bh).cuda(), nxt=nxt)
+    hb.conv_im2col_fused(torch.from_numpy(x).cuda(), g1, 32, hb.F32, W1, ep, ws1)
+    out = torch.full((M, F2), float("nan"), device="cuda")
+    hb.gemm(nxt, W2, out, _gemm_ws(hb, nxt, W2))
+    torch.cuda.synchronize()
+    rows = oracle.im2col(x, 3, 3, (1, 1), (1, 1))
+    da, sa = oracle.quantize(rows, 32)
+    c1, abs1 = oracle.hbmm_from_quantized(da, sa, 32, dw1, sw1, 32)
+    fine = gu.elementwise_magnitude(da, 32, dw1, 32, C * 9)
+    y1 = np.maximum(c1, 0.0)
+    z_ref = y1 * bs.astype(np.float64) + bh.astype(np.float64)
+    band = np.abs(bs) * (RTOL * abs1 + gu.FOLDED_FLOOR_ULPS * gu.U * fine) + 4 * gu.U * (np.abs(y1 * bs) + np.abs(bh)) + 1e-30
+    gu.check_next_operand(nxt, z_ref, band, bn, False)
+    # layer 2 from what was stored
+    sg = oracle.unpack(gu.host_bits(nxt.bits), F1)
+    dg = nxt.scales.cpu().numpy().astype(np.float64)[:, : F1 // bn]
+    c2, abs2 = oracle.hbmm_from_quantized(dg, sg, bn, dw2, sw2, bn)
+    gu.assert_close_rel_absref(out.cpu().numpy(), c2, abs2, RTOL, "pointwise layer",
+                               gu.elementwise_magnitude(dg, bn, dw2, bn, F1))
 
 
 @pytest.mark.parametrize("beta_a,xbf16", [(32, False), (1, True)])
