@@ -493,6 +493,43 @@ def side_measurements(torch, hbmm, inputs, peaks, iters: int):
     out.append({"kernel": "conv2_x_eq3_grouping_beta_a8: hbmm_binarize_dense + hbmm_conv_im2col(beta_a=1)", "shape": [Bc * Hc * Hc, Nc, Cc * 9],
                 "ms": round(ms3, 5), "bound": "tensor", "achieved": ach, "peak": bf16_tflops, "unit": "TFLOP/s", "frac": ach / bf16_tflops})
     del xm, am, Cc_out, amap, a, gy, gx
+    # Two dense-activation convolutions (conv3_x -> conv3_x) with ReLU and the next block's batch-norm map between them:
+    # chained through the epilogue (NHWC bf16 written by layer 1, read directly by layer 2) against the unfused
+    # sequence (fp32 NHWC product, the map / rounding / NHWC -> NCHW permutation as torch element-wise kernels, then the
+    # second convolution with its own layout copy).
+    sh = inputs.resnet18_convs(64)[1]
+    xc = torch.randn((sh.B, sh.C, sh.H, sh.W), device="cuda", generator=g).to(torch.bfloat16)
+    W1 = hbmm.quantize(torch.randn((sh.N, sh.K), device="cuda", generator=g) * (2.0 / sh.K) ** 0.5, hbmm.alloc_operand(sh.N, sh.K, BETA, hbmm.F32))
+    W2 = hbmm.quantize(torch.randn((sh.N, sh.N * 9), device="cuda", generator=g) * (2.0 / (sh.N * 9)) ** 0.5, hbmm.alloc_operand(sh.N, sh.N * 9, BETA, hbmm.F32))
+    bs = torch.rand(sh.N, device="cuda", generator=g) + 0.5
+    bh = torch.randn(sh.N, device="cuda", generator=g) * 0.2
+    geom3 = hbmm.make_geom(sh.B, sh.C, sh.H, sh.W, 3, 3, (1, 1), (1, 1))
+    ws1 = torch.empty(hbmm.conv_workspace_bytes(geom3, 1, hbmm.F32, W1), dtype=torch.uint8, device="cuda")
+    ws2 = torch.empty(hbmm.conv_workspace_bytes(geom3, 1, hbmm.F32, W2), dtype=torch.uint8, device="cuda")
+    zc = torch.empty((sh.M, sh.N), device="cuda", dtype=torch.bfloat16)
+    c1 = torch.empty((sh.M, sh.N), device="cuda")
+    c2 = torch.empty((sh.M, sh.N), device="cuda")
+    epc = hbmm.make_epilogue(hbmm.ACT_RELU, bs, bh, out=zc)
+    PREPF = hbmm.CONV_WEIGHTS_PREPARED
+
+    def chain_fused(flags):
+        hbmm.conv_im2col_fused(xc, geom3, 1, hbmm.F32, W1, epc, ws1, flags=flags)
+        hbmm.conv_im2col(zc.view(sh.B, sh.H, sh.W, sh.N), geom3, 1, hbmm.F32, W2, c2, ws2, flags=flags | hbmm.CONV_INPUT_NHWC)
+
+    def chain_unfused(flags):
+        hbmm.conv_im2col(xc, geom3, 1, hbmm.F32, W1, c1, ws1, flags=flags)
+        zt = (torch.relu(c1) * bs + bh).to(torch.bfloat16).view(sh.B, sh.H, sh.W, sh.N).permute(0, 3, 1, 2).contiguous()
+        hbmm.conv_im2col(zt, geom3, 1, hbmm.F32, W2, c2, ws2, flags=flags)
+
+    chain_fused(0)
+    ms_f = time_loop(torch, lambda: chain_fused(PREPF), iters)
+    chain_unfused(0)
+    ms_u = time_loop(torch, lambda: chain_unfused(PREPF), iters)
+    out.append({"kernel": "conv3_x -> relu -> bn -> conv3_x (bf16 activations): chained through the epilogue, 2 launches", "ms": round(ms_f, 5),
+                "tflops": 4.0 * sh.M * sh.N * sh.K / (ms_f * 1e-3) / 1e12})
+    out.append({"kernel": "conv3_x -> relu -> bn -> conv3_x (bf16 activations): unfused (fp32 product, torch element-wise + permute, layout copy)",
+                "ms": round(ms_u, 5), "tflops": 4.0 * sh.M * sh.N * sh.K / (ms_u * 1e-3) / 1e12})
+    del xc, zc, c1, c2, ws1, ws2
     # Exact-scale variants on the four convolution matrices (seeded device-generated operands of the same shapes):
     # HBMM with integer group dots and a per-group fp32 scale step (HBMM_PATH_TENSOR) beside the default
     # folded-scale kernel, and HBWN on the dense bf16 im2col matrix with three bf16 weight pieces (scales to 2^-26,
@@ -924,6 +961,14 @@ def run_ours(args):
     for _ in range(max(args.warmup, 3) - 1):
         step2(hbmm, layers, PREP)
     torch.cuda.synchronize()
+    if args.profile_step:
+        # the timed schedule and nothing else (no breakdown, side rows or CPU timing): for a profiler's launch list
+        for _ in range(args.steps):
+            step2(hbmm, layers, PREP)
+        torch.cuda.synchronize()
+        assert hbmm.last_device_error() == 0
+        print(json.dumps({"profile_step": True, "steps": args.steps, "launches_per_step": LAUNCHES_PER_STEP}))
+        return 0
 
     def barrier():
         if world > 1:
@@ -1087,6 +1132,8 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--profile-step", action="store_true",
+                    help="run the warm-up and the timed steps only, no measurement: for a profiler's launch list")
     ap.add_argument("--profile-layer", default=None,
                     help="run only this layer (conv2_x .. conv5_x), few launches, no measurement: for profiler captures")
     args = ap.parse_args()
