@@ -24,7 +24,7 @@
 //                 MMA takes its A operand from there: the activation operand never passes through shared
 //                 memory, whose bandwidth bounded the kernel while it did), with the global loads issued
 //                 several stages ahead
-//   warps 14-17 : scouts: one thread per tile row finds the row's largest scale (the power of two that
+//   warps 14-15 : scouts: one thread per two tile rows finds a row's largest scale (the power of two that
 //                 normalises the row) a few tiles ahead of everyone else
 //   warp  12    : TMEM allocation and the single MMA-issuing thread
 //   warp  13    : one thread streams the prepared W stages (cp.async.bulk, completion on the stage's
@@ -53,7 +53,7 @@ constexpr int kFirstProducerWarp = kEpilogueWarps;
 constexpr int kMmaWarp = kEpilogueWarps + kProducerWarps;   // 12
 constexpr int kLoaderWarp = kMmaWarp + 1;                   // 13
 constexpr int kFirstScoutWarp = kLoaderWarp + 1;            // 14..17
-constexpr int kScoutWarps = 4;
+constexpr int kScoutWarps = 2;                              // 16 warps in all: 128 registers per thread
 constexpr int kThreads = (kFirstScoutWarp + kScoutWarps) * 32;
 // Stages of packed words + scales each producer thread keeps in flight; fewer when a word has many scales.
 template <int SUBW> struct DepthFor { static constexpr int value = SUBW == 1 ? 4 : (SUBW <= 4 ? 2 : 1); };
@@ -68,6 +68,7 @@ prepare_w_fold_kernel(const Args g, unsigned char* __restrict__ out, float* __re
 // the row pointers of the tile it is in.
 struct StageCursor {
   int64_t ti, st;            // tile (in this CTA's sequence) and stage inside it
+  int64_t end;               // one past the last stage of the segment (ti)
   const uint32_t* bptr;      // packed words of this thread's row
   int64_t srow;              // first scale of the row
   bool in;                   // the row exists
@@ -76,7 +77,9 @@ struct StageCursor {
 // ASUB: scale groups per packed word of A (1: groups of whole words; 2 .. 16: beta_a = 16 .. 2).
 // FUSE: the epilogue runs the activation / affine map / dense or binarized output chain of epilogue.cuh instead of
 // storing the product as fp32.
-template <int TN, int ASUB, bool FUSE>
+// BAL: the balanced schedule (runs of (tile, stage) pairs, partial tiles reduced by the last CTA to arrive); the plain
+// instantiation carries none of its code.
+template <int TN, int ASUB, bool FUSE, bool BAL>
 __global__ void __launch_bounds__(kThreads, 1)
 hbmm_fold_kernel(const Args g) {
   using S = Smem<TN>;
@@ -100,7 +103,27 @@ hbmm_fold_kernel(const Args g) {
   const int64_t tiles_n = (g.N + TN - 1) / TN, tiles_m = (g.M + TM - 1) / TM;
   const int64_t n_tiles = tiles_m * tiles_n;
   const int64_t n_stages = (g.n_words + WPS - 1) / WPS;      // per tile
-  const int64_t my_tiles = blockIdx.x < n_tiles ? (n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+  // The CTA's work is a list of segments (tile, first stage, one past the last stage).  Plain schedule: whole tiles
+  // blockIdx.x, blockIdx.x + gridDim.x, ...  Balanced schedule: the run [u0, u1) of the tile-major (tile, stage)
+  // sequence -- consecutive tiles, the first possibly entered mid-way, the last possibly left early.
+  constexpr bool balanced = BAL;
+  const int64_t u0 = balanced ? static_cast<int64_t>(blockIdx.x) * g.sk_units : 0;
+  const int64_t u_end = balanced ? ((u0 + g.sk_units < n_tiles * n_stages) ? u0 + g.sk_units : n_tiles * n_stages) : 0;
+  const int64_t sk_t0 = balanced ? u0 / n_stages : 0;                                  // first tile of the run
+  const int64_t sk_first = balanced ? u0 - sk_t0 * n_stages : 0;                       // first stage inside it
+  const int64_t sk_t1 = (balanced && u_end > u0) ? (u_end - 1) / n_stages : 0;         // last tile of the run
+  const int64_t sk_last_end = (balanced && u_end > u0) ? u_end - sk_t1 * n_stages : 0; // one past its last stage
+  const int64_t my_tiles = balanced ? (u_end > u0 ? sk_t1 - sk_t0 + 1 : 0)
+                                    : (blockIdx.x < n_tiles ? (n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0);
+  const int64_t my_stages = balanced ? (u_end > u0 ? u_end - u0 : 0) : my_tiles * n_stages;
+  // Order of work in a balanced run: the two tiles shared with the neighbouring runs first (the tail of the run's first
+  // tile, then the head of its last), the whole tiles after them -- so partial accumulators are handed in early and
+  // the CTA that completes a shared tile does so in the shadow of the MMAs of its whole tiles, not at the kernel's end.
+  const bool reorder = balanced && my_tiles >= 3;
+  auto seg_nat = [&](int64_t ti) -> int64_t { return !reorder ? ti : (ti == 0 ? 0 : (ti == 1 ? my_tiles - 1 : ti - 1)); };
+  auto seg_tile = [&](int64_t ti) -> int64_t { return balanced ? sk_t0 + seg_nat(ti) : blockIdx.x + ti * gridDim.x; };
+  auto seg_begin = [&](int64_t ti) -> int64_t { return (balanced && ti < my_tiles && seg_nat(ti) == 0) ? sk_first : 0; };
+  auto seg_end = [&](int64_t ti) -> int64_t { return (balanced && ti < my_tiles && seg_nat(ti) == my_tiles - 1) ? sk_last_end : n_stages; };
 
   pdl_launch_dependents();      // the next kernel of the stream may start its own set-up
   if (tid == 0) {
@@ -137,20 +160,27 @@ hbmm_fold_kernel(const Args g) {
     const uint32_t t_lane = static_cast<uint32_t>((warp & 3) * 32) << 16;     // this warp's quarter of the TMEM lanes = its tile rows
     const uint32_t n_words = static_cast<uint32_t>(g.n_words), gw = static_cast<uint32_t>(g.a_gw);
     const bool vec_scales = ASUB == 1 && !g.a_bf16 && gw == 1;      // one fp32 scale per word: a stage's two scales are one 8-byte load
-    const int64_t total = my_tiles * n_stages;
+    const int64_t total = my_stages;
     auto set_tile = [&](StageCursor& c) {
-      const int64_t tile = blockIdx.x + c.ti * gridDim.x;
+      const int64_t tile = seg_tile(c.ti);
       const int64_t m = (tile / tiles_n) * TM + p;
       c.in = c.ti < my_tiles && m < g.M;
       c.bptr = g.a_bits + (c.in ? m : 0) * g.lda_w;
       c.srow = (c.in ? m : 0) * g.lda_s;
     };
-    auto advance = [&](StageCursor& c) {
-      c.st += 2;
-      if (c.st >= n_stages) {
-        do { c.st -= n_stages; c.ti++; } while (c.st >= n_stages);
+    auto carry_over = [&](StageCursor& c) {        // moves a stage index past its segment's end into the segments after it
+      if (c.st >= c.end) {
+        if (!balanced) {
+          do { c.st -= n_stages; c.ti++; } while (c.st >= n_stages);
+        } else {
+          do { const int64_t over = c.st - c.end; c.ti++; c.st = seg_begin(c.ti) + over; c.end = seg_end(c.ti); } while (c.st >= c.end);
+        }
         set_tile(c);
       }
+    };
+    auto advance = [&](StageCursor& c) {
+      c.st += 2;
+      carry_over(c);
     };
     // raw scales of the stage's two words: sc[0 .. ASUB) of the first, sc[ASUB .. 2 ASUB) of the second
     auto fetch = [&](const StageCursor& c, uint2& w, float (&sc)[2 * ASUB]) {
@@ -183,8 +213,8 @@ hbmm_fold_kernel(const Args g) {
       }
     };
     StageCursor pf, cur;
-    pf.ti = 0; pf.st = q;
-    if (pf.st >= n_stages) { do { pf.st -= n_stages; pf.ti++; } while (pf.st >= n_stages); }
+    pf.ti = 0; pf.st = seg_begin(0) + q; pf.end = seg_end(0);      // the stage walk continues from segment to segment
+    carry_over(pf);
     set_tile(pf);
     cur = pf;
     uint2 w[kDepth];
@@ -243,16 +273,25 @@ hbmm_fold_kernel(const Args g) {
     // =========================== scouts ===========================
     // One thread per tile row finds the row's largest scale and stores the two powers of two, up to
     // kRowSlots tiles ahead of the epilogue.
-    const int p = tid - kFirstScoutWarp * 32;
+    const int p0 = tid - kFirstScoutWarp * 32;
     for (int64_t ti = 0; ti < my_tiles; ti++) {
       const int slot = static_cast<int>(ti & (kRowSlots - 1));
       if (ti >= kRowSlots && !mbar_wait(&rowempty[slot], static_cast<uint32_t>(((ti / kRowSlots) & 1) ^ 1), abort_flag, 8)) break;
-      const int64_t tile = blockIdx.x + ti * gridDim.x;
-      const int64_t m = (tile / tiles_n) * TM + p;
-      float up = 0.0f, down = 1.0f;
-      if (m < g.M) norm_factors(row_max_scale(g.a_scales, g.a_bf16, m * g.lda_s, g.lda_s), up, down);
-      rowup[slot * TM + p] = up;
-      rowdown[slot * TM + p] = down;
+      const int64_t tile = seg_tile(ti);
+      {
+        // rows p0 and p0 + 64, scanned together so that both rows' loads are in flight at once
+        const int64_t ma = (tile / tiles_n) * TM + p0, mb = ma + kScoutWarps * 32;
+        float xa, xb;
+        row_max_scale2(g.a_scales, g.a_bf16, (ma < g.M ? ma : 0) * g.lda_s, (mb < g.M ? mb : 0) * g.lda_s, g.lda_s, xa, xb);
+        float up = 0.0f, down = 1.0f;
+        if (ma < g.M) norm_factors(xa, up, down);
+        rowup[slot * TM + p0] = up;
+        rowdown[slot * TM + p0] = down;
+        up = 0.0f; down = 1.0f;
+        if (mb < g.M) norm_factors(xb, up, down);
+        rowup[slot * TM + p0 + kScoutWarps * 32] = up;
+        rowdown[slot * TM + p0 + kScoutWarps * 32] = down;
+      }
       __syncwarp();
       if (lane == 0) mbar_arrive(&rowfull[slot]);
     }
@@ -262,9 +301,10 @@ hbmm_fold_kernel(const Args g) {
       int64_t gst = 0;
       bool ok = true;
       for (int64_t ti = 0; ti < my_tiles && ok; ti++) {
-        const int64_t tile = blockIdx.x + ti * gridDim.x;
+        const int64_t tile = seg_tile(ti);
         const unsigned char* src = g.w_prep + (tile % tiles_n) * n_stages * S::B_STAGE;
-        for (int64_t st = 0; st < n_stages; st++, gst++) {
+        const int64_t st_end = seg_end(ti);
+        for (int64_t st = seg_begin(ti); st < st_end; st++, gst++) {
           const int s = static_cast<int>(gst % STAGES);
           if (gst >= STAGES && !mbar_wait(&empty[s], static_cast<uint32_t>(((gst / STAGES) & 1) ^ 1), abort_flag, 6)) { ok = false; break; }
           mbar_arrive_expect_tx(&full[s], S::B_STAGE);
@@ -296,7 +336,6 @@ hbmm_fold_kernel(const Args g) {
       const uint32_t db_lo = static_cast<uint32_t>(db0);
       const uint32_t full_a = smem_u32(full), empty_a = smem_u32(empty), tfull_a = smem_u32(tfull), tempty_a = smem_u32(tempty);
       const bool leader = lane == 0;
-      const uint32_t n_st = static_cast<uint32_t>(n_stages);
       uint32_t s = 0, full_par = 0;
       bool ok = true;
       for (int64_t ti = 0; ti < my_tiles && ok; ti++) {
@@ -306,6 +345,7 @@ hbmm_fold_kernel(const Args g) {
           tc_fence_after();
         }
         const uint32_t d_tmem = tmem_base + buf * S::ACC_COLS;
+        const uint32_t n_st = static_cast<uint32_t>(seg_end(ti) - seg_begin(ti));      // the segment starts a fresh accumulation
         for (uint32_t st = 0; st < n_st; st++) {
           if (!mbar_wait_a(full_a + s * 8, full_par, abort_flag, 2)) { ok = false; break; }
           tc_fence_after();
@@ -350,7 +390,7 @@ hbmm_fold_kernel(const Args g) {
     for (int64_t ti = 0; ti < my_tiles; ti++) {
       const uint32_t buf = static_cast<uint32_t>(ti & 1);
       const int slot = static_cast<int>(ti & (kRowSlots - 1));
-      const int64_t tile = blockIdx.x + ti * gridDim.x;
+      const int64_t tile = seg_tile(ti);
       const int64_t m = (tile / tiles_n) * TM + row, nb = (tile % tiles_n) * TN;
       // the tile's column factors go through shared memory (one copy per warp, so no warp waits for
       // another): requested before the wait for the accumulator, read back as broadcasts
@@ -379,9 +419,8 @@ hbmm_fold_kernel(const Args g) {
       if (lane == 0) mbar_arrive(&rowempty[slot]);
       float* dst = g.C + m * g.ldc + nb;
       float carry = 0.0f;                                   // |z| sum of a group wider than a 32-column chunk
-#pragma unroll
-      for (int c = 0; c < TN / 32; c++) {
-        uint32_t v1[32];
+      // raw accumulator of chunk c (32 columns of this thread's row): the two stacked blocks added for the narrow tile
+      auto load_chunk = [&](int c, uint32_t (&v1)[32]) {
         const uint32_t t_addr = tmem_base + t_lane + buf * S::ACC_COLS + c * 32;
         tmem_ld32(t_addr, v1);
         if constexpr (S::STACKED) {      // the A1 W2 block sits TN columns further on
@@ -393,6 +432,9 @@ hbmm_fold_kernel(const Args g) {
         } else {
           tmem_ld_wait();
         }
+      };
+      // the tile's complete accumulator values of chunk c -> the output (powers of two divided out; epilogue chain or fp32 store)
+      auto finish = [&](int c, const uint32_t (&v1)[32]) {
         if constexpr (FUSE) {
           if (m < g.M) {
             // the product of the chunk's 32 columns, then activation, affine map and dense or binarized output
@@ -427,10 +469,61 @@ hbmm_fold_kernel(const Args g) {
                 if (n + e < g.N) dst[c * 32 + j + e] = o[e];
           }
         }
+      };
+      const bool whole = !BAL || (seg_begin(ti) == 0 && seg_end(ti) == n_stages);
+      if (whole) {
+#pragma unroll
+        for (int c = 0; c < TN / 32; c++) {
+          uint32_t v1[32];
+          load_chunk(c, v1);
+          finish(c, v1);
+        }
+        tc_fence_before();
+        __syncwarp();          // also: every lane is done with the warp's column factors
+        if (lane == 0) mbar_arrive(&tempty[buf]);
+      } else if constexpr (BAL) {
+        // Part of the tile's K range: the raw partial accumulator goes to this CTA's slot (first slot for the tile
+        // its run starts in, second for the tile it ends in), the accumulator is handed back, and the warp
+        // counts itself in.  Whoever arrives last adds the tile's partials in CTA order -- the same sum whoever
+        // that is -- and finishes the rows.  Nobody waits for anybody.
+        // slot layout [column][row]: a warp's store of one column is 32 consecutive floats
+        float* slot = g.sk_partials + static_cast<int64_t>(2 * blockIdx.x + (seg_nat(ti) == 0 ? 0 : 1)) * (TM * TN) + row;
+#pragma unroll
+        for (int c = 0; c < TN / 32; c++) {
+          uint32_t v1[32];
+          load_chunk(c, v1);
+#pragma unroll
+          for (int j = 0; j < 32; j++) __stcg(slot + (c * 32 + j) * TM, __uint_as_float(v1[j]));
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tempty[buf]);
+        __threadfence();       // the partial is visible device-wide before the count says so
+        __syncwarp();
+        const int64_t c_first = (tile * n_stages) / g.sk_units, c_last = ((tile + 1) * n_stages - 1) / g.sk_units;
+        int arrived = 0;
+        if (lane == 0) arrived = atomicAdd(g.sk_counters + tile * kEpilogueWarps + warp, 1);
+        arrived = __shfl_sync(0xFFFFFFFFu, arrived, 0);
+        if (arrived == static_cast<int>(c_last - c_first)) {
+          __threadfence();
+#pragma unroll 1
+          for (int c = 0; c < TN / 32; c++) {
+            uint32_t v1[32];
+#pragma unroll
+            for (int j = 0; j < 32; j++) v1[j] = 0u;                 // +0.0f
+            for (int64_t cc = c_first; cc <= c_last; cc++) {
+              const int64_t first_tile_of_cc = (cc * g.sk_units) / n_stages;
+              const float* src = g.sk_partials + (2 * cc + (first_tile_of_cc == tile ? 0 : 1)) * (TM * TN) + (c * 32) * TM + row;
+#pragma unroll
+              for (int j = 0; j < 32; j++) v1[j] = __float_as_uint(__uint_as_float(v1[j]) + __ldcg(src + j * TM));
+            }
+            finish(c, v1);
+          }
+          if (lane == 0) g.sk_counters[tile * kEpilogueWarps + warp] = 0;      // as the next launch expects to find it
+        }
+        __syncwarp();          // every lane is done with the warp's column factors
       }
-      tc_fence_before();
-      __syncwarp();          // also: every lane is done with the warp's column factors
-      if (lane == 0) mbar_arrive(&tempty[buf]);
+
     }
   }
 
@@ -476,6 +569,7 @@ Args make_args(const PackedView& A, const PackedView& W, float* C, int64_t ldc) 
   g.w_prep = nullptr;
   g.w_down = nullptr;
   g.ep = plain_epilogue();
+  g.sk_units = 0; g.sk_counters = nullptr; g.sk_counter_count = 0; g.sk_partials = nullptr;
   return g;
 }
 
@@ -484,25 +578,66 @@ size_t stage_bytes(const Args& g) {
   const int64_t tiles_n = (g.N + TN - 1) / TN, n_stages = (g.n_words + WPS - 1) / WPS;
   return static_cast<size_t>(tiles_n * n_stages) * Smem<TN>::B_STAGE;
 }
+// Balanced schedule: worth its reduction traffic when the tiles are few waves of the machine and a tile's K walk is
+// long enough to cut.  The workspace is sized for any device of up to kMaxBalancedCtas multiprocessors.
+constexpr int64_t kMaxBalancedCtas = 256;
+constexpr int64_t kBalancedWaves = 4;
+constexpr int64_t kBalancedMinStages = 4;
 template <int TN>
-size_t prep_bytes(const Args& g) {
-  return stage_bytes<TN>(g) + static_cast<size_t>((g.N + TN - 1) / TN) * TN * sizeof(float);
+int64_t tile_count(const Args& g) { return ((g.M + TM - 1) / TM) * ((g.N + TN - 1) / TN); }
+template <int TN>
+bool balanced_possible(const Args& g, int64_t sms) {
+  const int64_t n_stages = (g.n_words + WPS - 1) / WPS;
+  return sms <= kMaxBalancedCtas && n_stages >= kBalancedMinStages && tile_count<TN>(g) < kBalancedWaves * sms;
+}
+template <int TN>
+size_t counters_bytes(const Args& g) { return (static_cast<size_t>(tile_count<TN>(g)) * kEpilogueWarps * sizeof(int32_t) + 255) / 256 * 256; }
+template <int TN>
+size_t balanced_bytes(const Args& g) {
+  if (!balanced_possible<TN>(g, kMaxBalancedCtas)) return 0;
+  const int64_t n_stages = (g.n_words + WPS - 1) / WPS, units = tile_count<TN>(g) * n_stages;
+  const int64_t ctas = units < kMaxBalancedCtas ? units : kMaxBalancedCtas;
+  return counters_bytes<TN>(g) + static_cast<size_t>(2 * ctas) * TM * TN * sizeof(float);
+}
+// [W stages][one float per weight row][counters][partial slots]
+template <int TN>
+size_t down_offset(const Args& g) { return stage_bytes<TN>(g); }
+template <int TN>
+size_t balanced_offset(const Args& g) {
+  return (stage_bytes<TN>(g) + static_cast<size_t>((g.N + TN - 1) / TN) * TN * sizeof(float) + 255) / 256 * 256;
+}
+template <int TN>
+size_t prep_bytes(const Args& g) { return balanced_offset<TN>(g) + balanced_bytes<TN>(g); }
+// Points the argument block at the balanced schedule's part of the workspace (when the shape has one).
+template <int TN>
+void set_balanced_area(Args& g, void* workspace) {
+  if (balanced_bytes<TN>(g) == 0) return;
+  unsigned char* area = static_cast<unsigned char*>(workspace) + balanced_offset<TN>(g);
+  g.sk_counters = reinterpret_cast<int32_t*>(area);
+  g.sk_counter_count = tile_count<TN>(g) * kEpilogueWarps;
+  g.sk_partials = reinterpret_cast<float*>(area + counters_bytes<TN>(g));
 }
 
 template <int TN, int ASUB, bool FUSE = false>
 cudaError_t launch_fold(Args g, void* workspace, cudaStream_t stream, bool w_prepared) {
   using S = Smem<TN>;
+  constexpr bool kHasBalanced = ASUB == 1;           // the balanced schedule is built for activation groups of whole words
   static DeviceOnce configured;
   int dev = 0, sms = 0;
   if (current_device(&dev, &sms) != cudaSuccess) return cudaErrorInvalidDevice;
   if (configured.pending(dev)) {
-    cudaError_t e = cudaFuncSetAttribute(hbmm_fold_kernel<TN, ASUB, FUSE>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::BYTES);
+    cudaError_t e = cudaFuncSetAttribute(hbmm_fold_kernel<TN, ASUB, FUSE, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::BYTES);
     if (e != cudaSuccess) return e;
+    if (kHasBalanced) {
+      e = cudaFuncSetAttribute(hbmm_fold_kernel<TN, ASUB, FUSE, kHasBalanced>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::BYTES);
+      if (e != cudaSuccess) return e;
+    }
     configured.mark(dev);
   }
   const int64_t tiles_n = (g.N + TN - 1) / TN, n_stages = (g.n_words + WPS - 1) / WPS;
   unsigned char* stages = static_cast<unsigned char*>(workspace);
   float* down = reinterpret_cast<float*>(stages + stage_bytes<TN>(g));
+  set_balanced_area<TN>(g, workspace);
   if (!w_prepared) {
     dim3 pgrid(static_cast<unsigned>((n_stages + kPrepStages - 1) / kPrepStages), static_cast<unsigned>(tiles_n));
     prepare_w_fold_kernel<TN><<<pgrid, TN, 0, stream>>>(g, stages, down);
@@ -510,8 +645,19 @@ cudaError_t launch_fold(Args g, void* workspace, cudaStream_t stream, bool w_pre
   g.w_prep = stages;
   g.w_down = down;
   const int64_t tiles = ((g.M + TM - 1) / TM) * tiles_n;
+  // equal runs of (tile, stage) pairs, one per CTA, when that shortens the longest CTA's walk by a tenth or more
+  const int64_t units = tiles * n_stages;
+  int64_t ctas = units / kBalancedMinStages < sms ? units / kBalancedMinStages : sms;
+  if (ctas < 1) ctas = 1;
+  const int64_t run = (units + ctas - 1) / ctas;
+  const int64_t plain_walk = ((tiles + sms - 1) / sms) * n_stages;
+  if (kHasBalanced && balanced_possible<TN>(g, sms) && run * 10 <= plain_walk * 9) {
+    ctas = (units + run - 1) / run;                     // no CTA without work
+    g.sk_units = run;
+    return launch_pdl(hbmm_fold_kernel<TN, ASUB, FUSE, kHasBalanced>, dim3(static_cast<unsigned>(ctas)), dim3(kThreads), S::BYTES, stream, g);
+  }
   const unsigned grid = static_cast<unsigned>(tiles < sms ? tiles : sms);   // one persistent CTA per SM
-  return launch_pdl(hbmm_fold_kernel<TN, ASUB, FUSE>, dim3(grid), dim3(kThreads), S::BYTES, stream, g);
+  return launch_pdl(hbmm_fold_kernel<TN, ASUB, FUSE, false>, dim3(grid), dim3(kThreads), S::BYTES, stream, g);
 }
 
 template <int TN>
@@ -571,6 +717,7 @@ void gemm_fold_prep_job(const PackedView& A, const PackedView& W, void* workspac
   job->n_stages = static_cast<int32_t>((n_stages + kPrepStages - 1) / kPrepStages);    // tasks per column tile
   job->tiles_n = static_cast<int32_t>((job->f.N + job->tn - 1) / job->tn);
   job->out_down = reinterpret_cast<float*>(job->out + (job->tn == 64 ? stage_bytes<64>(job->f) : stage_bytes<128>(job->f)));
+  if (job->tn == 64) set_balanced_area<64>(job->f, workspace); else set_balanced_area<128>(job->f, workspace);
 }
 
 cudaError_t launch_wait_expiry_selftest(cudaStream_t stream) {

@@ -86,6 +86,36 @@ __device__ __forceinline__ float row_max_scale(const void* s, int bf16, int64_t 
   return __uint_as_float(mx);
 }
 
+// The same for two rows at once (both rows' loads in flight together).
+__device__ __forceinline__ void row_max_scale2(const void* s, int bf16, int64_t off_a, int64_t off_b, int64_t ld, float& max_a, float& max_b) {
+  uint32_t ma = 0, mb = 0;
+  if (bf16) {
+    const uint4* pa = reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned short*>(s) + off_a);
+    const uint4* pb = reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned short*>(s) + off_b);
+#pragma unroll 2
+    for (int64_t i = 0; i < ld / 8; i++) {
+      const uint4 va = __ldg(pa + i), vb = __ldg(pb + i);
+      const uint32_t wa[4] = {va.x, va.y, va.z, va.w}, wb[4] = {vb.x, vb.y, vb.z, vb.w};
+#pragma unroll
+      for (int e = 0; e < 4; e++) {
+        ma = max(ma, wa[e] << 16); ma = max(ma, wa[e] & 0xFFFF0000u);
+        mb = max(mb, wb[e] << 16); mb = max(mb, wb[e] & 0xFFFF0000u);
+      }
+    }
+  } else {
+    const uint4* pa = reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(s) + off_a);
+    const uint4* pb = reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(s) + off_b);
+#pragma unroll 2
+    for (int64_t i = 0; i < ld / 4; i++) {
+      const uint4 va = __ldg(pa + i), vb = __ldg(pb + i);
+      ma = max(max(ma, va.x), max(va.y, max(va.z, va.w)));
+      mb = max(max(mb, vb.x), max(vb.y, max(vb.z, vb.w)));
+    }
+  }
+  max_a = __uint_as_float(ma);
+  max_b = __uint_as_float(mb);
+}
+
 // Powers of two for a row whose largest scale is mx: mx * up lies in [2^14, 2^15), down = 1 / up.
 // Rows whose scales are all below 2^-100 (an all-zero row included) are treated as if their largest
 // were 2^-100, which keeps both factors normal numbers.
@@ -243,6 +273,11 @@ __device__ __forceinline__ void prepare_w_task(const Args& g, unsigned char* __r
   float up = 0.0f, down = 1.0f;
   if (in) norm_factors(row_max_scale(g.w_scales, g.w_bf16, n * g.ldw_s, g.ldw_s), up, down);
   if (chunk == 0) w_down[n] = down;
+  if (g.sk_counters != nullptr) {
+    // the per-tile arrival counters of the balanced schedule start at zero; every launch leaves them there
+    const int64_t n_chunks = (n_stages + kPrepStages - 1) / kPrepStages, tiles_n = (g.N + TN - 1) / TN;
+    for (int64_t i = (tile_n * n_chunks + chunk) * TN + p; i < g.sk_counter_count; i += tiles_n * n_chunks * TN) g.sk_counters[i] = 0;
+  }
   const int64_t st0 = chunk * kPrepStages;
   const int64_t st1 = st0 + kPrepStages < n_stages ? st0 + kPrepStages : n_stages;
   for (int64_t st = st0; st < st1; st++) {

@@ -123,6 +123,14 @@ struct FoldArgs {
   const unsigned char* w_prep;   // W expanded into [n tile][stage][stage bytes]
   const float* w_down;           // per weight row: the power of two that undoes its normalisation
   EpiArgs ep;                    // what the epilogue does with a finished tile (ep.mode == kEpiPlain: store C as fp32)
+  // Balanced schedule (sk_units > 0): the (tile, stage) pairs of the whole product, tile-major, are cut into
+  // equal runs of sk_units, one per CTA, so a tile's K range may be shared by several CTAs.  A CTA that holds only
+  // part of a tile stores its raw partial accumulator in its own slot of sk_partials and counts itself in
+  // sk_counters[tile][epilogue warp]; the last one to arrive adds the tile's partials in CTA order and finishes it.
+  int64_t sk_units;
+  int32_t* sk_counters;          // [tiles][4]: zeroed by the weight expansion, left at zero by every launch
+  int64_t sk_counter_count;
+  float* sk_partials;            // [2 * CTAs][128][TN]
 };
 // The weight expansion as a job another kernel can run: n_stages x tiles_n tasks of tn threads each
 // (n_stages counts tasks per column tile: single stages of the e4m3 layout, runs of stages of the folded one).
