@@ -565,7 +565,10 @@ def side_measurements(torch, hbmm, inputs, peaks, iters: int):
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
 # (same kernels, same workload); entries are dropped when a kernel changes after its capture.
 NCU_DRAM_BYTES = {
-    ("hbmm_contraction", "conv2_x"): 32.373e6 + 2.103e6,     # profiles/hbmm_fold_kernel_conv2_x.md
+    ("hbmm_contraction", "conv2_x"): 32.339e6 + 3.121e6,     # profiles/conv2_x_conv3_x_kernels.md
+    ("hbmm_contraction", "conv3_x"): 15.173e6 + 0.318e6,
+    ("hbwn_conv", "conv2_x"): 25.924e6 + 3.368e6,            # the contraction kernel of the call (the layout copy is a launch of its own)
+    ("front_end_pack", "conv2_x"): 51.502e6 + 2.750e6,
 }
 
 
