@@ -59,7 +59,8 @@ typedef enum {
   HBMM_PATH_TENSOR_PREPARED = 4, /* HBMM_PATH_TENSOR, and the caller states that the workspace still holds
                            the expanded weight operand an earlier HBMM_PATH_TENSOR / AUTO call with the
                            same W, the same kind of A and this workspace left there (W unchanged
-                           since): the expansion kernel is skipped.  Results are undefined otherwise.  */
+                           since, that call completed without a device-side error): the expansion
+                           kernel is skipped.  Results are undefined otherwise.                       */
   HBMM_PATH_FOLDED = 5, /* tcgen05, both operands packed: every group scale, times a power of two chosen
                            per row, is split into two fp16 pieces (22 significant bits) and folded into
                            the +-1 elements, so that Eq. 7's sum over groups is one fp32 accumulation of
@@ -77,7 +78,9 @@ typedef enum {
                            scale to 2^-17 instead of 2^-26; activations carry 2^-9), 128-column
                            tiles; what HBMM_PATH_AUTO picks for dense bf16 activations.              */
   HBMM_PATH_FOLDED_PREPARED = 6 /* HBMM_PATH_FOLDED with the expanded weights of an earlier
-                           HBMM_PATH_FOLDED / AUTO call reused, as HBMM_PATH_TENSOR_PREPARED          */
+                           HBMM_PATH_FOLDED / AUTO call reused, as HBMM_PATH_TENSOR_PREPARED (the
+                           arrival counters of the shared tiles, which every completed call leaves at
+                           zero, are part of what is reused)                                           */
 } hbmm_path;
 
 /*
@@ -180,9 +183,11 @@ hbmm_status hbmm_binarize_dense(const float *x, int64_t ldx, int64_t rows, int64
 /* Bytes of scratch hbmm_gemm wants for these operands (host pointer `bytes`).  The tensor-core
  * contractions keep the weight operand there, expanded once per call into the tile layout their
  * kernels stream (HBMM: 4 K bytes per weight row, two fp16 pieces; HBWN: 6 K bytes per weight row,
- * three bf16 pieces); 0 when no path needs scratch.  hbmm_gemm still works without it (workspace NULL
- * or too small): it then runs the integer-pipe path (HBMM) or the warp-level kernels (HBWN).
- * The workspace must be 16-byte aligned. */
+ * three bf16 pieces); 0 when no path needs scratch.  For products of few output tiles (fewer than about
+ * a thousand tiles of 128 x 128 or 128 x 64 outputs) the packed x packed figure also holds the slots in
+ * which CTAs that share a tile's K range exchange partial sums (up to 32 MB).  hbmm_gemm still works
+ * without a workspace (NULL or too small): it then runs the integer-pipe path (HBMM) or the warp-level
+ * kernels (HBWN).  The workspace must be 16-byte aligned. */
 hbmm_status hbmm_gemm_workspace_bytes(const hbmm_operand *A, const hbmm_operand *W, size_t *bytes);
 
 /*
