@@ -380,6 +380,224 @@ hbwn_umma_kernel(const Args g, const __grid_constant__ CUtensorMap a_map) {
   }
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// Stride-1 convolution of a 64-channel image with at most 64 filters (the first residual stage of the
+// ResNet workload): every filter tap reads the SAME staged input rows.
+//
+// Output positions are numbered over the zero-padded image, P = (b * Hp + y) * Wp + x with Hp = H + 2 ph and
+// Wp = W + 2 pw, so that the input pixel of tap (i, j) of position P is position P + i Wp + j whatever P is.
+// A tile is 128 consecutive positions; its inputs are the 128 + (kh - 1) Wp + (kw - 1) <= 256 consecutive
+// positions from P0.  Positions are staged in blocks of 128 (one im2col-mode tensor copy whose bounding box is
+// the padded image: 128-byte rows of 64 channels, zeros outside the tensor); a CTA walks a contiguous run of
+// tiles, so block t + 1 is both the halo of tile t and the body of tile t + 1 and every block is fetched once.
+// The MMA of tap (i, j) reads its 128 x 64 activation tile at a start address shifted by (i Wp + j) rows: the
+// 128-byte swizzle is a function of the shared-memory address alone, so a start on any row boundary reads the
+// rows as they were written.  Blocks live in a ring of four slots; a fifth slot behind the last one mirrors
+// slot 0, so that the window of a tile in slot 3 continues in contiguous memory.  The input is read once
+// instead of once per tap (a 3 x 3 filter: 16 KB instead of 144 KB per tile) and the copies run up to three
+// tiles ahead of the MMAs; the weight pieces of all taps stay resident in shared memory.  Positions in the
+// padding columns and rows (x >= Wo or y >= Ho) are computed like the others and dropped by the epilogue.
+constexpr int kRing = 4;                // ring slots; slot kRing mirrors slot 0
+constexpr int kBlockBytes = TM * 128;   // one block of 128 positions x 64 channels
+struct HaloArgs {
+  int32_t Wp, Hp, HpWp, Ho, Wo, B;
+  int32_t kh, kw, ph, pw;
+  int64_t positions;                    // B * Hp * Wp
+  int64_t tiles_per_cta;
+};
+
+template <int NP>
+__global__ void __launch_bounds__(kThreads, 1)
+hbwn_halo_kernel(const Args g, const HaloArgs h, const __grid_constant__ CUtensorMap a_map) {
+  constexpr int TN = 64;
+  using S = Smem<TN, NP>;
+  extern __shared__ __align__(1024) unsigned char smem[];
+  // [ring slots 0..3][mirror of slot 0][weight pieces of every tap][barriers]
+  constexpr int off_b = (kRing + 1) * kBlockBytes;
+  const int off_bar = off_b + g.taps * S::B_STAGE;
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + off_bar);
+  uint64_t* empty = full + kRing;
+  uint64_t* tfull = empty + kRing;
+  uint64_t* tempty = tfull + 2;
+  uint64_t* drain = tempty + 2;
+  uint64_t* wfull = drain + 1;
+  uint32_t* tmem_base_ptr = reinterpret_cast<uint32_t*>(wfull + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_base_ptr + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int64_t n_tiles = (h.positions + TM - 1) / TM;
+  const int64_t tile0 = blockIdx.x * h.tiles_per_cta;
+  const int64_t my_tiles = tile0 < n_tiles ? (n_tiles - tile0 < h.tiles_per_cta ? n_tiles - tile0 : h.tiles_per_cta) : 0;
+
+  pdl_launch_dependents();
+  if (tid == 0) {
+    for (int s = 0; s < kRing; s++) {
+      mbar_init(&full[s], 1);           // the loader's expect_tx arrival; the copies complete the bytes
+      mbar_init(&empty[s], 1);          // MMA commit
+    }
+    for (int b = 0; b < 2; b++) { mbar_init(&tfull[b], 1); mbar_init(&tempty[b], 4); }
+    mbar_init(drain, 1);
+    mbar_init(wfull, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == kMmaWarp) {
+    tmem_alloc(tmem_base_ptr, S::TMEM_COLS);
+    tmem_relinquish();
+  }
+  pdl_wait();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_base_ptr;
+
+  if (warp == kLoaderWarp) {
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&a_map) : "memory");
+      int64_t issued = 0;
+      bool ok = true;
+      if (my_tiles > 0) {
+        mbar_arrive_expect_tx(wfull, static_cast<uint32_t>(g.taps) * S::B_STAGE);
+        for (int t = 0; t < g.taps; t++)
+          bulk_copy_g2s(smem + off_b + t * S::B_STAGE, g.w_prep + static_cast<int64_t>(t) * S::B_STAGE, S::B_STAGE, wfull);
+      }
+      // block k of this CTA = positions (tile0 + k) * 128 ...; one more block than tiles (the last tile's halo)
+      const int64_t n_blocks = my_tiles > 0 ? my_tiles + 1 : 0;
+      const int64_t p_first = tile0 * TM;
+      int32_t b = static_cast<int32_t>(p_first / h.HpWp);
+      const int32_t rem = static_cast<int32_t>(p_first - static_cast<int64_t>(b) * h.HpWp);
+      int32_t y = rem / h.Wp, x = rem - y * h.Wp;
+      for (int64_t k = 0; k < n_blocks; k++) {
+        const int s = static_cast<int>(k & (kRing - 1));
+        if (k >= kRing && !mbar_wait(&empty[s], static_cast<uint32_t>(((k / kRing) & 1) ^ 1), abort_flag, 1)) { ok = false; break; }
+        const bool mirror = s == 0 && k > 0;                  // also the continuation of the tile in the last slot
+        mbar_arrive_expect_tx(&full[s], mirror ? 2u * kBlockBytes : 1u * kBlockBytes);
+        tma_load_im2col_4d(smem + s * kBlockBytes, &a_map, 0, x - h.pw, y - h.ph, b, 0, 0, &full[s]);
+        if (mirror) tma_load_im2col_4d(smem + kRing * kBlockBytes, &a_map, 0, x - h.pw, y - h.ph, b, 0, 0, &full[s]);
+        issued++;
+        x += TM;
+        while (x >= h.Wp) { x -= h.Wp; if (++y == h.Hp) { y = 0; b++; } }
+      }
+      if (!ok || *abort_flag) {
+        // aborted: the copies already issued must land before the CTA's shared memory goes away
+        if (my_tiles > 0) mbar_wait_quiet(wfull, 0, kDrainPolls);
+        const int64_t pending = issued < kRing ? issued : kRing;
+        for (int64_t q = 1; q <= pending; q++) {
+          const int64_t idx = issued - q;
+          mbar_wait_quiet(&full[idx & (kRing - 1)], static_cast<uint32_t>((idx / kRing) & 1), kDrainPolls);
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == kMmaWarp) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = instr_desc(S::NST, kFmtBF16);
+      const uint64_t da0 = smem_desc(smem_u32(smem)), db0 = smem_desc(smem_u32(smem + off_b));
+      const uint64_t da_hi = da0 & 0xFFFFFFFF00000000ull, db_hi = db0 & 0xFFFFFFFF00000000ull;
+      const uint32_t da_lo = static_cast<uint32_t>(da0), db_lo = static_cast<uint32_t>(db0);
+      bool ok = true;
+      if (my_tiles > 0) ok = mbar_wait(wfull, 0, abort_flag, 6) && mbar_wait(&full[0], 0, abort_flag, 2);
+      for (int64_t ti = 0; ti < my_tiles && ok; ti++) {
+        const uint32_t buf = static_cast<uint32_t>(ti & 1);
+        if (ti >= 2) {      // the epilogue must have drained this accumulator (used by tile ti - 2)
+          if (!mbar_wait(&tempty[buf], static_cast<uint32_t>(((ti >> 1) & 1) ^ 1), abort_flag, 3)) { ok = false; break; }
+        }
+        // the tile's own block arrived for the tile before (or above); its halo is block ti + 1
+        const uint32_t s = static_cast<uint32_t>(ti & (kRing - 1));
+        const int64_t k1 = ti + 1;
+        if (!mbar_wait(&full[k1 & (kRing - 1)], static_cast<uint32_t>((k1 / kRing) & 1), abort_flag, 2)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * S::NST;
+        const uint32_t win_lo = da_lo + s * (kBlockBytes >> 4);       // slot 3 continues into the mirror slot
+        int32_t fi = 0, fj = 0;
+        for (int32_t t = 0; t < g.taps; t++) {
+          const uint32_t a_lo = win_lo + static_cast<uint32_t>(fi * h.Wp + fj) * 8u;      // 128-byte rows in 16-byte units
+          const uint32_t b_lo = db_lo + static_cast<uint32_t>(t) * (S::B_STAGE >> 4);
+#pragma unroll
+          for (int ks = 0; ks < KB / 16; ks++)
+            umma_bf16(d_tmem, da_hi | (a_lo + ks * 2), db_hi | (b_lo + ks * 2), idesc, (t | ks) != 0 ? 1u : 0u);
+          if (++fj == h.kw) { fj = 0; fi++; }
+        }
+        umma_commit(&empty[s]);
+        umma_commit(&tfull[buf]);
+      }
+      umma_commit(drain);
+      if (!mbar_wait_quiet(drain, 0, g_spin_limit < kDrainPolls ? kDrainPolls : g_spin_limit)) {
+        atomicCAS(&g_error_word, 0, 4);
+        *abort_flag = 1;
+      }
+    }
+    __syncwarp();
+  } else if (warp < 4) {
+    const int row = warp * 32 + lane;
+    const uint32_t t_lane = static_cast<uint32_t>(warp * 32) << 16;
+    for (int64_t ti = 0; ti < my_tiles; ti++) {
+      const uint32_t buf = static_cast<uint32_t>(ti & 1);
+      // where this thread's position lies in the padded image, and whether it is an output at all
+      const int64_t p = (tile0 + ti) * TM + row;
+      const int32_t b = static_cast<int32_t>(p / h.HpWp);
+      const int32_t rem = static_cast<int32_t>(p - static_cast<int64_t>(b) * h.HpWp);
+      const int32_t y = rem / h.Wp, x = rem - y * h.Wp;
+      const bool valid = b < h.B && y < h.Ho && x < h.Wo;
+      const int64_t m = (static_cast<int64_t>(b) * h.Ho + y) * h.Wo + x;
+      if (!mbar_wait(&tfull[buf], static_cast<uint32_t>((ti >> 1) & 1), abort_flag, 5)) break;
+      tc_fence_after();
+      float* dst = g.C + m * g.ldc;
+      float carry = 0.0f;
+#pragma unroll
+      for (int c = 0; c < TN / 32; c++) {
+        uint32_t v[NP][32];
+        const uint32_t t_addr = tmem_base + t_lane + buf * S::NST + c * 32;
+#pragma unroll
+        for (int i = 0; i < NP; i++) tmem_ld32(t_addr + i * TN, v[i]);
+        tmem_ld_wait();
+        if (valid && g.ep.mode != kEpiPlain) {
+          float cv[32], fs[32], fh[32];
+#pragma unroll
+          for (int e = 0; e < 32; e++) {
+            float acc = __uint_as_float(v[NP - 1][e]);
+#pragma unroll
+            for (int i = NP - 2; i >= 0; i--) acc += __uint_as_float(v[i][e]);
+            cv[e] = acc;
+            const int64_t n = c * 32 + e;
+            fs[e] = (g.ep.bn_scale && n < g.N) ? __ldg(g.ep.bn_scale + n) : 1.0f;
+            fh[e] = (g.ep.bn_shift && n < g.N) ? __ldg(g.ep.bn_shift + n) : 0.0f;
+          }
+          epi::finish_chunk(g.ep, cv, fs, fh, m, c * 32, g.N, c == TN / 32 - 1, TN, carry);
+        } else if (valid) {
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            float o[4];
+#pragma unroll
+            for (int e = 0; e < 4; e++) {    // smallest pieces first
+              float acc = __uint_as_float(v[NP - 1][j + e]);
+#pragma unroll
+              for (int i = NP - 2; i >= 0; i--) acc += __uint_as_float(v[i][j + e]);
+              o[e] = acc;
+            }
+            const int64_t n = c * 32 + j;
+            if (g.c_vec && n + 3 < g.N)
+              *reinterpret_cast<float4*>(dst + n) = make_float4(o[0], o[1], o[2], o[3]);
+            else
+              for (int e = 0; e < 4; e++)
+                if (n + e < g.N) dst[n + e] = o[e];
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tempty[buf]);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == kMmaWarp) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, S::TMEM_COLS);
+  }
+}
+
 Args make_args(const DenseView& A, const PackedView& W, float* C, int64_t ldc) {
   Args g;
   g.a = reinterpret_cast<const __nv_bfloat16*>(A.data); g.lda = A.ld;
@@ -434,6 +652,42 @@ bool make_conv_map(const void* x_nhwc, const ConvGeom& c, int Cp, CUtensorMap* m
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tensor map of the shared-patch kernel: the same NHWC image, but the base pixels walk the whole zero-padded
+// image (Wp x Hp positions per image) and one copy brings `rows` consecutive positions.
+bool make_halo_map(const void* x_nhwc, const ConvGeom& c, int Cp, int rows, CUtensorMap* map) {
+  EncodeIm2colFn fn = encode_im2col_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[4] = {static_cast<cuuint64_t>(c.C), static_cast<cuuint64_t>(c.W), static_cast<cuuint64_t>(c.H),
+                              static_cast<cuuint64_t>(c.B)};
+  const cuuint64_t strides[3] = {static_cast<cuuint64_t>(Cp) * 2, static_cast<cuuint64_t>(c.W) * Cp * 2,
+                                 static_cast<cuuint64_t>(c.H) * c.W * Cp * 2};
+  const int lower[2] = {-c.pw, -c.ph};
+  const int upper[2] = {c.pw, c.ph};
+  const cuuint32_t elem[4] = {1, 1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(x_nhwc), dims, strides, lower, upper, KB,
+            static_cast<cuuint32_t>(rows), elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+constexpr int kHaloSmemMax = 227 * 1024;
+
+// Whether the shared-rows kernel takes this convolution, and its geometry: stride 1, exactly one 64-channel
+// block, one 64-column tile, a tile's window within two blocks of 128 positions, and the five ring slots
+// beside the resident weight pieces in shared memory.
+bool plan_halo(const ConvGeom& c, int64_t N, HaloArgs* h) {
+  if (c.sh != 1 || c.sw != 1 || c.C != KB || N > 64 || c.ph > 127 || c.pw > 127) return false;
+  const int64_t Wp = static_cast<int64_t>(c.W) + 2 * c.pw, Hp = static_cast<int64_t>(c.H) + 2 * c.ph;
+  if (static_cast<int64_t>(c.kh - 1) * Wp + (c.kw - 1) > TM || Hp * Wp >= (int64_t{1} << 31)) return false;
+  const int64_t smem = static_cast<int64_t>(kRing + 1) * kBlockBytes + static_cast<int64_t>(c.kh) * c.kw * Smem<64, 2>::B_STAGE + 256;
+  if (smem > kHaloSmemMax) return false;
+  h->Wp = static_cast<int32_t>(Wp); h->Hp = static_cast<int32_t>(Hp); h->HpWp = static_cast<int32_t>(Hp * Wp);
+  h->Ho = c.Ho; h->Wo = c.Wo; h->B = c.B;
+  h->kh = c.kh; h->kw = c.kw; h->ph = c.ph; h->pw = c.pw;
+  h->positions = static_cast<int64_t>(c.B) * Hp * Wp;
+  h->tiles_per_cta = 0;
+  return true;
+}
+
 Args make_conv_args(const ConvGeom& c, const PackedView& W, float* C, int64_t ldc) {
   Args g;
   g.a = nullptr; g.lda = 0;
@@ -453,7 +707,7 @@ Args make_conv_args(const ConvGeom& c, const PackedView& W, float* C, int64_t ld
 
 template <int TN, int NP>
 cudaError_t launch(Args g, const CUtensorMap& a_map, void* workspace, cudaStream_t stream, const CopyArgs* copy = nullptr,
-                   bool w_prepared = false) {
+                   bool w_prepared = false, const HaloArgs* halo = nullptr) {
   using S = Smem<TN, NP>;
   constexpr int kResBytes = 225 * 1024;
   static DeviceOnce configured;
@@ -478,6 +732,23 @@ cudaError_t launch(Args g, const CUtensorMap& a_map, void* workspace, cudaStream
     prepare_w_pieces_kernel<TN, NP><<<pgrid, 256, 0, stream>>>(g, static_cast<unsigned char*>(workspace));
   }
   g.w_prep = static_cast<const unsigned char*>(workspace);
+  if constexpr (TN == 64 && NP == 2) {
+    if (halo) {
+      static DeviceOnce halo_configured;
+      if (halo_configured.pending(dev)) {
+        const cudaError_t e = cudaFuncSetAttribute(hbwn_halo_kernel<NP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kHaloSmemMax);
+        if (e != cudaSuccess) return e;
+        halo_configured.mark(dev);
+      }
+      const int64_t used = static_cast<int64_t>(kRing + 1) * kBlockBytes + static_cast<int64_t>(g.taps) * S::B_STAGE + 256;
+      const int bytes = static_cast<int>(used > 120 * 1024 ? used : 120 * 1024);          // one CTA per SM
+      const int64_t tiles = (halo->positions + TM - 1) / TM;
+      HaloArgs hh = *halo;
+      hh.tiles_per_cta = (tiles + sms - 1) / sms;                                          // contiguous runs
+      const int64_t ctas = (tiles + hh.tiles_per_cta - 1) / hh.tiles_per_cta;
+      return launch_pdl(hbwn_halo_kernel<NP>, dim3(static_cast<unsigned>(ctas)), dim3(kThreads), bytes, stream, g, hh, a_map);
+    }
+  }
   const int64_t tiles = ((g.M + TM - 1) / TM) * tiles_n;
   const unsigned grid = static_cast<unsigned>(tiles < sms ? tiles : sms);
   // a single column tile whose pieces fit beside the activation ring stays resident in shared memory
@@ -488,9 +759,9 @@ cudaError_t launch(Args g, const CUtensorMap& a_map, void* workspace, cudaStream
 
 // exact: three pieces, 64-column tiles.  Otherwise two pieces: 128-column tiles when there are more than 64 columns.
 cudaError_t launch_any(const Args& g, const CUtensorMap& a_map, void* workspace, cudaStream_t stream, const CopyArgs* copy, bool w_prepared,
-                       bool exact) {
+                       bool exact, const HaloArgs* halo = nullptr) {
   if (exact) return launch<64, 3>(g, a_map, workspace, stream, copy, w_prepared);
-  if (g.N <= 64) return launch<64, 2>(g, a_map, workspace, stream, copy, w_prepared);
+  if (g.N <= 64) return launch<64, 2>(g, a_map, workspace, stream, copy, w_prepared, halo);
   return launch<128, 2>(g, a_map, workspace, stream, copy, w_prepared);
 }
 
@@ -541,19 +812,22 @@ cudaError_t launch_hbwn_umma_conv(const void* x, int x_bf16, void* x_nhwc, int C
   Args g = make_conv_args(c, W, C, ldc);
   if (ep) g.ep = *ep;
   CUtensorMap a_map;
-  if (input_is_nhwc) {
-    // the caller's tensor already is the NHWC bf16 image the tensor copies read (channel pitch Cp): no layout copy
-    if (!make_conv_map(x, c, Cp, &a_map)) return cudaErrorNotSupported;
-    return launch_any(g, a_map, workspace, stream, nullptr, w_prepared, false);
-  }
-  if (!make_conv_map(x_nhwc, c, Cp, &a_map)) return cudaErrorNotSupported;
+  // more row tiles than SMs on a stride-1, 64-channel, 64-filter layer: the kernel that stages one patch per tile
+  HaloArgs halo;
+  int dev = 0, sms = 0;
+  if (current_device(&dev, &sms) != cudaSuccess) return cudaErrorInvalidDevice;
+  const bool use_halo = plan_halo(c, g.N, &halo) && (g.M + TM - 1) / TM > sms;
+  const void* image = input_is_nhwc ? x : x_nhwc;
+  if (use_halo ? !make_halo_map(image, c, Cp, TM, &a_map) : !make_conv_map(image, c, Cp, &a_map)) return cudaErrorNotSupported;
+  // input_is_nhwc: the caller's tensor already is the NHWC bf16 image the tensor copies read (channel pitch Cp)
+  if (input_is_nhwc) return launch_any(g, a_map, workspace, stream, nullptr, w_prepared, false, use_halo ? &halo : nullptr);
   CopyArgs cp;
   cp.x = x; cp.x_bf16 = x_bf16; cp.C = c.C; cp.Cp = Cp; cp.HW = static_cast<int64_t>(c.H) * c.W;
   cp.out = static_cast<unsigned short*>(x_nhwc);
   cp.gx = static_cast<int32_t>((cp.HW + kNhwcPB - 1) / kNhwcPB);
   cp.gy = (Cp + kNhwcCB - 1) / kNhwcCB;
   cp.n_copy = static_cast<int64_t>(cp.gx) * cp.gy * c.B;
-  return launch_any(g, a_map, workspace, stream, &cp, w_prepared, false);
+  return launch_any(g, a_map, workspace, stream, &cp, w_prepared, false, use_halo ? &halo : nullptr);
 }
 
 cudaError_t hbwn_umma_health(int op, int* value) {

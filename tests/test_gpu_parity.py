@@ -352,6 +352,13 @@ CONV_CASES = [
     (1, 64, 12, 12, 16, 1, 1, 1, 0, 1, 64, True, True),     # 1x1
     (2, 64, 6, 6, 24, 5, 5, 1, 2, 1, 1600, True, True),     # 5x5, one weight group per row
     (5, 192, 14, 14, 130, 3, 3, 1, 1, 1, 96, False, True),  # three blocks, several tiles per image, post-ReLU
+    # HBWN, 64 channels, at most 64 filters, stride 1, more row tiles than SMs: every tap reads one staged run of
+    # input rows (positions numbered over the padded image; tiles cross image rows, images and the end)
+    (8, 64, 50, 50, 40, 3, 3, 1, 1, 1, 32, True, True),     # ragged filters
+    (10, 64, 47, 45, 64, 3, 3, 1, 0, 1, 64, True, False),   # no padding, odd extents, fp32 input
+    (6, 64, 56, 56, 24, 3, 3, 1, 2, 1, 32, False, True),    # padding wider than the filter needs, post-ReLU
+    (8, 64, 51, 51, 33, 2, 2, 1, 0, 1, 32, True, True),     # 2 x 2 filter
+    (6, 64, 60, 60, 16, 1, 1, 1, 0, 1, 32, True, True),     # 1 x 1: no halo at all
 ]
 
 
@@ -722,7 +729,7 @@ def _nhwc_to_nchw(z, B, Ho, Wo):
     return np.ascontiguousarray(z.reshape(B, Ho, Wo, -1).transpose(0, 3, 1, 2))
 
 
-@pytest.mark.parametrize("B,C,H,F1,F2", [(3, 64, 12, 64, 72), (2, 128, 7, 128, 40)])
+@pytest.mark.parametrize("B,C,H,F1,F2", [(3, 64, 12, 64, 72), (2, 128, 7, 128, 40), (7, 64, 54, 64, 48)])
 def test_two_dense_activation_convolutions_chained_through_the_epilogue(hb, B, C, H, F1, F2):
     """Layer 1: convolution (bf16 activations x Hadamard-binary weights) -> ReLU -> the next block's batch-norm map ->
     NHWC bf16, written by the epilogue.  Layer 2 reads that tensor as it is (HBMM_CONV_INPUT_NHWC).  Layer 1 is held to
