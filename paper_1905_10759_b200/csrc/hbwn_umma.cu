@@ -381,6 +381,245 @@ hbwn_umma_kernel(const Args g, const __grid_constant__ CUtensorMap a_map) {
 }
 
 // ---------------------------------------------------------------------------------------------------------
+// The same contraction on CTA pairs.  The single-CTA kernel above is bound by shared-memory traffic: per
+// 64-element stage of a 128 x 128 tile it writes 48 KB (16 KB of activations, 32 KB of stacked weight pieces)
+// and the tensor core reads them back, 96 KB against 512 clocks of MMA issue.  Two CTAs on neighbouring SMs
+// that work on vertically adjacent row tiles need the SAME weight stage, so they run as a cluster of two and
+// issue one 256 x 256 x 16 MMA (tcgen05 cta_group::2): each CTA stages its own 128 activation rows and only
+// ONE of the two weight pieces (the MMA reads the second operand's halves from both CTAs' shared memories), 32 KB
+// per stage and CTA, and the ring holds six stages instead of four.  Each CTA's tensor memory receives its own
+// 128 rows of the 256 stacked columns, so the epilogue is unchanged.
+//   rank 0: its loader thread posts the expected bytes of BOTH CTAs' copies on its `full` barrier, its MMA
+//           thread issues every MMA of the pair and commits to the `empty` / `tfull` barriers of both CTAs;
+//   rank 1: its loader thread fetches its tiles with copies that complete on rank 0's `full` barrier (no
+//           multicast: every CTA fetches what it stages itself); its MMA warp only owns the TMEM allocation;
+//   both  : the epilogue warps drain their CTA's accumulator and arrive on rank 0's `tempty` barrier.
+template <int TN, int NP>
+struct PairSmem {
+  static constexpr int NST = NP * TN;                      // stacked weight rows = MMA N
+  static constexpr int A_STAGE = TM * 128;                 // this CTA's 128 activation rows
+  static constexpr int B_HALF = (NST / 2) * 128;           // this CTA's half of the stacked weight rows
+  static constexpr int STAGE = A_STAGE + B_HALF;
+  static constexpr int STAGES = (200 * 1024) / STAGE;
+  static constexpr int OFF_A = 0;
+  static constexpr int OFF_B = STAGES * A_STAGE;
+  static constexpr int OFF_BAR = STAGES * STAGE;
+  static constexpr int NBAR = 2 * STAGES + 4 + 1;          // full, empty, tfull[2], tempty[2], drain
+  static constexpr int BYTES = OFF_BAR + NBAR * 8 + 16;
+  static constexpr int TMEM_COLS = 512;
+  static_assert(NST == 256 && B_HALF == Smem<TN, NP>::B_PIECE, "each CTA of the pair stages exactly one weight piece");
+};
+
+template <int TN, int NP>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+hbwn_pair_kernel(const Args g, const __grid_constant__ CUtensorMap a_map, const __grid_constant__ CUtensorMap b_map) {
+  using S = PairSmem<TN, NP>;
+  constexpr int STAGES = S::STAGES;
+  extern __shared__ __align__(1024) unsigned char smem[];
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + S::OFF_BAR);
+  uint64_t* empty = full + STAGES;
+  uint64_t* tfull = empty + STAGES;
+  uint64_t* tempty = tfull + 2;
+  uint64_t* drain = tempty + 2;
+  uint32_t* tmem_base_ptr = reinterpret_cast<uint32_t*>(drain + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_base_ptr + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int64_t pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int64_t tiles_n = (g.N + TN - 1) / TN, tiles_m = (g.M + 2 * TM - 1) / (2 * TM);     // tiles of 256 rows
+  const int64_t n_tiles = tiles_m * tiles_n;
+  const int64_t n_kb = g.n_kb;
+  const int64_t my_tiles = pair < n_tiles ? (n_tiles - pair + n_pairs - 1) / n_pairs : 0;
+
+  pdl_launch_dependents();
+  if (tid == 0) {
+    for (int s = 0; s < STAGES; s++) {
+      mbar_init(&full[s], 1);           // rank 0: its loader's expect_tx arrival; the copies of both CTAs complete the bytes
+      mbar_init(&empty[s], 1);          // MMA commit (to both CTAs)
+    }
+    for (int b = 0; b < 2; b++) { mbar_init(&tfull[b], 1); mbar_init(&tempty[b], 8); }     // 4 epilogue warps x 2 CTAs
+    mbar_init(drain, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == kMmaWarp) {
+    tmem_alloc_pair(tmem_base_ptr, S::TMEM_COLS);
+    tmem_relinquish_pair();
+  }
+  pdl_wait();
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                  // both CTAs' barriers exist before either signals the other
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_base_ptr;
+
+  if (warp == kLoaderWarp) {
+    // =========================== loader (both CTAs) ===========================
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&a_map) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&b_map) : "memory");
+      const uint32_t full0 = mapa_rank(smem_u32(full), 0);          // rank 0's `full` barriers
+      int s = 0;
+      uint32_t round = 0;
+      int64_t issued = 0;
+      bool ok = true;
+      for (int64_t ti = 0; ti < my_tiles && ok; ti++) {
+        const int64_t tile = pair + ti * n_pairs;
+        const int64_t tile_m = tile / tiles_n, tile_n = tile - tile_m * tiles_n;
+        const int64_t m0 = tile_m * (2 * TM) + rank * TM;
+        // rows of the weight-piece matrix: [column tile][k block][piece][TN rows]; this CTA stages piece `rank`
+        int32_t b_row = static_cast<int32_t>((tile_n * n_kb * NP + rank) * TN);
+        int32_t b = 0, h0 = 0, w0 = 0;
+        if (g.conv) {
+          b = static_cast<int32_t>(m0 / g.HoWo);
+          const int32_t rem = static_cast<int32_t>(m0 - static_cast<int64_t>(b) * g.HoWo);
+          const int32_t yo = rem / g.Wo, xo = rem - yo * g.Wo;
+          h0 = yo * g.sh - g.ph;
+          w0 = xo * g.sw - g.pw;
+        }
+        int32_t cb = 0, fi = 0, fj = 0;
+        for (int32_t kb = 0; kb < static_cast<int32_t>(n_kb); kb++) {
+          if (round > 0 && !mbar_wait(&empty[s], (round & 1) ^ 1, abort_flag, 1)) { ok = false; break; }
+          if (rank == 0) mbar_arrive_expect_tx(&full[s], 2 * S::STAGE);
+          const uint32_t bar = full0 + s * 8;
+          if (g.conv)
+            tma_load_im2col_4d_pair(smem + S::OFF_A + s * S::A_STAGE, &a_map, cb * KB, w0, h0, b, static_cast<uint16_t>(fj),
+                                    static_cast<uint16_t>(fi), bar);
+          else
+            tma_load_2d_pair(smem + S::OFF_A + s * S::A_STAGE, &a_map, kb * KB, static_cast<int32_t>(m0), bar);
+          tma_load_2d_pair(smem + S::OFF_B + s * S::B_HALF, &b_map, 0, b_row, bar);
+          b_row += NP * TN;
+          issued++;
+          if (++cb == g.cblocks) { cb = 0; if (++fj == g.kw) { fj = 0; fi++; } }
+          if (++s == STAGES) { s = 0; round++; }
+        }
+      }
+      if (!ok || *abort_flag) {
+        // aborted: copies already issued must land before this CTA's shared memory goes away.  Rank 0 can watch
+        // its barriers; rank 1 cannot see them and gives its own copies a fixed time that is far longer than a copy.
+        if (rank == 0) {
+          const int64_t pending = issued < STAGES ? issued : STAGES;
+          for (int64_t q = 1; q <= pending; q++) {
+            const int64_t idx = issued - q;
+            mbar_wait_quiet(&full[idx % STAGES], static_cast<uint32_t>((idx / STAGES) & 1), kDrainPolls);
+          }
+        } else {
+          for (int q = 0; q < 64; q++) __nanosleep(1000);
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == kMmaWarp) {
+    // =========================== MMA issuer (rank 0) ===========================
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = instr_desc_pair(S::NST, kFmtBF16);
+      const uint64_t da0 = smem_desc(smem_u32(smem + S::OFF_A)), db0 = smem_desc(smem_u32(smem + S::OFF_B));
+      const uint64_t da_hi = da0 & 0xFFFFFFFF00000000ull, db_hi = db0 & 0xFFFFFFFF00000000ull;
+      const uint32_t da_lo = static_cast<uint32_t>(da0), db_lo = static_cast<uint32_t>(db0);
+      const uint32_t full_a = smem_u32(full), empty_a = smem_u32(empty), tfull_a = smem_u32(tfull), tempty_a = smem_u32(tempty);
+      uint32_t s = 0, full_par = 0;
+      bool ok = true;
+      for (int64_t ti = 0; ti < my_tiles && ok; ti++) {
+        const uint32_t buf = static_cast<uint32_t>(ti & 1);
+        if (ti >= 2) {      // the epilogues of both CTAs must have drained this accumulator (used by tile ti - 2)
+          if (!mbar_wait_a(tempty_a + buf * 8, static_cast<uint32_t>(((ti >> 1) & 1) ^ 1), abort_flag, 3)) { ok = false; break; }
+          tc_fence_after();
+        }
+        const uint32_t d_tmem = tmem_base + buf * S::NST;
+        for (int64_t kb = 0; kb < n_kb; kb++) {
+          if (!mbar_wait_a(full_a + s * 8, full_par, abort_flag, 2)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_lo = da_lo + s * (S::A_STAGE >> 4);
+          const uint32_t b_lo = db_lo + s * (S::B_HALF >> 4);
+#pragma unroll
+          for (int ks = 0; ks < KB / 16; ks++)
+            umma_bf16_pair(d_tmem, da_hi | (a_lo + ks * 2), db_hi | (b_lo + ks * 2), idesc, (kb | ks) != 0 ? 1u : 0u);
+          umma_commit_pair_mc(empty_a + s * 8, 3);
+          if (++s == STAGES) { s = 0; full_par ^= 1; }
+        }
+        if (ok) umma_commit_pair_mc(tfull_a + buf * 8, 3);
+      }
+      // every MMA issued so far has retired (in both CTAs) before tensor memory is released -- also after an abort
+      umma_commit_pair(smem_u32(drain));
+      if (!mbar_wait_quiet(drain, 0, g_spin_limit < kDrainPolls ? kDrainPolls : g_spin_limit)) {
+        atomicCAS(&g_error_word, 0, 4);
+        *abort_flag = 1;
+      }
+    }
+    __syncwarp();
+  } else if (warp < 4) {
+    // =========================== epilogue (both CTAs) ===========================
+    const int row = warp * 32 + lane;
+    const uint32_t t_lane = static_cast<uint32_t>(warp * 32) << 16;
+    const uint32_t tempty0 = mapa_rank(smem_u32(tempty), 0);        // rank 0's `tempty` barriers
+    for (int64_t ti = 0; ti < my_tiles; ti++) {
+      const uint32_t buf = static_cast<uint32_t>(ti & 1);
+      if (!mbar_wait(&tfull[buf], static_cast<uint32_t>((ti >> 1) & 1), abort_flag, 5)) break;
+      tc_fence_after();
+      const int64_t tile = pair + ti * n_pairs;
+      const int64_t m = (tile / tiles_n) * (2 * TM) + rank * TM + row, nb = (tile % tiles_n) * TN;
+      float* dst = g.C + m * g.ldc + nb;
+      float carry = 0.0f;
+#pragma unroll
+      for (int c = 0; c < TN / 32; c++) {
+        uint32_t v[NP][32];
+        const uint32_t t_addr = tmem_base + t_lane + buf * S::NST + c * 32;
+#pragma unroll
+        for (int i = 0; i < NP; i++) tmem_ld32(t_addr + i * TN, v[i]);
+        tmem_ld_wait();
+        if (m < g.M && g.ep.mode != kEpiPlain) {
+          float cv[32], fs[32], fh[32];
+#pragma unroll
+          for (int e = 0; e < 32; e++) {
+            float acc = __uint_as_float(v[NP - 1][e]);
+#pragma unroll
+            for (int i = NP - 2; i >= 0; i--) acc += __uint_as_float(v[i][e]);
+            cv[e] = acc;
+            const int64_t n = nb + c * 32 + e;
+            fs[e] = (g.ep.bn_scale && n < g.N) ? __ldg(g.ep.bn_scale + n) : 1.0f;
+            fh[e] = (g.ep.bn_shift && n < g.N) ? __ldg(g.ep.bn_shift + n) : 0.0f;
+          }
+          epi::finish_chunk(g.ep, cv, fs, fh, m, nb + c * 32, g.N, c == TN / 32 - 1, nb + TN, carry);
+        } else if (m < g.M) {
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            float o[4];
+#pragma unroll
+            for (int e = 0; e < 4; e++) {    // smallest pieces first
+              float acc = __uint_as_float(v[NP - 1][j + e]);
+#pragma unroll
+              for (int i = NP - 2; i >= 0; i--) acc += __uint_as_float(v[i][j + e]);
+              o[e] = acc;
+            }
+            const int64_t n = nb + c * 32 + j;
+            if (g.c_vec && n + 3 < g.N)
+              *reinterpret_cast<float4*>(dst + c * 32 + j) = make_float4(o[0], o[1], o[2], o[3]);
+            else
+              for (int e = 0; e < 4; e++)
+                if (n + e < g.N) dst[c * 32 + j + e] = o[e];
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(tempty0 + buf * 8);
+    }
+  }
+
+  // Neither CTA may leave while the other can still reach into it (rank 0's MMAs read rank 1's shared memory and
+  // write its tensor memory; rank 1's copies and epilogue warps signal rank 0's barriers): rank 0 arrives here
+  // only after its drain wait.
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == kMmaWarp) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, S::TMEM_COLS);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------
 // Stride-1 convolution of a 64-channel image with at most 64 filters (the first residual stage of the
 // ResNet workload): every filter tap reads the SAME staged input rows.
 //
@@ -669,6 +908,21 @@ bool make_halo_map(const void* x_nhwc, const ConvGeom& c, int Cp, int rows, CUte
             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tensor map of the prepared weight pieces for the CTA-pair kernel: rows of 128 bytes (64 bf16) in the order the
+// preparation kernel wrote them, already swizzled, so the copy uses no swizzle of its own; one box = one piece of
+// one stage (TN rows).
+bool make_pieces_map(const void* w_prep, int64_t rows, int box_rows, CUtensorMap* map) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn || rows >= (int64_t{1} << 31)) return false;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(KB), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {128};
+  const cuuint32_t box[2] = {KB, static_cast<cuuint32_t>(box_rows)};
+  const cuuint32_t elem[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(w_prep), dims, strides, box, elem,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 constexpr int kHaloSmemMax = 227 * 1024;
 
 // Whether the shared-rows kernel takes this convolution, and its geometry: stride 1, exactly one 64-channel
@@ -747,6 +1001,23 @@ cudaError_t launch(Args g, const CUtensorMap& a_map, void* workspace, cudaStream
       hh.tiles_per_cta = (tiles + sms - 1) / sms;                                          // contiguous runs
       const int64_t ctas = (tiles + hh.tiles_per_cta - 1) / hh.tiles_per_cta;
       return launch_pdl(hbwn_halo_kernel<NP>, dim3(static_cast<unsigned>(ctas)), dim3(kThreads), bytes, stream, g, hh, a_map);
+    }
+  }
+  if constexpr (TN == 128 && NP == 2) {
+    // at least two row tiles: CTA pairs that share each weight stage
+    if (g.M > TM && sms >= 2) {
+      using P = PairSmem<TN, NP>;
+      static DeviceOnce pair_configured;
+      if (pair_configured.pending(dev)) {
+        const cudaError_t e = cudaFuncSetAttribute(hbwn_pair_kernel<TN, NP>, cudaFuncAttributeMaxDynamicSharedMemorySize, P::BYTES);
+        if (e != cudaSuccess) return e;
+        pair_configured.mark(dev);
+      }
+      CUtensorMap b_map;
+      if (!make_pieces_map(g.w_prep, tiles_n * n_kb * NP * TN, TN, &b_map)) return cudaErrorNotSupported;
+      const int64_t pair_tiles = ((g.M + 2 * TM - 1) / (2 * TM)) * tiles_n;
+      const int64_t pairs = pair_tiles < sms / 2 ? pair_tiles : sms / 2;
+      return launch_pdl(hbwn_pair_kernel<TN, NP>, dim3(static_cast<unsigned>(2 * pairs)), dim3(kThreads), P::BYTES, stream, g, a_map, b_map);
     }
   }
   const int64_t tiles = ((g.M + TM - 1) / TM) * tiles_n;

@@ -204,6 +204,64 @@ __device__ __forceinline__ void umma_bf16_overwrite(uint32_t d_tmem, uint64_t a_
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc) : "memory");
 }
 
+// ---- CTA pairs: a cluster of two CTAs on neighbouring SMs issues one MMA over 256 rows (128 per CTA) whose
+// second operand is split between the two CTAs' shared memories, so each CTA stages and serves half of it.
+// The CTA of cluster rank 0 issues the MMAs and owns the barriers the copies of both CTAs complete on.
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// every thread of both CTAs
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of the same shared-memory location in the CTA of the given cluster rank (shared::cluster window)
+__device__ __forceinline__ uint32_t mapa_rank(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// Tensor memory of both CTAs at once: the same warp of each CTA executes these with the same arguments.
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t* dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols));
+}
+__device__ __forceinline__ void tmem_relinquish_pair() { asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::); }
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t addr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols));
+}
+// D[tmem of both CTAs] (+)= A * B^T, 256 x N x 16: each CTA's descriptor addresses name its own 128 rows of A and
+// its own N / 2 rows of B.  Issued by one thread of the rank-0 CTA.
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrives, once the pair's MMAs issued so far have completed, on the barrier at this address in every CTA of the mask.
+__device__ __forceinline__ void umma_commit_pair_mc(uint32_t bar, uint16_t cta_mask) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(cta_mask) : "memory");
+}
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// Tensor copies into this CTA's shared memory whose bytes complete on a barrier of either CTA of the pair
+// (`bar` is a shared::cluster address).  No multicast: each CTA fetches its own tiles.
+__device__ __forceinline__ void tma_load_2d_pair(void* dst, const void* tensor_map, int32_t x, int32_t y, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(smem_u32(dst)), "l"(tensor_map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_im2col_4d_pair(void* dst, const void* tensor_map, int32_t c, int32_t w, int32_t h, int32_t n,
+                                                        uint16_t w_off, uint16_t h_off, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.4d.im2col.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6], {%7, %8};"
+               ::"r"(smem_u32(dst)), "l"(tensor_map), "r"(c), "r"(w), "r"(h), "r"(n), "r"(bar), "h"(w_off), "h"(h_off)
+               : "memory");
+}
+
 // Operand tiles in shared memory use the 128-byte-swizzled K-major layout of the tensor core: a row is
 // 128 contiguous bytes (the four K-words of a stage, 32 bytes each), rows follow each other, and the
 // 16-byte piece c of row r is stored at piece position c ^ (r % 8).  A tile starts on a 1024-byte
@@ -227,6 +285,11 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
 __host__ __device__ constexpr uint32_t instr_desc(int n, uint32_t ab_format) {
   return (1u << 4) | (ab_format << 7) | (ab_format << 10) | (static_cast<uint32_t>(n >> 3) << 17) |
          (static_cast<uint32_t>(TM >> 4) << 24);
+}
+// The same for a CTA pair: M = 256 (128 rows in each CTA).
+__host__ __device__ constexpr uint32_t instr_desc_pair(int n, uint32_t ab_format) {
+  return (1u << 4) | (ab_format << 7) | (ab_format << 10) | (static_cast<uint32_t>(n >> 3) << 17) |
+         (static_cast<uint32_t>((2 * TM) >> 4) << 24);
 }
 constexpr uint32_t kFmtE4M3 = 0, kFmtBF16 = 1;   // kind::f8f6f4 / kind::f16 operand codes
 constexpr uint32_t kFmtF16 = 0;                  // kind::f16 with fp16 operands
