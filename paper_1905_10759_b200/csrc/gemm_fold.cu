@@ -36,6 +36,7 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include "kernels.h"
+#include "tensor_map.h"
 #include "umma_common.cuh"
 #include "gemm_fold_prep.cuh"
 #include "epilogue.cuh"
@@ -58,10 +59,69 @@ constexpr int kThreads = (kFirstScoutWarp + kScoutWarps) * 32;
 // Stages of packed words + scales each producer thread keeps in flight; fewer when a word has many scales.
 template <int SUBW> struct DepthFor { static constexpr int value = SUBW == 1 ? 4 : (SUBW <= 4 ? 2 : 1); };
 
+// Sub-word groups (beta_a = 32 / ASUB): a stage of a tile needs 2 ASUB scales per row -- up to 128 bytes a row, 16 KB a
+// stage, against 1 KB of packed words.  Loaded by the producer threads themselves (one row per lane) these are
+// hundreds of scattered 16-byte requests per stage with nothing to hide their latency behind; instead the loader
+// thread brings the stage's [128 rows][2 ASUB] block of fp32 scales with one tensor copy into a ring beside the
+// weight stages, and the producers read their rows from shared memory.  The copy swizzles the rows' 16-byte
+// pieces (by the row number, as wide as the row is long), so 8 consecutive rows read 8 different bank groups.
+constexpr int kStagedFrom = 4;          // groups per word from which the scales go through shared memory (beta_a <= 8)
+constexpr int64_t kRowMaxFrom = 512;    // scales per row from which a kernel of its own finds the rows' largest scales
+template <int TN, int ASUB>
+struct ScaleRing {
+  static constexpr int ROW_BYTES = 8 * ASUB;                       // two words' scales
+  static constexpr int STAGE = TM * ROW_BYTES;
+  // The ring is deeper than the ring of weight stages: the block of stage g + LEAD is requested when stage g's weight
+  // copy is (its slot last served stage g - STAGES, whose MMAs -- hence whose producers -- are done by then).
+  static constexpr int NS = ASUB == 16 ? Smem<TN>::STAGES + 1 : 2 * Smem<TN>::STAGES;
+  static constexpr int LEAD = NS - Smem<TN>::STAGES;
+  static constexpr int OFF = (Smem<TN>::USED + 1023) / 1024 * 1024;
+  static constexpr int OFF_BAR = OFF + NS * STAGE;                 // sfull[NS]
+  static constexpr int BYTES = ASUB == 1 ? Smem<TN>::BYTES : OFF_BAR + NS * 8 + 16;
+  // byte offset of the 16-byte piece c of row p inside a stage block
+  __device__ static __forceinline__ int piece(int p, int c) {
+    if (ASUB == 16) return p * 128 + ((c ^ (p & 7)) << 4);
+    if (ASUB == 8) return p * 64 + ((c ^ ((p >> 1) & 3)) << 4);
+    if (ASUB == 4) return p * 32 + ((c ^ ((p >> 2) & 1)) << 4);
+    return p * 16;
+  }
+};
+
 template <int TN>
 __global__ void __launch_bounds__(TN)
 prepare_w_fold_kernel(const Args g, unsigned char* __restrict__ out, float* __restrict__ w_down) {
   prepare_w_task<TN>(g, out, w_down, blockIdx.x, blockIdx.y, threadIdx.x);
+}
+
+// Largest scale of every row of an operand with many scales per row (sub-word groups): one warp per row, consecutive
+// lanes on consecutive 16-byte vectors.  Scales are >= 0, so their bit patterns order like the values; entries past the
+// last group are stored zeros.
+__global__ void __launch_bounds__(256)
+row_max_kernel(const float* __restrict__ scales, int64_t ld, int64_t M, float* __restrict__ out) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int lane = threadIdx.x & 31;
+  const int64_t m = static_cast<int64_t>(blockIdx.x) * 8 + (threadIdx.x >> 5);
+  if (m >= M) return;
+  const uint4* p = reinterpret_cast<const uint4*>(scales + m * ld);
+  const int64_t n_vec = ld / 4;
+  uint32_t x0 = 0, x1 = 0, x2 = 0, x3 = 0;
+  int64_t j = lane;
+  for (; j + 96 < n_vec; j += 128) {
+    const uint4 a = __ldg(p + j), b = __ldg(p + j + 32), c = __ldg(p + j + 64), d = __ldg(p + j + 96);
+    x0 = max(max(x0, a.x), max(a.y, max(a.z, a.w)));
+    x1 = max(max(x1, b.x), max(b.y, max(b.z, b.w)));
+    x2 = max(max(x2, c.x), max(c.y, max(c.z, c.w)));
+    x3 = max(max(x3, d.x), max(d.y, max(d.z, d.w)));
+  }
+  for (; j < n_vec; j += 32) {
+    const uint4 a = __ldg(p + j);
+    x0 = max(max(x0, a.x), max(a.y, max(a.z, a.w)));
+  }
+  uint32_t x = max(max(x0, x1), max(x2, x3));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x = max(x, __shfl_xor_sync(0xFFFFFFFFu, x, o));
+  if (lane == 0) out[m] = __uint_as_float(x);
 }
 
 // Walks the stages a producer thread owns (every second stage of the CTA's stream of tiles) and keeps
@@ -81,12 +141,15 @@ struct StageCursor {
 // instantiation carries none of its code.
 template <int TN, int ASUB, bool FUSE, bool BAL>
 __global__ void __launch_bounds__(kThreads, 1)
-hbmm_fold_kernel(const Args g) {
+hbmm_fold_kernel(const Args g, const __grid_constant__ CUtensorMap s_map) {
   using S = Smem<TN>;
+  using SR = ScaleRing<TN, ASUB>;
+  const bool staged = ASUB > 1 && g.a_staged;                    // the stage's scales come through shared memory
   constexpr int kDepth = DepthFor<ASUB>::value;
   constexpr int STAGES = S::STAGES;
   extern __shared__ __align__(1024) unsigned char smem[];
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + S::OFF_BAR);
+  uint64_t* sfull = reinterpret_cast<uint64_t*>(smem + (ASUB > 1 ? SR::OFF_BAR : S::OFF_BAR));   // the scale block of a stage has arrived
   uint64_t* empty = full + STAGES;
   uint64_t* tfull = empty + STAGES;
   uint64_t* tempty = tfull + 2;
@@ -133,6 +196,8 @@ hbmm_fold_kernel(const Args g) {
     }
     for (int b = 0; b < 2; b++) { mbar_init(&tfull[b], 1); mbar_init(&tempty[b], kEpilogueWarps); }
     mbar_init(drain, 1);
+    if (ASUB > 1)
+      for (int s = 0; s < SR::NS; s++) mbar_init(&sfull[s], 1);        // the loader's expect_tx arrival; the copy completes the bytes
     for (int r = 0; r < kRowSlots; r++) { mbar_init(&rowfull[r], kScoutWarps); mbar_init(&rowempty[r], kEpilogueWarps); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -190,7 +255,9 @@ hbmm_fold_kernel(const Args g) {
       const uint32_t wi = static_cast<uint32_t>(c.st) * WPS;
       if (c.in && wi < n_words) {
         w = __ldg(reinterpret_cast<const uint2*>(c.bptr + wi));      // the row is padded with zero words to a multiple of four
-        if (ASUB > 1) {
+        if (ASUB > 1 && staged) {
+          // the scales arrive in shared memory
+        } else if (ASUB > 1) {
           // K is a multiple of 32 here, so every word has all its ASUB groups
           float lo[ASUB], hi[ASUB];
           load_scaled<(ASUB > 1 ? ASUB : 2)>(g.a_scales, g.a_bf16, c.srow + static_cast<int64_t>(wi) * ASUB, 1.0f,
@@ -242,6 +309,19 @@ hbmm_fold_kernel(const Args g) {
           if (ok) {
             // stage s: columns [0, 32) piece 1, [32, 64) piece 2; word slot q in columns 16 q .. 16 q + 15 of its piece
             const uint32_t a_col = tmem_base + t_lane + S::A_BASE + static_cast<uint32_t>(s) * S::A_COLS;
+            if (ASUB > 1 && staged) {
+              // this row's 2 ASUB scales of the stage, from the block the loader's tensor copy laid down
+              const int ss = static_cast<int>(my % SR::NS);
+              if (!mbar_wait(&sfull[ss], static_cast<uint32_t>((my / SR::NS) & 1), abort_flag, 9)) ok = false;
+              ok = __all_sync(0xFFFFFFFFu, ok);
+              if (!ok) break;
+              const unsigned char* blk = smem + SR::OFF + ss * SR::STAGE;
+#pragma unroll
+              for (int c = 0; c < (2 * ASUB) / 4; c++) {
+                const float4 v = *reinterpret_cast<const float4*>(blk + SR::piece(p, c));
+                sc[u][4 * c] = v.x; sc[u][4 * c + 1] = v.y; sc[u][4 * c + 2] = v.z; sc[u][4 * c + 3] = v.w;
+              }
+            }
 #pragma unroll
             for (int qw = 0; qw < WPS; qw++) {
               uint32_t p1[16], p2[16];
@@ -278,7 +358,18 @@ hbmm_fold_kernel(const Args g) {
       const int slot = static_cast<int>(ti & (kRowSlots - 1));
       if (ti >= kRowSlots && !mbar_wait(&rowempty[slot], static_cast<uint32_t>(((ti / kRowSlots) & 1) ^ 1), abort_flag, 8)) break;
       const int64_t tile = seg_tile(ti);
-      {
+      if (ASUB > 1 && g.a_rowmax) {
+        // long rows of scales: a kernel of its own has reduced every row to its largest scale
+        const int64_t ma = (tile / tiles_n) * TM + p0, mb = ma + kScoutWarps * 32;
+        float up = 0.0f, down = 1.0f;
+        if (ma < g.M) norm_factors(__ldg(g.a_rowmax + ma), up, down);
+        rowup[slot * TM + p0] = up;
+        rowdown[slot * TM + p0] = down;
+        up = 0.0f; down = 1.0f;
+        if (mb < g.M) norm_factors(__ldg(g.a_rowmax + mb), up, down);
+        rowup[slot * TM + p0 + kScoutWarps * 32] = up;
+        rowdown[slot * TM + p0 + kScoutWarps * 32] = down;
+      } else {
         // rows p0 and p0 + 64, scanned together so that both rows' loads are in flight at once
         const int64_t ma = (tile / tiles_n) * TM + p0, mb = ma + kScoutWarps * 32;
         float xa, xb;
@@ -300,6 +391,19 @@ hbmm_fold_kernel(const Args g) {
     if (lane == 0) {
       int64_t gst = 0;
       bool ok = true;
+      // sub-word groups: the next scale block to request -- [128 rows][2 ASUB scales] of one stage; rows past M and groups
+      // past the last one arrive as zeros
+      int64_t sc_ti = 0, sc_st = seg_begin(0), sc_g = 0;
+      auto issue_scales = [&]() {
+        const int slot = static_cast<int>(sc_g % SR::NS);
+        mbar_arrive_expect_tx(&sfull[slot], SR::STAGE);
+        tma_load_2d(smem + SR::OFF + slot * SR::STAGE, &s_map, static_cast<int32_t>(sc_st * (2 * ASUB)),
+                    static_cast<int32_t>((seg_tile(sc_ti) / tiles_n) * TM), &sfull[slot]);
+        sc_g++;
+        if (++sc_st >= seg_end(sc_ti)) { sc_ti++; sc_st = seg_begin(sc_ti); }
+      };
+      if (ASUB > 1 && staged)
+        for (int i = 0; i < SR::LEAD && sc_g < my_stages; i++) issue_scales();
       for (int64_t ti = 0; ti < my_tiles && ok; ti++) {
         const int64_t tile = seg_tile(ti);
         const unsigned char* src = g.w_prep + (tile % tiles_n) * n_stages * S::B_STAGE;
@@ -309,9 +413,17 @@ hbmm_fold_kernel(const Args g) {
           if (gst >= STAGES && !mbar_wait(&empty[s], static_cast<uint32_t>(((gst / STAGES) & 1) ^ 1), abort_flag, 6)) { ok = false; break; }
           mbar_arrive_expect_tx(&full[s], S::B_STAGE);
           bulk_copy_g2s(smem + S::OFF_B + s * S::B_STAGE, src + st * S::B_STAGE, S::B_STAGE, &full[s]);
+          if (ASUB > 1 && staged && sc_g < my_stages) issue_scales();      // the block of stage gst + LEAD
         }
       }
       if (!ok || *abort_flag) {
+        if (ASUB > 1 && staged) {
+          const int64_t pend = sc_g < SR::NS ? sc_g : SR::NS;
+          for (int64_t q = 1; q <= pend; q++) {
+            const int64_t idx = sc_g - q;
+            mbar_wait_quiet(&sfull[idx % SR::NS], static_cast<uint32_t>((idx / SR::NS) & 1), kDrainPolls);
+          }
+        }
         // aborted: the copies already issued (at most one per stage) must land before the CTA's shared memory
         // goes away.  Their barriers also count producer arrivals that may never come, so each wait is a
         // short bounded one that ignores the abort flag: it ends when the phase completes or after a time
@@ -570,6 +682,7 @@ Args make_args(const PackedView& A, const PackedView& W, float* C, int64_t ldc) 
   g.w_down = nullptr;
   g.ep = plain_epilogue();
   g.sk_units = 0; g.sk_counters = nullptr; g.sk_counter_count = 0; g.sk_partials = nullptr;
+  g.a_staged = 0; g.a_rowmax = nullptr;
   return g;
 }
 
@@ -606,8 +719,13 @@ template <int TN>
 size_t balanced_offset(const Args& g) {
   return (stage_bytes<TN>(g) + static_cast<size_t>((g.N + TN - 1) / TN) * TN * sizeof(float) + 255) / 256 * 256;
 }
+// ... then, for activation groups shorter than a word, one float per activation row (its largest scale)
 template <int TN>
-size_t prep_bytes(const Args& g) { return balanced_offset<TN>(g) + balanced_bytes<TN>(g); }
+size_t rowmax_offset(const Args& g) { return (balanced_offset<TN>(g) + balanced_bytes<TN>(g) + 255) / 256 * 256; }
+template <int TN>
+size_t prep_bytes(const Args& g) {
+  return g.a_sub > 1 ? rowmax_offset<TN>(g) + static_cast<size_t>(g.M) * sizeof(float) : balanced_offset<TN>(g) + balanced_bytes<TN>(g);
+}
 // Points the argument block at the balanced schedule's part of the workspace (when the shape has one).
 template <int TN>
 void set_balanced_area(Args& g, void* workspace) {
@@ -622,14 +740,16 @@ template <int TN, int ASUB, bool FUSE = false>
 cudaError_t launch_fold(Args g, void* workspace, cudaStream_t stream, bool w_prepared) {
   using S = Smem<TN>;
   constexpr bool kHasBalanced = ASUB == 1;           // the balanced schedule is built for activation groups of whole words
+  constexpr int kBytes = ScaleRing<TN, ASUB>::BYTES;
+  static_assert(kBytes <= 227 * 1024, "weight stages and the scale ring fit one CTA's shared memory");
   static DeviceOnce configured;
   int dev = 0, sms = 0;
   if (current_device(&dev, &sms) != cudaSuccess) return cudaErrorInvalidDevice;
   if (configured.pending(dev)) {
-    cudaError_t e = cudaFuncSetAttribute(hbmm_fold_kernel<TN, ASUB, FUSE, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::BYTES);
+    cudaError_t e = cudaFuncSetAttribute(hbmm_fold_kernel<TN, ASUB, FUSE, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kBytes);
     if (e != cudaSuccess) return e;
     if (kHasBalanced) {
-      e = cudaFuncSetAttribute(hbmm_fold_kernel<TN, ASUB, FUSE, kHasBalanced>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::BYTES);
+      e = cudaFuncSetAttribute(hbmm_fold_kernel<TN, ASUB, FUSE, kHasBalanced>, cudaFuncAttributeMaxDynamicSharedMemorySize, kBytes);
       if (e != cudaSuccess) return e;
     }
     configured.mark(dev);
@@ -644,6 +764,32 @@ cudaError_t launch_fold(Args g, void* workspace, cudaStream_t stream, bool w_pre
   }
   g.w_prep = stages;
   g.w_down = down;
+  // sub-word groups: the activation scales as a 2-D tensor [M][lda_s] of fp32 for the per-stage block copies
+  CUtensorMap s_map = {};
+  g.a_staged = 0;
+  if (ASUB >= kStagedFrom && !g.a_bf16 && reinterpret_cast<uintptr_t>(g.a_scales) % 16 == 0 && g.lda_s % 4 == 0 &&
+      g.lda_s < (int64_t{1} << 31) && g.M < (int64_t{1} << 31)) {
+    if (EncodeTiledFn fn = encode_tiled_fn()) {
+      const cuuint64_t dims[2] = {static_cast<cuuint64_t>(g.lda_s), static_cast<cuuint64_t>(g.M)};
+      const cuuint64_t strides[1] = {static_cast<cuuint64_t>(g.lda_s) * 4};
+      const cuuint32_t box[2] = {2 * ASUB, TM};
+      const cuuint32_t elem[2] = {1, 1};
+      const CUtensorMapSwizzle swz_mode = ASUB == 16 ? CU_TENSOR_MAP_SWIZZLE_128B : (ASUB == 8 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                          : (ASUB == 4 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE));
+      if (fn(&s_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(g.a_scales), dims, strides, box, elem,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, swz_mode, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS)
+        g.a_staged = 1;
+    }
+  }
+  g.a_rowmax = nullptr;
+  if (ASUB > 1 && !g.a_bf16 && g.lda_s % 4 == 0 && g.lda_s >= kRowMaxFrom && reinterpret_cast<uintptr_t>(g.a_scales) % 16 == 0) {
+    // many scales per row: reduce the rows to their largest scale in a kernel of its own, at streaming bandwidth
+    g.a_rowmax = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + rowmax_offset<TN>(g));
+    const cudaError_t e = launch_pdl(row_max_kernel, dim3(static_cast<unsigned>((g.M + 7) / 8)), dim3(256), 0, stream,
+                                     reinterpret_cast<const float*>(g.a_scales), g.lda_s, g.M, g.a_rowmax);
+    if (e != cudaSuccess) return e;
+  }
   const int64_t tiles = ((g.M + TM - 1) / TM) * tiles_n;
   // equal runs of (tile, stage) pairs, one per CTA, when that shortens the longest CTA's walk by a tenth or more
   const int64_t units = tiles * n_stages;
@@ -654,10 +800,10 @@ cudaError_t launch_fold(Args g, void* workspace, cudaStream_t stream, bool w_pre
   if (kHasBalanced && balanced_possible<TN>(g, sms) && run * 10 <= plain_walk * 9) {
     ctas = (units + run - 1) / run;                     // no CTA without work
     g.sk_units = run;
-    return launch_pdl(hbmm_fold_kernel<TN, ASUB, FUSE, kHasBalanced>, dim3(static_cast<unsigned>(ctas)), dim3(kThreads), S::BYTES, stream, g);
+    return launch_pdl(hbmm_fold_kernel<TN, ASUB, FUSE, kHasBalanced>, dim3(static_cast<unsigned>(ctas)), dim3(kThreads), kBytes, stream, g, s_map);
   }
   const unsigned grid = static_cast<unsigned>(tiles < sms ? tiles : sms);   // one persistent CTA per SM
-  return launch_pdl(hbmm_fold_kernel<TN, ASUB, FUSE, false>, dim3(grid), dim3(kThreads), S::BYTES, stream, g);
+  return launch_pdl(hbmm_fold_kernel<TN, ASUB, FUSE, false>, dim3(grid), dim3(kThreads), kBytes, stream, g, s_map);
 }
 
 template <int TN>

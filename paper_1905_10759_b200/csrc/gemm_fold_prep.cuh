@@ -105,8 +105,20 @@ __device__ __forceinline__ void row_max_scale2(const void* s, int bf16, int64_t 
   } else {
     const uint4* pa = reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(s) + off_a);
     const uint4* pb = reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(s) + off_b);
-#pragma unroll 2
-    for (int64_t i = 0; i < ld / 4; i++) {
+    // eight 16-byte loads of each row in flight: rows of a few hundred scales are scanned at a rate set by how much
+    // is in flight, and the scouts have little else in registers
+    int64_t i = 0;
+    for (; i + 8 <= ld / 4; i += 8) {
+      uint4 va[8], vb[8];
+#pragma unroll
+      for (int u = 0; u < 8; u++) { va[u] = __ldg(pa + i + u); vb[u] = __ldg(pb + i + u); }
+#pragma unroll
+      for (int u = 0; u < 8; u++) {
+        ma = max(max(ma, va[u].x), max(va[u].y, max(va[u].z, va[u].w)));
+        mb = max(max(mb, vb[u].x), max(vb[u].y, max(vb[u].z, vb[u].w)));
+      }
+    }
+    for (; i < ld / 4; i++) {
       const uint4 va = __ldg(pa + i), vb = __ldg(pb + i);
       ma = max(max(ma, va.x), max(va.y, max(va.z, va.w)));
       mb = max(max(mb, vb.x), max(vb.y, max(vb.z, vb.w)));

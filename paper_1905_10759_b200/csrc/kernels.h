@@ -131,6 +131,8 @@ struct FoldArgs {
   int32_t* sk_counters;          // [tiles][4]: zeroed by the weight expansion, left at zero by every launch
   int64_t sk_counter_count;
   float* sk_partials;            // [2 * CTAs][128][TN]
+  float* a_rowmax;               // sub-word groups: largest scale of every activation row (nullptr: the scouts scan the rows)
+  int32_t a_staged;              // sub-word groups: the activation scales of a stage reach the producers through shared memory
 };
 // The weight expansion as a job another kernel can run: n_stages x tiles_n tasks of tn threads each
 // (n_stages counts tasks per column tile: single stages of the e4m3 layout, runs of stages of the folded one).

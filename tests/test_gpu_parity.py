@@ -169,6 +169,12 @@ GEMM_CASES = [
     (33, 40, 100, 4, 8, 0),          # K no multiple of 32: integer-pipe path only
     (50, 60, 320, 320, 16, 0),       # one group per row against beta 16
     (300, 130, 640, 32, 8, 0),       # finer weight groups
+    # sub-word activation groups whose scales reach the producers through shared memory (beta_a <= 8), several tiles,
+    # ragged rows; 512 or more scales per row: the rows' largest scales come from a kernel of their own
+    (300, 130, 1152, 8, 8, 0),
+    (260, 72, 2048, 2, 16, 0),       # 1024 scales per row
+    (150, 200, 4608, 8, 32, 0),      # 576 scales per row, tail stage of one word... K = 144 words
+    (140, 64, 1056, 4, 4, 0),        # odd number of words: the last stage holds one word
 ]
 
 
