@@ -496,7 +496,7 @@ hbmm_status conv_checked(const void* x, int32_t x_dtype, const hbmm_conv_geom* g
       UmmaPrepJob job{};
       gemm_fold_prep_job(av, wv, gemm_ws, &job);
       if (job.n_stages * job.tiles_n <= 4096) {
-        if (launch_im2col_quantize_tma(x, cg, A.bits, A.ld_words, A.scales, A.ld_scales, a_scale_dtype == HBMM_BF16, s,
+        if (launch_im2col_quantize_tma(x, cg, beta_a, A.bits, A.ld_words, A.scales, A.ld_scales, a_scale_dtype == HBMM_BF16, s,
                                        w_prepared ? nullptr : &job) != cudaSuccess)
           return HBMM_ERR_CUDA;
         if (pack_only) return HBMM_OK;

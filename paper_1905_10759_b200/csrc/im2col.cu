@@ -379,7 +379,7 @@ cudaError_t launch_im2col_quantize(const void* x, int x_bf16, const ConvGeom& g,
   const int64_t beta_eff = beta >= K ? K : beta;
   const int64_t G = num_groups(K, beta);
   if (im2col_quantize_tma_supported(x, x_bf16, g, beta))
-    return launch_im2col_quantize_tma(x, g, bits, ld_words, scales, ld_scales, scale_bf16, stream);
+    return launch_im2col_quantize_tma(x, g, beta, bits, ld_words, scales, ld_scales, scale_bf16, stream);
   if (beta == 32 && beta < K && g.sw == 1) {
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);

@@ -1,5 +1,5 @@
-// Packed convolution front end (beta = 32, fp32 NCHW input) with the input tile staged by tensor
-// copies.  A work item is RB output rows of one image and a range of 32-channel chunks.  For every
+// Packed convolution front end (fp32 NCHW input; groups of 2, 4, 8, 16 elements or of whole K-words) with the
+// input tile staged by tensor copies.  A work item is RB output rows of one image and a range of 32-channel chunks.  For every
 // chunk one 4-D tensor copy brings [32 channels][rows_in input rows][pitch columns] into shared
 // memory, zero halo included (the copy starts left of and above the image where the padding asks
 // for it, and whatever lies outside the tensor arrives as zeros).  Two persistent CTAs per SM: a
@@ -35,7 +35,43 @@ struct Plan {
   int ring;               // tile buffers per CTA
   int flat;               // 1: whole channel planes staged by one bulk copy per chunk, no halo (pitch = W, rows_in = H)
   int tile_stride;        // floats between ring buffers (tile rounded up to 128 bytes)
+  int sub;                // scale groups per K-word (beta = 32 / sub), 1 for groups of whole words
+  int gw;                 // K-words per scale group (beta = 32 * gw), 1 for groups of at most a word
+  int vec_scales;         // sub > 1: a word's fp32 scales may leave as 16-byte (8-byte for sub = 2) stores
 };
+
+// One K-word of a full 32-channel chunk whose groups are shorter than a word: the packed word, and the word's SUB
+// group means stored straight to the operand's scale row (`dst`: the word's first scale).
+template <int SUB>
+__device__ __forceinline__ void gather_word_sub(int taps, bool flat, int w, uint32_t addr, uint32_t cs_bytes, uint32_t pitch_bytes,
+                                                uint32_t pm, uint32_t& word, void* scales, int scale_bf16, int64_t idx, bool vec) {
+  float sums[SUB];
+  if (taps == 9) {
+    if (flat) gather_word_dispatch_sub<3, 3, true, SUB>(w, addr, cs_bytes, pitch_bytes, pm, word, sums);
+    else gather_word_dispatch_sub<3, 3, false, SUB>(w, addr, cs_bytes, pitch_bytes, 0u, word, sums);
+  } else {
+    if (flat) gather_word_dispatch_sub<1, 1, true, SUB>(w, addr, cs_bytes, pitch_bytes, pm, word, sums);
+    else gather_word_dispatch_sub<1, 1, false, SUB>(w, addr, cs_bytes, pitch_bytes, 0u, word, sums);
+  }
+  constexpr float inv = static_cast<float>(SUB) / 32.0f;          // 1 / beta
+#pragma unroll
+  for (int i = 0; i < SUB; i++) sums[i] *= inv;
+  if (vec) {
+    float* d = reinterpret_cast<float*>(scales) + idx;
+    if constexpr (SUB == 2) {
+      *reinterpret_cast<float2*>(d) = make_float2(sums[0], sums[1]);
+    } else {
+#pragma unroll
+      for (int i = 0; i < SUB; i += 4) *reinterpret_cast<float4*>(d + i) = make_float4(sums[i], sums[i + 1], sums[i + 2], sums[i + 3]);
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < SUB; i++) {
+      if (scale_bf16) reinterpret_cast<__nv_bfloat16*>(scales)[idx + i] = __float2bfloat16_rn(sums[i]);
+      else reinterpret_cast<float*>(scales)[idx + i] = sums[i];
+    }
+  }
+}
 
 __device__ __forceinline__ void store_scale(void* scales, int bf16, int64_t idx, float v) {
   if (bf16) reinterpret_cast<__nv_bfloat16*>(scales)[idx] = __float2bfloat16_rn(v);
@@ -63,6 +99,9 @@ __device__ __forceinline__ ItemCoords item_coords(int item, const Plan& tp) {
   return c;
 }
 
+// GROUPS: 0 -- groups of exactly one K-word; 1 -- groups shorter than a word; 2 -- groups of several words.  The three are
+// separate instantiations so that the one-word kernel carries none of the others' code or registers.
+template <int GROUPS>
 __global__ void __launch_bounds__(kThreadsTma, 2)
 im2col_quantize_tma_kernel(const __grid_constant__ CUtensorMap x_map, const float* __restrict__ x, const ConvGeom g, const Plan tp,
                            const __grid_constant__ UmmaPrepJob prep, int n_prep, int n_items, int ring,
@@ -206,17 +245,45 @@ im2col_quantize_tma_kernel(const __grid_constant__ CUtensorMap x_map, const floa
           const int po = pixoff[pix];                          // tile offset of the pixel's first tap, in elements
           const uint32_t pm = pixmask[pix];
           uint32_t word = 0;
-          float mean;
-          if (cc == kCC && g.kh == 3 && g.kw == 3) {
+          float mean = 0.0f;
+          const int word_abs = static_cast<int>(static_cast<int64_t>(ic.chunk_first) * kCC * taps / 32) + words_done + w;
+          const int64_t m_pix = (static_cast<int64_t>(ic.b) * g.Ho + ic.yo0) * g.Wo + pix;
+          if (GROUPS == 1 && cc == kCC && (taps == 9 ? (g.kh == 3 && g.kw == 3) : taps == 1)) {
+            // groups shorter than a word: the word's means go straight to the scale row
+            const int64_t sidx = m_pix * ld_scales + static_cast<int64_t>(word_abs) * tp.sub;
+            const uint32_t a = t_addr + po * 4;
+            const bool vec = tp.vec_scales != 0;
+            switch (tp.sub) {
+              case 2: gather_word_sub<2>(taps, tp.flat != 0, w, a, cs * 4, tp.pitch * 4, pm, word, scales, scale_bf16, sidx, vec); break;
+              case 4: gather_word_sub<4>(taps, tp.flat != 0, w, a, cs * 4, tp.pitch * 4, pm, word, scales, scale_bf16, sidx, vec); break;
+              case 8: gather_word_sub<8>(taps, tp.flat != 0, w, a, cs * 4, tp.pitch * 4, pm, word, scales, scale_bf16, sidx, vec); break;
+              default: gather_word_sub<16>(taps, tp.flat != 0, w, a, cs * 4, tp.pitch * 4, pm, word, scales, scale_bf16, sidx, vec); break;
+            }
+          } else if (GROUPS == 1) {
+            // any filter size, short last chunk: group by group (the last group of the row may be short)
+            const float* base = t + po;
+            const unsigned short* o = off + k_begin;
+            const int beta = 32 / tp.sub;
+            for (int e0 = 0; e0 < nk; e0 += beta) {
+              const int cnt = (nk - e0 < beta) ? nk - e0 : beta;
+              float sum = 0.0f;
+              for (int e = e0; e < e0 + cnt; e++) {
+                const float v = base[o[e]];
+                word |= (v >= 0.0f ? 1u : 0u) << e;
+                sum += fabsf(v);
+              }
+              store_scale(scales, scale_bf16, m_pix * ld_scales + static_cast<int64_t>(word_abs) * tp.sub + e0 / beta, sum / static_cast<float>(cnt));
+            }
+          } else if (cc == kCC && g.kh == 3 && g.kw == 3) {
             float sum;
             if (tp.flat) gather_word_dispatch<3, 3, true>(w, t_addr + po * 4, cs * 4, tp.pitch * 4, pm, word, sum);
             else gather_word_dispatch<3, 3, false>(w, t_addr + po * 4, cs * 4, tp.pitch * 4, 0u, word, sum);
-            mean = sum * 0.03125f;
+            mean = GROUPS == 2 ? sum : sum * 0.03125f;
           } else if (cc == kCC && taps == 1) {
             float sum;
             if (tp.flat) gather_word_dispatch<1, 1, true>(w, t_addr + po * 4, cs * 4, tp.pitch * 4, pm, word, sum);
             else gather_word_dispatch<1, 1, false>(w, t_addr + po * 4, cs * 4, tp.pitch * 4, 0u, word, sum);
-            mean = sum * 0.03125f;
+            mean = GROUPS == 2 ? sum : sum * 0.03125f;
           } else {
             const float* base = t + po;
             const unsigned short* o = off + k_begin;
@@ -236,9 +303,10 @@ im2col_quantize_tma_kernel(const __grid_constant__ CUtensorMap x_map, const floa
               s0 += fabsf(v);
             }
             mean = ((s0 + s1) + (s2 + s3)) / static_cast<float>(nk);
+            if (GROUPS == 2) mean = (s0 + s1) + (s2 + s3);
           }
           out_bits[pix * ldo + words_done + w] = word;
-          out_scale[pix * ldo + words_done + w] = mean;
+          out_scale[pix * ldo + words_done + w] = mean;          // gw > 1: the word's sum of |x| (see the two fast branches)
         }
         pw += dpw; w += dw;
         if (pw >= pix_warps) { pw -= pix_warps; w++; }
@@ -275,7 +343,38 @@ im2col_quantize_tma_kernel(const __grid_constant__ CUtensorMap x_map, const floa
         bits[(m_base + pix) * ld_words + word0 + w] = (w < words_done) ? out_bits[pix * ldo + w] : 0u;
       }
     }
-    if (!scale_bf16 && (word0 & 3) == 0 && (run_scale & 3) == 0) {
+    if (GROUPS == 1) {
+      // the means were stored by the gather; the last channel range zeroes the row's padding
+      if (wrote_last) {
+        const int64_t K = static_cast<int64_t>(g.C) * taps;
+        const int beta = 32 / tp.sub;
+        const int64_t G = (K + beta - 1) / beta;
+        const int pad = static_cast<int>(ld_scales - G);
+        for (int idx = tid; idx < pixels * pad; idx += nthr) {
+          const int pix = idx / pad, q = idx - pix * pad;
+          store_scale(scales, scale_bf16, (m_base + pix) * ld_scales + G + q, 0.0f);
+        }
+      }
+    } else if (GROUPS == 2) {
+      // groups of gw words: add the words' sums (word0 is a multiple of gw, and so is the item's word count unless
+      // it ends the row); the row's last group may be short
+      const int64_t K = static_cast<int64_t>(g.C) * taps;
+      const int64_t beta = 32LL * tp.gw;
+      const int64_t group0 = word0 / tp.gw;
+      const int n_groups = (words_done + tp.gw - 1) / tp.gw;
+      const int run = wrote_last ? static_cast<int>(ld_scales - group0) : n_groups;
+      for (int idx = tid; idx < pixels * run; idx += nthr) {
+        const int pix = idx / run, q = idx - pix * run;
+        float v = 0.0f;
+        if (q < n_groups) {
+          const int w_end = ((q + 1) * tp.gw < words_done) ? (q + 1) * tp.gw : words_done;
+          for (int w = q * tp.gw; w < w_end; w++) v += out_scale[pix * ldo + w];
+          const int64_t left = K - (group0 + q) * beta;
+          v /= static_cast<float>(left < beta ? left : beta);
+        }
+        store_scale(scales, scale_bf16, (m_base + pix) * ld_scales + group0 + q, v);
+      }
+    } else if (!scale_bf16 && (word0 & 3) == 0 && (run_scale & 3) == 0) {
       const int q_per = run_scale >> 2;
       float* sc = reinterpret_cast<float*>(scales);
       for (int idx = tid; idx < pixels * q_per; idx += nthr) {
@@ -302,9 +401,12 @@ im2col_quantize_tma_kernel(const __grid_constant__ CUtensorMap x_map, const floa
 
 inline int round_up4(int v) { return (v + 3) / 4 * 4; }
 
-bool make_plan(const ConvGeom& g, int sms, bool flat, Plan* out, size_t* smem_bytes) {
+bool make_plan(const ConvGeom& g, int sms, bool flat, int32_t beta, Plan* out, size_t* smem_bytes) {
   Plan p;
   p.flat = flat ? 1 : 0;
+  p.sub = beta < 32 ? 32 / beta : 1;
+  p.gw = beta > 32 ? beta / 32 : 1;
+  p.vec_scales = 0;
   if (flat) {
     p.RB = g.Ho;                                               // an item covers the whole image
     p.rows_in = g.H;
@@ -324,9 +426,14 @@ bool make_plan(const ConvGeom& g, int sms, bool flat, Plan* out, size_t* smem_by
   const int64_t row_blocks = static_cast<int64_t>(g.B) * p.yo_blocks;
   int splits = 1;
   while (row_blocks * splits < 2LL * sms && splits * 2 <= p.n_chunks) splits *= 2;
-  p.chunks_per_split = (p.n_chunks + splits - 1) / splits;
-  p.splits = (p.n_chunks + p.chunks_per_split - 1) / p.chunks_per_split;
   const int taps = g.kh * g.kw;
+  p.chunks_per_split = (p.n_chunks + splits - 1) / splits;
+  // groups of several words must not straddle two channel ranges
+  while (splits > 1 && (p.chunks_per_split * taps) % p.gw != 0) {
+    splits /= 2;
+    p.chunks_per_split = (p.n_chunks + splits - 1) / splits;
+  }
+  p.splits = (p.n_chunks + p.chunks_per_split - 1) / p.chunks_per_split;
   const int64_t tile_elems = static_cast<int64_t>(kCC) * p.rows_in * p.pitch;
   p.tile_stride = static_cast<int>((tile_elems + 31) / 32 * 32);
   const int64_t max_pixels = static_cast<int64_t>(p.RB) * g.Wo;
@@ -346,35 +453,37 @@ bool make_plan(const ConvGeom& g, int sms, bool flat, Plan* out, size_t* smem_by
 // 0: not supported, 1: tensor-copy tiles with halo, 2: flat channel planes
 int tma_mode(const void* x, int x_bf16, const ConvGeom& g, int32_t beta) {
   const int64_t K = static_cast<int64_t>(g.C) * g.kh * g.kw;
-  if (x_bf16 || beta != 32 || beta >= K || g.sw != 1 || reinterpret_cast<uintptr_t>(x) % 16 != 0) return 0;
+  const bool beta_ok = beta == 2 || beta == 4 || beta == 8 || beta == 16 || (beta >= 32 && beta % 32 == 0 && beta / 32 <= 64);
+  if (x_bf16 || !beta_ok || beta >= K || g.sw != 1 || reinterpret_cast<uintptr_t>(x) % 16 != 0) return 0;
   Plan p;
   size_t smem;
   int dev = 0, sms = 0;
   if (current_device(&dev, &sms) != cudaSuccess) return 0;       // the plan's channel split follows the device's SM count
-  if (g.W % 4 == 0 && encode_tiled_fn() != nullptr && make_plan(g, sms, false, &p, &smem)) return 1;
+  if (g.W % 4 == 0 && encode_tiled_fn() != nullptr && make_plan(g, sms, false, beta, &p, &smem)) return 1;
   // small images whose rows are not multiples of 16 bytes: whole planes, masked 3x3 / 1x1 gather
   const bool filt = (g.kh == 3 && g.kw == 3) || (g.kh == 1 && g.kw == 1);
-  if (filt && g.C % kCC == 0 && (static_cast<int64_t>(g.C) * g.H * g.W) % 4 == 0 && make_plan(g, sms, true, &p, &smem)) return 2;
+  if (filt && g.C % kCC == 0 && (static_cast<int64_t>(g.C) * g.H * g.W) % 4 == 0 && make_plan(g, sms, true, beta, &p, &smem)) return 2;
   return 0;
 }
 
 }  // namespace
 
-// fp32 input, stride 1 along x, groups of exactly one K-word; rows that are multiples of 16 bytes (a
+// fp32 input, stride 1 along x, groups of 2, 4, 8, 16 elements or of whole K-words (fewer than the row has); rows that are multiples of 16 bytes (a
 // tensor map wants 16-byte strides), or small images with 3x3 / 1x1 filters and whole 32-channel chunks.
 bool im2col_quantize_tma_supported(const void* x, int x_bf16, const ConvGeom& g, int32_t beta) {
   return tma_mode(x, x_bf16, g, beta) != 0;
 }
 
-cudaError_t launch_im2col_quantize_tma(const void* x, const ConvGeom& g, uint32_t* bits, int64_t ld_words, void* scales,
+cudaError_t launch_im2col_quantize_tma(const void* x, const ConvGeom& g, int32_t beta, uint32_t* bits, int64_t ld_words, void* scales,
                                        int64_t ld_scales, int scale_bf16, cudaStream_t stream, const UmmaPrepJob* prep) {
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const int mode = tma_mode(x, 0, g, 32);
+  const int mode = tma_mode(x, 0, g, beta);
   Plan p;
   size_t smem;
-  if (mode == 0 || !make_plan(g, sms, mode == 2, &p, &smem)) return cudaErrorNotSupported;
+  if (mode == 0 || !make_plan(g, sms, mode == 2, beta, &p, &smem)) return cudaErrorNotSupported;
+  p.vec_scales = (p.sub > 1 && !scale_bf16 && reinterpret_cast<uintptr_t>(scales) % 16 == 0 && ld_scales % 4 == 0) ? 1 : 0;
   CUtensorMap map{};
   if (mode == 1) {
     const cuuint64_t dims[4] = {static_cast<cuuint64_t>(g.W), static_cast<cuuint64_t>(g.H), static_cast<cuuint64_t>(g.C),
@@ -390,7 +499,9 @@ cudaError_t launch_im2col_quantize_tma(const void* x, const ConvGeom& g, uint32_
   }
   static DeviceOnce configured;
   if (configured.pending(dev)) {
-    cudaError_t e = cudaFuncSetAttribute(im2col_quantize_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 104 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(im2col_quantize_tma_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 104 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(im2col_quantize_tma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 104 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(im2col_quantize_tma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 104 * 1024);
     if (e != cudaSuccess) return e;
     configured.mark(dev);
   }
@@ -404,7 +515,8 @@ cudaError_t launch_im2col_quantize_tma(const void* x, const ConvGeom& g, uint32_
     n_prep = job.n_stages * job.tiles_n;
     if (n_prep > 4096) return cudaErrorNotSupported;       // the caller expands large weight operands on its own
   }
-  return launch_pdl(im2col_quantize_tma_kernel, dim3(grid + n_prep), dim3(kThreadsTma), smem, stream, map, static_cast<const float*>(x), g, p,
+  auto kernel = p.sub > 1 ? im2col_quantize_tma_kernel<1> : (p.gw > 1 ? im2col_quantize_tma_kernel<2> : im2col_quantize_tma_kernel<0>);
+  return launch_pdl(kernel, dim3(grid + n_prep), dim3(kThreadsTma), smem, stream, map, static_cast<const float*>(x), g, p,
                     job, n_prep, static_cast<int>(n_items), p.ring, bits, ld_words, scales, ld_scales, scale_bf16);
 }
 

@@ -208,7 +208,7 @@ cudaError_t launch_im2col_quantize(const void* x, int x_bf16, const ConvGeom& g,
 // The packed front end with its input tile staged by tensor copies (fp32 input, beta = 32).
 bool im2col_quantize_tma_supported(const void* x, int x_bf16, const ConvGeom& g, int32_t beta);
 // prep (optional): weight-expansion tasks of the contraction that follows, run by extra CTAs of the launch.
-cudaError_t launch_im2col_quantize_tma(const void* x, const ConvGeom& g, uint32_t* bits, int64_t ld_words, void* scales,
+cudaError_t launch_im2col_quantize_tma(const void* x, const ConvGeom& g, int32_t beta, uint32_t* bits, int64_t ld_words, void* scales,
                                        int64_t ld_scales, int scale_bf16, cudaStream_t stream, const UmmaPrepJob* prep = nullptr);
 cudaError_t im2col_tma_health(int op, int* value);
 // Register-only arithmetic loop for measuring a unit's issue rate (kind 0: XOR + POPC, 1: fp32 add, 2: fp32

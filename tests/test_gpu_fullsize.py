@@ -65,6 +65,42 @@ def test_resnet_conv_hbmm_full_batch(hb, li, signed):
         gu.assert_close_rel_absref(C[lo: lo + per_image].cpu().numpy(), c_ref, absref, RTOL, "%s image %d" % (s.name, b))
 
 
+@pytest.mark.parametrize("li,ba,bw", [(0, 4, 4), (1, 2, 16), (2, 16, 16), (3, 64, 64), (1, 128, 32)])
+def test_resnet_conv_hbmm_full_batch_at_other_group_sizes(hb, li, ba, bw):
+    """The paper's own group sizes (Section 5: beta_a / beta_w of 2 .. 16) and groups of several words through the
+    convolution entry at batch 64: packed activations bit for bit, their scales to the quantizer's bound, the product
+    to 1e-5 R, on whole images."""
+    gu = _gu()
+    s = inputs.resnet18_convs(64)[li]
+    x = inputs.conv_activation(s, inputs.SEEDS["resnet_hbmm"][0] + 70 + li, signed=True)
+    w = inputs.he_normal(s.N, s.K, inputs.SEEDS["resnet_hbmm"][1] + 70 + li)
+    Wop = hb.quantize(torch.from_numpy(w).cuda(), hb.alloc_operand(s.N, s.K, bw, hb.F32))
+    geom = hb.make_geom(s.B, s.C, s.H, s.W, s.kh, s.kw, (s.stride, s.stride), (s.pad, s.pad))
+    ws = torch.empty(hb.conv_workspace_bytes(geom, ba, hb.F32, Wop), dtype=torch.uint8, device="cuda")
+    C = torch.empty((s.M, s.N), device="cuda")
+    hb.conv_im2col(torch.from_numpy(x).cuda(), geom, ba, hb.F32, Wop, C, ws)
+    torch.cuda.synchronize()
+    assert hb.last_device_error() == 0
+    _, _, lw, ls = hb.operand_bytes(s.M, s.K, ba, hb.F32)
+    bits_bytes = (s.M * lw * 4 + 255) // 256 * 256          # the scales follow the packed words on a 256-byte boundary
+    bits = ws[: s.M * lw * 4].view(torch.int32).reshape(s.M, lw)
+    scales = ws[bits_bytes: bits_bytes + s.M * ls * 4].view(torch.float32).reshape(s.M, ls)
+    G = oracle.n_groups(s.K, ba)
+    per_image = s.M // s.B
+    dw, sw = oracle.quantize(w, bw)
+    for b in (0, s.B - 1):
+        rows = oracle.im2col(x[b:b + 1], s.kh, s.kw, (s.stride, s.stride), (s.pad, s.pad))
+        da, sa = oracle.quantize(rows, ba)
+        lo = b * per_image
+        assert np.array_equal(gu.host_bits(bits[lo: lo + per_image]), oracle.pack(sa, lw)), "packed activations of image %d" % b
+        sg = scales[lo: lo + per_image].cpu().numpy().astype(np.float64)
+        assert np.all(sg[:, G:] == 0.0)
+        assert np.all(np.abs(sg[:, :G] - da) <= 12 * gu.U * da + 1e-30)
+        c_ref, absref = oracle.hbmm_from_quantized(sg[:, :G], sa, ba, oracle.round_scales(dw, "f32"), sw, bw)
+        fine = gu.elementwise_magnitude(sg[:, :G], ba, dw, bw, s.K)
+        gu.assert_close_rel_absref(C[lo: lo + per_image].cpu().numpy(), c_ref, absref, RTOL, "%s image %d beta %d/%d" % (s.name, b, ba, bw), fine)
+
+
 @pytest.mark.parametrize("li", [0, 1, 2, 3])
 def test_resnet_conv_hbwn_full_batch(hb, li):
     gu = _gu()

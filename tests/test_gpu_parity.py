@@ -351,6 +351,17 @@ CONV_CASES = [
     (3, 96, 14, 14, 40, 3, 3, 1, 1, 32, 32, True, False),
     (2, 32, 9, 10, 16, 1, 1, 1, 0, 32, 32, True, False),
     (2, 64, 7, 7, 24, 3, 3, 1, 0, 32, 32, None, False),     # no padding, zeros of both signs
+    # the same front end with groups shorter than a word (means stored from the gather) and of several words (sums of
+    # the words' sums), tiles with halo and whole planes, full and short last chunks, channel ranges
+    (2, 96, 20, 20, 40, 3, 3, 1, 1, 4, 4, True, False),
+    (2, 96, 20, 20, 40, 3, 3, 1, 1, 64, 64, True, False),
+    (2, 128, 12, 12, 24, 3, 3, 1, 1, 128, 32, True, False),  # 1152 = 9 groups of 128
+    (3, 70, 16, 12, 33, 3, 3, 1, 0, 8, 32, True, False),     # last chunk of 6 channels, K = 630: last group of 6
+    (3, 70, 16, 12, 33, 3, 3, 1, 0, 128, 64, True, False),   # K = 630: last group of 118
+    (2, 40, 8, 8, 24, 5, 5, 1, 2, 16, 16, True, False),      # 5x5
+    (1, 64, 12, 12, 16, 1, 1, 1, 0, 8, 8, True, False),      # 1x1
+    (2, 64, 7, 7, 24, 3, 3, 1, 1, 2, 2, None, False),        # whole planes, zeros of both signs
+    (3, 96, 14, 14, 40, 3, 3, 1, 1, 96, 32, True, False),    # groups of three words
     # HBWN with whole 64-channel blocks: no im2col matrix, tiles fetched by im2col-mode tensor copies
     (3, 128, 7, 7, 72, 3, 3, 1, 1, 1, 32, True, False),     # two channel blocks, tiles span images, ragged M and N
     (2, 64, 9, 9, 40, 3, 3, 2, 0, 1, 32, True, True),       # stride 2, no padding
