@@ -444,7 +444,7 @@ def side_measurements(torch, hbmm, inputs, peaks, iters: int):
         by = (4.0 + ob) * amap.numel()
         out.append({"kernel": "hbmm_binarize_dense/beta8_%s" % name, "shape": list(amap.shape), "ms": round(ms, 5), "bound": "hbm",
                     "achieved": by / (ms * 1e-3) / 1e9, "peak": hbm_gbs, "unit": "GB/s", "frac": by / (ms * 1e-3) / 1e9 / hbm_gbs})
-    for ba, bw in ((16, 16), (4, 4), (2, 16)):
+    for ba, bw in ((16, 16), (8, 8), (4, 4), (2, 16)):
         A = hbmm.quantize(a, hbmm.alloc_operand(M, K, ba, hbmm.F32))
         W = hbmm.quantize(w, hbmm.alloc_operand(N, K, bw, hbmm.F32))
         ws = torch.empty(max(hbmm.gemm_workspace_bytes(A, W), 16), dtype=torch.uint8, device="cuda")
@@ -454,6 +454,22 @@ def side_measurements(torch, hbmm, inputs, peaks, iters: int):
         ach = 2.0 * M * N * K / (ms * 1e-3) / 1e12
         out.append({"kernel": "hbmm_fold_kernel/beta_a%d_beta_w%d" % (ba, bw), "shape": [M, N, K], "ms": round(ms, 5), "bound": "tensor",
                     "achieved": ach, "peak": bf16_tflops, "unit": "TFLOP/s", "frac": ach / bf16_tflops})
+    # the whole convolution call (packing front end + contraction) on conv3_x at the group sizes of the paper's experiments
+    # (Section 5: beta_a / beta_w = 16/16, 4/4, 2/16) and at 64/64, beside 32/32
+    sh3 = inputs.resnet18_convs(64)[1]
+    x3 = torch.randn((sh3.B, sh3.C, sh3.H, sh3.W), device="cuda", generator=g)
+    geomc = hbmm.make_geom(sh3.B, sh3.C, sh3.H, sh3.W, 3, 3, (1, 1), (1, 1))
+    c3 = torch.empty((sh3.M, sh3.N), device="cuda")
+    for ba, bw in ((32, 32), (64, 64), (16, 16), (4, 4), (2, 16)):
+        W3 = hbmm.quantize(w, hbmm.alloc_operand(N, K, bw, hbmm.F32))
+        ws3 = torch.empty(hbmm.conv_workspace_bytes(geomc, ba, hbmm.F32, W3), dtype=torch.uint8, device="cuda")
+        hbmm.conv_im2col(x3, geomc, ba, hbmm.F32, W3, c3, ws3)
+        ms = time_loop(torch, lambda: hbmm.conv_im2col(x3, geomc, ba, hbmm.F32, W3, c3, ws3, flags=hbmm.CONV_WEIGHTS_PREPARED), iters)
+        msp = time_loop(torch, lambda: hbmm.conv_im2col(x3, geomc, ba, hbmm.F32, W3, None, ws3,
+                                                        flags=hbmm.CONV_WEIGHTS_PREPARED | hbmm.CONV_PACK_ONLY), iters)
+        out.append({"kernel": "hbmm_conv_im2col/conv3_x/beta_a%d_beta_w%d" % (ba, bw), "shape": [M, N, K], "ms": round(ms, 5),
+                    "ms_front_end_alone": round(msp, 5), "tops": 2.0 * M * N * K / (ms * 1e-3) / 1e12})
+    del x3, c3
     # AlexNet-style fully connected layer at batch 256 (4096 -> 4096, beta 64): product + binarization of its
     # rows for the next layer, as two calls (fp32 product stored, then hbmm_quantize) and fused in the epilogue
     Mf, Kf, Nf, bf = 256, 4096, 4096, 64
@@ -565,10 +581,12 @@ def side_measurements(torch, hbmm, inputs, peaks, iters: int):
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
 # (same kernels, same workload); entries are dropped when a kernel changes after its capture.
 NCU_DRAM_BYTES = {
-    ("hbmm_contraction", "conv2_x"): 32.339e6 + 3.121e6,     # profiles/conv2_x_conv3_x_kernels.md
-    ("hbmm_contraction", "conv3_x"): 15.173e6 + 0.318e6,
-    ("hbwn_conv", "conv2_x"): 25.924e6 + 3.368e6,            # the contraction kernel of the call (the layout copy is a launch of its own)
-    ("front_end_pack", "conv2_x"): 51.502e6 + 2.750e6,
+    ("hbmm_contraction", "conv2_x"): 32.340e6 + 1.998e6,     # profiles/conv2_x_conv3_x_kernels.md
+    ("hbmm_contraction", "conv3_x"): 15.174e6 + 0.314e6,
+    ("hbwn_conv", "conv2_x"): 25.998e6 + 3.054e6,            # the contraction kernel of the call (the layout copy is a launch of its own)
+    ("hbwn_conv", "conv3_x"): 13.531e6 + 0.005e6,
+    ("front_end_pack", "conv2_x"): 51.502e6 + 2.789e6,
+    ("front_end_pack", "conv3_x"): 25.837e6,
 }
 
 
