@@ -612,8 +612,10 @@ def roofline_for(kind: str, li: int, shape, ms: float, peaks, rates):
 
     Both contractions run on the tensor cores (HBMM: two fp16 pieces per operand carrying sign and group
     scale; HBWN: bf16 activations x two bf16 weight pieces), so they are set against the measured dense
-    16-bit GEMM peak.  `achieved` counts the ALGORITHMIC operations 2 M N K; the HBMM kernel issues four
-    times that on the tensor pipe (2 x 2 pieces), the HBWN kernel twice.  Beside it: the fraction of the
+    16-bit GEMM peak.  `achieved` counts the ALGORITHMIC operations 2 M N K; the HBMM kernel issues three
+    times that on the tensor pipe (three cross products of the operands' pieces), the HBWN kernel twice:
+    `frac_of_peak_in_issued_tensor_work` is `frac` times that factor, i.e. how busy the tensor pipe is with
+    the work the formulation gives it.  Beside it: the fraction of the
     popcount / HBM roofline for HBMM (one population count per output and K-word at the MEASURED rate of the
     integer pipe, or the algorithmic bytes at the HBM copy bandwidth, whichever is slower) and of the fp32-add
     / HBM roofline for HBWN (one addition per output and K-element at the measured rate)."""
@@ -627,7 +629,7 @@ def roofline_for(kind: str, li: int, shape, ms: float, peaks, rates):
         return {"kernel": "hbmm_fold_kernel/%s" % shape.name, "bound": "tensor", "achieved": ach,
                 "peak": bf16_tflops, "unit": "TFLOP/s", "frac": ach / bf16_tflops, "traffic": None,
                 "peak_source": "%s bf16 GEMM peak (fp16 operands, same rate)" % hbm_src,
-                "tensor_pipe_work_factor": 4,
+                "tensor_pipe_work_factor": 3, "frac_of_peak_in_issued_tensor_work": 3 * ach / bf16_tflops,
                 "frac_of_popcount_hbm_roofline": rf["t_roof_us"] / (ms * 1e3),
                 "frac_of_popcount_hbm_roofline_at_max_clock": rf["t_roof_us_at_max_clock"] / (ms * 1e3),
                 "popcount_hbm_roofline": rf, "timing": "L2-cold (ring of buffer sets larger than L2), weights already expanded"}
@@ -637,9 +639,10 @@ def roofline_for(kind: str, li: int, shape, ms: float, peaks, rates):
         ach = ops / (ms * 1e-3) / 1e12
         by = 2.0 * shape.B * shape.C * shape.H * shape.W + N * K / 8.0 + 4.0 * N * G + 4.0 * M * N
         t_roof = max(by / (hbm_gbs * 1e9), M * N * float(K) / rates["fadd"]["ops_per_s"])
-        return {"kernel": "hbwn_umma_kernel(im2col tensor copies)/%s" % shape.name, "bound": "tensor", "achieved": ach,
+        return {"kernel": "hbwn tcgen05 kernels (layout copy + contraction)/%s" % shape.name, "bound": "tensor", "achieved": ach,
                 "peak": bf16_tflops, "unit": "TFLOP/s", "frac": ach / bf16_tflops, "traffic": None,
                 "peak_source": "%s bf16 GEMM peak" % hbm_src, "tensor_pipe_work_factor": 2,
+                "frac_of_peak_in_issued_tensor_work": 2 * ach / bf16_tflops,
                 "frac_of_fp32_add_hbm_roofline": t_roof / (ms * 1e-3), "timing": "L2-cold, whole call (layout copy + contraction)"}
     x_bytes = 4.0 * shape.B * shape.C * shape.H * shape.W
     lw = ((K + 31) // 32 + 3) // 4 * 4
@@ -1079,7 +1082,8 @@ def run_ours(args):
     roof["traffic"] = NCU_DRAM_BYTES.get((dominant, shapes[li].name))
     roof["share_of_step"] = totals[dominant] / sum(totals.values())
     kernels = {}
-    keep = ("bound", "achieved", "peak", "unit", "frac", "frac_of_popcount_hbm_roofline", "frac_of_popcount_hbm_roofline_at_max_clock",
+    keep = ("bound", "achieved", "peak", "unit", "frac", "frac_of_peak_in_issued_tensor_work", "frac_of_popcount_hbm_roofline",
+            "frac_of_popcount_hbm_roofline_at_max_clock",
             "frac_of_fp32_add_hbm_roofline", "timing")
     for kind in families + ("hbmm_conv_call",):
         kernels[kind] = [dict(layer=s.name, ms=round(t, 5), **{k: v for k, v in roofline_for(kind, i, s, t, peaks, rates).items() if k in keep})
