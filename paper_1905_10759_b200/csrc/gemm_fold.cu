@@ -696,6 +696,7 @@ size_t stage_bytes(const Args& g) {
 constexpr int64_t kMaxBalancedCtas = 256;
 constexpr int64_t kBalancedWaves = 4;
 constexpr int64_t kBalancedMinStages = 4;
+constexpr int64_t kBalancedMaxShare = 4;
 template <int TN>
 int64_t tile_count(const Args& g) { return ((g.M + TM - 1) / TM) * ((g.N + TN - 1) / TN); }
 template <int TN>
@@ -795,7 +796,11 @@ cudaError_t launch_fold(Args g, void* workspace, cudaStream_t stream, bool w_pre
   const int64_t units = tiles * n_stages;
   int64_t ctas = units / kBalancedMinStages < sms ? units / kBalancedMinStages : sms;
   if (ctas < 1) ctas = 1;
-  const int64_t run = (units + ctas - 1) / ctas;
+  int64_t run = (units + ctas - 1) / ctas;
+  // a tile is shared by at most kBalancedMaxShare + 1 CTAs: the CTA that completes it adds the others' partial
+  // accumulators one after the other, which costs more than the shorter walk saves beyond that
+  const int64_t min_run = (n_stages + kBalancedMaxShare - 1) / kBalancedMaxShare;
+  if (run < min_run) run = min_run;
   const int64_t plain_walk = ((tiles + sms - 1) / sms) * n_stages;
   if (kHasBalanced && balanced_possible<TN>(g, sms) && run * 10 <= plain_walk * 9) {
     ctas = (units + run - 1) / run;                     // no CTA without work
