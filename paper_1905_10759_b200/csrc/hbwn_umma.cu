@@ -147,12 +147,13 @@ prepare_w_pieces_kernel(const Args g, unsigned char* __restrict__ out) {
 struct CopyArgs {
   const void* x; int32_t x_bf16, C, Cp; int64_t HW; unsigned short* out;
   int32_t gx, gy;          // pixel blocks and channel blocks per image
+  int32_t pb;              // pixels per block
   int64_t n_copy;
 };
-template <int TN, int NP>
+template <int TN, int NP, int PB>
 __global__ void __launch_bounds__(256)
 nhwc_and_pieces_kernel(const CopyArgs c, const Args g, unsigned char* __restrict__ w_out) {
-  __shared__ unsigned short tile[kNhwcCB][kNhwcPitch];
+  __shared__ unsigned short tile[kNhwcCB][nhwc_pitch(PB)];
   const int64_t blk = blockIdx.x;
   pdl_launch_dependents();
   pdl_wait();                   // the workspace may still be in use by the kernel before this one
@@ -160,7 +161,7 @@ nhwc_and_pieces_kernel(const CopyArgs c, const Args g, unsigned char* __restrict
     const int64_t per_image = static_cast<int64_t>(c.gx) * c.gy;
     const int64_t b = blk / per_image, r = blk - b * per_image;
     const int cblock = static_cast<int>(r / c.gx);
-    nchw_to_nhwc_block(c.x, c.x_bf16, c.C, c.HW, c.Cp, c.out, b, cblock, r - static_cast<int64_t>(cblock) * c.gx, tile);
+    nchw_to_nhwc_block<PB>(c.x, c.x_bf16, c.C, c.HW, c.Cp, c.out, b, cblock, r - static_cast<int64_t>(cblock) * c.gx, tile);
   } else {
     const int64_t j = blk - c.n_copy;
     const int64_t tile_n = j / g.n_kb;
@@ -979,8 +980,11 @@ cudaError_t launch(Args g, const CUtensorMap& a_map, void* workspace, cudaStream
   if (copy) {
     const int64_t blocks = copy->n_copy + (w_prepared ? 0 : n_kb * tiles_n);     // prepared weights: the copy blocks only
     if (blocks > 0x7fffffff) return cudaErrorNotSupported;
-    const cudaError_t e = launch_pdl(nhwc_and_pieces_kernel<TN, NP>, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, stream, *copy, g,
-                                     static_cast<unsigned char*>(workspace));
+    const cudaError_t e = copy->pb == kNhwcPBLarge
+        ? launch_pdl(nhwc_and_pieces_kernel<TN, NP, kNhwcPBLarge>, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, stream, *copy, g,
+                     static_cast<unsigned char*>(workspace))
+        : launch_pdl(nhwc_and_pieces_kernel<TN, NP, kNhwcPBSmall>, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, stream, *copy, g,
+                     static_cast<unsigned char*>(workspace));
     if (e != cudaSuccess) return e;
   } else if (!w_prepared) {
     prepare_w_pieces_kernel<TN, NP><<<pgrid, 256, 0, stream>>>(g, static_cast<unsigned char*>(workspace));
@@ -1095,7 +1099,8 @@ cudaError_t launch_hbwn_umma_conv(const void* x, int x_bf16, void* x_nhwc, int C
   CopyArgs cp;
   cp.x = x; cp.x_bf16 = x_bf16; cp.C = c.C; cp.Cp = Cp; cp.HW = static_cast<int64_t>(c.H) * c.W;
   cp.out = static_cast<unsigned short*>(x_nhwc);
-  cp.gx = static_cast<int32_t>((cp.HW + kNhwcPB - 1) / kNhwcPB);
+  cp.pb = nhwc_pixels_per_block(cp.HW);
+  cp.gx = static_cast<int32_t>((cp.HW + cp.pb - 1) / cp.pb);
   cp.gy = (Cp + kNhwcCB - 1) / kNhwcCB;
   cp.n_copy = static_cast<int64_t>(cp.gx) * cp.gy * c.B;
   return launch_any(g, a_map, workspace, stream, &cp, w_prepared, false, use_halo ? &halo : nullptr);
