@@ -454,6 +454,11 @@ def side_measurements(torch, hbmm, inputs, peaks, iters: int):
         ach = 2.0 * M * N * K / (ms * 1e-3) / 1e12
         out.append({"kernel": "hbmm_fold_kernel/beta_a%d_beta_w%d" % (ba, bw), "shape": [M, N, K], "ms": round(ms, 5), "bound": "tensor",
                     "achieved": ach, "peak": bf16_tflops, "unit": "TFLOP/s", "frac": ach / bf16_tflops})
+        if ba != 8:
+            # the same product with no workspace: masked popcounts on the integer pipe, one multiply-add per output and group
+            msp = time_loop(torch, lambda: hbmm.gemm_ex(A, W, C, hbmm.PATH_POPC), max(3, iters // 4))
+            out.append({"kernel": "gemm_popc_sub_kernel (no workspace)/beta_a%d_beta_w%d" % (ba, bw), "shape": [M, N, K], "ms": round(msp, 5),
+                        "tops": 2.0 * M * N * K / (msp * 1e-3) / 1e12, "multiply_adds_per_output": K // min(ba, bw)})
     # the whole convolution call (packing front end + contraction) on conv3_x at the group sizes of the paper's experiments
     # (Section 5: beta_a / beta_w = 16/16, 4/4, 2/16) and at 64/64, beside 32/32
     sh3 = inputs.resnet18_convs(64)[1]
